@@ -1,0 +1,169 @@
+/*
+ * vgc.h -- C ABI of the variance-based gradient compression hot path for NVIDIA B200 (sm_100a).
+ *
+ * Method: Tsuzuku, Imachi, Akiba, "Variance-based Gradient Compression for Efficient Distributed
+ * Deep Learning".  Per training step and per worker the library computes
+ *   (1) the mini-batch sum of squared per-example gradients of a dense or conv layer
+ *       (the right-hand side of Eq. 2 / the "v_i +=" line of Algorithm 1),
+ *   (2) one pass of Algorithm 1 over the flat parameter buffer: accumulate the residual r and
+ *       the variance estimate v, apply the send test r^2 > alpha*v, reset or decay, compact the
+ *       selected elements and encode them with the 4-bit quantiser of Sec. 4.2 / 4.4 into
+ *       32-bit (value, index) words,
+ *   (3) the decode-and-sum half of CommunicateAndUpdate (Sec. 4.3) over W such messages.
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer owned by the caller unless a parameter says "host".
+ *     The library allocates nothing, keeps no state between calls and never synchronises:
+ *     each call only enqueues work on `stream` and returns.
+ *   - Pointers to fp32 / u32 arrays must be 16-byte aligned (whole allocations are).
+ *   - Return value: a vgc_status detected on the host before anything is enqueued, or
+ *     VGC_ERR_CUDA when a launch failed.  Conditions found on the device are OR-ed into the
+ *     caller's *dev_status word (VGC_DEV_*), which the caller zeroes and reads.
+ *   - Workspaces hold no information between calls; the same workspace may serve successive
+ *     calls on one stream.  Calls that overlap on the GPU need separate workspaces.
+ */
+#ifndef VGC_H_
+#define VGC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* cudaStream_t without pulling in the CUDA headers */
+typedef struct CUstream_st *vgc_stream_t;
+
+typedef enum {
+    VGC_OK = 0,
+    VGC_ERR_INVALID_ARG = 1, /* null / misaligned pointer, negative size, n > 2^28, bad alpha or zeta */
+    VGC_ERR_UNSUPPORTED = 2, /* shape outside what the kernels cover                               */
+    VGC_ERR_WORKSPACE = 3,   /* workspace smaller than the matching *_workspace_bytes()             */
+    VGC_ERR_CUDA = 4         /* a CUDA call failed; cudaGetLastError() has the detail               */
+} vgc_status;
+
+/* bits OR-ed into *dev_status by kernels */
+#define VGC_DEV_CAPACITY 1u /* staging or word buffer too small: message truncated, state still correct */
+#define VGC_DEV_TIMEOUT 2u  /* a bounded wait between thread blocks gave up: outputs of this call invalid */
+#define VGC_DEV_RANGE 4u    /* decode met an index >= n: that word was skipped                           */
+
+/* group_exp value of a weight tensor from which nothing was sent */
+#define VGC_EXP_NONE INT32_MIN
+
+/* largest flat buffer: the word keeps 28 bits for the index (Sec. 4.2, "the rest 28-bits") */
+#define VGC_MAX_PARAMS (1u << 28)
+
+const char *vgc_status_string(int status);
+/* 1000*major + minor of this library */
+int vgc_version(void);
+
+/* ---------------------------------------------------------------------------------------------
+ * (1) Squared per-example gradient sums.
+ *
+ * Dense layer y_z = W x_z, delta_z = df_z/dy_z: the gradient of example z for W[j][i] is
+ * delta[z][j]*x[z][i], so  S[j][i] = scale * sum_z delta[z][j]^2 * x[z][i]^2  -- the sum of squared
+ * per-example gradients that Eq. 2 and Algorithm 1 ("v_i += sum (grad_i f_z / B)^2") need, obtained
+ * as one contraction of squared operands without forming any per-example gradient.  Cost
+ * N_params*|B| multiply-adds, the leading term of Sec. 5.  Algorithm 1 divides each example's
+ * gradient by B: pass scale = 1/B^2 when delta carries no 1/B.
+ *
+ *   x      [B][in]   fp32 row-major        delta  [B][out]  fp32 row-major
+ *   S      [out][in] fp32 row-major (the layer's slice of the flat buffer)
+ *   accumulate  0: S = result   1: S += result
+ *   ws / ws_bytes  scratch of at least vgc_sqgrad_linear_workspace_bytes(B, in, out)
+ *
+ * Result within 1e-5 relative of the exact sum.  B, in, out >= 1 (any of them 0: no-op, OK).
+ * ------------------------------------------------------------------------------------------- */
+size_t vgc_sqgrad_linear_workspace_bytes(int B, int in, int out);
+vgc_status vgc_sqgrad_linear(const float *x, const float *delta, int B, int in, int out,
+                             float scale, int accumulate, float *S,
+                             void *ws, size_t ws_bytes, vgc_stream_t stream);
+
+/* Conv layer (cross-correlation, zero padding, dilation 1, groups 1).  The paper does not treat
+ * conv layers; this entry point takes every (example, output position) pair as one sample:
+ *   S[o][c][kh][kw] = scale * sum_z sum_{ho,wo} delta[z][o][ho][wo]^2 * x[z][c][ho*sh+kh-ph][wo*sw+kw-pw]^2
+ * which is the contraction of squared im2col inputs with squared errors, and equals the
+ * per-example sum of squares whenever there is a single output position.
+ *
+ *   x      [B][C][H][W]        fp32 NCHW        delta  [B][Cout][Ho][Wo]  fp32
+ *   S      [Cout][C][Kh][Kw]   fp32 (OIHW, the layer's slice of the flat buffer)
+ *   Ho = (H + 2*pad_h - Kh)/stride_h + 1, Wo likewise; both must be >= 1.
+ * ------------------------------------------------------------------------------------------- */
+size_t vgc_sqgrad_conv_workspace_bytes(int B, int C, int H, int W, int Cout, int Kh, int Kw,
+                                       int stride_h, int stride_w, int pad_h, int pad_w);
+vgc_status vgc_sqgrad_conv(const float *x, const float *delta, int B, int C, int H, int W, int Cout,
+                           int Kh, int Kw, int stride_h, int stride_w, int pad_h, int pad_w,
+                           float scale, int accumulate, float *S,
+                           void *ws, size_t ws_bytes, vgc_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * (2) Compressor: one step of Algorithm 1 ("Basic") over the flat buffer, then Encode().
+ *
+ * For every parameter i, in IEEE binary32, round-to-nearest-even, one operation at a time, no FMA:
+ *     r1 = r[i] + g[i];  v1 = v[i] + s[i];
+ *     send = (r1*r1 > alpha*v1)                       -- strict, Eq. 2
+ *     send:  value_i = r1; r[i] = 0; v[i] = 0        else:  r[i] = r1; v[i] = v1*zeta
+ * Encode (Sec. 4.2, bit-level recipe of Sec. 4.4), per weight tensor k = [offsets[k], offsets[k+1]):
+ *     M_k = max |value_i| over the elements of k being sent;  E_k = floor(log2 M_k) (exponent field)
+ *     e   = min(E_k, exponent of |value_i| after adding 1 at the top mantissa bit)   -- nearer power
+ *           of two, midpoint up, cut at 2^E_k;   d = E_k - e;   d > 7: nothing is emitted for i
+ *     word = i << 4 | sign << 3 | d               -- 28-bit index, 1 sign bit, 3 exponent bits
+ * Words come out in ascending index order; the output is a deterministic function of the inputs.
+ *
+ *   g, s          [n] fp32: this step's sum of per-example gradients / B and sum of their squares
+ *   r, v          [n] fp32 state, updated in place (all zeros before the first step)
+ *   group_offsets [K+1] u32 on the device, offsets[0] = 0, offsets[K] = n, non-decreasing
+ *   stage_capacity  how many elements passing the test the workspace can stage (n is always enough)
+ *   out           HOST struct of device pointers, see below
+ *   ws            at least vgc_compress_workspace_bytes(n, K, stage_capacity)
+ *
+ * n == 0: no-op, OK (counters are not written).  n > VGC_MAX_PARAMS, alpha < 0, non-finite alpha or
+ * zeta, K < 1, null or misaligned pointers: VGC_ERR_INVALID_ARG.  When the staging area or the word
+ * buffer is too small the message is truncated, VGC_DEV_CAPACITY is set, *nnz still holds the count
+ * that was needed (exact unless staging overflowed), and r, v are updated exactly as if it had fit.
+ * Inputs containing NaN or Inf are outside the contract; s >= 0 and v >= 0 are assumed.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    uint32_t *words;       /* out [capacity]: packed words, ascending index                          */
+    uint32_t capacity;     /*                 how many words fit                                     */
+    int32_t *group_exp;    /* out [K]: floor(log2 M_k), or VGC_EXP_NONE                              */
+    uint32_t *nnz;         /* out [1]: words emitted                                                 */
+    uint32_t *n_criterion; /* out [1]: elements that passed the send test                            */
+    uint32_t *n_dropped;   /* out [1]: of those, how many the quantiser rounded to zero (d > 7)      */
+    uint8_t *mask;         /* optional out [n] (may be NULL): 1 where the send test passed           */
+    uint32_t *dev_status;  /* in/out [1]: VGC_DEV_* bits are OR-ed in                                */
+} vgc_message;
+
+size_t vgc_compress_workspace_bytes(size_t n, int K, size_t stage_capacity);
+vgc_status vgc_compress(const float *g, const float *s, float *r, float *v, size_t n,
+                        const uint32_t *group_offsets, int K, float alpha, float zeta,
+                        size_t stage_capacity, const vgc_message *out,
+                        void *ws, size_t ws_bytes, vgc_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * (3) Decoder: the decode-and-sum half of CommunicateAndUpdate (Sec. 4.3; Fig. 1 caption).
+ *
+ * For every word of every message w:  u[idx] += scale * (-1)^sign * 2^(group_exp_w[k] - d), k the
+ * tensor that holds idx.  The W messages are summed ("allreduce" semantics of Sec. 4.3 realised
+ * after an allgatherv); scale = 1/W gives the mean.  Additions into one element may happen in any
+ * order (fp32 atomics), so results match a sequential sum to rounding only.
+ *
+ *   msgs   HOST array of W views; each view holds DEVICE pointers; the word count is read on the device
+ *   u      [n] fp32, accumulated in place (the caller zeroes it when a fresh sum is wanted)
+ * Words whose index is >= n are skipped and VGC_DEV_RANGE is set.  W == 0 or n == 0: no-op, OK.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    const uint32_t *words;    /* [*nnz] packed words                           */
+    const uint32_t *nnz;      /* [1] number of words                           */
+    const int32_t *group_exp; /* [K]                                           */
+} vgc_message_view;
+
+vgc_status vgc_decode_accumulate(const vgc_message_view *msgs, int W,
+                                 const uint32_t *group_offsets, int K, float scale,
+                                 float *u, size_t n, uint32_t *dev_status, vgc_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VGC_H_ */

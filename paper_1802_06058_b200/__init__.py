@@ -1,0 +1,252 @@
+"""Variance-based gradient compression hot path on NVIDIA B200 -- Python binding.
+
+Thin ctypes marshalling over the C ABI declared in ``include/vgc.h`` (same entry-point names).
+Every step of the path runs in the CUDA library ``libvgc.so`` built from ``csrc/``; this module
+only checks tensors, passes pointers and sizes, and raises on a non-zero status.  PyTorch is
+used for device memory and streams.  There is no CPU fallback: if the library is missing or
+was not built, every call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+from ._build import LIB_PATH, build  # noqa: F401  (build is re-exported)
+
+VGC_OK = 0
+VGC_DEV_CAPACITY = 1
+VGC_DEV_TIMEOUT = 2
+VGC_DEV_RANGE = 4
+VGC_EXP_NONE = -(2 ** 31)
+VGC_MAX_PARAMS = 1 << 28
+
+EXPORTS = [
+    "vgc_status_string", "vgc_version",
+    "vgc_sqgrad_linear_workspace_bytes", "vgc_sqgrad_linear",
+    "vgc_sqgrad_conv_workspace_bytes", "vgc_sqgrad_conv",
+    "vgc_compress_workspace_bytes", "vgc_compress",
+    "vgc_decode_accumulate",
+]
+
+
+class VgcError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({_status_string(status)})")
+
+
+class _MessageStruct(ctypes.Structure):      # mirrors vgc_message
+    _fields_ = [("words", ctypes.c_void_p), ("capacity", ctypes.c_uint32), ("group_exp", ctypes.c_void_p),
+                ("nnz", ctypes.c_void_p), ("n_criterion", ctypes.c_void_p), ("n_dropped", ctypes.c_void_p),
+                ("mask", ctypes.c_void_p), ("dev_status", ctypes.c_void_p)]
+
+
+class _ViewStruct(ctypes.Structure):         # mirrors vgc_message_view
+    _fields_ = [("words", ctypes.c_void_p), ("nnz", ctypes.c_void_p), ("group_exp", ctypes.c_void_p)]
+
+
+_lib = None
+
+
+def load_library():
+    """Load libvgc.so (raises if it has not been built) and declare the entry points."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: run paper_1802_06058_b200.build() "
+                           "(needs nvcc); there is no fallback path")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i, f, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.vgc_status_string.argtypes = [i]; lib.vgc_status_string.restype = ctypes.c_char_p
+    lib.vgc_version.argtypes = []; lib.vgc_version.restype = i
+    lib.vgc_sqgrad_linear_workspace_bytes.argtypes = [i, i, i]
+    lib.vgc_sqgrad_linear_workspace_bytes.restype = sz
+    lib.vgc_sqgrad_linear.argtypes = [vp, vp, i, i, i, f, i, vp, vp, sz, vp]
+    lib.vgc_sqgrad_linear.restype = i
+    lib.vgc_sqgrad_conv_workspace_bytes.argtypes = [i] * 11
+    lib.vgc_sqgrad_conv_workspace_bytes.restype = sz
+    lib.vgc_sqgrad_conv.argtypes = [vp, vp] + [i] * 11 + [f, i, vp, vp, sz, vp]
+    lib.vgc_sqgrad_conv.restype = i
+    lib.vgc_compress_workspace_bytes.argtypes = [sz, i, sz]
+    lib.vgc_compress_workspace_bytes.restype = sz
+    lib.vgc_compress.argtypes = [vp, vp, vp, vp, sz, vp, i, f, f, sz, ctypes.POINTER(_MessageStruct), vp, sz, vp]
+    lib.vgc_compress.restype = i
+    lib.vgc_decode_accumulate.argtypes = [ctypes.POINTER(_ViewStruct), i, vp, i, f, vp, sz, vp, vp]
+    lib.vgc_decode_accumulate.restype = i
+    _lib = lib
+    return lib
+
+
+def _status_string(status: int) -> str:
+    try:
+        return load_library().vgc_status_string(int(status)).decode()
+    except Exception:  # pragma: no cover
+        return "?"
+
+
+def _check(status: int, where: str):
+    if status != VGC_OK:
+        raise VgcError(status, where)
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> int:
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _ws(ws: Optional[torch.Tensor]):
+    if ws is None:
+        return None, 0
+    if not ws.is_cuda or not ws.is_contiguous():
+        raise ValueError("workspace must be a contiguous CUDA tensor")
+    return ws.data_ptr(), ws.numel() * ws.element_size()
+
+
+def vgc_version() -> int:
+    return load_library().vgc_version()
+
+
+# ------------------------------------------------------------------------------------------ (1)
+def vgc_sqgrad_linear_workspace_bytes(B: int, n_in: int, n_out: int) -> int:
+    return load_library().vgc_sqgrad_linear_workspace_bytes(B, n_in, n_out)
+
+
+def vgc_sqgrad_linear(x, delta, scale: float, S, accumulate: bool = False, ws=None, stream=None):
+    """S[out,in] (+)= scale * sum_z delta[z,:]^2 (outer) x[z,:]^2 ; x [B,in], delta [B,out]."""
+    B, n_in = x.shape
+    B2, n_out = delta.shape
+    if B != B2 or S.numel() != n_in * n_out:
+        raise ValueError("shape mismatch")
+    wp, wb = _ws(ws)
+    st = load_library().vgc_sqgrad_linear(_dev(x, torch.float32, "x"), _dev(delta, torch.float32, "delta"),
+                                          B, n_in, n_out, float(scale), int(bool(accumulate)),
+                                          _dev(S, torch.float32, "S"), wp, wb, _stream(stream))
+    _check(st, "vgc_sqgrad_linear")
+    return S
+
+
+def vgc_sqgrad_conv_workspace_bytes(B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw) -> int:
+    return load_library().vgc_sqgrad_conv_workspace_bytes(B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw)
+
+
+def vgc_sqgrad_conv(x, delta, kernel, stride, padding, scale: float, S, accumulate: bool = False,
+                    ws=None, stream=None):
+    """S[Cout,C,Kh,Kw] (+)= scale * sum over (example, output position) of squared contributions."""
+    B, C, H, W = x.shape
+    B2, Cout, Ho, Wo = delta.shape
+    Kh, Kw = kernel
+    sh, sw = stride
+    ph, pw = padding
+    if B != B2 or S.numel() != Cout * C * Kh * Kw:
+        raise ValueError("shape mismatch")
+    if Ho != (H + 2 * ph - Kh) // sh + 1 or Wo != (W + 2 * pw - Kw) // sw + 1:
+        raise ValueError("delta spatial shape does not match the convolution geometry")
+    wp, wb = _ws(ws)
+    st = load_library().vgc_sqgrad_conv(_dev(x, torch.float32, "x"), _dev(delta, torch.float32, "delta"),
+                                        B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, float(scale),
+                                        int(bool(accumulate)), _dev(S, torch.float32, "S"), wp, wb,
+                                        _stream(stream))
+    _check(st, "vgc_sqgrad_conv")
+    return S
+
+
+# ------------------------------------------------------------------------------------------ (2)
+class MessageBuffers:
+    """Device buffers behind a vgc_message: words, per-group exponents, counters, optional mask.
+
+    ``counters`` is int32[4] on the device: nnz, n_criterion, n_dropped, dev_status."""
+
+    def __init__(self, capacity: int, K: int, n: int = 0, with_mask: bool = False, device="cuda"):
+        self.capacity = int(capacity)
+        self.K = int(K)
+        self.words = torch.empty(max(self.capacity, 1), dtype=torch.int32, device=device)
+        self.group_exp = torch.empty(max(self.K, 1), dtype=torch.int32, device=device)
+        self.counters = torch.zeros(4, dtype=torch.int32, device=device)
+        self.mask = torch.zeros(n, dtype=torch.uint8, device=device) if with_mask else None
+
+    def struct(self) -> _MessageStruct:
+        c = self.counters.data_ptr()
+        return _MessageStruct(self.words.data_ptr(), self.capacity, self.group_exp.data_ptr(), c, c + 4, c + 8,
+                              self.mask.data_ptr() if self.mask is not None else None, c + 12)
+
+    def view(self) -> _ViewStruct:
+        return _ViewStruct(self.words.data_ptr(), self.counters.data_ptr(), self.group_exp.data_ptr())
+
+    def read(self):
+        """Device -> host copy (synchronises): dict with words (numpy uint32), group_exp, counters."""
+        nnz, n_criterion, n_dropped, dev_status = (int(c) & 0xFFFFFFFF for c in self.counters.tolist())
+        kept = min(nnz, self.capacity)
+        return {"words": self.words[:kept].cpu().numpy().view("uint32"),
+                "group_exp": self.group_exp[:self.K].cpu().numpy(),
+                "nnz": nnz, "n_criterion": n_criterion, "n_dropped": n_dropped, "dev_status": dev_status,
+                "mask": None if self.mask is None else self.mask.cpu().numpy()}
+
+
+def vgc_compress_workspace_bytes(n: int, K: int, stage_capacity: Optional[int] = None) -> int:
+    return load_library().vgc_compress_workspace_bytes(n, K, n if stage_capacity is None else stage_capacity)
+
+
+def vgc_compress(g, s, r, v, group_offsets, alpha: float, zeta: float, out: MessageBuffers, ws,
+                 stage_capacity: Optional[int] = None, stream=None):
+    """One step of Algorithm 1 over the flat buffer + Encode(); r, v updated in place."""
+    n = g.numel()
+    if s.numel() != n or r.numel() != n or v.numel() != n:
+        raise ValueError("g, s, r, v must have the same length")
+    K = group_offsets.numel() - 1
+    if out.K != K:
+        raise ValueError("message buffers were made for a different number of groups")
+    if out.mask is not None and out.mask.numel() != n:
+        raise ValueError("mask length")
+    wp, wb = _ws(ws)
+    msg = out.struct()
+    st = load_library().vgc_compress(_dev(g, torch.float32, "g"), _dev(s, torch.float32, "s"),
+                                     _dev(r, torch.float32, "r"), _dev(v, torch.float32, "v"), n,
+                                     _dev(group_offsets, torch.int32, "group_offsets"), K, float(alpha),
+                                     float(zeta), n if stage_capacity is None else int(stage_capacity),
+                                     ctypes.byref(msg), wp, wb, _stream(stream))
+    _check(st, "vgc_compress")
+    return out
+
+
+# ------------------------------------------------------------------------------------------ (3)
+def vgc_decode_accumulate(messages: Sequence, group_offsets, scale: float, u, dev_status, stream=None):
+    """u[idx] += scale * decoded value over all words of all messages.
+
+    ``messages``: MessageBuffers objects, or (words int32, nnz int32[1], group_exp int32) tensor triples.
+    ``dev_status``: int32[1] device tensor (zeroed by the caller) receiving VGC_DEV_* bits."""
+    W = len(messages)
+    views = (_ViewStruct * max(W, 1))()
+    for w, m in enumerate(messages):
+        if isinstance(m, MessageBuffers):
+            views[w] = m.view()
+        else:
+            words, nnz, gexp = m
+            views[w] = _ViewStruct(_dev(words, torch.int32, "words"), _dev(nnz, torch.int32, "nnz"),
+                                   _dev(gexp, torch.int32, "group_exp"))
+    K = group_offsets.numel() - 1
+    st = load_library().vgc_decode_accumulate(views, W, _dev(group_offsets, torch.int32, "group_offsets"), K,
+                                              float(scale), _dev(u, torch.float32, "u"), u.numel(),
+                                              _dev(dev_status, torch.int32, "dev_status"), _stream(stream))
+    _check(st, "vgc_decode_accumulate")
+    return u
+
+
+def offsets_tensor(offsets, device="cuda") -> torch.Tensor:
+    """Group offsets (uint32 values < 2^31) as the int32 device tensor the binding passes."""
+    import numpy as np
+    return torch.from_numpy(np.asarray(offsets, dtype=np.int64).astype(np.int32)).to(device)

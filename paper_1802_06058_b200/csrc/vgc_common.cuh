@@ -1,0 +1,124 @@
+// Shared device/host helpers of the vgc CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "vgc.h"
+
+#ifndef __CUDA_ARCH__
+#define VGC_HOST_ONLY 1
+#endif
+
+namespace vgc {
+
+constexpr int kWarp = 32;
+
+// Upper bound on polls of a flag written by another thread block.  Each poll sleeps ~64 ns
+// once the fast retries are used up, so the bound is of the order of a second; after it the
+// waiter records VGC_DEV_TIMEOUT and carries on with a value of zero instead of hanging.
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+#define VGC_CUDA_OK(expr)                          \
+    do {                                           \
+        if ((expr) != cudaSuccess) return VGC_ERR_CUDA; \
+    } while (0)
+
+__device__ __forceinline__ uint32_t lane_id() { return threadIdx.x & 31; }
+
+__device__ __forceinline__ uint64_t ld_volatile_u64(const uint64_t *p)
+{
+    uint64_t v;
+    asm volatile("ld.volatile.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_volatile_u64(uint64_t *p, uint64_t v)
+{
+    asm volatile("st.volatile.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_volatile_u32(const uint32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.volatile.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Streaming (evict-first) 128-bit accesses for data touched once per call.
+__device__ __forceinline__ float4 ld_stream_f4(const float *p)
+{
+    float4 v;
+    asm volatile("ld.global.cs.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream_f4(float *p, float4 v)
+{
+    asm volatile("st.global.cs.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+                 : "memory");
+}
+
+// Index of the weight tensor holding flat index i: the k with offs[k] <= i < offs[k+1].
+// offs has K+1 non-decreasing entries, offs[0] = 0; empty tensors are skipped.
+__device__ __forceinline__ int group_of(const uint32_t *offs, int K, uint32_t i)
+{
+    int lo = 0, hi = K;   // invariant: offs[lo] <= i, answer in [lo, hi)
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (offs[mid] <= i) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// Decoupled look-back over per-tile status words {flag:2 | value:32}.  Called by one full
+// warp.  Publishes this tile's aggregate, sums the aggregates of the preceding tiles until
+// one with a complete prefix is met, publishes the inclusive prefix and returns the
+// exclusive one.  Tiles must have been numbered in the order their blocks started (ticket
+// from an atomic counter), so every tile waited for is already running.
+constexpr uint64_t kFlagAgg = 1ull << 32;
+constexpr uint64_t kFlagPrefix = 2ull << 32;
+
+__device__ __forceinline__ uint32_t lookback_exclusive(uint64_t *status, uint32_t tile, uint32_t total,
+                                                       uint32_t *dev_status)
+{
+    const uint32_t lane = lane_id();
+    if (tile == 0) {
+        if (lane == 0) st_volatile_u64(status, kFlagPrefix | total);
+        return 0;
+    }
+    if (lane == 0) st_volatile_u64(status + tile, kFlagAgg | total);
+    uint32_t excl = 0;
+    int64_t pos = (int64_t)tile - 1;
+    bool timed_out = false;
+    while (true) {
+        int64_t idx = pos - lane;
+        uint64_t st = kFlagPrefix;                 // tiles "before 0" carry an empty prefix
+        if (idx >= 0) {
+            st = ld_volatile_u64(status + idx);
+            uint32_t spins = 0;
+            while ((st >> 32) == 0) {
+                if (++spins > kSpinLimit) { timed_out = true; st = kFlagPrefix; break; }
+                if (spins > 16) __nanosleep(64);
+                st = ld_volatile_u64(status + idx);
+            }
+        }
+        const uint32_t has_prefix = __ballot_sync(0xffffffffu, (st >> 32) == 2);
+        uint32_t contrib = (uint32_t)st;
+        if (has_prefix) {
+            const uint32_t first = __ffs(has_prefix) - 1;     // nearest tile with a full prefix
+            if (lane > first) contrib = 0;
+        }
+        excl += __reduce_add_sync(0xffffffffu, contrib);
+        if (has_prefix) break;
+        pos -= 32;
+    }
+    if (__any_sync(0xffffffffu, timed_out) && lane == 0) atomicOr(dev_status, VGC_DEV_TIMEOUT);
+    if (lane == 0) st_volatile_u64(status + tile, kFlagPrefix | (uint64_t)(excl + total));
+    return excl;
+}
+
+}  // namespace vgc

@@ -1,0 +1,89 @@
+// C ABI of the squared per-example gradient sums (argument checks and kernel choice).
+#include "vgc_common.cuh"
+
+namespace vgc {
+size_t simt_workspace_bytes(int M, int N, int K);
+vgc_status simt_sqgrad_linear(const float *x, const float *delta, int B, int in, int out, float scale,
+                              int accumulate, float *S, void *ws, size_t ws_bytes, cudaStream_t st);
+vgc_status simt_sqgrad_conv(const float *x, const float *delta, int B, int C, int H, int W, int Cout,
+                            int Kh, int Kw, int sh, int sw, int ph, int pw, int Ho, int Wo, float scale,
+                            int accumulate, float *S, void *ws, size_t ws_bytes, cudaStream_t st);
+}  // namespace vgc
+
+using namespace vgc;
+
+namespace {
+bool conv_shape_ok(int B, int C, int H, int W, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw,
+                   int *Ho, int *Wo)
+{
+    if (B < 0 || C < 0 || H < 1 || W < 1 || Cout < 0 || Kh < 1 || Kw < 1 || sh < 1 || sw < 1 || ph < 0 || pw < 0)
+        return false;
+    if (H + 2 * ph < Kh || W + 2 * pw < Kw) return false;
+    *Ho = (H + 2 * ph - Kh) / sh + 1;
+    *Wo = (W + 2 * pw - Kw) / sw + 1;
+    const long long k = (long long)B * *Ho * *Wo, n = (long long)C * Kh * Kw;
+    return k < (1LL << 31) && n < (1LL << 31) && (long long)Cout * n < (1LL << 40);
+}
+}  // namespace
+
+extern "C" size_t vgc_sqgrad_linear_workspace_bytes(int B, int in, int out)
+{
+    if (B <= 0 || in <= 0 || out <= 0) return 0;
+    return round_up(simt_workspace_bytes(out, in, B), 256);
+}
+
+extern "C" vgc_status vgc_sqgrad_linear(const float *x, const float *delta, int B, int in, int out,
+                                        float scale, int accumulate, float *S,
+                                        void *ws, size_t ws_bytes, vgc_stream_t stream)
+{
+    if (B < 0 || in < 0 || out < 0) return VGC_ERR_INVALID_ARG;
+    if (in == 0 || out == 0) return VGC_OK;
+    if (!S || !aligned16(S)) return VGC_ERR_INVALID_ARG;
+    if (B > 0 && (!x || !delta || !aligned16(x) || !aligned16(delta))) return VGC_ERR_INVALID_ARG;
+    if (!(scale == scale)) return VGC_ERR_INVALID_ARG;
+    if (ws_bytes < vgc_sqgrad_linear_workspace_bytes(B, in, out) || (ws_bytes && !ws)) return VGC_ERR_WORKSPACE;
+    return simt_sqgrad_linear(x, delta, B, in, out, scale, accumulate, S, ws, ws_bytes,
+                              reinterpret_cast<cudaStream_t>(stream));
+}
+
+extern "C" size_t vgc_sqgrad_conv_workspace_bytes(int B, int C, int H, int W, int Cout, int Kh, int Kw,
+                                                  int stride_h, int stride_w, int pad_h, int pad_w)
+{
+    int Ho, Wo;
+    if (!conv_shape_ok(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, &Ho, &Wo)) return 0;
+    if (B == 0 || C == 0 || Cout == 0) return 0;
+    return round_up(simt_workspace_bytes(Cout, C * Kh * Kw, B * Ho * Wo), 256);
+}
+
+extern "C" vgc_status vgc_sqgrad_conv(const float *x, const float *delta, int B, int C, int H, int W, int Cout,
+                                      int Kh, int Kw, int stride_h, int stride_w, int pad_h, int pad_w,
+                                      float scale, int accumulate, float *S,
+                                      void *ws, size_t ws_bytes, vgc_stream_t stream)
+{
+    int Ho, Wo;
+    if (!conv_shape_ok(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, &Ho, &Wo))
+        return VGC_ERR_INVALID_ARG;
+    if (C == 0 || Cout == 0) return VGC_OK;
+    if (!S || !aligned16(S)) return VGC_ERR_INVALID_ARG;
+    if (B > 0 && (!x || !delta || !aligned16(x) || !aligned16(delta))) return VGC_ERR_INVALID_ARG;
+    if (!(scale == scale)) return VGC_ERR_INVALID_ARG;
+    if (ws_bytes < vgc_sqgrad_conv_workspace_bytes(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w) ||
+        (ws_bytes && !ws))
+        return VGC_ERR_WORKSPACE;
+    return simt_sqgrad_conv(x, delta, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho, Wo, scale,
+                            accumulate, S, ws, ws_bytes, reinterpret_cast<cudaStream_t>(stream));
+}
+
+extern "C" const char *vgc_status_string(int status)
+{
+    switch (status) {
+        case VGC_OK: return "ok";
+        case VGC_ERR_INVALID_ARG: return "invalid argument";
+        case VGC_ERR_UNSUPPORTED: return "unsupported shape";
+        case VGC_ERR_WORKSPACE: return "workspace too small";
+        case VGC_ERR_CUDA: return "CUDA error";
+        default: return "unknown status";
+    }
+}
+
+extern "C" int vgc_version(void) { return 1000; }

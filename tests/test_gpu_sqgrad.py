@@ -1,0 +1,102 @@
+"""GPU parity: squared per-example gradient sums against the CPU oracle (relative 1e-5)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1802_06058_b200 as vgc
+
+pytestmark = pytest.mark.gpu
+RTOL = 1e-5
+
+
+def _ws(nbytes):
+    return torch.empty(max(nbytes, 16), dtype=torch.uint8, device="cuda")
+
+
+def _check(got, want):
+    want64 = want.astype(np.float64)
+    err = np.abs(got.astype(np.float64) - want64)
+    assert np.all(err <= RTOL * np.abs(want64)), float((err / np.maximum(np.abs(want64), 1e-300)).max())
+    assert np.all(got[want == 0] == 0)
+
+
+def run_linear(x, d, scale, S0=None):
+    B, n_in = x.shape
+    n_out = d.shape[1]
+    S = torch.empty(n_out, n_in, device="cuda") if S0 is None else S0.clone()
+    ws = _ws(vgc.vgc_sqgrad_linear_workspace_bytes(B, n_in, n_out))
+    vgc.vgc_sqgrad_linear(x, d, scale, S, accumulate=S0 is not None, ws=ws)
+    return S.cpu().numpy()
+
+
+def run_conv(x, d, k, s, p, scale, S0=None):
+    B, C, H, W = x.shape
+    Cout = d.shape[1]
+    S = torch.empty(Cout, C, k, k, device="cuda") if S0 is None else S0.clone()
+    ws = _ws(vgc.vgc_sqgrad_conv_workspace_bytes(B, C, H, W, Cout, k, k, s, s, p, p))
+    vgc.vgc_sqgrad_conv(x, d, (k, k), (s, s), (p, p), scale, S, accumulate=S0 is not None, ws=ws)
+    return S.cpu().numpy()
+
+
+@pytest.mark.parametrize("B,n_in,n_out", [(32, 256, 128), (128, 784, 1024), (128, 1024, 10), (1, 5, 3),
+                                          (7, 130, 67), (64, 1000, 333), (300, 64, 64), (2, 1, 1)])
+def test_linear(B, n_in, n_out):
+    gen = torch.Generator(device="cuda"); gen.manual_seed(B * 131 + n_in)
+    x = torch.randn(B, n_in, device="cuda", generator=gen).clamp_(min=0)     # ReLU-dead inputs
+    d = torch.randn(B, n_out, device="cuda", generator=gen) * 1e-3
+    x[:, 0] = 0
+    got = run_linear(x, d, 1.0 / (B * B))
+    want = oracle.sqgrad_linear(x.cpu().numpy(), d.cpu().numpy(), scale=1.0 / (B * B))
+    _check(got, want)
+
+
+def test_linear_accumulate_and_all_ones():
+    B, n_in, n_out = 4096, 72, 40
+    ones = run_linear(torch.ones(B, n_in, device="cuda"), torch.ones(B, n_out, device="cuda"), 0.5)
+    assert np.all(ones == 0.5 * B)
+    x = torch.randn(16, n_in, device="cuda"); d = torch.randn(16, n_out, device="cuda")
+    S0 = torch.rand(n_out, n_in, device="cuda")
+    got = run_linear(x, d, 0.25, S0=S0)
+    want = S0.cpu().numpy().copy()
+    oracle.sqgrad_linear(x.cpu().numpy(), d.cpu().numpy(), scale=0.25, out=want)
+    _check(got, want)
+
+
+CONV_SHAPES = [  # B, C, H, Cout, k, stride, pad
+    (2, 3, 9, 4, 3, 1, 1), (3, 5, 8, 6, 1, 1, 0), (2, 4, 9, 3, 1, 2, 0), (2, 3, 20, 8, 7, 2, 3),
+    (4, 16, 14, 24, 3, 2, 1), (2, 64, 14, 64, 3, 1, 1), (2, 70, 7, 130, 1, 1, 0), (3, 8, 5, 5, 5, 1, 0),
+    (1, 1, 3, 1, 3, 1, 1),
+]
+
+
+@pytest.mark.parametrize("B,C,H,Cout,k,s,p", CONV_SHAPES)
+def test_conv(B, C, H, Cout, k, s, p):
+    gen = torch.Generator(device="cuda"); gen.manual_seed(C * 1000 + H)
+    Ho = (H + 2 * p - k) // s + 1
+    x = torch.randn(B, C, H, H, device="cuda", generator=gen).abs_()
+    d = torch.randn(B, Cout, Ho, Ho, device="cuda", generator=gen) * 1e-4
+    got = run_conv(x, d, k, s, p, 1.0 / (B * B))
+    want = oracle.sqgrad_conv(x.cpu().numpy(), d.cpu().numpy(), (k, k), (s, s), (p, p), scale=1.0 / (B * B))
+    _check(got, want)
+
+
+def test_conv_rectangular_geometry_and_accumulate():
+    B, C, H, W, Cout = 2, 3, 10, 7, 4
+    Kh, Kw, sh, sw, ph, pw = 3, 2, 2, 1, 1, 0
+    Ho, Wo = (H + 2 * ph - Kh) // sh + 1, (W + 2 * pw - Kw) // sw + 1
+    x = torch.randn(B, C, H, W, device="cuda"); d = torch.randn(B, Cout, Ho, Wo, device="cuda")
+    S0 = torch.rand(Cout, C, Kh, Kw, device="cuda")
+    S = S0.clone()
+    ws = _ws(vgc.vgc_sqgrad_conv_workspace_bytes(B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw))
+    vgc.vgc_sqgrad_conv(x, d, (Kh, Kw), (sh, sw), (ph, pw), 2.0, S, accumulate=True, ws=ws)
+    want = S0.cpu().numpy().copy()
+    oracle.sqgrad_conv(x.cpu().numpy(), d.cpu().numpy(), (Kh, Kw), (sh, sw), (ph, pw), scale=2.0, out=want)
+    _check(S.cpu().numpy(), want)
+
+
+def test_long_reduction_all_ones_is_exact():
+    # K = 2*224*224 = 100352 terms of exactly 1: any one-sided rounding in the accumulation shows up
+    x = torch.ones(2, 4, 224, 224, device="cuda"); d = torch.ones(2, 8, 224, 224, device="cuda")
+    got = run_conv(x, d, 1, 1, 0, 1.0)
+    assert np.all(got == 2 * 224 * 224)
