@@ -1,0 +1,473 @@
+#!/usr/bin/env python
+"""Benchmark of the variance-based gradient compression hot path on B200.
+
+One "step" is one pass of the whole hot path over one mini-batch of synthetic input:
+squared per-example gradient sums for every layer (vgc_sqgrad_conv / vgc_sqgrad_linear) into
+the flat buffer s, one compressor step over the flat buffer (vgc_compress), and the decode of
+W packed messages into the dense update (vgc_decode_accumulate).
+
+Default workload: the ResNet-50-shaped flat buffer (53 conv + 1 fc weight tensors, 25.5 M
+weights, batch 32, 224x224 input) -- the paper's ImageNet workload shape and the only
+configuration that exercises all three parts at a size that is not cache resident.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet50|mlp|dense|vgg16]
+    python bench.py --impl reference ...      # times the CPU oracle on a bounded sample
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+METRIC = "hot-path throughput (sqgrad + compress + decode), parameters per second"
+UNIT = "Gparam/s"
+
+WORKLOADS = {
+    # name: (config id, layer table, batch, x kind, delta std, W messages, alpha)
+    "dense": (0, "dense_layers", 32, "normal", 1e-2, 4, 2.0),
+    "mlp": (1, "mlp_layers", 128, "relu_normal", 1e-3, 8, 2.0),
+    "resnet50": (2, "resnet50_layers", 32, "half_normal", 1e-4, 8, 2.0),
+    "vgg16": (3, "vgg16_layers", 64, "half_normal", 1e-4, 0, 2.0),      # compress only
+}
+ZETA = 0.999
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for row in self.rows:
+            if len(row) < 7:
+                continue
+            try:
+                sm.append(float(row[0])); smax.append(float(row[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, row[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------------
+# the pipeline under test
+# ----------------------------------------------------------------------------------------------
+class HotPath:
+    """All device buffers of one worker and the launches of one step."""
+
+    def __init__(self, name: str, worker: int, n_input_sets: int, n_g_sets: int, device="cuda"):
+        import paper_1802_06058_b200 as vgc
+        from paper_1802_06058_b200 import workloads
+        self.vgc, self.wl = vgc, workloads
+        cfg, table, self.batch, x_kind, delta_std, self.W, self.alpha = WORKLOADS[name]
+        self.name, self.cfg = name, cfg
+        self.layers = getattr(workloads, table)()
+        self.offsets = workloads.group_offsets(self.layers)
+        self.n = int(self.offsets[-1])
+        self.K = len(self.layers)
+        self.offs_dev = vgc.offsets_tensor(self.offsets)
+        self.compress_only = name == "vgg16"
+        dev = device
+        B = self.batch
+        self.scale = 1.0 / (B * B)
+        f32 = dict(dtype=torch.float32, device=dev)
+        self.s = torch.zeros(self.n, **f32)
+        self.r = torch.zeros(self.n, **f32)
+        self.v = torch.zeros(self.n, **f32)
+        self.u = torch.zeros(self.n, **f32)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.out = vgc.MessageBuffers(self.n, self.K, self.n, with_mask=False, device=dev)
+        self.ws_c = torch.empty(vgc.vgc_compress_workspace_bytes(self.n, self.K), dtype=torch.uint8, device=dev)
+        self.flops_useful = 0
+        self.inputs = []
+        if self.compress_only:
+            gs = [workloads.per_parameter_gs(self.n, B, delta_std, workloads.seed_for(cfg, worker, t, 0, 2), dev)
+                  for t in range(n_g_sets)]
+            self.g_sets = [g for g, _ in gs]
+            self.s_sets = [s for _, s in gs]
+            self.ws_s = None
+        else:
+            ws_bytes = 16
+            for li, spec in enumerate(self.layers):
+                M, N, K = spec.gemm_mnk(B)
+                self.flops_useful += 2 * M * N * K
+                if spec.kind == "conv":
+                    ws_bytes = max(ws_bytes, vgc.vgc_sqgrad_conv_workspace_bytes(
+                        B, spec.cin, spec.hin, spec.hin, spec.cout, spec.k, spec.k, spec.stride, spec.stride,
+                        spec.pad, spec.pad))
+                else:
+                    ws_bytes = max(ws_bytes, vgc.vgc_sqgrad_linear_workspace_bytes(B, spec.cin, spec.cout))
+            self.ws_s = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+            for t in range(n_input_sets):
+                self.inputs.append([workloads.layer_inputs(spec, B, cfg, worker, t, li, x_kind, delta_std, dev)
+                                    for li, spec in enumerate(self.layers)])
+            # g is an input of the compressor made by the harness: one noise draw per step whose
+            # variance matches the squared-gradient sums (g_t = z_t * sqrt(s)), like a mini-batch
+            # gradient under pure noise
+            self.sqgrad(0)
+            root_s = self.s.sqrt()
+            gen = torch.Generator(device=dev); gen.manual_seed(workloads.seed_for(cfg, worker, 0, 0, 3))
+            self.g_sets = [torch.empty(self.n, **f32).normal_(generator=gen).mul_(root_s) for _ in range(n_g_sets)]
+            self.s_sets = None
+        # messages of the other W-1 workers: generated inputs (their own noise draws, compressed once)
+        self.others = []
+        if self.W > 1:
+            root_s = (self.s if self.s_sets is None else self.s_sets[0]).sqrt()
+            rr = torch.zeros(self.n, **f32); vv = torch.zeros(self.n, **f32)
+            for w in range(1, self.W):
+                gen = torch.Generator(device=dev); gen.manual_seed(workloads.seed_for(cfg, worker + w, 0, 0, 3))
+                gw = torch.empty(self.n, **f32).normal_(generator=gen).mul_(root_s)
+                rr.zero_(); vv.zero_()
+                mb = vgc.MessageBuffers(self.n, self.K, self.n, device=dev)
+                vgc.vgc_compress(gw, self.s if self.s_sets is None else self.s_sets[0], rr, vv, self.offs_dev,
+                                 self.alpha, ZETA, mb, self.ws_c)
+                torch.cuda.synchronize()
+                nnz = int(mb.counters[0].item())
+                mb.words = mb.words[:max(nnz, 4)].clone()          # keep only what was written
+                self.others.append(mb)
+            del rr, vv
+
+    # -- launches -------------------------------------------------------------------------------
+    def sqgrad(self, t: int):
+        vgc = self.vgc
+        if self.compress_only:
+            return
+        ins = self.inputs[t % len(self.inputs)]
+        for li, spec in enumerate(self.layers):
+            x, delta = ins[li]
+            S = self.s[int(self.offsets[li]):int(self.offsets[li + 1])]
+            if spec.kind == "conv":
+                vgc.vgc_sqgrad_conv(x, delta, (spec.k, spec.k), (spec.stride, spec.stride), (spec.pad, spec.pad),
+                                    self.scale, S, ws=self.ws_s)
+            else:
+                vgc.vgc_sqgrad_linear(x, delta, self.scale, S, ws=self.ws_s)
+
+    def compress(self, t: int):
+        s = self.s if self.s_sets is None else self.s_sets[t % len(self.s_sets)]
+        self.vgc.vgc_compress(self.g_sets[t % len(self.g_sets)], s, self.r, self.v, self.offs_dev, self.alpha,
+                              ZETA, self.out, self.ws_c)
+
+    def decode(self, t: int):
+        if self.W == 0:
+            return
+        self.u.zero_()
+        self.vgc.vgc_decode_accumulate([self.out] + self.others, self.offs_dev, 1.0 / self.W, self.u, self.status)
+
+    def step(self, t: int, marks=None):
+        self.sqgrad(t)
+        if marks: marks[0].record()
+        self.compress(t)
+        if marks: marks[1].record()
+        self.decode(t)
+        if marks: marks[2].record()
+
+
+def run_device_timed(hp: HotPath, steps: int, warmup: int, dist_on: bool):
+    vgc = hp.vgc
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    for t in range(warmup):
+        hp.step(t)
+    torch.cuda.synchronize()
+    if dist_on:
+        torch.distributed.barrier()
+    torch.cuda.synchronize()
+    marks = [[ev() for _ in range(4)] for _ in range(steps)]
+    launches0 = vgc.vgc_kernel_launch_count()
+    start, stop = ev(), ev()
+    start.record()
+    for i in range(steps):
+        marks[i][3].record()
+        hp.step(warmup + i, marks[i])
+    stop.record()
+    torch.cuda.synchronize()
+    if dist_on:
+        torch.distributed.barrier()
+    launches = vgc.vgc_kernel_launch_count() - launches0
+    total_ms = start.elapsed_time(stop)
+    sq = [m[3].elapsed_time(m[0]) for m in marks]
+    co = [m[0].elapsed_time(m[1]) for m in marks]
+    de = [m[1].elapsed_time(m[2]) for m in marks]
+    return total_ms, sq, co, de, launches
+
+
+def run_e2e(hp: HotPath, steps: int, warmup: int):
+    """Same step, but every step first copies its inputs from pinned host memory to the device and
+    ends with a device->host read of the message (counters, then the packed words)."""
+    if hp.compress_only:
+        host_sets = [[(hp.g_sets[i].cpu().pin_memory(), hp.s_sets[i].cpu().pin_memory())] for i in range(1)]
+    else:
+        host_sets = [[(x.cpu().pin_memory(), d.cpu().pin_memory()) for x, d in hp.inputs[0]]]
+    g_host = hp.g_sets[0].cpu().pin_memory()
+    words_host = torch.empty(hp.n, dtype=torch.int32).pin_memory()
+    counters_host = torch.empty(4, dtype=torch.int32).pin_memory()
+    h2d = g_host.numel() * 4 + sum(a.numel() * 4 + b.numel() * 4 for a, b in host_sets[0])
+    if hp.compress_only:
+        h2d -= g_host.numel() * 4         # g is already one of the pair
+    d2h_total = 0
+
+    def one(t):
+        nonlocal d2h_total
+        if hp.compress_only:
+            hp.g_sets[0].copy_(host_sets[0][0][0], non_blocking=True)
+            hp.s_sets[0].copy_(host_sets[0][0][1], non_blocking=True)
+        else:
+            for (xd, dd), (xh, dh) in zip(hp.inputs[0], host_sets[0]):
+                xd.copy_(xh, non_blocking=True); dd.copy_(dh, non_blocking=True)
+            hp.g_sets[0].copy_(g_host, non_blocking=True)
+        hp.sqgrad(0); hp.compress(0); hp.decode(0)
+        counters_host.copy_(hp.out.counters, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        nnz = min(int(counters_host[0]), hp.n)
+        words_host[:nnz].copy_(hp.out.words[:nnz], non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        d2h_total += 16 + 4 * nnz
+
+    for t in range(warmup):
+        one(t)
+    torch.cuda.synchronize()
+    d2h_total = 0
+    t0 = time.perf_counter()
+    for t in range(steps):
+        one(t)
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    return dt * 1e3 / steps, h2d, d2h_total // max(steps, 1)
+
+
+# ----------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline and --impl reference)
+# ----------------------------------------------------------------------------------------------
+def oracle_sample_time(name: str, hp_like=None):
+    """Times the oracle, as it stands, on a bounded sample of the workload.  Returns
+    (estimated seconds per full step, description, threads)."""
+    import oracle
+    from paper_1802_06058_b200 import workloads
+    cfg, table, B, x_kind, delta_std, W, alpha = WORKLOADS[name]
+    layers = getattr(workloads, table)()
+    offsets = workloads.group_offsets(layers)
+    n = int(offsets[-1])
+    rng = np.random.default_rng(0)
+    # compress + decode at full size on noise inputs (one step each)
+    g = rng.standard_normal(n, dtype=np.float32)
+    s = (rng.standard_normal(n, dtype=np.float32) ** 2)
+    r = np.zeros(n, np.float32); v = np.zeros(n, np.float32)
+    t0 = time.perf_counter()
+    msg = oracle.compress(g, s, r, v, offsets, alpha, ZETA, want_mask=False)
+    t_compress = time.perf_counter() - t0
+    t_decode = 0.0
+    if W:
+        u = np.zeros(n, np.float32)
+        t0 = time.perf_counter()
+        oracle.decode_accumulate([(msg.words, msg.group_exp)], offsets, 1.0 / W, u)
+        t_decode = (time.perf_counter() - t0) * W
+    # sqgrad: measure multiply-add rate on a few layers at reduced batch, extrapolate by MAC count
+    t_sq, desc = 0.0, ""
+    if name != "vgg16":
+        total_macs = sum(np.prod(l.gemm_mnk(B)) for l in layers)
+        picks = layers if len(layers) <= 3 else [layers[i] for i in (2, len(layers) // 2, len(layers) - 2)]
+        bs = B if len(layers) <= 3 else 1
+        macs, secs = 0, 0.0
+        for li, spec in enumerate(picks):
+            x, d = workloads.layer_inputs(spec, bs, cfg, 0, 0, li, x_kind, delta_std, "cpu")
+            t0 = time.perf_counter()
+            if spec.kind == "conv":
+                oracle.sqgrad_conv(x.numpy(), d.numpy(), (spec.k, spec.k), (spec.stride, spec.stride),
+                                   (spec.pad, spec.pad), scale=1.0)
+            else:
+                oracle.sqgrad_linear(x.numpy(), d.numpy(), scale=1.0)
+            secs += time.perf_counter() - t0
+            macs += int(np.prod(spec.gemm_mnk(bs)))
+        t_sq = total_macs / (macs / secs)
+        desc = (f"sqgrad: {len(picks)} layers ({', '.join(p.name for p in picks)}) at batch {bs}, "
+                f"{macs / secs / 1e9:.2f} GMAC/s extrapolated to {total_macs / 1e9:.1f} GMAC; ")
+    desc += f"compress at full n={n} ({t_compress:.2f} s)"
+    if W:
+        desc += f"; decode of one message x W={W} ({t_decode:.2f} s)"
+    return t_sq + t_compress + t_decode, desc, 1, n
+
+
+def reference_arm(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    times = []
+    for i in range(args.warmup + args.steps):
+        sec, desc, threads, n = oracle_sample_time(args.workload)
+        if i >= args.warmup:
+            times.append(sec)
+    sec = statistics.mean(times)
+    value = n / sec / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": args.workload, "n_params": n},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="vgc", choices=["vgc", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        reference_arm(args)
+        return
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    dist_on = world > 1
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the hot path")
+    torch.cuda.set_device(local_rank)
+    if dist_on:
+        torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    import paper_1802_06058_b200 as vgc
+    vgc.load_library()
+    pk = peaks()
+    hp = HotPath(args.workload, worker=rank * 16, n_input_sets=1, n_g_sets=max(4, min(args.steps + args.warmup, 16)))
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    total_ms, sq, co, de, launches = run_device_timed(hp, args.steps, max(args.warmup, 3), dist_on)
+    clocks = sampler.stop()
+    counters = hp.out.read()
+    ms_per_step = total_ms / args.steps
+    if dist_on:
+        t = torch.tensor([ms_per_step], device="cuda")
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms_per_step = float(t.item())
+
+    n = hp.n
+    value = world * n / (ms_per_step * 1e-3) / 1e9
+    sq_ms, co_ms, de_ms = statistics.mean(sq), statistics.mean(co), statistics.mean(de)
+    nnz_a, nnz = counters["n_criterion"], counters["nnz"]
+    sum_nnz = nnz + sum(int(o.words.numel()) for o in hp.others) if hp.W else 0
+    compress_bytes = 24 * n + 8 * nnz_a + 4 * nnz
+    decode_bytes = 12 * sum_nnz + 4 * n * (1 if hp.W else 0)       # words + read-modify-write of u + clearing u
+    sections = {
+        "sqgrad_ms": sq_ms, "compress_ms": co_ms, "decode_ms": de_ms,
+        "sqgrad_useful_tflops": hp.flops_useful / (sq_ms * 1e-3) / 1e12 if sq_ms > 0 and hp.flops_useful else None,
+        "compress_gparam_s": n / (co_ms * 1e-3) / 1e9,
+        "compress_gbs": compress_bytes / (co_ms * 1e-3) / 1e9,
+        "compress_frac_of_measured_hbm": compress_bytes / (co_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+        "decode_gelem_s": sum_nnz / (de_ms * 1e-3) / 1e9 if hp.W else None,
+        "decode_gbs": decode_bytes / (de_ms * 1e-3) / 1e9 if hp.W else None,
+        "compress_decode_gparam_s": n / ((co_ms + de_ms) * 1e-3) / 1e9,
+        "compress_decode_frac_of_measured_hbm": (compress_bytes + decode_bytes) / ((co_ms + de_ms) * 1e-3) / 1e9 / pk["hbm_gbs"],
+        "send_density": nnz_a / n, "nnz": nnz, "n_dropped": counters["n_dropped"], "sum_nnz_decoded": sum_nnz,
+        "dev_status": counters["dev_status"],
+    }
+    # dominant kernel of the step
+    if sq_ms >= co_ms + de_ms and hp.flops_useful:
+        tf32_peak = pk["bf16_tflops_sustained"] / 2.0          # nominal tf32 : bf16 ratio is 1 : 2
+        ach = hp.flops_useful / (sq_ms * 1e-3) / 1e12
+        roofline = {"kernel": "sqgrad (all layers of one step)", "bound": "tensor", "achieved": ach,
+                    "peak": tf32_peak, "unit": "TFLOP/s", "frac": ach / tf32_peak, "traffic": None,
+                    "peak_source": f"{pk['source']} bf16 sustained x 1/2 (tf32 nominal ratio)",
+                    "note": "useful flops 2*M*N*K per layer; a 3xTF32 scheme issues 3x this"}
+    else:
+        ach = compress_bytes / (co_ms * 1e-3) / 1e9
+        roofline = {"kernel": "compress_phase_a+b", "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"],
+                    "unit": "GB/s", "frac": ach / pk["hbm_gbs"], "traffic": None,
+                    "peak_source": f"{pk['source']} copy bandwidth"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32 (tf32x3 products where tensor cores are used)",
+            "data": "synthetic",
+            "config": {"workload": args.workload, "n_params": n, "batch": hp.batch, "W": hp.W, "alpha": hp.alpha,
+                       "zeta": ZETA, "groups": hp.K,
+                       "l2": "inputs larger than L2 (no flush)" if n * 16 > 126e6 else "state fits in L2 (no flush): cache-resident numbers"},
+            "gpu_launches": int(launches), "clocks": clocks, "sections": sections, "roofline": roofline}
+
+    if not args.no_e2e:
+        e2e_ms, h2d, d2h = run_e2e(hp, min(args.steps, 5), 1)
+        if dist_on:
+            t = torch.tensor([e2e_ms], device="cuda")
+            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        line["e2e"] = {"value": world * n / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
+                       "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sec, desc, threads, _ = oracle_sample_time(args.workload)
+        line["cpu_baseline"] = {"value": n / sec / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": desc, "host_cores_available": os.cpu_count()}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist_on:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -44,7 +44,7 @@ typedef enum {
 } vgc_status;
 
 /* bits OR-ed into *dev_status by kernels */
-#define VGC_DEV_CAPACITY 1u /* staging or word buffer too small: message truncated, state still correct */
+#define VGC_DEV_CAPACITY 1u /* word buffer too small: message truncated, state still correct             */
 #define VGC_DEV_TIMEOUT 2u  /* a bounded wait between thread blocks gave up: outputs of this call invalid */
 #define VGC_DEV_RANGE 4u    /* decode met an index >= n: that word was skipped                           */
 
@@ -57,6 +57,9 @@ typedef enum {
 const char *vgc_status_string(int status);
 /* 1000*major + minor of this library */
 int vgc_version(void);
+/* Kernels enqueued by this library since it was loaded (host-side bookkeeping for benchmarks;
+ * not thread-safe, no paper counterpart). */
+uint64_t vgc_kernel_launch_count(void);
 
 /* ---------------------------------------------------------------------------------------------
  * (1) Squared per-example gradient sums.
@@ -114,14 +117,14 @@ vgc_status vgc_sqgrad_conv(const float *x, const float *delta, int B, int C, int
  *   g, s          [n] fp32: this step's sum of per-example gradients / B and sum of their squares
  *   r, v          [n] fp32 state, updated in place (all zeros before the first step)
  *   group_offsets [K+1] u32 on the device, offsets[0] = 0, offsets[K] = n, non-decreasing
- *   stage_capacity  how many elements passing the test the workspace can stage (n is always enough)
  *   out           HOST struct of device pointers, see below
- *   ws            at least vgc_compress_workspace_bytes(n, K, stage_capacity)
+ *   ws            at least vgc_compress_workspace_bytes(n, K) (about 8 bytes per parameter: every
+ *                 tile of the buffer owns a staging segment that could hold all of its elements)
  *
  * n == 0: no-op, OK (counters are not written).  n > VGC_MAX_PARAMS, alpha < 0, non-finite alpha or
- * zeta, K < 1, null or misaligned pointers: VGC_ERR_INVALID_ARG.  When the staging area or the word
- * buffer is too small the message is truncated, VGC_DEV_CAPACITY is set, *nnz still holds the count
- * that was needed (exact unless staging overflowed), and r, v are updated exactly as if it had fit.
+ * zeta, K < 1, null or misaligned pointers: VGC_ERR_INVALID_ARG.  When the word buffer is too small
+ * the message is truncated, VGC_DEV_CAPACITY is set, *nnz still holds the count that was needed, and
+ * r, v are updated exactly as if it had fit.
  * Inputs containing NaN or Inf are outside the contract; s >= 0 and v >= 0 are assumed.
  * ------------------------------------------------------------------------------------------- */
 typedef struct {
@@ -135,11 +138,10 @@ typedef struct {
     uint32_t *dev_status;  /* in/out [1]: VGC_DEV_* bits are OR-ed in                                */
 } vgc_message;
 
-size_t vgc_compress_workspace_bytes(size_t n, int K, size_t stage_capacity);
+size_t vgc_compress_workspace_bytes(size_t n, int K);
 vgc_status vgc_compress(const float *g, const float *s, float *r, float *v, size_t n,
                         const uint32_t *group_offsets, int K, float alpha, float zeta,
-                        size_t stage_capacity, const vgc_message *out,
-                        void *ws, size_t ws_bytes, vgc_stream_t stream);
+                        const vgc_message *out, void *ws, size_t ws_bytes, vgc_stream_t stream);
 
 /* ---------------------------------------------------------------------------------------------
  * (3) Decoder: the decode-and-sum half of CommunicateAndUpdate (Sec. 4.3; Fig. 1 caption).

@@ -24,7 +24,7 @@ VGC_EXP_NONE = -(2 ** 31)
 VGC_MAX_PARAMS = 1 << 28
 
 EXPORTS = [
-    "vgc_status_string", "vgc_version",
+    "vgc_status_string", "vgc_version", "vgc_kernel_launch_count",
     "vgc_sqgrad_linear_workspace_bytes", "vgc_sqgrad_linear",
     "vgc_sqgrad_conv_workspace_bytes", "vgc_sqgrad_conv",
     "vgc_compress_workspace_bytes", "vgc_compress",
@@ -63,6 +63,7 @@ def load_library():
     vp, i, f, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
     lib.vgc_status_string.argtypes = [i]; lib.vgc_status_string.restype = ctypes.c_char_p
     lib.vgc_version.argtypes = []; lib.vgc_version.restype = i
+    lib.vgc_kernel_launch_count.argtypes = []; lib.vgc_kernel_launch_count.restype = ctypes.c_uint64
     lib.vgc_sqgrad_linear_workspace_bytes.argtypes = [i, i, i]
     lib.vgc_sqgrad_linear_workspace_bytes.restype = sz
     lib.vgc_sqgrad_linear.argtypes = [vp, vp, i, i, i, f, i, vp, vp, sz, vp]
@@ -71,9 +72,9 @@ def load_library():
     lib.vgc_sqgrad_conv_workspace_bytes.restype = sz
     lib.vgc_sqgrad_conv.argtypes = [vp, vp] + [i] * 11 + [f, i, vp, vp, sz, vp]
     lib.vgc_sqgrad_conv.restype = i
-    lib.vgc_compress_workspace_bytes.argtypes = [sz, i, sz]
+    lib.vgc_compress_workspace_bytes.argtypes = [sz, i]
     lib.vgc_compress_workspace_bytes.restype = sz
-    lib.vgc_compress.argtypes = [vp, vp, vp, vp, sz, vp, i, f, f, sz, ctypes.POINTER(_MessageStruct), vp, sz, vp]
+    lib.vgc_compress.argtypes = [vp, vp, vp, vp, sz, vp, i, f, f, ctypes.POINTER(_MessageStruct), vp, sz, vp]
     lib.vgc_compress.restype = i
     lib.vgc_decode_accumulate.argtypes = [ctypes.POINTER(_ViewStruct), i, vp, i, f, vp, sz, vp, vp]
     lib.vgc_decode_accumulate.restype = i
@@ -119,6 +120,10 @@ def _ws(ws: Optional[torch.Tensor]):
 
 def vgc_version() -> int:
     return load_library().vgc_version()
+
+
+def vgc_kernel_launch_count() -> int:
+    return load_library().vgc_kernel_launch_count()
 
 
 # ------------------------------------------------------------------------------------------ (1)
@@ -197,12 +202,11 @@ class MessageBuffers:
                 "mask": None if self.mask is None else self.mask.cpu().numpy()}
 
 
-def vgc_compress_workspace_bytes(n: int, K: int, stage_capacity: Optional[int] = None) -> int:
-    return load_library().vgc_compress_workspace_bytes(n, K, n if stage_capacity is None else stage_capacity)
+def vgc_compress_workspace_bytes(n: int, K: int) -> int:
+    return load_library().vgc_compress_workspace_bytes(n, K)
 
 
-def vgc_compress(g, s, r, v, group_offsets, alpha: float, zeta: float, out: MessageBuffers, ws,
-                 stage_capacity: Optional[int] = None, stream=None):
+def vgc_compress(g, s, r, v, group_offsets, alpha: float, zeta: float, out: MessageBuffers, ws, stream=None):
     """One step of Algorithm 1 over the flat buffer + Encode(); r, v updated in place."""
     n = g.numel()
     if s.numel() != n or r.numel() != n or v.numel() != n:
@@ -217,8 +221,7 @@ def vgc_compress(g, s, r, v, group_offsets, alpha: float, zeta: float, out: Mess
     st = load_library().vgc_compress(_dev(g, torch.float32, "g"), _dev(s, torch.float32, "s"),
                                      _dev(r, torch.float32, "r"), _dev(v, torch.float32, "v"), n,
                                      _dev(group_offsets, torch.int32, "group_offsets"), K, float(alpha),
-                                     float(zeta), n if stage_capacity is None else int(stage_capacity),
-                                     ctypes.byref(msg), wp, wb, _stream(stream))
+                                     float(zeta), ctypes.byref(msg), wp, wb, _stream(stream))
     _check(st, "vgc_compress")
     return out
 

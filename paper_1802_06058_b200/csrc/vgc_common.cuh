@@ -28,6 +28,10 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
         if ((expr) != cudaSuccess) return VGC_ERR_CUDA; \
     } while (0)
 
+// Number of kernels this library has enqueued since it was loaded (benchmark bookkeeping).
+extern unsigned long long g_launches;
+inline void count_launch(unsigned k = 1) { g_launches += k; }
+
 __device__ __forceinline__ uint32_t lane_id() { return threadIdx.x & 31; }
 
 __device__ __forceinline__ uint64_t ld_volatile_u64(const uint64_t *p)
@@ -74,15 +78,25 @@ __device__ __forceinline__ int group_of(const uint32_t *offs, int K, uint32_t i)
     return lo;
 }
 
-// Decoupled look-back over per-tile status words {flag:2 | value:32}.  Called by one full
+// Decoupled look-back over per-tile status words {flag:2 | payload:62}.  Called by one full
 // warp.  Publishes this tile's aggregate, sums the aggregates of the preceding tiles until
 // one with a complete prefix is met, publishes the inclusive prefix and returns the
-// exclusive one.  Tiles must have been numbered in the order their blocks started (ticket
-// from an atomic counter), so every tile waited for is already running.
-constexpr uint64_t kFlagAgg = 1ull << 32;
-constexpr uint64_t kFlagPrefix = 2ull << 32;
+// exclusive one.  Payloads add as plain 64-bit integers (several packed counters are fine
+// as long as no field overflows into its neighbour).  Tiles must have been numbered in the
+// order their blocks started (ticket from an atomic counter), so every tile waited for is
+// already running; every wait is bounded all the same.
+constexpr uint64_t kFlagAgg = 1ull << 62;
+constexpr uint64_t kFlagPrefix = 2ull << 62;
+constexpr uint64_t kPayloadMask = (1ull << 62) - 1;
 
-__device__ __forceinline__ uint32_t lookback_exclusive(uint64_t *status, uint32_t tile, uint32_t total,
+__device__ __forceinline__ uint64_t warp_sum_u64(uint64_t x)
+{
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) x += __shfl_xor_sync(0xffffffffu, x, d);
+    return x;
+}
+
+__device__ __forceinline__ uint64_t lookback_exclusive(uint64_t *status, uint32_t tile, uint64_t total,
                                                        uint32_t *dev_status)
 {
     const uint32_t lane = lane_id();
@@ -91,7 +105,7 @@ __device__ __forceinline__ uint32_t lookback_exclusive(uint64_t *status, uint32_
         return 0;
     }
     if (lane == 0) st_volatile_u64(status + tile, kFlagAgg | total);
-    uint32_t excl = 0;
+    uint64_t excl = 0;
     int64_t pos = (int64_t)tile - 1;
     bool timed_out = false;
     while (true) {
@@ -100,24 +114,24 @@ __device__ __forceinline__ uint32_t lookback_exclusive(uint64_t *status, uint32_
         if (idx >= 0) {
             st = ld_volatile_u64(status + idx);
             uint32_t spins = 0;
-            while ((st >> 32) == 0) {
+            while ((st >> 62) == 0) {
                 if (++spins > kSpinLimit) { timed_out = true; st = kFlagPrefix; break; }
                 if (spins > 16) __nanosleep(64);
                 st = ld_volatile_u64(status + idx);
             }
         }
-        const uint32_t has_prefix = __ballot_sync(0xffffffffu, (st >> 32) == 2);
-        uint32_t contrib = (uint32_t)st;
+        const uint32_t has_prefix = __ballot_sync(0xffffffffu, (st >> 62) == 2);
+        uint64_t contrib = st & kPayloadMask;
         if (has_prefix) {
             const uint32_t first = __ffs(has_prefix) - 1;     // nearest tile with a full prefix
             if (lane > first) contrib = 0;
         }
-        excl += __reduce_add_sync(0xffffffffu, contrib);
+        excl += warp_sum_u64(contrib);
         if (has_prefix) break;
         pos -= 32;
     }
     if (__any_sync(0xffffffffu, timed_out) && lane == 0) atomicOr(dev_status, VGC_DEV_TIMEOUT);
-    if (lane == 0) st_volatile_u64(status + tile, kFlagPrefix | (uint64_t)(excl + total));
+    if (lane == 0) st_volatile_u64(status + tile, kFlagPrefix | (excl + total));
     return excl;
 }
 

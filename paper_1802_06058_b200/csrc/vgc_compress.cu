@@ -4,12 +4,14 @@
 //
 // Two kernels on one stream:
 //   phase A  streams g, s, r, v once (16 B read + 8 B written per parameter), applies the send
-//            test, writes r, v back and compacts the selected (index, value) pairs IN INDEX
-//            ORDER into a staging area; a per-tensor atomicMax on |value| bit patterns yields
-//            M_k.  Ordered compaction across thread blocks uses a decoupled look-back over
-//            per-tile counts, with tiles numbered by an atomic ticket.
+//            test and writes r, v back.  Each tile of 2048 parameters compacts its selected
+//            (index, value) pairs, in index order, into its own 2048-slot segment of a staging
+//            area and records how many there are; a per-tensor atomicMax on |value| bit
+//            patterns yields M_k.  Thread blocks never wait for one another here.
 //   phase B  runs over the staged pairs only: quantises against E_k = floor(log2 M_k), drops
-//            d > 7, compacts again in order and packs the words.
+//            d > 7 and packs the words in ascending index order.  One warp owns one segment;
+//            positions across thread blocks come from a decoupled look-back over per-tile
+//            counts, with tiles numbered by an atomic ticket and every wait bounded.
 // The per-tensor maximum has to be complete before any value can be quantised, which is why
 // the work is split in two; the staged pairs are a small fraction of the buffer.
 #include "vgc_common.cuh"
@@ -17,38 +19,37 @@
 namespace vgc {
 
 constexpr int kThreads = 256;
-constexpr int kRowsA = 4;                            // float4 vectors per thread per tile
-constexpr int kTileA = kThreads * kRowsA * 4;        // 4096 parameters per tile
-constexpr int kRowsB = 8;                            // staged pairs per thread per tile
-constexpr int kTileB = kThreads * kRowsB;            // 2048 staged pairs per tile
+constexpr int kWarps = kThreads / kWarp;             // 8
+constexpr int kRowsA = 2;                            // float4 vectors per thread per tile
+constexpr int kTileA = kThreads * kRowsA * 4;        // 2048 parameters per tile = one staging segment
+constexpr int kSegPerTileB = kWarps;                 // phase B: one warp per segment
 constexpr int kOffsSmem = 1024;                      // group offsets cached in shared memory
 
 struct CompressHeader {      // first bytes of the workspace, zeroed by every call
-    uint32_t ticket_a;
     uint32_t ticket_b;
-    uint32_t nnz_a;          // elements that passed the send test
-    uint32_t pad;
+    uint32_t pad[3];
 };
 
 struct CompressLayout {
-    size_t gmax, status_a, status_b, stage_idx, stage_val, total;
-    size_t zero_bytes;       // header + gmax + both status arrays are cleared per call
+    size_t gmax, status_b, tile_count, stage_idx, stage_val, total;
+    size_t zero_bytes;       // header + gmax + status array are cleared per call
     uint32_t tiles_a, tiles_b;
 };
 
-static CompressLayout compress_layout(size_t n, int K, size_t stage_capacity)
+static CompressLayout compress_layout(size_t n, int K)
 {
     CompressLayout L;
     L.tiles_a = (uint32_t)((n + kTileA - 1) / kTileA);
-    L.tiles_b = (uint32_t)((stage_capacity + kTileB - 1) / kTileB);
+    L.tiles_b = (L.tiles_a + kSegPerTileB - 1) / kSegPerTileB;
     size_t off = sizeof(CompressHeader);
     L.gmax = off;          off = round_up(off + sizeof(uint32_t) * (size_t)K, 16);
-    L.status_a = off;      off += sizeof(uint64_t) * L.tiles_a;
     L.status_b = off;      off += sizeof(uint64_t) * L.tiles_b;
     off = round_up(off, 256);
     L.zero_bytes = off;
-    L.stage_idx = off;     off = round_up(off + sizeof(uint32_t) * stage_capacity, 256);
-    L.stage_val = off;     off = round_up(off + sizeof(uint32_t) * stage_capacity, 256);
+    L.tile_count = off;    off = round_up(off + sizeof(uint32_t) * L.tiles_a, 256);
+    const size_t slots = (size_t)L.tiles_a * kTileA;
+    L.stage_idx = off;     off = round_up(off + sizeof(uint32_t) * slots, 256);
+    L.stage_val = off;     off = round_up(off + sizeof(uint32_t) * slots, 256);
     L.total = off;
     return L;
 }
@@ -56,44 +57,31 @@ static CompressLayout compress_layout(size_t n, int K, size_t stage_capacity)
 // ------------------------------------------------------------------------------------------
 // phase A
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 compress_phase_a(const float *__restrict__ g, const float *__restrict__ s, float *__restrict__ r,
                  float *__restrict__ v, size_t n, const uint32_t *__restrict__ group_offsets, int K,
-                 float alpha, float zeta, CompressHeader *hdr, uint32_t *gmax, uint64_t *status,
-                 uint32_t *__restrict__ stage_idx, uint32_t *__restrict__ stage_val, size_t stage_capacity,
-                 uint8_t *__restrict__ mask, uint32_t *dev_status, uint32_t n_tiles)
+                 float alpha, float zeta, uint32_t *gmax, uint32_t *__restrict__ tile_count,
+                 uint32_t *__restrict__ stage_idx, uint32_t *__restrict__ stage_val,
+                 uint8_t *__restrict__ mask, uint32_t n_tiles)
 {
-    __shared__ uint32_t sm_idx[kTileA];
-    __shared__ uint32_t sm_val[kTileA];
     __shared__ uint32_t sm_offs[kOffsSmem];
-    __shared__ uint32_t sm_part[kRowsA * (kThreads / kWarp)];   // 32 per-(row, warp) counts
-    __shared__ uint32_t sm_tile[2];
-    __shared__ uint32_t sm_excl, sm_total, sm_gmax;
-    __shared__ int sm_klo, sm_khi;
+    __shared__ uint32_t sm_part[2][32];                 // per-(row, warp) counts, double buffered
+    __shared__ uint32_t sm_wmax[2][kWarps];
+    __shared__ int sm_grp[2];
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool offs_in_smem = (K + 1) <= kOffsSmem;
     if (offs_in_smem)
         for (int i = tid; i <= K; i += kThreads) sm_offs[i] = group_offsets[i];
     const uint32_t *offs = offs_in_smem ? sm_offs : group_offsets;
-    if (tid == 0) sm_tile[0] = atomicAdd(&hdr->ticket_a, 1u);
+    if (tid < 64) (&sm_part[0][0])[tid] = 0;            // entries past kRowsA*kWarps stay zero
     __syncthreads();
 
-    for (uint32_t it = 0;; ++it) {
-        const uint32_t tile = sm_tile[it & 1];
-        if (tile >= n_tiles) break;
+    uint32_t buf = 0;
+    for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, buf ^= 1) {
         const size_t base = (size_t)tile * kTileA;
-        if (tid == 0) {                                // ticket of the next tile, off the critical path
-            sm_tile[(it + 1) & 1] = atomicAdd(&hdr->ticket_a, 1u);
-            sm_gmax = 0;
-        }
-        if (tid == 32) {                               // weight tensors this tile touches
-            const size_t last = (base + kTileA < n ? base + kTileA : n) - 1;
-            sm_klo = group_of(offs, K, (uint32_t)base);
-            sm_khi = group_of(offs, K, (uint32_t)last);
-        }
 
-        // ---- load: thread t owns elements base + (j*256 + t)*4 + {0..3}, j = 0..3
+        // ---- load: thread t owns elements base + (j*256 + t)*4 + {0..3}
         float4 G[kRowsA], S[kRowsA], R[kRowsA], V[kRowsA];
 #pragma unroll
         for (int j = 0; j < kRowsA; ++j) {
@@ -114,6 +102,11 @@ compress_phase_a(const float *__restrict__ g, const float *__restrict__ s, float
                 G[j] = make_float4(tg[0], tg[1], tg[2], tg[3]);  S[j] = make_float4(ts[0], ts[1], ts[2], ts[3]);
                 R[j] = make_float4(tr[0], tr[1], tr[2], tr[3]);  V[j] = make_float4(tv[0], tv[1], tv[2], tv[3]);
             }
+        }
+        if (tid == 0) {                                 // weight tensor of this tile, or -1 if it spans several
+            const size_t last = (base + kTileA < n ? base + kTileA : n) - 1;
+            const int k = group_of(offs, K, (uint32_t)base);
+            sm_grp[buf] = (last < offs[k + 1]) ? k : -1;
         }
 
         // ---- Algorithm 1 loop body; every operation rounded on its own (no FMA)
@@ -164,111 +157,109 @@ compress_phase_a(const float *__restrict__ g, const float *__restrict__ s, float
             }
         }
 
-        // ---- ordered positions inside the tile: warp scan of the packed per-row counts
+        // ---- ordered positions inside the tile: warp scan of the packed per-row counts, then
+        //      every warp scans the 16 (row, warp) totals by itself (one barrier per tile)
         uint32_t incl = packed;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
             const uint32_t up = __shfl_up_sync(0xffffffffu, incl, d);
             if (lane >= d) incl += up;
         }
+        const uint32_t warp_max = __reduce_max_sync(0xffffffffu, my_max);
         if (lane == 31) {
 #pragma unroll
-            for (int j = 0; j < kRowsA; ++j) sm_part[j * (kThreads / kWarp) + warp] = (incl >> (8 * j)) & 0xFFu;
+            for (int j = 0; j < kRowsA; ++j) sm_part[buf][j * kWarps + warp] = (incl >> (8 * j)) & 0xFFu;
+            sm_wmax[buf][warp] = warp_max;
         }
-        const uint32_t warp_max = __reduce_max_sync(0xffffffffu, my_max);
-        __syncthreads();                                           // (1) parts, sm_gmax = 0, sm_klo/khi
-        if (lane == 0 && warp_max) atomicMax(&sm_gmax, warp_max);
-        if (warp == 0) {
-            const uint32_t t = sm_part[lane];
-            uint32_t ti = t;
+        __syncthreads();
+        const uint32_t part = sm_part[buf][lane];
+        uint32_t pincl = part;
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t up = __shfl_up_sync(0xffffffffu, ti, d);
-                if (lane >= d) ti += up;
-            }
-            const uint32_t total = __shfl_sync(0xffffffffu, ti, 31);
-            sm_part[lane] = ti - t;
-            const uint32_t excl = lookback_exclusive(status, tile, total, dev_status);
-            if (lane == 0) {
-                sm_excl = excl;
-                sm_total = total;
-                if (tile == n_tiles - 1) hdr->nnz_a = excl + total;
-                if ((size_t)excl + total > stage_capacity) atomicOr(dev_status, VGC_DEV_CAPACITY);
-            }
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xffffffffu, pincl, d);
+            if (lane >= d) pincl += up;
         }
-        __syncthreads();                                           // (2) offsets, prefix, sm_gmax
-        const uint32_t excl = sm_excl, total = sm_total;
-        const bool one_group = sm_klo == sm_khi;
-        if (tid == 0 && one_group && sm_gmax) atomicMax(&gmax[sm_klo], sm_gmax);
+        const uint32_t total = __shfl_sync(0xffffffffu, pincl, 31);
+        const uint32_t pexcl = pincl - part;
+        const int grp = sm_grp[buf];
+        uint32_t *seg_idx = stage_idx + base;
+        uint32_t *seg_val = stage_val + base;
 #pragma unroll
         for (int j = 0; j < kRowsA; ++j) {
+            const uint32_t row_base = __shfl_sync(0xffffffffu, pexcl, j * kWarps + warp);
             const uint32_t row_bits = (send_bits >> (4 * j)) & 0xFu;
             if (row_bits) {
                 const uint32_t e = (uint32_t)(base + (size_t)(j * kThreads + tid) * 4);
-                uint32_t at = sm_part[j * (kThreads / kWarp) + warp] + ((incl >> (8 * j)) & 0xFFu) -
-                              (uint32_t)__popc(row_bits);
+                uint32_t at = row_base + ((incl >> (8 * j)) & 0xFFu) - (uint32_t)__popc(row_bits);
                 const float *Gj = reinterpret_cast<const float *>(&G[j]);
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
                     if (row_bits & (1u << q)) {
                         const uint32_t bits = __float_as_uint(Gj[q]);
-                        sm_idx[at] = e + q;
-                        sm_val[at] = bits;
+                        seg_idx[at] = e + q;
+                        seg_val[at] = bits;
                         ++at;
-                        if (!one_group)
-                            atomicMax(&gmax[group_of(offs, K, e + q)], bits & 0x7FFFFFFFu);
+                        if (grp < 0) atomicMax(&gmax[group_of(offs, K, e + q)], bits & 0x7FFFFFFFu);
                     }
             }
         }
-        __syncthreads();                                           // (3) compacted tile in shared memory
-        for (uint32_t q = tid; q < total; q += kThreads) {
-            const size_t p = (size_t)excl + q;
-            if (p < stage_capacity) {
-                stage_idx[p] = sm_idx[q];
-                stage_val[p] = sm_val[q];
+        if (tid == 0) {
+            tile_count[tile] = total;
+            if (grp >= 0 && total) {
+                uint32_t m = 0;
+#pragma unroll
+                for (int w = 0; w < kWarps; ++w) m = max(m, sm_wmax[buf][w]);
+                if (m > ld_volatile_u32(gmax + grp)) atomicMax(gmax + grp, m);
             }
         }
-        __syncthreads();                                           // (4) before the next tile reuses smem
     }
 }
 
 // ------------------------------------------------------------------------------------------
 // phase B
 // ------------------------------------------------------------------------------------------
+// Quantise one staged pair: returns true if a word is emitted.
+__device__ __forceinline__ bool encode_pair(uint32_t idx, uint32_t bits, const uint32_t *offs, int K,
+                                            const uint32_t *gmax, int &k, int32_t &Ek, uint32_t &word)
+{
+    if (idx < offs[k] || idx >= offs[k + 1] || Ek == INT32_MIN) {
+        k = group_of(offs, K, idx);
+        Ek = (int32_t)((gmax[k] >> 23) & 0xFFu) - 127;                  // floor(log2 M_k)
+    }
+    const uint32_t a = bits & 0x7FFFFFFFu;
+    const int32_t e1 = (int32_t)((a + 0x00400000u) >> 23) - 127;        // nearer power of two, midpoint up
+    const int32_t e = e1 < Ek ? e1 : Ek;                                // cut at 2^E_k
+    const int32_t d = Ek - e;
+    word = (idx << 4) | ((bits >> 31) << 3) | (uint32_t)(d & 7);
+    return d <= 7;
+}
+
+constexpr uint64_t kPassedShift = 31;       // look-back payload: passed << 31 | kept (each < 2^29)
+
 __global__ void __launch_bounds__(kThreads)
 compress_phase_b(const uint32_t *__restrict__ group_offsets, int K, CompressHeader *hdr,
-                 const uint32_t *__restrict__ gmax, uint64_t *status,
+                 const uint32_t *__restrict__ gmax, const uint32_t *__restrict__ tile_count, uint32_t n_tiles_a,
                  const uint32_t *__restrict__ stage_idx, const uint32_t *__restrict__ stage_val,
-                 size_t stage_capacity, uint32_t *__restrict__ words, uint32_t capacity,
+                 uint64_t *status, uint32_t *__restrict__ words, uint32_t capacity,
                  int32_t *__restrict__ group_exp, uint32_t *nnz_out, uint32_t *n_criterion,
                  uint32_t *n_dropped, uint32_t *dev_status)
 {
-    __shared__ uint32_t sm_words[kTileB];
     __shared__ uint32_t sm_offs[kOffsSmem];
-    __shared__ uint32_t sm_part[kRowsB * (kThreads / kWarp)];   // 64 per-(row, warp) counts
+    __shared__ uint32_t sm_kept[kWarps], sm_passed[kWarps], sm_excl[kWarps];
     __shared__ uint32_t sm_tile[2];
-    __shared__ uint32_t sm_excl, sm_total;
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool offs_in_smem = (K + 1) <= kOffsSmem;
     if (offs_in_smem)
         for (int i = tid; i <= K; i += kThreads) sm_offs[i] = group_offsets[i];
     const uint32_t *offs = offs_in_smem ? sm_offs : group_offsets;
+    const uint32_t n_tiles = (n_tiles_a + kSegPerTileB - 1) / kSegPerTileB;
 
-    const uint32_t n_passed = hdr->nnz_a;                         // written by phase A
-    const uint32_t n_staged = n_passed < stage_capacity ? n_passed : (uint32_t)stage_capacity;
-    const uint32_t n_tiles = (n_staged + kTileB - 1) / kTileB;
-
-    if (blockIdx.x == 0) {
+    if (blockIdx.x == 0)
         for (int k = tid; k < K; k += kThreads) {
             const uint32_t m = gmax[k];
             group_exp[k] = m ? (int32_t)((m >> 23) & 0xFFu) - 127 : VGC_EXP_NONE;
         }
-        if (tid == 0) {
-            *n_criterion = n_passed;
-            if (n_tiles == 0) { *nnz_out = 0; *n_dropped = n_passed; }
-        }
-    }
     if (tid == 0) sm_tile[0] = atomicAdd(&hdr->ticket_b, 1u);
     __syncthreads();
 
@@ -277,64 +268,65 @@ compress_phase_b(const uint32_t *__restrict__ group_offsets, int K, CompressHead
         if (tile >= n_tiles) break;
         if (tid == 0) sm_tile[(it + 1) & 1] = atomicAdd(&hdr->ticket_b, 1u);
 
-        uint32_t word[kRowsB];
-        uint32_t keep_bits = 0;
-        uint32_t my_pos[kRowsB];
-#pragma unroll
-        for (int j = 0; j < kRowsB; ++j) {
-            const uint32_t q = tile * kTileB + j * kThreads + tid;
+        const uint32_t seg = tile * kSegPerTileB + warp;
+        const uint32_t count = seg < n_tiles_a ? tile_count[seg] : 0;
+        const uint32_t *seg_idx = stage_idx + (size_t)seg * kTileA;
+        const uint32_t *seg_val = stage_val + (size_t)seg * kTileA;
+
+        // pass 1: how many of this segment's pairs survive the quantiser
+        int k = 0;
+        int32_t Ek = INT32_MIN;
+        uint32_t kept = 0;
+        for (uint32_t q0 = 0; q0 < count; q0 += 32) {
+            const uint32_t q = q0 + lane;
             bool keep = false;
-            word[j] = 0;
-            if (q < n_staged) {
-                const uint32_t idx = stage_idx[q];
-                const uint32_t bits = stage_val[q];
-                const uint32_t m = gmax[group_of(offs, K, idx)];
-                const int32_t Ek = (int32_t)((m >> 23) & 0xFFu) - 127;       // floor(log2 M_k)
-                const uint32_t a = bits & 0x7FFFFFFFu;
-                const int32_t e1 = (int32_t)((a + 0x00400000u) >> 23) - 127; // nearer power of two
-                const int32_t e = e1 < Ek ? e1 : Ek;                         // cut at 2^E_k
-                const int32_t d = Ek - e;
-                keep = d <= 7;
-                word[j] = (idx << 4) | ((bits >> 31) << 3) | (uint32_t)(d & 7);
+            if (q < count) {
+                uint32_t word;
+                keep = encode_pair(seg_idx[q], seg_val[q], offs, K, gmax, k, Ek, word);
             }
-            const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
-            my_pos[j] = __popc(ballot & ((1u << lane) - 1u));
-            if (keep) keep_bits |= 1u << j;
-            if (lane == 0) sm_part[j * (kThreads / kWarp) + warp] = __popc(ballot);
+            kept += __popc(__ballot_sync(0xffffffffu, keep));
         }
+        if (lane == 0) { sm_kept[warp] = kept; sm_passed[warp] = count; }
         __syncthreads();                                           // (1)
         if (warp == 0) {
-            const uint32_t t0 = sm_part[2 * lane], t1 = sm_part[2 * lane + 1];
-            const uint32_t t = t0 + t1;
-            uint32_t ti = t;
+            const uint32_t mine = lane < kWarps ? sm_kept[lane] : 0;
+            const uint32_t pass = lane < kWarps ? sm_passed[lane] : 0;
+            uint32_t ki = mine, pi = pass;
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t up = __shfl_up_sync(0xffffffffu, ti, d);
-                if (lane >= d) ti += up;
+            for (int d = 1; d < kWarps; d <<= 1) {
+                const uint32_t ku = __shfl_up_sync(0xffffffffu, ki, d);
+                const uint32_t pu = __shfl_up_sync(0xffffffffu, pi, d);
+                if (lane >= d) { ki += ku; pi += pu; }
             }
-            const uint32_t total = __shfl_sync(0xffffffffu, ti, 31);
-            sm_part[2 * lane] = ti - t;
-            sm_part[2 * lane + 1] = ti - t + t0;
-            const uint32_t excl = lookback_exclusive(status, tile, total, dev_status);
+            const uint32_t tot_kept = __shfl_sync(0xffffffffu, ki, kWarps - 1);
+            const uint32_t tot_pass = __shfl_sync(0xffffffffu, pi, kWarps - 1);
+            const uint64_t excl = lookback_exclusive(status, tile, ((uint64_t)tot_pass << kPassedShift) | tot_kept,
+                                                     dev_status);
+            const uint32_t excl_kept = (uint32_t)(excl & ((1ull << kPassedShift) - 1));
+            const uint32_t excl_pass = (uint32_t)(excl >> kPassedShift);
+            if (lane < kWarps) sm_excl[lane] = excl_kept + ki - mine;
             if (lane == 0) {
-                sm_excl = excl;
-                sm_total = total;
                 if (tile == n_tiles - 1) {
-                    *nnz_out = excl + total;
-                    *n_dropped = n_passed - (excl + total);
+                    *nnz_out = excl_kept + tot_kept;
+                    *n_criterion = excl_pass + tot_pass;
+                    *n_dropped = (excl_pass + tot_pass) - (excl_kept + tot_kept);
                 }
-                if (excl + total > capacity) atomicOr(dev_status, VGC_DEV_CAPACITY);
+                if (excl_kept + tot_kept > capacity) atomicOr(dev_status, VGC_DEV_CAPACITY);
             }
         }
         __syncthreads();                                           // (2)
-        const uint32_t excl = sm_excl, total = sm_total;
-#pragma unroll
-        for (int j = 0; j < kRowsB; ++j)
-            if (keep_bits & (1u << j)) sm_words[sm_part[j * (kThreads / kWarp) + warp] + my_pos[j]] = word[j];
-        __syncthreads();                                           // (3)
-        for (uint32_t q = tid; q < total; q += kThreads)
-            if (excl + q < capacity) words[excl + q] = sm_words[q];
-        __syncthreads();                                           // (4)
+        // pass 2: same pairs again (cache hits), now with their final positions
+        uint32_t pos = sm_excl[warp];
+        for (uint32_t q0 = 0; q0 < count; q0 += 32) {
+            const uint32_t q = q0 + lane;
+            bool keep = false;
+            uint32_t word = 0;
+            if (q < count) keep = encode_pair(seg_idx[q], seg_val[q], offs, K, gmax, k, Ek, word);
+            const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
+            const uint32_t p = pos + __popc(ballot & ((1u << lane) - 1u));
+            if (keep && p < capacity) words[p] = word;
+            pos += __popc(ballot);
+        }
     }
 }
 
@@ -345,17 +337,15 @@ compress_phase_b(const uint32_t *__restrict__ group_offsets, int K, CompressHead
 // ------------------------------------------------------------------------------------------
 using namespace vgc;
 
-extern "C" size_t vgc_compress_workspace_bytes(size_t n, int K, size_t stage_capacity)
+extern "C" size_t vgc_compress_workspace_bytes(size_t n, int K)
 {
     if (K < 1) K = 1;
-    if (stage_capacity > n) stage_capacity = n;
-    return compress_layout(n, K, stage_capacity).total;
+    return compress_layout(n, K).total;
 }
 
 extern "C" vgc_status vgc_compress(const float *g, const float *s, float *r, float *v, size_t n,
                                    const uint32_t *group_offsets, int K, float alpha, float zeta,
-                                   size_t stage_capacity, const vgc_message *out,
-                                   void *ws, size_t ws_bytes, vgc_stream_t stream)
+                                   const vgc_message *out, void *ws, size_t ws_bytes, vgc_stream_t stream)
 {
     if (n == 0) return VGC_OK;
     if (n > VGC_MAX_PARAMS || K < 1 || !out) return VGC_ERR_INVALID_ARG;
@@ -369,15 +359,14 @@ extern "C" vgc_status vgc_compress(const float *g, const float *s, float *r, flo
     if (!aligned16(g) || !aligned16(s) || !aligned16(r) || !aligned16(v) || !aligned16(ws) ||
         (out->mask && (reinterpret_cast<uintptr_t>(out->mask) & 3u)))
         return VGC_ERR_INVALID_ARG;
-    if (stage_capacity > n) stage_capacity = n;
-    const CompressLayout L = compress_layout(n, K, stage_capacity);
+    const CompressLayout L = compress_layout(n, K);
     if (ws_bytes < L.total) return VGC_ERR_WORKSPACE;
 
     char *base = static_cast<char *>(ws);
     CompressHeader *hdr = reinterpret_cast<CompressHeader *>(base);
     uint32_t *gmax = reinterpret_cast<uint32_t *>(base + L.gmax);
-    uint64_t *status_a = reinterpret_cast<uint64_t *>(base + L.status_a);
     uint64_t *status_b = reinterpret_cast<uint64_t *>(base + L.status_b);
+    uint32_t *tile_count = reinterpret_cast<uint32_t *>(base + L.tile_count);
     uint32_t *stage_idx = reinterpret_cast<uint32_t *>(base + L.stage_idx);
     uint32_t *stage_val = reinterpret_cast<uint32_t *>(base + L.stage_val);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
@@ -391,15 +380,14 @@ extern "C" vgc_status vgc_compress(const float *g, const float *s, float *r, flo
     }
 
     VGC_CUDA_OK(cudaMemsetAsync(ws, 0, L.zero_bytes, st));
-    const uint32_t grid_a = L.tiles_a < (uint32_t)(sm_count * 4) ? L.tiles_a : (uint32_t)(sm_count * 4);
-    compress_phase_a<<<grid_a, kThreads, 0, st>>>(g, s, r, v, n, group_offsets, K, alpha, zeta, hdr, gmax,
-                                                  status_a, stage_idx, stage_val, stage_capacity, out->mask,
-                                                  out->dev_status, L.tiles_a);
-    uint32_t grid_b = L.tiles_b < (uint32_t)(sm_count * 4) ? L.tiles_b : (uint32_t)(sm_count * 4);
-    if (grid_b == 0) grid_b = 1;
-    compress_phase_b<<<grid_b, kThreads, 0, st>>>(group_offsets, K, hdr, gmax, status_b, stage_idx, stage_val,
-                                                  stage_capacity, out->words, out->capacity, out->group_exp,
+    const uint32_t grid_a = L.tiles_a < (uint32_t)(sm_count * 8) ? L.tiles_a : (uint32_t)(sm_count * 8);
+    compress_phase_a<<<grid_a, kThreads, 0, st>>>(g, s, r, v, n, group_offsets, K, alpha, zeta, gmax, tile_count,
+                                                  stage_idx, stage_val, out->mask, L.tiles_a);
+    const uint32_t grid_b = L.tiles_b < (uint32_t)(sm_count * 8) ? L.tiles_b : (uint32_t)(sm_count * 8);
+    compress_phase_b<<<grid_b, kThreads, 0, st>>>(group_offsets, K, hdr, gmax, tile_count, L.tiles_a, stage_idx,
+                                                  stage_val, status_b, out->words, out->capacity, out->group_exp,
                                                   out->nnz, out->n_criterion, out->n_dropped, out->dev_status);
+    count_launch(2);
     VGC_CUDA_OK(cudaGetLastError());
     return VGC_OK;
 }

@@ -102,6 +102,7 @@ extern "C" vgc_status vgc_decode_accumulate(const vgc_message_view *msgs, int W,
         if (per_msg < 1) per_msg = 1;
         dim3 grid((unsigned)per_msg, (unsigned)wb);
         decode_scatter<<<grid, kDecThreads, 0, st>>>(views, group_offsets, K, scale, u, n, dev_status);
+        count_launch();
     }
     VGC_CUDA_OK(cudaGetLastError());
     return VGC_OK;

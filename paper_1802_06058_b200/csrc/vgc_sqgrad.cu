@@ -87,3 +87,6 @@ extern "C" const char *vgc_status_string(int status)
 }
 
 extern "C" int vgc_version(void) { return 1000; }
+
+namespace vgc { unsigned long long g_launches = 0; }
+extern "C" uint64_t vgc_kernel_launch_count(void) { return vgc::g_launches; }

@@ -183,7 +183,9 @@ vgc_status simt_launch(const Ops &ops, int M, int N, int K, float scale, int acc
     if (grid.y > 65535u) return VGC_ERR_UNSUPPORTED;
     sqgrad_simt<Ops><<<grid, kSimtThreads, 0, st>>>(ops, M, N, K, k_per_split, scale, accumulate, S,
                                                     static_cast<float *>(ws));
+    count_launch();
     if (splits > 1) {
+        count_launch();
         const size_t mn = (size_t)M * N;
         sqgrad_combine_splits<<<(unsigned)((mn + 255) / 256), 256, 0, st>>>(static_cast<const float *>(ws), splits,
                                                                             mn, scale, accumulate, S);

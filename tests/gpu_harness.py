@@ -12,22 +12,20 @@ F32 = np.float32
 class GpuCompressor:
     """State + buffers for repeated vgc_compress calls on one flat buffer."""
 
-    def __init__(self, n, offsets, with_mask=True, capacity=None, stage_capacity=None):
+    def __init__(self, n, offsets, with_mask=True, capacity=None):
         self.n = n
         self.offsets = np.asarray(offsets, np.uint32)
         self.K = len(self.offsets) - 1
         self.offs_dev = vgc.offsets_tensor(self.offsets)
         self.r = torch.zeros(n, dtype=torch.float32, device="cuda")
         self.v = torch.zeros(n, dtype=torch.float32, device="cuda")
-        self.stage_capacity = n if stage_capacity is None else stage_capacity
         self.out = vgc.MessageBuffers(n if capacity is None else capacity, self.K, n, with_mask=with_mask)
-        ws_bytes = vgc.vgc_compress_workspace_bytes(n, self.K, self.stage_capacity)
+        ws_bytes = vgc.vgc_compress_workspace_bytes(n, self.K)
         self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
 
     def step(self, g, s, alpha, zeta):
         self.out.counters.zero_()
-        vgc.vgc_compress(g, s, self.r, self.v, self.offs_dev, alpha, zeta, self.out, self.ws,
-                         stage_capacity=self.stage_capacity)
+        vgc.vgc_compress(g, s, self.r, self.v, self.offs_dev, alpha, zeta, self.out, self.ws)
         return self.out.read()
 
 

@@ -39,9 +39,8 @@ def test_status_strings_and_version(lib):
 
 def test_workspace_queries_are_pure_host_functions(lib):
     n = 138344128
-    need = lib.vgc_compress_workspace_bytes(n, 16, n)
+    need = lib.vgc_compress_workspace_bytes(n, 16)
     assert 8 * n < need < 8 * n + (4 << 20)
-    assert lib.vgc_compress_workspace_bytes(n, 16, 1000) < (2 << 20)
     assert lib.vgc_sqgrad_linear_workspace_bytes(32, 256, 128) % 256 == 0
     assert lib.vgc_sqgrad_conv_workspace_bytes(32, 64, 56, 56, 64, 3, 3, 1, 1, 1, 1) > 0
     assert lib.vgc_sqgrad_conv_workspace_bytes(32, 64, 2, 2, 64, 3, 3, 1, 1, 0, 0) == 0   # kernel > image
@@ -51,7 +50,7 @@ def test_compress_rejects_bad_arguments_on_the_host(lib):
     fake = ctypes.c_void_p(0x1000)          # never dereferenced: every call below fails validation first
     msg = vgc._MessageStruct(0x1000, 16, 0x1000, 0x1000, 0x1000, 0x1000, None, 0x1000)
     call = lambda n, K, alpha, zeta, g=fake, ws=fake, ws_bytes=1 << 40: lib.vgc_compress(
-        g, fake, fake, fake, n, fake, K, alpha, zeta, n, ctypes.byref(msg), ws, ws_bytes, None)
+        g, fake, fake, fake, n, fake, K, alpha, zeta, ctypes.byref(msg), ws, ws_bytes, None)
     assert call(0, 1, 2.0, 0.999) == 0                        # empty buffer: no-op
     assert call((1 << 28) + 1, 1, 2.0, 0.999) == 1            # index would not fit 28 bits
     assert call(100, 0, 2.0, 0.999) == 1

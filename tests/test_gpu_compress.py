@@ -76,12 +76,11 @@ def test_capacity_overflow_keeps_state_and_reports_needed_count():
     assert got["nnz"] == want.nnz and got["n_criterion"] == want.n_criterion
     assert np.array_equal(got["words"], want.words[:1000])
     assert_same_state(small, cpu)
-    # staging area too small: state still exact, flag set
-    tiny = GpuCompressor(n, offs, stage_capacity=512)
-    got = tiny.step(g, s, 2.0, 0.999)
-    assert got["dev_status"] & vgc.VGC_DEV_CAPACITY
-    assert got["n_criterion"] == want.n_criterion
-    assert_same_state(tiny, cpu)
+    # no room at all
+    none = GpuCompressor(n, offs, capacity=0)
+    got = none.step(g, s, 2.0, 0.999)
+    assert got["dev_status"] == vgc.VGC_DEV_CAPACITY and got["nnz"] == want.nnz and got["words"].size == 0
+    assert_same_state(none, cpu)
 
 
 def test_checkpoint_resume_is_bit_identical():
