@@ -42,6 +42,8 @@ WORKLOADS = {
     "mlp": (1, "mlp_layers", 128, "relu_normal", 1e-3, 8, 2.0),
     "resnet50": (2, "resnet50_layers", 32, "half_normal", 1e-4, 8, 2.0),
     "vgg16": (3, "vgg16_layers", 64, "half_normal", 1e-4, 0, 2.0),      # compress only
+    # a flat buffer of --n-params weights in 16 equal tensors: compress + decode only (small profiling case)
+    "flat": (4, None, 64, "half_normal", 1e-4, 4, 2.0),
 }
 ZETA = 0.999
 
@@ -115,18 +117,23 @@ class ClockSampler:
 class HotPath:
     """All device buffers of one worker and the launches of one step."""
 
-    def __init__(self, name: str, worker: int, n_input_sets: int, n_g_sets: int, device="cuda"):
+    def __init__(self, name: str, worker: int, n_input_sets: int, n_g_sets: int, device="cuda",
+                 n_params: int = 1 << 25):
         import paper_1802_06058_b200 as vgc
         from paper_1802_06058_b200 import workloads
         self.vgc, self.wl = vgc, workloads
         cfg, table, self.batch, x_kind, delta_std, self.W, self.alpha = WORKLOADS[name]
         self.name, self.cfg = name, cfg
-        self.layers = getattr(workloads, table)()
-        self.offsets = workloads.group_offsets(self.layers)
+        if table is None:
+            self.layers = []
+            self.offsets = np.linspace(0, n_params, 17).astype(np.uint32)
+        else:
+            self.layers = getattr(workloads, table)()
+            self.offsets = workloads.group_offsets(self.layers)
         self.n = int(self.offsets[-1])
-        self.K = len(self.layers)
+        self.K = len(self.offsets) - 1
         self.offs_dev = vgc.offsets_tensor(self.offsets)
-        self.compress_only = name == "vgg16"
+        self.compress_only = name in ("vgg16", "flat")
         dev = device
         B = self.batch
         self.scale = 1.0 / (B * B)
@@ -297,14 +304,17 @@ def run_e2e(hp: HotPath, steps: int, warmup: int):
 # ----------------------------------------------------------------------------------------------
 # CPU oracle timing (cpu_baseline and --impl reference)
 # ----------------------------------------------------------------------------------------------
-def oracle_sample_time(name: str, hp_like=None):
+def oracle_sample_time(name: str, n_params: int = 1 << 25):
     """Times the oracle, as it stands, on a bounded sample of the workload.  Returns
     (estimated seconds per full step, description, threads)."""
     import oracle
     from paper_1802_06058_b200 import workloads
     cfg, table, B, x_kind, delta_std, W, alpha = WORKLOADS[name]
-    layers = getattr(workloads, table)()
-    offsets = workloads.group_offsets(layers)
+    if table is None:
+        layers, offsets = [], np.linspace(0, n_params, 17).astype(np.uint32)
+    else:
+        layers = getattr(workloads, table)()
+        offsets = workloads.group_offsets(layers)
     n = int(offsets[-1])
     rng = np.random.default_rng(0)
     # compress + decode at full size on noise inputs (one step each)
@@ -322,7 +332,7 @@ def oracle_sample_time(name: str, hp_like=None):
         t_decode = (time.perf_counter() - t0) * W
     # sqgrad: measure multiply-add rate on a few layers at reduced batch, extrapolate by MAC count
     t_sq, desc = 0.0, ""
-    if name != "vgg16":
+    if layers and name != "vgg16":
         total_macs = sum(np.prod(l.gemm_mnk(B)) for l in layers)
         picks = layers if len(layers) <= 3 else [layers[i] for i in (2, len(layers) // 2, len(layers) - 2)]
         bs = B if len(layers) <= 3 else 1
@@ -352,7 +362,7 @@ def reference_arm(args):
         return
     times = []
     for i in range(args.warmup + args.steps):
-        sec, desc, threads, n = oracle_sample_time(args.workload)
+        sec, desc, threads, n = oracle_sample_time(args.workload, args.n_params)
         if i >= args.warmup:
             times.append(sec)
     sec = statistics.mean(times)
@@ -374,6 +384,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="vgc", choices=["vgc", "reference"])
+    ap.add_argument("--n-params", type=int, default=1 << 25, help="size of the 'flat' workload")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -394,7 +405,8 @@ def main():
     import paper_1802_06058_b200 as vgc
     vgc.load_library()
     pk = peaks()
-    hp = HotPath(args.workload, worker=rank * 16, n_input_sets=1, n_g_sets=max(4, min(args.steps + args.warmup, 16)))
+    hp = HotPath(args.workload, worker=rank * 16, n_input_sets=1, n_g_sets=max(4, min(args.steps + args.warmup, 16)),
+                 n_params=args.n_params)
     torch.cuda.synchronize()
 
     sampler = ClockSampler(local_rank)
@@ -460,7 +472,7 @@ def main():
         line["e2e"] = {"value": world * n / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
                        "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        sec, desc, threads, _ = oracle_sample_time(args.workload)
+        sec, desc, threads, _ = oracle_sample_time(args.workload, args.n_params)
         line["cpu_baseline"] = {"value": n / sec / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
                                 "sample": desc, "host_cores_available": os.cpu_count()}
     if rank == 0:

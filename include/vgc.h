@@ -45,7 +45,7 @@ typedef enum {
 
 /* bits OR-ed into *dev_status by kernels */
 #define VGC_DEV_CAPACITY 1u /* word buffer too small: message truncated, state still correct             */
-#define VGC_DEV_TIMEOUT 2u  /* a bounded wait between thread blocks gave up: outputs of this call invalid */
+#define VGC_DEV_TIMEOUT 2u  /* a bounded wait inside a kernel gave up: outputs of this call are invalid    */
 #define VGC_DEV_RANGE 4u    /* decode met an index >= n: that word was skipped                           */
 
 /* group_exp value of a weight tensor from which nothing was sent */

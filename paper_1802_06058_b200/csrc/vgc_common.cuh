@@ -14,11 +14,6 @@ namespace vgc {
 
 constexpr int kWarp = 32;
 
-// Upper bound on polls of a flag written by another thread block.  Each poll sleeps ~64 ns
-// once the fast retries are used up, so the bound is of the order of a second; after it the
-// waiter records VGC_DEV_TIMEOUT and carries on with a value of zero instead of hanging.
-constexpr uint32_t kSpinLimit = 1u << 22;
-
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -78,61 +73,11 @@ __device__ __forceinline__ int group_of(const uint32_t *offs, int K, uint32_t i)
     return lo;
 }
 
-// Decoupled look-back over per-tile status words {flag:2 | payload:62}.  Called by one full
-// warp.  Publishes this tile's aggregate, sums the aggregates of the preceding tiles until
-// one with a complete prefix is met, publishes the inclusive prefix and returns the
-// exclusive one.  Payloads add as plain 64-bit integers (several packed counters are fine
-// as long as no field overflows into its neighbour).  Tiles must have been numbered in the
-// order their blocks started (ticket from an atomic counter), so every tile waited for is
-// already running; every wait is bounded all the same.
-constexpr uint64_t kFlagAgg = 1ull << 62;
-constexpr uint64_t kFlagPrefix = 2ull << 62;
-constexpr uint64_t kPayloadMask = (1ull << 62) - 1;
-
 __device__ __forceinline__ uint64_t warp_sum_u64(uint64_t x)
 {
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) x += __shfl_xor_sync(0xffffffffu, x, d);
     return x;
-}
-
-__device__ __forceinline__ uint64_t lookback_exclusive(uint64_t *status, uint32_t tile, uint64_t total,
-                                                       uint32_t *dev_status)
-{
-    const uint32_t lane = lane_id();
-    if (tile == 0) {
-        if (lane == 0) st_volatile_u64(status, kFlagPrefix | total);
-        return 0;
-    }
-    if (lane == 0) st_volatile_u64(status + tile, kFlagAgg | total);
-    uint64_t excl = 0;
-    int64_t pos = (int64_t)tile - 1;
-    bool timed_out = false;
-    while (true) {
-        int64_t idx = pos - lane;
-        uint64_t st = kFlagPrefix;                 // tiles "before 0" carry an empty prefix
-        if (idx >= 0) {
-            st = ld_volatile_u64(status + idx);
-            uint32_t spins = 0;
-            while ((st >> 62) == 0) {
-                if (++spins > kSpinLimit) { timed_out = true; st = kFlagPrefix; break; }
-                if (spins > 16) __nanosleep(64);
-                st = ld_volatile_u64(status + idx);
-            }
-        }
-        const uint32_t has_prefix = __ballot_sync(0xffffffffu, (st >> 62) == 2);
-        uint64_t contrib = st & kPayloadMask;
-        if (has_prefix) {
-            const uint32_t first = __ffs(has_prefix) - 1;     // nearest tile with a full prefix
-            if (lane > first) contrib = 0;
-        }
-        excl += warp_sum_u64(contrib);
-        if (has_prefix) break;
-        pos -= 32;
-    }
-    if (__any_sync(0xffffffffu, timed_out) && lane == 0) atomicOr(dev_status, VGC_DEV_TIMEOUT);
-    if (lane == 0) st_volatile_u64(status + tile, kFlagPrefix | (excl + total));
-    return excl;
 }
 
 }  // namespace vgc

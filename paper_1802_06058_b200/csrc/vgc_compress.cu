@@ -8,12 +8,15 @@
 //            (index, value) pairs, in index order, into its own 2048-slot segment of a staging
 //            area and records how many there are; a per-tensor atomicMax on |value| bit
 //            patterns yields M_k.  Thread blocks never wait for one another here.
-//   phase B  runs over the staged pairs only: quantises against E_k = floor(log2 M_k), drops
-//            d > 7 and packs the words in ascending index order.  One warp owns one segment;
-//            positions across thread blocks come from a decoupled look-back over per-tile
-//            counts, with tiles numbered by an atomic ticket and every wait bounded.
+//   phase B  runs over the staged pairs only, one warp per segment, in two kernels: "count"
+//            quantises against E_k = floor(log2 M_k) and records how many pairs of each
+//            segment survive (d <= 7); "emit" turns those counts into positions (a block sums
+//            the totals of the chunks before its own, then scans its 32 segments) and packs
+//            the words in ascending index order.
+// No thread block ever waits for another one: ordering comes from kernel boundaries only.
 // The per-tensor maximum has to be complete before any value can be quantised, which is why
-// the work is split in two; the staged pairs are a small fraction of the buffer.
+// the work is split; the staged pairs are a small fraction of the buffer and stay in L2
+// between the count and emit kernels.
 #include "vgc_common.cuh"
 
 namespace vgc {
@@ -22,31 +25,26 @@ constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / kWarp;             // 8
 constexpr int kRowsA = 2;                            // float4 vectors per thread per tile
 constexpr int kTileA = kThreads * kRowsA * 4;        // 2048 parameters per tile = one staging segment
-constexpr int kSegPerTileB = kWarps;                 // phase B: one warp per segment
+constexpr int kSegPerChunk = 32;                     // phase B: segments per thread block (4 per warp)
 constexpr int kOffsSmem = 1024;                      // group offsets cached in shared memory
 
-struct CompressHeader {      // first bytes of the workspace, zeroed by every call
-    uint32_t ticket_b;
-    uint32_t pad[3];
-};
-
 struct CompressLayout {
-    size_t gmax, status_b, tile_count, stage_idx, stage_val, total;
-    size_t zero_bytes;       // header + gmax + status array are cleared per call
-    uint32_t tiles_a, tiles_b;
+    size_t gmax, tile_count, kept_count, chunk_total, stage_idx, stage_val, total;
+    size_t zero_bytes;       // the per-tensor maxima are cleared per call
+    uint32_t tiles_a, chunks;
 };
 
 static CompressLayout compress_layout(size_t n, int K)
 {
     CompressLayout L;
     L.tiles_a = (uint32_t)((n + kTileA - 1) / kTileA);
-    L.tiles_b = (L.tiles_a + kSegPerTileB - 1) / kSegPerTileB;
-    size_t off = sizeof(CompressHeader);
-    L.gmax = off;          off = round_up(off + sizeof(uint32_t) * (size_t)K, 16);
-    L.status_b = off;      off += sizeof(uint64_t) * L.tiles_b;
-    off = round_up(off, 256);
+    L.chunks = (L.tiles_a + kSegPerChunk - 1) / kSegPerChunk;
+    size_t off = 0;
+    L.gmax = off;          off = round_up(off + sizeof(uint32_t) * (size_t)K, 256);
     L.zero_bytes = off;
     L.tile_count = off;    off = round_up(off + sizeof(uint32_t) * L.tiles_a, 256);
+    L.kept_count = off;    off = round_up(off + sizeof(uint32_t) * L.tiles_a, 256);
+    L.chunk_total = off;   off = round_up(off + sizeof(uint64_t) * L.chunks, 256);
     const size_t slots = (size_t)L.tiles_a * kTileA;
     L.stage_idx = off;     off = round_up(off + sizeof(uint32_t) * slots, 256);
     L.stage_val = off;     off = round_up(off + sizeof(uint32_t) * slots, 256);
@@ -234,99 +232,145 @@ __device__ __forceinline__ bool encode_pair(uint32_t idx, uint32_t bits, const u
     return d <= 7;
 }
 
-constexpr uint64_t kPassedShift = 31;       // look-back payload: passed << 31 | kept (each < 2^29)
+constexpr uint64_t kPassedShift = 32;       // chunk totals: passed << 32 | kept
+
+// One warp walks one segment in index order, four 32-wide slices per round so that the loads
+// of a round are in flight together.  EMIT: write the words from position `pos` on.
+// Returns the number of pairs kept.
+template <bool EMIT>
+__device__ __forceinline__ uint32_t walk_segment(const uint32_t *__restrict__ seg_idx,
+                                                 const uint32_t *__restrict__ seg_val, uint32_t count,
+                                                 const uint32_t *offs, int K, const uint32_t *gmax,
+                                                 uint32_t *__restrict__ words, uint32_t pos, uint32_t capacity)
+{
+    const uint32_t lane = lane_id();
+    int k = 0;
+    int32_t Ek = INT32_MIN;
+    uint32_t kept = 0;
+    for (uint32_t q0 = 0; q0 < count; q0 += 128) {
+        uint32_t idx[4], bits[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t q = q0 + u * 32 + lane;
+            idx[u] = 0; bits[u] = 0;
+            if (q < count) { idx[u] = seg_idx[q]; bits[u] = seg_val[q]; }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t q = q0 + u * 32 + lane;
+            bool keep = false;
+            uint32_t word = 0;
+            if (q < count) keep = encode_pair(idx[u], bits[u], offs, K, gmax, k, Ek, word);
+            const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
+            if (EMIT) {
+                const uint32_t p = pos + kept + __popc(ballot & ((1u << lane) - 1u));
+                if (keep && p < capacity) words[p] = word;
+            }
+            kept += __popc(ballot);
+        }
+    }
+    return kept;
+}
 
 __global__ void __launch_bounds__(kThreads)
-compress_phase_b(const uint32_t *__restrict__ group_offsets, int K, CompressHeader *hdr,
-                 const uint32_t *__restrict__ gmax, const uint32_t *__restrict__ tile_count, uint32_t n_tiles_a,
-                 const uint32_t *__restrict__ stage_idx, const uint32_t *__restrict__ stage_val,
-                 uint64_t *status, uint32_t *__restrict__ words, uint32_t capacity,
-                 int32_t *__restrict__ group_exp, uint32_t *nnz_out, uint32_t *n_criterion,
-                 uint32_t *n_dropped, uint32_t *dev_status)
+compress_count(const uint32_t *__restrict__ group_offsets, int K, const uint32_t *__restrict__ gmax,
+               const uint32_t *__restrict__ tile_count, uint32_t n_tiles_a,
+               const uint32_t *__restrict__ stage_idx, const uint32_t *__restrict__ stage_val,
+               uint32_t *__restrict__ kept_count, uint64_t *__restrict__ chunk_total,
+               int32_t *__restrict__ group_exp)
 {
     __shared__ uint32_t sm_offs[kOffsSmem];
-    __shared__ uint32_t sm_kept[kWarps], sm_passed[kWarps], sm_excl[kWarps];
-    __shared__ uint32_t sm_tile[2];
-
+    __shared__ unsigned long long sm_tot[kWarps];
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool offs_in_smem = (K + 1) <= kOffsSmem;
-    if (offs_in_smem)
+    if (offs_in_smem) {
         for (int i = tid; i <= K; i += kThreads) sm_offs[i] = group_offsets[i];
+        __syncthreads();
+    }
     const uint32_t *offs = offs_in_smem ? sm_offs : group_offsets;
-    const uint32_t n_tiles = (n_tiles_a + kSegPerTileB - 1) / kSegPerTileB;
-
     if (blockIdx.x == 0)
         for (int k = tid; k < K; k += kThreads) {
             const uint32_t m = gmax[k];
             group_exp[k] = m ? (int32_t)((m >> 23) & 0xFFu) - 127 : VGC_EXP_NONE;
         }
-    if (tid == 0) sm_tile[0] = atomicAdd(&hdr->ticket_b, 1u);
+    unsigned long long tot = 0;
+#pragma unroll 1
+    for (int i = 0; i < kSegPerChunk / kWarps; ++i) {
+        const uint32_t seg = blockIdx.x * kSegPerChunk + i * kWarps + warp;
+        if (seg >= n_tiles_a) break;
+        const uint32_t count = tile_count[seg];
+        const uint32_t kept = walk_segment<false>(stage_idx + (size_t)seg * kTileA, stage_val + (size_t)seg * kTileA,
+                                                  count, offs, K, gmax, nullptr, 0, 0);
+        if (lane == 0) kept_count[seg] = kept;
+        tot += ((unsigned long long)count << kPassedShift) | kept;
+    }
+    if (lane == 0) sm_tot[warp] = tot;
     __syncthreads();
-
-    for (uint32_t it = 0;; ++it) {
-        const uint32_t tile = sm_tile[it & 1];
-        if (tile >= n_tiles) break;
-        if (tid == 0) sm_tile[(it + 1) & 1] = atomicAdd(&hdr->ticket_b, 1u);
-
-        const uint32_t seg = tile * kSegPerTileB + warp;
-        const uint32_t count = seg < n_tiles_a ? tile_count[seg] : 0;
-        const uint32_t *seg_idx = stage_idx + (size_t)seg * kTileA;
-        const uint32_t *seg_val = stage_val + (size_t)seg * kTileA;
-
-        // pass 1: how many of this segment's pairs survive the quantiser
-        int k = 0;
-        int32_t Ek = INT32_MIN;
-        uint32_t kept = 0;
-        for (uint32_t q0 = 0; q0 < count; q0 += 32) {
-            const uint32_t q = q0 + lane;
-            bool keep = false;
-            if (q < count) {
-                uint32_t word;
-                keep = encode_pair(seg_idx[q], seg_val[q], offs, K, gmax, k, Ek, word);
-            }
-            kept += __popc(__ballot_sync(0xffffffffu, keep));
-        }
-        if (lane == 0) { sm_kept[warp] = kept; sm_passed[warp] = count; }
-        __syncthreads();                                           // (1)
-        if (warp == 0) {
-            const uint32_t mine = lane < kWarps ? sm_kept[lane] : 0;
-            const uint32_t pass = lane < kWarps ? sm_passed[lane] : 0;
-            uint32_t ki = mine, pi = pass;
+    if (tid == 0) {
+        unsigned long long t = 0;
 #pragma unroll
-            for (int d = 1; d < kWarps; d <<= 1) {
-                const uint32_t ku = __shfl_up_sync(0xffffffffu, ki, d);
-                const uint32_t pu = __shfl_up_sync(0xffffffffu, pi, d);
-                if (lane >= d) { ki += ku; pi += pu; }
-            }
-            const uint32_t tot_kept = __shfl_sync(0xffffffffu, ki, kWarps - 1);
-            const uint32_t tot_pass = __shfl_sync(0xffffffffu, pi, kWarps - 1);
-            const uint64_t excl = lookback_exclusive(status, tile, ((uint64_t)tot_pass << kPassedShift) | tot_kept,
-                                                     dev_status);
-            const uint32_t excl_kept = (uint32_t)(excl & ((1ull << kPassedShift) - 1));
-            const uint32_t excl_pass = (uint32_t)(excl >> kPassedShift);
-            if (lane < kWarps) sm_excl[lane] = excl_kept + ki - mine;
-            if (lane == 0) {
-                if (tile == n_tiles - 1) {
-                    *nnz_out = excl_kept + tot_kept;
-                    *n_criterion = excl_pass + tot_pass;
-                    *n_dropped = (excl_pass + tot_pass) - (excl_kept + tot_kept);
-                }
-                if (excl_kept + tot_kept > capacity) atomicOr(dev_status, VGC_DEV_CAPACITY);
+        for (int w = 0; w < kWarps; ++w) t += sm_tot[w];
+        chunk_total[blockIdx.x] = t;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+compress_emit(const uint32_t *__restrict__ group_offsets, int K, const uint32_t *__restrict__ gmax,
+              const uint32_t *__restrict__ tile_count, uint32_t n_tiles_a,
+              const uint32_t *__restrict__ stage_idx, const uint32_t *__restrict__ stage_val,
+              const uint32_t *__restrict__ kept_count, const uint64_t *__restrict__ chunk_total,
+              uint32_t *__restrict__ words, uint32_t capacity, uint32_t *nnz_out, uint32_t *n_criterion,
+              uint32_t *n_dropped, uint32_t *dev_status)
+{
+    __shared__ uint32_t sm_offs[kOffsSmem];
+    __shared__ unsigned long long sm_tot[kWarps];
+    __shared__ uint32_t sm_pos[kSegPerChunk];
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool offs_in_smem = (K + 1) <= kOffsSmem;
+    if (offs_in_smem)
+        for (int i = tid; i <= K; i += kThreads) sm_offs[i] = group_offsets[i];
+    const uint32_t *offs = offs_in_smem ? sm_offs : group_offsets;
+
+    // totals of all chunks before this one
+    unsigned long long before = 0;
+    for (uint32_t c = tid; c < blockIdx.x; c += kThreads) before += chunk_total[c];
+    before = warp_sum_u64(before);
+    if (lane == 0) sm_tot[warp] = before;
+    __syncthreads();
+    before = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) before += sm_tot[w];
+    const uint32_t kept_before = (uint32_t)(before & 0xFFFFFFFFull);
+
+    if (warp == 0) {                                   // positions of this chunk's 32 segments
+        const uint32_t seg = blockIdx.x * kSegPerChunk + lane;
+        const uint32_t mine = seg < n_tiles_a ? kept_count[seg] : 0;
+        uint32_t incl = mine;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += up;
+        }
+        sm_pos[lane] = kept_before + incl - mine;
+        if (lane == 31) {
+            const uint32_t end = kept_before + incl;
+            if (end > capacity) atomicOr(dev_status, VGC_DEV_CAPACITY);
+            if (blockIdx.x == gridDim.x - 1) {
+                const unsigned long long all = before + chunk_total[blockIdx.x];
+                *nnz_out = (uint32_t)(all & 0xFFFFFFFFull);
+                *n_criterion = (uint32_t)(all >> kPassedShift);
+                *n_dropped = (uint32_t)(all >> kPassedShift) - (uint32_t)(all & 0xFFFFFFFFull);
             }
         }
-        __syncthreads();                                           // (2)
-        // pass 2: same pairs again (cache hits), now with their final positions
-        uint32_t pos = sm_excl[warp];
-        for (uint32_t q0 = 0; q0 < count; q0 += 32) {
-            const uint32_t q = q0 + lane;
-            bool keep = false;
-            uint32_t word = 0;
-            if (q < count) keep = encode_pair(seg_idx[q], seg_val[q], offs, K, gmax, k, Ek, word);
-            const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
-            const uint32_t p = pos + __popc(ballot & ((1u << lane) - 1u));
-            if (keep && p < capacity) words[p] = word;
-            pos += __popc(ballot);
-        }
+    }
+    __syncthreads();
+#pragma unroll 1
+    for (int i = 0; i < kSegPerChunk / kWarps; ++i) {
+        const uint32_t local = i * kWarps + warp;
+        const uint32_t seg = blockIdx.x * kSegPerChunk + local;
+        if (seg >= n_tiles_a) break;
+        walk_segment<true>(stage_idx + (size_t)seg * kTileA, stage_val + (size_t)seg * kTileA, tile_count[seg],
+                           offs, K, gmax, words, sm_pos[local], capacity);
     }
 }
 
@@ -363,10 +407,10 @@ extern "C" vgc_status vgc_compress(const float *g, const float *s, float *r, flo
     if (ws_bytes < L.total) return VGC_ERR_WORKSPACE;
 
     char *base = static_cast<char *>(ws);
-    CompressHeader *hdr = reinterpret_cast<CompressHeader *>(base);
     uint32_t *gmax = reinterpret_cast<uint32_t *>(base + L.gmax);
-    uint64_t *status_b = reinterpret_cast<uint64_t *>(base + L.status_b);
     uint32_t *tile_count = reinterpret_cast<uint32_t *>(base + L.tile_count);
+    uint32_t *kept_count = reinterpret_cast<uint32_t *>(base + L.kept_count);
+    uint64_t *chunk_total = reinterpret_cast<uint64_t *>(base + L.chunk_total);
     uint32_t *stage_idx = reinterpret_cast<uint32_t *>(base + L.stage_idx);
     uint32_t *stage_val = reinterpret_cast<uint32_t *>(base + L.stage_val);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
@@ -383,11 +427,12 @@ extern "C" vgc_status vgc_compress(const float *g, const float *s, float *r, flo
     const uint32_t grid_a = L.tiles_a < (uint32_t)(sm_count * 8) ? L.tiles_a : (uint32_t)(sm_count * 8);
     compress_phase_a<<<grid_a, kThreads, 0, st>>>(g, s, r, v, n, group_offsets, K, alpha, zeta, gmax, tile_count,
                                                   stage_idx, stage_val, out->mask, L.tiles_a);
-    const uint32_t grid_b = L.tiles_b < (uint32_t)(sm_count * 8) ? L.tiles_b : (uint32_t)(sm_count * 8);
-    compress_phase_b<<<grid_b, kThreads, 0, st>>>(group_offsets, K, hdr, gmax, tile_count, L.tiles_a, stage_idx,
-                                                  stage_val, status_b, out->words, out->capacity, out->group_exp,
-                                                  out->nnz, out->n_criterion, out->n_dropped, out->dev_status);
-    count_launch(2);
+    compress_count<<<L.chunks, kThreads, 0, st>>>(group_offsets, K, gmax, tile_count, L.tiles_a, stage_idx,
+                                                  stage_val, kept_count, chunk_total, out->group_exp);
+    compress_emit<<<L.chunks, kThreads, 0, st>>>(group_offsets, K, gmax, tile_count, L.tiles_a, stage_idx,
+                                                 stage_val, kept_count, chunk_total, out->words, out->capacity,
+                                                 out->nnz, out->n_criterion, out->n_dropped, out->dev_status);
+    count_launch(3);
     VGC_CUDA_OK(cudaGetLastError());
     return VGC_OK;
 }
