@@ -1,4 +1,6 @@
 // C ABI of the squared per-example gradient sums (argument checks and kernel choice).
+#include <cstdlib>
+
 #include "vgc_common.cuh"
 
 namespace vgc {
@@ -8,11 +10,30 @@ vgc_status simt_sqgrad_linear(const float *x, const float *delta, int B, int in,
 vgc_status simt_sqgrad_conv(const float *x, const float *delta, int B, int C, int H, int W, int Cout,
                             int Kh, int Kw, int sh, int sw, int ph, int pw, int Ho, int Wo, float scale,
                             int accumulate, float *S, void *ws, size_t ws_bytes, cudaStream_t st);
+bool tc_linear_supported(int B, int in, int out);
+bool tc_conv_supported(int B, int C, int H, int W, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw);
+size_t tc_linear_workspace_bytes(int B, int in, int out);
+size_t tc_conv1x1_workspace_bytes(int B, int C, int P, int Cout);
+vgc_status tc_sqgrad_linear(const float *x, const float *delta, int B, int in, int out, float scale, int accumulate,
+                            float *S, void *ws, size_t ws_bytes, cudaStream_t st);
+vgc_status tc_sqgrad_conv1x1(const float *x, const float *delta, int B, int C, int P, int Cout, float scale,
+                             int accumulate, float *S, void *ws, size_t ws_bytes, cudaStream_t st);
 }  // namespace vgc
 
 using namespace vgc;
 
 namespace {
+// VGC_SQGRAD_PATH=simt forces the CUDA-core kernel (cross-checks, shapes under suspicion)
+bool use_tensor_cores()
+{
+    static int v = -1;
+    if (v < 0) {
+        const char *e = getenv("VGC_SQGRAD_PATH");
+        v = (e && e[0] == 's') ? 0 : 1;
+    }
+    return v == 1;
+}
+
 bool conv_shape_ok(int B, int C, int H, int W, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw,
                    int *Ho, int *Wo)
 {
@@ -29,7 +50,9 @@ bool conv_shape_ok(int B, int C, int H, int W, int Cout, int Kh, int Kw, int sh,
 extern "C" size_t vgc_sqgrad_linear_workspace_bytes(int B, int in, int out)
 {
     if (B <= 0 || in <= 0 || out <= 0) return 0;
-    return round_up(simt_workspace_bytes(out, in, B), 256);
+    size_t need = simt_workspace_bytes(out, in, B) + 256;
+    if (tc_linear_supported(B, in, out)) need = need > tc_linear_workspace_bytes(B, in, out) ? need : tc_linear_workspace_bytes(B, in, out);
+    return round_up(need > 256 ? need : 256, 256);
 }
 
 extern "C" vgc_status vgc_sqgrad_linear(const float *x, const float *delta, int B, int in, int out,
@@ -42,8 +65,12 @@ extern "C" vgc_status vgc_sqgrad_linear(const float *x, const float *delta, int 
     if (B > 0 && (!x || !delta || !aligned16(x) || !aligned16(delta))) return VGC_ERR_INVALID_ARG;
     if (!(scale == scale)) return VGC_ERR_INVALID_ARG;
     if (ws_bytes < vgc_sqgrad_linear_workspace_bytes(B, in, out) || (ws_bytes && !ws)) return VGC_ERR_WORKSPACE;
-    return simt_sqgrad_linear(x, delta, B, in, out, scale, accumulate, S, ws, ws_bytes,
-                              reinterpret_cast<cudaStream_t>(stream));
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (use_tensor_cores() && tc_linear_supported(B, in, out))
+        return tc_sqgrad_linear(x, delta, B, in, out, scale, accumulate, S, ws, ws_bytes, st);
+    VGC_CUDA_OK(cudaMemsetAsync(ws, 0, 4, st));          // status word: nothing to report on this path
+    return simt_sqgrad_linear(x, delta, B, in, out, scale, accumulate, S, static_cast<char *>(ws) + 256,
+                              ws_bytes - 256, st);
 }
 
 extern "C" size_t vgc_sqgrad_conv_workspace_bytes(int B, int C, int H, int W, int Cout, int Kh, int Kw,
@@ -52,7 +79,12 @@ extern "C" size_t vgc_sqgrad_conv_workspace_bytes(int B, int C, int H, int W, in
     int Ho, Wo;
     if (!conv_shape_ok(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, &Ho, &Wo)) return 0;
     if (B == 0 || C == 0 || Cout == 0) return 0;
-    return round_up(simt_workspace_bytes(Cout, C * Kh * Kw, B * Ho * Wo), 256);
+    size_t need = simt_workspace_bytes(Cout, C * Kh * Kw, B * Ho * Wo);
+    if (tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w)) {
+        const size_t t = tc_conv1x1_workspace_bytes(B, C, H * W, Cout);
+        need = need > t ? need : t;
+    }
+    return round_up(need + 256, 256);
 }
 
 extern "C" vgc_status vgc_sqgrad_conv(const float *x, const float *delta, int B, int C, int H, int W, int Cout,
@@ -70,8 +102,12 @@ extern "C" vgc_status vgc_sqgrad_conv(const float *x, const float *delta, int B,
     if (ws_bytes < vgc_sqgrad_conv_workspace_bytes(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w) ||
         (ws_bytes && !ws))
         return VGC_ERR_WORKSPACE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (B > 0 && use_tensor_cores() && tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w))
+        return tc_sqgrad_conv1x1(x, delta, B, C, H * W, Cout, scale, accumulate, S, ws, ws_bytes, st);
+    VGC_CUDA_OK(cudaMemsetAsync(ws, 0, 4, st));          // status word: nothing to report on this path
     return simt_sqgrad_conv(x, delta, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho, Wo, scale,
-                            accumulate, S, ws, ws_bytes, reinterpret_cast<cudaStream_t>(stream));
+                            accumulate, S, static_cast<char *>(ws) + 256, ws_bytes - 256, st);
 }
 
 extern "C" const char *vgc_status_string(int status)

@@ -14,6 +14,10 @@ def _ws(nbytes):
     return torch.empty(max(nbytes, 16), dtype=torch.uint8, device="cuda")
 
 
+def _status(ws):
+    return int(ws[:4].view(torch.int32).item())
+
+
 def _check(got, want):
     want64 = want.astype(np.float64)
     err = np.abs(got.astype(np.float64) - want64)
@@ -27,6 +31,7 @@ def run_linear(x, d, scale, S0=None):
     S = torch.empty(n_out, n_in, device="cuda") if S0 is None else S0.clone()
     ws = _ws(vgc.vgc_sqgrad_linear_workspace_bytes(B, n_in, n_out))
     vgc.vgc_sqgrad_linear(x, d, scale, S, accumulate=S0 is not None, ws=ws)
+    assert _status(ws) == 0
     return S.cpu().numpy()
 
 
@@ -36,11 +41,13 @@ def run_conv(x, d, k, s, p, scale, S0=None):
     S = torch.empty(Cout, C, k, k, device="cuda") if S0 is None else S0.clone()
     ws = _ws(vgc.vgc_sqgrad_conv_workspace_bytes(B, C, H, W, Cout, k, k, s, s, p, p))
     vgc.vgc_sqgrad_conv(x, d, (k, k), (s, s), (p, p), scale, S, accumulate=S0 is not None, ws=ws)
+    assert _status(ws) == 0
     return S.cpu().numpy()
 
 
 @pytest.mark.parametrize("B,n_in,n_out", [(32, 256, 128), (128, 784, 1024), (128, 1024, 10), (1, 5, 3),
-                                          (7, 130, 67), (64, 1000, 333), (300, 64, 64), (2, 1, 1)])
+                                          (7, 130, 67), (64, 1000, 333), (300, 64, 64), (2, 1, 1),
+                                          (32, 2048, 1000), (64, 36, 260), (1000, 128, 132)])
 def test_linear(B, n_in, n_out):
     gen = torch.Generator(device="cuda"); gen.manual_seed(B * 131 + n_in)
     x = torch.randn(B, n_in, device="cuda", generator=gen).clamp_(min=0)     # ReLU-dead inputs
@@ -67,6 +74,9 @@ CONV_SHAPES = [  # B, C, H, Cout, k, stride, pad
     (2, 3, 9, 4, 3, 1, 1), (3, 5, 8, 6, 1, 1, 0), (2, 4, 9, 3, 1, 2, 0), (2, 3, 20, 8, 7, 2, 3),
     (4, 16, 14, 24, 3, 2, 1), (2, 64, 14, 64, 3, 1, 1), (2, 70, 7, 130, 1, 1, 0), (3, 8, 5, 5, 5, 1, 0),
     (1, 1, 3, 1, 3, 1, 1),
+    # 1x1 / stride 1 / no padding: the tensor-core path (whole and ragged tiles, split reductions)
+    (2, 64, 8, 64, 1, 1, 0), (3, 256, 14, 64, 1, 1, 0), (2, 100, 12, 200, 1, 1, 0), (4, 64, 56, 64, 1, 1, 0),
+    (2, 8, 6, 8, 1, 1, 0), (5, 300, 10, 136, 1, 1, 0),
 ]
 
 
@@ -99,4 +109,7 @@ def test_long_reduction_all_ones_is_exact():
     # K = 2*224*224 = 100352 terms of exactly 1: any one-sided rounding in the accumulation shows up
     x = torch.ones(2, 4, 224, 224, device="cuda"); d = torch.ones(2, 8, 224, 224, device="cuda")
     got = run_conv(x, d, 1, 1, 0, 1.0)
+    assert np.all(got == 2 * 224 * 224)
+    x = torch.ones(2, 8, 224, 224, device="cuda"); d = torch.ones(2, 16, 224, 224, device="cuda")
+    got = run_conv(x, d, 1, 1, 0, 1.0)                      # tensor-core path
     assert np.all(got == 2 * 224 * 224)
