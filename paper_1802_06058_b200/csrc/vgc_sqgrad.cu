@@ -13,11 +13,12 @@ vgc_status simt_sqgrad_conv(const float *x, const float *delta, int B, int C, in
 bool tc_linear_supported(int B, int in, int out);
 bool tc_conv_supported(int B, int C, int H, int W, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw);
 size_t tc_linear_workspace_bytes(int B, int in, int out);
-size_t tc_conv1x1_workspace_bytes(int B, int C, int P, int Cout);
+size_t tc_conv_workspace_bytes(int B, int C, int Kh, int Kw, int P, int Cout);
 vgc_status tc_sqgrad_linear(const float *x, const float *delta, int B, int in, int out, float scale, int accumulate,
                             float *S, void *ws, size_t ws_bytes, cudaStream_t st);
-vgc_status tc_sqgrad_conv1x1(const float *x, const float *delta, int B, int C, int P, int Cout, float scale,
-                             int accumulate, float *S, void *ws, size_t ws_bytes, cudaStream_t st);
+vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int H, int W, int Cout, int Kh, int Kw,
+                          int sh, int sw, int ph, int pw, int Ho, int Wo, float scale, int accumulate, float *S,
+                          void *ws, size_t ws_bytes, cudaStream_t st);
 }  // namespace vgc
 
 using namespace vgc;
@@ -81,7 +82,7 @@ extern "C" size_t vgc_sqgrad_conv_workspace_bytes(int B, int C, int H, int W, in
     if (B == 0 || C == 0 || Cout == 0) return 0;
     size_t need = simt_workspace_bytes(Cout, C * Kh * Kw, B * Ho * Wo);
     if (tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w)) {
-        const size_t t = tc_conv1x1_workspace_bytes(B, C, H * W, Cout);
+        const size_t t = tc_conv_workspace_bytes(B, C, Kh, Kw, Ho * Wo, Cout);
         need = need > t ? need : t;
     }
     return round_up(need + 256, 256);
@@ -104,7 +105,8 @@ extern "C" vgc_status vgc_sqgrad_conv(const float *x, const float *delta, int B,
         return VGC_ERR_WORKSPACE;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     if (B > 0 && use_tensor_cores() && tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w))
-        return tc_sqgrad_conv1x1(x, delta, B, C, H * W, Cout, scale, accumulate, S, ws, ws_bytes, st);
+        return tc_sqgrad_conv(x, delta, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho, Wo, scale,
+                              accumulate, S, ws, ws_bytes, st);
     VGC_CUDA_OK(cudaMemsetAsync(ws, 0, 4, st));          // status word: nothing to report on this path
     return simt_sqgrad_conv(x, delta, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho, Wo, scale,
                             accumulate, S, static_cast<char *>(ws) + 256, ws_bytes - 256, st);

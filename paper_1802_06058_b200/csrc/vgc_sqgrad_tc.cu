@@ -15,11 +15,16 @@
 // fp32 registers while the next chunk accumulates into the second TMEM buffer.
 // Long reductions are split across blockIdx.z; partial tiles are combined in a fixed order.
 //
-// Operand layouts covered here (everything else takes the CUDA-core kernel):
-//   conv, 1x1 kernel, stride 1, no padding: A = delta[z][o][p], B = x[z][c][p]  (k = (z,p) innermost: K-major)
-//   dense layer:                            A = delta[z][out],  B = x[z][in]    (m / n innermost: MN-major)
+// Operand layouts:
+//   dense layer: A = delta[z][out], B = x[z][in]  (m / n innermost: MN-major tiles, both by TMA)
+//   conv layer:  A = delta[z][o][p], p = (ho,wo) innermost (K-major); B is the im2col view of x,
+//                row n = (c,kh,kw), column k = (z,ho,wo).  Each example contributes ceil(P/32) slices.
+//                A tile: TMA when the row pitch P*4 is a multiple of 16 bytes, else gathered.
+//                B tile: TMA for a 1x1 / stride 1 / unpadded kernel (then it is just x[z][c][p]);
+//                otherwise the transform warps gather it straight from global memory, four
+//                consecutive k per thread, zero outside the image -- im2col is never materialised.
 //
-// Warp roles (320 threads): 0 TMA producer, 1 MMA issuer + TMEM owner, 2-5 transform, 6-9 epilogue.
+// Warp roles (448 threads): 0 TMA producer, 1 MMA issuer + TMEM owner, 2-9 transform, 10-13 epilogue.
 // Every wait on an mbarrier is bounded; on expiry the block raises an abort flag, all roles fall
 // through to the common exit, outstanding TMA loads are waited for (bounded) and TMEM is freed.
 #include <cuda.h>
@@ -37,8 +42,9 @@ constexpr int kBN = 128;            // output columns per block (UMMA N)
 constexpr int kBK = 32;             // k per pipeline slice (= 128 bytes of fp32)
 constexpr int kRawStages = 3;
 constexpr int kOpStages = 2;
-constexpr int kThreadsTc = 320;
-constexpr int kTransformWarps = 4;
+constexpr int kThreadsTc = 448;
+constexpr int kTransformWarps = 8;
+constexpr int kTransformThreads = 32 * kTransformWarps;
 constexpr int kEpilogueWarps = 4;
 constexpr uint32_t kRawBytesA = kBM * kBK * 4;                      // 16 KB
 constexpr uint32_t kRawBytesB = kBN * kBK * 4;                      // 16 KB
@@ -59,6 +65,8 @@ struct Params {
     uint32_t tx_bytes;       // bytes the TMA loads of one slice deliver
     float scale;
     int accumulate;
+    const float *x, *delta;  // raw operands (gathered tiles)
+    int C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, Wo, P;     // conv geometry (gathered tiles)
     float *S;                // final output [M][N] (used when gridDim.z == 1)
     float *partial;          // [gridDim.z][M][N] otherwise
     uint32_t *error_flag;    // device word, set to 1 if a wait expired
@@ -180,10 +188,28 @@ __host__ __device__ constexpr uint32_t instr_desc(int major)
 }
 
 // ---- the kernel ------------------------------------------------------------------------------
-template <int kMajor>
+// One 16-byte chunk (4 consecutive k of one row) of a K-major 128-byte-swizzled tile.
+__device__ __forceinline__ uint32_t chunk_offset(int row, int kq) { return (uint32_t)row * 128u + (uint32_t)((kq ^ (row & 7)) << 4); }
+
+__device__ __forceinline__ void split_store(uint8_t *hi_tile, uint8_t *lo_tile, uint32_t off, float v0, float v1, float v2, float v3)
+{
+    const float q0 = __fmul_rn(v0, v0), q1 = __fmul_rn(v1, v1), q2 = __fmul_rn(v2, v2), q3 = __fmul_rn(v3, v3);
+    uint4 h, l;
+    h.x = to_tf32(q0); h.y = to_tf32(q1); h.z = to_tf32(q2); h.w = to_tf32(q3);
+    l.x = to_tf32(__fsub_rn(q0, __uint_as_float(h.x)));
+    l.y = to_tf32(__fsub_rn(q1, __uint_as_float(h.y)));
+    l.z = to_tf32(__fsub_rn(q2, __uint_as_float(h.z)));
+    l.w = to_tf32(__fsub_rn(q3, __uint_as_float(h.w)));
+    *reinterpret_cast<uint4 *>(hi_tile + off) = h;
+    *reinterpret_cast<uint4 *>(lo_tile + off) = l;
+}
+
+template <int kMajor, bool kGatherA, bool kGatherB>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const Params prm)
 {
+    static_assert(kMajor == kMajorK || (!kGatherA && !kGatherB), "gathered tiles are K-major");
+    constexpr bool kAnyTma = !kGatherA || !kGatherB;
     extern __shared__ uint8_t smem_raw_[];
     __shared__ __align__(8) uint64_t bars[2 * kRawStages + 2 * kOpStages + 5];
     __shared__ uint32_t tmem_base_slot;
@@ -226,7 +252,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 
     if (warp == 0) {
         // ================= TMA producer (one thread) =================
-        if (lane == 0) {
+        if (lane == 0 && kAnyTma) {
             int issued = 0;
             for (int i = 0; i < n_slices; ++i) {
                 const int st = i % kRawStages;
@@ -238,8 +264,8 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                 const int slice = slice_begin + i;
                 if (kMajor == kMajorK) {
                     const int z = slice / prm.p_slices, p0 = (slice - z * prm.p_slices) * kBK;
-                    tma_load_3d(dst_a, &map_a, full, p0, m0, z);
-                    tma_load_3d(dst_b, &map_b, full, p0, n0, z);
+                    if (!kGatherA) tma_load_3d(dst_a, &map_a, full, p0, m0, z);
+                    if (!kGatherB) tma_load_3d(dst_b, &map_b, full, p0, n0, z);
                 } else {
                     const int k0 = slice * kBK;
 #pragma unroll
@@ -307,33 +333,143 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         }
     } else if (warp < 2 + kTransformWarps) {
         // ================= transform warps: square and split into TF32 hi / lo =================
-        const uint32_t t = threadIdx.x - 64;                              // 0..127
+        const int t = (int)threadIdx.x - 64;                               // 0..255
+        const int kq = t & 7, row0 = t >> 3;                               // gathered chunks: rows row0 + 32*i, k = 4*kq..4*kq+3
+        constexpr int kRowsPerThread = kBM * 8 / kTransformThreads;        // 4
+
+        // ---- per-thread constants of the gathered tiles
+        int b_base[kRowsPerThread], b_dh[kRowsPerThread], b_dw[kRowsPerThread];
+        bool b_ok[kRowsPerThread], a_ok[kRowsPerThread];
+        int ho[4], wo[4];                    // output position of this thread's four k in the current slice
+        int ho_init[4], wo_init[4];
+        int q32 = 0, r32 = 0;
+        int z = 0, pblk = 0;
+        if (kGatherA || kGatherB) {
+            const int khw = prm.Kh * prm.Kw;
+#pragma unroll
+            for (int i = 0; i < kRowsPerThread; ++i) {
+                const int n = n0 + row0 + 32 * i;
+                b_ok[i] = n < prm.N;
+                const int nn = b_ok[i] ? n : 0;
+                const int c = nn / khw, rem = nn - c * khw;
+                const int kh = rem / prm.Kw, kw = rem - kh * prm.Kw;
+                b_dh[i] = kh - prm.ph;
+                b_dw[i] = kw - prm.pw;
+                b_base[i] = (c * prm.H + b_dh[i]) * prm.W + b_dw[i];
+                a_ok[i] = m0 + row0 + 32 * i < prm.M;
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                ho_init[j] = (kq * 4 + j) / prm.Wo;
+                wo_init[j] = (kq * 4 + j) - ho_init[j] * prm.Wo;
+            }
+            q32 = kBK / prm.Wo;
+            r32 = kBK - q32 * prm.Wo;
+            z = slice_begin / prm.p_slices;
+            pblk = slice_begin - z * prm.p_slices;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int p = pblk * kBK + kq * 4 + j;
+                ho[j] = p / prm.Wo;
+                wo[j] = p - ho[j] * prm.Wo;
+            }
+        }
+        float va[kGatherA ? kRowsPerThread : 1][4], vb[kGatherB ? kRowsPerThread : 1][4];
+
+        // loads of the gathered chunks of the slice the (z, pblk, ho, wo) state points at
+        auto gather = [&](float (&ga)[kGatherA ? kRowsPerThread : 1][4], float (&gb)[kGatherB ? kRowsPerThread : 1][4]) {
+            const int pbase = pblk * kBK + kq * 4;
+            if (kGatherB) {
+                const float *xz = prm.x + (size_t)z * prm.C * prm.H * prm.W;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const bool pv = pbase + j < prm.P;
+                    const int hs = ho[j] * prm.sh, ws = wo[j] * prm.sw;
+                    const int poff = hs * prm.W + ws;
+#pragma unroll
+                    for (int i = 0; i < kRowsPerThread; ++i) {
+                        const bool ok = pv && b_ok[i] && (unsigned)(hs + b_dh[i]) < (unsigned)prm.H &&
+                                        (unsigned)(ws + b_dw[i]) < (unsigned)prm.W;
+                        gb[i][j] = ok ? __ldg(xz + (b_base[i] + poff)) : 0.f;
+                    }
+                }
+            }
+            if (kGatherA) {
+#pragma unroll
+                for (int i = 0; i < kRowsPerThread; ++i) {
+                    const float *dr = prm.delta + ((size_t)z * prm.Cout + (m0 + row0 + 32 * i)) * prm.P + pbase;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) ga[i][j] = (a_ok[i] && pbase + j < prm.P) ? __ldg(dr + j) : 0.f;
+                }
+            }
+        };
+        auto advance = [&]() {
+            if (++pblk == prm.p_slices) {
+                pblk = 0;
+                ++z;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { ho[j] = ho_init[j]; wo[j] = wo_init[j]; }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    ho[j] += q32;
+                    wo[j] += r32;
+                    if (wo[j] >= prm.Wo) { wo[j] -= prm.Wo; ++ho[j]; }
+                }
+            }
+        };
+
+        if (kGatherA || kGatherB) gather(va, vb);
         for (int i = 0; i < n_slices; ++i) {
             const int rs = i % kRawStages, os = i % kOpStages;
-            if (!mbar_wait(smem_u32(&raw_full[rs]), (uint32_t)(i / kRawStages) & 1u, &abort_flag)) break;
+            float wa[kGatherA ? kRowsPerThread : 1][4], wb[kGatherB ? kRowsPerThread : 1][4];
+            if ((kGatherA || kGatherB) && i + 1 < n_slices) {           // next slice's loads fly during this transform
+                advance();
+                gather(wa, wb);
+            }
+            if (kAnyTma && !mbar_wait(smem_u32(&raw_full[rs]), (uint32_t)(i / kRawStages) & 1u, &abort_flag)) break;
             if (!mbar_wait(smem_u32(&op_empty[os]), ((uint32_t)(i / kOpStages) & 1u) ^ 1u, &abort_flag)) break;
-            const float4 *raw = reinterpret_cast<const float4 *>(smem_gen + rs * kRawStageBytes);
-            uint4 *hi = reinterpret_cast<uint4 *>(smem_gen + kRawStages * kRawStageBytes + os * kOpStageBytes);
-            uint4 *lo = hi + kRawStageBytes / 16;
+            uint8_t *raw = smem_gen + rs * kRawStageBytes;
+            uint8_t *hi = smem_gen + kRawStages * kRawStageBytes + os * kOpStageBytes;
+            uint8_t *lo = hi + kRawStageBytes;
+            // tiles that came by TMA: elementwise over their 16-byte chunks (layout is inherited)
+            {
+                const uint32_t c_begin = kGatherA ? kRawBytesA / 16 : 0;
+                const uint32_t c_end = kGatherB ? kRawBytesA / 16 : kRawStageBytes / 16;
 #pragma unroll 4
-            for (uint32_t c = t; c < kRawStageBytes / 16; c += 32 * kTransformWarps) {
-                const float4 v = raw[c];
-                const float q0 = __fmul_rn(v.x, v.x), q1 = __fmul_rn(v.y, v.y), q2 = __fmul_rn(v.z, v.z),
-                            q3 = __fmul_rn(v.w, v.w);
-                uint4 h, l;
-                h.x = to_tf32(q0); h.y = to_tf32(q1); h.z = to_tf32(q2); h.w = to_tf32(q3);
-                l.x = to_tf32(__fsub_rn(q0, __uint_as_float(h.x)));
-                l.y = to_tf32(__fsub_rn(q1, __uint_as_float(h.y)));
-                l.z = to_tf32(__fsub_rn(q2, __uint_as_float(h.z)));
-                l.w = to_tf32(__fsub_rn(q3, __uint_as_float(h.w)));
-                hi[c] = h;
-                lo[c] = l;
+                for (uint32_t c = c_begin + (uint32_t)t; c < c_end; c += kTransformThreads) {
+                    const float4 v = *reinterpret_cast<const float4 *>(raw + 16 * c);
+                    split_store(hi, lo, 16 * c, v.x, v.y, v.z, v.w);
+                }
+            }
+            if (kGatherA) {
+#pragma unroll
+                for (int r = 0; r < kRowsPerThread; ++r)
+                    split_store(hi, lo, chunk_offset(row0 + 32 * r, kq), va[r][0], va[r][1], va[r][2], va[r][3]);
+            }
+            if (kGatherB) {
+#pragma unroll
+                for (int r = 0; r < kRowsPerThread; ++r)
+                    split_store(hi + kRawBytesA, lo + kRawBytesA, chunk_offset(row0 + 32 * r, kq), vb[r][0], vb[r][1],
+                                vb[r][2], vb[r][3]);
             }
             fence_async_smem();                                   // generic-proxy writes -> tensor core reads
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(smem_u32(&op_full[os]));
-                mbar_arrive(smem_u32(&raw_empty[rs]));
+                if (kAnyTma) mbar_arrive(smem_u32(&raw_empty[rs]));
+            }
+            if (kGatherA) {
+#pragma unroll
+                for (int r = 0; r < kRowsPerThread; ++r)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) va[r][j] = wa[r][j];
+            }
+            if (kGatherB) {
+#pragma unroll
+                for (int r = 0; r < kRowsPerThread; ++r)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) vb[r][j] = wb[r][j];
             }
         }
     } else {
@@ -473,9 +609,11 @@ bool tc_linear_supported(int B, int in, int out)
 }
 bool tc_conv_supported(int B, int C, int H, int W, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw)
 {
-    const long P = (long)H * W;
-    return Kh == 1 && Kw == 1 && sh == 1 && sw == 1 && ph == 0 && pw == 0 && P >= 32 && P % 4 == 0 && B >= 1 &&
-           C >= 8 && Cout >= 8 && ((long)C * P) % 4 == 0;
+    const long Ho = (H + 2 * ph - Kh) / sh + 1, Wo = (W + 2 * pw - Kw) / sw + 1;
+    const long P = Ho * Wo, N = (long)C * Kh * Kw;
+    // 32-bit index arithmetic inside the kernel
+    return B >= 1 && C >= 1 && Cout >= 1 && (long)C * H * W < (1L << 30) && N < (1L << 24) &&
+           (long)B * ((P + kBK - 1) / kBK) < (1L << 30);
 }
 
 size_t tc_workspace_bytes(int M, int N, int k_slices)
@@ -484,34 +622,38 @@ size_t tc_workspace_bytes(int M, int N, int k_slices)
     return 256 + (p.splits > 1 ? (size_t)p.splits * M * N * sizeof(float) : 0);
 }
 
-static vgc_status tc_launch(int major, const CUtensorMap &ma, const CUtensorMap &mb, int M, int N, int k_slices,
-                            int p_slices, uint32_t tx_bytes, float scale, int accumulate, float *S, void *ws, size_t ws_bytes,
-                            cudaStream_t st)
+enum Variant { kDense, kConvTmaTma, kConvTmaGather, kConvGatherGather };
+
+static vgc_status tc_launch(Variant variant, const CUtensorMap &ma, const CUtensorMap &mb, Params prm, int M, int N,
+                            int k_slices, void *ws, size_t ws_bytes, cudaStream_t st)
 {
     const Plan plan = make_plan(M, N, k_slices);
     if (ws_bytes < tc_workspace_bytes(M, N, k_slices)) return VGC_ERR_WORKSPACE;
     static bool attr_set = false;
     if (!attr_set) {
-        VGC_CUDA_OK(cudaFuncSetAttribute(sqgrad_tc<kMajorK>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-        VGC_CUDA_OK(cudaFuncSetAttribute(sqgrad_tc<kMajorMN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        VGC_CUDA_OK(cudaFuncSetAttribute(sqgrad_tc<kMajorMN, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        VGC_CUDA_OK(cudaFuncSetAttribute(sqgrad_tc<kMajorK, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        VGC_CUDA_OK(cudaFuncSetAttribute(sqgrad_tc<kMajorK, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        VGC_CUDA_OK(cudaFuncSetAttribute(sqgrad_tc<kMajorK, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
         attr_set = true;
     }
-    Params prm;
     prm.M = M; prm.N = N; prm.k_slices = k_slices; prm.slices_per_split = plan.slices_per_split;
-    prm.p_slices = p_slices; prm.chunk = default_chunk(); prm.tx_bytes = tx_bytes; prm.scale = scale; prm.accumulate = accumulate;
-    prm.S = S;
+    prm.chunk = default_chunk();
     prm.error_flag = static_cast<uint32_t *>(ws);
     prm.partial = reinterpret_cast<float *>(static_cast<char *>(ws) + 256);
     VGC_CUDA_OK(cudaMemsetAsync(ws, 0, 4, st));
     dim3 grid((N + kBN - 1) / kBN, (M + kBM - 1) / kBM, plan.splits);
-    if (major == kMajorK)
-        sqgrad_tc<kMajorK><<<grid, kThreadsTc, kSmemBytes, st>>>(ma, mb, prm);
-    else
-        sqgrad_tc<kMajorMN><<<grid, kThreadsTc, kSmemBytes, st>>>(ma, mb, prm);
+    switch (variant) {
+        case kDense: sqgrad_tc<kMajorMN, false, false><<<grid, kThreadsTc, kSmemBytes, st>>>(ma, mb, prm); break;
+        case kConvTmaTma: sqgrad_tc<kMajorK, false, false><<<grid, kThreadsTc, kSmemBytes, st>>>(ma, mb, prm); break;
+        case kConvTmaGather: sqgrad_tc<kMajorK, false, true><<<grid, kThreadsTc, kSmemBytes, st>>>(ma, mb, prm); break;
+        case kConvGatherGather: sqgrad_tc<kMajorK, true, true><<<grid, kThreadsTc, kSmemBytes, st>>>(ma, mb, prm); break;
+    }
     count_launch();
     if (plan.splits > 1) {
         const size_t mn = (size_t)M * N;
-        sqgrad_tc_combine<<<(unsigned)((mn + 255) / 256), 256, 0, st>>>(prm.partial, plan.splits, mn, scale, accumulate, S);
+        sqgrad_tc_combine<<<(unsigned)((mn + 255) / 256), 256, 0, st>>>(prm.partial, plan.splits, mn, prm.scale,
+                                                                         prm.accumulate, prm.S);
         count_launch();
     }
     return cudaGetLastError() == cudaSuccess ? VGC_OK : VGC_ERR_CUDA;
@@ -529,29 +671,47 @@ vgc_status tc_sqgrad_linear(const float *x, const float *delta, int B, int in, i
     if (!make_map(&ma, delta, 2, dims_a, str_a, box, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) ||
         !make_map(&mb, x, 2, dims_b, str_b, box, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B))
         return VGC_ERR_CUDA;
-    return tc_launch(kMajorMN, ma, mb, out, in, (B + kBK - 1) / kBK, 0, kRawStageBytes, scale, accumulate, S, ws, ws_bytes, st);
+    Params prm = {};
+    prm.p_slices = 1; prm.tx_bytes = kRawStageBytes; prm.scale = scale; prm.accumulate = accumulate; prm.S = S;
+    return tc_launch(kDense, ma, mb, prm, out, in, (B + kBK - 1) / kBK, ws, ws_bytes, st);
 }
 
-size_t tc_conv1x1_workspace_bytes(int B, int C, int P, int Cout)
+size_t tc_conv_workspace_bytes(int B, int C, int Kh, int Kw, int P, int Cout)
 {
-    return tc_workspace_bytes(Cout, C, B * ((P + kBK - 1) / kBK));
+    return tc_workspace_bytes(Cout, C * Kh * Kw, B * ((P + kBK - 1) / kBK));
 }
 
-vgc_status tc_sqgrad_conv1x1(const float *x, const float *delta, int B, int C, int P, int Cout, float scale,
-                             int accumulate, float *S, void *ws, size_t ws_bytes, cudaStream_t st)
+vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int H, int W, int Cout, int Kh, int Kw,
+                          int sh, int sw, int ph, int pw, int Ho, int Wo, float scale, int accumulate, float *S,
+                          void *ws, size_t ws_bytes, cudaStream_t st)
 {
-    CUtensorMap ma, mb;
+    const int P = Ho * Wo, N = C * Kh * Kw;
     const int p_slices = (P + kBK - 1) / kBK;
-    const cuuint32_t box_a[3] = {(cuuint32_t)kBK, (cuuint32_t)(Cout < kBM ? Cout : kBM), 1};
-    const cuuint32_t box_b[3] = {(cuuint32_t)kBK, (cuuint32_t)(C < kBN ? C : kBN), 1};
-    const cuuint64_t dims_a[3] = {(cuuint64_t)P, (cuuint64_t)Cout, (cuuint64_t)B};
-    const cuuint64_t str_a[2] = {(cuuint64_t)P * 4, (cuuint64_t)Cout * P * 4};
-    const cuuint64_t dims_b[3] = {(cuuint64_t)P, (cuuint64_t)C, (cuuint64_t)B};
-    const cuuint64_t str_b[2] = {(cuuint64_t)P * 4, (cuuint64_t)C * P * 4};
-    if (!make_map(&ma, delta, 3, dims_a, str_a, box_a, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_map(&mb, x, 3, dims_b, str_b, box_b, CU_TENSOR_MAP_SWIZZLE_128B))
-        return VGC_ERR_CUDA;
-    return tc_launch(kMajorK, ma, mb, Cout, C, B * p_slices, p_slices, (box_a[1] + box_b[1]) * kBK * 4, scale, accumulate, S, ws, ws_bytes, st);
+    const bool a_tma = P >= kBK && P % 4 == 0;
+    const bool b_tma = a_tma && Kh == 1 && Kw == 1 && sh == 1 && sw == 1 && ph == 0 && pw == 0;
+    CUtensorMap ma = {}, mb = {};
+    uint32_t tx = 0;
+    if (a_tma) {
+        const cuuint32_t box_a[3] = {(cuuint32_t)kBK, (cuuint32_t)(Cout < kBM ? Cout : kBM), 1};
+        const cuuint64_t dims_a[3] = {(cuuint64_t)P, (cuuint64_t)Cout, (cuuint64_t)B};
+        const cuuint64_t str_a[2] = {(cuuint64_t)P * 4, (cuuint64_t)Cout * P * 4};
+        if (!make_map(&ma, delta, 3, dims_a, str_a, box_a, CU_TENSOR_MAP_SWIZZLE_128B)) return VGC_ERR_CUDA;
+        tx += box_a[1] * kBK * 4;
+    }
+    if (b_tma) {
+        const cuuint32_t box_b[3] = {(cuuint32_t)kBK, (cuuint32_t)(C < kBN ? C : kBN), 1};
+        const cuuint64_t dims_b[3] = {(cuuint64_t)P, (cuuint64_t)C, (cuuint64_t)B};
+        const cuuint64_t str_b[2] = {(cuuint64_t)P * 4, (cuuint64_t)C * P * 4};
+        if (!make_map(&mb, x, 3, dims_b, str_b, box_b, CU_TENSOR_MAP_SWIZZLE_128B)) return VGC_ERR_CUDA;
+        tx += box_b[1] * kBK * 4;
+    }
+    Params prm = {};
+    prm.p_slices = p_slices; prm.tx_bytes = tx; prm.scale = scale; prm.accumulate = accumulate; prm.S = S;
+    prm.x = x; prm.delta = delta;
+    prm.C = C; prm.H = H; prm.W = W; prm.Cout = Cout; prm.Kh = Kh; prm.Kw = Kw; prm.sh = sh; prm.sw = sw;
+    prm.ph = ph; prm.pw = pw; prm.Wo = Wo; prm.P = P;
+    const Variant v = b_tma ? kConvTmaTma : (a_tma ? kConvTmaGather : kConvGatherGather);
+    return tc_launch(v, ma, mb, prm, Cout, N, B * p_slices, ws, ws_bytes, st);
 }
 
 }  // namespace vgc
