@@ -118,7 +118,7 @@ class HotPath:
     """All device buffers of one worker and the launches of one step."""
 
     def __init__(self, name: str, worker: int, n_input_sets: int, n_g_sets: int, device="cuda",
-                 n_params: int = 1 << 25):
+                 n_params: int = 1 << 25, n_streams: int = 4):
         import paper_1802_06058_b200 as vgc
         from paper_1802_06058_b200 import workloads
         self.vgc, self.wl = vgc, workloads
@@ -164,7 +164,12 @@ class HotPath:
                         spec.pad, spec.pad))
                 else:
                     ws_bytes = max(ws_bytes, vgc.vgc_sqgrad_linear_workspace_bytes(B, spec.cin, spec.cout))
-            self.ws_s = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+            self.ws_s = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+            # independent layers are spread over a few streams (each with its own workspace) so that one
+            # layer's tail and the next one's start overlap; the whole step is then replayed as a CUDA graph
+            self.n_streams = n_streams
+            self.side = [torch.cuda.Stream() for _ in range(max(n_streams - 1, 0))]
+            self.ws_side = [torch.zeros(ws_bytes, dtype=torch.uint8, device=dev) for _ in self.side]
             for t in range(n_input_sets):
                 self.inputs.append([workloads.layer_inputs(spec, B, cfg, worker, t, li, x_kind, delta_std, dev)
                                     for li, spec in enumerate(self.layers)])
@@ -200,14 +205,56 @@ class HotPath:
         if self.compress_only:
             return
         ins = self.inputs[t % len(self.inputs)]
+        main = torch.cuda.current_stream()
+        for st in self.side:
+            st.wait_stream(main)
         for li, spec in enumerate(self.layers):
             x, delta = ins[li]
             S = self.s[int(self.offsets[li]):int(self.offsets[li + 1])]
+            lane = li % self.n_streams
+            stream = main if lane == 0 else self.side[lane - 1]
+            ws = self.ws_s if lane == 0 else self.ws_side[lane - 1]
             if spec.kind == "conv":
                 vgc.vgc_sqgrad_conv(x, delta, (spec.k, spec.k), (spec.stride, spec.stride), (spec.pad, spec.pad),
-                                    self.scale, S, ws=self.ws_s)
+                                    self.scale, S, ws=ws, stream=stream)
             else:
-                vgc.vgc_sqgrad_linear(x, delta, self.scale, S, ws=self.ws_s)
+                vgc.vgc_sqgrad_linear(x, delta, self.scale, S, ws=ws, stream=stream)
+        for st in self.side:
+            main.wait_stream(st)
+
+    def per_layer_times(self, reps: int = 5):
+        """Median device time of each layer's sqgrad call (ms), for profiling."""
+        vgc = self.vgc
+        out = []
+        ins = self.inputs[0]
+        for li, spec in enumerate(self.layers):
+            x, delta = ins[li]
+            S = self.s[int(self.offsets[li]):int(self.offsets[li + 1])]
+            def call():
+                if spec.kind == "conv":
+                    vgc.vgc_sqgrad_conv(x, delta, (spec.k, spec.k), (spec.stride, spec.stride), (spec.pad, spec.pad),
+                                        self.scale, S, ws=self.ws_s)
+                else:
+                    vgc.vgc_sqgrad_linear(x, delta, self.scale, S, ws=self.ws_s)
+            call(); torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                for _ in range(10):
+                    call()
+            times = []
+            for r in range(reps + 2):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                graph.replay()
+                e1.record()
+                torch.cuda.synchronize()
+                if r >= 2:
+                    times.append(e0.elapsed_time(e1) / 10)
+            M, N, K = spec.gemm_mnk(self.batch)
+            ms = statistics.median(times)
+            out.append({"layer": spec.name, "M": M, "N": N, "K": K, "ms": round(ms, 4),
+                        "useful_tflops": round(2 * M * N * K / (ms * 1e-3) / 1e12, 2)})
+        return out
 
     def compress(self, t: int):
         s = self.s if self.s_sets is None else self.s_sets[t % len(self.s_sets)]
@@ -229,9 +276,34 @@ class HotPath:
         if marks: marks[2].record()
 
 
-def run_device_timed(hp: HotPath, steps: int, warmup: int, dist_on: bool):
+class GraphedStep:
+    """The launches of one step captured once per input set and replayed (CUDA graph): the step is a
+    fixed sequence of ~60 small launches, so replaying removes the host launch cost from the loop."""
+
+    def __init__(self, hp: HotPath, n_variants: int):
+        self.graphs = []
+        self.launches = []
+        for t in range(n_variants):
+            hp.step(t)                                   # eager once: first-call set-up happens outside capture
+        torch.cuda.synchronize()
+        for t in range(n_variants):
+            before = hp.vgc.vgc_kernel_launch_count()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                hp.step(t)
+            self.launches.append(hp.vgc.vgc_kernel_launch_count() - before)
+            self.graphs.append(g)
+        self.hp = hp
+
+    def replay(self, t: int):
+        self.graphs[t % len(self.graphs)].replay()
+
+
+def run_device_timed(hp: HotPath, steps: int, warmup: int, dist_on: bool, use_graph: bool = True):
     vgc = hp.vgc
     ev = lambda: torch.cuda.Event(enable_timing=True)
+    if use_graph:
+        return run_graph_timed(hp, steps, warmup, dist_on)
     for t in range(warmup):
         hp.step(t)
     torch.cuda.synchronize()
@@ -255,6 +327,46 @@ def run_device_timed(hp: HotPath, steps: int, warmup: int, dist_on: bool):
     co = [m[0].elapsed_time(m[1]) for m in marks]
     de = [m[1].elapsed_time(m[2]) for m in marks]
     return total_ms, sq, co, de, launches
+
+
+def run_graph_timed(hp: HotPath, steps: int, warmup: int, dist_on: bool):
+    """Timed region = K graph replays (whole steps) bracketed by events; the per-section split comes from
+    a second, untimed pass in which each section is replayed as its own graph."""
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    n_var = len(hp.g_sets)
+    gs = GraphedStep(hp, n_var)
+    for t in range(warmup):
+        gs.replay(t)
+    torch.cuda.synchronize()
+    if dist_on:
+        torch.distributed.barrier()
+    torch.cuda.synchronize()
+    start, stop = ev(), ev()
+    start.record()
+    for i in range(steps):
+        gs.replay(warmup + i)
+    stop.record()
+    torch.cuda.synchronize()
+    if dist_on:
+        torch.distributed.barrier()
+    total_ms = start.elapsed_time(stop)
+    launches = sum(gs.launches[(warmup + i) % n_var] for i in range(steps))
+    # section split (outside the timed region): one graph per section
+    secs = []
+    for fn in (hp.sqgrad, hp.compress, hp.decode):
+        g = torch.cuda.CUDAGraph()
+        fn(0); torch.cuda.synchronize()
+        with torch.cuda.graph(g):
+            fn(0)
+        times = []
+        for r in range(max(steps, 5) + 2):
+            e0, e1 = ev(), ev()
+            e0.record(); g.replay(); e1.record()
+            torch.cuda.synchronize()
+            if r >= 2:
+                times.append(e0.elapsed_time(e1))
+        secs.append(times)
+    return total_ms, secs[0], secs[1], secs[2], launches
 
 
 def run_e2e(hp: HotPath, steps: int, warmup: int):
@@ -385,6 +497,9 @@ def main():
     ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="vgc", choices=["vgc", "reference"])
     ap.add_argument("--n-params", type=int, default=1 << 25, help="size of the 'flat' workload")
+    ap.add_argument("--per-layer", action="store_true", help="print per-layer sqgrad times instead of the bench line")
+    ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
+    ap.add_argument("--streams", type=int, default=4, help="streams the independent sqgrad layers are spread over")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -406,12 +521,20 @@ def main():
     vgc.load_library()
     pk = peaks()
     hp = HotPath(args.workload, worker=rank * 16, n_input_sets=1, n_g_sets=max(4, min(args.steps + args.warmup, 16)),
-                 n_params=args.n_params)
+                 n_params=args.n_params, n_streams=max(args.streams, 1))
     torch.cuda.synchronize()
+
+    if args.per_layer:
+        rows = hp.per_layer_times()
+        for row in rows:
+            print(json.dumps(row))
+        print(json.dumps({"total_ms": sum(r["ms"] for r in rows)}))
+        return
 
     sampler = ClockSampler(local_rank)
     sampler.start()
-    total_ms, sq, co, de, launches = run_device_timed(hp, args.steps, max(args.warmup, 3), dist_on)
+    total_ms, sq, co, de, launches = run_device_timed(hp, args.steps, max(args.warmup, 3), dist_on,
+                                                      use_graph=not args.no_graph)
     clocks = sampler.stop()
     counters = hp.out.read()
     ms_per_step = total_ms / args.steps
@@ -459,7 +582,8 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "f32 (tf32x3 products where tensor cores are used)",
             "data": "synthetic",
             "config": {"workload": args.workload, "n_params": n, "batch": hp.batch, "W": hp.W, "alpha": hp.alpha,
-                       "zeta": ZETA, "groups": hp.K,
+                       "zeta": ZETA, "groups": hp.K, "launch": "eager" if args.no_graph else "cuda graph replay",
+                       "sqgrad_streams": getattr(hp, "n_streams", 1),
                        "l2": "inputs larger than L2 (no flush)" if n * 16 > 126e6 else "state fits in L2 (no flush): cache-resident numbers"},
             "gpu_launches": int(launches), "clocks": clocks, "sections": sections, "roofline": roofline}
 

@@ -75,8 +75,9 @@ uint64_t vgc_kernel_launch_count(void);
  *   S      [out][in] fp32 row-major (the layer's slice of the flat buffer)
  *   accumulate  0: S = result   1: S += result
  *   ws / ws_bytes  scratch of at least vgc_sqgrad_linear_workspace_bytes(B, in, out) (never less than
- *                  256 bytes).  After the call the first 32-bit word of ws is a status word: 0, or
- *                  VGC_DEV_TIMEOUT if a bounded wait inside the kernel gave up (S is then invalid).
+ *                  256 bytes).  The first 32-bit word of ws is a status word the caller zeroes once
+ *                  (e.g. when allocating ws): kernels only ever OR bits into it -- VGC_DEV_TIMEOUT
+ *                  if a bounded wait inside a kernel gave up, in which case S is invalid.
  *
  * Result within 1e-5 relative of the exact sum.  B, in, out >= 1 (any of them 0: no-op, OK).
  * ------------------------------------------------------------------------------------------- */

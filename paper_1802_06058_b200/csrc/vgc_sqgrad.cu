@@ -69,7 +69,6 @@ extern "C" vgc_status vgc_sqgrad_linear(const float *x, const float *delta, int 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     if (use_tensor_cores() && tc_linear_supported(B, in, out))
         return tc_sqgrad_linear(x, delta, B, in, out, scale, accumulate, S, ws, ws_bytes, st);
-    VGC_CUDA_OK(cudaMemsetAsync(ws, 0, 4, st));          // status word: nothing to report on this path
     return simt_sqgrad_linear(x, delta, B, in, out, scale, accumulate, S, static_cast<char *>(ws) + 256,
                               ws_bytes - 256, st);
 }
@@ -107,7 +106,6 @@ extern "C" vgc_status vgc_sqgrad_conv(const float *x, const float *delta, int B,
     if (B > 0 && use_tensor_cores() && tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w))
         return tc_sqgrad_conv(x, delta, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho, Wo, scale,
                               accumulate, S, ws, ws_bytes, st);
-    VGC_CUDA_OK(cudaMemsetAsync(ws, 0, 4, st));          // status word: nothing to report on this path
     return simt_sqgrad_conv(x, delta, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho, Wo, scale,
                             accumulate, S, static_cast<char *>(ws) + 256, ws_bytes - 256, st);
 }

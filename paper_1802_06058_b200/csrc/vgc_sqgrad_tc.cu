@@ -17,12 +17,14 @@
 //
 // Operand layouts:
 //   dense layer: A = delta[z][out], B = x[z][in]  (m / n innermost: MN-major tiles, both by TMA)
-//   conv layer:  A = delta[z][o][p], p = (ho,wo) innermost (K-major); B is the im2col view of x,
-//                row n = (c,kh,kw), column k = (z,ho,wo).  Each example contributes ceil(P/32) slices.
-//                A tile: TMA when the row pitch P*4 is a multiple of 16 bytes, else gathered.
-//                B tile: TMA for a 1x1 / stride 1 / unpadded kernel (then it is just x[z][c][p]);
-//                otherwise the transform warps gather it straight from global memory, four
-//                consecutive k per thread, zero outside the image -- im2col is never materialised.
+//   conv layer:  the error tile is delta[z][o][p], p = (ho,wo) innermost (K-major); the input tile is
+//                the im2col view of x, row (c,kh,kw), column k = (z,ho,wo).  Each example contributes
+//                ceil(P/32) slices.  Error tile: TMA when the row pitch P*4 is a multiple of 16 bytes,
+//                else gathered.  Input tile: TMA for a 1x1 / stride 1 / unpadded kernel (then it is
+//                just x[z][c][p]); otherwise the transform warps gather it straight from global
+//                memory, four consecutive k per thread, zero outside the image -- im2col is never
+//                materialised.  With few output channels (Cout <= 64) the roles are swapped: the
+//                im2col rows become the 128-row A tile and the errors the narrow B tile.
 //
 // Warp roles (448 threads): 0 TMA producer, 1 MMA issuer + TMEM owner, 2-9 transform, 10-13 epilogue.
 // Every wait on an mbarrier is bounded; on expiry the block raises an abort flag, all roles fall
@@ -56,20 +58,23 @@ constexpr uint32_t kWaitLimit = 1u << 22;                           // polls bef
 
 enum { kMajorK = 0, kMajorMN = 1 };
 
+enum { kTma = 0, kGatherErr = 1, kGatherIm2col = 2 };      // how a tile gets its rows
+
 struct Params {
-    int M, N;
+    int M, N;                // rows of the A tile space / of the B tile space
     int k_slices;            // total 32-deep slices of the reduction
     int slices_per_split;
-    int p_slices;            // conv: slices per example (ceil(P/32)); dense: unused
+    int p_slices;            // conv: slices per example (ceil(P/32)); dense: 1
     int chunk;               // slices per accumulator drain
     uint32_t tx_bytes;       // bytes the TMA loads of one slice deliver
     float scale;
     int accumulate;
     const float *x, *delta;  // raw operands (gathered tiles)
     int C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, Wo, P;     // conv geometry (gathered tiles)
-    float *S;                // final output [M][N] (used when gridDim.z == 1)
-    float *partial;          // [gridDim.z][M][N] otherwise
-    uint32_t *error_flag;    // device word, set to 1 if a wait expired
+    float *S;                // result: element (m, n) lives at S[m*ld_m + n*ld_n]; one of the two is 1
+    long long ld_m, ld_n;
+    float *partial;          // split-K scratch [split][tile][column][row], used when gridDim.z > 1
+    uint32_t *status;        // device word; VGC_DEV_TIMEOUT is OR-ed in if a wait expired
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -180,11 +185,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
     return d;
 }
 
-// Instruction descriptor: D fp32, A and B tf32, given major-ness, M = 128, N = kBN.
-__host__ __device__ constexpr uint32_t instr_desc(int major)
+// Instruction descriptor: D fp32, A and B tf32, given major-ness, M = 128, N = n (multiple of 16).
+__host__ __device__ constexpr uint32_t instr_desc(int major, int n)
 {
     return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)major << 15) | ((uint32_t)major << 16) |
-           ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
 }
 
 // ---- the kernel ------------------------------------------------------------------------------
@@ -204,12 +209,74 @@ __device__ __forceinline__ void split_store(uint8_t *hi_tile, uint8_t *lo_tile, 
     *reinterpret_cast<uint4 *>(lo_tile + off) = l;
 }
 
-template <int kMajor, bool kGatherA, bool kGatherB>
+constexpr int kRowsPerThread = kBM * 8 / kTransformThreads;        // 4 gathered chunks per thread per tile
+
+// The four rows (row0 + 32*i) of a gathered tile that one transform thread owns.
+template <int kMode>
+struct GatherRows {
+    int base[kRowsPerThread], dh[kRowsPerThread], dw[kRowsPerThread];
+    bool ok[kRowsPerThread];
+
+    __device__ __forceinline__ void init(const Params &prm, int first_row, int limit)
+    {
+        if (kMode == kTma) return;
+        const int khw = prm.Kh * prm.Kw;
+#pragma unroll
+        for (int i = 0; i < kRowsPerThread; ++i) {
+            const int idx = first_row + 32 * i;
+            ok[i] = idx < limit;
+            const int ii = ok[i] ? idx : 0;
+            if (kMode == kGatherIm2col) {
+                const int c = ii / khw, rem = ii - c * khw;
+                const int kh = rem / prm.Kw, kw = rem - kh * prm.Kw;
+                dh[i] = kh - prm.ph;
+                dw[i] = kw - prm.pw;
+                base[i] = (c * prm.H + dh[i]) * prm.W + dw[i];
+            } else {
+                base[i] = ii;           // output channel
+                dh[i] = dw[i] = 0;
+            }
+        }
+    }
+    // loads this thread's 4 x 4 elements of the slice at (z, pbase .. pbase+3)
+    __device__ __forceinline__ void load(const Params &prm, int z, int pbase, const int (&ho)[4], const int (&wo)[4],
+                                         float (&v)[kRowsPerThread][4]) const
+    {
+        if (kMode == kGatherIm2col) {
+            const float *xz = prm.x + (size_t)z * prm.C * prm.H * prm.W;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const bool pv = pbase + j < prm.P;
+                const int hs = ho[j] * prm.sh, ws = wo[j] * prm.sw;
+                const int poff = hs * prm.W + ws;
+#pragma unroll
+                for (int i = 0; i < kRowsPerThread; ++i) {
+                    const bool in = pv && ok[i] && (unsigned)(hs + dh[i]) < (unsigned)prm.H &&
+                                    (unsigned)(ws + dw[i]) < (unsigned)prm.W;
+                    v[i][j] = in ? __ldg(xz + (base[i] + poff)) : 0.f;
+                }
+            }
+        } else if (kMode == kGatherErr) {
+#pragma unroll
+            for (int i = 0; i < kRowsPerThread; ++i) {
+                const float *dr = prm.delta + ((size_t)z * prm.Cout + base[i]) * prm.P + pbase;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) v[i][j] = (ok[i] && pbase + j < prm.P) ? __ldg(dr + j) : 0.f;
+            }
+        }
+    }
+};
+
+// ---- the kernel ------------------------------------------------------------------------------
+template <int kMajor, int kModeA, int kModeB>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const Params prm)
 {
-    static_assert(kMajor == kMajorK || (!kGatherA && !kGatherB), "gathered tiles are K-major");
+    static_assert(kMajor == kMajorK || (kModeA == kTma && kModeB == kTma), "gathered tiles are K-major");
+    constexpr bool kGatherA = kModeA != kTma, kGatherB = kModeB != kTma;
     constexpr bool kAnyTma = !kGatherA || !kGatherB;
+    constexpr bool kAnyGather = kGatherA || kGatherB;
+
     extern __shared__ uint8_t smem_raw_[];
     __shared__ __align__(8) uint64_t bars[2 * kRawStages + 2 * kOpStages + 5];
     __shared__ uint32_t tmem_base_slot;
@@ -226,6 +293,8 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     uint64_t *acc_full = op_empty + kOpStages, *acc_empty = acc_full + 2, *drain = acc_empty + 2;
 
     const int m0 = blockIdx.y * kBM, n0 = blockIdx.x * kBN;
+    const int n_valid = min(kBN, prm.N - n0);                              // columns of this tile that exist
+    const int n_act = (n_valid + 15) & ~15;                                // UMMA N (multiple of 16)
     const int slice_begin = blockIdx.z * prm.slices_per_split;
     const int slice_end = min(prm.k_slices, slice_begin + prm.slices_per_split);
     const int n_slices = slice_end - slice_begin;                           // >= 1 by construction
@@ -288,7 +357,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     } else if (warp == 1) {
         // ================= MMA issuer (one thread) =================
         if (lane == 0) {
-            constexpr uint32_t idesc = instr_desc(kMajor);
+            const uint32_t idesc = instr_desc(kMajor, n_act);
             // K-major: rows of 128 B, 8-row groups 1024 B apart (SBO); LBO unused.
             // MN-major: 32-wide column blocks 4096 B apart (LBO); 4-deep k groups 512 B apart (SBO).
             const uint32_t lbo = kMajor == kMajorK ? 16u : 4096u;
@@ -335,29 +404,14 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         // ================= transform warps: square and split into TF32 hi / lo =================
         const int t = (int)threadIdx.x - 64;                               // 0..255
         const int kq = t & 7, row0 = t >> 3;                               // gathered chunks: rows row0 + 32*i, k = 4*kq..4*kq+3
-        constexpr int kRowsPerThread = kBM * 8 / kTransformThreads;        // 4
-
-        // ---- per-thread constants of the gathered tiles
-        int b_base[kRowsPerThread], b_dh[kRowsPerThread], b_dw[kRowsPerThread];
-        bool b_ok[kRowsPerThread], a_ok[kRowsPerThread];
-        int ho[4], wo[4];                    // output position of this thread's four k in the current slice
+        GatherRows<kModeA> rows_a;
+        GatherRows<kModeB> rows_b;
+        rows_a.init(prm, m0 + row0, prm.M);
+        rows_b.init(prm, n0 + row0, prm.N);
+        int ho[4] = {0, 0, 0, 0}, wo[4] = {0, 0, 0, 0};                    // output position of this thread's four k
         int ho_init[4], wo_init[4];
-        int q32 = 0, r32 = 0;
-        int z = 0, pblk = 0;
-        if (kGatherA || kGatherB) {
-            const int khw = prm.Kh * prm.Kw;
-#pragma unroll
-            for (int i = 0; i < kRowsPerThread; ++i) {
-                const int n = n0 + row0 + 32 * i;
-                b_ok[i] = n < prm.N;
-                const int nn = b_ok[i] ? n : 0;
-                const int c = nn / khw, rem = nn - c * khw;
-                const int kh = rem / prm.Kw, kw = rem - kh * prm.Kw;
-                b_dh[i] = kh - prm.ph;
-                b_dw[i] = kw - prm.pw;
-                b_base[i] = (c * prm.H + b_dh[i]) * prm.W + b_dw[i];
-                a_ok[i] = m0 + row0 + 32 * i < prm.M;
-            }
+        int q32 = 0, r32 = 0, z = 0, pblk = 0;
+        if (kAnyGather) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 ho_init[j] = (kq * 4 + j) / prm.Wo;
@@ -374,35 +428,6 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                 wo[j] = p - ho[j] * prm.Wo;
             }
         }
-        float va[kGatherA ? kRowsPerThread : 1][4], vb[kGatherB ? kRowsPerThread : 1][4];
-
-        // loads of the gathered chunks of the slice the (z, pblk, ho, wo) state points at
-        auto gather = [&](float (&ga)[kGatherA ? kRowsPerThread : 1][4], float (&gb)[kGatherB ? kRowsPerThread : 1][4]) {
-            const int pbase = pblk * kBK + kq * 4;
-            if (kGatherB) {
-                const float *xz = prm.x + (size_t)z * prm.C * prm.H * prm.W;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const bool pv = pbase + j < prm.P;
-                    const int hs = ho[j] * prm.sh, ws = wo[j] * prm.sw;
-                    const int poff = hs * prm.W + ws;
-#pragma unroll
-                    for (int i = 0; i < kRowsPerThread; ++i) {
-                        const bool ok = pv && b_ok[i] && (unsigned)(hs + b_dh[i]) < (unsigned)prm.H &&
-                                        (unsigned)(ws + b_dw[i]) < (unsigned)prm.W;
-                        gb[i][j] = ok ? __ldg(xz + (b_base[i] + poff)) : 0.f;
-                    }
-                }
-            }
-            if (kGatherA) {
-#pragma unroll
-                for (int i = 0; i < kRowsPerThread; ++i) {
-                    const float *dr = prm.delta + ((size_t)z * prm.Cout + (m0 + row0 + 32 * i)) * prm.P + pbase;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) ga[i][j] = (a_ok[i] && pbase + j < prm.P) ? __ldg(dr + j) : 0.f;
-                }
-            }
-        };
         auto advance = [&]() {
             if (++pblk == prm.p_slices) {
                 pblk = 0;
@@ -418,22 +443,20 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                 }
             }
         };
-
-        if (kGatherA || kGatherB) gather(va, vb);
-        for (int i = 0; i < n_slices; ++i) {
+        auto gather = [&](float (&ga)[kRowsPerThread][4], float (&gb)[kRowsPerThread][4]) {
+            const int pbase = pblk * kBK + kq * 4;
+            rows_a.load(prm, z, pbase, ho, wo, ga);
+            rows_b.load(prm, z, pbase, ho, wo, gb);
+        };
+        // transform of slice i; gathered elements come in registers, TMA tiles from the raw stage
+        auto process = [&](int i, const float (&ga)[kRowsPerThread][4], const float (&gb)[kRowsPerThread][4]) -> bool {
             const int rs = i % kRawStages, os = i % kOpStages;
-            float wa[kGatherA ? kRowsPerThread : 1][4], wb[kGatherB ? kRowsPerThread : 1][4];
-            if ((kGatherA || kGatherB) && i + 1 < n_slices) {           // next slice's loads fly during this transform
-                advance();
-                gather(wa, wb);
-            }
-            if (kAnyTma && !mbar_wait(smem_u32(&raw_full[rs]), (uint32_t)(i / kRawStages) & 1u, &abort_flag)) break;
-            if (!mbar_wait(smem_u32(&op_empty[os]), ((uint32_t)(i / kOpStages) & 1u) ^ 1u, &abort_flag)) break;
+            if (kAnyTma && !mbar_wait(smem_u32(&raw_full[rs]), (uint32_t)(i / kRawStages) & 1u, &abort_flag)) return false;
+            if (!mbar_wait(smem_u32(&op_empty[os]), ((uint32_t)(i / kOpStages) & 1u) ^ 1u, &abort_flag)) return false;
             uint8_t *raw = smem_gen + rs * kRawStageBytes;
             uint8_t *hi = smem_gen + kRawStages * kRawStageBytes + os * kOpStageBytes;
             uint8_t *lo = hi + kRawStageBytes;
-            // tiles that came by TMA: elementwise over their 16-byte chunks (layout is inherited)
-            {
+            if (kAnyTma) {      // tiles that came by TMA: elementwise over their 16-byte chunks (layout is inherited)
                 const uint32_t c_begin = kGatherA ? kRawBytesA / 16 : 0;
                 const uint32_t c_end = kGatherB ? kRawBytesA / 16 : kRawStageBytes / 16;
 #pragma unroll 4
@@ -445,13 +468,13 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             if (kGatherA) {
 #pragma unroll
                 for (int r = 0; r < kRowsPerThread; ++r)
-                    split_store(hi, lo, chunk_offset(row0 + 32 * r, kq), va[r][0], va[r][1], va[r][2], va[r][3]);
+                    split_store(hi, lo, chunk_offset(row0 + 32 * r, kq), ga[r][0], ga[r][1], ga[r][2], ga[r][3]);
             }
             if (kGatherB) {
 #pragma unroll
                 for (int r = 0; r < kRowsPerThread; ++r)
-                    split_store(hi + kRawBytesA, lo + kRawBytesA, chunk_offset(row0 + 32 * r, kq), vb[r][0], vb[r][1],
-                                vb[r][2], vb[r][3]);
+                    split_store(hi + kRawBytesA, lo + kRawBytesA, chunk_offset(row0 + 32 * r, kq), gb[r][0], gb[r][1],
+                                gb[r][2], gb[r][3]);
             }
             fence_async_smem();                                   // generic-proxy writes -> tensor core reads
             __syncwarp();
@@ -459,17 +482,18 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                 mbar_arrive(smem_u32(&op_full[os]));
                 if (kAnyTma) mbar_arrive(smem_u32(&raw_empty[rs]));
             }
-            if (kGatherA) {
-#pragma unroll
-                for (int r = 0; r < kRowsPerThread; ++r)
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) va[r][j] = wa[r][j];
-            }
-            if (kGatherB) {
-#pragma unroll
-                for (int r = 0; r < kRowsPerThread; ++r)
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) vb[r][j] = wb[r][j];
+            return true;
+        };
+
+        // two register sets in turn: the loads of slice i+1 are in flight while slice i is transformed
+        float a0[kRowsPerThread][4], b0[kRowsPerThread][4], a1[kRowsPerThread][4], b1[kRowsPerThread][4];
+        if (kAnyGather) gather(a0, b0);
+        for (int i = 0; i < n_slices; i += 2) {
+            if (kAnyGather && i + 1 < n_slices) { advance(); gather(a1, b1); }
+            if (!process(i, a0, b0)) break;
+            if (i + 1 < n_slices) {
+                if (kAnyGather && i + 2 < n_slices) { advance(); gather(a0, b0); }
+                if (!process(i + 1, a1, b1)) break;
             }
         }
     } else {
@@ -487,33 +511,58 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             const uint32_t taddr = tmem_base + ((q * 32u) << 16) + (uint32_t)b * kBN;
 #pragma unroll
             for (int j0 = 0; j0 < kBN; j0 += 32) {
-                uint32_t r[32];
-                tc_ld_32x32(taddr + j0, r);
-                tc_wait_ld();
+                if (j0 < n_act) {
+                    uint32_t r[32];
+                    tc_ld_32x32(taddr + j0, r);
+                    tc_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) acc[j0 + j] = __fadd_rn(acc[j0 + j], __uint_as_float(r[j]));
+                    for (int j = 0; j < 32; ++j) acc[j0 + j] = __fadd_rn(acc[j0 + j], __uint_as_float(r[j]));
+                }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&acc_empty[b]));
         }
         if (ok) {
-            const int m = m0 + (int)(q * 32u + lane);
-            if (m < prm.M) {
-                const bool direct = gridDim.z == 1;
-                float *row = direct ? prm.S + (size_t)m * prm.N : prm.partial + ((size_t)blockIdx.z * prm.M + m) * prm.N;
-                const int n_valid = min(kBN, prm.N - n0);
-                if (direct) {
+            const int r_local = (int)(q * 32u + lane);
+            const int m = m0 + r_local;
+            if (gridDim.z > 1) {
+                // split-K scratch, column-major inside the tile: consecutive lanes -> consecutive addresses
+                const size_t tile = (size_t)blockIdx.z * (gridDim.x * gridDim.y) + (size_t)blockIdx.y * gridDim.x + blockIdx.x;
+                float *dst = prm.partial + tile * (kBM * kBN) + r_local;
+#pragma unroll
+                for (int j = 0; j < kBN; ++j)
+                    if (j < n_valid) dst[j * kBM] = acc[j];
+            } else if (prm.ld_m == 1) {
+                // result is contiguous along m: lanes write neighbouring addresses directly
+                if (m < prm.M) {
 #pragma unroll
                     for (int j = 0; j < kBN; ++j)
                         if (j < n_valid) {
+                            float *dst = prm.S + (size_t)m + (size_t)(n0 + j) * prm.ld_n;
                             const float res = __fmul_rn(prm.scale, acc[j]);
-                            row[n0 + j] = prm.accumulate ? __fadd_rn(row[n0 + j], res) : res;
+                            *dst = prm.accumulate ? __fadd_rn(*dst, res) : res;
                         }
-                } else {
+                }
+            } else {
+                // result is contiguous along n: transpose this warp's 32 x 128 block through shared memory
+                // (the operand stages are idle: the last accumulator was complete before we got here)
+                float *tile = reinterpret_cast<float *>(smem_gen + kRawStages * kRawStageBytes) + q * (32 * (kBN + 1));
 #pragma unroll
-                    for (int j = 0; j < kBN; ++j)
-                        if (j < n_valid) row[n0 + j] = acc[j];
+                for (int j = 0; j < kBN; ++j) tile[lane * (kBN + 1) + j] = __fmul_rn(prm.scale, acc[j]);
+                __syncwarp();
+                for (int r = 0; r < 32; ++r) {
+                    const int mr = m0 + (int)(q * 32u) + r;
+                    if (mr >= prm.M) break;
+                    float *dst = prm.S + (size_t)mr * prm.ld_m + n0;
+#pragma unroll
+                    for (int cblk = 0; cblk < kBN / 32; ++cblk) {
+                        const int j = cblk * 32 + (int)lane;
+                        if (j < n_valid) {
+                            const float res = tile[r * (kBN + 1) + j];
+                            dst[j] = prm.accumulate ? __fadd_rn(dst[j], res) : res;
+                        }
+                    }
                 }
             }
         }
@@ -526,20 +575,53 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
-    if (threadIdx.x == 0 && abort_flag) atomicExch(prm.error_flag, 1u);
+    if (threadIdx.x == 0 && abort_flag) atomicOr(prm.status, VGC_DEV_TIMEOUT);
 }
 
-// combine split-K partial tiles in a fixed order
+// Combine split-K partial tiles in a fixed order.  One block per 32 x 32 patch of a tile: partials are
+// read along rows (their unit stride), the result is written along whichever of m / n has unit stride.
 __global__ void __launch_bounds__(256)
-sqgrad_tc_combine(const float *__restrict__ partial, int splits, size_t mn, float scale, int accumulate,
-                  float *__restrict__ S)
+sqgrad_tc_combine(const float *__restrict__ partial, int splits, int tiles_x, int tiles_y, int M, int N, float scale,
+                  int accumulate, float *__restrict__ S, long long ld_m, long long ld_n)
 {
-    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= mn) return;
-    float sum = 0.f;
-    for (int z = 0; z < splits; ++z) sum = __fadd_rn(sum, partial[(size_t)z * mn + i]);
-    const float res = __fmul_rn(scale, sum);
-    S[i] = accumulate ? __fadd_rn(S[i], res) : res;
+    __shared__ float patch[32][33];
+    const int tile = blockIdx.x >> 4, sub = blockIdx.x & 15;
+    const int tx = tile % tiles_x, ty = tile / tiles_x;
+    const int r0 = (sub & 3) * 32, j0 = (sub >> 2) * 32;                  // patch origin inside the tile
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;              // 8 warps x 4 columns each
+    const size_t tiles = (size_t)tiles_x * tiles_y;
+    if (ty * kBM + r0 >= M || tx * kBN + j0 >= N) return;
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+        const int j = j0 + w * 4 + jj;
+        const float *src = partial + ((size_t)tile * kBN + j) * kBM + r0 + lane;
+        float sum = 0.f;
+        if (tx * kBN + j < N)
+            for (int z = 0; z < splits; ++z) sum = __fadd_rn(sum, src[(size_t)z * tiles * (kBM * kBN)]);
+        patch[w * 4 + jj][lane] = __fmul_rn(scale, sum);                   // patch[column][row]
+    }
+    __syncthreads();
+    if (ld_m == 1) {
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+            const int m = ty * kBM + r0 + lane, n = tx * kBN + j0 + w * 4 + jj;
+            if (m < M && n < N) {
+                float *dst = S + (size_t)m + (size_t)n * ld_n;
+                const float res = patch[w * 4 + jj][lane];
+                *dst = accumulate ? __fadd_rn(*dst, res) : res;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int rr = 0; rr < 4; ++rr) {
+            const int m = ty * kBM + r0 + w * 4 + rr, n = tx * kBN + j0 + lane;
+            if (m < M && n < N) {
+                float *dst = S + (size_t)m * ld_m + n;
+                const float res = patch[lane][w * 4 + rr];
+                *dst = accumulate ? __fadd_rn(*dst, res) : res;
+            }
+        }
+    }
 }
 
 // ---- host side --------------------------------------------------------------------------------
@@ -576,23 +658,25 @@ static int default_chunk()
     static int chunk = 0;
     if (!chunk) {
         const char *e = getenv("VGC_TC_CHUNK");
-        chunk = e ? atoi(e) : 4;
+        chunk = e ? atoi(e) : 8;
         if (chunk < 1) chunk = 1;
     }
     return chunk;
 }
 
 struct Plan {
-    int splits, slices_per_split, k_slices;
+    int splits, slices_per_split, k_slices, tiles_x, tiles_y;
 };
 
 static Plan make_plan(int M, int N, int k_slices)
 {
-    const long tiles = (long)((M + kBM - 1) / kBM) * ((N + kBN - 1) / kBN);
-    long want = (148 + tiles - 1) / tiles;                 // fill the SMs once
+    Plan p;
+    p.tiles_x = (N + kBN - 1) / kBN;
+    p.tiles_y = (M + kBM - 1) / kBM;
+    const long tiles = (long)p.tiles_x * p.tiles_y;
+    long want = 148 / tiles;                               // one block per SM: fill the SMs at most once
     if (want > k_slices) want = k_slices;
     if (want < 1) want = 1;
-    Plan p;
     p.k_slices = k_slices;
     p.slices_per_split = (int)((k_slices + want - 1) / want);
     p.splits = (k_slices + p.slices_per_split - 1) / p.slices_per_split;
@@ -616,44 +700,38 @@ bool tc_conv_supported(int B, int C, int H, int W, int Cout, int Kh, int Kw, int
            (long)B * ((P + kBK - 1) / kBK) < (1L << 30);
 }
 
-size_t tc_workspace_bytes(int M, int N, int k_slices)
+static size_t tc_workspace_bytes(int M, int N, int k_slices)
 {
     const Plan p = make_plan(M, N, k_slices);
-    return 256 + (p.splits > 1 ? (size_t)p.splits * M * N * sizeof(float) : 0);
+    return 256 + (p.splits > 1 ? (size_t)p.splits * p.tiles_x * p.tiles_y * kBM * kBN * sizeof(float) : 0);
 }
 
-enum Variant { kDense, kConvTmaTma, kConvTmaGather, kConvGatherGather };
+typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const Params);
 
-static vgc_status tc_launch(Variant variant, const CUtensorMap &ma, const CUtensorMap &mb, Params prm, int M, int N,
+static vgc_status tc_launch(KernelFn kernel, const CUtensorMap &ma, const CUtensorMap &mb, Params prm, int M, int N,
                             int k_slices, void *ws, size_t ws_bytes, cudaStream_t st)
 {
     const Plan plan = make_plan(M, N, k_slices);
     if (ws_bytes < tc_workspace_bytes(M, N, k_slices)) return VGC_ERR_WORKSPACE;
-    static bool attr_set = false;
-    if (!attr_set) {
-        VGC_CUDA_OK(cudaFuncSetAttribute(sqgrad_tc<kMajorMN, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-        VGC_CUDA_OK(cudaFuncSetAttribute(sqgrad_tc<kMajorK, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-        VGC_CUDA_OK(cudaFuncSetAttribute(sqgrad_tc<kMajorK, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-        VGC_CUDA_OK(cudaFuncSetAttribute(sqgrad_tc<kMajorK, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-        attr_set = true;
+    static KernelFn configured[16];
+    static int n_configured = 0;
+    bool seen = false;
+    for (int i = 0; i < n_configured; ++i) seen = seen || configured[i] == kernel;
+    if (!seen) {
+        VGC_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        if (n_configured < 16) configured[n_configured++] = kernel;
     }
     prm.M = M; prm.N = N; prm.k_slices = k_slices; prm.slices_per_split = plan.slices_per_split;
     prm.chunk = default_chunk();
-    prm.error_flag = static_cast<uint32_t *>(ws);
+    prm.status = static_cast<uint32_t *>(ws);
     prm.partial = reinterpret_cast<float *>(static_cast<char *>(ws) + 256);
-    VGC_CUDA_OK(cudaMemsetAsync(ws, 0, 4, st));
-    dim3 grid((N + kBN - 1) / kBN, (M + kBM - 1) / kBM, plan.splits);
-    switch (variant) {
-        case kDense: sqgrad_tc<kMajorMN, false, false><<<grid, kThreadsTc, kSmemBytes, st>>>(ma, mb, prm); break;
-        case kConvTmaTma: sqgrad_tc<kMajorK, false, false><<<grid, kThreadsTc, kSmemBytes, st>>>(ma, mb, prm); break;
-        case kConvTmaGather: sqgrad_tc<kMajorK, false, true><<<grid, kThreadsTc, kSmemBytes, st>>>(ma, mb, prm); break;
-        case kConvGatherGather: sqgrad_tc<kMajorK, true, true><<<grid, kThreadsTc, kSmemBytes, st>>>(ma, mb, prm); break;
-    }
+    dim3 grid(plan.tiles_x, plan.tiles_y, plan.splits);
+    kernel<<<grid, kThreadsTc, kSmemBytes, st>>>(ma, mb, prm);
     count_launch();
     if (plan.splits > 1) {
-        const size_t mn = (size_t)M * N;
-        sqgrad_tc_combine<<<(unsigned)((mn + 255) / 256), 256, 0, st>>>(prm.partial, plan.splits, mn, prm.scale,
-                                                                         prm.accumulate, prm.S);
+        sqgrad_tc_combine<<<(unsigned)(plan.tiles_x * plan.tiles_y * 16), 256, 0, st>>>(
+            prm.partial, plan.splits, plan.tiles_x, plan.tiles_y, M, N, prm.scale, prm.accumulate, prm.S, prm.ld_m,
+            prm.ld_n);
         count_launch();
     }
     return cudaGetLastError() == cudaSuccess ? VGC_OK : VGC_ERR_CUDA;
@@ -673,45 +751,70 @@ vgc_status tc_sqgrad_linear(const float *x, const float *delta, int B, int in, i
         return VGC_ERR_CUDA;
     Params prm = {};
     prm.p_slices = 1; prm.tx_bytes = kRawStageBytes; prm.scale = scale; prm.accumulate = accumulate; prm.S = S;
-    return tc_launch(kDense, ma, mb, prm, out, in, (B + kBK - 1) / kBK, ws, ws_bytes, st);
+    prm.ld_m = in; prm.ld_n = 1;
+    return tc_launch(sqgrad_tc<kMajorMN, kTma, kTma>, ma, mb, prm, out, in, (B + kBK - 1) / kBK, ws, ws_bytes, st);
 }
+
+// Cout <= 64: the im2col rows take the 128-row A tile and the errors the narrow B tile
+static bool conv_swapped(int Cout, int n_im2col) { return Cout <= 64 && n_im2col > Cout; }
 
 size_t tc_conv_workspace_bytes(int B, int C, int Kh, int Kw, int P, int Cout)
 {
-    return tc_workspace_bytes(Cout, C * Kh * Kw, B * ((P + kBK - 1) / kBK));
+    const int n_im2col = C * Kh * Kw, k_slices = B * ((P + kBK - 1) / kBK);
+    return conv_swapped(Cout, n_im2col) ? tc_workspace_bytes(n_im2col, Cout, k_slices)
+                                        : tc_workspace_bytes(Cout, n_im2col, k_slices);
 }
 
 vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int H, int W, int Cout, int Kh, int Kw,
                           int sh, int sw, int ph, int pw, int Ho, int Wo, float scale, int accumulate, float *S,
                           void *ws, size_t ws_bytes, cudaStream_t st)
 {
-    const int P = Ho * Wo, N = C * Kh * Kw;
+    const int P = Ho * Wo, n_im2col = C * Kh * Kw;
     const int p_slices = (P + kBK - 1) / kBK;
-    const bool a_tma = P >= kBK && P % 4 == 0;
-    const bool b_tma = a_tma && Kh == 1 && Kw == 1 && sh == 1 && sw == 1 && ph == 0 && pw == 0;
-    CUtensorMap ma = {}, mb = {};
+    static const int force_gather = getenv("VGC_TC_GATHER") ? atoi(getenv("VGC_TC_GATHER")) : 0;   // experiments
+    const bool err_tma = P >= kBK && P % 4 == 0 && !(force_gather & 1);
+    const bool in_tma = P >= kBK && P % 4 == 0 && !(force_gather & 2) && Kh == 1 && Kw == 1 && sh == 1 && sw == 1 &&
+                        ph == 0 && pw == 0;
+    const bool swapped = conv_swapped(Cout, n_im2col);
+    const int rows_err = swapped ? kBN : kBM, rows_in = swapped ? kBM : kBN;     // tile heights
+    CUtensorMap m_err = {}, m_in = {};
     uint32_t tx = 0;
-    if (a_tma) {
-        const cuuint32_t box_a[3] = {(cuuint32_t)kBK, (cuuint32_t)(Cout < kBM ? Cout : kBM), 1};
-        const cuuint64_t dims_a[3] = {(cuuint64_t)P, (cuuint64_t)Cout, (cuuint64_t)B};
-        const cuuint64_t str_a[2] = {(cuuint64_t)P * 4, (cuuint64_t)Cout * P * 4};
-        if (!make_map(&ma, delta, 3, dims_a, str_a, box_a, CU_TENSOR_MAP_SWIZZLE_128B)) return VGC_ERR_CUDA;
-        tx += box_a[1] * kBK * 4;
+    if (err_tma) {
+        const cuuint32_t box[3] = {(cuuint32_t)kBK, (cuuint32_t)(Cout < rows_err ? Cout : rows_err), 1};
+        const cuuint64_t dims[3] = {(cuuint64_t)P, (cuuint64_t)Cout, (cuuint64_t)B};
+        const cuuint64_t str[2] = {(cuuint64_t)P * 4, (cuuint64_t)Cout * P * 4};
+        if (!make_map(&m_err, delta, 3, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B)) return VGC_ERR_CUDA;
+        tx += box[1] * kBK * 4;
     }
-    if (b_tma) {
-        const cuuint32_t box_b[3] = {(cuuint32_t)kBK, (cuuint32_t)(C < kBN ? C : kBN), 1};
-        const cuuint64_t dims_b[3] = {(cuuint64_t)P, (cuuint64_t)C, (cuuint64_t)B};
-        const cuuint64_t str_b[2] = {(cuuint64_t)P * 4, (cuuint64_t)C * P * 4};
-        if (!make_map(&mb, x, 3, dims_b, str_b, box_b, CU_TENSOR_MAP_SWIZZLE_128B)) return VGC_ERR_CUDA;
-        tx += box_b[1] * kBK * 4;
+    if (in_tma) {
+        const cuuint32_t box[3] = {(cuuint32_t)kBK, (cuuint32_t)(C < rows_in ? C : rows_in), 1};
+        const cuuint64_t dims[3] = {(cuuint64_t)P, (cuuint64_t)C, (cuuint64_t)B};
+        const cuuint64_t str[2] = {(cuuint64_t)P * 4, (cuuint64_t)C * P * 4};
+        if (!make_map(&m_in, x, 3, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B)) return VGC_ERR_CUDA;
+        tx += box[1] * kBK * 4;
     }
     Params prm = {};
     prm.p_slices = p_slices; prm.tx_bytes = tx; prm.scale = scale; prm.accumulate = accumulate; prm.S = S;
     prm.x = x; prm.delta = delta;
     prm.C = C; prm.H = H; prm.W = W; prm.Cout = Cout; prm.Kh = Kh; prm.Kw = Kw; prm.sh = sh; prm.sw = sw;
     prm.ph = ph; prm.pw = pw; prm.Wo = Wo; prm.P = P;
-    const Variant v = b_tma ? kConvTmaTma : (a_tma ? kConvTmaGather : kConvGatherGather);
-    return tc_launch(v, ma, mb, prm, Cout, N, B * p_slices, ws, ws_bytes, st);
+    const int k_slices = B * p_slices;
+    const int e = err_tma ? kTma : kGatherErr, i = in_tma ? kTma : kGatherIm2col;
+    KernelFn fn = nullptr;
+    if (!swapped) {     // S[o][idx]: m = o, n = idx
+        prm.ld_m = n_im2col; prm.ld_n = 1;
+        if (e == kTma && i == kTma) fn = sqgrad_tc<kMajorK, kTma, kTma>;
+        else if (e == kTma) fn = sqgrad_tc<kMajorK, kTma, kGatherIm2col>;
+        else if (i == kTma) fn = sqgrad_tc<kMajorK, kGatherErr, kTma>;
+        else fn = sqgrad_tc<kMajorK, kGatherErr, kGatherIm2col>;
+        return tc_launch(fn, m_err, m_in, prm, Cout, n_im2col, k_slices, ws, ws_bytes, st);
+    }
+    prm.ld_m = 1; prm.ld_n = n_im2col;   // m = idx, n = o
+    if (e == kTma && i == kTma) fn = sqgrad_tc<kMajorK, kTma, kTma>;
+    else if (i == kTma) fn = sqgrad_tc<kMajorK, kTma, kGatherErr>;
+    else if (e == kTma) fn = sqgrad_tc<kMajorK, kGatherIm2col, kTma>;
+    else fn = sqgrad_tc<kMajorK, kGatherIm2col, kGatherErr>;
+    return tc_launch(fn, m_in, m_err, prm, n_im2col, Cout, k_slices, ws, ws_bytes, st);
 }
 
 }  // namespace vgc

@@ -11,7 +11,7 @@ RTOL = 1e-5
 
 
 def _ws(nbytes):
-    return torch.empty(max(nbytes, 16), dtype=torch.uint8, device="cuda")
+    return torch.zeros(max(nbytes, 256), dtype=torch.uint8, device="cuda")      # status word starts at 0
 
 
 def _status(ws):
