@@ -596,8 +596,18 @@ sqgrad_tc_combine(const float *__restrict__ partial, int splits, int tiles_x, in
         const int j = j0 + w * 4 + jj;
         const float *src = partial + ((size_t)tile * kBN + j) * kBM + r0 + lane;
         float sum = 0.f;
-        if (tx * kBN + j < N)
-            for (int z = 0; z < splits; ++z) sum = __fadd_rn(sum, src[(size_t)z * tiles * (kBM * kBN)]);
+        if (tx * kBN + j < N) {
+            const size_t stride = tiles * (size_t)(kBM * kBN);
+            int z = 0;
+            for (; z + 8 <= splits; z += 8) {               // eight loads in flight, summed in split order
+                float v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = __ldcs(src + (size_t)(z + u) * stride);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) sum = __fadd_rn(sum, v[u]);
+            }
+            for (; z < splits; ++z) sum = __fadd_rn(sum, __ldcs(src + (size_t)z * stride));
+        }
         patch[w * 4 + jj][lane] = __fmul_rn(scale, sum);                   // patch[column][row]
     }
     __syncthreads();
