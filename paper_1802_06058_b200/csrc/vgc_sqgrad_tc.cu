@@ -3,11 +3,12 @@
 //   D[m][n] = sum_k A(k,m)^2 * B(k,n)^2          (the contraction behind Eq. 2 / Algorithm 1's
 //                                                  "v_i +=" line; N_params*|B| multiply-adds, Sec. 5)
 // Operands stay fp32 in global memory.  Per 32-deep k slice a thread block
-//   1. TMA-loads the raw fp32 tiles of A (128 rows) and B (kBN rows) into shared memory
+//   1. TMA-loads the raw fp32 tiles of A (128 rows) and B (kBN rows) into a pipeline stage
 //      (128-byte swizzle, out-of-range parts filled with zeros),
 //   2. squares every element in fp32 and splits the square into two TF32 numbers hi + lo
-//      (hi = rna(x*x), lo = rna(x*x - hi)); the transform is elementwise, so the hi and lo tiles
-//      inherit the swizzled layout the tensor core wants,
+//      (hi = x*x rounded to 11 significant bits, lo = x*x - hi likewise); the transform is elementwise
+//      and in place (hi overwrites the raw tile, lo goes beside it), so both inherit the swizzled
+//      layout the tensor core wants,
 //   3. issues three tcgen05.mma per 8-deep step -- hi*hi, hi*lo, lo*hi -- into a TMEM
 //      accumulator (the dropped lo*lo term is 2^-22 relative).
 // The tensor core's fp32 accumulation is not trusted over long reductions: every kChunk k slices
@@ -42,17 +43,16 @@ namespace tc {
 constexpr int kBM = 128;            // output rows per block (UMMA M)
 constexpr int kBN = 128;            // output columns per block (UMMA N)
 constexpr int kBK = 32;             // k per pipeline slice (= 128 bytes of fp32)
-constexpr int kRawStages = 3;
-constexpr int kOpStages = 2;
+constexpr int kStages = 3;          // each stage: raw fp32 tiles, overwritten in place by hi, plus the lo tiles
 constexpr int kThreadsTc = 448;
 constexpr int kTransformWarps = 8;
 constexpr int kTransformThreads = 32 * kTransformWarps;
 constexpr int kEpilogueWarps = 4;
 constexpr uint32_t kRawBytesA = kBM * kBK * 4;                      // 16 KB
 constexpr uint32_t kRawBytesB = kBN * kBK * 4;                      // 16 KB
-constexpr uint32_t kRawStageBytes = kRawBytesA + kRawBytesB;        // 32 KB
-constexpr uint32_t kOpStageBytes = 2 * kRawStageBytes;              // hi block then lo block
-constexpr uint32_t kSmemBytes = kRawStages * kRawStageBytes + kOpStages * kOpStageBytes + 1024 /*align*/ + 256;
+constexpr uint32_t kRawStageBytes = kRawBytesA + kRawBytesB;        // 32 KB: [A raw/hi][B raw/hi]
+constexpr uint32_t kStageBytes = 2 * kRawStageBytes;                // 64 KB: ... then [A lo][B lo]
+constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256;
 constexpr uint32_t kTmemCols = 2 * kBN;                             // two accumulator buffers
 constexpr uint32_t kWaitLimit = 1u << 22;                           // polls before a wait gives up
 
@@ -75,6 +75,7 @@ struct Params {
     long long ld_m, ld_n;
     float *partial;          // split-K scratch [split][tile][column][row], used when gridDim.z > 1
     uint32_t *status;        // device word; VGC_DEV_TIMEOUT is OR-ed in if a wait expired
+    int debug;               // experiments: 1 skip MMAs, 2 skip transform math, 4 skip gathers
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -164,12 +165,9 @@ __device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-__device__ __forceinline__ uint32_t to_tf32(float x)
-{
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return r;
-}
+// fp32 -> tf32 (10 explicit mantissa bits), round to nearest with ties away from zero, as the integer
+// form of cvt.rna.tf32.f32: add half a tf32 ulp to the bit pattern and clear the 13 low bits.
+__device__ __forceinline__ uint32_t to_tf32(float x) { return (__float_as_uint(x) + 0x1000u) & 0xFFFFE000u; }
 
 // Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte offsets
 // (all >> 4), descriptor version 1, swizzle mode (2: 128-byte swizzle of 16-byte units, the K-major
@@ -278,19 +276,17 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     constexpr bool kAnyGather = kGatherA || kGatherB;
 
     extern __shared__ uint8_t smem_raw_[];
-    __shared__ __align__(8) uint64_t bars[2 * kRawStages + 2 * kOpStages + 5];
+    __shared__ __align__(8) uint64_t bars[3 * kStages + 5];
     __shared__ uint32_t tmem_base_slot;
     __shared__ volatile uint32_t abort_flag;
 
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (smem_u32(smem_raw_) + 1023u) & ~1023u;     // 1024-byte aligned tiles
     uint8_t *smem_gen = smem_raw_ + (smem_base - smem_u32(smem_raw_));
-    const uint32_t raw_base = smem_base;
-    const uint32_t op_base = smem_base + kRawStages * kRawStageBytes;
 
-    uint64_t *raw_full = bars, *raw_empty = bars + kRawStages;
-    uint64_t *op_full = bars + 2 * kRawStages, *op_empty = op_full + kOpStages;
-    uint64_t *acc_full = op_empty + kOpStages, *acc_empty = acc_full + 2, *drain = acc_empty + 2;
+    // per stage: raw_full (TMA landed) -> op_full (hi/lo written) -> empty (MMAs that read it retired)
+    uint64_t *raw_full = bars, *op_full = bars + kStages, *empty = bars + 2 * kStages;
+    uint64_t *acc_full = bars + 3 * kStages, *acc_empty = acc_full + 2, *drain = acc_empty + 2;
 
     const int m0 = blockIdx.y * kBM, n0 = blockIdx.x * kBN;
     const int n_valid = min(kBN, prm.N - n0);                              // columns of this tile that exist
@@ -302,8 +298,11 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        for (int i = 0; i < kRawStages; ++i) { mbar_init(smem_u32(&raw_full[i]), 1); mbar_init(smem_u32(&raw_empty[i]), kTransformWarps); }
-        for (int i = 0; i < kOpStages; ++i) { mbar_init(smem_u32(&op_full[i]), kTransformWarps); mbar_init(smem_u32(&op_empty[i]), 1); }
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(smem_u32(&raw_full[i]), 1);
+            mbar_init(smem_u32(&op_full[i]), kTransformWarps);
+            mbar_init(smem_u32(&empty[i]), 1);
+        }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&acc_full[i]), 1); mbar_init(smem_u32(&acc_empty[i]), kEpilogueWarps); }
         mbar_init(smem_u32(drain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -324,11 +323,11 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         if (lane == 0 && kAnyTma) {
             int issued = 0;
             for (int i = 0; i < n_slices; ++i) {
-                const int st = i % kRawStages;
-                const uint32_t ph = (uint32_t)(i / kRawStages) & 1u;
-                if (!mbar_wait(smem_u32(&raw_empty[st]), ph ^ 1u, &abort_flag)) break;
+                const int st = i % kStages;
+                const uint32_t ph = (uint32_t)(i / kStages) & 1u;
+                if (!mbar_wait(smem_u32(&empty[st]), ph ^ 1u, &abort_flag)) break;
                 const uint32_t full = smem_u32(&raw_full[st]);
-                const uint32_t dst_a = raw_base + st * kRawStageBytes, dst_b = dst_a + kRawBytesA;
+                const uint32_t dst_a = smem_base + st * kStageBytes, dst_b = dst_a + kRawBytesA;
                 mbar_expect_tx(full, prm.tx_bytes);
                 const int slice = slice_begin + i;
                 if (kMajor == kMajorK) {
@@ -346,10 +345,10 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             }
             // on an abort: loads already issued must land before the block may exit
             if (abort_flag) {
-                const int first = issued > kRawStages ? issued - kRawStages : 0;
+                const int first = issued > kStages ? issued - kStages : 0;
                 for (int i = first; i < issued; ++i) {
-                    const uint32_t bar = smem_u32(&raw_full[i % kRawStages]);
-                    const uint32_t ph = (uint32_t)(i / kRawStages) & 1u;
+                    const uint32_t bar = smem_u32(&raw_full[i % kStages]);
+                    const uint32_t ph = (uint32_t)(i / kStages) & 1u;
                     for (uint32_t t = 0; t < kWaitLimit && !mbar_try(bar, ph); ++t) {}
                 }
             }
@@ -374,14 +373,15 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                 const uint32_t d_tmem = tmem_base + (uint32_t)b * kBN;
                 const int chunk_end = min(n_slices, (c + 1) * prm.chunk);
                 for (bool first = true; i < chunk_end; ++i) {
-                    const int st = i % kOpStages;
-                    ok = mbar_wait(smem_u32(&op_full[st]), (uint32_t)(i / kOpStages) & 1u, &abort_flag);
+                    const int st = i % kStages;
+                    ok = mbar_wait(smem_u32(&op_full[st]), (uint32_t)(i / kStages) & 1u, &abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t hi_a = op_base + st * kOpStageBytes, hi_b = hi_a + kRawBytesA;
+                    const uint32_t hi_a = smem_base + st * kStageBytes, hi_b = hi_a + kRawBytesA;
                     const uint32_t lo_a = hi_a + kRawStageBytes, lo_b = lo_a + kRawBytesA;
 #pragma unroll
                     for (int kk = 0; kk < kBK / 8; ++kk) {
+                        if (prm.debug & 1) break;
                         const uint64_t da_hi = smem_desc(hi_a + kk * k_step, lbo, sbo, layout);
                         const uint64_t db_hi = smem_desc(hi_b + kk * k_step, lbo, sbo, layout);
                         const uint64_t da_lo = smem_desc(lo_a + kk * k_step, lbo, sbo, layout);
@@ -391,7 +391,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                         tc_mma_tf32(d_tmem, da_lo, db_hi, idesc, 1u);
                         first = false;
                     }
-                    tc_commit(smem_u32(&op_empty[st]));           // operand slot free once these MMAs retire
+                    tc_commit(smem_u32(&empty[st]));              // stage free once these MMAs retire
                 }
                 if (ok) tc_commit(smem_u32(&acc_full[b]));
             }
@@ -445,25 +445,37 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         };
         auto gather = [&](float (&ga)[kRowsPerThread][4], float (&gb)[kRowsPerThread][4]) {
             const int pbase = pblk * kBK + kq * 4;
+            if (prm.debug & 4) return;
             rows_a.load(prm, z, pbase, ho, wo, ga);
             rows_b.load(prm, z, pbase, ho, wo, gb);
         };
         // transform of slice i; gathered elements come in registers, TMA tiles from the raw stage
         auto process = [&](int i, const float (&ga)[kRowsPerThread][4], const float (&gb)[kRowsPerThread][4]) -> bool {
-            const int rs = i % kRawStages, os = i % kOpStages;
-            if (kAnyTma && !mbar_wait(smem_u32(&raw_full[rs]), (uint32_t)(i / kRawStages) & 1u, &abort_flag)) return false;
-            if (!mbar_wait(smem_u32(&op_empty[os]), ((uint32_t)(i / kOpStages) & 1u) ^ 1u, &abort_flag)) return false;
-            uint8_t *raw = smem_gen + rs * kRawStageBytes;
-            uint8_t *hi = smem_gen + kRawStages * kRawStageBytes + os * kOpStageBytes;
+            const int st = i % kStages;
+            const uint32_t ph = (uint32_t)(i / kStages) & 1u;
+            // a stage is ours once its TMA tiles landed (the producer waited for it to be empty), or, with
+            // nothing coming by TMA, once the MMAs that last read it retired
+            if (kAnyTma ? !mbar_wait(smem_u32(&raw_full[st]), ph, &abort_flag)
+                        : !mbar_wait(smem_u32(&empty[st]), ph ^ 1u, &abort_flag))
+                return false;
+            uint8_t *hi = smem_gen + st * kStageBytes;           // raw tiles live here and become the hi tiles
             uint8_t *lo = hi + kRawStageBytes;
-            if (kAnyTma) {      // tiles that came by TMA: elementwise over their 16-byte chunks (layout is inherited)
-                const uint32_t c_begin = kGatherA ? kRawBytesA / 16 : 0;
-                const uint32_t c_end = kGatherB ? kRawBytesA / 16 : kRawStageBytes / 16;
-#pragma unroll 4
-                for (uint32_t c = c_begin + (uint32_t)t; c < c_end; c += kTransformThreads) {
-                    const float4 v = *reinterpret_cast<const float4 *>(raw + 16 * c);
-                    split_store(hi, lo, 16 * c, v.x, v.y, v.z, v.w);
-                }
+            if (prm.debug & 2) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&op_full[st]));
+                return true;
+            }
+            if (kAnyTma) {      // tiles that came by TMA: elementwise, in place, over their 16-byte chunks
+                constexpr uint32_t c_begin = kGatherA ? kRawBytesA / 16 : 0;
+                constexpr uint32_t c_end = kGatherB ? kRawBytesA / 16 : kRawStageBytes / 16;
+                constexpr int kPerThread = c_end > c_begin ? (c_end - c_begin) / kTransformThreads : 1;
+                float4 v[kPerThread];
+#pragma unroll
+                for (int u = 0; u < kPerThread; ++u)
+                    v[u] = *reinterpret_cast<const float4 *>(hi + 16 * (c_begin + (uint32_t)t + u * kTransformThreads));
+#pragma unroll
+                for (int u = 0; u < kPerThread; ++u)
+                    split_store(hi, lo, 16 * (c_begin + (uint32_t)t + u * kTransformThreads), v[u].x, v[u].y, v[u].z, v[u].w);
             }
             if (kGatherA) {
 #pragma unroll
@@ -478,10 +490,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             }
             fence_async_smem();                                   // generic-proxy writes -> tensor core reads
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(smem_u32(&op_full[os]));
-                if (kAnyTma) mbar_arrive(smem_u32(&raw_empty[rs]));
-            }
+            if (lane == 0) mbar_arrive(smem_u32(&op_full[st]));
             return true;
         };
 
@@ -546,8 +555,8 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                 }
             } else {
                 // result is contiguous along n: transpose this warp's 32 x 128 block through shared memory
-                // (the operand stages are idle: the last accumulator was complete before we got here)
-                float *tile = reinterpret_cast<float *>(smem_gen + kRawStages * kRawStageBytes) + q * (32 * (kBN + 1));
+                // (the pipeline stages are idle: the last accumulator was complete before we got here)
+                float *tile = reinterpret_cast<float *>(smem_gen) + q * (32 * (kBN + 1));
 #pragma unroll
                 for (int j = 0; j < kBN; ++j) tile[lane * (kBN + 1) + j] = __fmul_rn(prm.scale, acc[j]);
                 __syncwarp();
@@ -733,6 +742,7 @@ static vgc_status tc_launch(KernelFn kernel, const CUtensorMap &ma, const CUtens
     }
     prm.M = M; prm.N = N; prm.k_slices = k_slices; prm.slices_per_split = plan.slices_per_split;
     prm.chunk = default_chunk();
+    { static const int dbg = getenv("VGC_TC_DEBUG") ? atoi(getenv("VGC_TC_DEBUG")) : 0; prm.debug = dbg; }
     prm.status = static_cast<uint32_t *>(ws);
     prm.partial = reinterpret_cast<float *>(static_cast<char *>(ws) + 256);
     dim3 grid(plan.tiles_x, plan.tiles_y, plan.splits);
