@@ -43,16 +43,26 @@ namespace tc {
 constexpr int kBM = 128;            // output rows per block (UMMA M)
 constexpr int kBN = 128;            // output columns per block (UMMA N)
 constexpr int kBK = 32;             // k per pipeline slice (= 128 bytes of fp32)
-constexpr int kStages = 3;          // each stage: raw fp32 tiles, overwritten in place by hi, plus the lo tiles
+#ifndef VGC_TC_RAW_SLOTS
+#define VGC_TC_RAW_SLOTS 5
+#endif
+#ifndef VGC_TC_LO_SLOTS
+#define VGC_TC_LO_SLOTS 2
+#endif
+// The pipeline is bound by how many bytes are in flight, so the raw tiles get as many slots as fit:
+// a raw slot holds the fp32 tiles of one slice (overwritten in place by their hi parts), a lo slot the
+// lo parts, which only exist between the transform and the MMAs that consume them.
+constexpr int kRawSlots = VGC_TC_RAW_SLOTS;
+constexpr int kLoSlots = VGC_TC_LO_SLOTS;
 constexpr int kThreadsTc = 448;
 constexpr int kTransformWarps = 8;
 constexpr int kTransformThreads = 32 * kTransformWarps;
 constexpr int kEpilogueWarps = 4;
 constexpr uint32_t kRawBytesA = kBM * kBK * 4;                      // 16 KB
 constexpr uint32_t kRawBytesB = kBN * kBK * 4;                      // 16 KB
-constexpr uint32_t kRawStageBytes = kRawBytesA + kRawBytesB;        // 32 KB: [A raw/hi][B raw/hi]
-constexpr uint32_t kStageBytes = 2 * kRawStageBytes;                // 64 KB: ... then [A lo][B lo]
-constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256;
+constexpr uint32_t kRawStageBytes = kRawBytesA + kRawBytesB;        // 32 KB: [A raw/hi][B raw/hi], same for lo
+constexpr uint32_t kLoBase = kRawSlots * kRawStageBytes;            // lo slots follow the raw slots
+constexpr uint32_t kSmemBytes = (kRawSlots + kLoSlots) * kRawStageBytes + 1024 /*align*/ + 128;
 constexpr uint32_t kTmemCols = 2 * kBN;                             // two accumulator buffers
 constexpr uint32_t kWaitLimit = 1u << 22;                           // polls before a wait gives up
 
@@ -75,6 +85,7 @@ struct Params {
     long long ld_m, ld_n;
     float *partial;          // split-K scratch [split][tile][column][row], used when gridDim.z > 1
     uint32_t *status;        // device word; VGC_DEV_TIMEOUT is OR-ed in if a wait expired
+    int prefetch;            // slices ahead of the TMA loads that are prefetched into L2 (0: off)
     int debug;               // experiments: 1 skip MMAs, 2 skip transform math, 4 skip gathers
 };
 
@@ -129,6 +140,13 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
+}
+
+// L2 prefetch of a tile that a later TMA load will fetch (no shared memory, no barrier involved)
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap *map, int c0, int c1, int c2)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(c0), "r"(c1), "r"(c2)
+                 : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -276,7 +294,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     constexpr bool kAnyGather = kGatherA || kGatherB;
 
     extern __shared__ uint8_t smem_raw_[];
-    __shared__ __align__(8) uint64_t bars[3 * kStages + 5];
+    __shared__ __align__(8) uint64_t bars[3 * kRawSlots + kLoSlots + 5];
     __shared__ uint32_t tmem_base_slot;
     __shared__ volatile uint32_t abort_flag;
 
@@ -284,9 +302,11 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     const uint32_t smem_base = (smem_u32(smem_raw_) + 1023u) & ~1023u;     // 1024-byte aligned tiles
     uint8_t *smem_gen = smem_raw_ + (smem_base - smem_u32(smem_raw_));
 
-    // per stage: raw_full (TMA landed) -> op_full (hi/lo written) -> empty (MMAs that read it retired)
-    uint64_t *raw_full = bars, *op_full = bars + kStages, *empty = bars + 2 * kStages;
-    uint64_t *acc_full = bars + 3 * kStages, *acc_empty = acc_full + 2, *drain = acc_empty + 2;
+    // per raw slot: raw_full (TMA landed) -> op_full (hi/lo written) -> empty (MMAs that read it retired);
+    // per lo slot: lo_empty (MMAs that read it retired)
+    uint64_t *raw_full = bars, *op_full = bars + kRawSlots, *empty = bars + 2 * kRawSlots;
+    uint64_t *lo_empty = bars + 3 * kRawSlots;
+    uint64_t *acc_full = lo_empty + kLoSlots, *acc_empty = acc_full + 2, *drain = acc_empty + 2;
 
     const int m0 = blockIdx.y * kBM, n0 = blockIdx.x * kBN;
     const int n_valid = min(kBN, prm.N - n0);                              // columns of this tile that exist
@@ -298,11 +318,12 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        for (int i = 0; i < kStages; ++i) {
+        for (int i = 0; i < kRawSlots; ++i) {
             mbar_init(smem_u32(&raw_full[i]), 1);
             mbar_init(smem_u32(&op_full[i]), kTransformWarps);
             mbar_init(smem_u32(&empty[i]), 1);
         }
+        for (int i = 0; i < kLoSlots; ++i) mbar_init(smem_u32(&lo_empty[i]), 1);
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&acc_full[i]), 1); mbar_init(smem_u32(&acc_empty[i]), kEpilogueWarps); }
         mbar_init(smem_u32(drain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -323,17 +344,23 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         if (lane == 0 && kAnyTma) {
             int issued = 0;
             for (int i = 0; i < n_slices; ++i) {
-                const int st = i % kStages;
-                const uint32_t ph = (uint32_t)(i / kStages) & 1u;
+                const int st = i % kRawSlots;
+                const uint32_t ph = (uint32_t)(i / kRawSlots) & 1u;
                 if (!mbar_wait(smem_u32(&empty[st]), ph ^ 1u, &abort_flag)) break;
                 const uint32_t full = smem_u32(&raw_full[st]);
-                const uint32_t dst_a = smem_base + st * kStageBytes, dst_b = dst_a + kRawBytesA;
+                const uint32_t dst_a = smem_base + st * kRawStageBytes, dst_b = dst_a + kRawBytesA;
                 mbar_expect_tx(full, prm.tx_bytes);
                 const int slice = slice_begin + i;
                 if (kMajor == kMajorK) {
                     const int z = slice / prm.p_slices, p0 = (slice - z * prm.p_slices) * kBK;
                     if (!kGatherA) tma_load_3d(dst_a, &map_a, full, p0, m0, z);
                     if (!kGatherB) tma_load_3d(dst_b, &map_b, full, p0, n0, z);
+                    if (prm.prefetch > 0 && i + prm.prefetch < n_slices) {      // warm L2 for a slice further ahead
+                        const int sl = slice + prm.prefetch;
+                        const int zp = sl / prm.p_slices, pp = (sl - zp * prm.p_slices) * kBK;
+                        if (!kGatherA) tma_prefetch_3d(&map_a, pp, m0, zp);
+                        if (!kGatherB) tma_prefetch_3d(&map_b, pp, n0, zp);
+                    }
                 } else {
                     const int k0 = slice * kBK;
 #pragma unroll
@@ -345,10 +372,10 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             }
             // on an abort: loads already issued must land before the block may exit
             if (abort_flag) {
-                const int first = issued > kStages ? issued - kStages : 0;
+                const int first = issued > kRawSlots ? issued - kRawSlots : 0;
                 for (int i = first; i < issued; ++i) {
-                    const uint32_t bar = smem_u32(&raw_full[i % kStages]);
-                    const uint32_t ph = (uint32_t)(i / kStages) & 1u;
+                    const uint32_t bar = smem_u32(&raw_full[i % kRawSlots]);
+                    const uint32_t ph = (uint32_t)(i / kRawSlots) & 1u;
                     for (uint32_t t = 0; t < kWaitLimit && !mbar_try(bar, ph); ++t) {}
                 }
             }
@@ -373,12 +400,12 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                 const uint32_t d_tmem = tmem_base + (uint32_t)b * kBN;
                 const int chunk_end = min(n_slices, (c + 1) * prm.chunk);
                 for (bool first = true; i < chunk_end; ++i) {
-                    const int st = i % kStages;
-                    ok = mbar_wait(smem_u32(&op_full[st]), (uint32_t)(i / kStages) & 1u, &abort_flag);
+                    const int st = i % kRawSlots, ls = i % kLoSlots;
+                    ok = mbar_wait(smem_u32(&op_full[st]), (uint32_t)(i / kRawSlots) & 1u, &abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t hi_a = smem_base + st * kStageBytes, hi_b = hi_a + kRawBytesA;
-                    const uint32_t lo_a = hi_a + kRawStageBytes, lo_b = lo_a + kRawBytesA;
+                    const uint32_t hi_a = smem_base + st * kRawStageBytes, hi_b = hi_a + kRawBytesA;
+                    const uint32_t lo_a = smem_base + kLoBase + ls * kRawStageBytes, lo_b = lo_a + kRawBytesA;
 #pragma unroll
                     for (int kk = 0; kk < kBK / 8; ++kk) {
                         if (prm.debug & 1) break;
@@ -391,7 +418,8 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                         tc_mma_tf32(d_tmem, da_lo, db_hi, idesc, 1u);
                         first = false;
                     }
-                    tc_commit(smem_u32(&empty[st]));              // stage free once these MMAs retire
+                    tc_commit(smem_u32(&empty[st]));              // both slots are free once these MMAs retire
+                    tc_commit(smem_u32(&lo_empty[ls]));
                 }
                 if (ok) tc_commit(smem_u32(&acc_full[b]));
             }
@@ -451,21 +479,22 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         };
         // transform of slice i; gathered elements come in registers, TMA tiles from the raw stage
         auto process = [&](int i, const float (&ga)[kRowsPerThread][4], const float (&gb)[kRowsPerThread][4]) -> bool {
-            const int st = i % kStages;
-            const uint32_t ph = (uint32_t)(i / kStages) & 1u;
-            // a stage is ours once its TMA tiles landed (the producer waited for it to be empty), or, with
-            // nothing coming by TMA, once the MMAs that last read it retired
+            const int st = i % kRawSlots, ls = i % kLoSlots;
+            const uint32_t ph = (uint32_t)(i / kRawSlots) & 1u;
+            // a raw slot is ours once its TMA tiles landed (the producer waited for it to be empty), or, with
+            // nothing coming by TMA, once the MMAs that last read it retired; likewise the lo slot
             if (kAnyTma ? !mbar_wait(smem_u32(&raw_full[st]), ph, &abort_flag)
                         : !mbar_wait(smem_u32(&empty[st]), ph ^ 1u, &abort_flag))
                 return false;
-            uint8_t *hi = smem_gen + st * kStageBytes;           // raw tiles live here and become the hi tiles
-            uint8_t *lo = hi + kRawStageBytes;
+            if (!mbar_wait(smem_u32(&lo_empty[ls]), ((uint32_t)(i / kLoSlots) & 1u) ^ 1u, &abort_flag)) return false;
+            uint8_t *hi = smem_gen + st * kRawStageBytes;        // raw tiles live here and become the hi tiles
+            uint8_t *lo = smem_gen + kLoBase + ls * kRawStageBytes;
             if (prm.debug & 2) {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&op_full[st]));
                 return true;
             }
-            if (kAnyTma) {      // tiles that came by TMA: elementwise, in place, over their 16-byte chunks
+            if (kAnyTma && !(prm.debug & 8)) {      // tiles that came by TMA: elementwise, in place, over their 16-byte chunks
                 constexpr uint32_t c_begin = kGatherA ? kRawBytesA / 16 : 0;
                 constexpr uint32_t c_end = kGatherB ? kRawBytesA / 16 : kRawStageBytes / 16;
                 constexpr int kPerThread = c_end > c_begin ? (c_end - c_begin) / kTransformThreads : 1;
@@ -488,7 +517,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                     split_store(hi + kRawBytesA, lo + kRawBytesA, chunk_offset(row0 + 32 * r, kq), gb[r][0], gb[r][1],
                                 gb[r][2], gb[r][3]);
             }
-            fence_async_smem();                                   // generic-proxy writes -> tensor core reads
+            if (!(prm.debug & 32)) fence_async_smem();            // generic-proxy writes -> tensor core reads
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&op_full[st]));
             return true;
@@ -742,6 +771,7 @@ static vgc_status tc_launch(KernelFn kernel, const CUtensorMap &ma, const CUtens
     }
     prm.M = M; prm.N = N; prm.k_slices = k_slices; prm.slices_per_split = plan.slices_per_split;
     prm.chunk = default_chunk();
+    { static const int pf = getenv("VGC_TC_PREFETCH") ? atoi(getenv("VGC_TC_PREFETCH")) : 0; prm.prefetch = pf; }
     { static const int dbg = getenv("VGC_TC_DEBUG") ? atoi(getenv("VGC_TC_DEBUG")) : 0; prm.debug = dbg; }
     prm.status = static_cast<uint32_t *>(ws);
     prm.partial = reinterpret_cast<float *>(static_cast<char *>(ws) + 256);
