@@ -63,7 +63,11 @@ constexpr uint32_t kRawBytesB = kBN * kBK * 4;                      // 16 KB
 constexpr uint32_t kRawStageBytes = kRawBytesA + kRawBytesB;        // 32 KB: [A raw/hi][B raw/hi], same for lo
 constexpr uint32_t kLoBase = kRawSlots * kRawStageBytes;            // lo slots follow the raw slots
 constexpr uint32_t kSmemBytes = (kRawSlots + kLoSlots) * kRawStageBytes + 1024 /*align*/ + 128;
-constexpr uint32_t kTmemCols = 2 * kBN;                             // two accumulator buffers
+// With the A operand in tensor memory a lo slot holds the B tile only, so twice as many fit; the A
+// operand ring in TMEM has the same number of slots and shares their barrier.
+constexpr int kLoSlotsAT = 2 * kLoSlots;
+constexpr uint32_t kTmemColsA = 64;                                 // per slot: 32 columns hi + 32 columns lo
+constexpr uint32_t kTmemCols = 512;                                 // two accumulator buffers + the A operand ring
 constexpr uint32_t kWaitLimit = 1u << 22;                           // polls before a wait gives up
 
 enum { kMajorK = 0, kMajorMN = 1 };
@@ -167,6 +171,29 @@ __device__ __forceinline__ void tc_mma_tf32(uint32_t d_tmem, uint64_t a_desc, ui
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// same with the A operand read from tensor memory (lane = row, one 32-bit column per k)
+__device__ __forceinline__ void tc_mma_tf32_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 lanes x 16 columns: each thread stores 16 registers into its lane's row
+__device__ __forceinline__ void tc_st_32x16(uint32_t taddr, const uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
 // 32 lanes x 32 columns of 32-bit accumulators -> 32 registers per thread (thread = lane = row)
 __device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
 {
@@ -284,17 +311,20 @@ struct GatherRows {
 };
 
 // ---- the kernel ------------------------------------------------------------------------------
-template <int kMajor, int kModeA, int kModeB>
+template <int kMajor, int kModeA, int kModeB, bool kATmem>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const Params prm)
 {
     static_assert(kMajor == kMajorK || (kModeA == kTma && kModeB == kTma), "gathered tiles are K-major");
+    static_assert(!kATmem || (kMajor == kMajorK && kModeA == kTma), "A goes to tensor memory from a K-major TMA tile");
+    constexpr int kLoN = kATmem ? kLoSlotsAT : kLoSlots;                  // lo slots (and A operand slots in TMEM)
+    constexpr uint32_t kLoBytes = kATmem ? kRawBytesB : kRawStageBytes;  // bytes of one lo slot
     constexpr bool kGatherA = kModeA != kTma, kGatherB = kModeB != kTma;
     constexpr bool kAnyTma = !kGatherA || !kGatherB;
     constexpr bool kAnyGather = kGatherA || kGatherB;
 
     extern __shared__ uint8_t smem_raw_[];
-    __shared__ __align__(8) uint64_t bars[3 * kRawSlots + kLoSlots + 5];
+    __shared__ __align__(8) uint64_t bars[3 * kRawSlots + kLoSlotsAT + 5];
     __shared__ uint32_t tmem_base_slot;
     __shared__ volatile uint32_t abort_flag;
 
@@ -306,7 +336,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     // per lo slot: lo_empty (MMAs that read it retired)
     uint64_t *raw_full = bars, *op_full = bars + kRawSlots, *empty = bars + 2 * kRawSlots;
     uint64_t *lo_empty = bars + 3 * kRawSlots;
-    uint64_t *acc_full = lo_empty + kLoSlots, *acc_empty = acc_full + 2, *drain = acc_empty + 2;
+    uint64_t *acc_full = lo_empty + kLoSlotsAT, *acc_empty = acc_full + 2, *drain = acc_empty + 2;
 
     const int m0 = blockIdx.y * kBM, n0 = blockIdx.x * kBN;
     const int n_valid = min(kBN, prm.N - n0);                              // columns of this tile that exist
@@ -323,7 +353,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             mbar_init(smem_u32(&op_full[i]), kTransformWarps);
             mbar_init(smem_u32(&empty[i]), 1);
         }
-        for (int i = 0; i < kLoSlots; ++i) mbar_init(smem_u32(&lo_empty[i]), 1);
+        for (int i = 0; i < kLoSlotsAT; ++i) mbar_init(smem_u32(&lo_empty[i]), 1);
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&acc_full[i]), 1); mbar_init(smem_u32(&acc_empty[i]), kEpilogueWarps); }
         mbar_init(smem_u32(drain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -400,22 +430,29 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                 const uint32_t d_tmem = tmem_base + (uint32_t)b * kBN;
                 const int chunk_end = min(n_slices, (c + 1) * prm.chunk);
                 for (bool first = true; i < chunk_end; ++i) {
-                    const int st = i % kRawSlots, ls = i % kLoSlots;
+                    const int st = i % kRawSlots, ls = i % kLoN;
                     ok = mbar_wait(smem_u32(&op_full[st]), (uint32_t)(i / kRawSlots) & 1u, &abort_flag);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t hi_a = smem_base + st * kRawStageBytes, hi_b = hi_a + kRawBytesA;
-                    const uint32_t lo_a = smem_base + kLoBase + ls * kRawStageBytes, lo_b = lo_a + kRawBytesA;
+                    const uint32_t lo_a = smem_base + kLoBase + ls * kLoBytes, lo_b = kATmem ? lo_a : lo_a + kRawBytesA;
+                    const uint32_t ta_hi = tmem_base + 2 * kBN + ls * kTmemColsA, ta_lo = ta_hi + 32;
 #pragma unroll
                     for (int kk = 0; kk < kBK / 8; ++kk) {
                         if (prm.debug & 1) break;
-                        const uint64_t da_hi = smem_desc(hi_a + kk * k_step, lbo, sbo, layout);
                         const uint64_t db_hi = smem_desc(hi_b + kk * k_step, lbo, sbo, layout);
-                        const uint64_t da_lo = smem_desc(lo_a + kk * k_step, lbo, sbo, layout);
                         const uint64_t db_lo = smem_desc(lo_b + kk * k_step, lbo, sbo, layout);
-                        tc_mma_tf32(d_tmem, da_hi, db_hi, idesc, first ? 0u : 1u);
-                        tc_mma_tf32(d_tmem, da_hi, db_lo, idesc, 1u);
-                        tc_mma_tf32(d_tmem, da_lo, db_hi, idesc, 1u);
+                        if (kATmem) {
+                            tc_mma_tf32_ts(d_tmem, ta_hi + kk * 8, db_hi, idesc, first ? 0u : 1u);
+                            tc_mma_tf32_ts(d_tmem, ta_hi + kk * 8, db_lo, idesc, 1u);
+                            tc_mma_tf32_ts(d_tmem, ta_lo + kk * 8, db_hi, idesc, 1u);
+                        } else {
+                            const uint64_t da_hi = smem_desc(hi_a + kk * k_step, lbo, sbo, layout);
+                            const uint64_t da_lo = smem_desc(lo_a + kk * k_step, lbo, sbo, layout);
+                            tc_mma_tf32(d_tmem, da_hi, db_hi, idesc, first ? 0u : 1u);
+                            tc_mma_tf32(d_tmem, da_hi, db_lo, idesc, 1u);
+                            tc_mma_tf32(d_tmem, da_lo, db_hi, idesc, 1u);
+                        }
                         first = false;
                     }
                     tc_commit(smem_u32(&empty[st]));              // both slots are free once these MMAs retire
@@ -479,32 +516,60 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         };
         // transform of slice i; gathered elements come in registers, TMA tiles from the raw stage
         auto process = [&](int i, const float (&ga)[kRowsPerThread][4], const float (&gb)[kRowsPerThread][4]) -> bool {
-            const int st = i % kRawSlots, ls = i % kLoSlots;
+            const int st = i % kRawSlots, ls = i % kLoN;
             const uint32_t ph = (uint32_t)(i / kRawSlots) & 1u;
             // a raw slot is ours once its TMA tiles landed (the producer waited for it to be empty), or, with
             // nothing coming by TMA, once the MMAs that last read it retired; likewise the lo slot
             if (kAnyTma ? !mbar_wait(smem_u32(&raw_full[st]), ph, &abort_flag)
                         : !mbar_wait(smem_u32(&empty[st]), ph ^ 1u, &abort_flag))
                 return false;
-            if (!mbar_wait(smem_u32(&lo_empty[ls]), ((uint32_t)(i / kLoSlots) & 1u) ^ 1u, &abort_flag)) return false;
+            if (!mbar_wait(smem_u32(&lo_empty[ls]), ((uint32_t)(i / kLoN) & 1u) ^ 1u, &abort_flag)) return false;
             uint8_t *hi = smem_gen + st * kRawStageBytes;        // raw tiles live here and become the hi tiles
-            uint8_t *lo = smem_gen + kLoBase + ls * kRawStageBytes;
+            // lo tiles: [A lo][B lo], or the B tile alone when A lives in tensor memory (then `lo` points
+            // one A tile below the slot so that the same chunk offsets address the B part)
+            uint8_t *lo = smem_gen + kLoBase + ls * kLoBytes - (kATmem ? kRawBytesA : 0);
             if (prm.debug & 2) {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&op_full[st]));
                 return true;
             }
+            if (kATmem) {
+                // A: this thread's row (TMEM lane) and half of the slice's 32 k -> hi / lo straight into TMEM
+                tc_fence_after();
+                const uint32_t q = warp & 3, h = (warp - 2) >> 2;
+                const int m_local = (int)(q * 32 + lane);
+                const uint8_t *arow = hi + m_local * 128;
+                float4 c4[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) c4[u] = *reinterpret_cast<const float4 *>(arow + (((4 * h + u) ^ (m_local & 7)) << 4));
+                uint32_t h16[16], l16[16];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const float e[4] = {c4[u].x, c4[u].y, c4[u].z, c4[u].w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float sq = __fmul_rn(e[j], e[j]);
+                        h16[4 * u + j] = to_tf32(sq);
+                        l16[4 * u + j] = to_tf32(__fsub_rn(sq, __uint_as_float(h16[4 * u + j])));
+                    }
+                }
+                const uint32_t taddr = tmem_base + ((q * 32u) << 16) + 2 * kBN + ls * kTmemColsA + 16 * h;
+                tc_st_32x16(taddr, h16);
+                tc_st_32x16(taddr + 32, l16);
+            }
             if (kAnyTma && !(prm.debug & 8)) {      // tiles that came by TMA: elementwise, in place, over their 16-byte chunks
-                constexpr uint32_t c_begin = kGatherA ? kRawBytesA / 16 : 0;
+                constexpr uint32_t c_begin = (kGatherA || kATmem) ? kRawBytesA / 16 : 0;
                 constexpr uint32_t c_end = kGatherB ? kRawBytesA / 16 : kRawStageBytes / 16;
                 constexpr int kPerThread = c_end > c_begin ? (c_end - c_begin) / kTransformThreads : 1;
-                float4 v[kPerThread];
+                if (c_end > c_begin) {
+                    float4 v[kPerThread];
 #pragma unroll
-                for (int u = 0; u < kPerThread; ++u)
-                    v[u] = *reinterpret_cast<const float4 *>(hi + 16 * (c_begin + (uint32_t)t + u * kTransformThreads));
+                    for (int u = 0; u < kPerThread; ++u)
+                        v[u] = *reinterpret_cast<const float4 *>(hi + 16 * (c_begin + (uint32_t)t + u * kTransformThreads));
 #pragma unroll
-                for (int u = 0; u < kPerThread; ++u)
-                    split_store(hi, lo, 16 * (c_begin + (uint32_t)t + u * kTransformThreads), v[u].x, v[u].y, v[u].z, v[u].w);
+                    for (int u = 0; u < kPerThread; ++u)
+                        split_store(hi, lo, 16 * (c_begin + (uint32_t)t + u * kTransformThreads), v[u].x, v[u].y, v[u].z, v[u].w);
+                }
             }
             if (kGatherA) {
 #pragma unroll
@@ -517,6 +582,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                     split_store(hi + kRawBytesA, lo + kRawBytesA, chunk_offset(row0 + 32 * r, kq), gb[r][0], gb[r][1],
                                 gb[r][2], gb[r][3]);
             }
+            if (kATmem) { tc_wait_st(); tc_fence_before(); }      // TMEM stores complete and ordered before the signal
             if (!(prm.debug & 32)) fence_async_smem();            // generic-proxy writes -> tensor core reads
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&op_full[st]));
@@ -802,7 +868,7 @@ vgc_status tc_sqgrad_linear(const float *x, const float *delta, int B, int in, i
     Params prm = {};
     prm.p_slices = 1; prm.tx_bytes = kRawStageBytes; prm.scale = scale; prm.accumulate = accumulate; prm.S = S;
     prm.ld_m = in; prm.ld_n = 1;
-    return tc_launch(sqgrad_tc<kMajorMN, kTma, kTma>, ma, mb, prm, out, in, (B + kBK - 1) / kBK, ws, ws_bytes, st);
+    return tc_launch(sqgrad_tc<kMajorMN, kTma, kTma, false>, ma, mb, prm, out, in, (B + kBK - 1) / kBK, ws, ws_bytes, st);
 }
 
 // Cout <= 64: the im2col rows take the 128-row A tile and the errors the narrow B tile
@@ -825,6 +891,7 @@ vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int 
     const bool err_tma = P >= kBK && P % 4 == 0 && !(force_gather & 1);
     const bool in_tma = P >= kBK && P % 4 == 0 && !(force_gather & 2) && Kh == 1 && Kw == 1 && sh == 1 && sw == 1 &&
                         ph == 0 && pw == 0;
+    static const bool a_tmem = !(getenv("VGC_TC_ATMEM") && atoi(getenv("VGC_TC_ATMEM")) == 0);   // experiments
     const bool swapped = conv_swapped(Cout, n_im2col);
     const int rows_err = swapped ? kBN : kBM, rows_in = swapped ? kBM : kBN;     // tile heights
     CUtensorMap m_err = {}, m_in = {};
@@ -853,17 +920,17 @@ vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int 
     KernelFn fn = nullptr;
     if (!swapped) {     // S[o][idx]: m = o, n = idx
         prm.ld_m = n_im2col; prm.ld_n = 1;
-        if (e == kTma && i == kTma) fn = sqgrad_tc<kMajorK, kTma, kTma>;
-        else if (e == kTma) fn = sqgrad_tc<kMajorK, kTma, kGatherIm2col>;
-        else if (i == kTma) fn = sqgrad_tc<kMajorK, kGatherErr, kTma>;
-        else fn = sqgrad_tc<kMajorK, kGatherErr, kGatherIm2col>;
+        if (e == kTma && i == kTma) fn = a_tmem ? sqgrad_tc<kMajorK, kTma, kTma, true> : sqgrad_tc<kMajorK, kTma, kTma, false>;
+        else if (e == kTma) fn = a_tmem ? sqgrad_tc<kMajorK, kTma, kGatherIm2col, true> : sqgrad_tc<kMajorK, kTma, kGatherIm2col, false>;
+        else if (i == kTma) fn = sqgrad_tc<kMajorK, kGatherErr, kTma, false>;
+        else fn = sqgrad_tc<kMajorK, kGatherErr, kGatherIm2col, false>;
         return tc_launch(fn, m_err, m_in, prm, Cout, n_im2col, k_slices, ws, ws_bytes, st);
     }
     prm.ld_m = 1; prm.ld_n = n_im2col;   // m = idx, n = o
-    if (e == kTma && i == kTma) fn = sqgrad_tc<kMajorK, kTma, kTma>;
-    else if (i == kTma) fn = sqgrad_tc<kMajorK, kTma, kGatherErr>;
-    else if (e == kTma) fn = sqgrad_tc<kMajorK, kGatherIm2col, kTma>;
-    else fn = sqgrad_tc<kMajorK, kGatherIm2col, kGatherErr>;
+    if (e == kTma && i == kTma) fn = a_tmem ? sqgrad_tc<kMajorK, kTma, kTma, true> : sqgrad_tc<kMajorK, kTma, kTma, false>;
+    else if (i == kTma) fn = a_tmem ? sqgrad_tc<kMajorK, kTma, kGatherErr, true> : sqgrad_tc<kMajorK, kTma, kGatherErr, false>;
+    else if (e == kTma) fn = sqgrad_tc<kMajorK, kGatherIm2col, kTma, false>;
+    else fn = sqgrad_tc<kMajorK, kGatherIm2col, kGatherErr, false>;
     return tc_launch(fn, m_in, m_err, prm, n_im2col, Cout, k_slices, ws, ws_bytes, st);
 }
 
