@@ -6,7 +6,8 @@
 //   1. TMA-loads the raw fp32 tiles of A (128 rows) and B (kBN rows) into a pipeline stage
 //      (128-byte swizzle, out-of-range parts filled with zeros),
 //   2. squares every element in fp32 and splits the square into two TF32 numbers hi + lo
-//      (hi = x*x rounded to 11 significant bits, lo = x*x - hi likewise); the transform is elementwise
+//      (hi = x*x rounded to 11 significant bits, lo = x*x - hi, of which the tensor core reads the
+//      leading 11 bits); the transform is elementwise
 //      and in place (hi overwrites the raw tile, lo goes beside it), so both inherit the swizzled
 //      layout the tensor core wants,
 //   3. issues three tcgen05.mma per 8-deep step -- hi*hi, hi*lo, lo*hi -- into a TMEM
@@ -121,11 +122,17 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait.  Returns false when it gave up or when another role already raised the abort flag.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
+// After a few immediate retries the waiter sleeps `sleep_ns` between polls so that it does not take
+// issue slots from the warps it is waiting for.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                          uint32_t sleep_ns = 32)
 {
     for (uint32_t i = 0; i < kWaitLimit; ++i) {
         if (mbar_try(bar, parity)) return true;
-        if (*abort_flag) return false;
+        if (i >= 4) {
+            if (*abort_flag) return false;
+            __nanosleep(sleep_ns);
+        }
     }
     *abort_flag = 1;
     return false;
@@ -244,10 +251,12 @@ __device__ __forceinline__ void split_store(uint8_t *hi_tile, uint8_t *lo_tile, 
     const float q0 = __fmul_rn(v0, v0), q1 = __fmul_rn(v1, v1), q2 = __fmul_rn(v2, v2), q3 = __fmul_rn(v3, v3);
     uint4 h, l;
     h.x = to_tf32(q0); h.y = to_tf32(q1); h.z = to_tf32(q2); h.w = to_tf32(q3);
-    l.x = to_tf32(__fsub_rn(q0, __uint_as_float(h.x)));
-    l.y = to_tf32(__fsub_rn(q1, __uint_as_float(h.y)));
-    l.z = to_tf32(__fsub_rn(q2, __uint_as_float(h.z)));
-    l.w = to_tf32(__fsub_rn(q3, __uint_as_float(h.w)));
+    // lo = q - hi is exact in fp32; the tensor core reads only its upper 19 bits, an error of at most
+    // 2^-10 * |lo| <= 2^-22 * q whose sign follows lo (no systematic bias)
+    l.x = __float_as_uint(__fsub_rn(q0, __uint_as_float(h.x)));
+    l.y = __float_as_uint(__fsub_rn(q1, __uint_as_float(h.y)));
+    l.z = __float_as_uint(__fsub_rn(q2, __uint_as_float(h.z)));
+    l.w = __float_as_uint(__fsub_rn(q3, __uint_as_float(h.w)));
     *reinterpret_cast<uint4 *>(hi_tile + off) = h;
     *reinterpret_cast<uint4 *>(lo_tile + off) = l;
 }
@@ -376,7 +385,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             for (int i = 0; i < n_slices; ++i) {
                 const int st = i % kRawSlots;
                 const uint32_t ph = (uint32_t)(i / kRawSlots) & 1u;
-                if (!mbar_wait(smem_u32(&empty[st]), ph ^ 1u, &abort_flag)) break;
+                if (!mbar_wait(smem_u32(&empty[st]), ph ^ 1u, &abort_flag, 64)) break;
                 const uint32_t full = smem_u32(&raw_full[st]);
                 const uint32_t dst_a = smem_base + st * kRawStageBytes, dst_b = dst_a + kRawBytesA;
                 mbar_expect_tx(full, prm.tx_bytes);
@@ -550,7 +559,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                     for (int j = 0; j < 4; ++j) {
                         const float sq = __fmul_rn(e[j], e[j]);
                         h16[4 * u + j] = to_tf32(sq);
-                        l16[4 * u + j] = to_tf32(__fsub_rn(sq, __uint_as_float(h16[4 * u + j])));
+                        l16[4 * u + j] = __float_as_uint(__fsub_rn(sq, __uint_as_float(h16[4 * u + j])));
                     }
                 }
                 const uint32_t taddr = tmem_base + ((q * 32u) << 16) + 2 * kBN + ls * kTmemColsA + 16 * h;
@@ -609,7 +618,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         bool ok = true;
         for (int c = 0; c < n_chunks && ok; ++c) {
             const int b = c & 1;
-            ok = mbar_wait(smem_u32(&acc_full[b]), (uint32_t)(c >> 1) & 1u, &abort_flag);
+            ok = mbar_wait(smem_u32(&acc_full[b]), (uint32_t)(c >> 1) & 1u, &abort_flag, 256);
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((q * 32u) << 16) + (uint32_t)b * kBN;
@@ -682,58 +691,53 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     if (threadIdx.x == 0 && abort_flag) atomicOr(prm.status, VGC_DEV_TIMEOUT);
 }
 
-// Combine split-K partial tiles in a fixed order.  One block per 32 x 32 patch of a tile: partials are
-// read along rows (their unit stride), the result is written along whichever of m / n has unit stride.
+// Combine split-K partial tiles in a fixed order.  One block per 32 x 8 patch of a tile, one output per
+// thread: partials are read along rows (their unit stride), the result is written along whichever of
+// m / n has unit stride.
 __global__ void __launch_bounds__(256)
 sqgrad_tc_combine(const float *__restrict__ partial, int splits, int tiles_x, int tiles_y, int M, int N, float scale,
                   int accumulate, float *__restrict__ S, long long ld_m, long long ld_n)
 {
-    __shared__ float patch[32][33];
-    const int tile = blockIdx.x >> 4, sub = blockIdx.x & 15;
+    __shared__ float patch[8][33];
+    const int tile = blockIdx.x >> 6, sub = blockIdx.x & 63;
     const int tx = tile % tiles_x, ty = tile / tiles_x;
-    const int r0 = (sub & 3) * 32, j0 = (sub >> 2) * 32;                  // patch origin inside the tile
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;              // 8 warps x 4 columns each
+    const int r0 = (sub & 3) * 32, j0 = (sub >> 2) * 8;                   // patch origin inside the tile
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;              // lane -> row, warp -> column
     const size_t tiles = (size_t)tiles_x * tiles_y;
     if (ty * kBM + r0 >= M || tx * kBN + j0 >= N) return;
-#pragma unroll
-    for (int jj = 0; jj < 4; ++jj) {
-        const int j = j0 + w * 4 + jj;
+    const int j = j0 + w;
+    float sum = 0.f;
+    if (tx * kBN + j < N) {
         const float *src = partial + ((size_t)tile * kBN + j) * kBM + r0 + lane;
-        float sum = 0.f;
-        if (tx * kBN + j < N) {
-            const size_t stride = tiles * (size_t)(kBM * kBN);
-            int z = 0;
-            for (; z + 8 <= splits; z += 8) {               // eight loads in flight, summed in split order
-                float v[8];
+        const size_t stride = tiles * (size_t)(kBM * kBN);
+        int z = 0;
+        for (; z + 8 <= splits; z += 8) {                   // eight loads in flight, summed in split order
+            float v[8];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) v[u] = __ldcs(src + (size_t)(z + u) * stride);
+            for (int u = 0; u < 8; ++u) v[u] = __ldcs(src + (size_t)(z + u) * stride);
 #pragma unroll
-                for (int u = 0; u < 8; ++u) sum = __fadd_rn(sum, v[u]);
-            }
-            for (; z < splits; ++z) sum = __fadd_rn(sum, __ldcs(src + (size_t)z * stride));
+            for (int u = 0; u < 8; ++u) sum = __fadd_rn(sum, v[u]);
         }
-        patch[w * 4 + jj][lane] = __fmul_rn(scale, sum);                   // patch[column][row]
+        for (; z < splits; ++z) sum = __fadd_rn(sum, __ldcs(src + (size_t)z * stride));
     }
-    __syncthreads();
+    const float res = __fmul_rn(scale, sum);
     if (ld_m == 1) {
-#pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-            const int m = ty * kBM + r0 + lane, n = tx * kBN + j0 + w * 4 + jj;
-            if (m < M && n < N) {
-                float *dst = S + (size_t)m + (size_t)n * ld_n;
-                const float res = patch[w * 4 + jj][lane];
-                *dst = accumulate ? __fadd_rn(*dst, res) : res;
-            }
+        const int m = ty * kBM + r0 + lane, n = tx * kBN + j;
+        if (m < M && n < N) {
+            float *dst = S + (size_t)m + (size_t)n * ld_n;
+            *dst = accumulate ? __fadd_rn(*dst, res) : res;
         }
-    } else {
-#pragma unroll
-        for (int rr = 0; rr < 4; ++rr) {
-            const int m = ty * kBM + r0 + w * 4 + rr, n = tx * kBN + j0 + lane;
-            if (m < M && n < N) {
-                float *dst = S + (size_t)m * ld_m + n;
-                const float res = patch[lane][w * 4 + rr];
-                *dst = accumulate ? __fadd_rn(*dst, res) : res;
-            }
+        return;
+    }
+    patch[w][lane] = res;                                                  // patch[column][row]
+    __syncthreads();
+    {
+        const int c = threadIdx.x & 7, r = threadIdx.x >> 3;              // 8 consecutive columns per row
+        const int m = ty * kBM + r0 + r, n = tx * kBN + j0 + c;
+        if (m < M && n < N) {
+            float *dst = S + (size_t)m * ld_m + n;
+            const float out = patch[c][r];
+            *dst = accumulate ? __fadd_rn(*dst, out) : out;
         }
     }
 }
@@ -845,7 +849,7 @@ static vgc_status tc_launch(KernelFn kernel, const CUtensorMap &ma, const CUtens
     kernel<<<grid, kThreadsTc, kSmemBytes, st>>>(ma, mb, prm);
     count_launch();
     if (plan.splits > 1) {
-        sqgrad_tc_combine<<<(unsigned)(plan.tiles_x * plan.tiles_y * 16), 256, 0, st>>>(
+        sqgrad_tc_combine<<<(unsigned)(plan.tiles_x * plan.tiles_y * 64), 256, 0, st>>>(
             prm.partial, plan.splits, plan.tiles_x, plan.tiles_y, M, N, prm.scale, prm.accumulate, prm.S, prm.ld_m,
             prm.ld_n);
         count_launch();
