@@ -146,6 +146,33 @@ vgc_status vgc_compress(const float *g, const float *s, float *r, float *v, size
                         const uint32_t *group_offsets, int K, float alpha, float zeta,
                         const vgc_message *out, void *ws, size_t ws_bytes, vgc_stream_t stream);
 
+/* vgc_compress without a workspace argument.  (No counterpart in the paper: this is a packaging
+ * variant of the call above for hosts that cannot allocate.)
+ *
+ * Who needs it: callers that are not in a position to allocate device memory where they call the
+ * library -- programs whose device memory was planned and handed out in full beforehand, plug-ins
+ * invoked in the middle of another framework's step where an allocation would stall the device or is
+ * not permitted, and hosts that only ever lend the library the tensors of the call.  Here the scratch
+ * is a fixed array inside the library image: every GPU that loads the library sets aside
+ * 8 * VGC_COMPRESS_STATIC_MAX_PARAMS bytes (plus a few tens of KB) until the process exits.
+ *
+ *   - Same arguments, results and error rules as vgc_compress, minus ws / ws_bytes.
+ *   - n > VGC_COMPRESS_STATIC_MAX_PARAMS or K > VGC_COMPRESS_STATIC_MAX_GROUPS: VGC_ERR_UNSUPPORTED
+ *     (nothing is enqueued).
+ *   - The call itself performs no allocation of any kind.  The first call on each device looks up
+ *     the device address of the array (one cudaGetSymbolAddress, with that device current); make that
+ *     first call before any stream capture starts.
+ *   - All calls on a device share the one array and it keeps whatever the previous call left in it
+ *     (the call clears the part that must start at zero).  Two calls that overlap on the GPU -- other
+ *     streams, other host threads -- race on it: serialise them, or use vgc_compress with separate
+ *     workspaces.
+ */
+#define VGC_COMPRESS_STATIC_MAX_PARAMS (1u << 21)
+#define VGC_COMPRESS_STATIC_MAX_GROUPS 1024
+vgc_status vgc_compress_static(const float *g, const float *s, float *r, float *v, size_t n,
+                               const uint32_t *group_offsets, int K, float alpha, float zeta,
+                               const vgc_message *out, vgc_stream_t stream);
+
 /* ---------------------------------------------------------------------------------------------
  * (3) Decoder: the decode-and-sum half of CommunicateAndUpdate (Sec. 4.3; Fig. 1 caption).
  *

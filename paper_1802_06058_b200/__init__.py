@@ -27,7 +27,7 @@ EXPORTS = [
     "vgc_status_string", "vgc_version", "vgc_kernel_launch_count",
     "vgc_sqgrad_linear_workspace_bytes", "vgc_sqgrad_linear",
     "vgc_sqgrad_conv_workspace_bytes", "vgc_sqgrad_conv",
-    "vgc_compress_workspace_bytes", "vgc_compress",
+    "vgc_compress_workspace_bytes", "vgc_compress", "vgc_compress_static",
     "vgc_decode_accumulate",
 ]
 
@@ -76,6 +76,8 @@ def load_library():
     lib.vgc_compress_workspace_bytes.restype = sz
     lib.vgc_compress.argtypes = [vp, vp, vp, vp, sz, vp, i, f, f, ctypes.POINTER(_MessageStruct), vp, sz, vp]
     lib.vgc_compress.restype = i
+    lib.vgc_compress_static.argtypes = [vp, vp, vp, vp, sz, vp, i, f, f, ctypes.POINTER(_MessageStruct), vp]
+    lib.vgc_compress_static.restype = i
     lib.vgc_decode_accumulate.argtypes = [ctypes.POINTER(_ViewStruct), i, vp, i, f, vp, sz, vp, vp]
     lib.vgc_decode_accumulate.restype = i
     _lib = lib
@@ -223,6 +225,31 @@ def vgc_compress(g, s, r, v, group_offsets, alpha: float, zeta: float, out: Mess
                                      _dev(group_offsets, torch.int32, "group_offsets"), K, float(alpha),
                                      float(zeta), ctypes.byref(msg), wp, wb, _stream(stream))
     _check(st, "vgc_compress")
+    return out
+
+
+VGC_COMPRESS_STATIC_MAX_PARAMS = 1 << 21
+VGC_COMPRESS_STATIC_MAX_GROUPS = 1024
+
+
+def vgc_compress_static(g, s, r, v, group_offsets, alpha: float, zeta: float, out: MessageBuffers, stream=None):
+    """vgc_compress for callers that cannot allocate a workspace (memory planned up front, plug-ins
+    running inside someone else's step, hosts that lend only the call's tensors): the scratch is a fixed
+    array inside the library, so n is limited to VGC_COMPRESS_STATIC_MAX_PARAMS.  Nothing is allocated by
+    this call -- the binding passes pointers only.  Calls on one device share the scratch: do not let
+    two of them overlap on the GPU.  Make the first call on a device outside any stream capture."""
+    n = g.numel()
+    if s.numel() != n or r.numel() != n or v.numel() != n:
+        raise ValueError("g, s, r, v must have the same length")
+    K = group_offsets.numel() - 1
+    if out.K != K:
+        raise ValueError("message buffers were made for a different number of groups")
+    msg = out.struct()
+    st = load_library().vgc_compress_static(_dev(g, torch.float32, "g"), _dev(s, torch.float32, "s"),
+                                            _dev(r, torch.float32, "r"), _dev(v, torch.float32, "v"), n,
+                                            _dev(group_offsets, torch.int32, "group_offsets"), K, float(alpha),
+                                            float(zeta), ctypes.byref(msg), _stream(stream))
+    _check(st, "vgc_compress_static")
     return out
 
 

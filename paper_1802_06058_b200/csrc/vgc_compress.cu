@@ -436,3 +436,45 @@ extern "C" vgc_status vgc_compress(const float *g, const float *s, float *r, flo
     VGC_CUDA_OK(cudaGetLastError());
     return VGC_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// Allocation-free variant of vgc_compress: the scratch lives in the library image
+// ------------------------------------------------------------------------------------------
+// Some callers cannot hand the library a workspace because they cannot allocate device memory at the
+// point where they call it: code running under a memory plan fixed ahead of time (every byte of the
+// device budget already assigned), plug-ins called from inside another framework's step where
+// cudaMalloc would synchronise the device or is simply forbidden, and embedding hosts that expose
+// only the tensors they pass in.  For them the scratch of vgc_compress is a fixed array that every
+// GPU loading this library reserves until the process exits; its size bounds the buffer length.
+namespace vgc {
+constexpr size_t kStaticMaxParams = VGC_COMPRESS_STATIC_MAX_PARAMS;
+constexpr int kStaticMaxGroups = VGC_COMPRESS_STATIC_MAX_GROUPS;
+// worst-case layout: per-tensor maxima, per-tile counts, chunk totals, 8 bytes of staging per parameter
+constexpr size_t kStaticScratchBytes = 8 * kStaticMaxParams + (kStaticMaxParams / kTileA) * 8 + kStaticMaxGroups * 4 + 64 * 1024;
+static __device__ __align__(256) unsigned char g_compress_scratch[kStaticScratchBytes];
+}  // namespace vgc
+
+extern "C" vgc_status vgc_compress_static(const float *g, const float *s, float *r, float *v, size_t n,
+                                          const uint32_t *group_offsets, int K, float alpha, float zeta,
+                                          const vgc_message *out, vgc_stream_t stream)
+{
+    if (n > kStaticMaxParams || K > kStaticMaxGroups) return VGC_ERR_UNSUPPORTED;
+    if (n == 0) return VGC_OK;
+    if (K < 1) return VGC_ERR_INVALID_ARG;
+    if (compress_layout(n, K).total > kStaticScratchBytes) return VGC_ERR_UNSUPPORTED;
+    // Host code sees g_compress_scratch only as a stand-in for the device array: the address a kernel can
+    // use has to be asked for, once per device, with that device current.
+    constexpr int kMaxDevices = 64;
+    static void *scratch_of_device[kMaxDevices] = {};
+    int dev = -1;
+    VGC_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return VGC_ERR_UNSUPPORTED;
+    if (!scratch_of_device[dev]) {
+        void *p = nullptr;
+        VGC_CUDA_OK(cudaGetSymbolAddress(&p, g_compress_scratch));
+        if (!p) return VGC_ERR_CUDA;
+        scratch_of_device[dev] = p;
+    }
+    return vgc_compress(g, s, r, v, n, group_offsets, K, alpha, zeta, out, scratch_of_device[dev], kStaticScratchBytes,
+                        stream);
+}
