@@ -195,6 +195,29 @@ vgc_status vgc_decode_accumulate(const vgc_message_view *msgs, int W,
                                  const uint32_t *group_offsets, int K, float scale,
                                  float *u, size_t n, uint32_t *dev_status, vgc_stream_t stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * One worker step from HOST buffers (end-to-end form of (1) + (2); Algorithm 1 from CalcGrad()'s
+ * outputs to the encoded message).  For each layer, in order: copy x and delta from host memory into
+ * the given device buffers, compute the layer's squared-gradient sums into its slice of s_dev (layer
+ * l is weight tensor l of the flat buffer, K == n_layers); then copy g from the host, run vgc_compress
+ * and copy the message back: counters_host[4] = {nnz, n_criterion, n_dropped, dev_status} and the
+ * first min(nnz, capacity) words into words_host.  Host buffers should be pinned.  Unlike the other
+ * entry points this one WAITS for the stream (twice: the word count has to reach the host before the
+ * words can be copied).  `out` holds device pointers as for vgc_compress; r, v are device state.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    int is_conv;                 /* 0: dense layer (C = in, Cout = out; H, W, K*, stride, pad ignored) */
+    int B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w;
+    const float *x_host, *delta_host; /* host: x [B][C][H][W] or [B][in]; delta [B][Cout][Ho][Wo] or [B][out] */
+    float *x_dev, *delta_dev;         /* device staging of the same sizes */
+} vgc_layer_host;
+
+vgc_status vgc_step_host(const vgc_layer_host *layers, int n_layers, const float *g_host, float *g_dev,
+                         float *s_dev, float *r, float *v, size_t n, const uint32_t *group_offsets, int K,
+                         float alpha, float zeta, float scale, const vgc_message *out, uint32_t *words_host,
+                         uint32_t *counters_host, void *ws_sqgrad, size_t ws_sqgrad_bytes, void *ws_compress,
+                         size_t ws_compress_bytes, vgc_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

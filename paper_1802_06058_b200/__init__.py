@@ -28,7 +28,7 @@ EXPORTS = [
     "vgc_sqgrad_linear_workspace_bytes", "vgc_sqgrad_linear",
     "vgc_sqgrad_conv_workspace_bytes", "vgc_sqgrad_conv",
     "vgc_compress_workspace_bytes", "vgc_compress", "vgc_compress_static",
-    "vgc_decode_accumulate",
+    "vgc_decode_accumulate", "vgc_step_host",
 ]
 
 
@@ -42,6 +42,13 @@ class _MessageStruct(ctypes.Structure):      # mirrors vgc_message
     _fields_ = [("words", ctypes.c_void_p), ("capacity", ctypes.c_uint32), ("group_exp", ctypes.c_void_p),
                 ("nnz", ctypes.c_void_p), ("n_criterion", ctypes.c_void_p), ("n_dropped", ctypes.c_void_p),
                 ("mask", ctypes.c_void_p), ("dev_status", ctypes.c_void_p)]
+
+
+class _LayerHostStruct(ctypes.Structure):    # mirrors vgc_layer_host
+    _fields_ = [(name, ctypes.c_int) for name in ("is_conv", "B", "C", "H", "W", "Cout", "Kh", "Kw", "stride_h",
+                                                  "stride_w", "pad_h", "pad_w")] + \
+               [("x_host", ctypes.c_void_p), ("delta_host", ctypes.c_void_p), ("x_dev", ctypes.c_void_p),
+                ("delta_dev", ctypes.c_void_p)]
 
 
 class _ViewStruct(ctypes.Structure):         # mirrors vgc_message_view
@@ -78,6 +85,9 @@ def load_library():
     lib.vgc_compress.restype = i
     lib.vgc_compress_static.argtypes = [vp, vp, vp, vp, sz, vp, i, f, f, ctypes.POINTER(_MessageStruct), vp]
     lib.vgc_compress_static.restype = i
+    lib.vgc_step_host.argtypes = [ctypes.POINTER(_LayerHostStruct), i, vp, vp, vp, vp, vp, sz, vp, i, f, f, f,
+                                  ctypes.POINTER(_MessageStruct), vp, vp, vp, sz, vp, sz, vp]
+    lib.vgc_step_host.restype = i
     lib.vgc_decode_accumulate.argtypes = [ctypes.POINTER(_ViewStruct), i, vp, i, f, vp, sz, vp, vp]
     lib.vgc_decode_accumulate.restype = i
     _lib = lib
@@ -274,6 +284,40 @@ def vgc_decode_accumulate(messages: Sequence, group_offsets, scale: float, u, de
                                               _dev(dev_status, torch.int32, "dev_status"), _stream(stream))
     _check(st, "vgc_decode_accumulate")
     return u
+
+
+def _host(t: torch.Tensor, dtype, name: str) -> int:
+    if not isinstance(t, torch.Tensor) or t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"{name} must be a contiguous CPU tensor of {dtype}")
+    return t.data_ptr()
+
+
+def vgc_step_host(layers, g_host, g_dev, s_dev, r, v, group_offsets, alpha, zeta, scale, out: MessageBuffers,
+                  words_host, counters_host, ws_sqgrad, ws_compress, stream=None):
+    """One worker step from host buffers.  ``layers``: list of dicts with keys is_conv, B, C, H, W, Cout,
+    Kh, Kw, stride, pad, x_host, delta_host (CPU, ideally pinned) and x_dev, delta_dev (CUDA staging).
+    Returns (nnz, n_criterion, n_dropped, dev_status) as read back into ``counters_host``."""
+    arr = (_LayerHostStruct * max(len(layers), 1))()
+    for k, L in enumerate(layers):
+        arr[k] = _LayerHostStruct(int(L["is_conv"]), L["B"], L["C"], L.get("H", 1), L.get("W", 1), L["Cout"],
+                                  L.get("Kh", 1), L.get("Kw", 1), L.get("stride", 1), L.get("stride", 1),
+                                  L.get("pad", 0), L.get("pad", 0),
+                                  _host(L["x_host"], torch.float32, "x_host"), _host(L["delta_host"], torch.float32, "delta_host"),
+                                  _dev(L["x_dev"], torch.float32, "x_dev"), _dev(L["delta_dev"], torch.float32, "delta_dev"))
+    n = g_dev.numel()
+    K = group_offsets.numel() - 1
+    wsp, wsb = _ws(ws_sqgrad)
+    wcp, wcb = _ws(ws_compress)
+    msg = out.struct()
+    st = load_library().vgc_step_host(arr, len(layers), _host(g_host, torch.float32, "g_host"),
+                                      _dev(g_dev, torch.float32, "g_dev"), _dev(s_dev, torch.float32, "s_dev"),
+                                      _dev(r, torch.float32, "r"), _dev(v, torch.float32, "v"), n,
+                                      _dev(group_offsets, torch.int32, "group_offsets"), K, float(alpha), float(zeta),
+                                      float(scale), ctypes.byref(msg), _host(words_host, torch.int32, "words_host"),
+                                      _host(counters_host, torch.int32, "counters_host"), wsp, wsb, wcp, wcb,
+                                      _stream(stream))
+    _check(st, "vgc_step_host")
+    return tuple(int(c) & 0xFFFFFFFF for c in counters_host.tolist())
 
 
 def offsets_tensor(offsets, device="cuda") -> torch.Tensor:

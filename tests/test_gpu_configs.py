@@ -1,0 +1,230 @@
+"""GPU parity on the five benchmark configurations at their stated sizes, through the C ABI.
+
+Squared-gradient sums: relative 1e-5 (whole matrices where the oracle finishes in seconds, sampled entries
+otherwise).  Compressor: bit-exact in lock-step -- at every step the GPU-produced (g, s) bytes are copied to
+the host and fed to the oracle, so both state machines stay identical by induction.  Decoder: absolute 1e-6."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1802_06058_b200 as vgc
+from paper_1802_06058_b200 import workloads
+from gpu_harness import GpuCompressor, OracleCompressor, assert_same_message, assert_same_state
+
+pytestmark = pytest.mark.gpu
+F32 = np.float32
+ZETA = 0.999
+
+
+def _zeros_ws(nbytes):
+    return torch.zeros(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+
+
+def sqgrad_layer(spec, x, delta, scale, S, ws):
+    if spec.kind == "conv":
+        vgc.vgc_sqgrad_conv(x, delta, (spec.k, spec.k), (spec.stride, spec.stride), (spec.pad, spec.pad), scale, S, ws=ws)
+    else:
+        vgc.vgc_sqgrad_linear(x, delta, scale, S, ws=ws)
+
+
+def layer_ws(layers, B):
+    need = 256
+    for spec in layers:
+        if spec.kind == "conv":
+            need = max(need, vgc.vgc_sqgrad_conv_workspace_bytes(B, spec.cin, spec.hin, spec.hin, spec.cout, spec.k,
+                                                                 spec.k, spec.stride, spec.stride, spec.pad, spec.pad))
+        else:
+            need = max(need, vgc.vgc_sqgrad_linear_workspace_bytes(B, spec.cin, spec.cout))
+    return _zeros_ws(need)
+
+
+def assert_close_rel(got, want, rtol=1e-5):
+    want64 = want.astype(np.float64)
+    err = np.abs(got.astype(np.float64) - want64)
+    assert np.all(err <= rtol * np.abs(want64)), float((err / np.maximum(np.abs(want64), 1e-300)).max())
+
+
+def run_dense_pipeline(layers, B, x_kind, delta_std, cfg, worker, steps, alpha, check_sqgrad_every=1):
+    """sqgrad per layer + compress for `steps` steps; returns the GPU compressor (its `out` holds the last message)
+    and the oracle's last message."""
+    offs = workloads.group_offsets(layers)
+    n = int(offs[-1])
+    gpu, cpu = GpuCompressor(n, offs), OracleCompressor(n, offs)
+    s = torch.empty(n, device="cuda")
+    ws = layer_ws(layers, B)
+    scale = 1.0 / (B * B)
+    want = None
+    for t in range(steps):
+        g_parts = []
+        for li, spec in enumerate(layers):
+            x, d = workloads.layer_inputs(spec, B, cfg, worker, t, li, x_kind, delta_std, "cuda")
+            S = s[int(offs[li]):int(offs[li + 1])]
+            sqgrad_layer(spec, x, d, scale, S, ws)
+            g_parts.append(workloads.mean_gradient(spec, x, d))
+            if t % check_sqgrad_every == 0:
+                ref = oracle.sqgrad_linear(x.cpu().numpy(), d.cpu().numpy(), scale=scale)
+                assert_close_rel(S.cpu().numpy().reshape(ref.shape), ref)
+        assert int(ws[:4].view(torch.int32).item()) == 0
+        g = torch.cat(g_parts)
+        got = gpu.step(g, s, alpha, ZETA)
+        want = cpu.step(g.cpu().numpy(), s.cpu().numpy(), alpha, ZETA)
+        assert_same_message(got, want)
+        assert_same_state(gpu, cpu)
+    return gpu, want, offs
+
+
+def decode_and_check(comps, cpu_msgs, offs, n, scale):
+    u = torch.zeros(n, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    vgc.vgc_decode_accumulate([c.out for c in comps], comps[0].offs_dev, scale, u, status)
+    ref = np.zeros(n, F32)
+    oracle.decode_accumulate(cpu_msgs, offs, scale, ref)
+    assert int(status.item()) == 0
+    assert np.abs(u.cpu().numpy().astype(np.float64) - ref).max() <= 1e-6
+
+
+def test_config1_dense_layer_10_steps_then_decode_4_messages():
+    layers, B, W = workloads.dense_layers(), 32, 4
+    comps, msgs = [], []
+    for w in range(W):
+        gpu, want, offs = run_dense_pipeline(layers, B, "normal", 1e-2, cfg=0, worker=w, steps=10, alpha=2.0)
+        comps.append(gpu); msgs.append((want.words, want.group_exp))
+        assert want.nnz > 0
+    decode_and_check(comps, msgs, offs, 32768, 1.0)
+
+
+def test_config2_mlp_100_steps_then_decode_8_messages():
+    layers, B, W = workloads.mlp_layers(), 128, 8
+    comps, msgs = [], []
+    for w in range(W):
+        # worker 0 runs the full 100 steps (sqgrad checked every 10th step), the others 3 steps each
+        steps = 100 if w == 0 else 3
+        gpu, want, offs = run_dense_pipeline(layers, B, "relu_normal", 1e-3, cfg=1, worker=w, steps=steps, alpha=2.0,
+                                             check_sqgrad_every=10)
+        comps.append(gpu); msgs.append((want.words, want.group_exp))
+    assert int(offs[-1]) == 1861632
+    decode_and_check(comps, msgs, offs, 1861632, 1.0 / W)
+
+
+def test_config3_resnet50_sampled_sqgrad_and_alpha_sweep():
+    layers, B = workloads.resnet50_layers(), 32
+    offs = workloads.group_offsets(layers)
+    n = int(offs[-1])
+    assert n == 25502912 and len(layers) == 54
+    s = torch.empty(n, device="cuda")
+    ws = layer_ws(layers, B)
+    scale = 1.0 / (B * B)
+    rng = np.random.default_rng(3)
+    for li, spec in enumerate(layers):
+        x, d = workloads.layer_inputs(spec, B, 2, 0, 0, li, "half_normal", 1e-4, "cuda")
+        S = s[int(offs[li]):int(offs[li + 1])]
+        sqgrad_layer(spec, x, d, scale, S, ws)
+        idx = np.unique(np.concatenate([rng.integers(0, spec.n_params, 24), [0, spec.n_params - 1]]))
+        got = S.cpu().numpy()[idx]
+        if spec.kind == "conv":
+            ref = oracle.sqgrad_conv_entries(x.cpu().numpy(), d.cpu().numpy(), (spec.k, spec.k), (spec.stride, spec.stride),
+                                             (spec.pad, spec.pad), scale, idx)
+        else:
+            ref = oracle.sqgrad_linear(x.cpu().numpy(), d.cpu().numpy(), scale=scale).reshape(-1)[idx]
+        assert_close_rel(got, ref)
+        del x, d
+    assert int(ws[:4].view(torch.int32).item()) == 0
+    assert bool((s >= 0).all())
+    # compress over the whole flat buffer for three steps, alpha sweep; g is a noise draw with variance s
+    root_s = s.sqrt()
+    for alpha in (1.0, 2.0, 4.0):
+        gpu, cpu = GpuCompressor(n, offs, with_mask=False), OracleCompressor(n, offs)
+        s_host = s.cpu().numpy()
+        for t in range(3):
+            gen = torch.Generator(device="cuda"); gen.manual_seed(workloads.seed_for(2, 0, t, 0, 3))
+            g = torch.empty(n, device="cuda").normal_(generator=gen).mul_(root_s)
+            got = gpu.step(g, s, alpha, ZETA)
+            want = cpu.step(g.cpu().numpy(), s_host, alpha, ZETA, want_mask=False)
+            assert_same_message(got, want, check_mask=False)
+        assert_same_state(gpu, cpu)
+        density = want.n_criterion / n
+        assert 0.005 < density < 0.5
+
+
+def test_config4_vgg16_flat_buffer_compress_only():
+    layers = workloads.vgg16_layers()
+    offs = workloads.group_offsets(layers)
+    n = int(offs[-1])
+    assert n == 138344128 and len(layers) == 16
+    gpu, cpu = GpuCompressor(n, offs, with_mask=False), OracleCompressor(n, offs)
+    for t in range(2):
+        g, s = workloads.per_parameter_gs(n, 64, 1e-4, workloads.seed_for(3, 0, t, 0, 2), "cuda")
+        got = gpu.step(g, s, 2.0, ZETA)
+        want = cpu.step(g.cpu().numpy(), s.cpu().numpy(), 2.0, ZETA, want_mask=False)
+        assert_same_message(got, want, check_mask=False)
+        del g, s
+    assert_same_state(gpu, cpu)
+
+
+@pytest.mark.parametrize("net,W,density", [("resnet50", 4, 1e-4), ("resnet50", 16, 1e-3), ("resnet50", 64, 1e-2),
+                                           ("vgg16", 4, 1e-2), ("vgg16", 64, 1e-3)])
+def test_config5_decode_sweep(net, W, density):
+    layers = workloads.resnet50_layers() if net == "resnet50" else workloads.vgg16_layers()
+    offs = workloads.group_offsets(layers)
+    n = int(offs[-1])
+    offs_dev = vgc.offsets_tensor(offs)
+    msgs = [workloads.random_message(n, offs, density, workloads.seed_for(4, w, 0, 0, 2), "cuda") for w in range(W)]
+    counts = [torch.tensor([m[0].numel()], dtype=torch.int32, device="cuda") for m in msgs]
+    u = torch.zeros(n, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    vgc.vgc_decode_accumulate([(m[0], c, m[1]) for m, c in zip(msgs, counts)], offs_dev, 1.0 / W, u, status)
+    ref = np.zeros(n, F32)
+    oracle.decode_accumulate([(m[0].cpu().numpy().view(np.uint32), m[1].cpu().numpy()) for m in msgs], offs, 1.0 / W, ref)
+    assert int(status.item()) == 0
+    assert np.abs(u.cpu().numpy().astype(np.float64) - ref).max() <= 1e-6
+
+
+def test_config5_max_contention_all_messages_share_one_index_set():
+    layers = workloads.resnet50_layers()
+    offs = workloads.group_offsets(layers)
+    n, W = int(offs[-1]), 16
+    mask = torch.empty(n, device="cuda").uniform_(generator=torch.Generator(device="cuda").manual_seed(5)) < 1e-3
+    msgs = [workloads.random_message(n, offs, 1e-3, workloads.seed_for(4, w, 1, 0, 2), "cuda", index_mask=mask)
+            for w in range(W)]
+    counts = [torch.tensor([m[0].numel()], dtype=torch.int32, device="cuda") for m in msgs]
+    u = torch.zeros(n, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    vgc.vgc_decode_accumulate([(m[0], c, m[1]) for m, c in zip(msgs, counts)], vgc.offsets_tensor(offs), 1.0, u, status)
+    ref = np.zeros(n, F32)
+    oracle.decode_accumulate([(m[0].cpu().numpy().view(np.uint32), m[1].cpu().numpy()) for m in msgs], offs, 1.0, ref)
+    assert np.abs(u.cpu().numpy().astype(np.float64) - ref).max() <= 1e-6
+
+
+def test_step_host_matches_device_path():
+    """vgc_step_host (inputs in pinned host memory, message read back) against the device-pointer calls."""
+    layers, B = workloads.mlp_layers(), 128
+    offs = workloads.group_offsets(layers)
+    n, K = int(offs[-1]), len(layers)
+    scale = 1.0 / (B * B)
+    ws_s, ws_c = layer_ws(layers, B), torch.empty(vgc.vgc_compress_workspace_bytes(n, K), dtype=torch.uint8, device="cuda")
+    offs_dev = vgc.offsets_tensor(offs)
+    dev_inputs = [workloads.layer_inputs(spec, B, 1, 0, 0, li, "relu_normal", 1e-3, "cuda") for li, spec in enumerate(layers)]
+    g = torch.cat([workloads.mean_gradient(spec, x, d) for spec, (x, d) in zip(layers, dev_inputs)])
+    # device path
+    s = torch.empty(n, device="cuda"); r = torch.zeros(n, device="cuda"); v = torch.zeros(n, device="cuda")
+    for li, (spec, (x, d)) in enumerate(zip(layers, dev_inputs)):
+        sqgrad_layer(spec, x, d, scale, s[int(offs[li]):int(offs[li + 1])], ws_s)
+    out = vgc.MessageBuffers(n, K, n)
+    vgc.vgc_compress(g, s, r, v, offs_dev, 2.0, ZETA, out, ws_c)
+    want = out.read()
+    # host path
+    host_layers = []
+    for spec, (x, d) in zip(layers, dev_inputs):
+        host_layers.append({"is_conv": False, "B": B, "C": spec.cin, "Cout": spec.cout,
+                            "x_host": x.cpu().pin_memory(), "delta_host": d.cpu().pin_memory(),
+                            "x_dev": torch.empty_like(x), "delta_dev": torch.empty_like(d)})
+    s2 = torch.empty(n, device="cuda"); r2 = torch.zeros(n, device="cuda"); v2 = torch.zeros(n, device="cuda")
+    out2 = vgc.MessageBuffers(n, K, n)
+    words_host = torch.zeros(n, dtype=torch.int32).pin_memory()
+    counters_host = torch.zeros(4, dtype=torch.int32).pin_memory()
+    nnz, n_crit, n_drop, status = vgc.vgc_step_host(host_layers, g.cpu().pin_memory(), torch.empty(n, device="cuda"), s2, r2, v2,
+                                                    offs_dev, 2.0, ZETA, scale, out2, words_host, counters_host, ws_s, ws_c)
+    assert status == 0 and (nnz, n_crit, n_drop) == (want["nnz"], want["n_criterion"], want["n_dropped"])
+    assert np.array_equal(words_host[:nnz].numpy().view(np.uint32), want["words"])
+    assert torch.equal(r, r2) and torch.equal(v, v2) and torch.equal(s, s2)
