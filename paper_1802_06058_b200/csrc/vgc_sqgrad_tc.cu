@@ -86,6 +86,8 @@ struct Params {
     int accumulate;
     const float *x, *delta;  // raw operands (gathered tiles)
     int C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, Wo, P;     // conv geometry (gathered tiles)
+    int chw;                 // C*H*W
+    unsigned wo_magic;       // floor(2^32 / Wo) + 1: p / Wo == umulhi(p, wo_magic) for p * Wo < 2^32
     float *S;                // result: element (m, n) lives at S[m*ld_m + n*ld_n]; one of the two is 1
     long long ld_m, ld_n;
     float *partial;          // split-K scratch [split][tile][column][row], used when gridDim.z > 1
@@ -242,7 +244,6 @@ __host__ __device__ constexpr uint32_t instr_desc(int major, int n)
            ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
 }
 
-// ---- the kernel ------------------------------------------------------------------------------
 // One 16-byte chunk (4 consecutive k of one row) of a K-major 128-byte-swizzled tile.
 __device__ __forceinline__ uint32_t chunk_offset(int row, int kq) { return (uint32_t)row * 128u + (uint32_t)((kq ^ (row & 7)) << 4); }
 
@@ -285,36 +286,36 @@ struct GatherRows {
                 dw[i] = kw - prm.pw;
                 base[i] = (c * prm.H + dh[i]) * prm.W + dw[i];
             } else {
-                base[i] = ii;           // output channel
+                base[i] = ii * prm.P;   // offset of the output channel's plane
                 dh[i] = dw[i] = 0;
             }
         }
     }
-    // loads this thread's 4 x 4 elements of the slice at (z, pbase .. pbase+3)
-    __device__ __forceinline__ void load(const Params &prm, int z, int pbase, const int (&ho)[4], const int (&wo)[4],
-                                         float (&v)[kRowsPerThread][4]) const
+    // loads this thread's 4 rows x 4 consecutive k: example z, output positions pbase .. pbase+3
+    __device__ __forceinline__ void load(const Params &prm, int z, int pbase, float (&v)[kRowsPerThread][4]) const
     {
         if (kMode == kGatherIm2col) {
-            const float *xz = prm.x + (size_t)z * prm.C * prm.H * prm.W;
+            const float *xz = prm.x + (size_t)z * prm.chw;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const bool pv = pbase + j < prm.P;
-                const int hs = ho[j] * prm.sh, ws = wo[j] * prm.sw;
-                const int poff = hs * prm.W + ws;
+                const int p = pbase + j;
+                const int ho = prm.Wo == 1 ? p : (int)__umulhi((unsigned)p, prm.wo_magic), wo = p - ho * prm.Wo;
+                const int hs = ho * prm.sh, ws = wo * prm.sw;
+                const float *xp = xz + (hs * prm.W + ws);
+                const bool pv = p < prm.P;
 #pragma unroll
                 for (int i = 0; i < kRowsPerThread; ++i) {
                     const bool in = pv && ok[i] && (unsigned)(hs + dh[i]) < (unsigned)prm.H &&
                                     (unsigned)(ws + dw[i]) < (unsigned)prm.W;
-                    v[i][j] = in ? __ldg(xz + (base[i] + poff)) : 0.f;
+                    v[i][j] = in ? __ldg(xp + base[i]) : 0.f;
                 }
             }
         } else if (kMode == kGatherErr) {
+            const float *dz = prm.delta + (size_t)z * prm.Cout * prm.P + pbase;
 #pragma unroll
-            for (int i = 0; i < kRowsPerThread; ++i) {
-                const float *dr = prm.delta + ((size_t)z * prm.Cout + base[i]) * prm.P + pbase;
+            for (int i = 0; i < kRowsPerThread; ++i)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) v[i][j] = (ok[i] && pbase + j < prm.P) ? __ldg(dr + j) : 0.f;
-            }
+                for (int j = 0; j < 4; ++j) v[i][j] = (ok[i] && pbase + j < prm.P) ? __ldg(dz + (base[i] + j)) : 0.f;
         }
     }
 };
@@ -482,46 +483,20 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         GatherRows<kModeB> rows_b;
         rows_a.init(prm, m0 + row0, prm.M);
         rows_b.init(prm, n0 + row0, prm.N);
-        int ho[4] = {0, 0, 0, 0}, wo[4] = {0, 0, 0, 0};                    // output position of this thread's four k
-        int ho_init[4], wo_init[4];
-        int q32 = 0, r32 = 0, z = 0, pblk = 0;
+        // where the current slice sits: example z, 32-wide block pblk of that example's output positions
+        int z = 0, pblk = 0;
         if (kAnyGather) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                ho_init[j] = (kq * 4 + j) / prm.Wo;
-                wo_init[j] = (kq * 4 + j) - ho_init[j] * prm.Wo;
-            }
-            q32 = kBK / prm.Wo;
-            r32 = kBK - q32 * prm.Wo;
             z = slice_begin / prm.p_slices;
             pblk = slice_begin - z * prm.p_slices;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int p = pblk * kBK + kq * 4 + j;
-                ho[j] = p / prm.Wo;
-                wo[j] = p - ho[j] * prm.Wo;
-            }
         }
         auto advance = [&]() {
-            if (++pblk == prm.p_slices) {
-                pblk = 0;
-                ++z;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) { ho[j] = ho_init[j]; wo[j] = wo_init[j]; }
-            } else {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    ho[j] += q32;
-                    wo[j] += r32;
-                    if (wo[j] >= prm.Wo) { wo[j] -= prm.Wo; ++ho[j]; }
-                }
-            }
+            if (++pblk == prm.p_slices) { pblk = 0; ++z; }
         };
         auto gather = [&](float (&ga)[kRowsPerThread][4], float (&gb)[kRowsPerThread][4]) {
-            const int pbase = pblk * kBK + kq * 4;
             if (prm.debug & 4) return;
-            rows_a.load(prm, z, pbase, ho, wo, ga);
-            rows_b.load(prm, z, pbase, ho, wo, gb);
+            const int pbase = pblk * kBK + kq * 4;
+            rows_a.load(prm, z, pbase, ga);
+            rows_b.load(prm, z, pbase, gb);
         };
         // transform of slice i; gathered elements come in registers, TMA tiles from the raw stage
         auto process = [&](int i, const float (&ga)[kRowsPerThread][4], const float (&gb)[kRowsPerThread][4]) -> bool {
@@ -890,12 +865,13 @@ vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int 
                           void *ws, size_t ws_bytes, cudaStream_t st)
 {
     const int P = Ho * Wo, n_im2col = C * Kh * Kw;
-    const int p_slices = (P + kBK - 1) / kBK;
     static const int force_gather = getenv("VGC_TC_GATHER") ? atoi(getenv("VGC_TC_GATHER")) : 0;   // experiments
     const bool err_tma = P >= kBK && P % 4 == 0 && !(force_gather & 1);
     const bool in_tma = P >= kBK && P % 4 == 0 && !(force_gather & 2) && Kh == 1 && Kw == 1 && sh == 1 && sw == 1 &&
                         ph == 0 && pw == 0;
     static const bool a_tmem = !(getenv("VGC_TC_ATMEM") && atoi(getenv("VGC_TC_ATMEM")) == 0);   // experiments
+    const int p_slices = (P + kBK - 1) / kBK;
+    const int k_slices = B * p_slices;
     const bool swapped = conv_swapped(Cout, n_im2col);
     const int rows_err = swapped ? kBN : kBM, rows_in = swapped ? kBM : kBN;     // tile heights
     CUtensorMap m_err = {}, m_in = {};
@@ -919,7 +895,8 @@ vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int 
     prm.x = x; prm.delta = delta;
     prm.C = C; prm.H = H; prm.W = W; prm.Cout = Cout; prm.Kh = Kh; prm.Kw = Kw; prm.sh = sh; prm.sw = sw;
     prm.ph = ph; prm.pw = pw; prm.Wo = Wo; prm.P = P;
-    const int k_slices = B * p_slices;
+    prm.chw = C * H * W;
+    prm.wo_magic = (unsigned)(0x100000000ull / (unsigned)Wo) + 1u;
     const int e = err_tma ? kTma : kGatherErr, i = in_tma ? kTma : kGatherIm2col;
     KernelFn fn = nullptr;
     if (!swapped) {     // S[o][idx]: m = o, n = idx
