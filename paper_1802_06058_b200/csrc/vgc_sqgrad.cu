@@ -27,12 +27,8 @@ namespace {
 // VGC_SQGRAD_PATH=simt forces the CUDA-core kernel (cross-checks, shapes under suspicion)
 bool use_tensor_cores()
 {
-    static int v = -1;
-    if (v < 0) {
-        const char *e = getenv("VGC_SQGRAD_PATH");
-        v = (e && e[0] == 's') ? 0 : 1;
-    }
-    return v == 1;
+    const char *e = getenv("VGC_SQGRAD_PATH");
+    return !(e && e[0] == 's');
 }
 
 bool conv_shape_ok(int B, int C, int H, int W, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw,

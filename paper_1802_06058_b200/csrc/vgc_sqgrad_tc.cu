@@ -92,8 +92,6 @@ struct Params {
     long long ld_m, ld_n;
     float *partial;          // split-K scratch [split][tile][column][row], used when gridDim.z > 1
     uint32_t *status;        // device word; VGC_DEV_TIMEOUT is OR-ed in if a wait expired
-    int prefetch;            // slices ahead of the TMA loads that are prefetched into L2 (0: off)
-    int debug;               // experiments: 1 skip MMAs, 2 skip transform math, 4 skip gathers
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -153,13 +151,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
-}
-
-// L2 prefetch of a tile that a later TMA load will fetch (no shared memory, no barrier involved)
-__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap *map, int c0, int c1, int c2)
-{
-    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(c0), "r"(c1), "r"(c2)
-                 : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -395,12 +386,6 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                     const int z = slice / prm.p_slices, p0 = (slice - z * prm.p_slices) * kBK;
                     if (!kGatherA) tma_load_3d(dst_a, &map_a, full, p0, m0, z);
                     if (!kGatherB) tma_load_3d(dst_b, &map_b, full, p0, n0, z);
-                    if (prm.prefetch > 0 && i + prm.prefetch < n_slices) {      // warm L2 for a slice further ahead
-                        const int sl = slice + prm.prefetch;
-                        const int zp = sl / prm.p_slices, pp = (sl - zp * prm.p_slices) * kBK;
-                        if (!kGatherA) tma_prefetch_3d(&map_a, pp, m0, zp);
-                        if (!kGatherB) tma_prefetch_3d(&map_b, pp, n0, zp);
-                    }
                 } else {
                     const int k0 = slice * kBK;
 #pragma unroll
@@ -449,7 +434,6 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                     const uint32_t ta_hi = tmem_base + 2 * kBN + ls * kTmemColsA, ta_lo = ta_hi + 32;
 #pragma unroll
                     for (int kk = 0; kk < kBK / 8; ++kk) {
-                        if (prm.debug & 1) break;
                         const uint64_t db_hi = smem_desc(hi_b + kk * k_step, lbo, sbo, layout);
                         const uint64_t db_lo = smem_desc(lo_b + kk * k_step, lbo, sbo, layout);
                         if (kATmem) {
@@ -493,7 +477,6 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             if (++pblk == prm.p_slices) { pblk = 0; ++z; }
         };
         auto gather = [&](float (&ga)[kRowsPerThread][4], float (&gb)[kRowsPerThread][4]) {
-            if (prm.debug & 4) return;
             const int pbase = pblk * kBK + kq * 4;
             rows_a.load(prm, z, pbase, ga);
             rows_b.load(prm, z, pbase, gb);
@@ -512,11 +495,6 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             // lo tiles: [A lo][B lo], or the B tile alone when A lives in tensor memory (then `lo` points
             // one A tile below the slot so that the same chunk offsets address the B part)
             uint8_t *lo = smem_gen + kLoBase + ls * kLoBytes - (kATmem ? kRawBytesA : 0);
-            if (prm.debug & 2) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&op_full[st]));
-                return true;
-            }
             if (kATmem) {
                 // A: this thread's row (TMEM lane) and half of the slice's 32 k -> hi / lo straight into TMEM
                 tc_fence_after();
@@ -541,7 +519,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                 tc_st_32x16(taddr, h16);
                 tc_st_32x16(taddr + 32, l16);
             }
-            if (kAnyTma && !(prm.debug & 8)) {      // tiles that came by TMA: elementwise, in place, over their 16-byte chunks
+            if (kAnyTma) {      // tiles that came by TMA: elementwise, in place, over their 16-byte chunks
                 constexpr uint32_t c_begin = (kGatherA || kATmem) ? kRawBytesA / 16 : 0;
                 constexpr uint32_t c_end = kGatherB ? kRawBytesA / 16 : kRawStageBytes / 16;
                 constexpr int kPerThread = c_end > c_begin ? (c_end - c_begin) / kTransformThreads : 1;
@@ -567,7 +545,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                                 gb[r][2], gb[r][3]);
             }
             if (kATmem) { tc_wait_st(); tc_fence_before(); }      // TMEM stores complete and ordered before the signal
-            if (!(prm.debug & 32)) fence_async_smem();            // generic-proxy writes -> tensor core reads
+            fence_async_smem();                                   // generic-proxy writes -> tensor core reads
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&op_full[st]));
             return true;
@@ -816,8 +794,6 @@ static vgc_status tc_launch(KernelFn kernel, const CUtensorMap &ma, const CUtens
     }
     prm.M = M; prm.N = N; prm.k_slices = k_slices; prm.slices_per_split = plan.slices_per_split;
     prm.chunk = default_chunk();
-    { static const int pf = getenv("VGC_TC_PREFETCH") ? atoi(getenv("VGC_TC_PREFETCH")) : 0; prm.prefetch = pf; }
-    { static const int dbg = getenv("VGC_TC_DEBUG") ? atoi(getenv("VGC_TC_DEBUG")) : 0; prm.debug = dbg; }
     prm.status = static_cast<uint32_t *>(ws);
     prm.partial = reinterpret_cast<float *>(static_cast<char *>(ws) + 256);
     dim3 grid(plan.tiles_x, plan.tiles_y, plan.splits);
@@ -865,11 +841,14 @@ vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int 
                           void *ws, size_t ws_bytes, cudaStream_t st)
 {
     const int P = Ho * Wo, n_im2col = C * Kh * Kw;
-    static const int force_gather = getenv("VGC_TC_GATHER") ? atoi(getenv("VGC_TC_GATHER")) : 0;   // experiments
+    // VGC_TC_GATHER (bit 0: error tile, bit 1: input tile) forces the gathered form of a tile and
+    // VGC_TC_ATMEM=0 keeps the A operand in shared memory: every variant computes the same thing, the
+    // switches exist so that tests can reach each of them on any shape.
+    const int force_gather = getenv("VGC_TC_GATHER") ? atoi(getenv("VGC_TC_GATHER")) : 0;
     const bool err_tma = P >= kBK && P % 4 == 0 && !(force_gather & 1);
     const bool in_tma = P >= kBK && P % 4 == 0 && !(force_gather & 2) && Kh == 1 && Kw == 1 && sh == 1 && sw == 1 &&
                         ph == 0 && pw == 0;
-    static const bool a_tmem = !(getenv("VGC_TC_ATMEM") && atoi(getenv("VGC_TC_ATMEM")) == 0);   // experiments
+    const bool a_tmem = !(getenv("VGC_TC_ATMEM") && atoi(getenv("VGC_TC_ATMEM")) == 0);
     const int p_slices = (P + kBK - 1) / kBK;
     const int k_slices = B * p_slices;
     const bool swapped = conv_swapped(Cout, n_im2col);

@@ -113,3 +113,21 @@ def test_long_reduction_all_ones_is_exact():
     x = torch.ones(2, 8, 224, 224, device="cuda"); d = torch.ones(2, 16, 224, 224, device="cuda")
     got = run_conv(x, d, 1, 1, 0, 1.0)                      # tensor-core path
     assert np.all(got == 2 * 224 * 224)
+
+
+@pytest.mark.parametrize("env", [{"VGC_TC_ATMEM": "0"}, {"VGC_TC_GATHER": "1"}, {"VGC_TC_GATHER": "2"},
+                                 {"VGC_TC_GATHER": "3"}, {"VGC_SQGRAD_PATH": "simt"}])
+@pytest.mark.parametrize("B,C,H,Cout,k,s,p", [(3, 96, 12, 160, 1, 1, 0), (2, 40, 12, 48, 3, 1, 1), (2, 72, 16, 200, 3, 2, 1)])
+def test_every_kernel_variant_gives_the_same_statistic(monkeypatch, env, B, C, H, Cout, k, s, p):
+    """The library picks a kernel form per layer (TMA or gathered tiles, A operand in shared or tensor memory,
+    roles swapped for few output channels, CUDA-core kernel); the switches force each form on shapes that would
+    otherwise take another one."""
+    for key, val in env.items():
+        monkeypatch.setenv(key, val)
+    gen = torch.Generator(device="cuda"); gen.manual_seed(C + H)
+    Ho = (H + 2 * p - k) // s + 1
+    x = torch.randn(B, C, H, H, device="cuda", generator=gen).abs_()
+    d = torch.randn(B, Cout, Ho, Ho, device="cuda", generator=gen) * 1e-4
+    got = run_conv(x, d, k, s, p, 0.5)
+    want = oracle.sqgrad_conv(x.cpu().numpy(), d.cpu().numpy(), (k, k), (s, s), (p, p), scale=0.5)
+    _check(got, want)
