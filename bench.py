@@ -586,22 +586,30 @@ def main():
         "send_density": nnz_a / n, "nnz": nnz, "n_dropped": counters["n_dropped"], "sum_nnz_decoded": sum_nnz,
         "dev_status": counters["dev_status"],
     }
+    # DRAM traffic measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum), per launch group:
+    # profiles/sqgrad_tc_resnet50_pass.md (one pass over the 54 ResNet-50 layers) and
+    # profiles/compress_flat_n33554432.md (scaled by n: the traffic is proportional to the buffer length)
+    NCU_SQGRAD_PASS_BYTES_RESNET50 = 3.21e9
+    NCU_COMPRESS_BYTES_PER_PARAM = (537.7e6 + 233.9e6 + 20.7e6 + 20.7e6) / 33554432
+    compress_roofline = {"kernel": "compress_phase_a + compress_count + compress_emit", "bound": "hbm",
+                         "achieved": compress_bytes / (co_ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                         "frac": compress_bytes / (co_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+                         "traffic": NCU_COMPRESS_BYTES_PER_PARAM * n,
+                         "algorithmic_bytes": compress_bytes, "peak_source": f"{pk['source']} copy bandwidth, of measured"}
     # dominant kernel of the step
     if sq_ms >= co_ms + de_ms and hp.flops_useful:
         tf32_peak = pk["bf16_tflops_sustained"] / 2.0          # nominal tf32 : bf16 ratio is 1 : 2
         ach = hp.flops_useful / (sq_ms * 1e-3) / 1e12
         roofline = {"kernel": "sqgrad_tc (all layers of one step)", "bound": "tensor", "achieved": ach,
-                    "peak": tf32_peak, "unit": "TFLOP/s", "frac": ach / tf32_peak, "traffic": None,
+                    "peak": tf32_peak, "unit": "TFLOP/s", "frac": ach / tf32_peak,
+                    "traffic": NCU_SQGRAD_PASS_BYTES_RESNET50 if args.workload == "resnet50" else None,
                     "issued_tflops": 3 * ach, "issued_frac": 3 * ach / tf32_peak,
-                    "peak_source": f"{pk['source']} bf16 sustained x 1/2 (tf32 nominal ratio)",
+                    "peak_source": f"{pk['source']} bf16 sustained x 1/2 (tf32 nominal ratio), of measured",
                     "note": "achieved = algorithmic flops 2*M*N*K per layer / sqgrad time; the 3xTF32 scheme "
-                            "issues 3 tensor-core products per algorithmic one (issued_frac = tensor-pipe load)"}
+                            "issues 3 tensor-core products per algorithmic one (issued_frac = tensor-pipe load); "
+                            "traffic = DRAM bytes of the 103 launches of one pass"}
     else:
-        ach = compress_bytes / (co_ms * 1e-3) / 1e9
-        roofline = {"kernel": "compress_phase_a+b", "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"],
-                    "unit": "GB/s", "frac": ach / pk["hbm_gbs"], "traffic": None,
-                    "peak_source": f"{pk['source']} copy bandwidth"}
-
+        roofline = compress_roofline
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32 (tf32x3 products where tensor cores are used)",
@@ -610,7 +618,8 @@ def main():
                        "zeta": ZETA, "groups": hp.K, "launch": "eager" if args.no_graph else "cuda graph replay",
                        "sqgrad_streams": getattr(hp, "n_streams", 1),
                        "l2": "inputs larger than L2 (no flush)" if n * 16 > 126e6 else "state fits in L2 (no flush): cache-resident numbers"},
-            "gpu_launches": int(launches), "clocks": clocks, "sections": sections, "roofline": roofline}
+            "gpu_launches": int(launches), "clocks": clocks, "sections": sections, "roofline": roofline,
+            "roofline_compress": compress_roofline}
 
     if not args.no_e2e:
         e2e_ms, h2d, d2h = run_e2e(hp, min(args.steps, 5), 1)
