@@ -181,7 +181,8 @@ vgc_status vgc_compress_static(const float *g, const float *s, float *r, float *
  * after an allgatherv); scale = 1/W gives the mean.  Additions into one element may happen in any
  * order (fp32 atomics), so results match a sequential sum to rounding only.
  *
- *   msgs   HOST array of W views; each view holds DEVICE pointers; the word count is read on the device
+ *   msgs   HOST array of W views; each view holds DEVICE pointers; the word count is read on the device.
+ *          Words must be in ascending index order, as vgc_compress emits them.
  *   u      [n] fp32, accumulated in place (the caller zeroes it when a fresh sum is wanted)
  * Words whose index is >= n are skipped and VGC_DEV_RANGE is set.  W == 0 or n == 0: no-op, OK.
  * ------------------------------------------------------------------------------------------- */

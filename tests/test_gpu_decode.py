@@ -89,3 +89,15 @@ def test_round_trip_of_compressed_messages():
     oracle.decode_accumulate(cpu_msgs, offs, 1.0 / W, want)
     assert int(status.item()) == 0
     assert np.abs(u.cpu().numpy().astype(np.float64) - want).max() <= ATOL
+
+
+def test_scatter_form_agrees_with_the_default_merge_form(monkeypatch):
+    n, W = 400003, 5
+    offs = random_offsets(np.random.default_rng(21), n, 9)
+    msgs = [workloads.random_message(n, offs, 0.15 if w % 2 else 0.002, seed=900 + w, device="cuda") for w in range(W)]
+    merged, want, status, _ = _decode_both(n, offs, msgs, 0.5)
+    monkeypatch.setenv("VGC_DECODE_PATH", "scatter")
+    scattered, _, status2, _ = _decode_both(n, offs, msgs, 0.5)
+    assert status == 0 and status2 == 0
+    assert np.abs(merged.astype(np.float64) - want).max() <= ATOL
+    assert np.abs(scattered.astype(np.float64) - want).max() <= ATOL
