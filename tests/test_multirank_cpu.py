@@ -28,7 +28,7 @@ assert gathered[0] != gathered[1]
 assert workloads.seed_for(2, 16, 0, 3, 0) == workloads.seed_for(2, 16, 0, 3, 0)
 dist.barrier()
 dist.destroy_process_group()
-print("rank", rank, "ok")
+sys.stdout.write("rank%dok\n" % rank); sys.stdout.flush()
 """
 
 
@@ -55,7 +55,7 @@ def test_max_over_ranks_and_seeding_world_size_2(tmp_path):
     script.write_text(WORKER.format(root=ROOT))
     res = _torchrun([str(script)])
     assert res.returncode == 0, res.stdout + res.stderr
-    assert "rank 0 ok" in res.stdout and "rank 1 ok" in res.stdout
+    assert "rank0ok" in res.stdout and "rank1ok" in res.stdout
 
 
 def test_reference_arm_under_torchrun_prints_one_line_from_rank_0():
