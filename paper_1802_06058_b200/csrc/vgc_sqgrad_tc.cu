@@ -745,7 +745,11 @@ static Plan make_plan(int M, int N, int k_slices)
     p.tiles_x = (N + kBN - 1) / kBN;
     p.tiles_y = (M + kBM - 1) / kBM;
     const long tiles = (long)p.tiles_x * p.tiles_y;
-    long want = 148 / tiles;                               // one block per SM: fill the SMs at most once
+    // blocks of one launch: one per SM fills the device once; a caller that runs several layers side by side
+    // (separate streams and workspaces) may ask for fewer, longer blocks through VGC_TC_BLOCKS
+    const char *env = getenv("VGC_TC_BLOCKS");
+    const long target = env && atoi(env) > 0 ? atoi(env) : 148;
+    long want = target / tiles;
     if (want > k_slices) want = k_slices;
     if (want < 1) want = 1;
     p.k_slices = k_slices;
