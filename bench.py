@@ -134,6 +134,7 @@ class HotPath:
         self.K = len(self.offsets) - 1
         self.offs_dev = vgc.offsets_tensor(self.offsets)
         self.compress_only = name in ("vgg16", "flat")
+        self.fused = False
         dev = device
         B = self.batch
         self.scale = 1.0 / (B * B)
@@ -200,25 +201,27 @@ class HotPath:
             del rr, vv
 
     # -- launches -------------------------------------------------------------------------------
-    def sqgrad(self, t: int):
+    def sqgrad(self, t: int, into_v: bool = False):
+        """Squared-gradient sums of every layer into s (or, fused form, added straight into v)."""
         vgc = self.vgc
         if self.compress_only:
             return
+        target = self.v if into_v else self.s
         ins = self.inputs[t % len(self.inputs)]
         main = torch.cuda.current_stream()
         for st in self.side:
             st.wait_stream(main)
         for li, spec in enumerate(self.layers):
             x, delta = ins[li]
-            S = self.s[int(self.offsets[li]):int(self.offsets[li + 1])]
+            S = target[int(self.offsets[li]):int(self.offsets[li + 1])]
             lane = li % self.n_streams
             stream = main if lane == 0 else self.side[lane - 1]
             ws = self.ws_s if lane == 0 else self.ws_side[lane - 1]
             if spec.kind == "conv":
                 vgc.vgc_sqgrad_conv(x, delta, (spec.k, spec.k), (spec.stride, spec.stride), (spec.pad, spec.pad),
-                                    self.scale, S, ws=ws, stream=stream)
+                                    self.scale, S, accumulate=into_v, ws=ws, stream=stream)
             else:
-                vgc.vgc_sqgrad_linear(x, delta, self.scale, S, ws=ws, stream=stream)
+                vgc.vgc_sqgrad_linear(x, delta, self.scale, S, accumulate=into_v, ws=ws, stream=stream)
         for st in self.side:
             main.wait_stream(st)
 
@@ -256,8 +259,8 @@ class HotPath:
                         "useful_tflops": round(2 * M * N * K / (ms * 1e-3) / 1e12, 2)})
         return out
 
-    def compress(self, t: int):
-        s = self.s if self.s_sets is None else self.s_sets[t % len(self.s_sets)]
+    def compress(self, t: int, fused: bool = False):
+        s = None if fused else (self.s if self.s_sets is None else self.s_sets[t % len(self.s_sets)])
         self.vgc.vgc_compress(self.g_sets[t % len(self.g_sets)], s, self.r, self.v, self.offs_dev, self.alpha,
                               ZETA, self.out, self.ws_c)
 
@@ -268,9 +271,10 @@ class HotPath:
         self.vgc.vgc_decode_accumulate([self.out] + self.others, self.offs_dev, 1.0 / self.W, self.u, self.status)
 
     def step(self, t: int, marks=None):
-        self.sqgrad(t)
+        fused = self.fused and not self.compress_only
+        self.sqgrad(t, into_v=fused)
         if marks: marks[0].record()
-        self.compress(t)
+        self.compress(t, fused=fused)
         if marks: marks[1].record()
         self.decode(t)
         if marks: marks[2].record()
@@ -526,6 +530,8 @@ def main():
     ap.add_argument("--per-layer", action="store_true", help="print per-layer sqgrad times instead of the bench line")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--streams", type=int, default=4, help="streams the independent sqgrad layers are spread over")
+    ap.add_argument("--fused", action="store_true",
+                    help="sqgrad adds its sums straight into v and vgc_compress runs without s (12 B read per parameter)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -548,6 +554,7 @@ def main():
     pk = peaks()
     hp = HotPath(args.workload, worker=rank * 16, n_input_sets=1, n_g_sets=max(4, min(args.steps + args.warmup, 16)),
                  n_params=args.n_params, n_streams=max(args.streams, 1))
+    hp.fused = args.fused
     torch.cuda.synchronize()
 
     if args.per_layer:
@@ -617,6 +624,7 @@ def main():
             "config": {"workload": args.workload, "n_params": n, "batch": hp.batch, "W": hp.W, "alpha": hp.alpha,
                        "zeta": ZETA, "groups": hp.K, "launch": "eager" if args.no_graph else "cuda graph replay",
                        "sqgrad_streams": getattr(hp, "n_streams", 1),
+                       "fused_sqgrad_into_v": bool(args.fused),
                        "l2": "inputs larger than L2 (no flush)" if n * 16 > 126e6 else "state fits in L2 (no flush): cache-resident numbers"},
             "gpu_launches": int(launches), "clocks": clocks, "sections": sections, "roofline": roofline,
             "roofline_compress": compress_roofline}

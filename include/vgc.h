@@ -118,6 +118,9 @@ vgc_status vgc_sqgrad_conv(const float *x, const float *delta, int B, int C, int
  * Words come out in ascending index order; the output is a deterministic function of the inputs.
  *
  *   g, s          [n] fp32: this step's sum of per-example gradients / B and sum of their squares
+ *                 s may be NULL: then v must already hold v + s (the sqgrad calls with accumulate = 1
+ *                 and S pointing into v do exactly that one fp32 addition), and the pass reads 4 bytes
+ *                 per parameter less; results are identical bit for bit
  *   r, v          [n] fp32 state, updated in place (all zeros before the first step)
  *   group_offsets [K+1] u32 on the device, offsets[0] = 0, offsets[K] = n, non-decreasing
  *   out           HOST struct of device pointers, see below

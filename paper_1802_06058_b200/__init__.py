@@ -219,9 +219,10 @@ def vgc_compress_workspace_bytes(n: int, K: int) -> int:
 
 
 def vgc_compress(g, s, r, v, group_offsets, alpha: float, zeta: float, out: MessageBuffers, ws, stream=None):
-    """One step of Algorithm 1 over the flat buffer + Encode(); r, v updated in place."""
+    """One step of Algorithm 1 over the flat buffer + Encode(); r, v updated in place.
+    ``s=None``: v already contains this step's squared-gradient sums (sqgrad with accumulate into v)."""
     n = g.numel()
-    if s.numel() != n or r.numel() != n or v.numel() != n:
+    if (s is not None and s.numel() != n) or r.numel() != n or v.numel() != n:
         raise ValueError("g, s, r, v must have the same length")
     K = group_offsets.numel() - 1
     if out.K != K:
@@ -230,7 +231,7 @@ def vgc_compress(g, s, r, v, group_offsets, alpha: float, zeta: float, out: Mess
         raise ValueError("mask length")
     wp, wb = _ws(ws)
     msg = out.struct()
-    st = load_library().vgc_compress(_dev(g, torch.float32, "g"), _dev(s, torch.float32, "s"),
+    st = load_library().vgc_compress(_dev(g, torch.float32, "g"), None if s is None else _dev(s, torch.float32, "s"),
                                      _dev(r, torch.float32, "r"), _dev(v, torch.float32, "v"), n,
                                      _dev(group_offsets, torch.int32, "group_offsets"), K, float(alpha),
                                      float(zeta), ctypes.byref(msg), wp, wb, _stream(stream))

@@ -55,6 +55,9 @@ static CompressLayout compress_layout(size_t n, int K)
 // ------------------------------------------------------------------------------------------
 // phase A
 // ------------------------------------------------------------------------------------------
+// kHasS = false: the caller accumulated this step's squared-gradient sums straight into v (the sqgrad entry
+// points with accumulate = 1), so the pass reads 12 instead of 16 bytes per parameter.
+template <bool kHasS>
 __global__ void __launch_bounds__(kThreads, 4)
 compress_phase_a(const float *__restrict__ g, const float *__restrict__ s, float *__restrict__ r,
                  float *__restrict__ v, size_t n, const uint32_t *__restrict__ group_offsets, int K,
@@ -86,7 +89,7 @@ compress_phase_a(const float *__restrict__ g, const float *__restrict__ s, float
             const size_t e = base + (size_t)(j * kThreads + tid) * 4;
             if (e + 3 < n) {
                 G[j] = ld_stream_f4(g + e);
-                S[j] = ld_stream_f4(s + e);
+                if (kHasS) S[j] = ld_stream_f4(s + e);
                 R[j] = *reinterpret_cast<const float4 *>(r + e);
                 V[j] = *reinterpret_cast<const float4 *>(v + e);
             } else {
@@ -94,7 +97,7 @@ compress_phase_a(const float *__restrict__ g, const float *__restrict__ s, float
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     const bool in = e + q < n;
-                    tg[q] = in ? g[e + q] : 0.f;  ts[q] = in ? s[e + q] : 0.f;
+                    tg[q] = in ? g[e + q] : 0.f;  ts[q] = (kHasS && in) ? s[e + q] : 0.f;
                     tr[q] = in ? r[e + q] : 0.f;  tv[q] = in ? v[e + q] : 0.f;
                 }
                 G[j] = make_float4(tg[0], tg[1], tg[2], tg[3]);  S[j] = make_float4(ts[0], ts[1], ts[2], ts[3]);
@@ -122,7 +125,7 @@ compress_phase_a(const float *__restrict__ g, const float *__restrict__ s, float
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const float r1 = __fadd_rn(Rj[q], Gj[q]);
-                const float v1 = __fadd_rn(Vj[q], Sj[q]);
+                const float v1 = kHasS ? __fadd_rn(Vj[q], Sj[q]) : Vj[q];
                 const float lhs = __fmul_rn(r1, r1);
                 const float rhs = __fmul_rn(alpha, v1);
                 const bool send = (lhs > rhs) && (e + q < n);
@@ -396,11 +399,11 @@ extern "C" vgc_status vgc_compress(const float *g, const float *s, float *r, flo
     if (!(alpha >= 0.f) || !(alpha <= 3.402823466e38f) || !(zeta == zeta) || !(zeta >= -3.402823466e38f) ||
         !(zeta <= 3.402823466e38f))
         return VGC_ERR_INVALID_ARG;
-    if (!g || !s || !r || !v || !group_offsets || !ws) return VGC_ERR_INVALID_ARG;
+    if (!g || !r || !v || !group_offsets || !ws) return VGC_ERR_INVALID_ARG;
     if (!out->group_exp || !out->nnz || !out->n_criterion || !out->n_dropped || !out->dev_status)
         return VGC_ERR_INVALID_ARG;
     if (out->capacity && !out->words) return VGC_ERR_INVALID_ARG;
-    if (!aligned16(g) || !aligned16(s) || !aligned16(r) || !aligned16(v) || !aligned16(ws) ||
+    if (!aligned16(g) || (s && !aligned16(s)) || !aligned16(r) || !aligned16(v) || !aligned16(ws) ||
         (out->mask && (reinterpret_cast<uintptr_t>(out->mask) & 3u)))
         return VGC_ERR_INVALID_ARG;
     const CompressLayout L = compress_layout(n, K);
@@ -425,8 +428,12 @@ extern "C" vgc_status vgc_compress(const float *g, const float *s, float *r, flo
 
     VGC_CUDA_OK(cudaMemsetAsync(ws, 0, L.zero_bytes, st));
     const uint32_t grid_a = L.tiles_a < (uint32_t)(sm_count * 8) ? L.tiles_a : (uint32_t)(sm_count * 8);
-    compress_phase_a<<<grid_a, kThreads, 0, st>>>(g, s, r, v, n, group_offsets, K, alpha, zeta, gmax, tile_count,
-                                                  stage_idx, stage_val, out->mask, L.tiles_a);
+    if (s)
+        compress_phase_a<true><<<grid_a, kThreads, 0, st>>>(g, s, r, v, n, group_offsets, K, alpha, zeta, gmax, tile_count,
+                                                            stage_idx, stage_val, out->mask, L.tiles_a);
+    else
+        compress_phase_a<false><<<grid_a, kThreads, 0, st>>>(g, nullptr, r, v, n, group_offsets, K, alpha, zeta, gmax,
+                                                             tile_count, stage_idx, stage_val, out->mask, L.tiles_a);
     compress_count<<<L.chunks, kThreads, 0, st>>>(group_offsets, K, gmax, tile_count, L.tiles_a, stage_idx,
                                                   stage_val, kept_count, chunk_total, out->group_exp);
     compress_emit<<<L.chunks, kThreads, 0, st>>>(group_offsets, K, gmax, tile_count, L.tiles_a, stage_idx,

@@ -602,13 +602,20 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             } else if (prm.ld_m == 1) {
                 // result is contiguous along m: lanes write neighbouring addresses directly
                 if (m < prm.M) {
+                    float *col = prm.S + (size_t)m + (size_t)n0 * prm.ld_n;
 #pragma unroll
-                    for (int j = 0; j < kBN; ++j)
-                        if (j < n_valid) {
-                            float *dst = prm.S + (size_t)m + (size_t)(n0 + j) * prm.ld_n;
-                            const float res = __fmul_rn(prm.scale, acc[j]);
-                            *dst = prm.accumulate ? __fadd_rn(*dst, res) : res;
-                        }
+                    for (int j0 = 0; j0 < kBN; j0 += 16) {        // old values sixteen at a time, all loads in flight
+                        float old[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            old[j] = (prm.accumulate && j0 + j < n_valid) ? col[(size_t)(j0 + j) * prm.ld_n] : 0.f;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (j0 + j < n_valid) {
+                                const float res = __fmul_rn(prm.scale, acc[j0 + j]);
+                                col[(size_t)(j0 + j) * prm.ld_n] = prm.accumulate ? __fadd_rn(old[j], res) : res;
+                            }
+                    }
                 }
             } else {
                 // result is contiguous along n: transpose this warp's 32 x 128 block through shared memory
@@ -617,16 +624,29 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 #pragma unroll
                 for (int j = 0; j < kBN; ++j) tile[lane * (kBN + 1) + j] = __fmul_rn(prm.scale, acc[j]);
                 __syncwarp();
-                for (int r = 0; r < 32; ++r) {
-                    const int mr = m0 + (int)(q * 32u) + r;
-                    if (mr >= prm.M) break;
-                    float *dst = prm.S + (size_t)mr * prm.ld_m + n0;
+                for (int r0 = 0; r0 < 32; r0 += 8) {              // eight rows at a time, all loads in flight
+                    float old[8][kBN / 32];
 #pragma unroll
-                    for (int cblk = 0; cblk < kBN / 32; ++cblk) {
-                        const int j = cblk * 32 + (int)lane;
-                        if (j < n_valid) {
-                            const float res = tile[r * (kBN + 1) + j];
-                            dst[j] = prm.accumulate ? __fadd_rn(dst[j], res) : res;
+                    for (int rr = 0; rr < 8; ++rr) {
+                        const int mr = m0 + (int)(q * 32u) + r0 + rr;
+                        const float *src = prm.S + (size_t)mr * prm.ld_m + n0;
+#pragma unroll
+                        for (int cblk = 0; cblk < kBN / 32; ++cblk) {
+                            const int j = cblk * 32 + (int)lane;
+                            old[rr][cblk] = (prm.accumulate && mr < prm.M && j < n_valid) ? src[j] : 0.f;
+                        }
+                    }
+#pragma unroll
+                    for (int rr = 0; rr < 8; ++rr) {
+                        const int mr = m0 + (int)(q * 32u) + r0 + rr;
+                        float *dst = prm.S + (size_t)mr * prm.ld_m + n0;
+#pragma unroll
+                        for (int cblk = 0; cblk < kBN / 32; ++cblk) {
+                            const int j = cblk * 32 + (int)lane;
+                            if (mr < prm.M && j < n_valid) {
+                                const float res = tile[(r0 + rr) * (kBN + 1) + j];
+                                dst[j] = prm.accumulate ? __fadd_rn(old[rr][cblk], res) : res;
+                            }
                         }
                     }
                 }

@@ -113,3 +113,32 @@ def test_without_mask_and_on_a_side_stream():
     side.synchronize()
     want = cpu.step(g.cpu().numpy(), s.cpu().numpy(), 2.0, 0.999)
     assert_same_message(got, want)
+
+
+def test_sqgrad_accumulated_into_v_then_compress_without_s():
+    """The fused form: the squared-gradient kernels add their result straight into v (accumulate = 1) and the
+    compressor is called without s.  v + s is one fp32 addition either way, so everything matches bit for bit."""
+    from paper_1802_06058_b200 import workloads
+    layers, B = workloads.mlp_layers(), 128
+    offs = workloads.group_offsets(layers)
+    n, scale = int(offs[-1]), 1.0 / (B * B)
+    plain, cpu = GpuCompressor(n, offs), OracleCompressor(n, offs)
+    fused = GpuCompressor(n, offs)
+    ws = torch.zeros(1 << 26, dtype=torch.uint8, device="cuda")
+    s = torch.empty(n, device="cuda")
+    for t in range(4):
+        ins = [workloads.layer_inputs(spec, B, 1, 0, t, li, "relu_normal", 1e-3, "cuda") for li, spec in enumerate(layers)]
+        g = torch.cat([workloads.mean_gradient(spec, x, d) for spec, (x, d) in zip(layers, ins)])
+        for li, (spec, (x, d)) in enumerate(zip(layers, ins)):
+            lo, hi = int(offs[li]), int(offs[li + 1])
+            vgc.vgc_sqgrad_linear(x, d, scale, s[lo:hi], ws=ws)
+            vgc.vgc_sqgrad_linear(x, d, scale, fused.v[lo:hi], accumulate=True, ws=ws)
+        got_plain = plain.step(g, s, 2.0, 0.999)
+        fused.out.counters.zero_()
+        vgc.vgc_compress(g, None, fused.r, fused.v, fused.offs_dev, 2.0, 0.999, fused.out, fused.ws)
+        got_fused = fused.out.read()
+        want = cpu.step(g.cpu().numpy(), s.cpu().numpy(), 2.0, 0.999)
+        assert_same_message(got_plain, want)
+        assert_same_message(got_fused, want)
+        assert_same_state(plain, cpu)
+        assert_same_state(fused, cpu)
