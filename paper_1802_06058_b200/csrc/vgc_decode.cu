@@ -80,7 +80,7 @@ decode_scatter(const __grid_constant__ DecodeViews views, const uint32_t *__rest
 //     inside a message are distinct), and the tile is written back -- u is read and written once,
 //     coalesced, however many words hit it, and the sum is formed in message order.
 // ------------------------------------------------------------------------------------------
-constexpr int kMergeTile = 8192;                 // elements of u per shared-memory tile (32 KB)
+constexpr int kMergeTile = 4096;                 // elements of u per shared-memory tile (16 KB)
 constexpr int kMergeWarps = kDecThreads / 32;
 
 // first position in [0, count) whose index is >= bound (count if none); whole warp, 32-ary search
@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(kDecThreads)
 decode_merge(const __grid_constant__ DecodeViews views, int W, const uint32_t *__restrict__ group_offsets, int K,
              float scale, float *__restrict__ u, size_t n, uint32_t chunk_elems, uint32_t *dev_status)
 {
-    __shared__ float tile[kMergeTile];
+    __shared__ __align__(16) float tile[kMergeTile];
     __shared__ uint32_t sm_offs[kDecOffsSmem];
     __shared__ uint32_t run_begin[kMaxViews], run_end[kMaxViews];
     __shared__ uint32_t total_words;
@@ -122,17 +122,17 @@ decode_merge(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
     const size_t hi = lo + chunk_elems < n ? lo + chunk_elems : n;
     const bool last_chunk = hi == n;
 
-    // ---- the run of every message inside [lo, hi)
+    // ---- where every message's run enters [lo, hi); the run ends where its indices reach hi, which the
+    // tile loop finds as it goes.  Dense or sparse is decided for the whole call from the messages' sizes.
     for (int w = warp; w < W; w += kMergeWarps) {
         const uint32_t *words = views.words[w];
         const uint32_t count = *views.nnz[w];
         const uint32_t b = warp_lower_bound(words, count, (uint32_t)lo);
-        const uint32_t e = b + warp_lower_bound(words + b, count - b, (uint32_t)hi);
         if (lane == 0) {
             run_begin[w] = b;
-            run_end[w] = e;
-            atomicAdd(&total_words, e - b);
-            if (last_chunk && e < count) atomicOr(dev_status, VGC_DEV_RANGE);      // indices >= n: skipped
+            run_end[w] = count;
+            atomicAdd(&total_words, count);
+            if (last_chunk && count && (words[count - 1] >> 4) >= n) atomicOr(dev_status, VGC_DEV_RANGE);   // skipped
         }
     }
     __syncthreads();
@@ -146,15 +146,18 @@ decode_merge(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
         return __fmul_rn(scale, __uint_as_float(((uint32_t)(e + 127) << 23) | ((word & 8u) << 28)));
     };
 
-    if ((size_t)total * 8 < hi - lo) {
-        // ---- sparse chunk: not worth moving the whole range through shared memory
+    if ((size_t)total * 8 < n) {
+        // ---- sparse messages: not worth moving u through shared memory
         for (int w = warp; w < W; w += kMergeWarps) {
             const uint32_t *words = views.words[w];
             const int32_t *gexp = views.group_exp[w];
             int k = 0;
-            for (uint32_t i = run_begin[w] + lane; i < run_end[w]; i += 32) {
-                const uint32_t word = words[i];
-                atomicAdd(u + (word >> 4), value_of(word, gexp, k));
+            for (uint32_t i0 = run_begin[w]; i0 < run_end[w]; i0 += 32) {       // warp-uniform trip count
+                const uint32_t i = i0 + lane;
+                const uint32_t word = i < run_end[w] ? words[i] : 0xFFFFFFFFu;
+                const bool in = i < run_end[w] && (word >> 4) < hi;
+                if (in) atomicAdd(u + (word >> 4), value_of(word, gexp, k));
+                if (!__all_sync(0xffffffffu, in)) break;             // sorted: the rest belongs to later chunks
             }
         }
         return;
@@ -163,57 +166,125 @@ decode_merge(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
     // ---- dense chunk: tile by tile through shared memory.  Messages are applied one after the other, in
     // message order, by the whole block: inside one message the indices are distinct, so plain
     // read-modify-writes suffice and every element sees its additions in the order w = 0, 1, ... --
-    // the result does not depend on scheduling.
-    __shared__ uint32_t cur[kMaxViews], t_end[kMaxViews];
-    for (int w = threadIdx.x; w < W; w += kDecThreads) cur[w] = run_begin[w];
+    // the result does not depend on scheduling.  A message's words of a tile are the head of what is left of
+    // its run: the block loads a window of kPre*256 words, applies those below the tile's end and counts them.
+    __shared__ uint32_t cur[kMaxViews], taken[kMaxViews];
+    for (int w = threadIdx.x; w < W; w += kDecThreads) { cur[w] = run_begin[w]; taken[w] = 0; }
+    constexpr int kPre = 4;                          // words per thread in one window
+    constexpr int kGroup = 8;                        // messages whose windows are in flight together
+    constexpr int kVec = kMergeTile / 4 / kDecThreads;   // float4 per thread per tile
+    const float4 *u4 = reinterpret_cast<const float4 *>(u);          // u is 16-byte aligned, tiles are whole
+    float4 ahead[kVec];                              // next tile of u, loaded while the current one is processed
+    auto fetch_tile = [&](size_t t0) {
+#pragma unroll
+        for (int q = 0; q < kVec; ++q) {
+            const size_t i = t0 + 4 * (threadIdx.x + q * kDecThreads);
+            if (i + 3 < hi) ahead[q] = u4[i / 4];
+            else {
+                float e[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) e[c] = i + c < hi ? u[i + c] : 0.f;
+                ahead[q] = make_float4(e[0], e[1], e[2], e[3]);
+            }
+        }
+    };
+    fetch_tile(lo);
     __syncthreads();
-    constexpr int kPre = 4;                          // words per thread and message held in registers
-    constexpr int kGroup = 8;                        // messages whose words are in flight together
     for (size_t t0 = lo; t0 < hi; t0 += kMergeTile) {
         const uint32_t t_len = (uint32_t)(hi - t0 < kMergeTile ? hi - t0 : kMergeTile);
         const uint32_t t_hi = (uint32_t)(t0 + t_len);
-        for (uint32_t i = threadIdx.x; i < t_len; i += kDecThreads) tile[i] = u[t0 + i];
-        for (int w = warp; w < W; w += kMergeWarps) {        // where each message's run leaves this tile
-            const uint32_t b = cur[w];
-            const uint32_t e = b + warp_lower_bound(views.words[w] + b, run_end[w] - b, t_hi);
-            if (lane == 0) t_end[w] = e;
-        }
-        __syncthreads();
-        for (int w0 = 0; w0 < W; w0 += kGroup) {             // the words of kGroup messages are fetched together ...
-            uint32_t held[kGroup][kPre];
+        int tile_group = group_of(offs, K, (uint32_t)t0);    // weight tensor of the tile, -1 if it spans several
+        if (t_hi - 1 >= offs[tile_group + 1]) tile_group = -1;
 #pragma unroll
-            for (int g = 0; g < kGroup; ++g) {
-                const int w = w0 + g < W ? w0 + g : W - 1;
-                const uint32_t *words = views.words[w];
-                const uint32_t b = cur[w], e = t_end[w];
+        for (int q = 0; q < kVec; ++q) reinterpret_cast<float4 *>(tile)[threadIdx.x + q * kDecThreads] = ahead[q];
+        if (t0 + kMergeTile < hi) fetch_tile(t0 + kMergeTile);
+        __syncthreads();
+
+        // one window of one message: apply the words below t_hi, return how many this thread applied
+        auto apply = [&](int w, const uint32_t (&win)[kPre], uint32_t base) -> uint32_t {
+            const int32_t *gexp = views.group_exp[w];
+            const uint32_t e = run_end[w];
+            uint32_t mine = 0;
+            if (tile_group >= 0) {
+                const uint32_t ebits = (uint32_t)(gexp[tile_group] + 127) << 23;   // one exponent for the tile
 #pragma unroll
                 for (int j = 0; j < kPre; ++j) {
-                    const uint32_t i = b + threadIdx.x + j * kDecThreads;
-                    held[g][j] = i < e ? words[i] : 0u;
-                }
-            }
-#pragma unroll
-            for (int g = 0; g < kGroup; ++g) {                // ... and applied one message after the other
-                const int w = w0 + g;
-                if (w < W) {
-                    const uint32_t *words = views.words[w];
-                    const int32_t *gexp = views.group_exp[w];
-                    const uint32_t b = cur[w], e = t_end[w];
-                    int k = 0;
-#pragma unroll
-                    for (int j = 0; j < kPre; ++j)
-                        if (b + threadIdx.x + j * kDecThreads < e)
-                            tile[(held[g][j] >> 4) - (uint32_t)t0] += value_of(held[g][j], gexp, k);
-                    for (uint32_t i = b + threadIdx.x + kPre * kDecThreads; i < e; i += kDecThreads) {
-                        const uint32_t word = words[i];
-                        tile[(word >> 4) - (uint32_t)t0] += value_of(word, gexp, k);
+                    const uint32_t word = win[j];
+                    if (base + threadIdx.x + j * kDecThreads < e && (word >> 4) < t_hi) {
+                        const float val = __uint_as_float((ebits - ((word & 7u) << 23)) | ((word & 8u) << 28));
+                        tile[(word >> 4) - (uint32_t)t0] += __fmul_rn(scale, val);
+                        ++mine;
                     }
                 }
-                __syncthreads();
+            } else {
+                int k = 0;
+#pragma unroll
+                for (int j = 0; j < kPre; ++j) {
+                    const uint32_t word = win[j];
+                    if (base + threadIdx.x + j * kDecThreads < e && (word >> 4) < t_hi) {
+                        tile[(word >> 4) - (uint32_t)t0] += value_of(word, gexp, k);
+                        ++mine;
+                    }
+                }
+            }
+            return mine;
+        };
+        auto load_window = [&](int w, uint32_t base, uint32_t (&win)[kPre]) {
+            const uint32_t *words = views.words[w];
+            const uint32_t e = run_end[w];
+#pragma unroll
+            for (int j = 0; j < kPre; ++j) {
+                const uint32_t i = base + threadIdx.x + j * kDecThreads;
+                win[j] = i < e ? words[i] : 0xFFFFFFFFu;
+            }
+        };
+
+        for (int w0 = 0; w0 < W; w0 += kGroup) {
+            uint32_t held[kGroup][kPre];
+#pragma unroll
+            for (int g = 0; g < kGroup; ++g) load_window(w0 + g < W ? w0 + g : W - 1, cur[w0 + g < W ? w0 + g : W - 1], held[g]);
+#pragma unroll
+            for (int g = 0; g < kGroup; ++g) {
+                const int w = w0 + g;
+                if (w < W) {                                         // uniform over the block
+                    uint32_t base = cur[w];
+                    uint32_t mine = apply(w, held[g], base);
+                    // block total of `mine`: warp sums, then shared counter
+                    uint32_t wsum = mine;
+#pragma unroll
+                    for (int d = 16; d >= 1; d >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, d);
+                    if (lane == 0 && wsum) atomicAdd(&taken[w], wsum);
+                    __syncthreads();
+                    // a full window means the tile may hold more words of this message
+                    while (taken[w] == (base - cur[w]) + kPre * kDecThreads) {
+                        base += kPre * kDecThreads;
+                        uint32_t win[kPre];
+                        load_window(w, base, win);
+                        mine = apply(w, win, base);
+                        wsum = mine;
+#pragma unroll
+                        for (int d = 16; d >= 1; d >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, d);
+                        __syncthreads();                             // everyone has read taken[w]
+                        if (lane == 0 && wsum) atomicAdd(&taken[w], wsum);
+                        __syncthreads();
+                    }
+                }
             }
         }
-        for (uint32_t i = threadIdx.x; i < t_len; i += kDecThreads) u[t0 + i] = tile[i];
-        for (int w = threadIdx.x; w < W; w += kDecThreads) cur[w] = t_end[w];
+#pragma unroll
+        for (int q = 0; q < kVec; ++q) {
+            const size_t i = t0 + 4 * (threadIdx.x + q * kDecThreads);
+            const float4 val = reinterpret_cast<const float4 *>(tile)[threadIdx.x + q * kDecThreads];
+            if (i + 3 < hi) reinterpret_cast<float4 *>(u)[i / 4] = val;
+            else {
+                const float e[4] = {val.x, val.y, val.z, val.w};
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    if (i + c < hi) u[i + c] = e[c];
+            }
+        }
+        __syncthreads();
+        for (int w = threadIdx.x; w < W; w += kDecThreads) { cur[w] += taken[w]; taken[w] = 0; }
         __syncthreads();
     }
 }
@@ -227,7 +298,7 @@ extern "C" vgc_status vgc_decode_accumulate(const vgc_message_view *msgs, int W,
                                             float *u, size_t n, uint32_t *dev_status, vgc_stream_t stream)
 {
     if (W == 0 || n == 0) return VGC_OK;
-    if (W < 0 || K < 1 || n > VGC_MAX_PARAMS || !msgs || !group_offsets || !u || !dev_status)
+    if (W < 0 || K < 1 || n > VGC_MAX_PARAMS || !msgs || !group_offsets || !u || !dev_status || !aligned16(u))
         return VGC_ERR_INVALID_ARG;
     if (!(scale == scale)) return VGC_ERR_INVALID_ARG;
     for (int w = 0; w < W; ++w)
@@ -257,7 +328,7 @@ extern "C" vgc_status vgc_decode_accumulate(const vgc_message_view *msgs, int W,
             dim3 grid((unsigned)per_msg, (unsigned)wb);
             decode_scatter<<<grid, kDecThreads, 0, st>>>(views, group_offsets, K, scale, u, n, dev_status);
         } else {
-            // one chunk per block, about four blocks per SM, whole tiles per chunk
+            // one chunk per block, four blocks per SM (all resident at once), whole tiles per chunk
             size_t chunk = (n + (size_t)sm_count * 4 - 1) / ((size_t)sm_count * 4);
             chunk = (chunk + kMergeTile - 1) / kMergeTile * kMergeTile;
             const unsigned blocks = (unsigned)((n + chunk - 1) / chunk);
