@@ -579,7 +579,8 @@ def main():
     nnz_a, nnz = counters["n_criterion"], counters["nnz"]
     sum_nnz = nnz + sum(int(o.words.numel()) for o in hp.others) if hp.W else 0
     compress_bytes = 24 * n + 8 * nnz_a + 4 * nnz
-    decode_bytes = 12 * sum_nnz + 4 * n * (1 if hp.W else 0)       # words + read-modify-write of u + clearing u
+    # decode: 4 B per word + one read and one write of u (merge form) + the 4 B/element clearing of u before it
+    decode_bytes = (4 * sum_nnz + 12 * n) if hp.W else 0
     sections = {
         "sqgrad_ms": sq_ms, "compress_ms": co_ms, "decode_ms": de_ms,
         "sqgrad_useful_tflops": hp.flops_useful / (sq_ms * 1e-3) / 1e12 if sq_ms > 0 and hp.flops_useful else None,
