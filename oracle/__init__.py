@@ -60,6 +60,13 @@ def _load():
         lib.oracle_decode_accumulate.argtypes = [ctypes.POINTER(u32p), u32p, ctypes.POINTER(i32p), i,
                                                  u32p, i, ctypes.c_float, f32p, ctypes.c_uint64]
         lib.oracle_decode_accumulate.restype = ctypes.c_uint64
+        lib.oracle_compress_hybrid.argtypes = [f32p, f32p, f32p, f32p, ctypes.c_uint64, ctypes.c_float,
+                                               ctypes.c_float, ctypes.c_float, i, u32p, ctypes.c_uint64, u32p,
+                                               ctypes.POINTER(ctypes.c_uint8)]
+        lib.oracle_compress_hybrid.restype = ctypes.c_int
+        lib.oracle_decode_hybrid.argtypes = [ctypes.POINTER(u32p), u32p, i, ctypes.c_float, ctypes.c_float, f32p,
+                                             ctypes.c_uint64]
+        lib.oracle_decode_hybrid.restype = ctypes.c_uint64
         _lib = lib
     return _lib
 
@@ -203,3 +210,35 @@ def decode_accumulate(messages, group_offsets, scale, u):
     return int(_load().oracle_decode_accumulate(wptrs, _ptr(nnz, ctypes.c_uint32), eptrs, W,
                                                 _ptr(offs, ctypes.c_uint32), K, float(scale),
                                                 _ptr(u, ctypes.c_float), u.size))
+
+
+def compress_hybrid(g, s, r, v, alpha, zeta, tau, pre_update_r=True, capacity=None, want_mask=True):
+    """One step of the hybrid algorithm (Algorithm 2); r and v are updated IN PLACE.  Returns a Message whose
+    words are index << 4 | sign << 3 (group_exp is empty, n_criterion == nnz)."""
+    g = _f32(g, "g"); s = _f32(s, "s")
+    n = g.size
+    cap = n if capacity is None else int(capacity)
+    words = np.zeros(max(cap, 1), np.uint32)
+    cnt = np.zeros(1, np.uint32)
+    mask = np.zeros(max(n, 1), np.uint8) if want_mask else None
+    over = _load().oracle_compress_hybrid(
+        _ptr(g, ctypes.c_float), _ptr(s, ctypes.c_float), _ptr(r, ctypes.c_float), _ptr(v, ctypes.c_float), n,
+        float(alpha), float(zeta), float(tau), int(bool(pre_update_r)), _ptr(words, ctypes.c_uint32), cap,
+        _ptr(cnt, ctypes.c_uint32), _ptr(mask, ctypes.c_uint8) if want_mask else None)
+    nnz = int(cnt[0])
+    return Message(words[:min(nnz, cap)].copy(), np.zeros(0, np.int32), nnz, nnz, 0, mask[:n] if want_mask else None,
+                   bool(over))
+
+
+def decode_hybrid(word_arrays, tau, scale, u):
+    """u[idx] += scale * (+-tau) for every word of every message (message order); u IN PLACE."""
+    W = len(word_arrays)
+    u32p = ctypes.POINTER(ctypes.c_uint32)
+    keep = [np.ascontiguousarray(w, dtype=np.uint32) for w in word_arrays]
+    ptrs = (u32p * max(W, 1))()
+    nnz = np.zeros(max(W, 1), np.uint32)
+    for k, w in enumerate(keep):
+        ptrs[k] = _ptr(w, ctypes.c_uint32)
+        nnz[k] = w.size
+    return int(_load().oracle_decode_hybrid(ptrs, _ptr(nnz, ctypes.c_uint32), W, float(tau), float(scale),
+                                            _ptr(u, ctypes.c_float), u.size))

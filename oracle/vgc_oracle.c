@@ -22,10 +22,14 @@
  *   oracle_compress             Algorithm 1 (Basic) loop body + Sec. 4.2 quantisation with
  *                               the Sec. 4.4 bit-level recipe + the 4+28-bit word of Sec. 4.2.
  *   oracle_decode_accumulate    decode half of CommunicateAndUpdate (Sec. 4.3, Fig. 1 caption).
+ *   oracle_compress_hybrid      Algorithm 2 (Hybrid) loop body with the variance correction of Sec. 4.5.
+ *   oracle_decode_hybrid        its receiver side: every word adds +-tau.
  *
  * Parity pins (tests/, run without a GPU): the Appendix B worked example; closed forms
  * of the Algorithm 1 state machine; equivalence of Eq. 2 with Eq. 1 via the last line of
- * Appendix A; residual accounting; brute-force per-example gradients for the squared sums.
+ * Appendix A; residual accounting; brute-force per-example gradients for the squared sums;
+ * for the hybrid: its reduction to the plain threshold method (alpha = 0), the "(a-b)^2" identity
+ * of Sec. 4.5 on single samples, the never-send limits, agreement with Algorithm 1's test at tau = 0.
  * Conventions the paper leaves open (scope of M_k, bit positions in the word, width of
  * the per-group exponent) are choices of this build: "parity unpinned" for those three.
  */
@@ -264,5 +268,69 @@ uint64_t oracle_decode_accumulate(const uint32_t *const *words, const uint32_t *
             u[idx] = u[idx] + term;
         }
     }
+    return bad;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Hybrid of the variance test with a fixed threshold (Algorithm 2, Sec. 4.5) */
+/* ------------------------------------------------------------------------- */
+
+/* One step over the flat buffer.  An element is sent when |r| > tau AND r^2 > alpha*v; what is
+ * sent is Sign(r) (the receiver adds +-tau), r keeps the remainder r - Sign(r)*tau, and the
+ * sum of squares is corrected as Sec. 4.5 derives it ("a^2 -> (a-b)^2"):
+ *     v <- max(v - 2*|r|*tau + tau^2, 0)
+ * with |r| the accumulated sum BEFORE the subtraction (pre_update_r != 0, the reading the
+ * derivation fixes: for a single sample v = r^2 it gives exactly (|r| - tau)^2), or AFTER it
+ * (pre_update_r == 0, the statement order of the Algorithm 2 listing).  v decays every step.
+ * Words: index << 4 | sign << 3, ascending index.  Returns 1 if the message did not fit. */
+int oracle_compress_hybrid(const float *g, const float *s, float *r, float *v, uint64_t n,
+                           float alpha, float zeta, float tau, int pre_update_r,
+                           uint32_t *words, uint64_t capacity, uint32_t *nnz, uint8_t *mask)
+{
+    uint32_t emitted = 0;
+    int overflow = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        float r1 = r[i] + g[i];
+        float v1 = v[i] + s[i];
+        float absr = float_of(bits_of(r1) & 0x7FFFFFFFu);
+        float lhs = r1 * r1;
+        float rhs = alpha * v1;
+        int send = (absr > tau) && (lhs > rhs);
+        if (send) {
+            uint32_t neg = bits_of(r1) >> 31;
+            uint32_t word = ((uint32_t)i << 4) | (neg << 3);
+            if (emitted < capacity) words[emitted] = word; else overflow = 1;
+            ++emitted;
+            float r2 = neg ? r1 + tau : r1 - tau;          /* r -= Sign(r) * tau */
+            float a = pre_update_r ? absr : float_of(bits_of(r2) & 0x7FFFFFFFu);
+            float twice = 2.0f * a;
+            float cross = twice * tau;
+            float diff = v1 - cross;
+            float tsq = tau * tau;
+            float corr = diff + tsq;
+            v1 = corr > 0.0f ? corr : 0.0f;
+            r1 = r2;
+        }
+        if (mask) mask[i] = (uint8_t)send;
+        r[i] = r1;
+        v[i] = v1 * zeta;                                   /* decay at every step */
+    }
+    *nnz = emitted;
+    return overflow;
+}
+
+/* Receiver side of the hybrid: every word adds scale * (+-tau) to its element. */
+uint64_t oracle_decode_hybrid(const uint32_t *const *words, const uint32_t *nnz, int W, float tau,
+                              float scale, float *u, uint64_t n)
+{
+    uint64_t bad = 0;
+    for (int w = 0; w < W; ++w)
+        for (uint32_t q = 0; q < nnz[w]; ++q) {
+            uint32_t word = words[w][q], idx = word >> 4;
+            if (idx >= n) { ++bad; continue; }
+            float value = ((word >> 3) & 1u) ? -tau : tau;
+            float term = scale * value;
+            u[idx] = u[idx] + term;
+        }
     return bad;
 }
