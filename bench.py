@@ -118,7 +118,7 @@ class HotPath:
     """All device buffers of one worker and the launches of one step."""
 
     def __init__(self, name: str, worker: int, n_input_sets: int, n_g_sets: int, device="cuda",
-                 n_params: int = 1 << 25, n_streams: int = 4):
+                 n_params: int = 1 << 25, n_streams: int = 4, algorithm: str = "basic"):
         import paper_1802_06058_b200 as vgc
         from paper_1802_06058_b200 import workloads
         self.vgc, self.wl = vgc, workloads
@@ -135,6 +135,8 @@ class HotPath:
         self.offs_dev = vgc.offsets_tensor(self.offsets)
         self.compress_only = name in ("vgg16", "flat")
         self.fused = False
+        self.hybrid = algorithm == "hybrid"                # Algorithm 2 instead of Algorithm 1
+        self.tau = 0.0
         dev = device
         B = self.batch
         self.scale = 1.0 / (B * B)
@@ -144,8 +146,12 @@ class HotPath:
         self.v = torch.zeros(self.n, **f32)
         self.u = torch.zeros(self.n, **f32)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
-        self.out = vgc.MessageBuffers(self.n, self.K, self.n, with_mask=False, device=dev)
-        self.ws_c = torch.empty(vgc.vgc_compress_workspace_bytes(self.n, self.K), dtype=torch.uint8, device=dev)
+        if self.hybrid:
+            self.out = vgc.HybridMessageBuffers(self.n, self.n, with_mask=False, device=dev)
+        else:
+            self.out = vgc.MessageBuffers(self.n, self.K, self.n, with_mask=False, device=dev)
+        self.ws_c = torch.empty(max(vgc.vgc_compress_workspace_bytes(self.n, self.K),
+                                    vgc.vgc_compress_hybrid_workspace_bytes(self.n)), dtype=torch.uint8, device=dev)
         self.flops_useful = 0
         self.inputs = []
         if self.compress_only:
@@ -184,6 +190,10 @@ class HotPath:
             self.s_sets = None
         # messages of the other W-1 workers: generated inputs (their own noise draws, compressed once)
         self.others = []
+        if self.hybrid:
+            # the fixed threshold of the hybrid: the median noise scale of the buffer, so that about half
+            # of the parameters can reach it at all
+            self.tau = float((self.s if self.s_sets is None else self.s_sets[0]).sqrt().median().item())
         if self.W > 1:
             root_s = (self.s if self.s_sets is None else self.s_sets[0]).sqrt()
             rr = torch.zeros(self.n, **f32); vv = torch.zeros(self.n, **f32)
@@ -191,9 +201,14 @@ class HotPath:
                 gen = torch.Generator(device=dev); gen.manual_seed(workloads.seed_for(cfg, worker + w, 0, 0, 3))
                 gw = torch.empty(self.n, **f32).normal_(generator=gen).mul_(root_s)
                 rr.zero_(); vv.zero_()
-                mb = vgc.MessageBuffers(self.n, self.K, self.n, device=dev)
-                vgc.vgc_compress(gw, self.s if self.s_sets is None else self.s_sets[0], rr, vv, self.offs_dev,
-                                 self.alpha, ZETA, mb, self.ws_c)
+                if self.hybrid:
+                    mb = vgc.HybridMessageBuffers(self.n, self.n, device=dev)
+                    vgc.vgc_compress_hybrid(gw, self.s if self.s_sets is None else self.s_sets[0], rr, vv,
+                                            self.alpha, ZETA, self.tau, mb, self.ws_c)
+                else:
+                    mb = vgc.MessageBuffers(self.n, self.K, self.n, device=dev)
+                    vgc.vgc_compress(gw, self.s if self.s_sets is None else self.s_sets[0], rr, vv, self.offs_dev,
+                                     self.alpha, ZETA, mb, self.ws_c)
                 torch.cuda.synchronize()
                 nnz = int(mb.counters[0].item())
                 mb.words = mb.words[:max(nnz, 4)].clone()          # keep only what was written
@@ -261,6 +276,10 @@ class HotPath:
 
     def compress(self, t: int, fused: bool = False):
         s = None if fused else (self.s if self.s_sets is None else self.s_sets[t % len(self.s_sets)])
+        if self.hybrid:
+            self.vgc.vgc_compress_hybrid(self.g_sets[t % len(self.g_sets)], s, self.r, self.v, self.alpha, ZETA,
+                                         self.tau, self.out, self.ws_c)
+            return
         self.vgc.vgc_compress(self.g_sets[t % len(self.g_sets)], s, self.r, self.v, self.offs_dev, self.alpha,
                               ZETA, self.out, self.ws_c)
 
@@ -268,6 +287,9 @@ class HotPath:
         if self.W == 0:
             return
         self.u.zero_()
+        if self.hybrid:
+            self.vgc.vgc_decode_accumulate_hybrid([self.out] + self.others, self.tau, 1.0 / self.W, self.u, self.status)
+            return
         self.vgc.vgc_decode_accumulate([self.out] + self.others, self.offs_dev, 1.0 / self.W, self.u, self.status)
 
     def step(self, t: int, marks=None):
@@ -532,6 +554,9 @@ def main():
     ap.add_argument("--streams", type=int, default=4, help="streams the independent sqgrad layers are spread over")
     ap.add_argument("--fused", action="store_true",
                     help="sqgrad adds its sums straight into v and vgc_compress runs without s (12 B read per parameter)")
+    ap.add_argument("--algorithm", default="basic", choices=["basic", "hybrid"],
+                    help="hybrid: Algorithm 2 (fixed threshold tau + variance criterion) for the compress and decode "
+                         "sections; device-timed only (no end-to-end or CPU leg)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -553,7 +578,9 @@ def main():
     vgc.load_library()
     pk = peaks()
     hp = HotPath(args.workload, worker=rank * 16, n_input_sets=1, n_g_sets=max(4, min(args.steps + args.warmup, 16)),
-                 n_params=args.n_params, n_streams=max(args.streams, 1))
+                 n_params=args.n_params, n_streams=max(args.streams, 1), algorithm=args.algorithm)
+    if hp.hybrid:
+        args.no_e2e = args.no_cpu_baseline = True
     hp.fused = args.fused
     torch.cuda.synchronize()
 
@@ -570,6 +597,8 @@ def main():
                                                       use_graph=not args.no_graph)
     clocks = sampler.stop()
     counters = hp.out.read()
+    if hp.hybrid:
+        counters.update(n_criterion=counters["nnz"], n_dropped=0)
     ms_per_step = total_ms / args.steps
     ms_per_step = max_over_ranks(ms_per_step, "cuda")
 
@@ -579,6 +608,8 @@ def main():
     nnz_a, nnz = counters["n_criterion"], counters["nnz"]
     sum_nnz = nnz + sum(int(o.words.numel()) for o in hp.others) if hp.W else 0
     compress_bytes = 24 * n + 8 * nnz_a + 4 * nnz
+    if hp.hybrid:                                          # the staged word is written, read and written again
+        compress_bytes = 24 * n + 12 * nnz
     # decode: 4 B per word + one read and one write of u (merge form) + the 4 B/element clearing of u before it
     decode_bytes = (4 * sum_nnz + 12 * n) if hp.W else 0
     sections = {
@@ -623,7 +654,7 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "f32 (tf32x3 products where tensor cores are used)",
             "data": "synthetic",
             "config": {"workload": args.workload, "n_params": n, "batch": hp.batch, "W": hp.W, "alpha": hp.alpha,
-                       "zeta": ZETA, "groups": hp.K, "launch": "eager" if args.no_graph else "cuda graph replay",
+                       "zeta": ZETA, "groups": hp.K, "algorithm": args.algorithm, "tau": hp.tau, "launch": "eager" if args.no_graph else "cuda graph replay",
                        "sqgrad_streams": getattr(hp, "n_streams", 1),
                        "fused_sqgrad_into_v": bool(args.fused),
                        "l2": "inputs larger than L2 (no flush)" if n * 16 > 126e6 else "state fits in L2 (no flush): cache-resident numbers"},

@@ -222,6 +222,49 @@ vgc_status vgc_step_host(const vgc_layer_host *layers, int n_layers, const float
                          uint32_t *counters_host, void *ws_sqgrad, size_t ws_sqgrad_bytes, void *ws_compress,
                          size_t ws_compress_bytes, vgc_stream_t stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * (4) Hybrid algorithm (Algorithm 2; Sec. 4.5): the variance criterion combined with the fixed
+ * threshold tau of Strom's method.  Per parameter, every operation one rounded fp32 operation:
+ *
+ *   r1 = r + g;  v1 = v + s
+ *   send = |r1| > tau  and  r1*r1 > alpha*v1          (both strict)
+ *   if send:  emit Sign(r1);  r2 = r1 - Sign(r1)*tau
+ *             v1 = max((v1 - (2*a)*tau) + tau*tau, 0)     a = |r1|, or |r2| when
+ *                                                          correction_from_updated_r != 0
+ *             r1 = r2
+ *   r = r1;  v = v1 * zeta                             (v decays at every step, sent or not)
+ *
+ * a = |r1| is the reading under which the correction is the "(a - b)^2" of Sec. 4.5 for a single
+ * sample (v - 2|r|tau + tau^2 = (|r| - tau)^2 when v = r^2); a = |r2| follows the order in which the
+ * listing of Algorithm 2 states the two updates.  The message carries no magnitudes: each 32-bit word
+ * is  index << 4 | sign << 3  (low three bits zero), ascending index -- the same container as the
+ * basic algorithm's words, a choice of this library (the paper does not print the hybrid's format).
+ *
+ *   s       may be NULL, as for vgc_compress (the squared sums were accumulated into v already)
+ *   out     DEVICE pointers: words [capacity], nnz [1], mask [n] or NULL (needs 4-byte alignment),
+ *           dev_status [1] (sticky; VGC_DEV_CAPACITY when more than capacity elements were sent: nnz
+ *           still counts them all, the first `capacity` words are valid, r and v are updated for all)
+ *   ws      DEVICE scratch of vgc_compress_hybrid_workspace_bytes(n) bytes, 16-byte aligned
+ * tau must be finite and >= 0; alpha, zeta as for vgc_compress.  Asynchronous on `stream`.
+ *
+ * vgc_decode_accumulate_hybrid:  u[idx] += scale * (-1)^sign * tau  for every word of every message
+ * (views' group_exp is not read and may be NULL); otherwise as vgc_decode_accumulate.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    uint32_t *words;       /* [capacity] out */
+    uint32_t capacity;
+    uint32_t *nnz;         /* [1] out: elements sent */
+    uint8_t *mask;         /* [n] out or NULL: 1 where the element was sent */
+    uint32_t *dev_status;  /* [1] sticky VGC_DEV_* bits */
+} vgc_hybrid_message;
+
+size_t vgc_compress_hybrid_workspace_bytes(size_t n);
+vgc_status vgc_compress_hybrid(const float *g, const float *s, float *r, float *v, size_t n, float alpha,
+                               float zeta, float tau, int correction_from_updated_r,
+                               const vgc_hybrid_message *out, void *ws, size_t ws_bytes, vgc_stream_t stream);
+vgc_status vgc_decode_accumulate_hybrid(const vgc_message_view *msgs, int W, float tau, float scale, float *u,
+                                        size_t n, uint32_t *dev_status, vgc_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -29,6 +29,7 @@ EXPORTS = [
     "vgc_sqgrad_conv_workspace_bytes", "vgc_sqgrad_conv",
     "vgc_compress_workspace_bytes", "vgc_compress", "vgc_compress_static",
     "vgc_decode_accumulate", "vgc_step_host",
+    "vgc_compress_hybrid_workspace_bytes", "vgc_compress_hybrid", "vgc_decode_accumulate_hybrid",
 ]
 
 
@@ -49,6 +50,11 @@ class _LayerHostStruct(ctypes.Structure):    # mirrors vgc_layer_host
                                                   "stride_w", "pad_h", "pad_w")] + \
                [("x_host", ctypes.c_void_p), ("delta_host", ctypes.c_void_p), ("x_dev", ctypes.c_void_p),
                 ("delta_dev", ctypes.c_void_p)]
+
+
+class _HybridMessageStruct(ctypes.Structure):    # mirrors vgc_hybrid_message
+    _fields_ = [("words", ctypes.c_void_p), ("capacity", ctypes.c_uint32), ("nnz", ctypes.c_void_p),
+                ("mask", ctypes.c_void_p), ("dev_status", ctypes.c_void_p)]
 
 
 class _ViewStruct(ctypes.Structure):         # mirrors vgc_message_view
@@ -90,6 +96,12 @@ def load_library():
     lib.vgc_step_host.restype = i
     lib.vgc_decode_accumulate.argtypes = [ctypes.POINTER(_ViewStruct), i, vp, i, f, vp, sz, vp, vp]
     lib.vgc_decode_accumulate.restype = i
+    lib.vgc_compress_hybrid_workspace_bytes.argtypes = [sz]
+    lib.vgc_compress_hybrid_workspace_bytes.restype = sz
+    lib.vgc_compress_hybrid.argtypes = [vp, vp, vp, vp, sz, f, f, f, i, ctypes.POINTER(_HybridMessageStruct), vp, sz, vp]
+    lib.vgc_compress_hybrid.restype = i
+    lib.vgc_decode_accumulate_hybrid.argtypes = [ctypes.POINTER(_ViewStruct), i, f, f, vp, sz, vp, vp]
+    lib.vgc_decode_accumulate_hybrid.restype = i
     _lib = lib
     return lib
 
@@ -284,6 +296,69 @@ def vgc_decode_accumulate(messages: Sequence, group_offsets, scale: float, u, de
                                               float(scale), _dev(u, torch.float32, "u"), u.numel(),
                                               _dev(dev_status, torch.int32, "dev_status"), _stream(stream))
     _check(st, "vgc_decode_accumulate")
+    return u
+
+
+# ------------------------------------------------------------------------------------------ (4)
+class HybridMessageBuffers:
+    """Device buffers behind a vgc_hybrid_message.  ``counters`` is int32[2]: nnz, dev_status."""
+
+    def __init__(self, capacity: int, n: int = 0, with_mask: bool = False, device="cuda"):
+        self.capacity = int(capacity)
+        self.words = torch.empty(max(self.capacity, 1), dtype=torch.int32, device=device)
+        self.counters = torch.zeros(2, dtype=torch.int32, device=device)
+        self.mask = torch.zeros(n, dtype=torch.uint8, device=device) if with_mask else None
+
+    def struct(self) -> _HybridMessageStruct:
+        c = self.counters.data_ptr()
+        return _HybridMessageStruct(self.words.data_ptr(), self.capacity, c,
+                                    self.mask.data_ptr() if self.mask is not None else None, c + 4)
+
+    def view(self) -> _ViewStruct:
+        return _ViewStruct(self.words.data_ptr(), self.counters.data_ptr(), None)
+
+    def read(self):
+        nnz, dev_status = (int(c) & 0xFFFFFFFF for c in self.counters.tolist())
+        return {"words": self.words[:min(nnz, self.capacity)].cpu().numpy().view("uint32"), "nnz": nnz,
+                "dev_status": dev_status, "mask": None if self.mask is None else self.mask.cpu().numpy()}
+
+
+def vgc_compress_hybrid_workspace_bytes(n: int) -> int:
+    return load_library().vgc_compress_hybrid_workspace_bytes(n)
+
+
+def vgc_compress_hybrid(g, s, r, v, alpha: float, zeta: float, tau: float, out: HybridMessageBuffers, ws,
+                        correction_from_updated_r: bool = False, stream=None):
+    """One step of Algorithm 2 over the flat buffer; r, v updated in place.  ``s=None`` as for vgc_compress."""
+    n = g.numel()
+    if (s is not None and s.numel() != n) or r.numel() != n or v.numel() != n:
+        raise ValueError("g, s, r, v must have the same length")
+    if out.mask is not None and out.mask.numel() != n:
+        raise ValueError("mask length")
+    wp, wb = _ws(ws)
+    msg = out.struct()
+    st = load_library().vgc_compress_hybrid(
+        _dev(g, torch.float32, "g"), None if s is None else _dev(s, torch.float32, "s"), _dev(r, torch.float32, "r"),
+        _dev(v, torch.float32, "v"), n, float(alpha), float(zeta), float(tau), int(bool(correction_from_updated_r)),
+        ctypes.byref(msg), wp, wb, _stream(stream))
+    _check(st, "vgc_compress_hybrid")
+    return out
+
+
+def vgc_decode_accumulate_hybrid(messages: Sequence, tau: float, scale: float, u, dev_status, stream=None):
+    """u[idx] += scale * (+-tau) over all words of all messages (HybridMessageBuffers or (words, nnz) pairs)."""
+    W = len(messages)
+    views = (_ViewStruct * max(W, 1))()
+    for w, m in enumerate(messages):
+        if isinstance(m, HybridMessageBuffers):
+            views[w] = m.view()
+        else:
+            words, nnz = m
+            views[w] = _ViewStruct(_dev(words, torch.int32, "words"), _dev(nnz, torch.int32, "nnz"), None)
+    st = load_library().vgc_decode_accumulate_hybrid(views, W, float(tau), float(scale), _dev(u, torch.float32, "u"),
+                                                     u.numel(), _dev(dev_status, torch.int32, "dev_status"),
+                                                     _stream(stream))
+    _check(st, "vgc_decode_accumulate_hybrid")
     return u
 
 

@@ -23,27 +23,34 @@ struct DecodeViews {
     const int32_t *group_exp[kMaxViews];
 };
 
+// kHybrid: messages of the hybrid algorithm (Algorithm 2) -- every word stands for +-tau, no exponents.
+template <bool kHybrid>
 __device__ __forceinline__ void decode_one(uint32_t word, const uint32_t *offs, const int32_t *gexp, int K,
-                                           int &k, float scale, float *u, size_t n, bool &bad)
+                                           int &k, float scale, float tau, float *u, size_t n, bool &bad)
 {
     const uint32_t idx = word >> 4;
     if (idx >= n) { bad = true; return; }
+    if (kHybrid) {
+        atomicAdd(u + idx, __fmul_rn(scale, (word & 8u) ? -tau : tau));
+        return;
+    }
     if (idx < offs[k] || idx >= offs[k + 1]) k = group_of(offs, K, idx);
     const int32_t e = gexp[k] - (int32_t)(word & 7u);
     const float value = __uint_as_float(((uint32_t)(e + 127) << 23) | ((word & 8u) << 28));
     atomicAdd(u + idx, __fmul_rn(scale, value));
 }
 
+template <bool kHybrid>
 __global__ void __launch_bounds__(kDecThreads)
 decode_scatter(const __grid_constant__ DecodeViews views, const uint32_t *__restrict__ group_offsets, int K,
-               float scale, float *__restrict__ u, size_t n, uint32_t *dev_status)
+               float scale, float tau, float *__restrict__ u, size_t n, uint32_t *dev_status)
 {
     __shared__ uint32_t sm_offs[kDecOffsSmem];
     __shared__ int32_t sm_exp[kDecOffsSmem];
     const int w = blockIdx.y;
     const uint32_t *__restrict__ words = views.words[w];
     const uint32_t count = *views.nnz[w];
-    const bool in_smem = (K + 1) <= kDecOffsSmem;
+    const bool in_smem = !kHybrid && (K + 1) <= kDecOffsSmem;
     if (in_smem) {
         for (int i = threadIdx.x; i <= K; i += kDecThreads) sm_offs[i] = group_offsets[i];
         for (int i = threadIdx.x; i < K; i += kDecThreads) sm_exp[i] = views.group_exp[w][i];
@@ -58,13 +65,13 @@ decode_scatter(const __grid_constant__ DecodeViews views, const uint32_t *__rest
     const uint32_t n_vec = vec_ok ? count / 4 : 0;
     for (uint32_t q = blockIdx.x * kDecThreads + threadIdx.x; q < n_vec; q += gridDim.x * kDecThreads) {
         const uint4 w4 = *reinterpret_cast<const uint4 *>(words + 4 * (size_t)q);
-        decode_one(w4.x, offs, gexp, K, k, scale, u, n, bad);
-        decode_one(w4.y, offs, gexp, K, k, scale, u, n, bad);
-        decode_one(w4.z, offs, gexp, K, k, scale, u, n, bad);
-        decode_one(w4.w, offs, gexp, K, k, scale, u, n, bad);
+        decode_one<kHybrid>(w4.x, offs, gexp, K, k, scale, tau, u, n, bad);
+        decode_one<kHybrid>(w4.y, offs, gexp, K, k, scale, tau, u, n, bad);
+        decode_one<kHybrid>(w4.z, offs, gexp, K, k, scale, tau, u, n, bad);
+        decode_one<kHybrid>(w4.w, offs, gexp, K, k, scale, tau, u, n, bad);
     }
     for (uint32_t q = 4 * n_vec + blockIdx.x * kDecThreads + threadIdx.x; q < count; q += gridDim.x * kDecThreads)
-        decode_one(words[q], offs, gexp, K, k, scale, u, n, bad);
+        decode_one<kHybrid>(words[q], offs, gexp, K, k, scale, tau, u, n, bad);
     if (bad) atomicOr(dev_status, VGC_DEV_RANGE);
 }
 
@@ -101,9 +108,10 @@ __device__ __forceinline__ uint32_t warp_lower_bound(const uint32_t *__restrict_
     return lo;
 }
 
+template <bool kHybrid>
 __global__ void __launch_bounds__(kDecThreads)
 decode_merge(const __grid_constant__ DecodeViews views, int W, const uint32_t *__restrict__ group_offsets, int K,
-             float scale, float *__restrict__ u, size_t n, uint32_t chunk_elems, uint32_t *dev_status)
+             float scale, float tau, float *__restrict__ u, size_t n, uint32_t chunk_elems, uint32_t *dev_status)
 {
     __shared__ __align__(16) float tile[kMergeTile];
     __shared__ uint32_t sm_offs[kDecOffsSmem];
@@ -111,7 +119,7 @@ decode_merge(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
     __shared__ uint32_t total_words;
 
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const bool in_smem = (K + 1) <= kDecOffsSmem;
+    const bool in_smem = !kHybrid && (K + 1) <= kDecOffsSmem;
     if (in_smem)
         for (int i = threadIdx.x; i <= K; i += kDecThreads) sm_offs[i] = group_offsets[i];
     const uint32_t *offs = in_smem ? sm_offs : group_offsets;
@@ -140,6 +148,7 @@ decode_merge(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
     if (total == 0) return;
 
     auto value_of = [&](uint32_t word, const int32_t *gexp, int &k) -> float {
+        if (kHybrid) return __fmul_rn(scale, (word & 8u) ? -tau : tau);
         const uint32_t idx = word >> 4;
         if (idx < offs[k] || idx >= offs[k + 1]) k = group_of(offs, K, idx);
         const int32_t e = gexp[k] - (int32_t)(word & 7u);
@@ -193,8 +202,11 @@ decode_merge(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
     for (size_t t0 = lo; t0 < hi; t0 += kMergeTile) {
         const uint32_t t_len = (uint32_t)(hi - t0 < kMergeTile ? hi - t0 : kMergeTile);
         const uint32_t t_hi = (uint32_t)(t0 + t_len);
-        int tile_group = group_of(offs, K, (uint32_t)t0);    // weight tensor of the tile, -1 if it spans several
-        if (t_hi - 1 >= offs[tile_group + 1]) tile_group = -1;
+        int tile_group = -1;                                  // weight tensor of the tile, -1 if it spans several
+        if (!kHybrid) {
+            tile_group = group_of(offs, K, (uint32_t)t0);
+            if (t_hi - 1 >= offs[tile_group + 1]) tile_group = -1;
+        }
 #pragma unroll
         for (int q = 0; q < kVec; ++q) reinterpret_cast<float4 *>(tile)[threadIdx.x + q * kDecThreads] = ahead[q];
         if (t0 + kMergeTile < hi) fetch_tile(t0 + kMergeTile);
@@ -293,17 +305,10 @@ decode_merge(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
 
 using namespace vgc;
 
-extern "C" vgc_status vgc_decode_accumulate(const vgc_message_view *msgs, int W,
-                                            const uint32_t *group_offsets, int K, float scale,
-                                            float *u, size_t n, uint32_t *dev_status, vgc_stream_t stream)
+namespace {
+vgc_status decode_launch(bool hybrid, const vgc_message_view *msgs, int W, const uint32_t *group_offsets, int K,
+                         float scale, float tau, float *u, size_t n, uint32_t *dev_status, cudaStream_t st)
 {
-    if (W == 0 || n == 0) return VGC_OK;
-    if (W < 0 || K < 1 || n > VGC_MAX_PARAMS || !msgs || !group_offsets || !u || !dev_status || !aligned16(u))
-        return VGC_ERR_INVALID_ARG;
-    if (!(scale == scale)) return VGC_ERR_INVALID_ARG;
-    for (int w = 0; w < W; ++w)
-        if (!msgs[w].words || !msgs[w].nnz || !msgs[w].group_exp) return VGC_ERR_INVALID_ARG;
-
     static int sm_count = 0;
     if (sm_count == 0) {
         int dev = 0, c = 0;
@@ -311,7 +316,6 @@ extern "C" vgc_status vgc_decode_accumulate(const vgc_message_view *msgs, int W,
         VGC_CUDA_OK(cudaDeviceGetAttribute(&c, cudaDevAttrMultiProcessorCount, dev));
         sm_count = c > 0 ? c : 148;
     }
-    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     for (int w0 = 0; w0 < W; w0 += kMaxViews) {
         const int wb = W - w0 < kMaxViews ? W - w0 : kMaxViews;
         DecodeViews views;
@@ -326,17 +330,50 @@ extern "C" vgc_status vgc_decode_accumulate(const vgc_message_view *msgs, int W,
             int per_msg = (sm_count * 8 + wb - 1) / wb;          // ~8 blocks per SM in total
             if (per_msg < 1) per_msg = 1;
             dim3 grid((unsigned)per_msg, (unsigned)wb);
-            decode_scatter<<<grid, kDecThreads, 0, st>>>(views, group_offsets, K, scale, u, n, dev_status);
+            if (hybrid)
+                decode_scatter<true><<<grid, kDecThreads, 0, st>>>(views, group_offsets, K, scale, tau, u, n, dev_status);
+            else
+                decode_scatter<false><<<grid, kDecThreads, 0, st>>>(views, group_offsets, K, scale, tau, u, n, dev_status);
         } else {
             // one chunk per block, four blocks per SM (all resident at once), whole tiles per chunk
             size_t chunk = (n + (size_t)sm_count * 4 - 1) / ((size_t)sm_count * 4);
             chunk = (chunk + kMergeTile - 1) / kMergeTile * kMergeTile;
             const unsigned blocks = (unsigned)((n + chunk - 1) / chunk);
-            decode_merge<<<blocks, kDecThreads, 0, st>>>(views, wb, group_offsets, K, scale, u, n, (uint32_t)chunk,
-                                                          dev_status);
+            if (hybrid)
+                decode_merge<true><<<blocks, kDecThreads, 0, st>>>(views, wb, group_offsets, K, scale, tau, u, n,
+                                                                    (uint32_t)chunk, dev_status);
+            else
+                decode_merge<false><<<blocks, kDecThreads, 0, st>>>(views, wb, group_offsets, K, scale, tau, u, n,
+                                                                     (uint32_t)chunk, dev_status);
         }
         count_launch();
     }
     VGC_CUDA_OK(cudaGetLastError());
     return VGC_OK;
+}
+}  // namespace
+
+extern "C" vgc_status vgc_decode_accumulate(const vgc_message_view *msgs, int W,
+                                            const uint32_t *group_offsets, int K, float scale,
+                                            float *u, size_t n, uint32_t *dev_status, vgc_stream_t stream)
+{
+    if (W == 0 || n == 0) return VGC_OK;
+    if (W < 0 || K < 1 || n > VGC_MAX_PARAMS || !msgs || !group_offsets || !u || !dev_status || !aligned16(u))
+        return VGC_ERR_INVALID_ARG;
+    if (!(scale == scale)) return VGC_ERR_INVALID_ARG;
+    for (int w = 0; w < W; ++w)
+        if (!msgs[w].words || !msgs[w].nnz || !msgs[w].group_exp) return VGC_ERR_INVALID_ARG;
+    return decode_launch(false, msgs, W, group_offsets, K, scale, 0.f, u, n, dev_status,
+                         reinterpret_cast<cudaStream_t>(stream));
+}
+
+extern "C" vgc_status vgc_decode_accumulate_hybrid(const vgc_message_view *msgs, int W, float tau, float scale,
+                                                   float *u, size_t n, uint32_t *dev_status, vgc_stream_t stream)
+{
+    if (W == 0 || n == 0) return VGC_OK;
+    if (W < 0 || n > VGC_MAX_PARAMS || !msgs || !u || !dev_status || !aligned16(u)) return VGC_ERR_INVALID_ARG;
+    if (!(scale == scale) || !(tau == tau)) return VGC_ERR_INVALID_ARG;
+    for (int w = 0; w < W; ++w)
+        if (!msgs[w].words || !msgs[w].nnz) return VGC_ERR_INVALID_ARG;
+    return decode_launch(true, msgs, W, nullptr, 0, scale, tau, u, n, dev_status, reinterpret_cast<cudaStream_t>(stream));
 }
