@@ -13,7 +13,7 @@ vgc_status simt_sqgrad_conv(const float *x, const float *delta, int B, int C, in
 bool tc_linear_supported(int B, int in, int out);
 bool tc_conv_supported(int B, int C, int H, int W, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw);
 size_t tc_linear_workspace_bytes(int B, int in, int out);
-size_t tc_conv_workspace_bytes(int B, int C, int Kh, int Kw, int P, int Cout);
+size_t tc_conv_workspace_bytes(int B, int C, int Kh, int Kw, int sh, int sw, int ph, int pw, int P, int Cout);
 vgc_status tc_sqgrad_linear(const float *x, const float *delta, int B, int in, int out, float scale, int accumulate,
                             float *S, void *ws, size_t ws_bytes, cudaStream_t st);
 vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int H, int W, int Cout, int Kh, int Kw,
@@ -77,7 +77,7 @@ extern "C" size_t vgc_sqgrad_conv_workspace_bytes(int B, int C, int H, int W, in
     if (B == 0 || C == 0 || Cout == 0) return 0;
     size_t need = simt_workspace_bytes(Cout, C * Kh * Kw, B * Ho * Wo);
     if (tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w)) {
-        const size_t t = tc_conv_workspace_bytes(B, C, Kh, Kw, Ho * Wo, Cout);
+        const size_t t = tc_conv_workspace_bytes(B, C, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho * Wo, Cout);
         need = need > t ? need : t;
     }
     return round_up(need + 256, 256);

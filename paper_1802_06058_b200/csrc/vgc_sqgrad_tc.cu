@@ -853,11 +853,96 @@ vgc_status tc_sqgrad_linear(const float *x, const float *delta, int B, int in, i
 // Cout <= 64: the im2col rows take the 128-row A tile and the errors the narrow B tile
 static bool conv_swapped(int Cout, int n_im2col) { return Cout <= 64 && n_im2col > Cout; }
 
-size_t tc_conv_workspace_bytes(int B, int C, int Kh, int Kw, int P, int Cout)
+// ---- repacking pre-pass for 1x1 convolutions whose tiles TMA cannot address in place ----------
+// A strided 1x1 convolution reads every (sh, sw)-th input position, and planes of P positions with P not
+// a multiple of 4 (7x7) have a row pitch TMA does not accept.  One small copy kernel per operand puts
+// them into a layout the TMA-fed kernel takes:
+//   kRepackPlanes   x_s[z][c][p] = x[z][c][(p / Wo) sh][(p % Wo) sw]: the input subsampled, examples kept
+//                   apart (the errors are used where they are)
+//   kRepackFlat     x_r[c][z P + p], d_r[o][z P + p]: channel-major, the (example, position) pairs of one
+//                   channel back to back -- the layer becomes a 1x1 convolution over ONE example with
+//                   B P positions, and its reduction has no per-example padding to whole slices
+enum { kRepackNone = 0, kRepackPlanes = 1, kRepackFlat = 2 };
+
+static int repack_mode(int B, int C, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw, int P)
+{
+    if (Kh != 1 || Kw != 1 || ph != 0 || pw != 0) return kRepackNone;
+    if ((long)B * C >= (1L << 31) || (long)B * Cout >= (1L << 31)) return kRepackNone;      // 32-bit row index
+    const char *e = getenv("VGC_TC_REPACK");
+    if (e && atoi(e) == 0) return kRepackNone;
+    const bool planes_ok = P >= kBK && P % 4 == 0;
+    if (planes_ok) return (sh > 1 || sw > 1) ? kRepackPlanes : kRepackNone;
+    const long flat = (long)B * P;
+    return (flat >= kBK && flat % 4 == 0 && flat < (1L << 30)) ? kRepackFlat : kRepackNone;
+}
+
+// out[a][b][p] = in[z][c][(p / Wo) sh W + (p % Wo) sw] with (a, b) = (z, c), or (c, z) when channel_major.
+// One warp per group of four rows of P positions (rows of the output are contiguous), lanes along p, eight
+// loads in flight per lane.
+__global__ void __launch_bounds__(256)
+sqgrad_repack(const float *__restrict__ in, float *__restrict__ out, int B, int C, int HW, int W, int Wo, int P,
+              int sh, int sw, int channel_major)
+{
+    constexpr int kRows = 4, kCols = 2;
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t rows = (uint32_t)B * (uint32_t)C;
+    const bool dense = sh == 1 && sw == 1 && W == Wo;                 // the plane is copied as it is
+    for (uint32_t row0 = (blockIdx.x * 8 + (threadIdx.x >> 5)) * kRows; row0 < rows; row0 += gridDim.x * 8 * kRows) {
+        const float *src[kRows];
+#pragma unroll
+        for (int r = 0; r < kRows; ++r) {
+            const uint32_t row = row0 + r < rows ? row0 + r : rows - 1;
+            uint32_t z, c;
+            if (channel_major) { c = row / (uint32_t)B; z = row - c * (uint32_t)B; }
+            else               { z = row / (uint32_t)C; c = row - z * (uint32_t)C; }
+            src[r] = in + ((size_t)z * C + c) * HW;
+        }
+        for (uint32_t p0 = 0; p0 < (uint32_t)P; p0 += 32 * kCols) {
+            float v[kRows][kCols];
+            uint32_t off[kCols];
+#pragma unroll
+            for (int u = 0; u < kCols; ++u) {
+                const uint32_t p = p0 + lane + 32u * u;
+                if (dense) off[u] = p;
+                else { const uint32_t ho = p / (uint32_t)Wo, wo = p - ho * (uint32_t)Wo; off[u] = ho * sh * W + wo * sw; }
+            }
+#pragma unroll
+            for (int r = 0; r < kRows; ++r)
+#pragma unroll
+                for (int u = 0; u < kCols; ++u)
+                    v[r][u] = (p0 + lane + 32u * u < (uint32_t)P) ? __ldg(src[r] + off[u]) : 0.f;
+#pragma unroll
+            for (int r = 0; r < kRows; ++r)
+#pragma unroll
+                for (int u = 0; u < kCols; ++u) {
+                    const uint32_t p = p0 + lane + 32u * u;
+                    if (row0 + r < rows && p < (uint32_t)P) out[(size_t)(row0 + r) * P + p] = v[r][u];
+                }
+        }
+    }
+}
+
+static size_t conv_workspace_plain(int B, int C, int Kh, int Kw, int P, int Cout)
 {
     const int n_im2col = C * Kh * Kw, k_slices = B * ((P + kBK - 1) / kBK);
     return conv_swapped(Cout, n_im2col) ? tc_workspace_bytes(n_im2col, Cout, k_slices)
                                         : tc_workspace_bytes(Cout, n_im2col, k_slices);
+}
+
+size_t tc_conv_workspace_bytes(int B, int C, int Kh, int Kw, int sh, int sw, int ph, int pw, int P, int Cout)
+{
+    // the larger of the in-place form and the repacked one, so that either can be chosen at call time
+    size_t need = conv_workspace_plain(B, C, Kh, Kw, P, Cout);
+    const int mode = repack_mode(B, C, Cout, Kh, Kw, sh, sw, ph, pw, P);
+    if (mode == kRepackPlanes) {
+        const size_t r = round_up(conv_workspace_plain(B, C, 1, 1, P, Cout), 256) + sizeof(float) * (size_t)B * C * P;
+        need = need > r ? need : r;
+    } else if (mode == kRepackFlat) {
+        const size_t r = round_up(conv_workspace_plain(1, C, 1, 1, B * P, Cout), 256) +
+                         round_up(sizeof(float) * (size_t)B * C * P, 256) + sizeof(float) * (size_t)B * Cout * P;
+        need = need > r ? need : r;
+    }
+    return need;
 }
 
 vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int H, int W, int Cout, int Kh, int Kw,
@@ -865,6 +950,27 @@ vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int 
                           void *ws, size_t ws_bytes, cudaStream_t st)
 {
     const int P = Ho * Wo, n_im2col = C * Kh * Kw;
+    const int mode = repack_mode(B, C, Cout, Kh, Kw, sh, sw, ph, pw, P);
+    if (mode != kRepackNone) {
+        const bool flat = mode == kRepackFlat;
+        const size_t inner = round_up(flat ? conv_workspace_plain(1, C, 1, 1, B * P, Cout)
+                                           : conv_workspace_plain(B, C, 1, 1, P, Cout), 256);
+        const size_t x_bytes = round_up(sizeof(float) * (size_t)B * C * P, 256);
+        const size_t d_bytes = flat ? sizeof(float) * (size_t)B * Cout * P : 0;
+        if (ws_bytes < inner + x_bytes + d_bytes) return VGC_ERR_WORKSPACE;
+        float *x_r = reinterpret_cast<float *>(static_cast<char *>(ws) + inner);
+        float *d_r = reinterpret_cast<float *>(static_cast<char *>(ws) + inner + x_bytes);
+        // one warp per row; a few rows per warp when there are many
+        auto blocks_for = [](size_t rows) { const size_t b = (rows + 31) / 32; return (unsigned)(b < 1 ? 1 : (b > 148 * 32 ? 148 * 32 : b)); };
+        sqgrad_repack<<<blocks_for((size_t)B * C), 256, 0, st>>>(x, x_r, B, C, H * W, W, Wo, P, sh, sw, flat ? 1 : 0);
+        count_launch();
+        if (flat) {
+            sqgrad_repack<<<blocks_for((size_t)B * Cout), 256, 0, st>>>(delta, d_r, B, Cout, P, Wo, Wo, P, 1, 1, 1);
+            count_launch();
+            return tc_sqgrad_conv(x_r, d_r, 1, C, B * P, 1, Cout, 1, 1, 1, 1, 0, 0, B * P, 1, scale, accumulate, S, ws, inner, st);
+        }
+        return tc_sqgrad_conv(x_r, delta, B, C, Ho, Wo, Cout, 1, 1, 1, 1, 0, 0, Ho, Wo, scale, accumulate, S, ws, inner, st);
+    }
     // VGC_TC_GATHER (bit 0: error tile, bit 1: input tile) forces the gathered form of a tile and
     // VGC_TC_ATMEM=0 keeps the A operand in shared memory: every variant computes the same thing, the
     // switches exist so that tests can reach each of them on any shape.

@@ -77,7 +77,11 @@ CONV_SHAPES = [  # B, C, H, Cout, k, stride, pad
     # 1x1 / stride 1 / no padding: the tensor-core path (whole and ragged tiles, split reductions)
     (2, 64, 8, 64, 1, 1, 0), (3, 256, 14, 64, 1, 1, 0), (2, 100, 12, 200, 1, 1, 0), (4, 64, 56, 64, 1, 1, 0),
     (2, 8, 6, 8, 1, 1, 0), (5, 300, 10, 136, 1, 1, 0),
+    # 1x1 layers that are repacked first: 7x7 planes (channel-major, flat reduction), strided (subsampled planes)
+    (4, 70, 7, 130, 1, 1, 0), (4, 48, 14, 200, 1, 2, 0), (2, 96, 16, 160, 1, 2, 0), (3, 64, 28, 40, 1, 2, 0),
+    (32, 160, 7, 144, 1, 1, 0),
 ]
+REPACKED = [(4, 70, 7, 130, 1, 1, 0), (4, 48, 14, 200, 1, 2, 0), (2, 96, 16, 160, 1, 2, 0), (3, 64, 28, 40, 1, 2, 0)]
 
 
 @pytest.mark.parametrize("B,C,H,Cout,k,s,p", CONV_SHAPES)
@@ -113,6 +117,22 @@ def test_long_reduction_all_ones_is_exact():
     x = torch.ones(2, 8, 224, 224, device="cuda"); d = torch.ones(2, 16, 224, 224, device="cuda")
     got = run_conv(x, d, 1, 1, 0, 1.0)                      # tensor-core path
     assert np.all(got == 2 * 224 * 224)
+
+
+@pytest.mark.parametrize("B,C,H,Cout,k,s,p", REPACKED)
+def test_repacked_and_in_place_forms_agree_with_the_oracle(monkeypatch, B, C, H, Cout, k, s, p):
+    gen = torch.Generator(device="cuda"); gen.manual_seed(C + H)
+    Ho = (H + 2 * p - k) // s + 1
+    x = torch.randn(B, C, H, H, device="cuda", generator=gen)
+    d = torch.randn(B, Cout, Ho, Ho, device="cuda", generator=gen) * 1e-3
+    want = oracle.sqgrad_conv(x.cpu().numpy(), d.cpu().numpy(), (k, k), (s, s), (p, p), scale=0.5)
+    S0 = torch.rand(Cout, C, k, k, device="cuda")
+    want_acc = S0.cpu().numpy().copy()
+    oracle.sqgrad_conv(x.cpu().numpy(), d.cpu().numpy(), (k, k), (s, s), (p, p), scale=0.5, out=want_acc)
+    for repack in ("1", "0"):
+        monkeypatch.setenv("VGC_TC_REPACK", repack)
+        _check(run_conv(x, d, k, s, p, 0.5), want)
+        _check(run_conv(x, d, k, s, p, 0.5, S0=S0), want_acc)
 
 
 @pytest.mark.parametrize("env", [{"VGC_TC_ATMEM": "0"}, {"VGC_TC_GATHER": "1"}, {"VGC_TC_GATHER": "2"},
