@@ -351,7 +351,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         abort_flag = 0;
         for (int i = 0; i < kRawSlots; ++i) {
             mbar_init(smem_u32(&raw_full[i]), 1);
-            mbar_init(smem_u32(&op_full[i]), kTransformWarps);
+            mbar_init(smem_u32(&op_full[i]), kAnyGather ? kTransformWarps : kTransformWarps / 2);
             mbar_init(smem_u32(&empty[i]), 1);
         }
         for (int i = 0; i < kLoSlotsAT; ++i) mbar_init(smem_u32(&lo_empty[i]), 1);
@@ -462,6 +462,12 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     } else if (warp < 2 + kTransformWarps) {
         // ================= transform warps: square and split into TF32 hi / lo =================
         const int t = (int)threadIdx.x - 64;                               // 0..255
+        // With nothing to gather the eight warps work as two groups of four that take alternate slices: the
+        // waits, fences and tensor-memory stores of one slice then overlap the arithmetic of the next one.
+        constexpr bool kTwoGroups = !kAnyGather;
+        constexpr int kTT = kTwoGroups ? kTransformThreads / 2 : kTransformThreads;   // threads sharing a slice
+        const int group = kTwoGroups ? (t >> 7) : 0;
+        const int tt = kTwoGroups ? (t & 127) : t;
         const int kq = t & 7, row0 = t >> 3;                               // gathered chunks: rows row0 + 32*i, k = 4*kq..4*kq+3
         GatherRows<kModeA> rows_a;
         GatherRows<kModeB> rows_b;
@@ -496,41 +502,51 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             // one A tile below the slot so that the same chunk offsets address the B part)
             uint8_t *lo = smem_gen + kLoBase + ls * kLoBytes - (kATmem ? kRawBytesA : 0);
             if (kATmem) {
-                // A: this thread's row (TMEM lane) and half of the slice's 32 k -> hi / lo straight into TMEM
+                // A: this thread's row (TMEM lane) and 16 of the slice's 32 k at a time -> hi / lo straight into
+                // TMEM (a warp of the two-group form takes both halves, otherwise its group number picks one)
                 tc_fence_after();
-                const uint32_t q = warp & 3, h = (warp - 2) >> 2;
+                const uint32_t q = warp & 3;
                 const int m_local = (int)(q * 32 + lane);
                 const uint8_t *arow = hi + m_local * 128;
-                float4 c4[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) c4[u] = *reinterpret_cast<const float4 *>(arow + (((4 * h + u) ^ (m_local & 7)) << 4));
-                uint32_t h16[16], l16[16];
+                for (int hh = 0; hh < (kTwoGroups ? 2 : 1); ++hh) {
+                    const uint32_t h = kTwoGroups ? (uint32_t)hh : (warp - 2) >> 2;
+                    float4 c4[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const float e[4] = {c4[u].x, c4[u].y, c4[u].z, c4[u].w};
+                    for (int u = 0; u < 4; ++u)
+                        c4[u] = *reinterpret_cast<const float4 *>(arow + (((4 * h + u) ^ (m_local & 7)) << 4));
+                    uint32_t h16[16], l16[16];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float sq = __fmul_rn(e[j], e[j]);
-                        h16[4 * u + j] = to_tf32(sq);
-                        l16[4 * u + j] = __float_as_uint(__fsub_rn(sq, __uint_as_float(h16[4 * u + j])));
+                    for (int u = 0; u < 4; ++u) {
+                        const float e[4] = {c4[u].x, c4[u].y, c4[u].z, c4[u].w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float sq = __fmul_rn(e[j], e[j]);
+                            h16[4 * u + j] = to_tf32(sq);
+                            l16[4 * u + j] = __float_as_uint(__fsub_rn(sq, __uint_as_float(h16[4 * u + j])));
+                        }
                     }
+                    const uint32_t taddr = tmem_base + ((q * 32u) << 16) + 2 * kBN + ls * kTmemColsA + 16 * h;
+                    tc_st_32x16(taddr, h16);
+                    tc_st_32x16(taddr + 32, l16);
                 }
-                const uint32_t taddr = tmem_base + ((q * 32u) << 16) + 2 * kBN + ls * kTmemColsA + 16 * h;
-                tc_st_32x16(taddr, h16);
-                tc_st_32x16(taddr + 32, l16);
             }
             if (kAnyTma) {      // tiles that came by TMA: elementwise, in place, over their 16-byte chunks
                 constexpr uint32_t c_begin = (kGatherA || kATmem) ? kRawBytesA / 16 : 0;
                 constexpr uint32_t c_end = kGatherB ? kRawBytesA / 16 : kRawStageBytes / 16;
-                constexpr int kPerThread = c_end > c_begin ? (c_end - c_begin) / kTransformThreads : 1;
+                constexpr int kPerThread = c_end > c_begin ? (c_end - c_begin) / kTT : 1;
+                constexpr int kBatch = kPerThread < 4 ? kPerThread : 4;              // chunks in registers at a time
                 if (c_end > c_begin) {
-                    float4 v[kPerThread];
 #pragma unroll
-                    for (int u = 0; u < kPerThread; ++u)
-                        v[u] = *reinterpret_cast<const float4 *>(hi + 16 * (c_begin + (uint32_t)t + u * kTransformThreads));
+                    for (int u0 = 0; u0 < kPerThread; u0 += kBatch) {
+                        float4 v[kBatch];
 #pragma unroll
-                    for (int u = 0; u < kPerThread; ++u)
-                        split_store(hi, lo, 16 * (c_begin + (uint32_t)t + u * kTransformThreads), v[u].x, v[u].y, v[u].z, v[u].w);
+                        for (int u = 0; u < kBatch; ++u)
+                            v[u] = *reinterpret_cast<const float4 *>(hi + 16 * (c_begin + (uint32_t)tt + (u0 + u) * kTT));
+#pragma unroll
+                        for (int u = 0; u < kBatch; ++u)
+                            split_store(hi, lo, 16 * (c_begin + (uint32_t)tt + (u0 + u) * kTT), v[u].x, v[u].y, v[u].z, v[u].w);
+                    }
                 }
             }
             if (kGatherA) {
@@ -554,6 +570,10 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         // two register sets in turn: the loads of slice i+1 are in flight while slice i is transformed
         float a0[kRowsPerThread][4], b0[kRowsPerThread][4], a1[kRowsPerThread][4], b1[kRowsPerThread][4];
         if (kAnyGather) gather(a0, b0);
+        if (kTwoGroups) {
+            for (int i = group; i < n_slices; i += 2)
+                if (!process(i, a0, b0)) break;
+        } else
         for (int i = 0; i < n_slices; i += 2) {
             if (kAnyGather && i + 1 < n_slices) { advance(); gather(a1, b1); }
             if (!process(i, a0, b0)) break;
