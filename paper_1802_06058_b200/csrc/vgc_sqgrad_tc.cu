@@ -67,6 +67,11 @@ constexpr uint32_t kSmemBytes = (kRawSlots + kLoSlots) * kRawStageBytes + 1024 /
 // With the A operand in tensor memory a lo slot holds the B tile only, so twice as many fit; the A
 // operand ring in TMEM has the same number of slots and shares their barrier.
 constexpr int kLoSlotsAT = 2 * kLoSlots;
+// Pure TMA form with A in tensor memory ("split rings"): the raw A tile is dead as soon as the transform has
+// read it, long before the MMAs of its slice retire.  It therefore gets a ring of its own that is freed
+// early, and the 16-KB units this saves hold more B tiles: more slices in flight from the same shared memory.
+constexpr int kSplitA = 4, kSplitB = 7, kSplitLo = 3;              // 16-KB units: A raw, B raw/hi, B lo (+ A in TMEM)
+static_assert((kSplitA + kSplitB + kSplitLo) * kRawBytesA <= (kRawSlots + kLoSlots) * kRawStageBytes, "smem budget");
 constexpr uint32_t kTmemColsA = 64;                                 // per slot: 32 columns hi + 32 columns lo
 constexpr uint32_t kTmemCols = 512;                                 // two accumulator buffers + the A operand ring
 constexpr uint32_t kWaitLimit = 1u << 22;                           // polls before a wait gives up
@@ -82,6 +87,7 @@ struct Params {
     int p_slices;            // conv: slices per example (ceil(P/32)); dense: 1
     int chunk;               // slices per accumulator drain
     uint32_t tx_bytes;       // bytes the TMA loads of one slice deliver
+    uint32_t tx_bytes_a;     // of which the A tile's
     float scale;
     int accumulate;
     const float *x, *delta;  // raw operands (gathered tiles)
@@ -318,14 +324,23 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 {
     static_assert(kMajor == kMajorK || (kModeA == kTma && kModeB == kTma), "gathered tiles are K-major");
     static_assert(!kATmem || (kMajor == kMajorK && kModeA == kTma), "A goes to tensor memory from a K-major TMA tile");
-    constexpr int kLoN = kATmem ? kLoSlotsAT : kLoSlots;                  // lo slots (and A operand slots in TMEM)
-    constexpr uint32_t kLoBytes = kATmem ? kRawBytesB : kRawStageBytes;  // bytes of one lo slot
     constexpr bool kGatherA = kModeA != kTma, kGatherB = kModeB != kTma;
     constexpr bool kAnyTma = !kGatherA || !kGatherB;
     constexpr bool kAnyGather = kGatherA || kGatherB;
+    constexpr bool kSplit = kATmem && !kAnyGather;                         // A raw tiles in a ring of their own
+    constexpr int kNB = kSplit ? kSplitB : kRawSlots;                      // slots of the raw / hi ring
+    constexpr int kLoN = kSplit ? kSplitLo : (kATmem ? kLoSlotsAT : kLoSlots);   // lo slots (and A slots in TMEM)
+    constexpr uint32_t kLoBytes = kATmem ? kRawBytesB : kRawStageBytes;  // bytes of one lo slot
+    // byte offsets of slot s: the [A][B] pair of the raw / hi ring (split form: only its B half exists, the
+    // offset points one A tile below it), the lo ring likewise, and the split form's A ring
+    auto pair_off = [](int s) -> uint32_t { return kSplit ? (uint32_t)(kSplitA + s - 1) * kRawBytesA : (uint32_t)s * kRawStageBytes; };
+    auto lo_off = [](int s) -> uint32_t {
+        return kSplit ? (uint32_t)(kSplitA + kSplitB + s - 1) * kRawBytesA
+                      : kLoBase + (uint32_t)s * kLoBytes - (kATmem ? kRawBytesA : 0u);
+    };
 
     extern __shared__ uint8_t smem_raw_[];
-    __shared__ __align__(8) uint64_t bars[3 * kRawSlots + kLoSlotsAT + 5];
+    __shared__ __align__(8) uint64_t bars[3 * kSplitB + kLoSlotsAT + 5 + 2 * kSplitA];
     __shared__ uint32_t tmem_base_slot;
     __shared__ volatile uint32_t abort_flag;
 
@@ -335,9 +350,10 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 
     // per raw slot: raw_full (TMA landed) -> op_full (hi/lo written) -> empty (MMAs that read it retired);
     // per lo slot: lo_empty (MMAs that read it retired)
-    uint64_t *raw_full = bars, *op_full = bars + kRawSlots, *empty = bars + 2 * kRawSlots;
-    uint64_t *lo_empty = bars + 3 * kRawSlots;
+    uint64_t *raw_full = bars, *op_full = bars + kNB, *empty = bars + 2 * kNB;
+    uint64_t *lo_empty = bars + 3 * kNB;
     uint64_t *acc_full = lo_empty + kLoSlotsAT, *acc_empty = acc_full + 2, *drain = acc_empty + 2;
+    uint64_t *a_full = drain + 1, *a_empty = a_full + kSplitA;             // split form: the A ring
 
     const int m0 = blockIdx.y * kBM, n0 = blockIdx.x * kBN;
     const int n_valid = min(kBN, prm.N - n0);                              // columns of this tile that exist
@@ -349,11 +365,16 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        for (int i = 0; i < kRawSlots; ++i) {
+        for (int i = 0; i < kNB; ++i) {
             mbar_init(smem_u32(&raw_full[i]), 1);
             mbar_init(smem_u32(&op_full[i]), kAnyGather ? kTransformWarps : kTransformWarps / 2);
             mbar_init(smem_u32(&empty[i]), 1);
         }
+        if (kSplit)
+            for (int i = 0; i < kSplitA; ++i) {
+                mbar_init(smem_u32(&a_full[i]), 1);
+                mbar_init(smem_u32(&a_empty[i]), kTransformWarps / 2);
+            }
         for (int i = 0; i < kLoSlotsAT; ++i) mbar_init(smem_u32(&lo_empty[i]), 1);
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&acc_full[i]), 1); mbar_init(smem_u32(&acc_empty[i]), kEpilogueWarps); }
         mbar_init(smem_u32(drain), 1);
@@ -375,13 +396,25 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         if (lane == 0 && kAnyTma) {
             int issued = 0;
             for (int i = 0; i < n_slices; ++i) {
-                const int st = i % kRawSlots;
-                const uint32_t ph = (uint32_t)(i / kRawSlots) & 1u;
+                const int st = i % kNB;
+                const uint32_t ph = (uint32_t)(i / kNB) & 1u;
                 if (!mbar_wait(smem_u32(&empty[st]), ph ^ 1u, &abort_flag, 64)) break;
                 const uint32_t full = smem_u32(&raw_full[st]);
-                const uint32_t dst_a = smem_base + st * kRawStageBytes, dst_b = dst_a + kRawBytesA;
-                mbar_expect_tx(full, prm.tx_bytes);
+                const uint32_t dst_a = smem_base + pair_off(st), dst_b = dst_a + kRawBytesA;
                 const int slice = slice_begin + i;
+                if (kSplit) {
+                    const int sa = i % kSplitA;
+                    if (!mbar_wait(smem_u32(&a_empty[sa]), ((uint32_t)(i / kSplitA) & 1u) ^ 1u, &abort_flag, 64)) break;
+                    const uint32_t full_a = smem_u32(&a_full[sa]);
+                    const int z = slice / prm.p_slices, p0 = (slice - z * prm.p_slices) * kBK;
+                    mbar_expect_tx(full_a, prm.tx_bytes_a);
+                    tma_load_3d(smem_base + (uint32_t)sa * kRawBytesA, &map_a, full_a, p0, m0, z);
+                    mbar_expect_tx(full, prm.tx_bytes - prm.tx_bytes_a);
+                    tma_load_3d(dst_b, &map_b, full, p0, n0, z);
+                    issued = i + 1;
+                    continue;
+                }
+                mbar_expect_tx(full, prm.tx_bytes);
                 if (kMajor == kMajorK) {
                     const int z = slice / prm.p_slices, p0 = (slice - z * prm.p_slices) * kBK;
                     if (!kGatherA) tma_load_3d(dst_a, &map_a, full, p0, m0, z);
@@ -397,11 +430,19 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             }
             // on an abort: loads already issued must land before the block may exit
             if (abort_flag) {
-                const int first = issued > kRawSlots ? issued - kRawSlots : 0;
+                const int first = issued > kNB ? issued - kNB : 0;
                 for (int i = first; i < issued; ++i) {
-                    const uint32_t bar = smem_u32(&raw_full[i % kRawSlots]);
-                    const uint32_t ph = (uint32_t)(i / kRawSlots) & 1u;
+                    const uint32_t bar = smem_u32(&raw_full[i % kNB]);
+                    const uint32_t ph = (uint32_t)(i / kNB) & 1u;
                     for (uint32_t t = 0; t < kWaitLimit && !mbar_try(bar, ph); ++t) {}
+                }
+                if (kSplit) {
+                    const int first_a = issued > kSplitA ? issued - kSplitA : 0;
+                    for (int i = first_a; i < issued; ++i) {
+                        const uint32_t bar = smem_u32(&a_full[i % kSplitA]);
+                        const uint32_t ph = (uint32_t)(i / kSplitA) & 1u;
+                        for (uint32_t t = 0; t < kWaitLimit && !mbar_try(bar, ph); ++t) {}
+                    }
                 }
             }
         }
@@ -425,12 +466,12 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                 const uint32_t d_tmem = tmem_base + (uint32_t)b * kBN;
                 const int chunk_end = min(n_slices, (c + 1) * prm.chunk);
                 for (bool first = true; i < chunk_end; ++i) {
-                    const int st = i % kRawSlots, ls = i % kLoN;
-                    ok = mbar_wait(smem_u32(&op_full[st]), (uint32_t)(i / kRawSlots) & 1u, &abort_flag);
+                    const int st = i % kNB, ls = i % kLoN;
+                    ok = mbar_wait(smem_u32(&op_full[st]), (uint32_t)(i / kNB) & 1u, &abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t hi_a = smem_base + st * kRawStageBytes, hi_b = hi_a + kRawBytesA;
-                    const uint32_t lo_a = smem_base + kLoBase + ls * kLoBytes, lo_b = kATmem ? lo_a : lo_a + kRawBytesA;
+                    const uint32_t hi_a = smem_base + pair_off(st), hi_b = hi_a + kRawBytesA;
+                    const uint32_t lo_a = smem_base + lo_off(ls), lo_b = lo_a + kRawBytesA;     // lo_a unused with A in TMEM
                     const uint32_t ta_hi = tmem_base + 2 * kBN + ls * kTmemColsA, ta_lo = ta_hi + 32;
 #pragma unroll
                     for (int kk = 0; kk < kBK / 8; ++kk) {
@@ -489,25 +530,27 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         };
         // transform of slice i; gathered elements come in registers, TMA tiles from the raw stage
         auto process = [&](int i, const float (&ga)[kRowsPerThread][4], const float (&gb)[kRowsPerThread][4]) -> bool {
-            const int st = i % kRawSlots, ls = i % kLoN;
-            const uint32_t ph = (uint32_t)(i / kRawSlots) & 1u;
+            const int st = i % kNB, ls = i % kLoN;
+            const uint32_t ph = (uint32_t)(i / kNB) & 1u;
+            const int sa = kSplit ? i % kSplitA : 0;
+            if (kSplit && !mbar_wait(smem_u32(&a_full[sa]), (uint32_t)(i / kSplitA) & 1u, &abort_flag)) return false;
             // a raw slot is ours once its TMA tiles landed (the producer waited for it to be empty), or, with
             // nothing coming by TMA, once the MMAs that last read it retired; likewise the lo slot
             if (kAnyTma ? !mbar_wait(smem_u32(&raw_full[st]), ph, &abort_flag)
                         : !mbar_wait(smem_u32(&empty[st]), ph ^ 1u, &abort_flag))
                 return false;
             if (!mbar_wait(smem_u32(&lo_empty[ls]), ((uint32_t)(i / kLoN) & 1u) ^ 1u, &abort_flag)) return false;
-            uint8_t *hi = smem_gen + st * kRawStageBytes;        // raw tiles live here and become the hi tiles
+            uint8_t *hi = smem_gen + pair_off(st);               // raw tiles live here and become the hi tiles
             // lo tiles: [A lo][B lo], or the B tile alone when A lives in tensor memory (then `lo` points
             // one A tile below the slot so that the same chunk offsets address the B part)
-            uint8_t *lo = smem_gen + kLoBase + ls * kLoBytes - (kATmem ? kRawBytesA : 0);
+            uint8_t *lo = smem_gen + lo_off(ls);
             if (kATmem) {
                 // A: this thread's row (TMEM lane) and 16 of the slice's 32 k at a time -> hi / lo straight into
                 // TMEM (a warp of the two-group form takes both halves, otherwise its group number picks one)
                 tc_fence_after();
                 const uint32_t q = warp & 3;
                 const int m_local = (int)(q * 32 + lane);
-                const uint8_t *arow = hi + m_local * 128;
+                const uint8_t *arow = (kSplit ? smem_gen + (uint32_t)sa * kRawBytesA : hi) + m_local * 128;
 #pragma unroll
                 for (int hh = 0; hh < (kTwoGroups ? 2 : 1); ++hh) {
                     const uint32_t h = kTwoGroups ? (uint32_t)hh : (warp - 2) >> 2;
@@ -529,6 +572,10 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                     const uint32_t taddr = tmem_base + ((q * 32u) << 16) + 2 * kBN + ls * kTmemColsA + 16 * h;
                     tc_st_32x16(taddr, h16);
                     tc_st_32x16(taddr + 32, l16);
+                }
+                if (kSplit) {                     // the raw A tile has been read: its slot may be refilled
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&a_empty[sa]));
                 }
             }
             if (kAnyTma) {      // tiles that came by TMA: elementwise, in place, over their 16-byte chunks
@@ -1004,13 +1051,14 @@ vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int 
     const bool swapped = conv_swapped(Cout, n_im2col);
     const int rows_err = swapped ? kBN : kBM, rows_in = swapped ? kBM : kBN;     // tile heights
     CUtensorMap m_err = {}, m_in = {};
-    uint32_t tx = 0;
+    uint32_t tx = 0, tx_err = 0;
     if (err_tma) {
         const cuuint32_t box[3] = {(cuuint32_t)kBK, (cuuint32_t)(Cout < rows_err ? Cout : rows_err), 1};
         const cuuint64_t dims[3] = {(cuuint64_t)P, (cuuint64_t)Cout, (cuuint64_t)B};
         const cuuint64_t str[2] = {(cuuint64_t)P * 4, (cuuint64_t)Cout * P * 4};
         if (!make_map(&m_err, delta, 3, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B)) return VGC_ERR_CUDA;
         tx += box[1] * kBK * 4;
+        tx_err = tx;
     }
     if (in_tma) {
         const cuuint32_t box[3] = {(cuuint32_t)kBK, (cuuint32_t)(C < rows_in ? C : rows_in), 1};
@@ -1020,7 +1068,8 @@ vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int 
         tx += box[1] * kBK * 4;
     }
     Params prm = {};
-    prm.p_slices = p_slices; prm.tx_bytes = tx; prm.scale = scale; prm.accumulate = accumulate; prm.S = S;
+    prm.p_slices = p_slices; prm.tx_bytes = tx; prm.scale = scale;
+    prm.tx_bytes_a = swapped ? tx - tx_err : tx_err; prm.accumulate = accumulate; prm.S = S;
     prm.x = x; prm.delta = delta;
     prm.C = C; prm.H = H; prm.W = W; prm.Cout = Cout; prm.Kh = Kh; prm.Kw = Kw; prm.sh = sh; prm.sw = sw;
     prm.ph = ph; prm.pw = pw; prm.Wo = Wo; prm.P = P;
