@@ -118,7 +118,7 @@ class HotPath:
     """All device buffers of one worker and the launches of one step."""
 
     def __init__(self, name: str, worker: int, n_input_sets: int, n_g_sets: int, device="cuda",
-                 n_params: int = 1 << 25, n_streams: int = 4, algorithm: str = "basic"):
+                 n_params: int = 1 << 25, n_streams: int = 4, algorithm: str = "basic", batch_layers: bool = True):
         import paper_1802_06058_b200 as vgc
         from paper_1802_06058_b200 import workloads
         self.vgc, self.wl = vgc, workloads
@@ -162,12 +162,22 @@ class HotPath:
             self.ws_s = None
         else:
             ws_bytes = 16
+            # conv layers of one geometry go to the library together (one launch per group of up to 8)
+            groups = {}
+            for li, spec in enumerate(self.layers):
+                key = (spec.kind, spec.cin, spec.cout, spec.k, spec.stride, spec.pad, spec.hin) if batch_layers and spec.kind == "conv" else li
+                groups.setdefault(key, []).append(li)
+            self.groups = [g[i:i + 8] for g in groups.values() for i in range(0, len(g), 8)]
+            # long groups first: the short ones fill the gaps at the end of the pass
+            self.groups.sort(key=lambda g: -sum(2 * np.prod(self.layers[li].gemm_mnk(B)) for li in g))
             for li, spec in enumerate(self.layers):
                 M, N, K = spec.gemm_mnk(B)
                 self.flops_useful += 2 * M * N * K
+            for g in self.groups:
+                spec = self.layers[g[0]]
                 if spec.kind == "conv":
-                    ws_bytes = max(ws_bytes, vgc.vgc_sqgrad_conv_workspace_bytes(
-                        B, spec.cin, spec.hin, spec.hin, spec.cout, spec.k, spec.k, spec.stride, spec.stride,
+                    ws_bytes = max(ws_bytes, vgc.vgc_sqgrad_conv_batch_workspace_bytes(
+                        len(g), B, spec.cin, spec.hin, spec.hin, spec.cout, spec.k, spec.k, spec.stride, spec.stride,
                         spec.pad, spec.pad))
                 else:
                     ws_bytes = max(ws_bytes, vgc.vgc_sqgrad_linear_workspace_bytes(B, spec.cin, spec.cout))
@@ -226,17 +236,19 @@ class HotPath:
         main = torch.cuda.current_stream()
         for st in self.side:
             st.wait_stream(main)
-        for li, spec in enumerate(self.layers):
-            x, delta = ins[li]
-            S = target[int(self.offsets[li]):int(self.offsets[li + 1])]
-            lane = li % self.n_streams
+        for gi, g in enumerate(self.groups):
+            spec = self.layers[g[0]]
+            Ss = [target[int(self.offsets[li]):int(self.offsets[li + 1])] for li in g]
+            lane = gi % self.n_streams
             stream = main if lane == 0 else self.side[lane - 1]
             ws = self.ws_s if lane == 0 else self.ws_side[lane - 1]
             if spec.kind == "conv":
-                vgc.vgc_sqgrad_conv(x, delta, (spec.k, spec.k), (spec.stride, spec.stride), (spec.pad, spec.pad),
-                                    self.scale, S, accumulate=into_v, ws=ws, stream=stream)
+                vgc.vgc_sqgrad_conv_batch([ins[li][0] for li in g], [ins[li][1] for li in g], (spec.k, spec.k),
+                                          (spec.stride, spec.stride), (spec.pad, spec.pad), self.scale, Ss,
+                                          accumulate=into_v, ws=ws, stream=stream)
             else:
-                vgc.vgc_sqgrad_linear(x, delta, self.scale, S, accumulate=into_v, ws=ws, stream=stream)
+                vgc.vgc_sqgrad_linear(ins[g[0]][0], ins[g[0]][1], self.scale, Ss[0], accumulate=into_v, ws=ws,
+                                      stream=stream)
         for st in self.side:
             main.wait_stream(st)
 
@@ -557,6 +569,8 @@ def main():
     ap.add_argument("--algorithm", default="basic", choices=["basic", "hybrid"],
                     help="hybrid: Algorithm 2 (fixed threshold tau + variance criterion) for the compress and decode "
                          "sections; device-timed only (no end-to-end or CPU leg)")
+    ap.add_argument("--no-batch", action="store_true",
+                    help="one library call per layer instead of one per group of same-shaped conv layers")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -578,7 +592,8 @@ def main():
     vgc.load_library()
     pk = peaks()
     hp = HotPath(args.workload, worker=rank * 16, n_input_sets=1, n_g_sets=max(4, min(args.steps + args.warmup, 16)),
-                 n_params=args.n_params, n_streams=max(args.streams, 1), algorithm=args.algorithm)
+                 n_params=args.n_params, n_streams=max(args.streams, 1), algorithm=args.algorithm,
+                 batch_layers=not args.no_batch)
     if hp.hybrid:
         args.no_e2e = args.no_cpu_baseline = True
     hp.fused = args.fused
@@ -656,6 +671,7 @@ def main():
             "config": {"workload": args.workload, "n_params": n, "batch": hp.batch, "W": hp.W, "alpha": hp.alpha,
                        "zeta": ZETA, "groups": hp.K, "algorithm": args.algorithm, "tau": hp.tau, "launch": "eager" if args.no_graph else "cuda graph replay",
                        "sqgrad_streams": getattr(hp, "n_streams", 1),
+                       "sqgrad_calls": len(getattr(hp, "groups", [])),
                        "fused_sqgrad_into_v": bool(args.fused),
                        "l2": "inputs larger than L2 (no flush)" if n * 16 > 126e6 else "state fits in L2 (no flush): cache-resident numbers"},
             "gpu_launches": int(launches), "clocks": clocks, "sections": sections, "roofline": roofline,

@@ -103,6 +103,21 @@ vgc_status vgc_sqgrad_conv(const float *x, const float *delta, int B, int C, int
                            float scale, int accumulate, float *S,
                            void *ws, size_t ws_bytes, vgc_stream_t stream);
 
+/* Several conv layers of ONE geometry in one call (the residual stages of a deep network repeat the same
+ * layer shapes): layer l computes what vgc_sqgrad_conv computes from x[l], delta[l] into S[l].  The tensor-
+ * core path runs up to 8 layers per kernel launch, which shortens the split of the reduction, the scratch
+ * traffic and the per-launch fixed cost; results are identical to n_layers single calls only up to the
+ * order of the fp32 partial sums (same 1e-5 bound).
+ *   x, delta, S   HOST arrays of n_layers DEVICE pointers (read during the call only)
+ *   ws            at least vgc_sqgrad_conv_batch_workspace_bytes(n_layers, ...) bytes; status word as above
+ * The layers' S ranges must not overlap.  n_layers == 0: no-op, OK. */
+size_t vgc_sqgrad_conv_batch_workspace_bytes(int n_layers, int B, int C, int H, int W, int Cout, int Kh, int Kw,
+                                             int stride_h, int stride_w, int pad_h, int pad_w);
+vgc_status vgc_sqgrad_conv_batch(int n_layers, const float *const *x, const float *const *delta, float *const *S,
+                                 int B, int C, int H, int W, int Cout, int Kh, int Kw, int stride_h, int stride_w,
+                                 int pad_h, int pad_w, float scale, int accumulate, void *ws, size_t ws_bytes,
+                                 vgc_stream_t stream);
+
 /* ---------------------------------------------------------------------------------------------
  * (2) Compressor: one step of Algorithm 1 ("Basic") over the flat buffer, then Encode().
  *

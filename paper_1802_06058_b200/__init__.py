@@ -27,6 +27,7 @@ EXPORTS = [
     "vgc_status_string", "vgc_version", "vgc_kernel_launch_count",
     "vgc_sqgrad_linear_workspace_bytes", "vgc_sqgrad_linear",
     "vgc_sqgrad_conv_workspace_bytes", "vgc_sqgrad_conv",
+    "vgc_sqgrad_conv_batch_workspace_bytes", "vgc_sqgrad_conv_batch",
     "vgc_compress_workspace_bytes", "vgc_compress", "vgc_compress_static",
     "vgc_decode_accumulate", "vgc_step_host",
     "vgc_compress_hybrid_workspace_bytes", "vgc_compress_hybrid", "vgc_decode_accumulate_hybrid",
@@ -85,6 +86,10 @@ def load_library():
     lib.vgc_sqgrad_conv_workspace_bytes.restype = sz
     lib.vgc_sqgrad_conv.argtypes = [vp, vp] + [i] * 11 + [f, i, vp, vp, sz, vp]
     lib.vgc_sqgrad_conv.restype = i
+    lib.vgc_sqgrad_conv_batch_workspace_bytes.argtypes = [i] * 12
+    lib.vgc_sqgrad_conv_batch_workspace_bytes.restype = sz
+    lib.vgc_sqgrad_conv_batch.argtypes = [i, vp, vp, vp] + [i] * 11 + [f, i, vp, sz, vp]
+    lib.vgc_sqgrad_conv_batch.restype = i
     lib.vgc_compress_workspace_bytes.argtypes = [sz, i]
     lib.vgc_compress_workspace_bytes.restype = sz
     lib.vgc_compress.argtypes = [vp, vp, vp, vp, sz, vp, i, f, f, ctypes.POINTER(_MessageStruct), vp, sz, vp]
@@ -192,6 +197,39 @@ def vgc_sqgrad_conv(x, delta, kernel, stride, padding, scale: float, S, accumula
                                         _stream(stream))
     _check(st, "vgc_sqgrad_conv")
     return S
+
+
+def vgc_sqgrad_conv_batch_workspace_bytes(n_layers, B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw) -> int:
+    return load_library().vgc_sqgrad_conv_batch_workspace_bytes(n_layers, B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw)
+
+
+def vgc_sqgrad_conv_batch(xs, deltas, kernel, stride, padding, scale: float, Ss, accumulate: bool = False,
+                          ws=None, stream=None):
+    """vgc_sqgrad_conv for several layers of one geometry (lists of tensors of equal shapes) in one call."""
+    n = len(xs)
+    if len(deltas) != n or len(Ss) != n:
+        raise ValueError("xs, deltas, Ss must have the same length")
+    if n == 0:
+        return Ss
+    B, C, H, W = xs[0].shape
+    B2, Cout, Ho, Wo = deltas[0].shape
+    Kh, Kw = kernel
+    sh, sw = stride
+    ph, pw = padding
+    if B != B2 or Ho != (H + 2 * ph - Kh) // sh + 1 or Wo != (W + 2 * pw - Kw) // sw + 1:
+        raise ValueError("delta shape does not match the convolution geometry")
+    for x, d, S in zip(xs, deltas, Ss):
+        if tuple(x.shape) != (B, C, H, W) or tuple(d.shape) != (B, Cout, Ho, Wo) or S.numel() != Cout * C * Kh * Kw:
+            raise ValueError("all layers of a batch must have the same shapes")
+    ptrs = ctypes.c_void_p * n
+    xp = ptrs(*[_dev(x, torch.float32, "x") for x in xs])
+    dp = ptrs(*[_dev(d, torch.float32, "delta") for d in deltas])
+    sp = ptrs(*[_dev(S, torch.float32, "S") for S in Ss])
+    wp, wb = _ws(ws)
+    st = load_library().vgc_sqgrad_conv_batch(n, xp, dp, sp, B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, float(scale),
+                                              int(bool(accumulate)), wp, wb, _stream(stream))
+    _check(st, "vgc_sqgrad_conv_batch")
+    return Ss
 
 
 # ------------------------------------------------------------------------------------------ (2)

@@ -13,12 +13,13 @@ vgc_status simt_sqgrad_conv(const float *x, const float *delta, int B, int C, in
 bool tc_linear_supported(int B, int in, int out);
 bool tc_conv_supported(int B, int C, int H, int W, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw);
 size_t tc_linear_workspace_bytes(int B, int in, int out);
-size_t tc_conv_workspace_bytes(int B, int C, int Kh, int Kw, int sh, int sw, int ph, int pw, int P, int Cout);
+size_t tc_conv_workspace_bytes(int n_layers, int B, int C, int Kh, int Kw, int sh, int sw, int ph, int pw, int P,
+                               int Cout);
 vgc_status tc_sqgrad_linear(const float *x, const float *delta, int B, int in, int out, float scale, int accumulate,
                             float *S, void *ws, size_t ws_bytes, cudaStream_t st);
-vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int H, int W, int Cout, int Kh, int Kw,
-                          int sh, int sw, int ph, int pw, int Ho, int Wo, float scale, int accumulate, float *S,
-                          void *ws, size_t ws_bytes, cudaStream_t st);
+vgc_status tc_sqgrad_conv(int n_layers, const float *const *x, const float *const *delta, float *const *S, int B, int C,
+                          int H, int W, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw, int Ho, int Wo,
+                          float scale, int accumulate, void *ws, size_t ws_bytes, cudaStream_t st);
 }  // namespace vgc
 
 using namespace vgc;
@@ -69,18 +70,55 @@ extern "C" vgc_status vgc_sqgrad_linear(const float *x, const float *delta, int 
                               ws_bytes - 256, st);
 }
 
-extern "C" size_t vgc_sqgrad_conv_workspace_bytes(int B, int C, int H, int W, int Cout, int Kh, int Kw,
-                                                  int stride_h, int stride_w, int pad_h, int pad_w)
+extern "C" size_t vgc_sqgrad_conv_batch_workspace_bytes(int n_layers, int B, int C, int H, int W, int Cout, int Kh,
+                                                        int Kw, int stride_h, int stride_w, int pad_h, int pad_w)
 {
     int Ho, Wo;
-    if (!conv_shape_ok(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, &Ho, &Wo)) return 0;
+    if (n_layers < 1 || !conv_shape_ok(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, &Ho, &Wo)) return 0;
     if (B == 0 || C == 0 || Cout == 0) return 0;
     size_t need = simt_workspace_bytes(Cout, C * Kh * Kw, B * Ho * Wo);
     if (tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w)) {
-        const size_t t = tc_conv_workspace_bytes(B, C, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho * Wo, Cout);
+        const size_t t = tc_conv_workspace_bytes(n_layers, B, C, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho * Wo, Cout);
         need = need > t ? need : t;
     }
     return round_up(need + 256, 256);
+}
+
+extern "C" size_t vgc_sqgrad_conv_workspace_bytes(int B, int C, int H, int W, int Cout, int Kh, int Kw,
+                                                  int stride_h, int stride_w, int pad_h, int pad_w)
+{
+    return vgc_sqgrad_conv_batch_workspace_bytes(1, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w);
+}
+
+extern "C" vgc_status vgc_sqgrad_conv_batch(int n_layers, const float *const *x, const float *const *delta,
+                                            float *const *S, int B, int C, int H, int W, int Cout, int Kh, int Kw,
+                                            int stride_h, int stride_w, int pad_h, int pad_w, float scale,
+                                            int accumulate, void *ws, size_t ws_bytes, vgc_stream_t stream)
+{
+    int Ho, Wo;
+    if (n_layers < 0 || !conv_shape_ok(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, &Ho, &Wo))
+        return VGC_ERR_INVALID_ARG;
+    if (n_layers == 0 || C == 0 || Cout == 0) return VGC_OK;
+    if (!x || !delta || !S || !(scale == scale)) return VGC_ERR_INVALID_ARG;
+    for (int l = 0; l < n_layers; ++l) {
+        if (!S[l] || !aligned16(S[l])) return VGC_ERR_INVALID_ARG;
+        if (B > 0 && (!x[l] || !delta[l] || !aligned16(x[l]) || !aligned16(delta[l]))) return VGC_ERR_INVALID_ARG;
+    }
+    if (ws_bytes < vgc_sqgrad_conv_batch_workspace_bytes(n_layers, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h,
+                                                         pad_w) ||
+        (ws_bytes && !ws))
+        return VGC_ERR_WORKSPACE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (B > 0 && use_tensor_cores() && tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w))
+        return tc_sqgrad_conv(n_layers, x, delta, S, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho, Wo,
+                              scale, accumulate, ws, ws_bytes, st);
+    for (int l = 0; l < n_layers; ++l) {        // CUDA-core kernel: layer after layer
+        const vgc_status rc = simt_sqgrad_conv(x[l], delta[l], B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w,
+                                               Ho, Wo, scale, accumulate, S[l], static_cast<char *>(ws) + 256,
+                                               ws_bytes - 256, st);
+        if (rc != VGC_OK) return rc;
+    }
+    return VGC_OK;
 }
 
 extern "C" vgc_status vgc_sqgrad_conv(const float *x, const float *delta, int B, int C, int H, int W, int Cout,
@@ -88,22 +126,8 @@ extern "C" vgc_status vgc_sqgrad_conv(const float *x, const float *delta, int B,
                                       float scale, int accumulate, float *S,
                                       void *ws, size_t ws_bytes, vgc_stream_t stream)
 {
-    int Ho, Wo;
-    if (!conv_shape_ok(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, &Ho, &Wo))
-        return VGC_ERR_INVALID_ARG;
-    if (C == 0 || Cout == 0) return VGC_OK;
-    if (!S || !aligned16(S)) return VGC_ERR_INVALID_ARG;
-    if (B > 0 && (!x || !delta || !aligned16(x) || !aligned16(delta))) return VGC_ERR_INVALID_ARG;
-    if (!(scale == scale)) return VGC_ERR_INVALID_ARG;
-    if (ws_bytes < vgc_sqgrad_conv_workspace_bytes(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w) ||
-        (ws_bytes && !ws))
-        return VGC_ERR_WORKSPACE;
-    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    if (B > 0 && use_tensor_cores() && tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w))
-        return tc_sqgrad_conv(x, delta, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho, Wo, scale,
-                              accumulate, S, ws, ws_bytes, st);
-    return simt_sqgrad_conv(x, delta, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho, Wo, scale,
-                            accumulate, S, static_cast<char *>(ws) + 256, ws_bytes - 256, st);
+    return vgc_sqgrad_conv_batch(1, &x, &delta, &S, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, scale,
+                                 accumulate, ws, ws_bytes, stream);
 }
 
 extern "C" const char *vgc_status_string(int status)

@@ -90,14 +90,21 @@ struct Params {
     uint32_t tx_bytes_a;     // of which the A tile's
     float scale;
     int accumulate;
-    const float *x, *delta;  // raw operands (gathered tiles)
+    int splits;              // blocks along the reduction per layer (blockIdx.z = layer * splits + split)
     int C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, Wo, P;     // conv geometry (gathered tiles)
     int chw;                 // C*H*W
     unsigned wo_magic;       // floor(2^32 / Wo) + 1: p / Wo == umulhi(p, wo_magic) for p * Wo < 2^32
-    float *S;                // result: element (m, n) lives at S[m*ld_m + n*ld_n]; one of the two is 1
-    long long ld_m, ld_n;
-    float *partial;          // split-K scratch [split][tile][column][row], used when gridDim.z > 1
+    long long ld_m, ld_n;    // result: element (m, n) lives at S[m*ld_m + n*ld_n]; one of the two is 1
+    float *partial;          // split-K scratch [layer][split][tile][column][row], used when splits > 1
     uint32_t *status;        // device word; VGC_DEV_TIMEOUT is OR-ed in if a wait expired
+};
+
+// Layers of one geometry computed by one launch: their tensor maps and pointers.
+constexpr int kMaxBatch = 8;
+struct Batch {
+    CUtensorMap a[kMaxBatch], b[kMaxBatch];
+    const float *x[kMaxBatch], *delta[kMaxBatch];   // raw operands (gathered tiles)
+    float *S[kMaxBatch];
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -266,10 +273,12 @@ template <int kMode>
 struct GatherRows {
     int base[kRowsPerThread], dh[kRowsPerThread], dw[kRowsPerThread];
     bool ok[kRowsPerThread];
+    const float *src;       // x (im2col rows) or delta (error rows) of this block's layer
 
-    __device__ __forceinline__ void init(const Params &prm, int first_row, int limit)
+    __device__ __forceinline__ void init(const Params &prm, const float *x, const float *delta, int first_row, int limit)
     {
         if (kMode == kTma) return;
+        src = kMode == kGatherIm2col ? x : delta;
         const int khw = prm.Kh * prm.Kw;
 #pragma unroll
         for (int i = 0; i < kRowsPerThread; ++i) {
@@ -292,7 +301,7 @@ struct GatherRows {
     __device__ __forceinline__ void load(const Params &prm, int z, int pbase, float (&v)[kRowsPerThread][4]) const
     {
         if (kMode == kGatherIm2col) {
-            const float *xz = prm.x + (size_t)z * prm.chw;
+            const float *xz = src + (size_t)z * prm.chw;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int p = pbase + j;
@@ -308,7 +317,7 @@ struct GatherRows {
                 }
             }
         } else if (kMode == kGatherErr) {
-            const float *dz = prm.delta + (size_t)z * prm.Cout * prm.P + pbase;
+            const float *dz = src + (size_t)z * prm.Cout * prm.P + pbase;
 #pragma unroll
             for (int i = 0; i < kRowsPerThread; ++i)
 #pragma unroll
@@ -320,7 +329,7 @@ struct GatherRows {
 // ---- the kernel ------------------------------------------------------------------------------
 template <int kMajor, int kModeA, int kModeB, bool kATmem>
 __global__ void __launch_bounds__(kThreadsTc, 1)
-sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const Params prm)
+sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
 {
     static_assert(kMajor == kMajorK || (kModeA == kTma && kModeB == kTma), "gathered tiles are K-major");
     static_assert(!kATmem || (kMajor == kMajorK && kModeA == kTma), "A goes to tensor memory from a K-major TMA tile");
@@ -358,7 +367,10 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     const int m0 = blockIdx.y * kBM, n0 = blockIdx.x * kBN;
     const int n_valid = min(kBN, prm.N - n0);                              // columns of this tile that exist
     const int n_act = (n_valid + 15) & ~15;                                // UMMA N (multiple of 16)
-    const int slice_begin = blockIdx.z * prm.slices_per_split;
+    const int layer = (int)blockIdx.z / prm.splits, split = (int)blockIdx.z - layer * prm.splits;
+    const CUtensorMap *map_a = &bt.a[layer], *map_b = &bt.b[layer];
+    float *const S = bt.S[layer];
+    const int slice_begin = split * prm.slices_per_split;
     const int slice_end = min(prm.k_slices, slice_begin + prm.slices_per_split);
     const int n_slices = slice_end - slice_begin;                           // >= 1 by construction
     const int n_chunks = (n_slices + prm.chunk - 1) / prm.chunk;
@@ -408,23 +420,23 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                     const uint32_t full_a = smem_u32(&a_full[sa]);
                     const int z = slice / prm.p_slices, p0 = (slice - z * prm.p_slices) * kBK;
                     mbar_expect_tx(full_a, prm.tx_bytes_a);
-                    tma_load_3d(smem_base + (uint32_t)sa * kRawBytesA, &map_a, full_a, p0, m0, z);
+                    tma_load_3d(smem_base + (uint32_t)sa * kRawBytesA, map_a, full_a, p0, m0, z);
                     mbar_expect_tx(full, prm.tx_bytes - prm.tx_bytes_a);
-                    tma_load_3d(dst_b, &map_b, full, p0, n0, z);
+                    tma_load_3d(dst_b, map_b, full, p0, n0, z);
                     issued = i + 1;
                     continue;
                 }
                 mbar_expect_tx(full, prm.tx_bytes);
                 if (kMajor == kMajorK) {
                     const int z = slice / prm.p_slices, p0 = (slice - z * prm.p_slices) * kBK;
-                    if (!kGatherA) tma_load_3d(dst_a, &map_a, full, p0, m0, z);
-                    if (!kGatherB) tma_load_3d(dst_b, &map_b, full, p0, n0, z);
+                    if (!kGatherA) tma_load_3d(dst_a, map_a, full, p0, m0, z);
+                    if (!kGatherB) tma_load_3d(dst_b, map_b, full, p0, n0, z);
                 } else {
                     const int k0 = slice * kBK;
 #pragma unroll
-                    for (int j = 0; j < kBM / 32; ++j) tma_load_2d(dst_a + j * 4096, &map_a, full, m0 + 32 * j, k0);
+                    for (int j = 0; j < kBM / 32; ++j) tma_load_2d(dst_a + j * 4096, map_a, full, m0 + 32 * j, k0);
 #pragma unroll
-                    for (int j = 0; j < kBN / 32; ++j) tma_load_2d(dst_b + j * 4096, &map_b, full, n0 + 32 * j, k0);
+                    for (int j = 0; j < kBN / 32; ++j) tma_load_2d(dst_b + j * 4096, map_b, full, n0 + 32 * j, k0);
                 }
                 issued = i + 1;
             }
@@ -512,8 +524,8 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         const int kq = t & 7, row0 = t >> 3;                               // gathered chunks: rows row0 + 32*i, k = 4*kq..4*kq+3
         GatherRows<kModeA> rows_a;
         GatherRows<kModeB> rows_b;
-        rows_a.init(prm, m0 + row0, prm.M);
-        rows_b.init(prm, n0 + row0, prm.N);
+        rows_a.init(prm, bt.x[layer], bt.delta[layer], m0 + row0, prm.M);
+        rows_b.init(prm, bt.x[layer], bt.delta[layer], n0 + row0, prm.N);
         // where the current slice sits: example z, 32-wide block pblk of that example's output positions
         int z = 0, pblk = 0;
         if (kAnyGather) {
@@ -659,7 +671,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         if (ok) {
             const int r_local = (int)(q * 32u + lane);
             const int m = m0 + r_local;
-            if (gridDim.z > 1) {
+            if (prm.splits > 1) {
                 // split-K scratch, column-major inside the tile: consecutive lanes -> consecutive addresses
                 const size_t tile = (size_t)blockIdx.z * (gridDim.x * gridDim.y) + (size_t)blockIdx.y * gridDim.x + blockIdx.x;
                 float *dst = prm.partial + tile * (kBM * kBN) + r_local;
@@ -669,7 +681,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             } else if (prm.ld_m == 1) {
                 // result is contiguous along m: lanes write neighbouring addresses directly
                 if (m < prm.M) {
-                    float *col = prm.S + (size_t)m + (size_t)n0 * prm.ld_n;
+                    float *col = S + (size_t)m + (size_t)n0 * prm.ld_n;
 #pragma unroll
                     for (int j0 = 0; j0 < kBN; j0 += 16) {        // old values sixteen at a time, all loads in flight
                         float old[16];
@@ -696,7 +708,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 #pragma unroll
                     for (int rr = 0; rr < 8; ++rr) {
                         const int mr = m0 + (int)(q * 32u) + r0 + rr;
-                        const float *src = prm.S + (size_t)mr * prm.ld_m + n0;
+                        const float *src = S + (size_t)mr * prm.ld_m + n0;
 #pragma unroll
                         for (int cblk = 0; cblk < kBN / 32; ++cblk) {
                             const int j = cblk * 32 + (int)lane;
@@ -706,7 +718,7 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 #pragma unroll
                     for (int rr = 0; rr < 8; ++rr) {
                         const int mr = m0 + (int)(q * 32u) + r0 + rr;
-                        float *dst = prm.S + (size_t)mr * prm.ld_m + n0;
+                        float *dst = S + (size_t)mr * prm.ld_m + n0;
 #pragma unroll
                         for (int cblk = 0; cblk < kBN / 32; ++cblk) {
                             const int j = cblk * 32 + (int)lane;
@@ -734,11 +746,15 @@ sqgrad_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 // Combine split-K partial tiles in a fixed order.  One block per 32 x 8 patch of a tile, one output per
 // thread: partials are read along rows (their unit stride), the result is written along whichever of
 // m / n has unit stride.
+struct ResultPtrs { float *S[kMaxBatch]; };
+
 __global__ void __launch_bounds__(256)
 sqgrad_tc_combine(const float *__restrict__ partial, int splits, int tiles_x, int tiles_y, int M, int N, float scale,
-                  int accumulate, float *__restrict__ S, long long ld_m, long long ld_n)
+                  int accumulate, const ResultPtrs results, long long ld_m, long long ld_n)
 {
     __shared__ float patch[8][33];
+    float *__restrict__ S = results.S[blockIdx.y];                         // blockIdx.y: layer of the batch
+    partial += (size_t)blockIdx.y * splits * ((size_t)tiles_x * tiles_y) * (kBM * kBN);
     const int tile = blockIdx.x >> 6, sub = blockIdx.x & 63;
     const int tx = tile % tiles_x, ty = tile / tiles_x;
     const int r0 = (sub & 3) * 32, j0 = (sub >> 2) * 8;                   // patch origin inside the tile
@@ -826,12 +842,12 @@ struct Plan {
     int splits, slices_per_split, k_slices, tiles_x, tiles_y;
 };
 
-static Plan make_plan(int M, int N, int k_slices)
+static Plan make_plan(int M, int N, int k_slices, int n_layers = 1)
 {
     Plan p;
     p.tiles_x = (N + kBN - 1) / kBN;
     p.tiles_y = (M + kBM - 1) / kBM;
-    const long tiles = (long)p.tiles_x * p.tiles_y;
+    const long tiles = (long)p.tiles_x * p.tiles_y * n_layers;          // output tiles of the whole launch
     // blocks of one launch: one per SM fills the device once; a caller that runs several layers side by side
     // (separate streams and workspaces) may ask for fewer, longer blocks through VGC_TC_BLOCKS
     const char *env = getenv("VGC_TC_BLOCKS");
@@ -862,19 +878,19 @@ bool tc_conv_supported(int B, int C, int H, int W, int Cout, int Kh, int Kw, int
            (long)B * ((P + kBK - 1) / kBK) < (1L << 30);
 }
 
-static size_t tc_workspace_bytes(int M, int N, int k_slices)
+static size_t tc_workspace_bytes(int M, int N, int k_slices, int n_layers = 1)
 {
-    const Plan p = make_plan(M, N, k_slices);
-    return 256 + (p.splits > 1 ? (size_t)p.splits * p.tiles_x * p.tiles_y * kBM * kBN * sizeof(float) : 0);
+    const Plan p = make_plan(M, N, k_slices, n_layers);
+    return 256 + (p.splits > 1 ? (size_t)n_layers * p.splits * p.tiles_x * p.tiles_y * kBM * kBN * sizeof(float) : 0);
 }
 
-typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const Params);
+typedef void (*KernelFn)(const Batch, const Params);
 
-static vgc_status tc_launch(KernelFn kernel, const CUtensorMap &ma, const CUtensorMap &mb, Params prm, int M, int N,
+static vgc_status tc_launch(KernelFn kernel, const Batch &bt, int n_layers, Params prm, int M, int N,
                             int k_slices, void *ws, size_t ws_bytes, cudaStream_t st)
 {
-    const Plan plan = make_plan(M, N, k_slices);
-    if (ws_bytes < tc_workspace_bytes(M, N, k_slices)) return VGC_ERR_WORKSPACE;
+    const Plan plan = make_plan(M, N, k_slices, n_layers);
+    if (ws_bytes < tc_workspace_bytes(M, N, k_slices, n_layers)) return VGC_ERR_WORKSPACE;
     static KernelFn configured[16];
     static int n_configured = 0;
     bool seen = false;
@@ -884,15 +900,18 @@ static vgc_status tc_launch(KernelFn kernel, const CUtensorMap &ma, const CUtens
         if (n_configured < 16) configured[n_configured++] = kernel;
     }
     prm.M = M; prm.N = N; prm.k_slices = k_slices; prm.slices_per_split = plan.slices_per_split;
+    prm.splits = plan.splits;
     prm.chunk = default_chunk();
     prm.status = static_cast<uint32_t *>(ws);
     prm.partial = reinterpret_cast<float *>(static_cast<char *>(ws) + 256);
-    dim3 grid(plan.tiles_x, plan.tiles_y, plan.splits);
-    kernel<<<grid, kThreadsTc, kSmemBytes, st>>>(ma, mb, prm);
+    dim3 grid(plan.tiles_x, plan.tiles_y, plan.splits * n_layers);
+    kernel<<<grid, kThreadsTc, kSmemBytes, st>>>(bt, prm);
     count_launch();
     if (plan.splits > 1) {
-        sqgrad_tc_combine<<<(unsigned)(plan.tiles_x * plan.tiles_y * 64), 256, 0, st>>>(
-            prm.partial, plan.splits, plan.tiles_x, plan.tiles_y, M, N, prm.scale, prm.accumulate, prm.S, prm.ld_m,
+        ResultPtrs results = {};
+        for (int l = 0; l < n_layers; ++l) results.S[l] = bt.S[l];
+        sqgrad_tc_combine<<<dim3((unsigned)(plan.tiles_x * plan.tiles_y * 64), (unsigned)n_layers), 256, 0, st>>>(
+            prm.partial, plan.splits, plan.tiles_x, plan.tiles_y, M, N, prm.scale, prm.accumulate, results, prm.ld_m,
             prm.ld_n);
         count_launch();
     }
@@ -904,17 +923,19 @@ size_t tc_linear_workspace_bytes(int B, int in, int out) { return tc_workspace_b
 vgc_status tc_sqgrad_linear(const float *x, const float *delta, int B, int in, int out, float scale, int accumulate,
                             float *S, void *ws, size_t ws_bytes, cudaStream_t st)
 {
-    CUtensorMap ma, mb;
+    Batch bt = {};
     const cuuint32_t box[2] = {32, (cuuint32_t)kBK};
     const cuuint64_t dims_a[2] = {(cuuint64_t)out, (cuuint64_t)B}, str_a[1] = {(cuuint64_t)out * 4};
     const cuuint64_t dims_b[2] = {(cuuint64_t)in, (cuuint64_t)B}, str_b[1] = {(cuuint64_t)in * 4};
-    if (!make_map(&ma, delta, 2, dims_a, str_a, box, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) ||
-        !make_map(&mb, x, 2, dims_b, str_b, box, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B))
+    if (!make_map(&bt.a[0], delta, 2, dims_a, str_a, box, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) ||
+        !make_map(&bt.b[0], x, 2, dims_b, str_b, box, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B))
         return VGC_ERR_CUDA;
+    bt.x[0] = x; bt.delta[0] = delta; bt.S[0] = S;
     Params prm = {};
-    prm.p_slices = 1; prm.tx_bytes = kRawStageBytes; prm.scale = scale; prm.accumulate = accumulate; prm.S = S;
+    prm.p_slices = 1; prm.tx_bytes = kRawStageBytes; prm.tx_bytes_a = kRawBytesA; prm.scale = scale;
+    prm.accumulate = accumulate;
     prm.ld_m = in; prm.ld_n = 1;
-    return tc_launch(sqgrad_tc<kMajorMN, kTma, kTma, false>, ma, mb, prm, out, in, (B + kBK - 1) / kBK, ws, ws_bytes, st);
+    return tc_launch(sqgrad_tc<kMajorMN, kTma, kTma, false>, bt, 1, prm, out, in, (B + kBK - 1) / kBK, ws, ws_bytes, st);
 }
 
 // Cout <= 64: the im2col rows take the 128-row A tile and the errors the narrow B tile
@@ -989,54 +1010,79 @@ sqgrad_repack(const float *__restrict__ in, float *__restrict__ out, int B, int 
     }
 }
 
-static size_t conv_workspace_plain(int B, int C, int Kh, int Kw, int P, int Cout)
+static size_t conv_workspace_plain(int n_layers, int B, int C, int Kh, int Kw, int P, int Cout)
 {
     const int n_im2col = C * Kh * Kw, k_slices = B * ((P + kBK - 1) / kBK);
-    return conv_swapped(Cout, n_im2col) ? tc_workspace_bytes(n_im2col, Cout, k_slices)
-                                        : tc_workspace_bytes(Cout, n_im2col, k_slices);
+    return conv_swapped(Cout, n_im2col) ? tc_workspace_bytes(n_im2col, Cout, k_slices, n_layers)
+                                        : tc_workspace_bytes(Cout, n_im2col, k_slices, n_layers);
 }
 
-size_t tc_conv_workspace_bytes(int B, int C, int Kh, int Kw, int sh, int sw, int ph, int pw, int P, int Cout)
+// Workspace of one launch over n_layers layers of this geometry (n_layers <= kMaxBatch).
+static size_t conv_workspace_group(int n_layers, int B, int C, int Kh, int Kw, int sh, int sw, int ph, int pw, int P,
+                                   int Cout)
 {
     // the larger of the in-place form and the repacked one, so that either can be chosen at call time
-    size_t need = conv_workspace_plain(B, C, Kh, Kw, P, Cout);
+    size_t need = conv_workspace_plain(n_layers, B, C, Kh, Kw, P, Cout);
     const int mode = repack_mode(B, C, Cout, Kh, Kw, sh, sw, ph, pw, P);
+    const size_t x_bytes = round_up(sizeof(float) * (size_t)B * C * P, 256);
+    const size_t d_bytes = round_up(sizeof(float) * (size_t)B * Cout * P, 256);
     if (mode == kRepackPlanes) {
-        const size_t r = round_up(conv_workspace_plain(B, C, 1, 1, P, Cout), 256) + sizeof(float) * (size_t)B * C * P;
+        const size_t r = round_up(conv_workspace_plain(n_layers, B, C, 1, 1, P, Cout), 256) + n_layers * x_bytes;
         need = need > r ? need : r;
     } else if (mode == kRepackFlat) {
-        const size_t r = round_up(conv_workspace_plain(1, C, 1, 1, B * P, Cout), 256) +
-                         round_up(sizeof(float) * (size_t)B * C * P, 256) + sizeof(float) * (size_t)B * Cout * P;
+        const size_t r = round_up(conv_workspace_plain(n_layers, 1, C, 1, 1, B * P, Cout), 256) +
+                         n_layers * (x_bytes + d_bytes);
         need = need > r ? need : r;
     }
     return need;
 }
 
-vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int H, int W, int Cout, int Kh, int Kw,
-                          int sh, int sw, int ph, int pw, int Ho, int Wo, float scale, int accumulate, float *S,
-                          void *ws, size_t ws_bytes, cudaStream_t st)
+size_t tc_conv_workspace_bytes(int n_layers, int B, int C, int Kh, int Kw, int sh, int sw, int ph, int pw, int P,
+                               int Cout)
+{
+    // more layers than one launch takes are processed group after group in the same workspace
+    const int first = n_layers < kMaxBatch ? n_layers : kMaxBatch;
+    size_t need = conv_workspace_group(first, B, C, Kh, Kw, sh, sw, ph, pw, P, Cout);
+    const int rest = n_layers > kMaxBatch ? n_layers % kMaxBatch : 0;
+    if (rest) {
+        const size_t r = conv_workspace_group(rest, B, C, Kh, Kw, sh, sw, ph, pw, P, Cout);
+        need = need > r ? need : r;
+    }
+    return need;
+}
+
+static vgc_status conv_group(int n_layers, const float *const *x, const float *const *delta, float *const *S, int B,
+                             int C, int H, int W, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw, int Ho,
+                             int Wo, float scale, int accumulate, void *ws, size_t ws_bytes, cudaStream_t st)
 {
     const int P = Ho * Wo, n_im2col = C * Kh * Kw;
     const int mode = repack_mode(B, C, Cout, Kh, Kw, sh, sw, ph, pw, P);
     if (mode != kRepackNone) {
         const bool flat = mode == kRepackFlat;
-        const size_t inner = round_up(flat ? conv_workspace_plain(1, C, 1, 1, B * P, Cout)
-                                           : conv_workspace_plain(B, C, 1, 1, P, Cout), 256);
+        const size_t inner = round_up(flat ? conv_workspace_plain(n_layers, 1, C, 1, 1, B * P, Cout)
+                                           : conv_workspace_plain(n_layers, B, C, 1, 1, P, Cout), 256);
         const size_t x_bytes = round_up(sizeof(float) * (size_t)B * C * P, 256);
-        const size_t d_bytes = flat ? sizeof(float) * (size_t)B * Cout * P : 0;
-        if (ws_bytes < inner + x_bytes + d_bytes) return VGC_ERR_WORKSPACE;
-        float *x_r = reinterpret_cast<float *>(static_cast<char *>(ws) + inner);
-        float *d_r = reinterpret_cast<float *>(static_cast<char *>(ws) + inner + x_bytes);
+        const size_t d_bytes = flat ? round_up(sizeof(float) * (size_t)B * Cout * P, 256) : 0;
+        if (ws_bytes < inner + n_layers * (x_bytes + d_bytes)) return VGC_ERR_WORKSPACE;
         // one warp per row; a few rows per warp when there are many
         auto blocks_for = [](size_t rows) { const size_t b = (rows + 31) / 32; return (unsigned)(b < 1 ? 1 : (b > 148 * 32 ? 148 * 32 : b)); };
-        sqgrad_repack<<<blocks_for((size_t)B * C), 256, 0, st>>>(x, x_r, B, C, H * W, W, Wo, P, sh, sw, flat ? 1 : 0);
-        count_launch();
-        if (flat) {
-            sqgrad_repack<<<blocks_for((size_t)B * Cout), 256, 0, st>>>(delta, d_r, B, Cout, P, Wo, Wo, P, 1, 1, 1);
+        const float *xr[kMaxBatch], *dr[kMaxBatch];
+        for (int l = 0; l < n_layers; ++l) {
+            char *base = static_cast<char *>(ws) + inner + (size_t)l * (x_bytes + d_bytes);
+            float *x_r = reinterpret_cast<float *>(base), *d_r = reinterpret_cast<float *>(base + x_bytes);
+            sqgrad_repack<<<blocks_for((size_t)B * C), 256, 0, st>>>(x[l], x_r, B, C, H * W, W, Wo, P, sh, sw, flat ? 1 : 0);
             count_launch();
-            return tc_sqgrad_conv(x_r, d_r, 1, C, B * P, 1, Cout, 1, 1, 1, 1, 0, 0, B * P, 1, scale, accumulate, S, ws, inner, st);
+            if (flat) {
+                sqgrad_repack<<<blocks_for((size_t)B * Cout), 256, 0, st>>>(delta[l], d_r, B, Cout, P, Wo, Wo, P, 1, 1, 1);
+                count_launch();
+            }
+            xr[l] = x_r;
+            dr[l] = flat ? d_r : delta[l];
         }
-        return tc_sqgrad_conv(x_r, delta, B, C, Ho, Wo, Cout, 1, 1, 1, 1, 0, 0, Ho, Wo, scale, accumulate, S, ws, inner, st);
+        if (flat)
+            return conv_group(n_layers, xr, dr, S, 1, C, B * P, 1, Cout, 1, 1, 1, 1, 0, 0, B * P, 1, scale, accumulate, ws,
+                              inner, st);
+        return conv_group(n_layers, xr, dr, S, B, C, Ho, Wo, Cout, 1, 1, 1, 1, 0, 0, Ho, Wo, scale, accumulate, ws, inner, st);
     }
     // VGC_TC_GATHER (bit 0: error tile, bit 1: input tile) forces the gathered form of a tile and
     // VGC_TC_ATMEM=0 keeps the A operand in shared memory: every variant computes the same thing, the
@@ -1050,27 +1096,29 @@ vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int 
     const int k_slices = B * p_slices;
     const bool swapped = conv_swapped(Cout, n_im2col);
     const int rows_err = swapped ? kBN : kBM, rows_in = swapped ? kBM : kBN;     // tile heights
-    CUtensorMap m_err = {}, m_in = {};
-    uint32_t tx = 0, tx_err = 0;
-    if (err_tma) {
-        const cuuint32_t box[3] = {(cuuint32_t)kBK, (cuuint32_t)(Cout < rows_err ? Cout : rows_err), 1};
-        const cuuint64_t dims[3] = {(cuuint64_t)P, (cuuint64_t)Cout, (cuuint64_t)B};
-        const cuuint64_t str[2] = {(cuuint64_t)P * 4, (cuuint64_t)Cout * P * 4};
-        if (!make_map(&m_err, delta, 3, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B)) return VGC_ERR_CUDA;
-        tx += box[1] * kBK * 4;
-        tx_err = tx;
-    }
-    if (in_tma) {
-        const cuuint32_t box[3] = {(cuuint32_t)kBK, (cuuint32_t)(C < rows_in ? C : rows_in), 1};
-        const cuuint64_t dims[3] = {(cuuint64_t)P, (cuuint64_t)C, (cuuint64_t)B};
-        const cuuint64_t str[2] = {(cuuint64_t)P * 4, (cuuint64_t)C * P * 4};
-        if (!make_map(&m_in, x, 3, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B)) return VGC_ERR_CUDA;
-        tx += box[1] * kBK * 4;
+    Batch bt = {};
+    uint32_t tx_err = 0, tx_in = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        CUtensorMap *m_err = swapped ? &bt.b[l] : &bt.a[l], *m_in = swapped ? &bt.a[l] : &bt.b[l];
+        if (err_tma) {
+            const cuuint32_t box[3] = {(cuuint32_t)kBK, (cuuint32_t)(Cout < rows_err ? Cout : rows_err), 1};
+            const cuuint64_t dims[3] = {(cuuint64_t)P, (cuuint64_t)Cout, (cuuint64_t)B};
+            const cuuint64_t str[2] = {(cuuint64_t)P * 4, (cuuint64_t)Cout * P * 4};
+            if (!make_map(m_err, delta[l], 3, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B)) return VGC_ERR_CUDA;
+            tx_err = box[1] * kBK * 4;
+        }
+        if (in_tma) {
+            const cuuint32_t box[3] = {(cuuint32_t)kBK, (cuuint32_t)(C < rows_in ? C : rows_in), 1};
+            const cuuint64_t dims[3] = {(cuuint64_t)P, (cuuint64_t)C, (cuuint64_t)B};
+            const cuuint64_t str[2] = {(cuuint64_t)P * 4, (cuuint64_t)C * P * 4};
+            if (!make_map(m_in, x[l], 3, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B)) return VGC_ERR_CUDA;
+            tx_in = box[1] * kBK * 4;
+        }
+        bt.x[l] = x[l]; bt.delta[l] = delta[l]; bt.S[l] = S[l];
     }
     Params prm = {};
-    prm.p_slices = p_slices; prm.tx_bytes = tx; prm.scale = scale;
-    prm.tx_bytes_a = swapped ? tx - tx_err : tx_err; prm.accumulate = accumulate; prm.S = S;
-    prm.x = x; prm.delta = delta;
+    prm.p_slices = p_slices; prm.tx_bytes = tx_err + tx_in; prm.scale = scale;
+    prm.tx_bytes_a = swapped ? tx_in : tx_err; prm.accumulate = accumulate;
     prm.C = C; prm.H = H; prm.W = W; prm.Cout = Cout; prm.Kh = Kh; prm.Kw = Kw; prm.sh = sh; prm.sw = sw;
     prm.ph = ph; prm.pw = pw; prm.Wo = Wo; prm.P = P;
     prm.chw = C * H * W;
@@ -1083,14 +1131,28 @@ vgc_status tc_sqgrad_conv(const float *x, const float *delta, int B, int C, int 
         else if (e == kTma) fn = a_tmem ? sqgrad_tc<kMajorK, kTma, kGatherIm2col, true> : sqgrad_tc<kMajorK, kTma, kGatherIm2col, false>;
         else if (i == kTma) fn = sqgrad_tc<kMajorK, kGatherErr, kTma, false>;
         else fn = sqgrad_tc<kMajorK, kGatherErr, kGatherIm2col, false>;
-        return tc_launch(fn, m_err, m_in, prm, Cout, n_im2col, k_slices, ws, ws_bytes, st);
+        return tc_launch(fn, bt, n_layers, prm, Cout, n_im2col, k_slices, ws, ws_bytes, st);
     }
     prm.ld_m = 1; prm.ld_n = n_im2col;   // m = idx, n = o
     if (e == kTma && i == kTma) fn = a_tmem ? sqgrad_tc<kMajorK, kTma, kTma, true> : sqgrad_tc<kMajorK, kTma, kTma, false>;
     else if (i == kTma) fn = a_tmem ? sqgrad_tc<kMajorK, kTma, kGatherErr, true> : sqgrad_tc<kMajorK, kTma, kGatherErr, false>;
     else if (e == kTma) fn = sqgrad_tc<kMajorK, kGatherIm2col, kTma, false>;
     else fn = sqgrad_tc<kMajorK, kGatherIm2col, kGatherErr, false>;
-    return tc_launch(fn, m_in, m_err, prm, n_im2col, Cout, k_slices, ws, ws_bytes, st);
+    return tc_launch(fn, bt, n_layers, prm, n_im2col, Cout, k_slices, ws, ws_bytes, st);
+}
+
+// n_layers layers of one geometry; x, delta, S are host arrays of device pointers
+vgc_status tc_sqgrad_conv(int n_layers, const float *const *x, const float *const *delta, float *const *S, int B, int C,
+                          int H, int W, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw, int Ho, int Wo,
+                          float scale, int accumulate, void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    for (int l0 = 0; l0 < n_layers; l0 += kMaxBatch) {
+        const int nl = n_layers - l0 < kMaxBatch ? n_layers - l0 : kMaxBatch;
+        const vgc_status rc = conv_group(nl, x + l0, delta + l0, S + l0, B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, Ho, Wo,
+                                         scale, accumulate, ws, ws_bytes, st);
+        if (rc != VGC_OK) return rc;
+    }
+    return VGC_OK;
 }
 
 }  // namespace vgc

@@ -151,3 +151,36 @@ def test_every_kernel_variant_gives_the_same_statistic(monkeypatch, env, B, C, H
     got = run_conv(x, d, k, s, p, 0.5)
     want = oracle.sqgrad_conv(x.cpu().numpy(), d.cpu().numpy(), (k, k), (s, s), (p, p), scale=0.5)
     _check(got, want)
+
+
+@pytest.mark.parametrize("n_layers", [1, 3, 9])
+@pytest.mark.parametrize("B,C,H,Cout,k,s,p", [(3, 96, 12, 160, 1, 1, 0), (2, 40, 12, 48, 3, 1, 1), (4, 70, 7, 130, 1, 1, 0),
+                                              (2, 96, 16, 160, 1, 2, 0), (2, 24, 9, 20, 3, 2, 1), (8, 256, 14, 64, 1, 1, 0)])
+def test_batch_of_layers_matches_the_oracle_layer_by_layer(n_layers, B, C, H, Cout, k, s, p):
+    gen = torch.Generator(device="cuda"); gen.manual_seed(n_layers * 100 + C)
+    Ho = (H + 2 * p - k) // s + 1
+    xs = [torch.randn(B, C, H, H, device="cuda", generator=gen) for _ in range(n_layers)]
+    ds = [torch.randn(B, Cout, Ho, Ho, device="cuda", generator=gen) * (10.0 ** -(l % 4)) for l in range(n_layers)]
+    flat = torch.rand(n_layers * Cout * C * k * k, device="cuda", generator=gen)
+    S0 = flat.clone()
+    Ss = [flat[l * Cout * C * k * k:(l + 1) * Cout * C * k * k] for l in range(n_layers)]
+    ws = _ws(vgc.vgc_sqgrad_conv_batch_workspace_bytes(n_layers, B, C, H, H, Cout, k, k, s, s, p, p))
+    for accumulate in (False, True):
+        flat.copy_(S0)
+        vgc.vgc_sqgrad_conv_batch(xs, ds, (k, k), (s, s), (p, p), 0.5, Ss, accumulate=accumulate, ws=ws)
+        assert _status(ws) == 0
+        for l in range(n_layers):
+            want = S0[l * Cout * C * k * k:(l + 1) * Cout * C * k * k].cpu().numpy().reshape(Cout, C, k, k).copy() \
+                if accumulate else None
+            want = oracle.sqgrad_conv(xs[l].cpu().numpy(), ds[l].cpu().numpy(), (k, k), (s, s), (p, p), scale=0.5, out=want)
+            _check(Ss[l].cpu().numpy().reshape(Cout, C, k, k), want)
+
+
+def test_batch_argument_checks():
+    x = torch.randn(2, 8, 6, 6, device="cuda"); d = torch.randn(2, 8, 6, 6, device="cuda")
+    S = torch.empty(8 * 8, device="cuda")
+    with pytest.raises(ValueError):
+        vgc.vgc_sqgrad_conv_batch([x, x], [d], (1, 1), (1, 1), (0, 0), 1.0, [S, S], ws=_ws(1 << 20))
+    with pytest.raises(vgc.VgcError):                         # workspace too small for two layers
+        vgc.vgc_sqgrad_conv_batch([x, x], [d, d], (1, 1), (1, 1), (0, 0), 1.0, [S, S.clone()], ws=_ws(256)[:16])
+    assert vgc.vgc_sqgrad_conv_batch([], [], (1, 1), (1, 1), (0, 0), 1.0, []) == []
