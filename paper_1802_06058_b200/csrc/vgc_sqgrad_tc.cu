@@ -78,7 +78,9 @@ constexpr uint32_t kWaitLimit = 1u << 22;                           // polls bef
 
 enum { kMajorK = 0, kMajorMN = 1 };
 
-enum { kTma = 0, kGatherErr = 1, kGatherIm2col = 2 };      // how a tile gets its rows
+// how a tile gets its rows; kGatherTaps4 / kGatherTaps2: im2col rows of a Kw = 3, stride 1, pad_w = 1 kernel
+// gathered three taps at a time (output width a multiple of 4 / of 2)
+enum { kTma = 0, kGatherErr = 1, kGatherIm2col = 2, kGatherTaps4 = 3, kGatherTaps2 = 4 };
 
 struct Params {
     int M, N;                // rows of the A tile space / of the B tile space
@@ -326,6 +328,118 @@ struct GatherRows {
     }
 };
 
+// Kw = 3, stride 1, pad_w = 1: the three rows (c, kh, kw = 0..2) of the im2col view read the same input row
+// shifted by one, so a thread takes whole triples: for 4 (or 2 + 2) consecutive output positions it loads
+// the input row segment once -- one aligned vector and its two neighbours -- and feeds all three rows from
+// it.  A thread owns the triples first_triple + grp + 32*i (i = 0, 1) of the tile's rows; triples that
+// straddle the tile's first or last row are handled by the row test at store time.
+template <int kSpan>          // output positions covered by one aligned vector load: 4 or 2
+struct GatherTaps {
+    int base[2], dh[2], row_local[2];
+    bool ok[2];
+    const float *src;
+
+    __device__ __forceinline__ void init(const Params &prm, const float *x, int tile_origin, int grp, int limit)
+    {
+        src = x;
+        const int first_triple = tile_origin / 3;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int T = first_triple + grp + 32 * i;               // triple = (c, kh)
+            ok[i] = 3 * T < limit;
+            const int tt = ok[i] ? T : 0;
+            const int c = tt / prm.Kh, kh = tt - c * prm.Kh;
+            dh[i] = kh - prm.ph;
+            base[i] = (c * prm.H + dh[i]) * prm.W;
+            row_local[i] = 3 * T - tile_origin;                      // tile row of the kw = 0 tap (may be -2, -1)
+        }
+    }
+    // v[i][0..7]: kSpan = 4: {left, m0, m1, m2, m3, right, -, -} for positions pbase..pbase+3;
+    //             kSpan = 2: {left, m0, m1, right} for pbase, pbase+1 and the same for pbase+2, pbase+3
+    __device__ __forceinline__ void load(const Params &prm, int z, int pbase, float (&v)[2][8]) const
+    {
+        const float *xz = src + (size_t)z * prm.chw;
+#pragma unroll
+        for (int s = 0; s < 4 / kSpan; ++s) {
+            const int p = pbase + s * kSpan;
+            const int ho = (int)__umulhi((unsigned)p, prm.wo_magic), wo = p - ho * prm.Wo;
+            const bool pv = p < prm.P;
+            const float *xp = xz + (ho * prm.W + wo);
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const bool in = pv && ok[i] && (unsigned)(ho + dh[i]) < (unsigned)prm.H;
+                const float *q = xp + base[i];
+                float *o = &v[i][s * 4];
+                if (kSpan == 4) {
+                    const float4 m = in ? __ldg(reinterpret_cast<const float4 *>(q)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    o[0] = (in && wo > 0) ? __ldg(q - 1) : 0.f;
+                    o[1] = m.x; o[2] = m.y; o[3] = m.z; o[4] = m.w;
+                    o[5] = (in && wo + 4 < prm.W) ? __ldg(q + 4) : 0.f;
+                } else {
+                    const float2 m = in ? __ldg(reinterpret_cast<const float2 *>(q)) : make_float2(0.f, 0.f);
+                    o[0] = (in && wo > 0) ? __ldg(q - 1) : 0.f;
+                    o[1] = m.x; o[2] = m.y;
+                    o[3] = (in && wo + 2 < prm.W) ? __ldg(q + 2) : 0.f;
+                }
+            }
+        }
+    }
+    // the four k of tap kw of triple i
+    __device__ __forceinline__ static void tap(const float (&v)[2][8], int i, int kw, float (&out)[4])
+    {
+        if (kSpan == 4) {
+            out[0] = v[i][kw]; out[1] = v[i][kw + 1]; out[2] = v[i][kw + 2]; out[3] = v[i][kw + 3];
+        } else {
+            out[0] = v[i][kw]; out[1] = v[i][kw + 1]; out[2] = v[i][4 + kw]; out[3] = v[i][4 + kw + 1];
+        }
+    }
+};
+
+template <int kMode> struct IsTaps { static constexpr bool value = kMode == kGatherTaps4 || kMode == kGatherTaps2; };
+
+// One interface over both gather forms: the registers of one slice, how they are loaded and where their
+// squared, split values go in a K-major swizzled tile.  row0 = t >> 3 and kq = t & 7 of transform thread t.
+template <int kMode, bool kTaps = IsTaps<kMode>::value>
+struct Gatherer {
+    struct Regs { float v[kRowsPerThread][4]; };
+    GatherRows<kMode> g;
+    __device__ __forceinline__ void init(const Params &prm, const float *x, const float *delta, int origin, int row0, int limit)
+    {
+        g.init(prm, x, delta, origin + row0, limit);
+    }
+    __device__ __forceinline__ void load(const Params &prm, int z, int pbase, Regs &r) const { g.load(prm, z, pbase, r.v); }
+    __device__ __forceinline__ void store(uint8_t *hi, uint8_t *lo, int row0, int kq, const Regs &r) const
+    {
+#pragma unroll
+        for (int i = 0; i < kRowsPerThread; ++i)
+            split_store(hi, lo, chunk_offset(row0 + 32 * i, kq), r.v[i][0], r.v[i][1], r.v[i][2], r.v[i][3]);
+    }
+};
+template <int kMode>
+struct Gatherer<kMode, true> {
+    struct Regs { float v[2][8]; };
+    GatherTaps<kMode == kGatherTaps4 ? 4 : 2> g;
+    __device__ __forceinline__ void init(const Params &prm, const float *x, const float *, int origin, int row0, int limit)
+    {
+        g.init(prm, x, origin, row0, limit);
+    }
+    __device__ __forceinline__ void load(const Params &prm, int z, int pbase, Regs &r) const { g.load(prm, z, pbase, r.v); }
+    __device__ __forceinline__ void store(uint8_t *hi, uint8_t *lo, int, int kq, const Regs &r) const
+    {
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int kw = 0; kw < 3; ++kw) {
+                const int row = g.row_local[i] + kw;
+                if ((unsigned)row < (unsigned)kBM) {                 // kBM == kBN rows in either tile
+                    float o[4];
+                    g.tap(r.v, i, kw, o);
+                    split_store(hi, lo, chunk_offset(row, kq), o[0], o[1], o[2], o[3]);
+                }
+            }
+    }
+};
+
 // ---- the kernel ------------------------------------------------------------------------------
 template <int kMajor, int kModeA, int kModeB, bool kATmem>
 __global__ void __launch_bounds__(kThreadsTc, 1)
@@ -522,10 +636,12 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         const int group = kTwoGroups ? (t >> 7) : 0;
         const int tt = kTwoGroups ? (t & 127) : t;
         const int kq = t & 7, row0 = t >> 3;                               // gathered chunks: rows row0 + 32*i, k = 4*kq..4*kq+3
-        GatherRows<kModeA> rows_a;
-        GatherRows<kModeB> rows_b;
-        rows_a.init(prm, bt.x[layer], bt.delta[layer], m0 + row0, prm.M);
-        rows_b.init(prm, bt.x[layer], bt.delta[layer], n0 + row0, prm.N);
+        Gatherer<kModeA> rows_a;
+        Gatherer<kModeB> rows_b;
+        typedef typename Gatherer<kModeA>::Regs RegsA;
+        typedef typename Gatherer<kModeB>::Regs RegsB;
+        rows_a.init(prm, bt.x[layer], bt.delta[layer], m0, row0, prm.M);
+        rows_b.init(prm, bt.x[layer], bt.delta[layer], n0, row0, prm.N);
         // where the current slice sits: example z, 32-wide block pblk of that example's output positions
         int z = 0, pblk = 0;
         if (kAnyGather) {
@@ -535,13 +651,13 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         auto advance = [&]() {
             if (++pblk == prm.p_slices) { pblk = 0; ++z; }
         };
-        auto gather = [&](float (&ga)[kRowsPerThread][4], float (&gb)[kRowsPerThread][4]) {
+        auto gather = [&](RegsA &ga, RegsB &gb) {
             const int pbase = pblk * kBK + kq * 4;
             rows_a.load(prm, z, pbase, ga);
             rows_b.load(prm, z, pbase, gb);
         };
         // transform of slice i; gathered elements come in registers, TMA tiles from the raw stage
-        auto process = [&](int i, const float (&ga)[kRowsPerThread][4], const float (&gb)[kRowsPerThread][4]) -> bool {
+        auto process = [&](int i, const RegsA &ga, const RegsB &gb) -> bool {
             const int st = i % kNB, ls = i % kLoN;
             const uint32_t ph = (uint32_t)(i / kNB) & 1u;
             const int sa = kSplit ? i % kSplitA : 0;
@@ -608,17 +724,8 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                     }
                 }
             }
-            if (kGatherA) {
-#pragma unroll
-                for (int r = 0; r < kRowsPerThread; ++r)
-                    split_store(hi, lo, chunk_offset(row0 + 32 * r, kq), ga[r][0], ga[r][1], ga[r][2], ga[r][3]);
-            }
-            if (kGatherB) {
-#pragma unroll
-                for (int r = 0; r < kRowsPerThread; ++r)
-                    split_store(hi + kRawBytesA, lo + kRawBytesA, chunk_offset(row0 + 32 * r, kq), gb[r][0], gb[r][1],
-                                gb[r][2], gb[r][3]);
-            }
+            if (kGatherA) rows_a.store(hi, lo, row0, kq, ga);
+            if (kGatherB) rows_b.store(hi + kRawBytesA, lo + kRawBytesA, row0, kq, gb);
             if (kATmem) { tc_wait_st(); tc_fence_before(); }      // TMEM stores complete and ordered before the signal
             fence_async_smem();                                   // generic-proxy writes -> tensor core reads
             __syncwarp();
@@ -627,7 +734,8 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         };
 
         // two register sets in turn: the loads of slice i+1 are in flight while slice i is transformed
-        float a0[kRowsPerThread][4], b0[kRowsPerThread][4], a1[kRowsPerThread][4], b1[kRowsPerThread][4];
+        RegsA a0, a1;
+        RegsB b0, b1;
         if (kAnyGather) gather(a0, b0);
         if (kTwoGroups) {
             for (int i = group; i < n_slices; i += 2)
@@ -1124,7 +1232,22 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
     prm.chw = C * H * W;
     prm.wo_magic = (unsigned)(0x100000000ull / (unsigned)Wo) + 1u;
     const int e = err_tma ? kTma : kGatherErr, i = in_tma ? kTma : kGatherIm2col;
+    // three taps at a time: Kw = 3, stride 1 along w with pad 1 (then Wo == W), output width even, errors by TMA
+    const char *taps_env = getenv("VGC_TC_TAPS");
+    const int taps = (!(taps_env && atoi(taps_env) == 0) && i == kGatherIm2col && e == kTma && Kw == 3 && sw == 1 &&
+                      sh == 1 && pw == 1 && Wo == W && W % 2 == 0 && a_tmem)
+                         ? (W % 4 == 0 ? 4 : 2) : 0;
     KernelFn fn = nullptr;
+    if (taps && !swapped) {
+        prm.ld_m = n_im2col; prm.ld_n = 1;
+        fn = taps == 4 ? sqgrad_tc<kMajorK, kTma, kGatherTaps4, true> : sqgrad_tc<kMajorK, kTma, kGatherTaps2, true>;
+        return tc_launch(fn, bt, n_layers, prm, Cout, n_im2col, k_slices, ws, ws_bytes, st);
+    }
+    if (taps && swapped) {
+        prm.ld_m = 1; prm.ld_n = n_im2col;
+        fn = taps == 4 ? sqgrad_tc<kMajorK, kGatherTaps4, kTma, false> : sqgrad_tc<kMajorK, kGatherTaps2, kTma, false>;
+        return tc_launch(fn, bt, n_layers, prm, n_im2col, Cout, k_slices, ws, ws_bytes, st);
+    }
     if (!swapped) {     // S[o][idx]: m = o, n = idx
         prm.ld_m = n_im2col; prm.ld_n = 1;
         if (e == kTma && i == kTma) fn = a_tmem ? sqgrad_tc<kMajorK, kTma, kTma, true> : sqgrad_tc<kMajorK, kTma, kTma, false>;

@@ -80,6 +80,10 @@ CONV_SHAPES = [  # B, C, H, Cout, k, stride, pad
     # 1x1 layers that are repacked first: 7x7 planes (channel-major, flat reduction), strided (subsampled planes)
     (4, 70, 7, 130, 1, 1, 0), (4, 48, 14, 200, 1, 2, 0), (2, 96, 16, 160, 1, 2, 0), (3, 64, 28, 40, 1, 2, 0),
     (32, 160, 7, 144, 1, 1, 0),
+    # 3x3, stride 1, pad 1 with an even width: three taps per gathered row segment (width % 4 == 0 and == 2,
+    # many and few output channels, tiles whose first row is not the first tap of a triple)
+    (2, 24, 16, 130, 3, 1, 1), (2, 24, 14, 130, 3, 1, 1), (3, 50, 8, 40, 3, 1, 1), (2, 50, 6, 200, 3, 1, 1),
+    (1, 130, 4, 70, 3, 1, 1),
 ]
 REPACKED = [(4, 70, 7, 130, 1, 1, 0), (4, 48, 14, 200, 1, 2, 0), (2, 96, 16, 160, 1, 2, 0), (3, 64, 28, 40, 1, 2, 0)]
 
@@ -136,7 +140,7 @@ def test_repacked_and_in_place_forms_agree_with_the_oracle(monkeypatch, B, C, H,
 
 
 @pytest.mark.parametrize("env", [{"VGC_TC_ATMEM": "0"}, {"VGC_TC_GATHER": "1"}, {"VGC_TC_GATHER": "2"},
-                                 {"VGC_TC_GATHER": "3"}, {"VGC_SQGRAD_PATH": "simt"}])
+                                 {"VGC_TC_GATHER": "3"}, {"VGC_SQGRAD_PATH": "simt"}, {"VGC_TC_TAPS": "0"}])
 @pytest.mark.parametrize("B,C,H,Cout,k,s,p", [(3, 96, 12, 160, 1, 1, 0), (2, 40, 12, 48, 3, 1, 1), (2, 72, 16, 200, 3, 2, 1)])
 def test_every_kernel_variant_gives_the_same_statistic(monkeypatch, env, B, C, H, Cout, k, s, p):
     """The library picks a kernel form per layer (TMA or gathered tiles, A operand in shared or tensor memory,
