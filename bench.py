@@ -161,6 +161,7 @@ class HotPath:
             self.s_sets = [s for _, s in gs]
             self.ws_s = None
         else:
+            vgc.vgc_sqgrad_plan_hint(n_streams)
             ws_bytes = 16
             # conv layers of one geometry go to the library together (one launch per group of up to 8)
             groups = {}
@@ -253,19 +254,20 @@ class HotPath:
             main.wait_stream(st)
 
     def per_layer_times(self, reps: int = 5):
-        """Median device time of each layer's sqgrad call (ms), for profiling."""
+        """Median device time of each sqgrad library call (a layer, or a group of same-shaped layers) in ms."""
         vgc = self.vgc
         out = []
         ins = self.inputs[0]
-        for li, spec in enumerate(self.layers):
-            x, delta = ins[li]
-            S = self.s[int(self.offsets[li]):int(self.offsets[li + 1])]
+        for g in self.groups:
+            spec = self.layers[g[0]]
+            Ss = [self.s[int(self.offsets[li]):int(self.offsets[li + 1])] for li in g]
             def call():
                 if spec.kind == "conv":
-                    vgc.vgc_sqgrad_conv(x, delta, (spec.k, spec.k), (spec.stride, spec.stride), (spec.pad, spec.pad),
-                                        self.scale, S, ws=self.ws_s)
+                    vgc.vgc_sqgrad_conv_batch([ins[li][0] for li in g], [ins[li][1] for li in g], (spec.k, spec.k),
+                                              (spec.stride, spec.stride), (spec.pad, spec.pad), self.scale, Ss,
+                                              ws=self.ws_s)
                 else:
-                    vgc.vgc_sqgrad_linear(x, delta, self.scale, S, ws=self.ws_s)
+                    vgc.vgc_sqgrad_linear(ins[g[0]][0], ins[g[0]][1], self.scale, Ss[0], ws=self.ws_s)
             call(); torch.cuda.synchronize()
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph):
@@ -282,8 +284,9 @@ class HotPath:
                     times.append(e0.elapsed_time(e1) / 10)
             M, N, K = spec.gemm_mnk(self.batch)
             ms = statistics.median(times)
-            out.append({"layer": spec.name, "M": M, "N": N, "K": K, "ms": round(ms, 4),
-                        "useful_tflops": round(2 * M * N * K / (ms * 1e-3) / 1e12, 2)})
+            out.append({"layer": "+".join(self.layers[li].name for li in g), "layers": len(g), "M": M, "N": N, "K": K,
+                        "ms": round(ms, 4),
+                        "useful_tflops": round(len(g) * 2 * M * N * K / (ms * 1e-3) / 1e12, 2)})
         return out
 
     def compress(self, t: int, fused: bool = False):
@@ -592,7 +595,7 @@ def main():
     vgc.load_library()
     pk = peaks()
     hp = HotPath(args.workload, worker=rank * 16, n_input_sets=1, n_g_sets=max(4, min(args.steps + args.warmup, 16)),
-                 n_params=args.n_params, n_streams=max(args.streams, 1), algorithm=args.algorithm,
+                 n_params=args.n_params, n_streams=1 if args.per_layer else max(args.streams, 1), algorithm=args.algorithm,
                  batch_layers=not args.no_batch)
     if hp.hybrid:
         args.no_e2e = args.no_cpu_baseline = True

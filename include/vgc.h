@@ -103,6 +103,12 @@ vgc_status vgc_sqgrad_conv(const float *x, const float *delta, int B, int C, int
                            float scale, int accumulate, float *S,
                            void *ws, size_t ws_bytes, vgc_stream_t stream);
 
+/* Planning hint (no counterpart in the paper): how many sqgrad calls the caller keeps in flight side by side
+ * on different streams, each with its own workspace (default 1).  Alone, a launch is planned so that its
+ * blocks fill whole waves over the SMs; next to other launches a partly filled last wave costs nothing, and
+ * the reduction is split less.  Process-wide; set it BEFORE asking for workspace sizes, which depend on it. */
+void vgc_sqgrad_plan_hint(int concurrent_launches);
+
 /* Several conv layers of ONE geometry in one call (the residual stages of a deep network repeat the same
  * layer shapes): layer l computes what vgc_sqgrad_conv computes from x[l], delta[l] into S[l].  The tensor-
  * core path runs up to 8 layers per kernel launch, which shortens the split of the reduction, the scratch

@@ -27,7 +27,7 @@ EXPORTS = [
     "vgc_status_string", "vgc_version", "vgc_kernel_launch_count",
     "vgc_sqgrad_linear_workspace_bytes", "vgc_sqgrad_linear",
     "vgc_sqgrad_conv_workspace_bytes", "vgc_sqgrad_conv",
-    "vgc_sqgrad_conv_batch_workspace_bytes", "vgc_sqgrad_conv_batch",
+    "vgc_sqgrad_conv_batch_workspace_bytes", "vgc_sqgrad_conv_batch", "vgc_sqgrad_plan_hint",
     "vgc_compress_workspace_bytes", "vgc_compress", "vgc_compress_static",
     "vgc_decode_accumulate", "vgc_step_host",
     "vgc_compress_hybrid_workspace_bytes", "vgc_compress_hybrid", "vgc_decode_accumulate_hybrid",
@@ -90,6 +90,7 @@ def load_library():
     lib.vgc_sqgrad_conv_batch_workspace_bytes.restype = sz
     lib.vgc_sqgrad_conv_batch.argtypes = [i, vp, vp, vp] + [i] * 11 + [f, i, vp, sz, vp]
     lib.vgc_sqgrad_conv_batch.restype = i
+    lib.vgc_sqgrad_plan_hint.argtypes = [i]; lib.vgc_sqgrad_plan_hint.restype = None
     lib.vgc_compress_workspace_bytes.argtypes = [sz, i]
     lib.vgc_compress_workspace_bytes.restype = sz
     lib.vgc_compress.argtypes = [vp, vp, vp, vp, sz, vp, i, f, f, ctypes.POINTER(_MessageStruct), vp, sz, vp]
@@ -197,6 +198,11 @@ def vgc_sqgrad_conv(x, delta, kernel, stride, padding, scale: float, S, accumula
                                         _stream(stream))
     _check(st, "vgc_sqgrad_conv")
     return S
+
+
+def vgc_sqgrad_plan_hint(concurrent_launches: int) -> None:
+    """Tell the planner how many sqgrad calls run side by side (streams with separate workspaces)."""
+    load_library().vgc_sqgrad_plan_hint(int(concurrent_launches))
 
 
 def vgc_sqgrad_conv_batch_workspace_bytes(n_layers, B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw) -> int:

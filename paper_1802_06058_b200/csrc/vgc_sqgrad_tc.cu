@@ -950,19 +950,41 @@ struct Plan {
     int splits, slices_per_split, k_slices, tiles_x, tiles_y;
 };
 
+// how many sqgrad launches the caller keeps in flight side by side (vgc_sqgrad_plan_hint)
+static int g_concurrent_launches = 1;
+
 static Plan make_plan(int M, int N, int k_slices, int n_layers = 1)
 {
     Plan p;
     p.tiles_x = (N + kBN - 1) / kBN;
     p.tiles_y = (M + kBM - 1) / kBM;
     const long tiles = (long)p.tiles_x * p.tiles_y * n_layers;          // output tiles of the whole launch
-    // blocks of one launch: one per SM fills the device once; a caller that runs several layers side by side
-    // (separate streams and workspaces) may ask for fewer, longer blocks through VGC_TC_BLOCKS
+    // Blocks run one per SM, wave after wave.  A caller that runs several launches side by side (separate
+    // streams and workspaces, vgc_sqgrad_plan_hint) may also plan for fewer SMs per launch through VGC_TC_BLOCKS.
     const char *env = getenv("VGC_TC_BLOCKS");
     const long target = env && atoi(env) > 0 ? atoi(env) : 148;
-    long want = target / tiles;
-    if (want > k_slices) want = k_slices;
-    if (want < 1) want = 1;
+    long want = 1;
+    if (g_concurrent_launches > 1) {
+        // next to other launches a partly filled wave costs nothing (their blocks take the idle SMs): split the
+        // reduction as far as one wave allows and no further -- every extra block pays its fixed cost again
+        want = target / tiles;
+        if (want > k_slices) want = k_slices;
+        if (want < 1) want = 1;
+    } else {
+        // alone, the launch pays for whole waves: take the split with the shortest estimated makespan,
+        // waves x (slices per block + a block's fixed cost, about 8 slices' worth, + about 5 more for writing
+        // and re-reading a partial tile) + the combine pass
+        long best = -1;
+        const long max_split = k_slices < 256 ? k_slices : 256;
+        for (long sp = 1; sp <= max_split; ++sp) {
+            const long per = (k_slices + sp - 1) / sp;
+            if ((k_slices + per - 1) / per != sp) continue;              // splits that would get no slices
+            if (sp > 1 && tiles * sp > 6 * target) break;                 // keeps the split-K scratch L2-sized
+            const long waves = (tiles * sp + target - 1) / target;
+            const long cost = waves * (per + 8 + (sp > 1 ? 5 : 0)) + (sp > 1 ? 6 : 0);
+            if (best < 0 || cost < best) { best = cost; want = sp; }
+        }
+    }
     p.k_slices = k_slices;
     p.slices_per_split = (int)((k_slices + want - 1) / want);
     p.splits = (k_slices + p.slices_per_split - 1) / p.slices_per_split;
@@ -972,6 +994,8 @@ static Plan make_plan(int M, int N, int k_slices, int n_layers = 1)
 }  // namespace tc
 
 using namespace tc;
+
+void tc_plan_hint(int concurrent_launches) { g_concurrent_launches = concurrent_launches > 1 ? concurrent_launches : 1; }
 
 bool tc_linear_supported(int B, int in, int out)
 {
