@@ -91,13 +91,16 @@ def test_round_trip_of_compressed_messages():
     assert np.abs(u.cpu().numpy().astype(np.float64) - want).max() <= ATOL
 
 
-def test_scatter_form_agrees_with_the_default_merge_form(monkeypatch):
-    n, W = 400003, 5
-    offs = random_offsets(np.random.default_rng(21), n, 9)
+@pytest.mark.parametrize("n,K,W", [(400003, 9, 5), (3 * 24576 * 2 + 5, 3, 9), (2500000, 40, 17)])
+def test_every_decode_form_agrees_with_the_oracle(monkeypatch, n, K, W):
+    """Default: large tiles through shared memory; VGC_DECODE_PATH=merge: the 4096-element tile form;
+    VGC_DECODE_PATH=scatter: one atomic per word."""
+    offs = random_offsets(np.random.default_rng(21), n, K)
     msgs = [workloads.random_message(n, offs, 0.15 if w % 2 else 0.002, seed=900 + w, device="cuda") for w in range(W)]
-    merged, want, status, _ = _decode_both(n, offs, msgs, 0.5)
-    monkeypatch.setenv("VGC_DECODE_PATH", "scatter")
-    scattered, _, status2, _ = _decode_both(n, offs, msgs, 0.5)
-    assert status == 0 and status2 == 0
-    assert np.abs(merged.astype(np.float64) - want).max() <= ATOL
-    assert np.abs(scattered.astype(np.float64) - want).max() <= ATOL
+    u0 = torch.randn(n, device="cuda") * 1e-2
+    for path in (None, "merge", "scatter"):
+        if path:
+            monkeypatch.setenv("VGC_DECODE_PATH", path)
+        got, want, status, _ = _decode_both(n, offs, msgs, 0.5, u0=u0)
+        assert status == 0
+        assert np.abs(got.astype(np.float64) - want).max() <= ATOL
