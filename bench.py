@@ -301,11 +301,11 @@ class HotPath:
     def decode(self, t: int):
         if self.W == 0:
             return
-        self.u.zero_()
+        # u = mean of the W messages, every element written (no clearing pass, u is not read)
         if self.hybrid:
-            self.vgc.vgc_decode_accumulate_hybrid([self.out] + self.others, self.tau, 1.0 / self.W, self.u, self.status)
+            self.vgc.vgc_decode_sum_hybrid([self.out] + self.others, self.tau, 1.0 / self.W, self.u, self.status)
             return
-        self.vgc.vgc_decode_accumulate([self.out] + self.others, self.offs_dev, 1.0 / self.W, self.u, self.status)
+        self.vgc.vgc_decode_sum([self.out] + self.others, self.offs_dev, 1.0 / self.W, self.u, self.status)
 
     def step(self, t: int, marks=None):
         fused = self.fused and not self.compress_only
@@ -628,8 +628,8 @@ def main():
     compress_bytes = 24 * n + 8 * nnz_a + 4 * nnz
     if hp.hybrid:                                          # the staged word is written, read and written again
         compress_bytes = 24 * n + 12 * nnz
-    # decode: 4 B per word + one read and one write of u (merge form) + the 4 B/element clearing of u before it
-    decode_bytes = (4 * sum_nnz + 12 * n) if hp.W else 0
+    # decode (vgc_decode_sum): 4 B per word + one write of u
+    decode_bytes = (4 * sum_nnz + 4 * n) if hp.W else 0
     sections = {
         "sqgrad_ms": sq_ms, "compress_ms": co_ms, "decode_ms": de_ms,
         "sqgrad_useful_tflops": hp.flops_useful / (sq_ms * 1e-3) / 1e12 if sq_ms > 0 and hp.flops_useful else None,

@@ -220,6 +220,12 @@ vgc_status vgc_decode_accumulate(const vgc_message_view *msgs, int W,
                                  const uint32_t *group_offsets, int K, float scale,
                                  float *u, size_t n, uint32_t *dev_status, vgc_stream_t stream);
 
+/* Same sum, written instead of added:  u = scale * (sum over all words of all messages)  -- every element of
+ * u is written (zero where no word points), so the caller need not clear u first and u is not read.  This is
+ * the dense update of Sec. 4.3 when nothing else has been accumulated into the buffer. */
+vgc_status vgc_decode_sum(const vgc_message_view *msgs, int W, const uint32_t *group_offsets, int K,
+                          float scale, float *u, size_t n, uint32_t *dev_status, vgc_stream_t stream);
+
 /* ---------------------------------------------------------------------------------------------
  * One worker step from HOST buffers (end-to-end form of (1) + (2); Algorithm 1 from CalcGrad()'s
  * outputs to the encoded message).  For each layer, in order: copy x and delta from host memory into
@@ -285,6 +291,9 @@ vgc_status vgc_compress_hybrid(const float *g, const float *s, float *r, float *
                                const vgc_hybrid_message *out, void *ws, size_t ws_bytes, vgc_stream_t stream);
 vgc_status vgc_decode_accumulate_hybrid(const vgc_message_view *msgs, int W, float tau, float scale, float *u,
                                         size_t n, uint32_t *dev_status, vgc_stream_t stream);
+/* vgc_decode_sum for hybrid messages: u = scale * (sum of +-tau), every element written. */
+vgc_status vgc_decode_sum_hybrid(const vgc_message_view *msgs, int W, float tau, float scale, float *u, size_t n,
+                                 uint32_t *dev_status, vgc_stream_t stream);
 
 #ifdef __cplusplus
 }

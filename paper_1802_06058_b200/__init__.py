@@ -31,6 +31,7 @@ EXPORTS = [
     "vgc_compress_workspace_bytes", "vgc_compress", "vgc_compress_static",
     "vgc_decode_accumulate", "vgc_step_host",
     "vgc_compress_hybrid_workspace_bytes", "vgc_compress_hybrid", "vgc_decode_accumulate_hybrid",
+    "vgc_decode_sum", "vgc_decode_sum_hybrid",
 ]
 
 
@@ -102,12 +103,16 @@ def load_library():
     lib.vgc_step_host.restype = i
     lib.vgc_decode_accumulate.argtypes = [ctypes.POINTER(_ViewStruct), i, vp, i, f, vp, sz, vp, vp]
     lib.vgc_decode_accumulate.restype = i
+    lib.vgc_decode_sum.argtypes = lib.vgc_decode_accumulate.argtypes
+    lib.vgc_decode_sum.restype = i
     lib.vgc_compress_hybrid_workspace_bytes.argtypes = [sz]
     lib.vgc_compress_hybrid_workspace_bytes.restype = sz
     lib.vgc_compress_hybrid.argtypes = [vp, vp, vp, vp, sz, f, f, f, i, ctypes.POINTER(_HybridMessageStruct), vp, sz, vp]
     lib.vgc_compress_hybrid.restype = i
     lib.vgc_decode_accumulate_hybrid.argtypes = [ctypes.POINTER(_ViewStruct), i, f, f, vp, sz, vp, vp]
     lib.vgc_decode_accumulate_hybrid.restype = i
+    lib.vgc_decode_sum_hybrid.argtypes = lib.vgc_decode_accumulate_hybrid.argtypes
+    lib.vgc_decode_sum_hybrid.restype = i
     _lib = lib
     return lib
 
@@ -321,11 +326,13 @@ def vgc_compress_static(g, s, r, v, group_offsets, alpha: float, zeta: float, ou
 
 
 # ------------------------------------------------------------------------------------------ (3)
-def vgc_decode_accumulate(messages: Sequence, group_offsets, scale: float, u, dev_status, stream=None):
+def vgc_decode_accumulate(messages: Sequence, group_offsets, scale: float, u, dev_status, stream=None,
+                          overwrite: bool = False):
     """u[idx] += scale * decoded value over all words of all messages.
 
     ``messages``: MessageBuffers objects, or (words int32, nnz int32[1], group_exp int32) tensor triples.
-    ``dev_status``: int32[1] device tensor (zeroed by the caller) receiving VGC_DEV_* bits."""
+    ``dev_status``: int32[1] device tensor (zeroed by the caller) receiving VGC_DEV_* bits.
+    ``overwrite``: write u = scale * sum instead (vgc_decode_sum): u is neither read nor needs clearing."""
     W = len(messages)
     views = (_ViewStruct * max(W, 1))()
     for w, m in enumerate(messages):
@@ -336,11 +343,17 @@ def vgc_decode_accumulate(messages: Sequence, group_offsets, scale: float, u, de
             views[w] = _ViewStruct(_dev(words, torch.int32, "words"), _dev(nnz, torch.int32, "nnz"),
                                    _dev(gexp, torch.int32, "group_exp"))
     K = group_offsets.numel() - 1
-    st = load_library().vgc_decode_accumulate(views, W, _dev(group_offsets, torch.int32, "group_offsets"), K,
-                                              float(scale), _dev(u, torch.float32, "u"), u.numel(),
-                                              _dev(dev_status, torch.int32, "dev_status"), _stream(stream))
-    _check(st, "vgc_decode_accumulate")
+    lib = load_library()
+    fn = lib.vgc_decode_sum if overwrite else lib.vgc_decode_accumulate
+    st = fn(views, W, _dev(group_offsets, torch.int32, "group_offsets"), K, float(scale), _dev(u, torch.float32, "u"),
+            u.numel(), _dev(dev_status, torch.int32, "dev_status"), _stream(stream))
+    _check(st, "vgc_decode_sum" if overwrite else "vgc_decode_accumulate")
     return u
+
+
+def vgc_decode_sum(messages: Sequence, group_offsets, scale: float, u, dev_status, stream=None):
+    """u = scale * (sum of all words of all messages); every element of u is written."""
+    return vgc_decode_accumulate(messages, group_offsets, scale, u, dev_status, stream, overwrite=True)
 
 
 # ------------------------------------------------------------------------------------------ (4)
@@ -389,7 +402,13 @@ def vgc_compress_hybrid(g, s, r, v, alpha: float, zeta: float, tau: float, out: 
     return out
 
 
-def vgc_decode_accumulate_hybrid(messages: Sequence, tau: float, scale: float, u, dev_status, stream=None):
+def vgc_decode_sum_hybrid(messages: Sequence, tau: float, scale: float, u, dev_status, stream=None):
+    """u = scale * (sum of +-tau over all words); every element of u is written."""
+    return vgc_decode_accumulate_hybrid(messages, tau, scale, u, dev_status, stream, overwrite=True)
+
+
+def vgc_decode_accumulate_hybrid(messages: Sequence, tau: float, scale: float, u, dev_status, stream=None,
+                                 overwrite: bool = False):
     """u[idx] += scale * (+-tau) over all words of all messages (HybridMessageBuffers or (words, nnz) pairs)."""
     W = len(messages)
     views = (_ViewStruct * max(W, 1))()
@@ -399,9 +418,10 @@ def vgc_decode_accumulate_hybrid(messages: Sequence, tau: float, scale: float, u
         else:
             words, nnz = m
             views[w] = _ViewStruct(_dev(words, torch.int32, "words"), _dev(nnz, torch.int32, "nnz"), None)
-    st = load_library().vgc_decode_accumulate_hybrid(views, W, float(tau), float(scale), _dev(u, torch.float32, "u"),
-                                                     u.numel(), _dev(dev_status, torch.int32, "dev_status"),
-                                                     _stream(stream))
+    lib = load_library()
+    fn = lib.vgc_decode_sum_hybrid if overwrite else lib.vgc_decode_accumulate_hybrid
+    st = fn(views, W, float(tau), float(scale), _dev(u, torch.float32, "u"), u.numel(),
+            _dev(dev_status, torch.int32, "dev_status"), _stream(stream))
     _check(st, "vgc_decode_accumulate_hybrid")
     return u
 

@@ -551,6 +551,11 @@ vgc_status decode_launch(bool hybrid, bool overwrite, const vgc_message_view *ms
         VGC_CUDA_OK(cudaDeviceGetAttribute(&c, cudaDevAttrMultiProcessorCount, dev));
         sm_count = c > 0 ? c : 148;
     }
+    const char *path_env = getenv("VGC_DECODE_PATH");
+    if (overwrite && (W == 0 || (path_env && (path_env[0] == 's' || path_env[0] == 'm')))) {
+        VGC_CUDA_OK(cudaMemsetAsync(u, 0, n * sizeof(float), st));   // the other forms only accumulate
+        overwrite = false;
+    }
     for (int w0 = 0; w0 < W; w0 += kMaxViews) {
         const int wb = W - w0 < kMaxViews ? W - w0 : kMaxViews;
         DecodeViews views;
@@ -632,5 +637,30 @@ extern "C" vgc_status vgc_decode_accumulate_hybrid(const vgc_message_view *msgs,
     for (int w = 0; w < W; ++w)
         if (!msgs[w].words || !msgs[w].nnz) return VGC_ERR_INVALID_ARG;
     return decode_launch(true, false, msgs, W, nullptr, 0, scale, tau, u, n, dev_status,
+                         reinterpret_cast<cudaStream_t>(stream));
+}
+
+extern "C" vgc_status vgc_decode_sum(const vgc_message_view *msgs, int W, const uint32_t *group_offsets, int K,
+                                     float scale, float *u, size_t n, uint32_t *dev_status, vgc_stream_t stream)
+{
+    if (n == 0) return VGC_OK;
+    if (W < 0 || K < 1 || n > VGC_MAX_PARAMS || (W > 0 && !msgs) || !group_offsets || !u || !dev_status || !aligned16(u))
+        return VGC_ERR_INVALID_ARG;
+    if (!(scale == scale)) return VGC_ERR_INVALID_ARG;
+    for (int w = 0; w < W; ++w)
+        if (!msgs[w].words || !msgs[w].nnz || !msgs[w].group_exp) return VGC_ERR_INVALID_ARG;
+    return decode_launch(false, true, msgs, W, group_offsets, K, scale, 0.f, u, n, dev_status,
+                         reinterpret_cast<cudaStream_t>(stream));
+}
+
+extern "C" vgc_status vgc_decode_sum_hybrid(const vgc_message_view *msgs, int W, float tau, float scale, float *u,
+                                            size_t n, uint32_t *dev_status, vgc_stream_t stream)
+{
+    if (n == 0) return VGC_OK;
+    if (W < 0 || n > VGC_MAX_PARAMS || (W > 0 && !msgs) || !u || !dev_status || !aligned16(u)) return VGC_ERR_INVALID_ARG;
+    if (!(scale == scale) || !(tau == tau)) return VGC_ERR_INVALID_ARG;
+    for (int w = 0; w < W; ++w)
+        if (!msgs[w].words || !msgs[w].nnz) return VGC_ERR_INVALID_ARG;
+    return decode_launch(true, true, msgs, W, nullptr, 0, scale, tau, u, n, dev_status,
                          reinterpret_cast<cudaStream_t>(stream));
 }

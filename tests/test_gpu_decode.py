@@ -104,3 +104,31 @@ def test_every_decode_form_agrees_with_the_oracle(monkeypatch, n, K, W):
         got, want, status, _ = _decode_both(n, offs, msgs, 0.5, u0=u0)
         assert status == 0
         assert np.abs(got.astype(np.float64) - want).max() <= ATOL
+
+
+@pytest.mark.parametrize("path", [None, "merge", "scatter"])
+@pytest.mark.parametrize("n,K,W,density", [(5, 1, 1, 1.0), (100003, 7, 4, 0.0005), (1 << 20, 54, 8, 0.1),
+                                           (2500001, 16, 70, 0.02)])
+def test_decode_sum_overwrites_whatever_u_held(monkeypatch, path, n, K, W, density):
+    if path:
+        monkeypatch.setenv("VGC_DECODE_PATH", path)
+    offs = random_offsets(np.random.default_rng(n + W), n, K)
+    msgs = [workloads.random_message(n, offs, density, seed=workloads.seed_for(6, w, 0, 0, 2), device="cuda")
+            for w in range(W)]
+    u = torch.full((n,), float("nan"), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    pad = torch.zeros(4, dtype=torch.int32, device="cuda")
+    triples = [(w if w.numel() else pad, torch.tensor([w.numel()], dtype=torch.int32, device="cuda"), e) for w, e in msgs]
+    vgc.vgc_decode_sum(triples, vgc.offsets_tensor(offs), 0.25, u, status)
+    want = np.zeros(n, F32)
+    oracle.decode_accumulate([(w.cpu().numpy().view(np.uint32), e.cpu().numpy()) for w, e in msgs], offs, 0.25, want)
+    assert int(status.item()) == 0
+    assert np.abs(u.cpu().numpy().astype(np.float64) - want).max() <= ATOL
+
+
+def test_decode_sum_of_no_messages_is_zero():
+    n = 12345
+    u = torch.full((n,), 3.0, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    vgc.vgc_decode_sum([], vgc.offsets_tensor(np.array([0, n], np.uint32)), 1.0, u, status)
+    assert float(u.abs().max().item()) == 0.0

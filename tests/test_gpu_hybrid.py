@@ -110,11 +110,12 @@ def hybrid_message(rng, n, density):
     return (idx << 4) | (sign << 3)
 
 
-@pytest.mark.parametrize("path", ["merge", "scatter"])
+@pytest.mark.parametrize("path", [None, "merge", "scatter"])
 @pytest.mark.parametrize("n,W,density", [(1, 1, 1.0), (4097, 3, 0.3), (300007, 8, 0.05), (300007, 2, 0.0005),
                                          ((1 << 21) + 3, 16, 0.02), (70000, 70, 0.2)])
 def test_decode(n, W, density, path, monkeypatch):
-    monkeypatch.setenv("VGC_DECODE_PATH", path)
+    if path:
+        monkeypatch.setenv("VGC_DECODE_PATH", path)
     rng = np.random.default_rng(n + W)
     msgs = [hybrid_message(rng, n, density) for _ in range(W)]
     tau, scale = 0.0123, 1.0 / W
@@ -147,5 +148,23 @@ def test_compress_then_decode_round_trip():
     u = torch.zeros(n, dtype=torch.float32, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     vgc.vgc_decode_accumulate_hybrid([wk.out for wk in workers], tau, 1.0 / W, u, status)
+    assert int(status.item()) == 0
+    np.testing.assert_allclose(u.cpu().numpy(), want, rtol=0, atol=1e-6)
+
+
+@pytest.mark.parametrize("n,W,density", [(4097, 3, 0.3), (300007, 2, 0.0005), ((1 << 21) + 3, 9, 0.05)])
+def test_decode_sum(n, W, density):
+    rng = np.random.default_rng(n + W)
+    msgs = [hybrid_message(rng, n, density) for _ in range(W)]
+    tau, scale = 0.0123, 1.0 / W
+    want = np.zeros(n, F32)
+    assert oracle.decode_hybrid(msgs, tau, scale, want) == 0
+    u = torch.full((n,), float("nan"), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dev = []
+    for m in msgs:
+        buf = np.zeros(max(m.size, 4), np.uint32); buf[:m.size] = m
+        dev.append((torch.from_numpy(buf.view(np.int32)).cuda(), torch.tensor([m.size], dtype=torch.int32, device="cuda")))
+    vgc.vgc_decode_sum_hybrid(dev, tau, scale, u, status)
     assert int(status.item()) == 0
     np.testing.assert_allclose(u.cpu().numpy(), want, rtol=0, atol=1e-6)
