@@ -646,7 +646,7 @@ def main():
     # DRAM traffic measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum), per launch group:
     # profiles/sqgrad_tc_resnet50_pass.md (one pass over the 54 ResNet-50 layers) and
     # profiles/compress_flat_n33554432.md (scaled by n: the traffic is proportional to the buffer length)
-    NCU_SQGRAD_PASS_BYTES_RESNET50 = 3.21e9
+    NCU_SQGRAD_PASS_BYTES_RESNET50 = 3.20e9
     NCU_COMPRESS_BYTES_PER_PARAM = (537.7e6 + 233.9e6 + 20.7e6 + 20.7e6) / 33554432
     compress_roofline = {"kernel": "compress_phase_a + compress_count + compress_emit", "bound": "hbm",
                          "achieved": compress_bytes / (co_ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
@@ -664,7 +664,7 @@ def main():
                     "peak_source": f"{pk['source']} bf16 sustained x 1/2 (tf32 nominal ratio), of measured",
                     "note": "achieved = algorithmic flops 2*M*N*K per layer / sqgrad time; the 3xTF32 scheme "
                             "issues 3 tensor-core products per algorithmic one (issued_frac = tensor-pipe load); "
-                            "traffic = DRAM bytes of the 103 launches of one pass"}
+                            "traffic = DRAM bytes of the 46 launches of one pass (profiles/launch_list_resnet50.md)"}
     else:
         roofline = compress_roofline
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
