@@ -1082,14 +1082,20 @@ static bool conv_swapped(int Cout, int n_im2col) { return Cout <= 64 && n_im2col
 //   kRepackFlat     x_r[c][z P + p], d_r[o][z P + p]: channel-major, the (example, position) pairs of one
 //                   channel back to back -- the layer becomes a 1x1 convolution over ONE example with
 //                   B P positions, and its reduction has no per-example padding to whole slices
-enum { kRepackNone = 0, kRepackPlanes = 1, kRepackFlat = 2 };
+//   kRepackPadW     a Kw = 3, stride-1, pad_w = 1 kernel on planes of odd width W (7x7): x and the errors are
+//                   copied into planes of width W4 = W rounded up to 4 with zero columns.  The zero input column
+//                   is the right-hand padding, the zero error columns contribute nothing, so the statistic is
+//                   unchanged -- and the padded layer has TMA-able error planes and takes the three-tap gather
+enum { kRepackNone = 0, kRepackPlanes = 1, kRepackFlat = 2, kRepackPadW = 3 };
 
-static int repack_mode(int B, int C, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw, int P)
+static int repack_mode(int B, int C, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw, int P, int W = 0, int Ho = 0)
 {
-    if (Kh != 1 || Kw != 1 || ph != 0 || pw != 0) return kRepackNone;
-    if ((long)B * C >= (1L << 31) || (long)B * Cout >= (1L << 31)) return kRepackNone;      // 32-bit row index
     const char *e = getenv("VGC_TC_REPACK");
     if (e && atoi(e) == 0) return kRepackNone;
+    if ((long)B * C >= (1L << 31) || (long)B * Cout >= (1L << 31)) return kRepackNone;      // 32-bit row index
+    if (Kw == 3 && sw == 1 && sh == 1 && pw == 1 && W % 2 == 1 && W >= 3 && (long)Ho * ((W + 3) / 4 * 4) >= kBK)
+        return kRepackPadW;
+    if (Kh != 1 || Kw != 1 || ph != 0 || pw != 0) return kRepackNone;
     const bool planes_ok = P >= kBK && P % 4 == 0;
     if (planes_ok) return (sh > 1 || sw > 1) ? kRepackPlanes : kRepackNone;
     const long flat = (long)B * P;
@@ -1101,12 +1107,12 @@ static int repack_mode(int B, int C, int Cout, int Kh, int Kw, int sh, int sw, i
 // loads in flight per lane.
 __global__ void __launch_bounds__(256)
 sqgrad_repack(const float *__restrict__ in, float *__restrict__ out, int B, int C, int HW, int W, int Wo, int P,
-              int sh, int sw, int channel_major)
+              int sh, int sw, int channel_major, int wo_valid)
 {
     constexpr int kRows = 4, kCols = 2;
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t rows = (uint32_t)B * (uint32_t)C;
-    const bool dense = sh == 1 && sw == 1 && W == Wo;                 // the plane is copied as it is
+    const bool dense = sh == 1 && sw == 1 && W == Wo && wo_valid == Wo;   // the plane is copied as it is
     for (uint32_t row0 = (blockIdx.x * 8 + (threadIdx.x >> 5)) * kRows; row0 < rows; row0 += gridDim.x * 8 * kRows) {
         const float *src[kRows];
 #pragma unroll
@@ -1120,17 +1126,23 @@ sqgrad_repack(const float *__restrict__ in, float *__restrict__ out, int B, int 
         for (uint32_t p0 = 0; p0 < (uint32_t)P; p0 += 32 * kCols) {
             float v[kRows][kCols];
             uint32_t off[kCols];
+            bool live[kCols];                                           // columns wo >= wo_valid are zero padding
 #pragma unroll
             for (int u = 0; u < kCols; ++u) {
                 const uint32_t p = p0 + lane + 32u * u;
+                live[u] = p < (uint32_t)P;
                 if (dense) off[u] = p;
-                else { const uint32_t ho = p / (uint32_t)Wo, wo = p - ho * (uint32_t)Wo; off[u] = ho * sh * W + wo * sw; }
+                else {
+                    const uint32_t ho = p / (uint32_t)Wo, wo = p - ho * (uint32_t)Wo;
+                    off[u] = ho * sh * W + wo * sw;
+                    live[u] = live[u] && wo < (uint32_t)wo_valid;
+                }
             }
 #pragma unroll
             for (int r = 0; r < kRows; ++r)
 #pragma unroll
                 for (int u = 0; u < kCols; ++u)
-                    v[r][u] = (p0 + lane + 32u * u < (uint32_t)P) ? __ldg(src[r] + off[u]) : 0.f;
+                    v[r][u] = live[u] ? __ldg(src[r] + off[u]) : 0.f;
 #pragma unroll
             for (int r = 0; r < kRows; ++r)
 #pragma unroll
@@ -1151,14 +1163,21 @@ static size_t conv_workspace_plain(int n_layers, int B, int C, int Kh, int Kw, i
 
 // Workspace of one launch over n_layers layers of this geometry (n_layers <= kMaxBatch).
 static size_t conv_workspace_group(int n_layers, int B, int C, int Kh, int Kw, int sh, int sw, int ph, int pw, int P,
-                                   int Cout)
+                                   int Cout, int Wo_)
 {
     // the larger of the in-place form and the repacked one, so that either can be chosen at call time
     size_t need = conv_workspace_plain(n_layers, B, C, Kh, Kw, P, Cout);
-    const int mode = repack_mode(B, C, Cout, Kh, Kw, sh, sw, ph, pw, P);
+    // the width W of the input equals the output width whenever kRepackPadW applies, and P / Wo = Ho
+    const int mode = repack_mode(B, C, Cout, Kh, Kw, sh, sw, ph, pw, P, Wo_, Wo_ ? P / Wo_ : 0);
     const size_t x_bytes = round_up(sizeof(float) * (size_t)B * C * P, 256);
     const size_t d_bytes = round_up(sizeof(float) * (size_t)B * Cout * P, 256);
-    if (mode == kRepackPlanes) {
+    if (mode == kRepackPadW) {
+        const int W4 = (Wo_ + 3) / 4 * 4, Ho = P / Wo_, H = Ho + Kh - 1 - 2 * ph;      // stride 1
+        const size_t xp = round_up(sizeof(float) * (size_t)B * C * H * W4, 256);
+        const size_t dp = round_up(sizeof(float) * (size_t)B * Cout * Ho * W4, 256);
+        const size_t r = round_up(conv_workspace_plain(n_layers, B, C, Kh, Kw, Ho * W4, Cout), 256) + n_layers * (xp + dp);
+        need = need > r ? need : r;
+    } else if (mode == kRepackPlanes) {
         const size_t r = round_up(conv_workspace_plain(n_layers, B, C, 1, 1, P, Cout), 256) + n_layers * x_bytes;
         need = need > r ? need : r;
     } else if (mode == kRepackFlat) {
@@ -1170,14 +1189,14 @@ static size_t conv_workspace_group(int n_layers, int B, int C, int Kh, int Kw, i
 }
 
 size_t tc_conv_workspace_bytes(int n_layers, int B, int C, int Kh, int Kw, int sh, int sw, int ph, int pw, int P,
-                               int Cout)
+                               int Cout, int Wo_)
 {
     // more layers than one launch takes are processed group after group in the same workspace
     const int first = n_layers < kMaxBatch ? n_layers : kMaxBatch;
-    size_t need = conv_workspace_group(first, B, C, Kh, Kw, sh, sw, ph, pw, P, Cout);
+    size_t need = conv_workspace_group(first, B, C, Kh, Kw, sh, sw, ph, pw, P, Cout, Wo_);
     const int rest = n_layers > kMaxBatch ? n_layers % kMaxBatch : 0;
     if (rest) {
-        const size_t r = conv_workspace_group(rest, B, C, Kh, Kw, sh, sw, ph, pw, P, Cout);
+        const size_t r = conv_workspace_group(rest, B, C, Kh, Kw, sh, sw, ph, pw, P, Cout, Wo_);
         need = need > r ? need : r;
     }
     return need;
@@ -1188,7 +1207,27 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
                              int Wo, float scale, int accumulate, void *ws, size_t ws_bytes, cudaStream_t st)
 {
     const int P = Ho * Wo, n_im2col = C * Kh * Kw;
-    const int mode = repack_mode(B, C, Cout, Kh, Kw, sh, sw, ph, pw, P);
+    const int mode = repack_mode(B, C, Cout, Kh, Kw, sh, sw, ph, pw, P, W, Ho);
+    // one warp per row; a few rows per warp when there are many
+    auto blocks_for = [](size_t rows) { const size_t b = (rows + 31) / 32; return (unsigned)(b < 1 ? 1 : (b > 148 * 32 ? 148 * 32 : b)); };
+    if (mode == kRepackPadW) {
+        const int W4 = (W + 3) / 4 * 4;
+        const size_t inner = round_up(conv_workspace_plain(n_layers, B, C, Kh, Kw, Ho * W4, Cout), 256);
+        const size_t xp = round_up(sizeof(float) * (size_t)B * C * H * W4, 256);
+        const size_t dp = round_up(sizeof(float) * (size_t)B * Cout * Ho * W4, 256);
+        if (ws_bytes < inner + n_layers * (xp + dp)) return VGC_ERR_WORKSPACE;
+        const float *xr[kMaxBatch], *dr[kMaxBatch];
+        for (int l = 0; l < n_layers; ++l) {
+            char *base = static_cast<char *>(ws) + inner + (size_t)l * (xp + dp);
+            float *x_p = reinterpret_cast<float *>(base), *d_p = reinterpret_cast<float *>(base + xp);
+            sqgrad_repack<<<blocks_for((size_t)B * C), 256, 0, st>>>(x[l], x_p, B, C, H * W, W, W4, H * W4, 1, 1, 0, W);
+            sqgrad_repack<<<blocks_for((size_t)B * Cout), 256, 0, st>>>(delta[l], d_p, B, Cout, Ho * Wo, Wo, W4, Ho * W4, 1, 1,
+                                                                       0, Wo);
+            count_launch(2);
+            xr[l] = x_p; dr[l] = d_p;
+        }
+        return conv_group(n_layers, xr, dr, S, B, C, H, W4, Cout, Kh, Kw, 1, 1, ph, 1, Ho, W4, scale, accumulate, ws, inner, st);
+    }
     if (mode != kRepackNone) {
         const bool flat = mode == kRepackFlat;
         const size_t inner = round_up(flat ? conv_workspace_plain(n_layers, 1, C, 1, 1, B * P, Cout)
@@ -1196,16 +1235,14 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
         const size_t x_bytes = round_up(sizeof(float) * (size_t)B * C * P, 256);
         const size_t d_bytes = flat ? round_up(sizeof(float) * (size_t)B * Cout * P, 256) : 0;
         if (ws_bytes < inner + n_layers * (x_bytes + d_bytes)) return VGC_ERR_WORKSPACE;
-        // one warp per row; a few rows per warp when there are many
-        auto blocks_for = [](size_t rows) { const size_t b = (rows + 31) / 32; return (unsigned)(b < 1 ? 1 : (b > 148 * 32 ? 148 * 32 : b)); };
         const float *xr[kMaxBatch], *dr[kMaxBatch];
         for (int l = 0; l < n_layers; ++l) {
             char *base = static_cast<char *>(ws) + inner + (size_t)l * (x_bytes + d_bytes);
             float *x_r = reinterpret_cast<float *>(base), *d_r = reinterpret_cast<float *>(base + x_bytes);
-            sqgrad_repack<<<blocks_for((size_t)B * C), 256, 0, st>>>(x[l], x_r, B, C, H * W, W, Wo, P, sh, sw, flat ? 1 : 0);
+            sqgrad_repack<<<blocks_for((size_t)B * C), 256, 0, st>>>(x[l], x_r, B, C, H * W, W, Wo, P, sh, sw, flat ? 1 : 0, Wo);
             count_launch();
             if (flat) {
-                sqgrad_repack<<<blocks_for((size_t)B * Cout), 256, 0, st>>>(delta[l], d_r, B, Cout, P, Wo, Wo, P, 1, 1, 1);
+                sqgrad_repack<<<blocks_for((size_t)B * Cout), 256, 0, st>>>(delta[l], d_r, B, Cout, P, Wo, Wo, P, 1, 1, 1, Wo);
                 count_launch();
             }
             xr[l] = x_r;

@@ -84,8 +84,11 @@ CONV_SHAPES = [  # B, C, H, Cout, k, stride, pad
     # many and few output channels, tiles whose first row is not the first tap of a triple)
     (2, 24, 16, 130, 3, 1, 1), (2, 24, 14, 130, 3, 1, 1), (3, 50, 8, 40, 3, 1, 1), (2, 50, 6, 200, 3, 1, 1),
     (1, 130, 4, 70, 3, 1, 1),
+    # 3x3, stride 1, pad 1 on odd widths: planes padded to a multiple of 4 columns first
+    (2, 40, 7, 130, 3, 1, 1), (4, 130, 7, 48, 3, 1, 1), (2, 16, 5, 72, 3, 1, 1),
 ]
-REPACKED = [(4, 70, 7, 130, 1, 1, 0), (4, 48, 14, 200, 1, 2, 0), (2, 96, 16, 160, 1, 2, 0), (3, 64, 28, 40, 1, 2, 0)]
+REPACKED = [(4, 70, 7, 130, 1, 1, 0), (4, 48, 14, 200, 1, 2, 0), (2, 96, 16, 160, 1, 2, 0), (3, 64, 28, 40, 1, 2, 0),
+            (2, 40, 7, 130, 3, 1, 1), (3, 24, 9, 20, 3, 1, 1)]
 
 
 @pytest.mark.parametrize("B,C,H,Cout,k,s,p", CONV_SHAPES)
