@@ -146,7 +146,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try(bar, parity)) return true;
         if (i >= 4) {
             if (*abort_flag) return false;
-            __nanosleep(sleep_ns);
+            if (sleep_ns) __nanosleep(sleep_ns);
         }
     }
     *abort_flag = 1;
@@ -195,6 +195,25 @@ __device__ __forceinline__ void tc_mma_tf32_ts(uint32_t d_tmem, uint32_t a_tmem,
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// the same two with "accumulate" fixed to true (no predicate to compute in the issuing thread)
+__device__ __forceinline__ void tc_mma_tf32_acc(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.eq.u32 p, 1, 1;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc)
+        : "memory");
+}
+__device__ __forceinline__ void tc_mma_tf32_ts_acc(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.eq.u32 p, 1, 1;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc)
         : "memory");
 }
 // 32 lanes x 16 columns: each thread stores 16 registers into its lane's row
@@ -472,7 +491,8 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
     uint8_t *smem_gen = smem_raw_ + (smem_base - smem_u32(smem_raw_));
 
     // per raw slot: raw_full (TMA landed) -> op_full (hi/lo written) -> empty (MMAs that read it retired);
-    // per lo slot: lo_empty (MMAs that read it retired)
+    // a lo slot (and its A slot in tensor memory) is free when the MMAs of the slice that used it last have
+    // retired, which is what that slice's `empty` barrier says: no barrier of its own, one commit per slice
     uint64_t *raw_full = bars, *op_full = bars + kNB, *empty = bars + 2 * kNB;
     uint64_t *lo_empty = bars + 3 * kNB;
     uint64_t *acc_full = lo_empty + kLoSlotsAT, *acc_empty = acc_full + 2, *drain = acc_empty + 2;
@@ -501,7 +521,7 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                 mbar_init(smem_u32(&a_full[i]), 1);
                 mbar_init(smem_u32(&a_empty[i]), kTransformWarps / 2);
             }
-        for (int i = 0; i < kLoSlotsAT; ++i) mbar_init(smem_u32(&lo_empty[i]), 1);
+        for (int i = 0; i < kLoSlotsAT; ++i) mbar_init(smem_u32(&lo_empty[i]), 1);      // unused, kept initialised
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&acc_full[i]), 1); mbar_init(smem_u32(&acc_empty[i]), kEpilogueWarps); }
         mbar_init(smem_u32(drain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -581,43 +601,52 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
             const uint32_t lbo = kMajor == kMajorK ? 16u : 4096u;
             const uint32_t sbo = kMajor == kMajorK ? 1024u : 512u;
             const uint32_t layout = kMajor == kMajorK ? 2u : 1u;
-            const uint32_t k_step = kMajor == kMajorK ? 32u : 1024u;        // bytes per 8-deep MMA step
-            int i = 0;
+            constexpr uint32_t k_step16 = (kMajor == kMajorK ? 32u : 1024u) >> 4;   // 16-byte units per 8-deep MMA step
+            // This one thread feeds the tensor pipe, so its instruction stream is kept short: the descriptor's
+            // upper word and the LBO field never change, the start-address field (address >> 4; shared memory
+            // is < 256 KB, so it cannot overflow its 14 bits) is one addition per operand and step.
+            const uint32_t desc_hi = (uint32_t)(smem_desc(0, lbo, sbo, layout) >> 32);
+            const uint32_t desc_lo0 = (uint32_t)smem_desc(0, lbo, sbo, layout);
+            auto desc_at = [&](uint32_t lo16) -> uint64_t { return ((uint64_t)desc_hi << 32) | (desc_lo0 + lo16); };
+            int i = 0, st = 0, ls = 0;                   // slice, its raw / hi slot, its lo slot
+            uint32_t st_phase = 0;
             bool ok = true;
             for (int c = 0; c < n_chunks && ok; ++c) {
                 const int b = c & 1;
-                ok = mbar_wait(smem_u32(&acc_empty[b]), ((uint32_t)(c >> 1) & 1u) ^ 1u, &abort_flag);
+                ok = mbar_wait(smem_u32(&acc_empty[b]), ((uint32_t)(c >> 1) & 1u) ^ 1u, &abort_flag, 0);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)b * kBN;
                 const int chunk_end = min(n_slices, (c + 1) * prm.chunk);
                 for (bool first = true; i < chunk_end; ++i) {
-                    const int st = i % kNB, ls = i % kLoN;
-                    ok = mbar_wait(smem_u32(&op_full[st]), (uint32_t)(i / kNB) & 1u, &abort_flag);
+                    ok = mbar_wait(smem_u32(&op_full[st]), st_phase, &abort_flag, 0);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t hi_a = smem_base + pair_off(st), hi_b = hi_a + kRawBytesA;
-                    const uint32_t lo_a = smem_base + lo_off(ls), lo_b = lo_a + kRawBytesA;     // lo_a unused with A in TMEM
+                    const uint32_t hi_a16 = (smem_base + pair_off(st)) >> 4, hi_b16 = hi_a16 + (kRawBytesA >> 4);
+                    const uint32_t lo_a16 = (smem_base + lo_off(ls)) >> 4, lo_b16 = lo_a16 + (kRawBytesA >> 4);   // lo_a unused with A in TMEM
                     const uint32_t ta_hi = tmem_base + 2 * kBN + ls * kTmemColsA, ta_lo = ta_hi + 32;
 #pragma unroll
                     for (int kk = 0; kk < kBK / 8; ++kk) {
-                        const uint64_t db_hi = smem_desc(hi_b + kk * k_step, lbo, sbo, layout);
-                        const uint64_t db_lo = smem_desc(lo_b + kk * k_step, lbo, sbo, layout);
+                        const uint64_t db_hi = desc_at(hi_b16 + kk * k_step16);
+                        const uint64_t db_lo = desc_at(lo_b16 + kk * k_step16);
                         if (kATmem) {
-                            tc_mma_tf32_ts(d_tmem, ta_hi + kk * 8, db_hi, idesc, first ? 0u : 1u);
-                            tc_mma_tf32_ts(d_tmem, ta_hi + kk * 8, db_lo, idesc, 1u);
-                            tc_mma_tf32_ts(d_tmem, ta_lo + kk * 8, db_hi, idesc, 1u);
+                            if (kk == 0) tc_mma_tf32_ts(d_tmem, ta_hi, db_hi, idesc, first ? 0u : 1u);
+                            else tc_mma_tf32_ts_acc(d_tmem, ta_hi + kk * 8, db_hi, idesc);
+                            tc_mma_tf32_ts_acc(d_tmem, ta_hi + kk * 8, db_lo, idesc);
+                            tc_mma_tf32_ts_acc(d_tmem, ta_lo + kk * 8, db_hi, idesc);
                         } else {
-                            const uint64_t da_hi = smem_desc(hi_a + kk * k_step, lbo, sbo, layout);
-                            const uint64_t da_lo = smem_desc(lo_a + kk * k_step, lbo, sbo, layout);
-                            tc_mma_tf32(d_tmem, da_hi, db_hi, idesc, first ? 0u : 1u);
-                            tc_mma_tf32(d_tmem, da_hi, db_lo, idesc, 1u);
-                            tc_mma_tf32(d_tmem, da_lo, db_hi, idesc, 1u);
+                            const uint64_t da_hi = desc_at(hi_a16 + kk * k_step16);
+                            const uint64_t da_lo = desc_at(lo_a16 + kk * k_step16);
+                            if (kk == 0) tc_mma_tf32(d_tmem, da_hi, db_hi, idesc, first ? 0u : 1u);
+                            else tc_mma_tf32_acc(d_tmem, da_hi, db_hi, idesc);
+                            tc_mma_tf32_acc(d_tmem, da_hi, db_lo, idesc);
+                            tc_mma_tf32_acc(d_tmem, da_lo, db_hi, idesc);
                         }
-                        first = false;
                     }
-                    tc_commit(smem_u32(&empty[st]));              // both slots are free once these MMAs retire
-                    tc_commit(smem_u32(&lo_empty[ls]));
+                    first = false;
+                    tc_commit(smem_u32(&empty[st]));              // raw, lo and TMEM-A slots are free once these MMAs retire
+                    if (++st == kNB) { st = 0; st_phase ^= 1u; }
+                    if (++ls == kLoN) ls = 0;
                 }
                 if (ok) tc_commit(smem_u32(&acc_full[b]));
             }
@@ -667,7 +696,10 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
             if (kAnyTma ? !mbar_wait(smem_u32(&raw_full[st]), ph, &abort_flag)
                         : !mbar_wait(smem_u32(&empty[st]), ph ^ 1u, &abort_flag))
                 return false;
-            if (!mbar_wait(smem_u32(&lo_empty[ls]), ((uint32_t)(i / kLoN) & 1u) ^ 1u, &abort_flag)) return false;
+            if (i >= kLoN) {      // the lo slot's previous user: slice i - kLoN
+                const int j = i - kLoN;
+                if (!mbar_wait(smem_u32(&empty[j % kNB]), (uint32_t)(j / kNB) & 1u, &abort_flag)) return false;
+            }
             uint8_t *hi = smem_gen + pair_off(st);               // raw tiles live here and become the hi tiles
             // lo tiles: [A lo][B lo], or the B tile alone when A lives in tensor memory (then `lo` points
             // one A tile below the slot so that the same chunk offsets address the B part)
