@@ -1134,14 +1134,32 @@ static int repack_mode(int B, int C, int Cout, int Kh, int Kw, int sh, int sw, i
     return (flat >= kBK && flat % 4 == 0 && flat < (1L << 30)) ? kRepackFlat : kRepackNone;
 }
 
+// One tensor to repack: out[a][b][p] = in[z][c][(p / Wo) sh W + (p % Wo) sw], zero where p % Wo >= wo_valid, with
+// (a, b) = (z, c), or (c, z) when channel_major.  All tensors of a layer group go into one launch.
+struct RepackJob {
+    const float *in;
+    float *out;
+    int C, HW, W, Wo, P, sh, sw, channel_major, wo_valid;
+};
+struct RepackJobs {
+    RepackJob job[2 * kMaxBatch];
+    int B;
+};
+
 // out[a][b][p] = in[z][c][(p / Wo) sh W + (p % Wo) sw] with (a, b) = (z, c), or (c, z) when channel_major.
 // One warp per group of four rows of P positions (rows of the output are contiguous), lanes along p, eight
 // loads in flight per lane.
 __global__ void __launch_bounds__(256)
-sqgrad_repack(const float *__restrict__ in, float *__restrict__ out, int B, int C, int HW, int W, int Wo, int P,
-              int sh, int sw, int channel_major, int wo_valid)
+sqgrad_repack(const __grid_constant__ RepackJobs jobs)
 {
     constexpr int kRows = 4, kCols = 2;
+    // blockIdx.y picks the tensor; its description is read once (a run-time index into kernel parameters
+    // is expensive, so nothing below touches `jobs` again)
+    const RepackJob job = jobs.job[blockIdx.y];
+    const float *__restrict__ in = job.in;
+    float *__restrict__ out = job.out;
+    const int B = jobs.B, C = job.C, HW = job.HW, W = job.W, Wo = job.Wo, P = job.P, sh = job.sh, sw = job.sw;
+    const int channel_major = job.channel_major, wo_valid = job.wo_valid;
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t rows = (uint32_t)B * (uint32_t)C;
     const bool dense = sh == 1 && sw == 1 && W == Wo && wo_valid == Wo;   // the plane is copied as it is
@@ -1249,15 +1267,17 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
         const size_t dp = round_up(sizeof(float) * (size_t)B * Cout * Ho * W4, 256);
         if (ws_bytes < inner + n_layers * (xp + dp)) return VGC_ERR_WORKSPACE;
         const float *xr[kMaxBatch], *dr[kMaxBatch];
+        RepackJobs jobs = {};
+        jobs.B = B;
         for (int l = 0; l < n_layers; ++l) {
             char *base = static_cast<char *>(ws) + inner + (size_t)l * (xp + dp);
             float *x_p = reinterpret_cast<float *>(base), *d_p = reinterpret_cast<float *>(base + xp);
-            sqgrad_repack<<<blocks_for((size_t)B * C), 256, 0, st>>>(x[l], x_p, B, C, H * W, W, W4, H * W4, 1, 1, 0, W);
-            sqgrad_repack<<<blocks_for((size_t)B * Cout), 256, 0, st>>>(delta[l], d_p, B, Cout, Ho * Wo, Wo, W4, Ho * W4, 1, 1,
-                                                                       0, Wo);
-            count_launch(2);
+            jobs.job[2 * l] = RepackJob{x[l], x_p, C, H * W, W, W4, H * W4, 1, 1, 0, W};
+            jobs.job[2 * l + 1] = RepackJob{delta[l], d_p, Cout, Ho * Wo, Wo, W4, Ho * W4, 1, 1, 0, Wo};
             xr[l] = x_p; dr[l] = d_p;
         }
+        sqgrad_repack<<<dim3(blocks_for((size_t)B * (C > Cout ? C : Cout)), 2 * n_layers), 256, 0, st>>>(jobs);
+        count_launch();
         return conv_group(n_layers, xr, dr, S, B, C, H, W4, Cout, Kh, Kw, 1, 1, ph, 1, Ho, W4, scale, accumulate, ws, inner, st);
     }
     if (mode != kRepackNone) {
@@ -1268,18 +1288,19 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
         const size_t d_bytes = flat ? round_up(sizeof(float) * (size_t)B * Cout * P, 256) : 0;
         if (ws_bytes < inner + n_layers * (x_bytes + d_bytes)) return VGC_ERR_WORKSPACE;
         const float *xr[kMaxBatch], *dr[kMaxBatch];
+        RepackJobs jobs = {};
+        jobs.B = B;
+        int n_jobs = 0;
         for (int l = 0; l < n_layers; ++l) {
             char *base = static_cast<char *>(ws) + inner + (size_t)l * (x_bytes + d_bytes);
             float *x_r = reinterpret_cast<float *>(base), *d_r = reinterpret_cast<float *>(base + x_bytes);
-            sqgrad_repack<<<blocks_for((size_t)B * C), 256, 0, st>>>(x[l], x_r, B, C, H * W, W, Wo, P, sh, sw, flat ? 1 : 0, Wo);
-            count_launch();
-            if (flat) {
-                sqgrad_repack<<<blocks_for((size_t)B * Cout), 256, 0, st>>>(delta[l], d_r, B, Cout, P, Wo, Wo, P, 1, 1, 1, Wo);
-                count_launch();
-            }
+            jobs.job[n_jobs++] = RepackJob{x[l], x_r, C, H * W, W, Wo, P, sh, sw, flat ? 1 : 0, Wo};
+            if (flat) jobs.job[n_jobs++] = RepackJob{delta[l], d_r, Cout, P, Wo, Wo, P, 1, 1, 1, Wo};
             xr[l] = x_r;
             dr[l] = flat ? d_r : delta[l];
         }
+        sqgrad_repack<<<dim3(blocks_for((size_t)B * (flat && Cout > C ? Cout : C)), n_jobs), 256, 0, st>>>(jobs);
+        count_launch();
         if (flat)
             return conv_group(n_layers, xr, dr, S, 1, C, B * P, 1, Cout, 1, 1, 1, 1, 0, 0, B * P, 1, scale, accumulate, ws,
                               inner, st);
