@@ -25,11 +25,12 @@ constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / kWarp;             // 8
 constexpr int kRowsA = 2;                            // float4 vectors per thread per tile
 constexpr int kTileA = kThreads * kRowsA * 4;        // 2048 parameters per tile = one staging segment
-constexpr int kSegPerChunk = 32;                     // phase B: segments per thread block (4 per warp)
+constexpr int kSegPerChunk = 32;                     // phase B: segments per thread block, one per warp
+constexpr int kThreadsB = kSegPerChunk * kWarp;      // 1024
 constexpr int kOffsSmem = 1024;                      // group offsets cached in shared memory
 
 struct CompressLayout {
-    size_t gmax, tile_count, kept_count, chunk_total, stage_idx, stage_val, total;
+    size_t gmax, tile_count, tile_min, kept_count, chunk_total, stage_idx, stage_val, total;
     size_t zero_bytes;       // the per-tensor maxima are cleared per call
     uint32_t tiles_a, chunks;
 };
@@ -43,6 +44,7 @@ static CompressLayout compress_layout(size_t n, int K)
     L.gmax = off;          off = round_up(off + sizeof(uint32_t) * (size_t)K, 256);
     L.zero_bytes = off;
     L.tile_count = off;    off = round_up(off + sizeof(uint32_t) * L.tiles_a, 256);
+    L.tile_min = off;      off = round_up(off + sizeof(int32_t) * L.tiles_a, 256);
     L.kept_count = off;    off = round_up(off + sizeof(uint32_t) * L.tiles_a, 256);
     L.chunk_total = off;   off = round_up(off + sizeof(uint64_t) * L.chunks, 256);
     const size_t slots = (size_t)L.tiles_a * kTileA;
@@ -62,12 +64,13 @@ __global__ void __launch_bounds__(kThreads, 4)
 compress_phase_a(const float *__restrict__ g, const float *__restrict__ s, float *__restrict__ r,
                  float *__restrict__ v, size_t n, const uint32_t *__restrict__ group_offsets, int K,
                  float alpha, float zeta, uint32_t *gmax, uint32_t *__restrict__ tile_count,
-                 uint32_t *__restrict__ stage_idx, uint32_t *__restrict__ stage_val,
+                 int32_t *__restrict__ tile_min, uint32_t *__restrict__ stage_idx, uint32_t *__restrict__ stage_val,
                  uint8_t *__restrict__ mask, uint32_t n_tiles)
 {
     __shared__ uint32_t sm_offs[kOffsSmem];
     __shared__ uint32_t sm_part[2][32];                 // per-(row, warp) counts, double buffered
     __shared__ uint32_t sm_wmax[2][kWarps];
+    __shared__ uint32_t sm_wmin[2][kWarps];             // smallest |value| bit pattern sent by each warp
     __shared__ int sm_grp[2];
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -113,7 +116,7 @@ compress_phase_a(const float *__restrict__ g, const float *__restrict__ s, float
         // ---- Algorithm 1 loop body; every operation rounded on its own (no FMA)
         uint32_t send_bits = 0;          // bit j*4+q
         uint32_t packed = 0;             // per-row counts, 8 bits each
-        uint32_t my_max = 0;
+        uint32_t my_max = 0, my_min = 0x7FFFFFFFu;
 #pragma unroll
         for (int j = 0; j < kRowsA; ++j) {
             const size_t e = base + (size_t)(j * kThreads + tid) * 4;
@@ -135,6 +138,7 @@ compress_phase_a(const float *__restrict__ g, const float *__restrict__ s, float
                 if (send) {
                     row_bits |= 1u << q;
                     my_max = max(my_max, __float_as_uint(r1) & 0x7FFFFFFFu);
+                    my_min = min(my_min, __float_as_uint(r1) & 0x7FFFFFFFu);
                 }
             }
             send_bits |= row_bits << (4 * j);
@@ -167,10 +171,12 @@ compress_phase_a(const float *__restrict__ g, const float *__restrict__ s, float
             if (lane >= d) incl += up;
         }
         const uint32_t warp_max = __reduce_max_sync(0xffffffffu, my_max);
+        const uint32_t warp_min = __reduce_min_sync(0xffffffffu, my_min);
         if (lane == 31) {
 #pragma unroll
             for (int j = 0; j < kRowsA; ++j) sm_part[buf][j * kWarps + warp] = (incl >> (8 * j)) & 0xFFu;
             sm_wmax[buf][warp] = warp_max;
+            sm_wmin[buf][warp] = warp_min;
         }
         __syncthreads();
         const uint32_t part = sm_part[buf][lane];
@@ -206,6 +212,13 @@ compress_phase_a(const float *__restrict__ g, const float *__restrict__ s, float
         }
         if (tid == 0) {
             tile_count[tile] = total;
+            // the rounded exponent (Sec. 4.2) of the smallest value sent from this tile: with it the counting
+            // pass knows without looking at the values whether any of them will be dropped (d > 7).  Tiles that
+            // span several tensors say "unknown".
+            uint32_t lo = 0x7FFFFFFFu;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) lo = min(lo, sm_wmin[buf][w]);
+            tile_min[tile] = grp >= 0 ? (int32_t)((lo + 0x00400000u) >> 23) - 127 : INT32_MIN;
             if (grp >= 0 && total) {
                 uint32_t m = 0;
 #pragma unroll
@@ -275,49 +288,60 @@ __device__ __forceinline__ uint32_t walk_segment(const uint32_t *__restrict__ se
     return kept;
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreadsB)
 compress_count(const uint32_t *__restrict__ group_offsets, int K, const uint32_t *__restrict__ gmax,
-               const uint32_t *__restrict__ tile_count, uint32_t n_tiles_a,
+               const uint32_t *__restrict__ tile_count, const int32_t *__restrict__ tile_min, uint32_t n_tiles_a,
                const uint32_t *__restrict__ stage_idx, const uint32_t *__restrict__ stage_val,
                uint32_t *__restrict__ kept_count, uint64_t *__restrict__ chunk_total,
                int32_t *__restrict__ group_exp)
 {
     __shared__ uint32_t sm_offs[kOffsSmem];
-    __shared__ unsigned long long sm_tot[kWarps];
+    __shared__ unsigned long long sm_tot[kSegPerChunk];
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool offs_in_smem = (K + 1) <= kOffsSmem;
     if (offs_in_smem) {
-        for (int i = tid; i <= K; i += kThreads) sm_offs[i] = group_offsets[i];
+        for (int i = tid; i <= K; i += kThreadsB) sm_offs[i] = group_offsets[i];
         __syncthreads();
     }
     const uint32_t *offs = offs_in_smem ? sm_offs : group_offsets;
     if (blockIdx.x == 0)
-        for (int k = tid; k < K; k += kThreads) {
+        for (int k = tid; k < K; k += kThreadsB) {
             const uint32_t m = gmax[k];
             group_exp[k] = m ? (int32_t)((m >> 23) & 0xFFu) - 127 : VGC_EXP_NONE;
         }
     unsigned long long tot = 0;
-#pragma unroll 1
-    for (int i = 0; i < kSegPerChunk / kWarps; ++i) {
-        const uint32_t seg = blockIdx.x * kSegPerChunk + i * kWarps + warp;
-        if (seg >= n_tiles_a) break;
+    const uint32_t seg = blockIdx.x * kSegPerChunk + warp;              // one warp per segment
+    if (seg < n_tiles_a) {
         const uint32_t count = tile_count[seg];
-        const uint32_t kept = walk_segment<false>(stage_idx + (size_t)seg * kTileA, stage_val + (size_t)seg * kTileA,
-                                                  count, offs, K, gmax, nullptr, 0, 0);
+        uint32_t kept = count;
+        if (count) {
+            // nothing is dropped when even the smallest value sent from the tile is within 7 binades of the
+            // tensor's exponent (d = E_k - e <= 7): then the values need not be read at all
+            const int32_t lowest = tile_min[seg];
+            bool walk = lowest == INT32_MIN;
+            if (!walk) {
+                const int k = group_of(offs, K, seg * (uint32_t)kTileA);
+                const int32_t Ek = (int32_t)((gmax[k] >> 23) & 0xFFu) - 127;
+                walk = lowest < Ek - 7;
+            }
+            if (walk)
+                kept = walk_segment<false>(stage_idx + (size_t)seg * kTileA, stage_val + (size_t)seg * kTileA, count, offs,
+                                           K, gmax, nullptr, 0, 0);
+        }
         if (lane == 0) kept_count[seg] = kept;
-        tot += ((unsigned long long)count << kPassedShift) | kept;
+        tot = ((unsigned long long)count << kPassedShift) | kept;
     }
     if (lane == 0) sm_tot[warp] = tot;
     __syncthreads();
     if (tid == 0) {
         unsigned long long t = 0;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) t += sm_tot[w];
+        for (int w = 0; w < kSegPerChunk; ++w) t += sm_tot[w];
         chunk_total[blockIdx.x] = t;
     }
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreadsB)
 compress_emit(const uint32_t *__restrict__ group_offsets, int K, const uint32_t *__restrict__ gmax,
               const uint32_t *__restrict__ tile_count, uint32_t n_tiles_a,
               const uint32_t *__restrict__ stage_idx, const uint32_t *__restrict__ stage_val,
@@ -326,23 +350,23 @@ compress_emit(const uint32_t *__restrict__ group_offsets, int K, const uint32_t 
               uint32_t *n_dropped, uint32_t *dev_status)
 {
     __shared__ uint32_t sm_offs[kOffsSmem];
-    __shared__ unsigned long long sm_tot[kWarps];
+    __shared__ unsigned long long sm_tot[kSegPerChunk];
     __shared__ uint32_t sm_pos[kSegPerChunk];
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool offs_in_smem = (K + 1) <= kOffsSmem;
     if (offs_in_smem)
-        for (int i = tid; i <= K; i += kThreads) sm_offs[i] = group_offsets[i];
+        for (int i = tid; i <= K; i += kThreadsB) sm_offs[i] = group_offsets[i];
     const uint32_t *offs = offs_in_smem ? sm_offs : group_offsets;
 
     // totals of all chunks before this one
     unsigned long long before = 0;
-    for (uint32_t c = tid; c < blockIdx.x; c += kThreads) before += chunk_total[c];
+    for (uint32_t c = tid; c < blockIdx.x; c += kThreadsB) before += chunk_total[c];
     before = warp_sum_u64(before);
     if (lane == 0) sm_tot[warp] = before;
     __syncthreads();
     before = 0;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) before += sm_tot[w];
+    for (int w = 0; w < kSegPerChunk; ++w) before += sm_tot[w];
     const uint32_t kept_before = (uint32_t)(before & 0xFFFFFFFFull);
 
     if (warp == 0) {                                   // positions of this chunk's 32 segments
@@ -367,14 +391,10 @@ compress_emit(const uint32_t *__restrict__ group_offsets, int K, const uint32_t 
         }
     }
     __syncthreads();
-#pragma unroll 1
-    for (int i = 0; i < kSegPerChunk / kWarps; ++i) {
-        const uint32_t local = i * kWarps + warp;
-        const uint32_t seg = blockIdx.x * kSegPerChunk + local;
-        if (seg >= n_tiles_a) break;
-        walk_segment<true>(stage_idx + (size_t)seg * kTileA, stage_val + (size_t)seg * kTileA, tile_count[seg],
-                           offs, K, gmax, words, sm_pos[local], capacity);
-    }
+    const uint32_t seg = blockIdx.x * kSegPerChunk + warp;              // one warp per segment
+    if (seg < n_tiles_a)
+        walk_segment<true>(stage_idx + (size_t)seg * kTileA, stage_val + (size_t)seg * kTileA, tile_count[seg], offs, K,
+                           gmax, words, sm_pos[warp], capacity);
 }
 
 }  // namespace vgc
@@ -412,6 +432,7 @@ extern "C" vgc_status vgc_compress(const float *g, const float *s, float *r, flo
     char *base = static_cast<char *>(ws);
     uint32_t *gmax = reinterpret_cast<uint32_t *>(base + L.gmax);
     uint32_t *tile_count = reinterpret_cast<uint32_t *>(base + L.tile_count);
+    int32_t *tile_min = reinterpret_cast<int32_t *>(base + L.tile_min);
     uint32_t *kept_count = reinterpret_cast<uint32_t *>(base + L.kept_count);
     uint64_t *chunk_total = reinterpret_cast<uint64_t *>(base + L.chunk_total);
     uint32_t *stage_idx = reinterpret_cast<uint32_t *>(base + L.stage_idx);
@@ -430,13 +451,14 @@ extern "C" vgc_status vgc_compress(const float *g, const float *s, float *r, flo
     const uint32_t grid_a = L.tiles_a < (uint32_t)(sm_count * 8) ? L.tiles_a : (uint32_t)(sm_count * 8);
     if (s)
         compress_phase_a<true><<<grid_a, kThreads, 0, st>>>(g, s, r, v, n, group_offsets, K, alpha, zeta, gmax, tile_count,
-                                                            stage_idx, stage_val, out->mask, L.tiles_a);
+                                                            tile_min, stage_idx, stage_val, out->mask, L.tiles_a);
     else
         compress_phase_a<false><<<grid_a, kThreads, 0, st>>>(g, nullptr, r, v, n, group_offsets, K, alpha, zeta, gmax,
-                                                             tile_count, stage_idx, stage_val, out->mask, L.tiles_a);
-    compress_count<<<L.chunks, kThreads, 0, st>>>(group_offsets, K, gmax, tile_count, L.tiles_a, stage_idx,
-                                                  stage_val, kept_count, chunk_total, out->group_exp);
-    compress_emit<<<L.chunks, kThreads, 0, st>>>(group_offsets, K, gmax, tile_count, L.tiles_a, stage_idx,
+                                                             tile_count, tile_min, stage_idx, stage_val, out->mask,
+                                                             L.tiles_a);
+    compress_count<<<L.chunks, kThreadsB, 0, st>>>(group_offsets, K, gmax, tile_count, tile_min, L.tiles_a, stage_idx,
+                                                   stage_val, kept_count, chunk_total, out->group_exp);
+    compress_emit<<<L.chunks, kThreadsB, 0, st>>>(group_offsets, K, gmax, tile_count, L.tiles_a, stage_idx,
                                                  stage_val, kept_count, chunk_total, out->words, out->capacity,
                                                  out->nnz, out->n_criterion, out->n_dropped, out->dev_status);
     count_launch(3);
@@ -457,7 +479,7 @@ namespace vgc {
 constexpr size_t kStaticMaxParams = VGC_COMPRESS_STATIC_MAX_PARAMS;
 constexpr int kStaticMaxGroups = VGC_COMPRESS_STATIC_MAX_GROUPS;
 // worst-case layout: per-tensor maxima, per-tile counts, chunk totals, 8 bytes of staging per parameter
-constexpr size_t kStaticScratchBytes = 8 * kStaticMaxParams + (kStaticMaxParams / kTileA) * 8 + kStaticMaxGroups * 4 + 64 * 1024;
+constexpr size_t kStaticScratchBytes = 8 * kStaticMaxParams + (kStaticMaxParams / kTileA) * 12 + kStaticMaxGroups * 4 + 64 * 1024;
 static __device__ __align__(256) unsigned char g_compress_scratch[kStaticScratchBytes];
 }  // namespace vgc
 
