@@ -118,7 +118,8 @@ class HotPath:
     """All device buffers of one worker and the launches of one step."""
 
     def __init__(self, name: str, worker: int, n_input_sets: int, n_g_sets: int, device="cuda",
-                 n_params: int = 1 << 25, n_streams: int = 4, algorithm: str = "basic", batch_layers: bool = True):
+                 n_params: int = 1 << 25, n_streams: int = 4, algorithm: str = "basic", batch_layers: bool = True,
+                 exact_conv: bool = False):
         import paper_1802_06058_b200 as vgc
         from paper_1802_06058_b200 import workloads
         self.vgc, self.wl = vgc, workloads
@@ -136,6 +137,8 @@ class HotPath:
         self.compress_only = name in ("vgg16", "flat")
         self.fused = False
         self.hybrid = algorithm == "hybrid"                # Algorithm 2 instead of Algorithm 1
+        self.exact_conv = exact_conv                       # per-example conv statistic (cross terms kept)
+        batch_layers = batch_layers and not exact_conv
         self.tau = 0.0
         dev = device
         B = self.batch
@@ -177,9 +180,10 @@ class HotPath:
             for g in self.groups:
                 spec = self.layers[g[0]]
                 if spec.kind == "conv":
-                    ws_bytes = max(ws_bytes, vgc.vgc_sqgrad_conv_batch_workspace_bytes(
-                        len(g), B, spec.cin, spec.hin, spec.hin, spec.cout, spec.k, spec.k, spec.stride, spec.stride,
-                        spec.pad, spec.pad))
+                    geo = (B, spec.cin, spec.hin, spec.hin, spec.cout, spec.k, spec.k, spec.stride, spec.stride,
+                           spec.pad, spec.pad)
+                    ws_bytes = max(ws_bytes, vgc.vgc_sqgrad_conv_exact_workspace_bytes(*geo) if exact_conv
+                                   else vgc.vgc_sqgrad_conv_batch_workspace_bytes(len(g), *geo))
                 else:
                     ws_bytes = max(ws_bytes, vgc.vgc_sqgrad_linear_workspace_bytes(B, spec.cin, spec.cout))
             self.ws_s = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
@@ -243,7 +247,11 @@ class HotPath:
             lane = gi % self.n_streams
             stream = main if lane == 0 else self.side[lane - 1]
             ws = self.ws_s if lane == 0 else self.ws_side[lane - 1]
-            if spec.kind == "conv":
+            if spec.kind == "conv" and self.exact_conv:
+                vgc.vgc_sqgrad_conv_exact(ins[g[0]][0], ins[g[0]][1], (spec.k, spec.k), (spec.stride, spec.stride),
+                                          (spec.pad, spec.pad), self.scale, Ss[0], accumulate=into_v, ws=ws,
+                                          stream=stream)
+            elif spec.kind == "conv":
                 vgc.vgc_sqgrad_conv_batch([ins[li][0] for li in g], [ins[li][1] for li in g], (spec.k, spec.k),
                                           (spec.stride, spec.stride), (spec.pad, spec.pad), self.scale, Ss,
                                           accumulate=into_v, ws=ws, stream=stream)
@@ -574,6 +582,9 @@ def main():
                          "sections; device-timed only (no end-to-end or CPU leg)")
     ap.add_argument("--no-batch", action="store_true",
                     help="one library call per layer instead of one per group of same-shaped conv layers")
+    ap.add_argument("--exact-conv", action="store_true",
+                    help="conv layers through vgc_sqgrad_conv_exact (per-example statistic, one call per layer); "
+                         "device-timed only")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -596,7 +607,9 @@ def main():
     pk = peaks()
     hp = HotPath(args.workload, worker=rank * 16, n_input_sets=1, n_g_sets=max(4, min(args.steps + args.warmup, 16)),
                  n_params=args.n_params, n_streams=1 if args.per_layer else max(args.streams, 1), algorithm=args.algorithm,
-                 batch_layers=not args.no_batch)
+                 batch_layers=not args.no_batch, exact_conv=args.exact_conv)
+    if args.exact_conv:
+        args.no_e2e = True
     if hp.hybrid:
         args.no_e2e = args.no_cpu_baseline = True
     hp.fused = args.fused
@@ -674,7 +687,7 @@ def main():
             "config": {"workload": args.workload, "n_params": n, "batch": hp.batch, "W": hp.W, "alpha": hp.alpha,
                        "zeta": ZETA, "groups": hp.K, "algorithm": args.algorithm, "tau": hp.tau, "launch": "eager" if args.no_graph else "cuda graph replay",
                        "sqgrad_streams": getattr(hp, "n_streams", 1),
-                       "sqgrad_calls": len(getattr(hp, "groups", [])),
+                       "sqgrad_calls": len(getattr(hp, "groups", [])), "conv_statistic": "per-example" if args.exact_conv else "per-position",
                        "fused_sqgrad_into_v": bool(args.fused),
                        "l2": "inputs larger than L2 (no flush)" if n * 16 > 126e6 else "state fits in L2 (no flush): cache-resident numbers"},
             "gpu_launches": int(launches), "clocks": clocks, "sections": sections, "roofline": roofline,

@@ -103,6 +103,24 @@ vgc_status vgc_sqgrad_conv(const float *x, const float *delta, int B, int C, int
                            float scale, int accumulate, float *S,
                            void *ws, size_t ws_bytes, vgc_stream_t stream);
 
+/* The per-example statistic of a conv layer, exactly as Eq. 2 / Algorithm 1 define it for any layer:
+ *   S[o][c][kh][kw] = scale * sum_z ( sum_{ho,wo} delta[z][o][ho][wo] * x[z][c][ho*sh+kh-ph][wo*sw+kw-pw] )^2
+ * i.e. the square of each example's whole weight gradient, cross terms between output positions included
+ * (vgc_sqgrad_conv drops them by treating every position as a sample; the two agree when Ho*Wo == 1).  Same
+ * tensor-core kernels and the same number of products: the operands are split into TF32 parts without being
+ * squared, an example's positions are reduced first, and the epilogue squares that sum and adds it to a running
+ * sum kept in tensor memory.  Arguments and layouts as for vgc_sqgrad_conv; workspace from
+ * vgc_sqgrad_conv_exact_workspace_bytes.  Accuracy: each example's gradient carries the 3xTF32 product error
+ * (about 2^-22 of the sum of |products|), so the result is within 1e-5 of the same statistic of |x| and |delta|
+ * (relative to the result itself only where an example's positions do not cancel).  Shapes the tensor-core
+ * path cannot take return VGC_ERR_UNSUPPORTED (there is no CUDA-core form of this entry point). */
+size_t vgc_sqgrad_conv_exact_workspace_bytes(int B, int C, int H, int W, int Cout, int Kh, int Kw,
+                                             int stride_h, int stride_w, int pad_h, int pad_w);
+vgc_status vgc_sqgrad_conv_exact(const float *x, const float *delta, int B, int C, int H, int W, int Cout,
+                                 int Kh, int Kw, int stride_h, int stride_w, int pad_h, int pad_w,
+                                 float scale, int accumulate, float *S,
+                                 void *ws, size_t ws_bytes, vgc_stream_t stream);
+
 /* Planning hint (no counterpart in the paper): how many sqgrad calls the caller keeps in flight side by side
  * on different streams, each with its own workspace (default 1).  Alone, a launch is planned so that its
  * blocks fill whole waves over the SMs; next to other launches a partly filled last wave costs nothing, and

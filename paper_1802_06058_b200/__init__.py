@@ -28,6 +28,7 @@ EXPORTS = [
     "vgc_sqgrad_linear_workspace_bytes", "vgc_sqgrad_linear",
     "vgc_sqgrad_conv_workspace_bytes", "vgc_sqgrad_conv",
     "vgc_sqgrad_conv_batch_workspace_bytes", "vgc_sqgrad_conv_batch", "vgc_sqgrad_plan_hint",
+    "vgc_sqgrad_conv_exact_workspace_bytes", "vgc_sqgrad_conv_exact",
     "vgc_compress_workspace_bytes", "vgc_compress", "vgc_compress_static",
     "vgc_decode_accumulate", "vgc_step_host",
     "vgc_compress_hybrid_workspace_bytes", "vgc_compress_hybrid", "vgc_decode_accumulate_hybrid",
@@ -92,6 +93,10 @@ def load_library():
     lib.vgc_sqgrad_conv_batch.argtypes = [i, vp, vp, vp] + [i] * 11 + [f, i, vp, sz, vp]
     lib.vgc_sqgrad_conv_batch.restype = i
     lib.vgc_sqgrad_plan_hint.argtypes = [i]; lib.vgc_sqgrad_plan_hint.restype = None
+    lib.vgc_sqgrad_conv_exact_workspace_bytes.argtypes = [i] * 11
+    lib.vgc_sqgrad_conv_exact_workspace_bytes.restype = sz
+    lib.vgc_sqgrad_conv_exact.argtypes = lib.vgc_sqgrad_conv.argtypes
+    lib.vgc_sqgrad_conv_exact.restype = i
     lib.vgc_compress_workspace_bytes.argtypes = [sz, i]
     lib.vgc_compress_workspace_bytes.restype = sz
     lib.vgc_compress.argtypes = [vp, vp, vp, vp, sz, vp, i, f, f, ctypes.POINTER(_MessageStruct), vp, sz, vp]
@@ -202,6 +207,31 @@ def vgc_sqgrad_conv(x, delta, kernel, stride, padding, scale: float, S, accumula
                                         int(bool(accumulate)), _dev(S, torch.float32, "S"), wp, wb,
                                         _stream(stream))
     _check(st, "vgc_sqgrad_conv")
+    return S
+
+
+def vgc_sqgrad_conv_exact_workspace_bytes(B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw) -> int:
+    return load_library().vgc_sqgrad_conv_exact_workspace_bytes(B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw)
+
+
+def vgc_sqgrad_conv_exact(x, delta, kernel, stride, padding, scale: float, S, accumulate: bool = False,
+                          ws=None, stream=None):
+    """S[Cout,C,Kh,Kw] (+)= scale * sum over examples of the squared per-example weight gradient."""
+    B, C, H, W = x.shape
+    B2, Cout, Ho, Wo = delta.shape
+    Kh, Kw = kernel
+    sh, sw = stride
+    ph, pw = padding
+    if B != B2 or S.numel() != Cout * C * Kh * Kw:
+        raise ValueError("shape mismatch")
+    if Ho != (H + 2 * ph - Kh) // sh + 1 or Wo != (W + 2 * pw - Kw) // sw + 1:
+        raise ValueError("delta spatial shape does not match the convolution geometry")
+    wp, wb = _ws(ws)
+    st = load_library().vgc_sqgrad_conv_exact(_dev(x, torch.float32, "x"), _dev(delta, torch.float32, "delta"),
+                                              B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, float(scale),
+                                              int(bool(accumulate)), _dev(S, torch.float32, "S"), wp, wb,
+                                              _stream(stream))
+    _check(st, "vgc_sqgrad_conv_exact")
     return S
 
 

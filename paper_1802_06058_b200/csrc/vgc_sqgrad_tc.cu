@@ -272,9 +272,13 @@ __host__ __device__ constexpr uint32_t instr_desc(int major, int n)
 // One 16-byte chunk (4 consecutive k of one row) of a K-major 128-byte-swizzled tile.
 __device__ __forceinline__ uint32_t chunk_offset(int row, int kq) { return (uint32_t)row * 128u + (uint32_t)((kq ^ (row & 7)) << 4); }
 
+// kSquare = false: the values themselves are split (per-example form: the products are summed over the positions of
+// an example first and squared afterwards), hi + lo = v with either sign
+template <bool kSquare = true>
 __device__ __forceinline__ void split_store(uint8_t *hi_tile, uint8_t *lo_tile, uint32_t off, float v0, float v1, float v2, float v3)
 {
-    const float q0 = __fmul_rn(v0, v0), q1 = __fmul_rn(v1, v1), q2 = __fmul_rn(v2, v2), q3 = __fmul_rn(v3, v3);
+    const float q0 = kSquare ? __fmul_rn(v0, v0) : v0, q1 = kSquare ? __fmul_rn(v1, v1) : v1;
+    const float q2 = kSquare ? __fmul_rn(v2, v2) : v2, q3 = kSquare ? __fmul_rn(v3, v3) : v3;
     uint4 h, l;
     h.x = to_tf32(q0); h.y = to_tf32(q1); h.z = to_tf32(q2); h.w = to_tf32(q3);
     // lo = q - hi is exact in fp32; the tensor core reads only its upper 19 bits, an error of at most
@@ -427,11 +431,12 @@ struct Gatherer {
         g.init(prm, x, delta, origin + row0, limit);
     }
     __device__ __forceinline__ void load(const Params &prm, int z, int pbase, Regs &r) const { g.load(prm, z, pbase, r.v); }
+    template <bool kSquare>
     __device__ __forceinline__ void store(uint8_t *hi, uint8_t *lo, int row0, int kq, const Regs &r) const
     {
 #pragma unroll
         for (int i = 0; i < kRowsPerThread; ++i)
-            split_store(hi, lo, chunk_offset(row0 + 32 * i, kq), r.v[i][0], r.v[i][1], r.v[i][2], r.v[i][3]);
+            split_store<kSquare>(hi, lo, chunk_offset(row0 + 32 * i, kq), r.v[i][0], r.v[i][1], r.v[i][2], r.v[i][3]);
     }
 };
 template <int kMode>
@@ -443,6 +448,7 @@ struct Gatherer<kMode, true> {
         g.init(prm, x, origin, row0, limit);
     }
     __device__ __forceinline__ void load(const Params &prm, int z, int pbase, Regs &r) const { g.load(prm, z, pbase, r.v); }
+    template <bool kSquare>
     __device__ __forceinline__ void store(uint8_t *hi, uint8_t *lo, int, int kq, const Regs &r) const
     {
 #pragma unroll
@@ -453,14 +459,17 @@ struct Gatherer<kMode, true> {
                 if ((unsigned)row < (unsigned)kBM) {                 // kBM == kBN rows in either tile
                     float o[4];
                     g.tap(r.v, i, kw, o);
-                    split_store(hi, lo, chunk_offset(row, kq), o[0], o[1], o[2], o[3]);
+                    split_store<kSquare>(hi, lo, chunk_offset(row, kq), o[0], o[1], o[2], o[3]);
                 }
             }
     }
 };
 
 // ---- the kernel ------------------------------------------------------------------------------
-template <int kMajor, int kModeA, int kModeB, bool kATmem>
+// kExact: the per-example statistic of a conv layer, S = scale * sum_z (sum_p delta x)^2 -- operands are split without
+// squaring, an accumulator is drained at least at every example's end, the epilogue sums the drains of one example
+// in registers and adds the square of that sum into a third accumulator kept in tensor memory.
+template <int kMajor, int kModeA, int kModeB, bool kATmem, bool kExact = false>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
 {
@@ -471,7 +480,9 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
     constexpr bool kAnyGather = kGatherA || kGatherB;
     constexpr bool kSplit = kATmem && !kAnyGather;                         // A raw tiles in a ring of their own
     constexpr int kNB = kSplit ? kSplitB : kRawSlots;                      // slots of the raw / hi ring
-    constexpr int kLoN = kSplit ? kSplitLo : (kATmem ? kLoSlotsAT : kLoSlots);   // lo slots (and A slots in TMEM)
+    // lo slots (and A slots in TMEM); the per-example form needs 128 TMEM columns for its sum of squares
+    constexpr int kLoN = (kExact && kATmem) ? 2 : kSplit ? kSplitLo : (kATmem ? kLoSlotsAT : kLoSlots);
+    constexpr uint32_t kSqCol = 2 * kBN + (kATmem ? 2 * kTmemColsA : 0);         // where that sum lives
     constexpr uint32_t kLoBytes = kATmem ? kRawBytesB : kRawStageBytes;  // bytes of one lo slot
     // byte offsets of slot s: the [A][B] pair of the raw / hi ring (split form: only its B half exists, the
     // offset points one A tile below it), the lo ring likewise, and the split form's A ring
@@ -507,7 +518,11 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
     const int slice_begin = split * prm.slices_per_split;
     const int slice_end = min(prm.k_slices, slice_begin + prm.slices_per_split);
     const int n_slices = slice_end - slice_begin;                           // >= 1 by construction
-    const int n_chunks = (n_slices + prm.chunk - 1) / prm.chunk;
+    // an accumulator is drained every prm.chunk slices, and (kExact) at the end of every example: the block's
+    // slices are segments of seg_len slices (whole examples -- the split is planned that way), each cut into cps chunks
+    const int seg_len = kExact ? prm.p_slices : n_slices;
+    const int cps = (seg_len + prm.chunk - 1) / prm.chunk;
+    const int n_chunks = (n_slices / seg_len) * cps;
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -617,7 +632,8 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)b * kBN;
-                const int chunk_end = min(n_slices, (c + 1) * prm.chunk);
+                const int seg = c / cps, cq = c - seg * cps;                // segment (example) and chunk inside it
+                const int chunk_end = seg * seg_len + min(seg_len, (cq + 1) * prm.chunk);
                 for (bool first = true; i < chunk_end; ++i) {
                     ok = mbar_wait(smem_u32(&op_full[st]), st_phase, &abort_flag, 0);
                     if (!ok) break;
@@ -724,7 +740,7 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                         const float e[4] = {c4[u].x, c4[u].y, c4[u].z, c4[u].w};
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            const float sq = __fmul_rn(e[j], e[j]);
+                            const float sq = kExact ? e[j] : __fmul_rn(e[j], e[j]);
                             h16[4 * u + j] = to_tf32(sq);
                             l16[4 * u + j] = __float_as_uint(__fsub_rn(sq, __uint_as_float(h16[4 * u + j])));
                         }
@@ -752,12 +768,12 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                             v[u] = *reinterpret_cast<const float4 *>(hi + 16 * (c_begin + (uint32_t)tt + (u0 + u) * kTT));
 #pragma unroll
                         for (int u = 0; u < kBatch; ++u)
-                            split_store(hi, lo, 16 * (c_begin + (uint32_t)tt + (u0 + u) * kTT), v[u].x, v[u].y, v[u].z, v[u].w);
+                            split_store<!kExact>(hi, lo, 16 * (c_begin + (uint32_t)tt + (u0 + u) * kTT), v[u].x, v[u].y, v[u].z, v[u].w);
                     }
                 }
             }
-            if (kGatherA) rows_a.store(hi, lo, row0, kq, ga);
-            if (kGatherB) rows_b.store(hi + kRawBytesA, lo + kRawBytesA, row0, kq, gb);
+            if (kGatherA) rows_a.template store<!kExact>(hi, lo, row0, kq, ga);
+            if (kGatherB) rows_b.template store<!kExact>(hi + kRawBytesA, lo + kRawBytesA, row0, kq, gb);
             if (kATmem) { tc_wait_st(); tc_fence_before(); }      // TMEM stores complete and ordered before the signal
             fence_async_smem();                                   // generic-proxy writes -> tensor core reads
             __syncwarp();
@@ -787,6 +803,15 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         float acc[kBN];
 #pragma unroll
         for (int j = 0; j < kBN; ++j) acc[j] = 0.f;
+        const uint32_t sq_addr = tmem_base + ((q * 32u) << 16) + kSqCol;  // kExact: this warp's rows of the sum of squares
+        if (kExact) {
+            uint32_t zero[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) zero[j] = 0u;
+#pragma unroll
+            for (int j0 = 0; j0 < kBN; j0 += 16) tc_st_32x16(sq_addr + j0, zero);
+            tc_wait_st();
+        }
         bool ok = true;
         for (int c = 0; c < n_chunks && ok; ++c) {
             const int b = c & 1;
@@ -807,6 +832,38 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&acc_empty[b]));
+            if (kExact && (c + 1) % cps == 0) {
+                // end of an example: acc holds its sum over positions; add the squares to the running sum in TMEM
+#pragma unroll
+                for (int j0 = 0; j0 < kBN; j0 += 32) {
+                    if (j0 < n_act) {
+                        uint32_t r[32];
+                        tc_ld_32x32(sq_addr + j0, r);
+                        tc_wait_ld();
+                        uint32_t w0[16], w1[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            w0[j] = __float_as_uint(__fadd_rn(__uint_as_float(r[j]), __fmul_rn(acc[j0 + j], acc[j0 + j])));
+                            w1[j] = __float_as_uint(__fadd_rn(__uint_as_float(r[16 + j]), __fmul_rn(acc[j0 + 16 + j], acc[j0 + 16 + j])));
+                        }
+                        tc_st_32x16(sq_addr + j0, w0);
+                        tc_st_32x16(sq_addr + j0 + 16, w1);
+                    }
+                }
+                tc_wait_st();
+#pragma unroll
+                for (int j = 0; j < kBN; ++j) acc[j] = 0.f;
+            }
+        }
+        if (kExact && ok) {        // the result is the sum of squares
+#pragma unroll
+            for (int j0 = 0; j0 < kBN; j0 += 32) {
+                uint32_t r[32];
+                tc_ld_32x32(sq_addr + j0, r);
+                tc_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) acc[j0 + j] = __uint_as_float(r[j]);
+            }
         }
         if (ok) {
             const int r_local = (int)(q * 32u + lane);
@@ -985,9 +1042,11 @@ struct Plan {
 // how many sqgrad launches the caller keeps in flight side by side (vgc_sqgrad_plan_hint)
 static int g_concurrent_launches = 1;
 
-static Plan make_plan(int M, int N, int k_slices, int n_layers = 1)
+// `unit`: slices that must stay in one block (the per-example form splits the reduction between examples only)
+static Plan make_plan(int M, int N, int k_slices_total, int n_layers = 1, int unit = 1)
 {
     Plan p;
+    const int k_slices = k_slices_total / unit;                          // planned in units
     p.tiles_x = (N + kBN - 1) / kBN;
     p.tiles_y = (M + kBM - 1) / kBM;
     const long tiles = (long)p.tiles_x * p.tiles_y * n_layers;          // output tiles of the whole launch
@@ -1013,13 +1072,14 @@ static Plan make_plan(int M, int N, int k_slices, int n_layers = 1)
             if ((k_slices + per - 1) / per != sp) continue;              // splits that would get no slices
             if (sp > 1 && tiles * sp > 6 * target) break;                 // keeps the split-K scratch L2-sized
             const long waves = (tiles * sp + target - 1) / target;
-            const long cost = waves * (per + 8 + (sp > 1 ? 5 : 0)) + (sp > 1 ? 6 : 0);
+            const long cost = waves * (per * unit + 8 + (sp > 1 ? 5 : 0)) + (sp > 1 ? 6 : 0);
             if (best < 0 || cost < best) { best = cost; want = sp; }
         }
     }
-    p.k_slices = k_slices;
-    p.slices_per_split = (int)((k_slices + want - 1) / want);
-    p.splits = (k_slices + p.slices_per_split - 1) / p.slices_per_split;
+    p.k_slices = k_slices_total;
+    const int per = (int)((k_slices + want - 1) / want);
+    p.slices_per_split = per * unit;
+    p.splits = (k_slices + per - 1) / per;
     return p;
 }
 
@@ -1042,26 +1102,26 @@ bool tc_conv_supported(int B, int C, int H, int W, int Cout, int Kh, int Kw, int
            (long)B * ((P + kBK - 1) / kBK) < (1L << 30);
 }
 
-static size_t tc_workspace_bytes(int M, int N, int k_slices, int n_layers = 1)
+static size_t tc_workspace_bytes(int M, int N, int k_slices, int n_layers = 1, int unit = 1)
 {
-    const Plan p = make_plan(M, N, k_slices, n_layers);
+    const Plan p = make_plan(M, N, k_slices, n_layers, unit);
     return 256 + (p.splits > 1 ? (size_t)n_layers * p.splits * p.tiles_x * p.tiles_y * kBM * kBN * sizeof(float) : 0);
 }
 
 typedef void (*KernelFn)(const Batch, const Params);
 
 static vgc_status tc_launch(KernelFn kernel, const Batch &bt, int n_layers, Params prm, int M, int N,
-                            int k_slices, void *ws, size_t ws_bytes, cudaStream_t st)
+                            int k_slices, void *ws, size_t ws_bytes, cudaStream_t st, int unit = 1)
 {
-    const Plan plan = make_plan(M, N, k_slices, n_layers);
-    if (ws_bytes < tc_workspace_bytes(M, N, k_slices, n_layers)) return VGC_ERR_WORKSPACE;
-    static KernelFn configured[16];
+    const Plan plan = make_plan(M, N, k_slices, n_layers, unit);
+    if (ws_bytes < tc_workspace_bytes(M, N, k_slices, n_layers, unit)) return VGC_ERR_WORKSPACE;
+    static KernelFn configured[32];
     static int n_configured = 0;
     bool seen = false;
     for (int i = 0; i < n_configured; ++i) seen = seen || configured[i] == kernel;
     if (!seen) {
         VGC_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-        if (n_configured < 16) configured[n_configured++] = kernel;
+        if (n_configured < 32) configured[n_configured++] = kernel;
     }
     prm.M = M; prm.N = N; prm.k_slices = k_slices; prm.slices_per_split = plan.slices_per_split;
     prm.splits = plan.splits;
@@ -1102,6 +1162,14 @@ vgc_status tc_sqgrad_linear(const float *x, const float *delta, int B, int in, i
     return tc_launch(sqgrad_tc<kMajorMN, kTma, kTma, false>, bt, 1, prm, out, in, (B + kBK - 1) / kBK, ws, ws_bytes, st);
 }
 
+// Set for the duration of a per-example (exact) call: planning, repacking and kernel choice consult it.
+static thread_local bool t_exact = false;
+struct ExactScope {
+    bool saved;
+    explicit ExactScope(bool on) : saved(t_exact) { t_exact = on; }
+    ~ExactScope() { t_exact = saved; }
+};
+
 // Cout <= 64: the im2col rows take the 128-row A tile and the errors the narrow B tile
 static bool conv_swapped(int Cout, int n_im2col) { return Cout <= 64 && n_im2col > Cout; }
 
@@ -1131,6 +1199,7 @@ static int repack_mode(int B, int C, int Cout, int Kh, int Kw, int sh, int sw, i
     const bool planes_ok = P >= kBK && P % 4 == 0;
     if (planes_ok) return (sh > 1 || sw > 1) ? kRepackPlanes : kRepackNone;
     const long flat = (long)B * P;
+    if (t_exact) return kRepackNone;                 // the flat form merges the examples' positions
     return (flat >= kBK && flat % 4 == 0 && flat < (1L << 30)) ? kRepackFlat : kRepackNone;
 }
 
@@ -1206,9 +1275,10 @@ sqgrad_repack(const __grid_constant__ RepackJobs jobs)
 
 static size_t conv_workspace_plain(int n_layers, int B, int C, int Kh, int Kw, int P, int Cout)
 {
-    const int n_im2col = C * Kh * Kw, k_slices = B * ((P + kBK - 1) / kBK);
-    return conv_swapped(Cout, n_im2col) ? tc_workspace_bytes(n_im2col, Cout, k_slices, n_layers)
-                                        : tc_workspace_bytes(Cout, n_im2col, k_slices, n_layers);
+    const int p_slices = (P + kBK - 1) / kBK, n_im2col = C * Kh * Kw, k_slices = B * p_slices;
+    const int unit = t_exact ? p_slices : 1;
+    return conv_swapped(Cout, n_im2col) ? tc_workspace_bytes(n_im2col, Cout, k_slices, n_layers, unit)
+                                        : tc_workspace_bytes(Cout, n_im2col, k_slices, n_layers, unit);
 }
 
 // Workspace of one launch over n_layers layers of this geometry (n_layers <= kMaxBatch).
@@ -1239,8 +1309,9 @@ static size_t conv_workspace_group(int n_layers, int B, int C, int Kh, int Kw, i
 }
 
 size_t tc_conv_workspace_bytes(int n_layers, int B, int C, int Kh, int Kw, int sh, int sw, int ph, int pw, int P,
-                               int Cout, int Wo_)
+                               int Cout, int Wo_, bool exact)
 {
+    ExactScope scope(exact);
     // more layers than one launch takes are processed group after group in the same workspace
     const int first = n_layers < kMaxBatch ? n_layers : kMaxBatch;
     size_t need = conv_workspace_group(first, B, C, Kh, Kw, sh, sw, ph, pw, P, Cout, Wo_);
@@ -1351,38 +1422,35 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
     const int taps = (!(taps_env && atoi(taps_env) == 0) && i == kGatherIm2col && e == kTma && Kw == 3 && sw == 1 &&
                       sh == 1 && pw == 1 && Wo == W && W % 2 == 0 && a_tmem)
                          ? (W % 4 == 0 ? 4 : 2) : 0;
+    const bool ex = t_exact;
+    const int unit = ex ? p_slices : 1;
     KernelFn fn = nullptr;
-    if (taps && !swapped) {
-        prm.ld_m = n_im2col; prm.ld_n = 1;
-        fn = taps == 4 ? sqgrad_tc<kMajorK, kTma, kGatherTaps4, true> : sqgrad_tc<kMajorK, kTma, kGatherTaps2, true>;
-        return tc_launch(fn, bt, n_layers, prm, Cout, n_im2col, k_slices, ws, ws_bytes, st);
-    }
-    if (taps && swapped) {
-        prm.ld_m = 1; prm.ld_n = n_im2col;
-        fn = taps == 4 ? sqgrad_tc<kMajorK, kGatherTaps4, kTma, false> : sqgrad_tc<kMajorK, kGatherTaps2, kTma, false>;
-        return tc_launch(fn, bt, n_layers, prm, n_im2col, Cout, k_slices, ws, ws_bytes, st);
-    }
+#define VGC_TC_FN(A, B_, AT) (ex ? (KernelFn)sqgrad_tc<kMajorK, A, B_, AT, true> : (KernelFn)sqgrad_tc<kMajorK, A, B_, AT, false>)
     if (!swapped) {     // S[o][idx]: m = o, n = idx
         prm.ld_m = n_im2col; prm.ld_n = 1;
-        if (e == kTma && i == kTma) fn = a_tmem ? sqgrad_tc<kMajorK, kTma, kTma, true> : sqgrad_tc<kMajorK, kTma, kTma, false>;
-        else if (e == kTma) fn = a_tmem ? sqgrad_tc<kMajorK, kTma, kGatherIm2col, true> : sqgrad_tc<kMajorK, kTma, kGatherIm2col, false>;
-        else if (i == kTma) fn = sqgrad_tc<kMajorK, kGatherErr, kTma, false>;
-        else fn = sqgrad_tc<kMajorK, kGatherErr, kGatherIm2col, false>;
-        return tc_launch(fn, bt, n_layers, prm, Cout, n_im2col, k_slices, ws, ws_bytes, st);
+        if (taps) fn = taps == 4 ? VGC_TC_FN(kTma, kGatherTaps4, true) : VGC_TC_FN(kTma, kGatherTaps2, true);
+        else if (e == kTma && i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kTma, true) : sqgrad_tc<kMajorK, kTma, kTma, false>;
+        else if (e == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kGatherIm2col, true) : sqgrad_tc<kMajorK, kTma, kGatherIm2col, false>;
+        else if (i == kTma) fn = VGC_TC_FN(kGatherErr, kTma, false);
+        else fn = VGC_TC_FN(kGatherErr, kGatherIm2col, false);
+        return tc_launch(fn, bt, n_layers, prm, Cout, n_im2col, k_slices, ws, ws_bytes, st, unit);
     }
     prm.ld_m = 1; prm.ld_n = n_im2col;   // m = idx, n = o
-    if (e == kTma && i == kTma) fn = a_tmem ? sqgrad_tc<kMajorK, kTma, kTma, true> : sqgrad_tc<kMajorK, kTma, kTma, false>;
-    else if (i == kTma) fn = a_tmem ? sqgrad_tc<kMajorK, kTma, kGatherErr, true> : sqgrad_tc<kMajorK, kTma, kGatherErr, false>;
-    else if (e == kTma) fn = sqgrad_tc<kMajorK, kGatherIm2col, kTma, false>;
-    else fn = sqgrad_tc<kMajorK, kGatherIm2col, kGatherErr, false>;
-    return tc_launch(fn, bt, n_layers, prm, n_im2col, Cout, k_slices, ws, ws_bytes, st);
+    if (taps) fn = taps == 4 ? VGC_TC_FN(kGatherTaps4, kTma, false) : VGC_TC_FN(kGatherTaps2, kTma, false);
+    else if (e == kTma && i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kTma, true) : sqgrad_tc<kMajorK, kTma, kTma, false>;
+    else if (i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kGatherErr, true) : sqgrad_tc<kMajorK, kTma, kGatherErr, false>;
+    else if (e == kTma) fn = VGC_TC_FN(kGatherIm2col, kTma, false);
+    else fn = VGC_TC_FN(kGatherIm2col, kGatherErr, false);
+#undef VGC_TC_FN
+    return tc_launch(fn, bt, n_layers, prm, n_im2col, Cout, k_slices, ws, ws_bytes, st, unit);
 }
 
 // n_layers layers of one geometry; x, delta, S are host arrays of device pointers
 vgc_status tc_sqgrad_conv(int n_layers, const float *const *x, const float *const *delta, float *const *S, int B, int C,
                           int H, int W, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw, int Ho, int Wo,
-                          float scale, int accumulate, void *ws, size_t ws_bytes, cudaStream_t st)
+                          float scale, int accumulate, void *ws, size_t ws_bytes, cudaStream_t st, bool exact)
 {
+    ExactScope scope(exact);
     for (int l0 = 0; l0 < n_layers; l0 += kMaxBatch) {
         const int nl = n_layers - l0 < kMaxBatch ? n_layers - l0 : kMaxBatch;
         const vgc_status rc = conv_group(nl, x + l0, delta + l0, S + l0, B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, Ho, Wo,
