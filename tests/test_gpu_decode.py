@@ -132,3 +132,23 @@ def test_decode_sum_of_no_messages_is_zero():
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     vgc.vgc_decode_sum([], vgc.offsets_tensor(np.array([0, n], np.uint32)), 1.0, u, status)
     assert float(u.abs().max().item()) == 0.0
+
+
+def test_exchange_and_decode_single_rank():
+    """Without a process group the exchange is the identity: the worker decodes its own message."""
+    from gpu_harness import GpuCompressor, OracleCompressor, noise_gs
+    from paper_1802_06058_b200 import exchange
+    n = 150001
+    offs = random_offsets(np.random.default_rng(3), n, 6)
+    gpu, cpu = GpuCompressor(n, offs), OracleCompressor(n, offs)
+    g, s = noise_gs(n, 4, seed=77)
+    gpu.out.counters.zero_()
+    vgc.vgc_compress(g, s, gpu.r, gpu.v, gpu.offs_dev, 2.0, 0.999, gpu.out, gpu.ws)
+    m = cpu.step(g.cpu().numpy(), s.cpu().numpy(), 2.0, 0.999)
+    u = torch.full((n,), float("nan"), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    exchange.exchange_and_decode(gpu.out, gpu.offs_dev, u, status)
+    want = np.zeros(n, F32)
+    oracle.decode_accumulate([(m.words, m.group_exp)], offs, 1.0, want)
+    assert int(status.item()) == 0
+    assert np.array_equal(u.cpu().numpy(), want)

@@ -67,3 +67,39 @@ def test_reference_arm_under_torchrun_prints_one_line_from_rank_0():
     rec = json.loads(lines[0])
     assert rec["impl"] == "reference" and rec["cpu_baseline"]["kind"] == "oracle"
     assert rec["e2e"]["h2d_bytes_per_step"] == 0 and rec["value"] > 0
+
+
+EXCHANGE_WORKER = r"""
+import os, sys
+sys.path.insert(0, {root!r})
+import numpy as np, torch, torch.distributed as dist
+from paper_1802_06058_b200 import exchange
+dist.init_process_group("gloo")
+rank, W = dist.get_rank(), dist.get_world_size()
+# messages of different lengths (rank 0: 5 words, rank 1: 11 words), K = 3 per-tensor exponents
+def message(r):
+    n = 5 + 6 * r
+    words = (torch.arange(n, dtype=torch.int32) * 7 + r) * 16 + r
+    return words, torch.tensor([n], dtype=torch.int32), torch.tensor([r, -r, 3 * r], dtype=torch.int32)
+words, nnz, gexp = message(rank)
+padded = torch.cat([words, torch.full((9,), -1, dtype=torch.int32)])        # capacity larger than the message
+for pad_to in (None, 16):
+    all_words, all_nnz, all_exp = exchange.allgather_messages(padded, nnz, gexp, pad_to=pad_to)
+    assert all_words.shape == (W, 11 if pad_to is None else 16), all_words.shape
+    for r in range(W):
+        w, c, e = message(r)
+        assert int(all_nnz[r]) == int(c[0])
+        assert torch.equal(all_words[r, :int(c[0])], w)
+        assert torch.equal(all_exp[r], e)
+dist.barrier()
+dist.destroy_process_group()
+sys.stdout.write("rank%dok\n" % rank); sys.stdout.flush()
+"""
+
+
+def test_allgather_of_messages_world_size_2(tmp_path):
+    script = tmp_path / "exchange_worker.py"
+    script.write_text(EXCHANGE_WORKER.format(root=ROOT))
+    res = _torchrun([str(script)])
+    assert res.returncode == 0, res.stdout + res.stderr
+    assert "rank0ok" in res.stdout and "rank1ok" in res.stdout
