@@ -183,7 +183,8 @@ class HotPath:
                     geo = (B, spec.cin, spec.hin, spec.hin, spec.cout, spec.k, spec.k, spec.stride, spec.stride,
                            spec.pad, spec.pad)
                     ws_bytes = max(ws_bytes, vgc.vgc_sqgrad_conv_exact_workspace_bytes(*geo) if exact_conv
-                                   else vgc.vgc_sqgrad_conv_batch_workspace_bytes(len(g), *geo))
+                                   else vgc.vgc_sqgrad_conv_batch_workspace_bytes(len(g), *geo),
+                                   vgc.vgc_sqgrad_conv_workspace_bytes(*geo))      # the end-to-end leg calls layer by layer
                 else:
                     ws_bytes = max(ws_bytes, vgc.vgc_sqgrad_linear_workspace_bytes(B, spec.cin, spec.cout))
             self.ws_s = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
