@@ -451,17 +451,36 @@ struct Gatherer<kMode, true> {
     template <bool kSquare>
     __device__ __forceinline__ void store(uint8_t *hi, uint8_t *lo, int, int kq, const Regs &r) const
     {
+        constexpr int kLoaded = kMode == kGatherTaps4 ? 6 : 8;      // segment elements held per triple
 #pragma unroll
-        for (int i = 0; i < 2; ++i)
+        for (int i = 0; i < 2; ++i) {
+            if (g.row_local[i] >= kBM || g.row_local[i] <= -3) continue;   // no row of this triple in the tile
+            // square and split every loaded element once; the three taps are shifted views of the same parts
+            uint32_t h[8], l[8];
+#pragma unroll
+            for (int e = 0; e < kLoaded; ++e) {
+                const float q = kSquare ? __fmul_rn(r.v[i][e], r.v[i][e]) : r.v[i][e];
+                h[e] = to_tf32(q);
+                l[e] = __float_as_uint(__fsub_rn(q, __uint_as_float(h[e])));
+            }
 #pragma unroll
             for (int kw = 0; kw < 3; ++kw) {
                 const int row = g.row_local[i] + kw;
                 if ((unsigned)row < (unsigned)kBM) {                 // kBM == kBN rows in either tile
-                    float o[4];
-                    g.tap(r.v, i, kw, o);
-                    split_store<kSquare>(hi, lo, chunk_offset(row, kq), o[0], o[1], o[2], o[3]);
+                    const uint32_t off = chunk_offset(row, kq);
+                    uint4 hv, lv;
+                    if (kMode == kGatherTaps4) {
+                        hv = make_uint4(h[kw], h[kw + 1], h[kw + 2], h[kw + 3]);
+                        lv = make_uint4(l[kw], l[kw + 1], l[kw + 2], l[kw + 3]);
+                    } else {
+                        hv = make_uint4(h[kw], h[kw + 1], h[4 + kw], h[4 + kw + 1]);
+                        lv = make_uint4(l[kw], l[kw + 1], l[4 + kw], l[4 + kw + 1]);
+                    }
+                    *reinterpret_cast<uint4 *>(hi + off) = hv;
+                    *reinterpret_cast<uint4 *>(lo + off) = lv;
                 }
             }
+        }
     }
 };
 
