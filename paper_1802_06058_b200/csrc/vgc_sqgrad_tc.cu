@@ -1406,7 +1406,14 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
     const bool a_tmem = !(getenv("VGC_TC_ATMEM") && atoi(getenv("VGC_TC_ATMEM")) == 0);
     const int p_slices = (P + kBK - 1) / kBK;
     const int k_slices = B * p_slices;
-    const bool swapped = conv_swapped(Cout, n_im2col);
+    // three taps at a time: Kw = 3, stride 1 along w with pad 1 (then Wo == W), output width even, errors by TMA
+    const char *taps_env = getenv("VGC_TC_TAPS");
+    const int taps = (!(taps_env && atoi(taps_env) == 0) && !in_tma && err_tma && Kw == 3 && sw == 1 && sh == 1 &&
+                      pw == 1 && Wo == W && W % 2 == 0 && a_tmem)
+                         ? (W % 4 == 0 ? 4 : 2) : 0;
+    // with few output channels the roles are swapped -- except in the three-tap form, where keeping the errors as
+    // the A operand (in tensor memory, half of its rows unused) measures faster than both operands in shared memory
+    const bool swapped = conv_swapped(Cout, n_im2col) && !taps;
     const int rows_err = swapped ? kBN : kBM, rows_in = swapped ? kBM : kBN;     // tile heights
     Batch bt = {};
     uint32_t tx_err = 0, tx_in = 0;
@@ -1436,11 +1443,6 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
     prm.chw = C * H * W;
     prm.wo_magic = (unsigned)(0x100000000ull / (unsigned)Wo) + 1u;
     const int e = err_tma ? kTma : kGatherErr, i = in_tma ? kTma : kGatherIm2col;
-    // three taps at a time: Kw = 3, stride 1 along w with pad 1 (then Wo == W), output width even, errors by TMA
-    const char *taps_env = getenv("VGC_TC_TAPS");
-    const int taps = (!(taps_env && atoi(taps_env) == 0) && i == kGatherIm2col && e == kTma && Kw == 3 && sw == 1 &&
-                      sh == 1 && pw == 1 && Wo == W && W % 2 == 0 && a_tmem)
-                         ? (W % 4 == 0 ? 4 : 2) : 0;
     const bool ex = t_exact;
     const int unit = ex ? p_slices : 1;
     KernelFn fn = nullptr;
@@ -1455,8 +1457,7 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
         return tc_launch(fn, bt, n_layers, prm, Cout, n_im2col, k_slices, ws, ws_bytes, st, unit);
     }
     prm.ld_m = 1; prm.ld_n = n_im2col;   // m = idx, n = o
-    if (taps) fn = taps == 4 ? VGC_TC_FN(kGatherTaps4, kTma, false) : VGC_TC_FN(kGatherTaps2, kTma, false);
-    else if (e == kTma && i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kTma, true) : sqgrad_tc<kMajorK, kTma, kTma, false>;
+    if (e == kTma && i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kTma, true) : sqgrad_tc<kMajorK, kTma, kTma, false>;
     else if (i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kGatherErr, true) : sqgrad_tc<kMajorK, kTma, kGatherErr, false>;
     else if (e == kTma) fn = VGC_TC_FN(kGatherIm2col, kTma, false);
     else fn = VGC_TC_FN(kGatherIm2col, kGatherErr, false);
