@@ -356,10 +356,12 @@ struct GatherRows {
 // the input row segment once -- one aligned vector and its two neighbours -- and feeds all three rows from
 // it.  A thread owns the triples first_triple + grp + 32*i (i = 0, 1) of the tile's rows; triples that
 // straddle the tile's first or last row are handled by the row test at store time.
-template <int kSpan>          // output positions covered by one aligned vector load: 4 or 2
+// kTriples = 2: 256 threads share a slice (triples grp + 32 i); kTriples = 3: 128 threads do (grp + 16 i).
+template <int kSpan, int kTriples>      // kSpan: output positions covered by one aligned vector load, 4 or 2
 struct GatherTaps {
-    int base[2], dh[2], row_local[2];
-    bool ok[2];
+    static constexpr int kStride = kTriples == 2 ? 32 : 16;
+    int base[kTriples], dh[kTriples], row_local[kTriples];
+    bool ok[kTriples];
     const float *src;
 
     __device__ __forceinline__ void init(const Params &prm, const float *x, int tile_origin, int grp, int limit)
@@ -367,8 +369,8 @@ struct GatherTaps {
         src = x;
         const int first_triple = tile_origin / 3;
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            const int T = first_triple + grp + 32 * i;               // triple = (c, kh)
+        for (int i = 0; i < kTriples; ++i) {
+            const int T = first_triple + grp + kStride * i;          // triple = (c, kh)
             ok[i] = 3 * T < limit;
             const int tt = ok[i] ? T : 0;
             const int c = tt / prm.Kh, kh = tt - c * prm.Kh;
@@ -379,7 +381,7 @@ struct GatherTaps {
     }
     // v[i][0..7]: kSpan = 4: {left, m0, m1, m2, m3, right, -, -} for positions pbase..pbase+3;
     //             kSpan = 2: {left, m0, m1, right} for pbase, pbase+1 and the same for pbase+2, pbase+3
-    __device__ __forceinline__ void load(const Params &prm, int z, int pbase, float (&v)[2][8]) const
+    __device__ __forceinline__ void load(const Params &prm, int z, int pbase, float (&v)[kTriples][8]) const
     {
         const float *xz = src + (size_t)z * prm.chw;
 #pragma unroll
@@ -389,7 +391,7 @@ struct GatherTaps {
             const bool pv = p < prm.P;
             const float *xp = xz + (ho * prm.W + wo);
 #pragma unroll
-            for (int i = 0; i < 2; ++i) {
+            for (int i = 0; i < kTriples; ++i) {
                 const bool in = pv && ok[i] && (unsigned)(ho + dh[i]) < (unsigned)prm.H;
                 const float *q = xp + base[i];
                 float *o = &v[i][s * 4];
@@ -408,7 +410,7 @@ struct GatherTaps {
         }
     }
     // the four k of tap kw of triple i
-    __device__ __forceinline__ static void tap(const float (&v)[2][8], int i, int kw, float (&out)[4])
+    __device__ __forceinline__ static void tap(const float (&v)[kTriples][8], int i, int kw, float (&out)[4])
     {
         if (kSpan == 4) {
             out[0] = v[i][kw]; out[1] = v[i][kw + 1]; out[2] = v[i][kw + 2]; out[3] = v[i][kw + 3];
@@ -422,7 +424,8 @@ template <int kMode> struct IsTaps { static constexpr bool value = kMode == kGat
 
 // One interface over both gather forms: the registers of one slice, how they are loaded and where their
 // squared, split values go in a K-major swizzled tile.  row0 = t >> 3 and kq = t & 7 of transform thread t.
-template <int kMode, bool kTaps = IsTaps<kMode>::value>
+// kHalf: the slice is shared by 128 threads instead of 256 (two transform groups on alternate slices)
+template <int kMode, bool kHalf = false, bool kTaps = IsTaps<kMode>::value>
 struct Gatherer {
     struct Regs { float v[kRowsPerThread][4]; };
     GatherRows<kMode> g;
@@ -439,10 +442,11 @@ struct Gatherer {
             split_store<kSquare>(hi, lo, chunk_offset(row0 + 32 * i, kq), r.v[i][0], r.v[i][1], r.v[i][2], r.v[i][3]);
     }
 };
-template <int kMode>
-struct Gatherer<kMode, true> {
-    struct Regs { float v[2][8]; };
-    GatherTaps<kMode == kGatherTaps4 ? 4 : 2> g;
+template <int kMode, bool kHalf>
+struct Gatherer<kMode, kHalf, true> {
+    static constexpr int kTriples = kHalf ? 3 : 2;
+    struct Regs { float v[kTriples][8]; };
+    GatherTaps<kMode == kGatherTaps4 ? 4 : 2, kTriples> g;
     __device__ __forceinline__ void init(const Params &prm, const float *x, const float *, int origin, int row0, int limit)
     {
         g.init(prm, x, origin, row0, limit);
@@ -453,7 +457,7 @@ struct Gatherer<kMode, true> {
     {
         constexpr int kLoaded = kMode == kGatherTaps4 ? 6 : 8;      // segment elements held per triple
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < kTriples; ++i) {
             if (g.row_local[i] >= kBM || g.row_local[i] <= -3) continue;   // no row of this triple in the tile
             // square and split every loaded element once; the three taps are shifted views of the same parts
             uint32_t h[8], l[8];
@@ -498,6 +502,8 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
     constexpr bool kAnyTma = !kGatherA || !kGatherB;
     constexpr bool kAnyGather = kGatherA || kGatherB;
     constexpr bool kSplit = kATmem && !kAnyGather;                         // A raw tiles in a ring of their own
+    // the transform warps work as two groups of four on alternate slices (else all eight on every slice)
+    constexpr bool kTwoGroups = !kAnyGather || (kModeB == kGatherTaps4 && kModeA == kTma);
     constexpr int kNB = kSplit ? kSplitB : kRawSlots;                      // slots of the raw / hi ring
     // lo slots (and A slots in TMEM); the per-example form needs 128 TMEM columns for its sum of squares
     constexpr int kLoN = (kExact && kATmem) ? 2 : kSplit ? kSplitLo : (kATmem ? kLoSlotsAT : kLoSlots);
@@ -547,7 +553,7 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         abort_flag = 0;
         for (int i = 0; i < kNB; ++i) {
             mbar_init(smem_u32(&raw_full[i]), 1);
-            mbar_init(smem_u32(&op_full[i]), kAnyGather ? kTransformWarps : kTransformWarps / 2);
+            mbar_init(smem_u32(&op_full[i]), kTwoGroups ? kTransformWarps / 2 : kTransformWarps);
             mbar_init(smem_u32(&empty[i]), 1);
         }
         if (kSplit)
@@ -695,15 +701,16 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         const int t = (int)threadIdx.x - 64;                               // 0..255
         // With nothing to gather the eight warps work as two groups of four that take alternate slices: the
         // waits, fences and tensor-memory stores of one slice then overlap the arithmetic of the next one.
-        constexpr bool kTwoGroups = !kAnyGather;
+        // The same split is used when the B tile is gathered three taps at a time (widths that are multiples of 4;
+        // the 2 + 2 form measures slower that way) next to a TMA-fed A tile.
         constexpr int kTT = kTwoGroups ? kTransformThreads / 2 : kTransformThreads;   // threads sharing a slice
         const int group = kTwoGroups ? (t >> 7) : 0;
         const int tt = kTwoGroups ? (t & 127) : t;
-        const int kq = t & 7, row0 = t >> 3;                               // gathered chunks: rows row0 + 32*i, k = 4*kq..4*kq+3
-        Gatherer<kModeA> rows_a;
-        Gatherer<kModeB> rows_b;
-        typedef typename Gatherer<kModeA>::Regs RegsA;
-        typedef typename Gatherer<kModeB>::Regs RegsB;
+        const int kq = tt & 7, row0 = tt >> 3;                             // gathered chunks: rows row0 + 32*i, k = 4*kq..4*kq+3
+        Gatherer<kModeA, kTwoGroups> rows_a;
+        Gatherer<kModeB, kTwoGroups> rows_b;
+        typedef typename Gatherer<kModeA, kTwoGroups>::Regs RegsA;
+        typedef typename Gatherer<kModeB, kTwoGroups>::Regs RegsB;
         rows_a.init(prm, bt.x[layer], bt.delta[layer], m0, row0, prm.M);
         rows_b.init(prm, bt.x[layer], bt.delta[layer], n0, row0, prm.N);
         // where the current slice sits: example z, 32-wide block pblk of that example's output positions
@@ -803,11 +810,23 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         // two register sets in turn: the loads of slice i+1 are in flight while slice i is transformed
         RegsA a0, a1;
         RegsB b0, b1;
-        if (kAnyGather) gather(a0, b0);
-        if (kTwoGroups) {
+        if (kTwoGroups && kAnyGather) {
+            // this group's slices: group, group + 2, ...; the loads of its next slice fly while one is transformed
+            for (int sk = 0; sk < group; ++sk) advance();
+            if (group < n_slices) gather(a0, b0);
+            for (int i = group; i < n_slices; i += 4) {
+                if (i + 2 < n_slices) { advance(); advance(); gather(a1, b1); }
+                if (!process(i, a0, b0)) break;
+                if (i + 2 < n_slices) {
+                    if (i + 4 < n_slices) { advance(); advance(); gather(a0, b0); }
+                    if (!process(i + 2, a1, b1)) break;
+                }
+            }
+        } else if (kTwoGroups) {
             for (int i = group; i < n_slices; i += 2)
                 if (!process(i, a0, b0)) break;
-        } else
+        } else {
+        if (kAnyGather) gather(a0, b0);
         for (int i = 0; i < n_slices; i += 2) {
             if (kAnyGather && i + 1 < n_slices) { advance(); gather(a1, b1); }
             if (!process(i, a0, b0)) break;
@@ -815,6 +834,7 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                 if (kAnyGather && i + 2 < n_slices) { advance(); gather(a0, b0); }
                 if (!process(i + 1, a1, b1)) break;
             }
+        }
         }
     } else {
         // ================= epilogue warps: drain chunks, accumulate in fp32 registers =================
