@@ -503,7 +503,7 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
     constexpr bool kAnyGather = kGatherA || kGatherB;
     constexpr bool kSplit = kATmem && !kAnyGather;                         // A raw tiles in a ring of their own
     // the transform warps work as two groups of four on alternate slices (else all eight on every slice)
-    constexpr bool kTwoGroups = !kAnyGather || (kModeB == kGatherTaps4 && kModeA == kTma);
+    constexpr bool kTwoGroups = !kAnyGather || (IsTaps<kModeB>::value && kModeA == kTma);
     constexpr int kNB = kSplit ? kSplitB : kRawSlots;                      // slots of the raw / hi ring
     // lo slots (and A slots in TMEM); the per-example form needs 128 TMEM columns for its sum of squares
     constexpr int kLoN = (kExact && kATmem) ? 2 : kSplit ? kSplitLo : (kATmem ? kLoSlotsAT : kLoSlots);
@@ -701,8 +701,7 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         const int t = (int)threadIdx.x - 64;                               // 0..255
         // With nothing to gather the eight warps work as two groups of four that take alternate slices: the
         // waits, fences and tensor-memory stores of one slice then overlap the arithmetic of the next one.
-        // The same split is used when the B tile is gathered three taps at a time (widths that are multiples of 4;
-        // the 2 + 2 form measures slower that way) next to a TMA-fed A tile.
+        // The same split is used when the B tile is gathered three taps at a time next to a TMA-fed A tile.
         constexpr int kTT = kTwoGroups ? kTransformThreads / 2 : kTransformThreads;   // threads sharing a slice
         const int group = kTwoGroups ? (t >> 7) : 0;
         const int tt = kTwoGroups ? (t & 127) : t;
@@ -811,16 +810,14 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         RegsA a0, a1;
         RegsB b0, b1;
         if (kTwoGroups && kAnyGather) {
-            // this group's slices: group, group + 2, ...; the loads of its next slice fly while one is transformed
+            // this group's slices: group, group + 2, ...
+            // one register set per thread: the other group's work covers this group's load latency (measured
+            // faster than two sets in turn)
             for (int sk = 0; sk < group; ++sk) advance();
-            if (group < n_slices) gather(a0, b0);
-            for (int i = group; i < n_slices; i += 4) {
-                if (i + 2 < n_slices) { advance(); advance(); gather(a1, b1); }
+            for (int i = group; i < n_slices; i += 2) {
+                gather(a0, b0);
                 if (!process(i, a0, b0)) break;
-                if (i + 2 < n_slices) {
-                    if (i + 4 < n_slices) { advance(); advance(); gather(a0, b0); }
-                    if (!process(i + 2, a1, b1)) break;
-                }
+                advance(); advance();
             }
         } else if (kTwoGroups) {
             for (int i = group; i < n_slices; i += 2)
