@@ -80,7 +80,9 @@ enum { kMajorK = 0, kMajorMN = 1 };
 
 // how a tile gets its rows; kGatherTaps4 / kGatherTaps2: im2col rows of a Kw = 3, stride 1, pad_w = 1 kernel
 // gathered three taps at a time (output width a multiple of 4 / of 2)
-enum { kTma = 0, kGatherErr = 1, kGatherIm2col = 2, kGatherTaps4 = 3, kGatherTaps2 = 4 };
+// kGatherTaps4S2 / kGatherTaps2S2: the same for stride 2 along w (input width twice the output width)
+enum { kTma = 0, kGatherErr = 1, kGatherIm2col = 2, kGatherTaps4 = 3, kGatherTaps2 = 4, kGatherTaps4S2 = 5,
+       kGatherTaps2S2 = 6 };
 
 struct Params {
     int M, N;                // rows of the A tile space / of the B tile space
@@ -360,6 +362,10 @@ struct GatherRows {
 template <int kSpan, int kTriples>      // kSpan: output positions covered by one aligned vector load, 4 or 2
 struct GatherTaps {
     static constexpr int kStride = kTriples == 2 ? 32 : 16;
+    static constexpr int kSlots = 8;                         // registers per triple
+    static constexpr int kLoaded = kSpan == 4 ? 6 : 8;       // of which loaded
+    // register that holds the input of tap kw for the j-th of the thread's four output positions
+    __device__ __forceinline__ static constexpr int idx(int kw, int j) { return kSpan == 4 ? kw + j : (j >> 1) * 4 + (j & 1) + kw; }
     int base[kTriples], dh[kTriples], row_local[kTriples];
     bool ok[kTriples];
     const float *src;
@@ -420,7 +426,73 @@ struct GatherTaps {
     }
 };
 
-template <int kMode> struct IsTaps { static constexpr bool value = kMode == kGatherTaps4 || kMode == kGatherTaps2; };
+// Stride 2 along w with Kw = 3, pad_w = 1 and W == 2 Wo: the 4 (or 2) output positions of a span read the input
+// columns 2 wo - 1 .. 2 wo + 7 (or + 3): one neighbour on the left and two (one) aligned 4-vectors, never past the
+// row's end.  Tap kw of output j is element 2 j + kw of that segment.
+template <int kSpan, int kTriples>
+struct GatherTapsS2 {
+    static constexpr int kStride = kTriples == 2 ? 32 : 16;
+    static constexpr int kPerSpan = kSpan == 4 ? 9 : 5;
+    static constexpr int kSlots = 10;
+    static constexpr int kLoaded = kSpan == 4 ? 9 : 10;
+    __device__ __forceinline__ static constexpr int idx(int kw, int j)
+    {
+        return kSpan == 4 ? 2 * j + kw : (j >> 1) * 5 + 2 * (j & 1) + kw;
+    }
+    int base[kTriples], dh[kTriples], row_local[kTriples];
+    bool ok[kTriples];
+    const float *src;
+
+    __device__ __forceinline__ void init(const Params &prm, const float *x, int tile_origin, int grp, int limit)
+    {
+        src = x;
+        const int first_triple = tile_origin / 3;
+#pragma unroll
+        for (int i = 0; i < kTriples; ++i) {
+            const int T = first_triple + grp + kStride * i;          // triple = (c, kh)
+            ok[i] = 3 * T < limit;
+            const int tt = ok[i] ? T : 0;
+            const int c = tt / prm.Kh, kh = tt - c * prm.Kh;
+            dh[i] = kh - prm.ph;
+            base[i] = (c * prm.H + dh[i]) * prm.W;
+            row_local[i] = 3 * T - tile_origin;
+        }
+    }
+    __device__ __forceinline__ void load(const Params &prm, int z, int pbase, float (&v)[kTriples][kSlots]) const
+    {
+        const float *xz = src + (size_t)z * prm.chw;
+#pragma unroll
+        for (int s = 0; s < 4 / kSpan; ++s) {
+            const int p = pbase + s * kSpan;
+            const int ho = (int)__umulhi((unsigned)p, prm.wo_magic), wo = p - ho * prm.Wo;
+            const bool pv = p < prm.P;
+            const int hs = ho * prm.sh;
+            const float *xp = xz + (hs * prm.W + 2 * wo);
+#pragma unroll
+            for (int i = 0; i < kTriples; ++i) {
+                const bool in = pv && ok[i] && (unsigned)(hs + dh[i]) < (unsigned)prm.H;
+                const float *q = xp + base[i];
+                float *o = &v[i][s * kPerSpan];
+                const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+                const float4 m0 = in ? __ldg(reinterpret_cast<const float4 *>(q)) : zero;
+                o[0] = (in && wo > 0) ? __ldg(q - 1) : 0.f;
+                o[1] = m0.x; o[2] = m0.y; o[3] = m0.z; o[4] = m0.w;
+                if (kSpan == 4) {
+                    const float4 m1 = in ? __ldg(reinterpret_cast<const float4 *>(q) + 1) : zero;
+                    o[5] = m1.x; o[6] = m1.y; o[7] = m1.z; o[8] = m1.w;
+                }
+            }
+        }
+    }
+};
+
+template <int kMode> struct IsTaps {
+    static constexpr bool value = kMode == kGatherTaps4 || kMode == kGatherTaps2 || kMode == kGatherTaps4S2 ||
+                                  kMode == kGatherTaps2S2;
+};
+template <int kMode, int kTriples> struct TapsOf { typedef GatherTaps<kMode == kGatherTaps4 ? 4 : 2, kTriples> type; };
+template <int kTriples> struct TapsOf<kGatherTaps4S2, kTriples> { typedef GatherTapsS2<4, kTriples> type; };
+template <int kTriples> struct TapsOf<kGatherTaps2S2, kTriples> { typedef GatherTapsS2<2, kTriples> type; };
 
 // One interface over both gather forms: the registers of one slice, how they are loaded and where their
 // squared, split values go in a K-major swizzled tile.  row0 = t >> 3 and kq = t & 7 of transform thread t.
@@ -445,8 +517,9 @@ struct Gatherer {
 template <int kMode, bool kHalf>
 struct Gatherer<kMode, kHalf, true> {
     static constexpr int kTriples = kHalf ? 3 : 2;
-    struct Regs { float v[kTriples][8]; };
-    GatherTaps<kMode == kGatherTaps4 ? 4 : 2, kTriples> g;
+    typedef typename TapsOf<kMode, kTriples>::type Impl;
+    struct Regs { float v[kTriples][Impl::kSlots]; };
+    Impl g;
     __device__ __forceinline__ void init(const Params &prm, const float *x, const float *, int origin, int row0, int limit)
     {
         g.init(prm, x, origin, row0, limit);
@@ -455,14 +528,13 @@ struct Gatherer<kMode, kHalf, true> {
     template <bool kSquare>
     __device__ __forceinline__ void store(uint8_t *hi, uint8_t *lo, int, int kq, const Regs &r) const
     {
-        constexpr int kLoaded = kMode == kGatherTaps4 ? 6 : 8;      // segment elements held per triple
 #pragma unroll
         for (int i = 0; i < kTriples; ++i) {
             if (g.row_local[i] >= kBM || g.row_local[i] <= -3) continue;   // no row of this triple in the tile
-            // square and split every loaded element once; the three taps are shifted views of the same parts
-            uint32_t h[8], l[8];
+            // square and split every loaded element once; the three taps are views of the same parts
+            uint32_t h[Impl::kSlots], l[Impl::kSlots];
 #pragma unroll
-            for (int e = 0; e < kLoaded; ++e) {
+            for (int e = 0; e < Impl::kLoaded; ++e) {
                 const float q = kSquare ? __fmul_rn(r.v[i][e], r.v[i][e]) : r.v[i][e];
                 h[e] = to_tf32(q);
                 l[e] = __float_as_uint(__fsub_rn(q, __uint_as_float(h[e])));
@@ -472,16 +544,10 @@ struct Gatherer<kMode, kHalf, true> {
                 const int row = g.row_local[i] + kw;
                 if ((unsigned)row < (unsigned)kBM) {                 // kBM == kBN rows in either tile
                     const uint32_t off = chunk_offset(row, kq);
-                    uint4 hv, lv;
-                    if (kMode == kGatherTaps4) {
-                        hv = make_uint4(h[kw], h[kw + 1], h[kw + 2], h[kw + 3]);
-                        lv = make_uint4(l[kw], l[kw + 1], l[kw + 2], l[kw + 3]);
-                    } else {
-                        hv = make_uint4(h[kw], h[kw + 1], h[4 + kw], h[4 + kw + 1]);
-                        lv = make_uint4(l[kw], l[kw + 1], l[4 + kw], l[4 + kw + 1]);
-                    }
-                    *reinterpret_cast<uint4 *>(hi + off) = hv;
-                    *reinterpret_cast<uint4 *>(lo + off) = lv;
+                    *reinterpret_cast<uint4 *>(hi + off) =
+                        make_uint4(h[Impl::idx(kw, 0)], h[Impl::idx(kw, 1)], h[Impl::idx(kw, 2)], h[Impl::idx(kw, 3)]);
+                    *reinterpret_cast<uint4 *>(lo + off) =
+                        make_uint4(l[Impl::idx(kw, 0)], l[Impl::idx(kw, 1)], l[Impl::idx(kw, 2)], l[Impl::idx(kw, 3)]);
                 }
             }
         }
@@ -1428,9 +1494,13 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
     const int taps = (!(taps_env && atoi(taps_env) == 0) && !in_tma && err_tma && Kw == 3 && sw == 1 && sh == 1 &&
                       pw == 1 && Wo == W && W % 2 == 0 && a_tmem)
                          ? (W % 4 == 0 ? 4 : 2) : 0;
+    // the same with stride 2 along w: W == 2 Wo, output width even
+    const int taps_s2 = (!(taps_env && atoi(taps_env) == 0) && !in_tma && err_tma && Kw == 3 && sw == 2 && pw == 1 &&
+                         W == 2 * Wo && Wo % 2 == 0 && a_tmem)
+                            ? (Wo % 4 == 0 ? 4 : 2) : 0;
     // with few output channels the roles are swapped -- except in the three-tap form, where keeping the errors as
     // the A operand (in tensor memory, half of its rows unused) measures faster than both operands in shared memory
-    const bool swapped = conv_swapped(Cout, n_im2col) && !taps;
+    const bool swapped = conv_swapped(Cout, n_im2col) && !taps && !taps_s2;
     const int rows_err = swapped ? kBN : kBM, rows_in = swapped ? kBM : kBN;     // tile heights
     Batch bt = {};
     uint32_t tx_err = 0, tx_in = 0;
@@ -1467,6 +1537,7 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
     if (!swapped) {     // S[o][idx]: m = o, n = idx
         prm.ld_m = n_im2col; prm.ld_n = 1;
         if (taps) fn = taps == 4 ? VGC_TC_FN(kTma, kGatherTaps4, true) : VGC_TC_FN(kTma, kGatherTaps2, true);
+        else if (taps_s2) fn = taps_s2 == 4 ? VGC_TC_FN(kTma, kGatherTaps4S2, true) : VGC_TC_FN(kTma, kGatherTaps2S2, true);
         else if (e == kTma && i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kTma, true) : sqgrad_tc<kMajorK, kTma, kTma, false>;
         else if (e == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kGatherIm2col, true) : sqgrad_tc<kMajorK, kTma, kGatherIm2col, false>;
         else if (i == kTma) fn = VGC_TC_FN(kGatherErr, kTma, false);

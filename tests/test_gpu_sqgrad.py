@@ -86,6 +86,8 @@ CONV_SHAPES = [  # B, C, H, Cout, k, stride, pad
     (1, 130, 4, 70, 3, 1, 1),
     # 3x3, stride 1, pad 1 on odd widths: planes padded to a multiple of 4 columns first
     (2, 40, 7, 130, 3, 1, 1), (4, 130, 7, 48, 3, 1, 1), (2, 16, 5, 72, 3, 1, 1),
+    # 3x3, stride 2, pad 1, input width twice the output width: three taps per gathered segment, stride-2 form
+    (2, 24, 12, 130, 3, 2, 1), (3, 50, 8, 40, 3, 2, 1), (2, 16, 24, 72, 3, 2, 1),
     # 7x7, stride 2, pad 3, few output channels: seven taps per gathered row segment
     (2, 3, 32, 16, 7, 2, 3), (1, 5, 24, 40, 7, 2, 3), (3, 20, 16, 64, 7, 2, 3),
 ]
