@@ -14,8 +14,8 @@ void tc_plan_hint(int concurrent_launches);
 bool tc_linear_supported(int B, int in, int out);
 bool tc_conv_supported(int B, int C, int H, int W, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw);
 size_t tc_linear_workspace_bytes(int B, int in, int out);
-size_t tc_conv_workspace_bytes(int n_layers, int B, int C, int Kh, int Kw, int sh, int sw, int ph, int pw, int P,
-                               int Cout, int Wo, bool exact = false);
+size_t tc_conv_workspace_bytes(int n_layers, int B, int C, int H, int W, int Kh, int Kw, int sh, int sw, int ph, int pw,
+                               int Ho, int Wo, int Cout, bool exact = false);
 vgc_status tc_sqgrad_linear(const float *x, const float *delta, int B, int in, int out, float scale, int accumulate,
                             float *S, void *ws, size_t ws_bytes, cudaStream_t st);
 vgc_status tc_sqgrad_conv(int n_layers, const float *const *x, const float *const *delta, float *const *S, int B, int C,
@@ -79,7 +79,7 @@ extern "C" size_t vgc_sqgrad_conv_batch_workspace_bytes(int n_layers, int B, int
     if (B == 0 || C == 0 || Cout == 0) return 0;
     size_t need = simt_workspace_bytes(Cout, C * Kh * Kw, B * Ho * Wo);
     if (tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w)) {
-        const size_t t = tc_conv_workspace_bytes(n_layers, B, C, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho * Wo, Cout, Wo);
+        const size_t t = tc_conv_workspace_bytes(n_layers, B, C, H, W, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho, Wo, Cout);
         need = need > t ? need : t;
     }
     return round_up(need + 256, 256);
@@ -138,7 +138,7 @@ extern "C" size_t vgc_sqgrad_conv_exact_workspace_bytes(int B, int C, int H, int
     if (!conv_shape_ok(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, &Ho, &Wo)) return 0;
     if (B == 0 || C == 0 || Cout == 0) return 0;
     if (!tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w)) return 0;
-    return round_up(tc_conv_workspace_bytes(1, B, C, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho * Wo, Cout, Wo, true) + 256,
+    return round_up(tc_conv_workspace_bytes(1, B, C, H, W, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho, Wo, Cout, true) + 256,
                     256);
 }
 

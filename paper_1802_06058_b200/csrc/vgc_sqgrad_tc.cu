@@ -1284,18 +1284,21 @@ static bool conv_swapped(int Cout, int n_im2col) { return Cout <= 64 && n_im2col
 //   kRepackFlat     x_r[c][z P + p], d_r[o][z P + p]: channel-major, the (example, position) pairs of one
 //                   channel back to back -- the layer becomes a 1x1 convolution over ONE example with
 //                   B P positions, and its reduction has no per-example padding to whole slices
-//   kRepackPadW     a Kw = 3, stride-1, pad_w = 1 kernel on planes of odd width W (7x7): x and the errors are
-//                   copied into planes of width W4 = W rounded up to 4 with zero columns.  The zero input column
-//                   is the right-hand padding, the zero error columns contribute nothing, so the statistic is
-//                   unchanged -- and the padded layer has TMA-able error planes and takes the three-tap gather
+//   kRepackPadW     a Kw = 3, pad_w = 1 kernel with stride 1 (W == Wo) or 2 (W == 2 Wo) whose output planes have
+//                   an odd width (7x7): the errors are copied into planes of width Wo4 = Wo rounded up to 4 and x
+//                   into planes of width stride * Wo4, new columns zero.  Zero input columns are what the padding
+//                   supplies anyway, zero error columns contribute nothing, so the statistic is unchanged -- and
+//                   the padded layer has TMA-able error planes and takes the three-tap gather
 enum { kRepackNone = 0, kRepackPlanes = 1, kRepackFlat = 2, kRepackPadW = 3 };
 
-static int repack_mode(int B, int C, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw, int P, int W = 0, int Ho = 0)
+static int repack_mode(int B, int C, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw, int P, int W = 0, int Ho = 0,
+                       int Wo = 0)
 {
     const char *e = getenv("VGC_TC_REPACK");
     if (e && atoi(e) == 0) return kRepackNone;
     if ((long)B * C >= (1L << 31) || (long)B * Cout >= (1L << 31)) return kRepackNone;      // 32-bit row index
-    if (Kw == 3 && sw == 1 && sh == 1 && pw == 1 && W % 2 == 1 && W >= 3 && (long)Ho * ((W + 3) / 4 * 4) >= kBK)
+    if (Kw == 3 && pw == 1 && Wo % 2 == 1 && Wo >= 3 && (long)Ho * ((Wo + 3) / 4 * 4) >= kBK &&
+        ((sw == 1 && sh == 1 && W == Wo) || (sw == 2 && W == 2 * Wo)))
         return kRepackPadW;
     if (Kh != 1 || Kw != 1 || ph != 0 || pw != 0) return kRepackNone;
     const bool planes_ok = P >= kBK && P % 4 == 0;
@@ -1385,19 +1388,18 @@ static size_t conv_workspace_plain(int n_layers, int B, int C, int Kh, int Kw, i
 
 // Workspace of one launch over n_layers layers of this geometry (n_layers <= kMaxBatch).
 static size_t conv_workspace_group(int n_layers, int B, int C, int Kh, int Kw, int sh, int sw, int ph, int pw, int P,
-                                   int Cout, int Wo_)
+                                   int Cout, int H, int W, int Ho, int Wo)
 {
     // the larger of the in-place form and the repacked one, so that either can be chosen at call time
     size_t need = conv_workspace_plain(n_layers, B, C, Kh, Kw, P, Cout);
-    // the width W of the input equals the output width whenever kRepackPadW applies, and P / Wo = Ho
-    const int mode = repack_mode(B, C, Cout, Kh, Kw, sh, sw, ph, pw, P, Wo_, Wo_ ? P / Wo_ : 0);
+    const int mode = repack_mode(B, C, Cout, Kh, Kw, sh, sw, ph, pw, P, W, Ho, Wo);
     const size_t x_bytes = round_up(sizeof(float) * (size_t)B * C * P, 256);
     const size_t d_bytes = round_up(sizeof(float) * (size_t)B * Cout * P, 256);
     if (mode == kRepackPadW) {
-        const int W4 = (Wo_ + 3) / 4 * 4, Ho = P / Wo_, H = Ho + Kh - 1 - 2 * ph;      // stride 1
-        const size_t xp = round_up(sizeof(float) * (size_t)B * C * H * W4, 256);
-        const size_t dp = round_up(sizeof(float) * (size_t)B * Cout * Ho * W4, 256);
-        const size_t r = round_up(conv_workspace_plain(n_layers, B, C, Kh, Kw, Ho * W4, Cout), 256) + n_layers * (xp + dp);
+        const int Wo4 = (Wo + 3) / 4 * 4;
+        const size_t xp = round_up(sizeof(float) * (size_t)B * C * H * (sw * Wo4), 256);
+        const size_t dp = round_up(sizeof(float) * (size_t)B * Cout * Ho * Wo4, 256);
+        const size_t r = round_up(conv_workspace_plain(n_layers, B, C, Kh, Kw, Ho * Wo4, Cout), 256) + n_layers * (xp + dp);
         need = need > r ? need : r;
     } else if (mode == kRepackPlanes) {
         const size_t r = round_up(conv_workspace_plain(n_layers, B, C, 1, 1, P, Cout), 256) + n_layers * x_bytes;
@@ -1410,16 +1412,17 @@ static size_t conv_workspace_group(int n_layers, int B, int C, int Kh, int Kw, i
     return need;
 }
 
-size_t tc_conv_workspace_bytes(int n_layers, int B, int C, int Kh, int Kw, int sh, int sw, int ph, int pw, int P,
-                               int Cout, int Wo_, bool exact)
+size_t tc_conv_workspace_bytes(int n_layers, int B, int C, int H, int W, int Kh, int Kw, int sh, int sw, int ph, int pw,
+                               int Ho, int Wo, int Cout, bool exact)
 {
+    const int P = Ho * Wo;
     ExactScope scope(exact);
     // more layers than one launch takes are processed group after group in the same workspace
     const int first = n_layers < kMaxBatch ? n_layers : kMaxBatch;
-    size_t need = conv_workspace_group(first, B, C, Kh, Kw, sh, sw, ph, pw, P, Cout, Wo_);
+    size_t need = conv_workspace_group(first, B, C, Kh, Kw, sh, sw, ph, pw, P, Cout, H, W, Ho, Wo);
     const int rest = n_layers > kMaxBatch ? n_layers % kMaxBatch : 0;
     if (rest) {
-        const size_t r = conv_workspace_group(rest, B, C, Kh, Kw, sh, sw, ph, pw, P, Cout, Wo_);
+        const size_t r = conv_workspace_group(rest, B, C, Kh, Kw, sh, sw, ph, pw, P, Cout, H, W, Ho, Wo);
         need = need > r ? need : r;
     }
     return need;
@@ -1430,14 +1433,14 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
                              int Wo, float scale, int accumulate, void *ws, size_t ws_bytes, cudaStream_t st)
 {
     const int P = Ho * Wo, n_im2col = C * Kh * Kw;
-    const int mode = repack_mode(B, C, Cout, Kh, Kw, sh, sw, ph, pw, P, W, Ho);
+    const int mode = repack_mode(B, C, Cout, Kh, Kw, sh, sw, ph, pw, P, W, Ho, Wo);
     // one warp per row; a few rows per warp when there are many
     auto blocks_for = [](size_t rows) { const size_t b = (rows + 31) / 32; return (unsigned)(b < 1 ? 1 : (b > 148 * 32 ? 148 * 32 : b)); };
     if (mode == kRepackPadW) {
-        const int W4 = (W + 3) / 4 * 4;
-        const size_t inner = round_up(conv_workspace_plain(n_layers, B, C, Kh, Kw, Ho * W4, Cout), 256);
-        const size_t xp = round_up(sizeof(float) * (size_t)B * C * H * W4, 256);
-        const size_t dp = round_up(sizeof(float) * (size_t)B * Cout * Ho * W4, 256);
+        const int Wo4 = (Wo + 3) / 4 * 4, Wx = sw * Wo4;              // padded widths of the errors and of x
+        const size_t inner = round_up(conv_workspace_plain(n_layers, B, C, Kh, Kw, Ho * Wo4, Cout), 256);
+        const size_t xp = round_up(sizeof(float) * (size_t)B * C * H * Wx, 256);
+        const size_t dp = round_up(sizeof(float) * (size_t)B * Cout * Ho * Wo4, 256);
         if (ws_bytes < inner + n_layers * (xp + dp)) return VGC_ERR_WORKSPACE;
         const float *xr[kMaxBatch], *dr[kMaxBatch];
         RepackJobs jobs = {};
@@ -1445,13 +1448,13 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
         for (int l = 0; l < n_layers; ++l) {
             char *base = static_cast<char *>(ws) + inner + (size_t)l * (xp + dp);
             float *x_p = reinterpret_cast<float *>(base), *d_p = reinterpret_cast<float *>(base + xp);
-            jobs.job[2 * l] = RepackJob{x[l], x_p, C, H * W, W, W4, H * W4, 1, 1, 0, W};
-            jobs.job[2 * l + 1] = RepackJob{delta[l], d_p, Cout, Ho * Wo, Wo, W4, Ho * W4, 1, 1, 0, Wo};
+            jobs.job[2 * l] = RepackJob{x[l], x_p, C, H * W, W, Wx, H * Wx, 1, 1, 0, W};
+            jobs.job[2 * l + 1] = RepackJob{delta[l], d_p, Cout, Ho * Wo, Wo, Wo4, Ho * Wo4, 1, 1, 0, Wo};
             xr[l] = x_p; dr[l] = d_p;
         }
         sqgrad_repack<<<dim3(blocks_for((size_t)B * (C > Cout ? C : Cout)), 2 * n_layers), 256, 0, st>>>(jobs);
         count_launch();
-        return conv_group(n_layers, xr, dr, S, B, C, H, W4, Cout, Kh, Kw, 1, 1, ph, 1, Ho, W4, scale, accumulate, ws, inner, st);
+        return conv_group(n_layers, xr, dr, S, B, C, H, Wx, Cout, Kh, Kw, sh, sw, ph, 1, Ho, Wo4, scale, accumulate, ws, inner, st);
     }
     if (mode != kRepackNone) {
         const bool flat = mode == kRepackFlat;

@@ -92,7 +92,7 @@ CONV_SHAPES = [  # B, C, H, Cout, k, stride, pad
     (2, 3, 32, 16, 7, 2, 3), (1, 5, 24, 40, 7, 2, 3), (3, 20, 16, 64, 7, 2, 3),
 ]
 REPACKED = [(4, 70, 7, 130, 1, 1, 0), (4, 48, 14, 200, 1, 2, 0), (2, 96, 16, 160, 1, 2, 0), (3, 64, 28, 40, 1, 2, 0),
-            (2, 40, 7, 130, 3, 1, 1), (3, 24, 9, 20, 3, 1, 1)]
+            (2, 40, 7, 130, 3, 1, 1), (3, 24, 9, 20, 3, 1, 1), (4, 16, 14, 24, 3, 2, 1), (2, 64, 14, 130, 3, 2, 1)]
 
 
 @pytest.mark.parametrize("B,C,H,Cout,k,s,p", CONV_SHAPES)

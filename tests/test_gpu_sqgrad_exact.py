@@ -17,7 +17,9 @@ SHAPES = [  # B, C, H, Cout, k, stride, pad
     (2, 24, 14, 130, 3, 1, 1),      # ... width % 4 == 2
     (2, 40, 12, 48, 3, 1, 1),       # 3x3 swapped
     (2, 40, 7, 130, 3, 1, 1),       # odd width: padded planes
-    (2, 72, 16, 200, 3, 2, 1),      # strided 3x3: element-wise gather
+    (2, 72, 16, 200, 3, 2, 1),      # strided 3x3: three taps at a time, stride-2 form
+    (2, 32, 14, 96, 3, 2, 1),       # ... with odd output width: padded planes first
+    (2, 20, 9, 40, 3, 2, 1),        # strided 3x3, odd input width: element-wise gather
     (2, 96, 16, 160, 1, 2, 0),      # strided 1x1: subsampled planes
     (2, 3, 32, 16, 7, 2, 3),        # first-layer shape
     (3, 16, 40, 24, 1, 1, 0),       # 50 slices per example: several drains inside one example
