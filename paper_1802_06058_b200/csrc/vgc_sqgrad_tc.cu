@@ -81,8 +81,9 @@ enum { kMajorK = 0, kMajorMN = 1 };
 // how a tile gets its rows; kGatherTaps4 / kGatherTaps2: im2col rows of a Kw = 3, stride 1, pad_w = 1 kernel
 // gathered three taps at a time (output width a multiple of 4 / of 2)
 // kGatherTaps4S2 / kGatherTaps2S2: the same for stride 2 along w (input width twice the output width)
+// kGatherTaps7S2: seven taps at a time for a Kw = 7, stride-2, pad-3 kernel (the first layer of the ImageNet networks)
 enum { kTma = 0, kGatherErr = 1, kGatherIm2col = 2, kGatherTaps4 = 3, kGatherTaps2 = 4, kGatherTaps4S2 = 5,
-       kGatherTaps2S2 = 6 };
+       kGatherTaps2S2 = 6, kGatherTaps7S2 = 7 };
 
 struct Params {
     int M, N;                // rows of the A tile space / of the B tile space
@@ -362,6 +363,7 @@ struct GatherRows {
 template <int kSpan, int kTriples>      // kSpan: output positions covered by one aligned vector load, 4 or 2
 struct GatherTaps {
     static constexpr int kStride = kTriples == 2 ? 32 : 16;
+    static constexpr int kKw = 3;
     static constexpr int kSlots = 8;                         // registers per triple
     static constexpr int kLoaded = kSpan == 4 ? 6 : 8;       // of which loaded
     // register that holds the input of tap kw for the j-th of the thread's four output positions
@@ -433,6 +435,7 @@ template <int kSpan, int kTriples>
 struct GatherTapsS2 {
     static constexpr int kStride = kTriples == 2 ? 32 : 16;
     static constexpr int kPerSpan = kSpan == 4 ? 9 : 5;
+    static constexpr int kKw = 3;
     static constexpr int kSlots = 10;
     static constexpr int kLoaded = kSpan == 4 ? 9 : 10;
     __device__ __forceinline__ static constexpr int idx(int kw, int j)
@@ -486,13 +489,66 @@ struct GatherTapsS2 {
     }
 };
 
+// Kw = 7, stride 2, pad_w = 3, W == 2 Wo, Wo a multiple of 4: the seven rows (c, kh, kw = 0..6) read, for four
+// consecutive output positions, the input columns 2 wo - 3 .. 2 wo + 9.  Four aligned 4-vectors from column 2 wo - 4
+// on cover them (each wholly inside or wholly outside the row); tap kw of output j is element 1 + 2 j + kw.
+// 128 threads share a slice; a thread owns the tuples first_tuple + grp + 16 i, i = 0, 1 (at most 20 touch a tile).
+template <int kTuples>
+struct GatherTaps7S2 {
+    static_assert(kTuples == 2, "used by the two-group form only");
+    static constexpr int kStride = 16;
+    static constexpr int kKw = 7;
+    static constexpr int kSlots = 16;
+    static constexpr int kLoaded = 14;
+    __device__ __forceinline__ static constexpr int idx(int kw, int j) { return 1 + 2 * j + kw; }
+    int base[kTuples], dh[kTuples], row_local[kTuples];
+    bool ok[kTuples];
+    const float *src;
+
+    __device__ __forceinline__ void init(const Params &prm, const float *x, int tile_origin, int grp, int limit)
+    {
+        src = x;
+        const int first_tuple = tile_origin / 7;
+#pragma unroll
+        for (int i = 0; i < kTuples; ++i) {
+            const int T = first_tuple + grp + kStride * i;           // tuple = (c, kh)
+            ok[i] = 7 * T < limit;
+            const int tt = ok[i] ? T : 0;
+            const int c = tt / prm.Kh, kh = tt - c * prm.Kh;
+            dh[i] = kh - prm.ph;
+            base[i] = (c * prm.H + dh[i]) * prm.W;
+            row_local[i] = 7 * T - tile_origin;
+        }
+    }
+    __device__ __forceinline__ void load(const Params &prm, int z, int pbase, float (&v)[kTuples][kSlots]) const
+    {
+        const int ho = (int)__umulhi((unsigned)pbase, prm.wo_magic), wo = pbase - ho * prm.Wo;
+        const int hs = ho * prm.sh;
+        const bool pv = pbase < prm.P;
+        const float *xp = src + (size_t)z * prm.chw + (hs * prm.W + 2 * wo - 4);
+        const int col0 = 2 * wo - 4;
+#pragma unroll
+        for (int i = 0; i < kTuples; ++i) {
+            const bool in = pv && ok[i] && (unsigned)(hs + dh[i]) < (unsigned)prm.H;
+            const float4 *q = reinterpret_cast<const float4 *>(xp + base[i]);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const bool inside = in && (unsigned)(col0 + 4 * u) < (unsigned)prm.W;
+                const float4 m = inside ? __ldg(q + u) : make_float4(0.f, 0.f, 0.f, 0.f);
+                v[i][4 * u] = m.x; v[i][4 * u + 1] = m.y; v[i][4 * u + 2] = m.z; v[i][4 * u + 3] = m.w;
+            }
+        }
+    }
+};
+
 template <int kMode> struct IsTaps {
     static constexpr bool value = kMode == kGatherTaps4 || kMode == kGatherTaps2 || kMode == kGatherTaps4S2 ||
-                                  kMode == kGatherTaps2S2;
+                                  kMode == kGatherTaps2S2 || kMode == kGatherTaps7S2;
 };
 template <int kMode, int kTriples> struct TapsOf { typedef GatherTaps<kMode == kGatherTaps4 ? 4 : 2, kTriples> type; };
 template <int kTriples> struct TapsOf<kGatherTaps4S2, kTriples> { typedef GatherTapsS2<4, kTriples> type; };
 template <int kTriples> struct TapsOf<kGatherTaps2S2, kTriples> { typedef GatherTapsS2<2, kTriples> type; };
+template <int kTriples> struct TapsOf<kGatherTaps7S2, kTriples> { typedef GatherTaps7S2<2> type; };
 
 // One interface over both gather forms: the registers of one slice, how they are loaded and where their
 // squared, split values go in a K-major swizzled tile.  row0 = t >> 3 and kq = t & 7 of transform thread t.
@@ -516,7 +572,7 @@ struct Gatherer {
 };
 template <int kMode, bool kHalf>
 struct Gatherer<kMode, kHalf, true> {
-    static constexpr int kTriples = kHalf ? 3 : 2;
+    static constexpr int kTriples = kMode == kGatherTaps7S2 ? 2 : kHalf ? 3 : 2;      // tuples of rows per thread
     typedef typename TapsOf<kMode, kTriples>::type Impl;
     struct Regs { float v[kTriples][Impl::kSlots]; };
     Impl g;
@@ -530,7 +586,7 @@ struct Gatherer<kMode, kHalf, true> {
     {
 #pragma unroll
         for (int i = 0; i < kTriples; ++i) {
-            if (g.row_local[i] >= kBM || g.row_local[i] <= -3) continue;   // no row of this triple in the tile
+            if (g.row_local[i] >= kBM || g.row_local[i] <= -Impl::kKw) continue;   // no row of this tuple in the tile
             // square and split every loaded element once; the three taps are views of the same parts
             uint32_t h[Impl::kSlots], l[Impl::kSlots];
 #pragma unroll
@@ -540,7 +596,7 @@ struct Gatherer<kMode, kHalf, true> {
                 l[e] = __float_as_uint(__fsub_rn(q, __uint_as_float(h[e])));
             }
 #pragma unroll
-            for (int kw = 0; kw < 3; ++kw) {
+            for (int kw = 0; kw < Impl::kKw; ++kw) {
                 const int row = g.row_local[i] + kw;
                 if ((unsigned)row < (unsigned)kBM) {                 // kBM == kBN rows in either tile
                     const uint32_t off = chunk_offset(row, kq);
@@ -1501,9 +1557,12 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
     const int taps_s2 = (!(taps_env && atoi(taps_env) == 0) && !in_tma && err_tma && Kw == 3 && sw == 2 && pw == 1 &&
                          W == 2 * Wo && Wo % 2 == 0 && a_tmem)
                             ? (Wo % 4 == 0 ? 4 : 2) : 0;
+    // seven taps at a time: Kw = 7, stride 2, pad 3
+    const bool taps7 = !(taps_env && atoi(taps_env) == 0) && !in_tma && err_tma && Kw == 7 && sw == 2 && pw == 3 &&
+                       W == 2 * Wo && Wo % 4 == 0 && a_tmem;
     // with few output channels the roles are swapped -- except in the three-tap form, where keeping the errors as
     // the A operand (in tensor memory, half of its rows unused) measures faster than both operands in shared memory
-    const bool swapped = conv_swapped(Cout, n_im2col) && !taps && !taps_s2;
+    const bool swapped = conv_swapped(Cout, n_im2col) && !taps && !taps_s2 && !taps7;
     const int rows_err = swapped ? kBN : kBM, rows_in = swapped ? kBM : kBN;     // tile heights
     Batch bt = {};
     uint32_t tx_err = 0, tx_in = 0;
@@ -1541,6 +1600,7 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
         prm.ld_m = n_im2col; prm.ld_n = 1;
         if (taps) fn = taps == 4 ? VGC_TC_FN(kTma, kGatherTaps4, true) : VGC_TC_FN(kTma, kGatherTaps2, true);
         else if (taps_s2) fn = taps_s2 == 4 ? VGC_TC_FN(kTma, kGatherTaps4S2, true) : VGC_TC_FN(kTma, kGatherTaps2S2, true);
+        else if (taps7) fn = VGC_TC_FN(kTma, kGatherTaps7S2, true);
         else if (e == kTma && i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kTma, true) : sqgrad_tc<kMajorK, kTma, kTma, false>;
         else if (e == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kGatherIm2col, true) : sqgrad_tc<kMajorK, kTma, kGatherIm2col, false>;
         else if (i == kTma) fn = VGC_TC_FN(kGatherErr, kTma, false);
