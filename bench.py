@@ -660,7 +660,7 @@ def main():
     # DRAM traffic measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum), per launch group:
     # profiles/sqgrad_tc_resnet50_pass.md (one pass over the 54 ResNet-50 layers) and
     # profiles/compress_flat_n33554432.md (scaled by n: the traffic is proportional to the buffer length)
-    NCU_SQGRAD_PASS_BYTES_RESNET50 = 3.20e9
+    NCU_SQGRAD_PASS_BYTES_RESNET50 = 3.23e9
     NCU_COMPRESS_BYTES_PER_PARAM = (537.7e6 + 233.9e6 + 20.7e6 + 20.7e6) / 33554432
     compress_roofline = {"kernel": "compress_phase_a + compress_count + compress_emit", "bound": "hbm",
                          "achieved": compress_bytes / (co_ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
@@ -682,7 +682,7 @@ def main():
                     "note": "achieved = algorithmic flops 2*M*N*K per layer / sqgrad time; frac = tensor-pipe load: the "
                             "3xTF32 scheme issues 3 tensor-core products per algorithmic one, so frac is also issued "
                             "flops / TF32 peak; against the plain TF32 peak the algorithmic rate is a third of it; "
-                            "traffic = DRAM bytes of the 46 launches of one pass (profiles/launch_list_resnet50.md)"}
+                            "traffic = DRAM bytes of the 49 launches of one pass (profiles/launch_list_resnet50.md)"}
     else:
         roofline = compress_roofline
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
