@@ -138,7 +138,6 @@ class HotPath:
         self.fused = False
         self.hybrid = algorithm == "hybrid"                # Algorithm 2 instead of Algorithm 1
         self.exact_conv = exact_conv                       # per-example conv statistic (cross terms kept)
-        batch_layers = batch_layers and not exact_conv
         self.tau = 0.0
         dev = device
         B = self.batch
@@ -182,8 +181,7 @@ class HotPath:
                 if spec.kind == "conv":
                     geo = (B, spec.cin, spec.hin, spec.hin, spec.cout, spec.k, spec.k, spec.stride, spec.stride,
                            spec.pad, spec.pad)
-                    ws_bytes = max(ws_bytes, vgc.vgc_sqgrad_conv_exact_workspace_bytes(*geo) if exact_conv
-                                   else vgc.vgc_sqgrad_conv_batch_workspace_bytes(len(g), *geo),
+                    ws_bytes = max(ws_bytes, vgc.vgc_sqgrad_conv_batch_workspace_bytes(len(g), *geo, exact=exact_conv),
                                    vgc.vgc_sqgrad_conv_workspace_bytes(*geo))      # the end-to-end leg calls layer by layer
                 else:
                     ws_bytes = max(ws_bytes, vgc.vgc_sqgrad_linear_workspace_bytes(B, spec.cin, spec.cout))
@@ -248,14 +246,10 @@ class HotPath:
             lane = gi % self.n_streams
             stream = main if lane == 0 else self.side[lane - 1]
             ws = self.ws_s if lane == 0 else self.ws_side[lane - 1]
-            if spec.kind == "conv" and self.exact_conv:
-                vgc.vgc_sqgrad_conv_exact(ins[g[0]][0], ins[g[0]][1], (spec.k, spec.k), (spec.stride, spec.stride),
-                                          (spec.pad, spec.pad), self.scale, Ss[0], accumulate=into_v, ws=ws,
-                                          stream=stream)
-            elif spec.kind == "conv":
+            if spec.kind == "conv":
                 vgc.vgc_sqgrad_conv_batch([ins[li][0] for li in g], [ins[li][1] for li in g], (spec.k, spec.k),
                                           (spec.stride, spec.stride), (spec.pad, spec.pad), self.scale, Ss,
-                                          accumulate=into_v, ws=ws, stream=stream)
+                                          accumulate=into_v, ws=ws, stream=stream, exact=self.exact_conv)
             else:
                 vgc.vgc_sqgrad_linear(ins[g[0]][0], ins[g[0]][1], self.scale, Ss[0], accumulate=into_v, ws=ws,
                                       stream=stream)
@@ -584,7 +578,7 @@ def main():
     ap.add_argument("--no-batch", action="store_true",
                     help="one library call per layer instead of one per group of same-shaped conv layers")
     ap.add_argument("--exact-conv", action="store_true",
-                    help="conv layers through vgc_sqgrad_conv_exact (per-example statistic, one call per layer); "
+                    help="conv layers through vgc_sqgrad_conv_exact_batch (per-example statistic); "
                          "device-timed only")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -120,6 +120,13 @@ vgc_status vgc_sqgrad_conv_exact(const float *x, const float *delta, int B, int 
                                  int Kh, int Kw, int stride_h, int stride_w, int pad_h, int pad_w,
                                  float scale, int accumulate, float *S,
                                  void *ws, size_t ws_bytes, vgc_stream_t stream);
+/* ... for several layers of one geometry in one call, as vgc_sqgrad_conv_batch. */
+size_t vgc_sqgrad_conv_exact_batch_workspace_bytes(int n_layers, int B, int C, int H, int W, int Cout, int Kh, int Kw,
+                                                   int stride_h, int stride_w, int pad_h, int pad_w);
+vgc_status vgc_sqgrad_conv_exact_batch(int n_layers, const float *const *x, const float *const *delta, float *const *S,
+                                       int B, int C, int H, int W, int Cout, int Kh, int Kw, int stride_h, int stride_w,
+                                       int pad_h, int pad_w, float scale, int accumulate, void *ws, size_t ws_bytes,
+                                       vgc_stream_t stream);
 
 /* Planning hint (no counterpart in the paper): how many sqgrad calls the caller keeps in flight side by side
  * on different streams, each with its own workspace (default 1).  Alone, a launch is planned so that its

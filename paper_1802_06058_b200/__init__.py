@@ -29,6 +29,7 @@ EXPORTS = [
     "vgc_sqgrad_conv_workspace_bytes", "vgc_sqgrad_conv",
     "vgc_sqgrad_conv_batch_workspace_bytes", "vgc_sqgrad_conv_batch", "vgc_sqgrad_plan_hint",
     "vgc_sqgrad_conv_exact_workspace_bytes", "vgc_sqgrad_conv_exact",
+    "vgc_sqgrad_conv_exact_batch_workspace_bytes", "vgc_sqgrad_conv_exact_batch",
     "vgc_compress_workspace_bytes", "vgc_compress", "vgc_compress_static",
     "vgc_decode_accumulate", "vgc_step_host",
     "vgc_compress_hybrid_workspace_bytes", "vgc_compress_hybrid", "vgc_decode_accumulate_hybrid",
@@ -97,6 +98,10 @@ def load_library():
     lib.vgc_sqgrad_conv_exact_workspace_bytes.restype = sz
     lib.vgc_sqgrad_conv_exact.argtypes = lib.vgc_sqgrad_conv.argtypes
     lib.vgc_sqgrad_conv_exact.restype = i
+    lib.vgc_sqgrad_conv_exact_batch_workspace_bytes.argtypes = [i] * 12
+    lib.vgc_sqgrad_conv_exact_batch_workspace_bytes.restype = sz
+    lib.vgc_sqgrad_conv_exact_batch.argtypes = lib.vgc_sqgrad_conv_batch.argtypes
+    lib.vgc_sqgrad_conv_exact_batch.restype = i
     lib.vgc_compress_workspace_bytes.argtypes = [sz, i]
     lib.vgc_compress_workspace_bytes.restype = sz
     lib.vgc_compress.argtypes = [vp, vp, vp, vp, sz, vp, i, f, f, ctypes.POINTER(_MessageStruct), vp, sz, vp]
@@ -240,13 +245,22 @@ def vgc_sqgrad_plan_hint(concurrent_launches: int) -> None:
     load_library().vgc_sqgrad_plan_hint(int(concurrent_launches))
 
 
-def vgc_sqgrad_conv_batch_workspace_bytes(n_layers, B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw) -> int:
-    return load_library().vgc_sqgrad_conv_batch_workspace_bytes(n_layers, B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw)
+def vgc_sqgrad_conv_batch_workspace_bytes(n_layers, B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, exact: bool = False) -> int:
+    lib = load_library()
+    fn = lib.vgc_sqgrad_conv_exact_batch_workspace_bytes if exact else lib.vgc_sqgrad_conv_batch_workspace_bytes
+    return fn(n_layers, B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw)
+
+
+def vgc_sqgrad_conv_exact_batch(xs, deltas, kernel, stride, padding, scale: float, Ss, accumulate: bool = False,
+                                ws=None, stream=None):
+    """vgc_sqgrad_conv_exact for several layers of one geometry in one call."""
+    return vgc_sqgrad_conv_batch(xs, deltas, kernel, stride, padding, scale, Ss, accumulate, ws, stream, exact=True)
 
 
 def vgc_sqgrad_conv_batch(xs, deltas, kernel, stride, padding, scale: float, Ss, accumulate: bool = False,
-                          ws=None, stream=None):
-    """vgc_sqgrad_conv for several layers of one geometry (lists of tensors of equal shapes) in one call."""
+                          ws=None, stream=None, exact: bool = False):
+    """vgc_sqgrad_conv for several layers of one geometry (lists of tensors of equal shapes) in one call
+    (``exact``: the per-example statistic, vgc_sqgrad_conv_exact_batch)."""
     n = len(xs)
     if len(deltas) != n or len(Ss) != n:
         raise ValueError("xs, deltas, Ss must have the same length")
@@ -267,9 +281,11 @@ def vgc_sqgrad_conv_batch(xs, deltas, kernel, stride, padding, scale: float, Ss,
     dp = ptrs(*[_dev(d, torch.float32, "delta") for d in deltas])
     sp = ptrs(*[_dev(S, torch.float32, "S") for S in Ss])
     wp, wb = _ws(ws)
-    st = load_library().vgc_sqgrad_conv_batch(n, xp, dp, sp, B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, float(scale),
-                                              int(bool(accumulate)), wp, wb, _stream(stream))
-    _check(st, "vgc_sqgrad_conv_batch")
+    lib = load_library()
+    fn = lib.vgc_sqgrad_conv_exact_batch if exact else lib.vgc_sqgrad_conv_batch
+    st = fn(n, xp, dp, sp, B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, float(scale), int(bool(accumulate)), wp, wb,
+            _stream(stream))
+    _check(st, "vgc_sqgrad_conv_exact_batch" if exact else "vgc_sqgrad_conv_batch")
     return Ss
 
 

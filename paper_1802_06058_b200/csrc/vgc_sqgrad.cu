@@ -131,15 +131,44 @@ extern "C" vgc_status vgc_sqgrad_conv(const float *x, const float *delta, int B,
                                  accumulate, ws, ws_bytes, stream);
 }
 
+extern "C" size_t vgc_sqgrad_conv_exact_batch_workspace_bytes(int n_layers, int B, int C, int H, int W, int Cout, int Kh,
+                                                              int Kw, int stride_h, int stride_w, int pad_h, int pad_w)
+{
+    int Ho, Wo;
+    if (n_layers < 1 || !conv_shape_ok(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, &Ho, &Wo)) return 0;
+    if (B == 0 || C == 0 || Cout == 0) return 0;
+    if (!tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w)) return 0;
+    return round_up(tc_conv_workspace_bytes(n_layers, B, C, H, W, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho, Wo, Cout, true) +
+                        256,
+                    256);
+}
+
 extern "C" size_t vgc_sqgrad_conv_exact_workspace_bytes(int B, int C, int H, int W, int Cout, int Kh, int Kw,
                                                         int stride_h, int stride_w, int pad_h, int pad_w)
 {
+    return vgc_sqgrad_conv_exact_batch_workspace_bytes(1, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w);
+}
+
+extern "C" vgc_status vgc_sqgrad_conv_exact_batch(int n_layers, const float *const *x, const float *const *delta,
+                                                  float *const *S, int B, int C, int H, int W, int Cout, int Kh, int Kw,
+                                                  int stride_h, int stride_w, int pad_h, int pad_w, float scale,
+                                                  int accumulate, void *ws, size_t ws_bytes, vgc_stream_t stream)
+{
     int Ho, Wo;
-    if (!conv_shape_ok(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, &Ho, &Wo)) return 0;
-    if (B == 0 || C == 0 || Cout == 0) return 0;
-    if (!tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w)) return 0;
-    return round_up(tc_conv_workspace_bytes(1, B, C, H, W, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho, Wo, Cout, true) + 256,
-                    256);
+    if (n_layers < 0 || !conv_shape_ok(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, &Ho, &Wo))
+        return VGC_ERR_INVALID_ARG;
+    if (n_layers == 0 || C == 0 || Cout == 0) return VGC_OK;
+    if (B < 1 || !x || !delta || !S || !(scale == scale)) return VGC_ERR_INVALID_ARG;
+    for (int l = 0; l < n_layers; ++l)
+        if (!S[l] || !aligned16(S[l]) || !x[l] || !delta[l] || !aligned16(x[l]) || !aligned16(delta[l]))
+            return VGC_ERR_INVALID_ARG;
+    if (!tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w)) return VGC_ERR_UNSUPPORTED;
+    if (ws_bytes < vgc_sqgrad_conv_exact_batch_workspace_bytes(n_layers, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h,
+                                                               pad_w) ||
+        !ws)
+        return VGC_ERR_WORKSPACE;
+    return tc_sqgrad_conv(n_layers, x, delta, S, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho, Wo, scale,
+                          accumulate, ws, ws_bytes, reinterpret_cast<cudaStream_t>(stream), true);
 }
 
 extern "C" vgc_status vgc_sqgrad_conv_exact(const float *x, const float *delta, int B, int C, int H, int W, int Cout,
@@ -147,17 +176,8 @@ extern "C" vgc_status vgc_sqgrad_conv_exact(const float *x, const float *delta, 
                                             float scale, int accumulate, float *S, void *ws, size_t ws_bytes,
                                             vgc_stream_t stream)
 {
-    int Ho, Wo;
-    if (!conv_shape_ok(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, &Ho, &Wo))
-        return VGC_ERR_INVALID_ARG;
-    if (C == 0 || Cout == 0) return VGC_OK;
-    if (!S || !aligned16(S) || !(scale == scale)) return VGC_ERR_INVALID_ARG;
-    if (B < 1 || !x || !delta || !aligned16(x) || !aligned16(delta)) return VGC_ERR_INVALID_ARG;
-    if (!tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w)) return VGC_ERR_UNSUPPORTED;
-    if (ws_bytes < vgc_sqgrad_conv_exact_workspace_bytes(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w) || !ws)
-        return VGC_ERR_WORKSPACE;
-    return tc_sqgrad_conv(1, &x, &delta, &S, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho, Wo, scale,
-                          accumulate, ws, ws_bytes, reinterpret_cast<cudaStream_t>(stream), true);
+    return vgc_sqgrad_conv_exact_batch(1, &x, &delta, &S, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, scale,
+                                       accumulate, ws, ws_bytes, stream);
 }
 
 extern "C" void vgc_sqgrad_plan_hint(int concurrent_launches) { tc_plan_hint(concurrent_launches); }

@@ -74,3 +74,23 @@ def test_one_position_equals_the_position_statistic():
     want = oracle.sqgrad_conv(x.cpu().numpy(), d.cpu().numpy(), (1, 1), (1, 1), (0, 0), scale=1.0).astype(np.float64)
     got = run(x, d, 1, 1, 0, 1.0).astype(np.float64)
     assert np.all(np.abs(got - want) <= 1e-5 * want)
+
+
+@pytest.mark.parametrize("n_layers", [3, 9])
+@pytest.mark.parametrize("B,C,H,Cout,k,s,p", [(3, 96, 12, 160, 1, 1, 0), (2, 24, 16, 130, 3, 1, 1), (2, 40, 7, 130, 3, 1, 1)])
+def test_exact_batch(n_layers, B, C, H, Cout, k, s, p):
+    gen = torch.Generator(device="cuda"); gen.manual_seed(n_layers + C)
+    Ho = (H + 2 * p - k) // s + 1
+    xs = [torch.randn(B, C, H, H, device="cuda", generator=gen) for _ in range(n_layers)]
+    ds = [torch.randn(B, Cout, Ho, Ho, device="cuda", generator=gen) * 1e-2 for _ in range(n_layers)]
+    Ss = [torch.empty(Cout, C, k, k, device="cuda") for _ in range(n_layers)]
+    ws = torch.zeros(vgc.vgc_sqgrad_conv_batch_workspace_bytes(n_layers, B, C, H, H, Cout, k, k, s, s, p, p, exact=True),
+                     dtype=torch.uint8, device="cuda")
+    vgc.vgc_sqgrad_conv_exact_batch(xs, ds, (k, k), (s, s), (p, p), 0.5, Ss, ws=ws)
+    assert int(ws[:4].view(torch.int32).item()) == 0
+    for l in range(n_layers):
+        xn, dn = xs[l].cpu().numpy(), ds[l].cpu().numpy()
+        want = oracle.sqgrad_conv_exact(xn, dn, (k, k), (s, s), (p, p), scale=0.5).astype(np.float64)
+        bound = oracle.sqgrad_conv_exact(np.abs(xn), np.abs(dn), (k, k), (s, s), (p, p), scale=0.5).astype(np.float64)
+        got = Ss[l].cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got - want) <= 1e-5 * bound)
