@@ -155,6 +155,7 @@ class HotPath:
         self.ws_c = torch.empty(max(vgc.vgc_compress_workspace_bytes(self.n, self.K),
                                     vgc.vgc_compress_hybrid_workspace_bytes(self.n)), dtype=torch.uint8, device=dev)
         self.flops_useful = 0
+        self.flops_issued = 0.0      # in TF32-product equivalents: what the tensor pipe is asked to do
         self.inputs = []
         if self.compress_only:
             gs = [workloads.per_parameter_gs(self.n, B, delta_std, workloads.seed_for(cfg, worker, t, 0, 2), dev)
@@ -176,6 +177,11 @@ class HotPath:
             for li, spec in enumerate(self.layers):
                 M, N, K = spec.gemm_mnk(B)
                 self.flops_useful += 2 * M * N * K
+                # fp32 accuracy costs three TF32 products per algorithmic one; the TMA-fed form (all 1x1 convs) takes
+                # its two cross terms in bf16, at half the TF32 cost each
+                bf16_cross = (spec.kind == "conv" and spec.k == 1 and not exact_conv
+                              and os.environ.get("VGC_TC_BF16", "1") != "0")
+                self.flops_issued += 2 * M * N * K * (2.0 if bf16_cross else 3.0)
             for g in self.groups:
                 spec = self.layers[g[0]]
                 if spec.kind == "conv":
@@ -666,22 +672,26 @@ def main():
         tf32_peak = pk["bf16_tflops_sustained"] / 2.0          # nominal tf32 : bf16 ratio is 1 : 2
         # The contraction must be fp32-accurate (1e-5), which costs three TF32 tensor-core products per
         # algorithmic product: the peak for this arithmetic is a third of the TF32 rate.
-        fp32x3_peak = tf32_peak / 3.0
+        issue_factor = hp.flops_issued / hp.flops_useful       # 3, or less where cross terms run as bf16 products
+        fp32x3_peak = tf32_peak / issue_factor
         ach = hp.flops_useful / (sq_ms * 1e-3) / 1e12
         roofline = {"kernel": "sqgrad_tc (all layers of one step)", "bound": "tensor", "achieved": ach,
                     "peak": fp32x3_peak, "unit": "TFLOP/s", "frac": ach / fp32x3_peak,
                     "traffic": NCU_SQGRAD_PASS_BYTES_RESNET50 if args.workload == "resnet50" else None,
-                    "issued_tflops": 3 * ach, "tf32_peak": tf32_peak, "algorithmic_frac_of_tf32_peak": ach / tf32_peak,
-                    "peak_source": f"{pk['source']} bf16 sustained x 1/2 (tf32 nominal ratio) x 1/3 (3xTF32), of measured",
-                    "note": "achieved = algorithmic flops 2*M*N*K per layer / sqgrad time; frac = tensor-pipe load: the "
-                            "3xTF32 scheme issues 3 tensor-core products per algorithmic one, so frac is also issued "
-                            "flops / TF32 peak; against the plain TF32 peak the algorithmic rate is a third of it; "
+                    "issued_tflops": issue_factor * ach, "issue_factor": issue_factor, "tf32_peak": tf32_peak,
+                    "frac_of_3xtf32_ceiling": ach / (tf32_peak / 3.0),
+                    "algorithmic_frac_of_tf32_peak": ach / tf32_peak,
+                    "peak_source": f"{pk['source']} bf16 sustained x 1/2 (tf32 nominal ratio) / issue_factor, of measured",
+                    "note": "achieved = algorithmic flops 2*M*N*K per layer / sqgrad time; frac = tensor-pipe load: "
+                            "fp32 accuracy takes 3 tensor-core products per algorithmic one (hi*hi in TF32 plus two "
+                            "cross terms: TF32, or bf16 at half the cost in the TMA-fed form), issue_factor is their "
+                            "flop-weighted cost in TF32 products, so frac is also issued work / TF32 peak; "
                             "traffic = DRAM bytes of the 49 launches of one pass (profiles/launch_list_resnet50.md)"}
     else:
         roofline = compress_roofline
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32 (tf32x3 products where tensor cores are used)",
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32 (split into tf32 hi*hi + tf32 or bf16 cross terms on the tensor cores)",
             "data": "synthetic",
             "config": {"workload": args.workload, "n_params": n, "batch": hp.batch, "W": hp.W, "alpha": hp.alpha,
                        "zeta": ZETA, "groups": hp.K, "algorithm": args.algorithm, "tau": hp.tau, "launch": "eager" if args.no_graph else "cuda graph replay",

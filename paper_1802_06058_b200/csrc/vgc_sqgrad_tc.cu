@@ -11,7 +11,9 @@
 //      and in place (hi overwrites the raw tile, lo goes beside it), so both inherit the swizzled
 //      layout the tensor core wants,
 //   3. issues three tcgen05.mma per 8-deep step -- hi*hi, hi*lo, lo*hi -- into a TMEM
-//      accumulator (the dropped lo*lo term is 2^-22 relative).
+//      accumulator (the dropped lo*lo term is 2^-22 relative).  In the TMA-fed K-major form the two
+//      cross terms use bf16 copies of hi and lo instead (kind::f16, 16 deep per instruction): a
+//      cross term is 2^-11 of the product, so 8-bit operands leave an error below 2^-18 of it.
 // The tensor core's fp32 accumulation is not trusted over long reductions: every kChunk k slices
 // the accumulator is drained by four epilogue warps (tcgen05.ld) and added, round-to-nearest, to
 // fp32 registers while the next chunk accumulates into the second TMEM buffer.
@@ -32,6 +34,7 @@
 // Every wait on an mbarrier is bounded; on expiry the block raises an abort flag, all roles fall
 // through to the common exit, outstanding TMA loads are waited for (bounded) and TMEM is freed.
 #include <cuda.h>
+#include <cuda_bf16.h>
 
 #include <cstdlib>
 
@@ -219,6 +222,30 @@ __device__ __forceinline__ void tc_mma_tf32_ts_acc(uint32_t d_tmem, uint32_t a_t
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc)
         : "memory");
 }
+// the same with bf16 operands (two k per 32-bit column of the A block in tensor memory, 16 k per instruction)
+__device__ __forceinline__ void tc_mma_bf16_ts_acc(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.eq.u32 p, 1, 1;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc)
+        : "memory");
+}
+// 32 lanes x 8 columns
+__device__ __forceinline__ void tc_st_32x8(uint32_t taddr, const uint32_t (&r)[8])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+        : "memory");
+}
+// two consecutive k as one 32-bit word of bf16 (round to nearest even): k in the low half, k + 1 in the high half
+__device__ __forceinline__ uint32_t pack_bf16(float k0, float k1)
+{
+    const __nv_bfloat162 v = __floats2bfloat162_rn(k0, k1);
+    return *reinterpret_cast<const uint32_t *>(&v);
+}
 // 32 lanes x 16 columns: each thread stores 16 registers into its lane's row
 __device__ __forceinline__ void tc_st_32x16(uint32_t taddr, const uint32_t (&r)[16])
 {
@@ -270,6 +297,12 @@ __host__ __device__ constexpr uint32_t instr_desc(int major, int n)
 {
     return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)major << 15) | ((uint32_t)major << 16) |
            ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+}
+
+// The same for bf16 operands (both K-major), used for the two cross terms of the bf16-cross form.
+__host__ __device__ constexpr uint32_t instr_desc_bf16(int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
 }
 
 // One 16-byte chunk (4 consecutive k of one row) of a K-major 128-byte-swizzled tile.
@@ -614,7 +647,11 @@ struct Gatherer<kMode, kHalf, true> {
 // kExact: the per-example statistic of a conv layer, S = scale * sum_z (sum_p delta x)^2 -- operands are split without
 // squaring, an accumulator is drained at least at every example's end, the epilogue sums the drains of one example
 // in registers and adds the square of that sum into a third accumulator kept in tensor memory.
-template <int kMajor, int kModeA, int kModeB, bool kATmem, bool kExact = false>
+// kBf: the two cross terms hi*lo and lo*hi are taken with bf16 operands (half the shared-memory reads and half the
+// tensor-pipe time of a tf32 product each; their rounding, 2^-9 relative on a term that is itself 2^-11 of the
+// product, stays below 2^-18 of the result).  A lo slot then holds [B hi as bf16][B lo as bf16], 8 KB each with
+// 64-byte rows, and an A slot in tensor memory [hi tf32: 32 columns][hi bf16: 16][lo bf16: 16].
+template <int kMajor, int kModeA, int kModeB, bool kATmem, bool kExact = false, bool kBf = false>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
 {
@@ -624,6 +661,7 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
     constexpr bool kAnyTma = !kGatherA || !kGatherB;
     constexpr bool kAnyGather = kGatherA || kGatherB;
     constexpr bool kSplit = kATmem && !kAnyGather;                         // A raw tiles in a ring of their own
+    static_assert(!kBf || (kSplit && !kExact), "bf16 cross terms: the TMA-fed form with A in tensor memory");
     // the transform warps work as two groups of four on alternate slices (else all eight on every slice)
     constexpr bool kTwoGroups = !kAnyGather || (IsTaps<kModeB>::value && kModeA == kTma);
     constexpr int kNB = kSplit ? kSplitB : kRawSlots;                      // slots of the raw / hi ring
@@ -770,6 +808,11 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
             const uint32_t desc_hi = (uint32_t)(smem_desc(0, lbo, sbo, layout) >> 32);
             const uint32_t desc_lo0 = (uint32_t)smem_desc(0, lbo, sbo, layout);
             auto desc_at = [&](uint32_t lo16) -> uint64_t { return ((uint64_t)desc_hi << 32) | (desc_lo0 + lo16); };
+            // bf16 tiles: K-major rows of 64 B with the 64-byte swizzle (mode 4), 8-row groups 512 B apart
+            const uint32_t idesc_bf = instr_desc_bf16(n_act);
+            const uint32_t desc_bf_hi = (uint32_t)(smem_desc(0, 16u, 512u, 4u) >> 32);
+            const uint32_t desc_bf_lo0 = (uint32_t)smem_desc(0, 16u, 512u, 4u);
+            auto desc_bf = [&](uint32_t lo16) -> uint64_t { return ((uint64_t)desc_bf_hi << 32) | (desc_bf_lo0 + lo16); };
             int i = 0, st = 0, ls = 0;                   // slice, its raw / hi slot, its lo slot
             uint32_t st_phase = 0;
             bool ok = true;
@@ -788,6 +831,21 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                     const uint32_t hi_a16 = (smem_base + pair_off(st)) >> 4, hi_b16 = hi_a16 + (kRawBytesA >> 4);
                     const uint32_t lo_a16 = (smem_base + lo_off(ls)) >> 4, lo_b16 = lo_a16 + (kRawBytesA >> 4);   // lo_a unused with A in TMEM
                     const uint32_t ta_hi = tmem_base + 2 * kBN + ls * kTmemColsA, ta_lo = ta_hi + 32;
+                    if (kBf) {
+#pragma unroll
+                        for (int kk = 0; kk < kBK / 8; ++kk) {
+                            const uint64_t db_hi = desc_at(hi_b16 + kk * k_step16);
+                            if (kk == 0) tc_mma_tf32_ts(d_tmem, ta_hi, db_hi, idesc, first ? 0u : 1u);
+                            else tc_mma_tf32_ts_acc(d_tmem, ta_hi + kk * 8, db_hi, idesc);
+                        }
+                        // cross terms, 16 k (32 bytes of a 64-byte row, 8 columns of tensor memory) per instruction
+                        const uint32_t bf_hi16 = lo_b16, bf_lo16 = lo_b16 + (kRawBytesB >> 5);
+#pragma unroll
+                        for (int kk = 0; kk < kBK / 16; ++kk) {
+                            tc_mma_bf16_ts_acc(d_tmem, ta_hi + 32 + kk * 8, desc_bf(bf_lo16 + kk * 2), idesc_bf);
+                            tc_mma_bf16_ts_acc(d_tmem, ta_hi + 48 + kk * 8, desc_bf(bf_hi16 + kk * 2), idesc_bf);
+                        }
+                    } else
 #pragma unroll
                     for (int kk = 0; kk < kBK / 8; ++kk) {
                         const uint64_t db_hi = desc_at(hi_b16 + kk * k_step16);
@@ -894,6 +952,17 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                     }
                     const uint32_t taddr = tmem_base + ((q * 32u) << 16) + 2 * kBN + ls * kTmemColsA + 16 * h;
                     tc_st_32x16(taddr, h16);
+                    if (kBf) {
+                        uint32_t hb[8], lb[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            hb[j] = pack_bf16(__uint_as_float(h16[2 * j]), __uint_as_float(h16[2 * j + 1]));
+                            lb[j] = pack_bf16(__uint_as_float(l16[2 * j]), __uint_as_float(l16[2 * j + 1]));
+                        }
+                        const uint32_t tb = taddr - 16 * h + 32 + 8 * h;
+                        tc_st_32x8(tb, hb);
+                        tc_st_32x8(tb + 16, lb);
+                    } else
                     tc_st_32x16(taddr + 32, l16);
                 }
                 if (kSplit) {                     // the raw A tile has been read: its slot may be refilled
@@ -901,6 +970,45 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                     if (lane == 0) mbar_arrive(smem_u32(&a_empty[sa]));
                 }
             }
+            if (kBf) {
+                // B tile: a thread takes pairs of adjacent 16-byte chunks (8 consecutive k of one row: the 128-byte
+                // swizzle permutes the two chunks of a pair only among themselves).  hi goes back in place as tf32;
+                // hi and lo as bf16 make one 16-byte chunk each, and under the 64-byte swizzle that chunk's place in
+                // its tile is the pair's place in the raw tile.  Half of each quarter-warp reads the second chunk of
+                // its pair first, which keeps the 16-byte accesses free of bank conflicts.
+                uint8_t *braw = hi + kRawBytesA, *bf_hi = lo + kRawBytesA, *bf_lo = bf_hi + kRawBytesB / 2;
+                const uint32_t s1 = (lane >> 2) & 1u;
+#pragma unroll
+                for (int u = 0; u < (int)(kRawBytesB / 32) / kTT; ++u) {
+                    const uint32_t p = (uint32_t)tt + (uint32_t)u * kTT;          // pair index = 4 * row + pair of the row
+                    const uint32_t offx = 32 * p + 16 * s1, offy = 32 * p + 16 * (s1 ^ 1u);
+                    const float4 x4 = *reinterpret_cast<const float4 *>(braw + offx);
+                    const float4 y4 = *reinterpret_cast<const float4 *>(braw + offy);
+                    const float ex[8] = {x4.x, x4.y, x4.z, x4.w, y4.x, y4.y, y4.z, y4.w};
+                    uint32_t h[8];
+                    float l[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const float sq = __fmul_rn(ex[j], ex[j]);
+                        h[j] = to_tf32(sq);
+                        l[j] = __fsub_rn(sq, __uint_as_float(h[j]));
+                    }
+                    *reinterpret_cast<uint4 *>(braw + offx) = make_uint4(h[0], h[1], h[2], h[3]);
+                    *reinterpret_cast<uint4 *>(braw + offy) = make_uint4(h[4], h[5], h[6], h[7]);
+                    const uint32_t hx0 = pack_bf16(__uint_as_float(h[0]), __uint_as_float(h[1]));
+                    const uint32_t hx1 = pack_bf16(__uint_as_float(h[2]), __uint_as_float(h[3]));
+                    const uint32_t hy0 = pack_bf16(__uint_as_float(h[4]), __uint_as_float(h[5]));
+                    const uint32_t hy1 = pack_bf16(__uint_as_float(h[6]), __uint_as_float(h[7]));
+                    const uint32_t lx0 = pack_bf16(l[0], l[1]), lx1 = pack_bf16(l[2], l[3]);
+                    const uint32_t ly0 = pack_bf16(l[4], l[5]), ly1 = pack_bf16(l[6], l[7]);
+                    // the chunk read first holds the lower k iff its place in the pair equals the row's parity
+                    const bool x_first = s1 == ((p >> 2) & 1u);
+                    *reinterpret_cast<uint4 *>(bf_hi + 16 * p) =
+                        x_first ? make_uint4(hx0, hx1, hy0, hy1) : make_uint4(hy0, hy1, hx0, hx1);
+                    *reinterpret_cast<uint4 *>(bf_lo + 16 * p) =
+                        x_first ? make_uint4(lx0, lx1, ly0, ly1) : make_uint4(ly0, ly1, lx0, lx1);
+                }
+            } else
             if (kAnyTma) {      // tiles that came by TMA: elementwise, in place, over their 16-byte chunks
                 constexpr uint32_t c_begin = (kGatherA || kATmem) ? kRawBytesA / 16 : 0;
                 constexpr uint32_t c_end = kGatherB ? kRawBytesA / 16 : kRawStageBytes / 16;
@@ -1329,6 +1437,13 @@ struct ExactScope {
 };
 
 // Cout <= 64: the im2col rows take the 128-row A tile and the errors the narrow B tile
+// cross terms of the TMA-fed form with bf16 operands unless VGC_TC_BF16=0
+static bool bf_cross()
+{
+    const char *e = getenv("VGC_TC_BF16");
+    return !(e && atoi(e) == 0);
+}
+
 static bool conv_swapped(int Cout, int n_im2col) { return Cout <= 64 && n_im2col > Cout; }
 
 // ---- repacking pre-pass for 1x1 convolutions whose tiles TMA cannot address in place ----------
@@ -1601,6 +1716,7 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
         if (taps) fn = taps == 4 ? VGC_TC_FN(kTma, kGatherTaps4, true) : VGC_TC_FN(kTma, kGatherTaps2, true);
         else if (taps_s2) fn = taps_s2 == 4 ? VGC_TC_FN(kTma, kGatherTaps4S2, true) : VGC_TC_FN(kTma, kGatherTaps2S2, true);
         else if (taps7) fn = VGC_TC_FN(kTma, kGatherTaps7S2, true);
+        else if (e == kTma && i == kTma && bf_cross() && !ex) fn = sqgrad_tc<kMajorK, kTma, kTma, true, false, true>;
         else if (e == kTma && i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kTma, true) : sqgrad_tc<kMajorK, kTma, kTma, false>;
         else if (e == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kGatherIm2col, true) : sqgrad_tc<kMajorK, kTma, kGatherIm2col, false>;
         else if (i == kTma) fn = VGC_TC_FN(kGatherErr, kTma, false);
@@ -1608,7 +1724,8 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
         return tc_launch(fn, bt, n_layers, prm, Cout, n_im2col, k_slices, ws, ws_bytes, st, unit);
     }
     prm.ld_m = 1; prm.ld_n = n_im2col;   // m = idx, n = o
-    if (e == kTma && i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kTma, true) : sqgrad_tc<kMajorK, kTma, kTma, false>;
+    if (e == kTma && i == kTma && bf_cross() && !ex) fn = sqgrad_tc<kMajorK, kTma, kTma, true, false, true>;
+    else if (e == kTma && i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kTma, true) : sqgrad_tc<kMajorK, kTma, kTma, false>;
     else if (i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kGatherErr, true) : sqgrad_tc<kMajorK, kTma, kGatherErr, false>;
     else if (e == kTma) fn = VGC_TC_FN(kGatherIm2col, kTma, false);
     else fn = VGC_TC_FN(kGatherIm2col, kGatherErr, false);

@@ -147,7 +147,7 @@ def test_repacked_and_in_place_forms_agree_with_the_oracle(monkeypatch, B, C, H,
 
 
 @pytest.mark.parametrize("env", [{"VGC_TC_ATMEM": "0"}, {"VGC_TC_GATHER": "1"}, {"VGC_TC_GATHER": "2"},
-                                 {"VGC_TC_GATHER": "3"}, {"VGC_SQGRAD_PATH": "simt"}, {"VGC_TC_TAPS": "0"}])
+                                 {"VGC_TC_GATHER": "3"}, {"VGC_SQGRAD_PATH": "simt"}, {"VGC_TC_TAPS": "0"}, {"VGC_TC_BF16": "0"}])
 @pytest.mark.parametrize("B,C,H,Cout,k,s,p", [(3, 96, 12, 160, 1, 1, 0), (2, 40, 12, 48, 3, 1, 1), (2, 72, 16, 200, 3, 2, 1)])
 def test_every_kernel_variant_gives_the_same_statistic(monkeypatch, env, B, C, H, Cout, k, s, p):
     """The library picks a kernel form per layer (TMA or gathered tiles, A operand in shared or tensor memory,
@@ -161,6 +161,20 @@ def test_every_kernel_variant_gives_the_same_statistic(monkeypatch, env, B, C, H
     d = torch.randn(B, Cout, Ho, Ho, device="cuda", generator=gen) * 1e-4
     got = run_conv(x, d, k, s, p, 0.5)
     want = oracle.sqgrad_conv(x.cpu().numpy(), d.cpu().numpy(), (k, k), (s, s), (p, p), scale=0.5)
+    _check(got, want)
+
+
+@pytest.mark.parametrize("bf16_cross", ["1", "0"])
+@pytest.mark.parametrize("xv,dv", [(1.2345678, 0.0031415926), (1.7320508, 0.0027182818), (0.99999994, 1.0000001)])
+def test_constant_inputs_rounding_errors_all_of_one_sign(monkeypatch, bf16_cross, xv, dv):
+    """Every product has the same rounding error when all inputs are equal, so nothing averages out: the error of
+    the split operands (and of the bf16 cross terms) shows at its full size and must still be inside the tolerance."""
+    monkeypatch.setenv("VGC_TC_BF16", bf16_cross)
+    B, C, H, Cout = 8, 128, 28, 256
+    x = torch.full((B, C, H, H), xv, device="cuda"); d = torch.full((B, Cout, H, H), dv, device="cuda")
+    got = run_conv(x, d, 1, 1, 0, 1.0 / B)
+    x2 = float(np.float32(xv)) ** 2; d2 = float(np.float32(dv)) ** 2        # exact squares of the fp32 inputs
+    want = np.full((Cout, C, 1, 1), (1.0 / B) * B * H * H * x2 * d2)
     _check(got, want)
 
 
