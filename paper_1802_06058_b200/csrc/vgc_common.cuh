@@ -4,6 +4,9 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <cstdio>
+#include <cstdlib>
+
 #include "vgc.h"
 
 #ifndef __CUDA_ARCH__
@@ -18,9 +21,18 @@ inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-#define VGC_CUDA_OK(expr)                          \
-    do {                                           \
-        if ((expr) != cudaSuccess) return VGC_ERR_CUDA; \
+// VGC_DEBUG=1 in the environment: a failing CUDA call is named on stderr before the status is returned
+inline void report_cuda_error(cudaError_t e, const char *what, const char *file, int line)
+{
+    if (getenv("VGC_DEBUG")) fprintf(stderr, "vgc: %s:%d: %s -> %s\n", file, line, what, cudaGetErrorString(e));
+}
+#define VGC_CUDA_OK(expr)                                                  \
+    do {                                                                   \
+        const cudaError_t vgc_e_ = (expr);                                 \
+        if (vgc_e_ != cudaSuccess) {                                       \
+            ::vgc::report_cuda_error(vgc_e_, #expr, __FILE__, __LINE__);   \
+            return VGC_ERR_CUDA;                                           \
+        }                                                                  \
     } while (0)
 
 // Number of kernels this library has enqueued since it was loaded (benchmark bookkeeping).

@@ -75,6 +75,11 @@ constexpr int kLoSlotsAT = 2 * kLoSlots;
 // early, and the 16-KB units this saves hold more B tiles: more slices in flight from the same shared memory.
 constexpr int kSplitA = 4, kSplitB = 7, kSplitLo = 3;              // 16-KB units: A raw, B raw/hi, B lo (+ A in TMEM)
 static_assert((kSplitA + kSplitB + kSplitLo) * kRawBytesA <= (kRawSlots + kLoSlots) * kRawStageBytes, "smem budget");
+// Pair form (two CTAs of a cluster share one 256 x 128 tile, tcgen05 cta_group::2): each CTA holds its own 128 A rows
+// and half of the B rows, so a B slot is 8 KB and the rings get deeper: A raw, B raw/hi, B bf16 (+ A in TMEM)
+constexpr int kPairA = 5, kPairB = 10, kPairLo = 4;
+constexpr uint32_t kPairBBytes = kRawBytesB / 2;
+static_assert(kPairA * kRawBytesA + (kPairB + kPairLo) * kPairBBytes <= (kRawSlots + kLoSlots) * kRawStageBytes, "smem budget");
 constexpr uint32_t kTmemColsA = 64;                                 // per slot: 32 columns hi + 32 columns lo
 constexpr uint32_t kTmemCols = 512;                                 // two accumulator buffers + the A operand ring
 constexpr uint32_t kWaitLimit = 1u << 22;                           // polls before a wait gives up
@@ -182,6 +187,63 @@ __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// ---- cluster of two CTAs (pair form) ----
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// arrive on the barrier at the same shared-memory offset in CTA `rank` of the cluster.  No cluster-scope release: what
+// the arrival publishes is read by the tensor core of the writing CTA (its shared memory after fence.proxy.async, its
+// tensor memory after tcgen05.wait::st), not by the other CTA's threads, and a cluster-wide release costs a full
+// memory barrier per arrival (measured: the pair form then runs 1.4x slower than single CTAs).
+__device__ __forceinline__ void mbar_arrive_cta(uint32_t bar, uint32_t rank)
+{
+    asm volatile(
+        "{\n\t.reg .b32 rem;\n\t"
+        "mapa.shared::cluster.u32 rem, %0, %1;\n\t"
+        "mbarrier.arrive.shared::cluster.b64 _, [rem];\n\t}"
+        ::"r"(bar), "r"(rank)
+        : "memory");
+}
+// commit of cta_group::2 MMAs: arrives on the barrier at this offset in both CTAs of the pair
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair_local(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// cta_group::2, A from tensor memory: D (256 rows over the two CTAs) (+)= A * B, B rows split between the CTAs
+__device__ __forceinline__ void tc_mma_pair_tf32_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                                    uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair_bf16_ts_acc(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.eq.u32 p, 1, 1;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc)
+        : "memory");
+}
+
 __device__ __forceinline__ void tc_mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                             uint32_t accumulate)
 {
@@ -293,16 +355,16 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 }
 
 // Instruction descriptor: D fp32, A and B tf32, given major-ness, M = 128, N = n (multiple of 16).
-__host__ __device__ constexpr uint32_t instr_desc(int major, int n)
+__host__ __device__ constexpr uint32_t instr_desc(int major, int n, int m = kBM)
 {
     return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)major << 15) | ((uint32_t)major << 16) |
-           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // The same for bf16 operands (both K-major), used for the two cross terms of the bf16-cross form.
-__host__ __device__ constexpr uint32_t instr_desc_bf16(int n)
+__host__ __device__ constexpr uint32_t instr_desc_bf16(int n, int m = kBM)
 {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // One 16-byte chunk (4 consecutive k of one row) of a K-major 128-byte-swizzled tile.
@@ -651,7 +713,12 @@ struct Gatherer<kMode, kHalf, true> {
 // tensor-pipe time of a tf32 product each; their rounding, 2^-9 relative on a term that is itself 2^-11 of the
 // product, stays below 2^-18 of the result).  A lo slot then holds [B hi as bf16][B lo as bf16], 8 KB each with
 // 64-byte rows, and an A slot in tensor memory [hi tf32: 32 columns][hi bf16: 16][lo bf16: 16].
-template <int kMajor, int kModeA, int kModeB, bool kATmem, bool kExact = false, bool kBf = false>
+// kPair: two CTAs of a cluster (neighbours along the grid's x, which holds the row tiles in this form) work on one 256 x 128 tile with cta_group::2 MMAs.
+// Each keeps its own 128 rows of A (tensor memory) and of the accumulators and loads / transforms only half of
+// the B rows, which halves the B share of the shared-memory traffic.  The even CTA issues the MMAs; the transform and
+// epilogue warps of the odd one signal its barriers through the cluster's shared-memory window, and a commit
+// arrives on the barriers of both.
+template <int kMajor, int kModeA, int kModeB, bool kATmem, bool kExact = false, bool kBf = false, bool kPair = false>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
 {
@@ -662,11 +729,13 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
     constexpr bool kAnyGather = kGatherA || kGatherB;
     constexpr bool kSplit = kATmem && !kAnyGather;                         // A raw tiles in a ring of their own
     static_assert(!kBf || (kSplit && !kExact), "bf16 cross terms: the TMA-fed form with A in tensor memory");
+    static_assert(!kPair || kBf, "the pair form exists for the TMA-fed form with bf16 cross terms");
+    constexpr int kNA = kPair ? kPairA : kSplitA;                          // slots of the raw A ring (split form)
     // the transform warps work as two groups of four on alternate slices (else all eight on every slice)
     constexpr bool kTwoGroups = !kAnyGather || (IsTaps<kModeB>::value && kModeA == kTma);
-    constexpr int kNB = kSplit ? kSplitB : kRawSlots;                      // slots of the raw / hi ring
+    constexpr int kNB = kPair ? kPairB : kSplit ? kSplitB : kRawSlots;     // slots of the raw / hi ring
     // lo slots (and A slots in TMEM); the per-example form needs 128 TMEM columns for its sum of squares
-    constexpr int kLoN = (kExact && kATmem) ? 2 : kSplit ? kSplitLo : (kATmem ? kLoSlotsAT : kLoSlots);
+    constexpr int kLoN = kPair ? kPairLo : (kExact && kATmem) ? 2 : kSplit ? kSplitLo : (kATmem ? kLoSlotsAT : kLoSlots);
     constexpr uint32_t kSqCol = 2 * kBN + (kATmem ? 2 * kTmemColsA : 0);         // where that sum lives
     constexpr uint32_t kLoBytes = kATmem ? kRawBytesB : kRawStageBytes;  // bytes of one lo slot
     // byte offsets of slot s: the [A][B] pair of the raw / hi ring (split form: only its B half exists, the
@@ -677,8 +746,17 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                       : kLoBase + (uint32_t)s * kLoBytes - (kATmem ? kRawBytesA : 0u);
     };
 
+    // bf16-cross form: where the B tile of raw slot s and the [hi bf16][lo bf16] tiles of lo slot s live
+    auto b_tile = [&](int s) -> uint32_t {
+        return kPair ? (uint32_t)kPairA * kRawBytesA + (uint32_t)s * kPairBBytes : pair_off(s) + kRawBytesA;
+    };
+    auto bf_tile = [&](int s) -> uint32_t {
+        return kPair ? (uint32_t)kPairA * kRawBytesA + (uint32_t)(kPairB + s) * kPairBBytes : lo_off(s) + kRawBytesA;
+    };
+    constexpr uint32_t kBTile = kPair ? kPairBBytes : kRawBytesB;          // bytes of this CTA's B tile
+
     extern __shared__ uint8_t smem_raw_[];
-    __shared__ __align__(8) uint64_t bars[3 * kSplitB + kLoSlotsAT + 5 + 2 * kSplitA];
+    __shared__ __align__(8) uint64_t bars[3 * kPairB + kLoSlotsAT + 5 + 2 * kPairA];
     __shared__ uint32_t tmem_base_slot;
     __shared__ volatile uint32_t abort_flag;
 
@@ -692,11 +770,17 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
     uint64_t *raw_full = bars, *op_full = bars + kNB, *empty = bars + 2 * kNB;
     uint64_t *lo_empty = bars + 3 * kNB;
     uint64_t *acc_full = lo_empty + kLoSlotsAT, *acc_empty = acc_full + 2, *drain = acc_empty + 2;
-    uint64_t *a_full = drain + 1, *a_empty = a_full + kSplitA;             // split form: the A ring
+    uint64_t *a_full = drain + 1, *a_empty = a_full + kNA;                 // split form: the A ring
+    // pair form: rank of this CTA in its cluster; rank 0 issues the MMAs and owns the barriers that both CTAs signal
+    const uint32_t cta_rank = kPair ? cluster_ctarank() : 0u;
 
-    const int m0 = blockIdx.y * kBM, n0 = blockIdx.x * kBN;
+    // tile coordinates: columns along the grid's x, rows along y; the pair form has them the other way round because
+    // the two CTAs of a pair, neighbours in rows, must be neighbours along x
+    const int tile_n = kPair ? (int)blockIdx.y : (int)blockIdx.x, tile_m = kPair ? (int)blockIdx.x : (int)blockIdx.y;
+    const int tiles_n = kPair ? (int)gridDim.y : (int)gridDim.x;
+    const int m0 = tile_m * kBM, n0 = tile_n * kBN;
     const int n_valid = min(kBN, prm.N - n0);                              // columns of this tile that exist
-    const int n_act = (n_valid + 15) & ~15;                                // UMMA N (multiple of 16)
+    const int n_act = kPair ? (n_valid + 31) & ~31 : (n_valid + 15) & ~15; // UMMA N (multiple of 16; of 32 for a pair)
     const int layer = (int)blockIdx.z / prm.splits, split = (int)blockIdx.z - layer * prm.splits;
     const CUtensorMap *map_a = &bt.a[layer], *map_b = &bt.b[layer];
     float *const S = bt.S[layer];
@@ -713,27 +797,35 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         abort_flag = 0;
         for (int i = 0; i < kNB; ++i) {
             mbar_init(smem_u32(&raw_full[i]), 1);
-            mbar_init(smem_u32(&op_full[i]), kTwoGroups ? kTransformWarps / 2 : kTransformWarps);
+            mbar_init(smem_u32(&op_full[i]), (kPair ? 2 : 1) * (kTwoGroups ? kTransformWarps / 2 : kTransformWarps));
             mbar_init(smem_u32(&empty[i]), 1);
         }
         if (kSplit)
-            for (int i = 0; i < kSplitA; ++i) {
+            for (int i = 0; i < kNA; ++i) {
                 mbar_init(smem_u32(&a_full[i]), 1);
                 mbar_init(smem_u32(&a_empty[i]), kTransformWarps / 2);
             }
         for (int i = 0; i < kLoSlotsAT; ++i) mbar_init(smem_u32(&lo_empty[i]), 1);      // unused, kept initialised
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&acc_full[i]), 1); mbar_init(smem_u32(&acc_empty[i]), kEpilogueWarps); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&acc_full[i]), 1); mbar_init(smem_u32(&acc_empty[i]), (kPair ? 2 : 1) * kEpilogueWarps); }
         mbar_init(smem_u32(drain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {      // TMEM: this warp allocates and, at the end, frees
+        if (kPair) {       // the same warp of both CTAs allocates for the pair
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                         "r"(kTmemCols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
                      "r"(kTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (kPair) cluster_sync_all();      // the other CTA's barriers are initialised before anything arrives on them
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
@@ -749,14 +841,16 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                 const uint32_t dst_a = smem_base + pair_off(st), dst_b = dst_a + kRawBytesA;
                 const int slice = slice_begin + i;
                 if (kSplit) {
-                    const int sa = i % kSplitA;
-                    if (!mbar_wait(smem_u32(&a_empty[sa]), ((uint32_t)(i / kSplitA) & 1u) ^ 1u, &abort_flag, 64)) break;
+                    const int sa = i % kNA;
+                    if (!mbar_wait(smem_u32(&a_empty[sa]), ((uint32_t)(i / kNA) & 1u) ^ 1u, &abort_flag, 64)) break;
                     const uint32_t full_a = smem_u32(&a_full[sa]);
                     const int z = slice / prm.p_slices, p0 = (slice - z * prm.p_slices) * kBK;
                     mbar_expect_tx(full_a, prm.tx_bytes_a);
                     tma_load_3d(smem_base + (uint32_t)sa * kRawBytesA, map_a, full_a, p0, m0, z);
                     mbar_expect_tx(full, prm.tx_bytes - prm.tx_bytes_a);
-                    tma_load_3d(dst_b, map_b, full, p0, n0, z);
+                    // pair form: this CTA's half of the tile's B rows
+                    if (kBf) tma_load_3d(smem_base + b_tile(st), map_b, full, p0, n0 + (kPair ? (int)cta_rank * (n_act >> 1) : 0), z);
+                    else tma_load_3d(dst_b, map_b, full, p0, n0, z);
                     issued = i + 1;
                     continue;
                 }
@@ -783,10 +877,10 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                     for (uint32_t t = 0; t < kWaitLimit && !mbar_try(bar, ph); ++t) {}
                 }
                 if (kSplit) {
-                    const int first_a = issued > kSplitA ? issued - kSplitA : 0;
+                    const int first_a = issued > kNA ? issued - kNA : 0;
                     for (int i = first_a; i < issued; ++i) {
-                        const uint32_t bar = smem_u32(&a_full[i % kSplitA]);
-                        const uint32_t ph = (uint32_t)(i / kSplitA) & 1u;
+                        const uint32_t bar = smem_u32(&a_full[i % kNA]);
+                        const uint32_t ph = (uint32_t)(i / kNA) & 1u;
                         for (uint32_t t = 0; t < kWaitLimit && !mbar_try(bar, ph); ++t) {}
                     }
                 }
@@ -794,8 +888,8 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         }
     } else if (warp == 1) {
         // ================= MMA issuer (one thread) =================
-        if (lane == 0) {
-            const uint32_t idesc = instr_desc(kMajor, n_act);
+        if (lane == 0 && cta_rank == 0) {
+            const uint32_t idesc = instr_desc(kMajor, n_act, kPair ? 2 * kBM : kBM);
             // K-major: rows of 128 B, 8-row groups 1024 B apart (SBO); LBO unused.
             // MN-major: 32-wide column blocks 4096 B apart (LBO); 4-deep k groups 512 B apart (SBO).
             const uint32_t lbo = kMajor == kMajorK ? 16u : 4096u;
@@ -809,7 +903,7 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
             const uint32_t desc_lo0 = (uint32_t)smem_desc(0, lbo, sbo, layout);
             auto desc_at = [&](uint32_t lo16) -> uint64_t { return ((uint64_t)desc_hi << 32) | (desc_lo0 + lo16); };
             // bf16 tiles: K-major rows of 64 B with the 64-byte swizzle (mode 4), 8-row groups 512 B apart
-            const uint32_t idesc_bf = instr_desc_bf16(n_act);
+            const uint32_t idesc_bf = instr_desc_bf16(n_act, kPair ? 2 * kBM : kBM);
             const uint32_t desc_bf_hi = (uint32_t)(smem_desc(0, 16u, 512u, 4u) >> 32);
             const uint32_t desc_bf_lo0 = (uint32_t)smem_desc(0, 16u, 512u, 4u);
             auto desc_bf = [&](uint32_t lo16) -> uint64_t { return ((uint64_t)desc_bf_hi << 32) | (desc_bf_lo0 + lo16); };
@@ -832,18 +926,25 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                     const uint32_t lo_a16 = (smem_base + lo_off(ls)) >> 4, lo_b16 = lo_a16 + (kRawBytesA >> 4);   // lo_a unused with A in TMEM
                     const uint32_t ta_hi = tmem_base + 2 * kBN + ls * kTmemColsA, ta_lo = ta_hi + 32;
                     if (kBf) {
+                        const uint32_t b16 = (smem_base + b_tile(st)) >> 4;
 #pragma unroll
                         for (int kk = 0; kk < kBK / 8; ++kk) {
-                            const uint64_t db_hi = desc_at(hi_b16 + kk * k_step16);
-                            if (kk == 0) tc_mma_tf32_ts(d_tmem, ta_hi, db_hi, idesc, first ? 0u : 1u);
+                            const uint64_t db_hi = desc_at(b16 + kk * k_step16);
+                            if (kPair) tc_mma_pair_tf32_ts(d_tmem, ta_hi + kk * 8, db_hi, idesc, (kk == 0 && first) ? 0u : 1u);
+                            else if (kk == 0) tc_mma_tf32_ts(d_tmem, ta_hi, db_hi, idesc, first ? 0u : 1u);
                             else tc_mma_tf32_ts_acc(d_tmem, ta_hi + kk * 8, db_hi, idesc);
                         }
                         // cross terms, 16 k (32 bytes of a 64-byte row, 8 columns of tensor memory) per instruction
-                        const uint32_t bf_hi16 = lo_b16, bf_lo16 = lo_b16 + (kRawBytesB >> 5);
+                        const uint32_t bf_hi16 = (smem_base + bf_tile(ls)) >> 4, bf_lo16 = bf_hi16 + (kBTile >> 5);
 #pragma unroll
                         for (int kk = 0; kk < kBK / 16; ++kk) {
-                            tc_mma_bf16_ts_acc(d_tmem, ta_hi + 32 + kk * 8, desc_bf(bf_lo16 + kk * 2), idesc_bf);
-                            tc_mma_bf16_ts_acc(d_tmem, ta_hi + 48 + kk * 8, desc_bf(bf_hi16 + kk * 2), idesc_bf);
+                            if (kPair) {
+                                tc_mma_pair_bf16_ts_acc(d_tmem, ta_hi + 32 + kk * 8, desc_bf(bf_lo16 + kk * 2), idesc_bf);
+                                tc_mma_pair_bf16_ts_acc(d_tmem, ta_hi + 48 + kk * 8, desc_bf(bf_hi16 + kk * 2), idesc_bf);
+                            } else {
+                                tc_mma_bf16_ts_acc(d_tmem, ta_hi + 32 + kk * 8, desc_bf(bf_lo16 + kk * 2), idesc_bf);
+                                tc_mma_bf16_ts_acc(d_tmem, ta_hi + 48 + kk * 8, desc_bf(bf_hi16 + kk * 2), idesc_bf);
+                            }
                         }
                     } else
 #pragma unroll
@@ -865,13 +966,16 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                         }
                     }
                     first = false;
+                    if (kPair) tc_commit_pair(smem_u32(&empty[st]));      // in both CTAs
+                    else
                     tc_commit(smem_u32(&empty[st]));              // raw, lo and TMEM-A slots are free once these MMAs retire
                     if (++st == kNB) { st = 0; st_phase ^= 1u; }
                     if (++ls == kLoN) ls = 0;
                 }
-                if (ok) tc_commit(smem_u32(&acc_full[b]));
+                if (ok) { if (kPair) tc_commit_pair(smem_u32(&acc_full[b])); else tc_commit(smem_u32(&acc_full[b])); }
             }
             if (!ok) {      // abort: MMAs already issued must retire before TMEM is freed
+                if (kPair) tc_commit_pair_local(smem_u32(drain)); else
                 tc_commit(smem_u32(drain));
                 for (uint32_t t = 0; t < kWaitLimit && !mbar_try(smem_u32(drain), 0); ++t) {}
             }
@@ -910,8 +1014,8 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         auto process = [&](int i, const RegsA &ga, const RegsB &gb) -> bool {
             const int st = i % kNB, ls = i % kLoN;
             const uint32_t ph = (uint32_t)(i / kNB) & 1u;
-            const int sa = kSplit ? i % kSplitA : 0;
-            if (kSplit && !mbar_wait(smem_u32(&a_full[sa]), (uint32_t)(i / kSplitA) & 1u, &abort_flag)) return false;
+            const int sa = kSplit ? i % kNA : 0;
+            if (kSplit && !mbar_wait(smem_u32(&a_full[sa]), (uint32_t)(i / kNA) & 1u, &abort_flag)) return false;
             // a raw slot is ours once its TMA tiles landed (the producer waited for it to be empty), or, with
             // nothing coming by TMA, once the MMAs that last read it retired; likewise the lo slot
             if (kAnyTma ? !mbar_wait(smem_u32(&raw_full[st]), ph, &abort_flag)
@@ -976,10 +1080,10 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                 // hi and lo as bf16 make one 16-byte chunk each, and under the 64-byte swizzle that chunk's place in
                 // its tile is the pair's place in the raw tile.  Half of each quarter-warp reads the second chunk of
                 // its pair first, which keeps the 16-byte accesses free of bank conflicts.
-                uint8_t *braw = hi + kRawBytesA, *bf_hi = lo + kRawBytesA, *bf_lo = bf_hi + kRawBytesB / 2;
+                uint8_t *braw = smem_gen + b_tile(st), *bf_hi = smem_gen + bf_tile(ls), *bf_lo = bf_hi + kBTile / 2;
                 const uint32_t s1 = (lane >> 2) & 1u;
 #pragma unroll
-                for (int u = 0; u < (int)(kRawBytesB / 32) / kTT; ++u) {
+                for (int u = 0; u < (int)(kBTile / 32) / kTT; ++u) {
                     const uint32_t p = (uint32_t)tt + (uint32_t)u * kTT;          // pair index = 4 * row + pair of the row
                     const uint32_t offx = 32 * p + 16 * s1, offy = 32 * p + 16 * (s1 ^ 1u);
                     const float4 x4 = *reinterpret_cast<const float4 *>(braw + offx);
@@ -1032,7 +1136,10 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
             if (kATmem) { tc_wait_st(); tc_fence_before(); }      // TMEM stores complete and ordered before the signal
             fence_async_smem();                                   // generic-proxy writes -> tensor core reads
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&op_full[st]));
+            if (lane == 0) {
+                if (kPair) mbar_arrive_cta(smem_u32(&op_full[st]), 0);     // the issuing CTA's barrier
+                else mbar_arrive(smem_u32(&op_full[st]));
+            }
             return true;
         };
 
@@ -1097,7 +1204,10 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&acc_empty[b]));
+            if (lane == 0) {
+                if (kPair) mbar_arrive_cta(smem_u32(&acc_empty[b]), 0);
+                else mbar_arrive(smem_u32(&acc_empty[b]));
+            }
             if (kExact && (c + 1) % cps == 0) {
                 // end of an example: acc holds its sum over positions; add the squares to the running sum in TMEM
 #pragma unroll
@@ -1136,7 +1246,7 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
             const int m = m0 + r_local;
             if (prm.splits > 1) {
                 // split-K scratch, column-major inside the tile: consecutive lanes -> consecutive addresses
-                const size_t tile = (size_t)blockIdx.z * (gridDim.x * gridDim.y) + (size_t)blockIdx.y * gridDim.x + blockIdx.x;
+                const size_t tile = (size_t)blockIdx.z * (gridDim.x * gridDim.y) + (size_t)tile_m * tiles_n + tile_n;
                 float *dst = prm.partial + tile * (kBM * kBN) + r_local;
 #pragma unroll
                 for (int j = 0; j < kBN; ++j)
@@ -1199,8 +1309,13 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
     // ---- common exit ----
     tc_fence_before();
     __syncthreads();
+    // pair form: the other CTA's tensor memory and shared memory are operands of this pair's MMAs and its barriers
+    // receive this CTA's arrivals, so neither CTA frees anything or leaves before both are done
+    if (kPair) cluster_sync_all();
     if (warp == 1) {
         tc_fence_after();
+        if (kPair) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        else
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
     if (threadIdx.x == 0 && abort_flag) atomicOr(prm.status, VGC_DEV_TIMEOUT);
@@ -1285,9 +1400,11 @@ static bool make_map(CUtensorMap *map, const float *base, int rank, const cuuint
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint32_t elem_strides[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<float *>(base), dims, strides_bytes, box,
-              elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    const CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<float *>(base), dims,
+                           strides_bytes, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (rc != CUDA_SUCCESS && getenv("VGC_DEBUG")) fprintf(stderr, "vgc: tensor map encode failed with CUresult %d\n", (int)rc);
+    return rc == CUDA_SUCCESS;
 }
 
 static int default_chunk()
@@ -1377,7 +1494,7 @@ static size_t tc_workspace_bytes(int M, int N, int k_slices, int n_layers = 1, i
 typedef void (*KernelFn)(const Batch, const Params);
 
 static vgc_status tc_launch(KernelFn kernel, const Batch &bt, int n_layers, Params prm, int M, int N,
-                            int k_slices, void *ws, size_t ws_bytes, cudaStream_t st, int unit = 1)
+                            int k_slices, void *ws, size_t ws_bytes, cudaStream_t st, int unit = 1, bool pair = false)
 {
     const Plan plan = make_plan(M, N, k_slices, n_layers, unit);
     if (ws_bytes < tc_workspace_bytes(M, N, k_slices, n_layers, unit)) return VGC_ERR_WORKSPACE;
@@ -1395,7 +1512,25 @@ static vgc_status tc_launch(KernelFn kernel, const Batch &bt, int n_layers, Para
     prm.status = static_cast<uint32_t *>(ws);
     prm.partial = reinterpret_cast<float *>(static_cast<char *>(ws) + 256);
     dim3 grid(plan.tiles_x, plan.tiles_y, plan.splits * n_layers);
-    kernel<<<grid, kThreadsTc, kSmemBytes, st>>>(bt, prm);
+    if (pair) {
+        // clusters of two CTAs, neighbours along x, which holds the row tiles in this form (the caller made sure
+        // their number is even)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid.y, grid.x, grid.z); cfg.blockDim = dim3(kThreadsTc); cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        if (getenv("VGC_DEBUG")) {
+            int n_clusters = -1;
+            const cudaError_t oe = cudaOccupancyMaxActiveClusters(&n_clusters, kernel, &cfg);
+            fprintf(stderr, "vgc: pair launch grid (%u, %u, %u), smem %u: max active clusters %d (%s)\n", grid.x, grid.y,
+                    grid.z, (unsigned)kSmemBytes, n_clusters, cudaGetErrorString(oe));
+        }
+        VGC_CUDA_OK(cudaLaunchKernelEx(&cfg, kernel, bt, prm));
+    } else {
+        kernel<<<grid, kThreadsTc, kSmemBytes, st>>>(bt, prm);
+    }
     count_launch();
     if (plan.splits > 1) {
         ResultPtrs results = {};
@@ -1405,7 +1540,8 @@ static vgc_status tc_launch(KernelFn kernel, const Batch &bt, int n_layers, Para
             prm.ld_n);
         count_launch();
     }
-    return cudaGetLastError() == cudaSuccess ? VGC_OK : VGC_ERR_CUDA;
+    VGC_CUDA_OK(cudaGetLastError());
+    return VGC_OK;
 }
 
 size_t tc_linear_workspace_bytes(int B, int in, int out) { return tc_workspace_bytes(out, in, (B + kBK - 1) / kBK); }
@@ -1443,6 +1579,13 @@ static bool bf_cross()
     const char *e = getenv("VGC_TC_BF16");
     return !(e && atoi(e) == 0);
 }
+// the TMA-fed form on pairs of CTAs (256 x 128 tiles) where the number of row tiles allows: VGC_TC_PAIR=1
+static bool pair_form()
+{
+    const char *e = getenv("VGC_TC_PAIR");
+    return e && atoi(e) != 0;
+}
+static bool even_row_tiles(int M) { return ((M + kBM - 1) / kBM) % 2 == 0; }
 
 static bool conv_swapped(int Cout, int n_im2col) { return Cout <= 64 && n_im2col > Cout; }
 
@@ -1677,8 +1820,17 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
                        W == 2 * Wo && Wo % 4 == 0 && a_tmem;
     // with few output channels the roles are swapped -- except in the three-tap form, where keeping the errors as
     // the A operand (in tensor memory, half of its rows unused) measures faster than both operands in shared memory
-    const bool swapped = conv_swapped(Cout, n_im2col) && !taps && !taps_s2 && !taps7;
-    const int rows_err = swapped ? kBN : kBM, rows_in = swapped ? kBM : kBN;     // tile heights
+    bool swapped = conv_swapped(Cout, n_im2col) && !taps && !taps_s2 && !taps7;
+    // both tiles by TMA, A in tensor memory, cross terms in bf16; on pairs of CTAs when the number of row tiles is
+    // even in one of the two orientations (both operands come the same way, so either can be the A side)
+    const bool tma_bf = err_tma && in_tma && a_tmem && bf_cross() && !t_exact;
+    bool pair = false;
+    if (tma_bf && pair_form()) {
+        if (even_row_tiles(swapped ? n_im2col : Cout)) pair = true;
+        else if (even_row_tiles(swapped ? Cout : n_im2col)) { pair = true; swapped = !swapped; }
+    }
+    // tile heights: 128 rows, or 64 for the B side of a pair (each CTA loads half of the tile's B rows)
+    const int rows_err = swapped ? (pair ? kBN / 2 : kBN) : kBM, rows_in = swapped ? kBM : (pair ? kBN / 2 : kBN);
     Batch bt = {};
     uint32_t tx_err = 0, tx_in = 0;
     for (int l = 0; l < n_layers; ++l) {
@@ -1716,21 +1868,21 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
         if (taps) fn = taps == 4 ? VGC_TC_FN(kTma, kGatherTaps4, true) : VGC_TC_FN(kTma, kGatherTaps2, true);
         else if (taps_s2) fn = taps_s2 == 4 ? VGC_TC_FN(kTma, kGatherTaps4S2, true) : VGC_TC_FN(kTma, kGatherTaps2S2, true);
         else if (taps7) fn = VGC_TC_FN(kTma, kGatherTaps7S2, true);
-        else if (e == kTma && i == kTma && bf_cross() && !ex) fn = sqgrad_tc<kMajorK, kTma, kTma, true, false, true>;
+        else if (tma_bf) fn = pair ? sqgrad_tc<kMajorK, kTma, kTma, true, false, true, true> : sqgrad_tc<kMajorK, kTma, kTma, true, false, true>;
         else if (e == kTma && i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kTma, true) : sqgrad_tc<kMajorK, kTma, kTma, false>;
         else if (e == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kGatherIm2col, true) : sqgrad_tc<kMajorK, kTma, kGatherIm2col, false>;
         else if (i == kTma) fn = VGC_TC_FN(kGatherErr, kTma, false);
         else fn = VGC_TC_FN(kGatherErr, kGatherIm2col, false);
-        return tc_launch(fn, bt, n_layers, prm, Cout, n_im2col, k_slices, ws, ws_bytes, st, unit);
+        return tc_launch(fn, bt, n_layers, prm, Cout, n_im2col, k_slices, ws, ws_bytes, st, unit, pair);
     }
     prm.ld_m = 1; prm.ld_n = n_im2col;   // m = idx, n = o
-    if (e == kTma && i == kTma && bf_cross() && !ex) fn = sqgrad_tc<kMajorK, kTma, kTma, true, false, true>;
+    if (tma_bf) fn = pair ? sqgrad_tc<kMajorK, kTma, kTma, true, false, true, true> : sqgrad_tc<kMajorK, kTma, kTma, true, false, true>;
     else if (e == kTma && i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kTma, true) : sqgrad_tc<kMajorK, kTma, kTma, false>;
     else if (i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kGatherErr, true) : sqgrad_tc<kMajorK, kTma, kGatherErr, false>;
     else if (e == kTma) fn = VGC_TC_FN(kGatherIm2col, kTma, false);
     else fn = VGC_TC_FN(kGatherIm2col, kGatherErr, false);
 #undef VGC_TC_FN
-    return tc_launch(fn, bt, n_layers, prm, n_im2col, Cout, k_slices, ws, ws_bytes, st, unit);
+    return tc_launch(fn, bt, n_layers, prm, n_im2col, Cout, k_slices, ws, ws_bytes, st, unit, pair);
 }
 
 // n_layers layers of one geometry; x, delta, S are host arrays of device pointers
