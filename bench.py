@@ -574,6 +574,9 @@ def main():
     ap.add_argument("--impl", default="vgc", choices=["vgc", "reference"])
     ap.add_argument("--n-params", type=int, default=1 << 25, help="size of the 'flat' workload")
     ap.add_argument("--per-layer", action="store_true", help="print per-layer sqgrad times instead of the bench line")
+    ap.add_argument("--mma-rates", action="store_true",
+                    help="print the measured time of one tcgen05.mma instruction per shape (the tensor-pipe ceiling "
+                         "the sqgrad kernel is bounded by) instead of the bench line")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--streams", type=int, default=4, help="streams the independent sqgrad layers are spread over")
     ap.add_argument("--fused", action="store_true",
@@ -604,6 +607,17 @@ def main():
         torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     import paper_1802_06058_b200 as vgc
+    if args.mma_rates:
+        if rank == 0:
+            sms = torch.cuda.get_device_properties(local_rank).multi_processor_count
+            for kind, name in ((0, "tf32 (8 k)"), (1, "bf16 (16 k)")):
+                for a_tmem in (False, True):
+                    for n_cols in (64, 128, 256):
+                        cyc, tf = vgc.vgc_probe_mma_rate(kind, a_tmem, n_cols, 4096, sms)
+                        print(json.dumps({"operands": name, "A_from": "tensor memory" if a_tmem else "shared memory",
+                                          "M": 128, "N": n_cols, "cycles_per_mma": round(cyc, 1),
+                                          "tflops_all_sms": round(tf, 1)}))
+        return
     vgc.load_library()
     pk = peaks()
     hp = HotPath(args.workload, worker=rank * 16, n_input_sets=1, n_g_sets=max(4, min(args.steps + args.warmup, 16)),

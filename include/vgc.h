@@ -134,6 +134,16 @@ vgc_status vgc_sqgrad_conv_exact_batch(int n_layers, const float *const *x, cons
  * the reduction is split less.  Process-wide; set it BEFORE asking for workspace sizes, which depend on it. */
 void vgc_sqgrad_plan_hint(int concurrent_launches);
 
+/* Diagnostic (no counterpart in the paper): how long one tcgen05.mma instruction with M = 128 occupies the tensor
+ * pipe of an SM -- the figure that bounds the squared-gradient contraction, whose ceiling depends on the instruction
+ * shape it can use and not only on the nominal flop rate.  kind 0: tf32 operands (8 k per instruction), 1: bf16 (16 k);
+ * a_tmem != 0: the A operand comes from tensor memory; n: the instruction's N (multiple of 16, <= 256).  `blocks`
+ * thread blocks (one per SM when blocks <= the SM count) each issue `reps` back-to-back MMAs on zero operands.
+ * Host pointers out: cycles per MMA seen by block 0, and the flop rate of the whole launch from its event time.
+ * Synchronises the device; uses the default stream.  VGC_ERR_INVALID_ARG for shapes outside the above,
+ * VGC_ERR_CUDA if a launch failed or the bounded wait for the MMAs gave up. */
+vgc_status vgc_probe_mma_rate(int kind, int a_tmem, int n, int reps, int blocks, double *cycles_per_mma, double *tflops);
+
 /* Several conv layers of ONE geometry in one call (the residual stages of a deep network repeat the same
  * layer shapes): layer l computes what vgc_sqgrad_conv computes from x[l], delta[l] into S[l].  The tensor-
  * core path runs up to 8 layers per kernel launch, which shortens the split of the reduction, the scratch

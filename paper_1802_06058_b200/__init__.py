@@ -33,7 +33,7 @@ EXPORTS = [
     "vgc_compress_workspace_bytes", "vgc_compress", "vgc_compress_static",
     "vgc_decode_accumulate", "vgc_step_host",
     "vgc_compress_hybrid_workspace_bytes", "vgc_compress_hybrid", "vgc_decode_accumulate_hybrid",
-    "vgc_decode_sum", "vgc_decode_sum_hybrid",
+    "vgc_decode_sum", "vgc_decode_sum_hybrid", "vgc_probe_mma_rate",
 ]
 
 
@@ -94,6 +94,8 @@ def load_library():
     lib.vgc_sqgrad_conv_batch.argtypes = [i, vp, vp, vp] + [i] * 11 + [f, i, vp, sz, vp]
     lib.vgc_sqgrad_conv_batch.restype = i
     lib.vgc_sqgrad_plan_hint.argtypes = [i]; lib.vgc_sqgrad_plan_hint.restype = None
+    lib.vgc_probe_mma_rate.argtypes = [i, i, i, i, i, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+    lib.vgc_probe_mma_rate.restype = i
     lib.vgc_sqgrad_conv_exact_workspace_bytes.argtypes = [i] * 11
     lib.vgc_sqgrad_conv_exact_workspace_bytes.restype = sz
     lib.vgc_sqgrad_conv_exact.argtypes = lib.vgc_sqgrad_conv.argtypes
@@ -243,6 +245,16 @@ def vgc_sqgrad_conv_exact(x, delta, kernel, stride, padding, scale: float, S, ac
 def vgc_sqgrad_plan_hint(concurrent_launches: int) -> None:
     """Tell the planner how many sqgrad calls run side by side (streams with separate workspaces)."""
     load_library().vgc_sqgrad_plan_hint(int(concurrent_launches))
+
+
+def vgc_probe_mma_rate(kind: int, a_tmem: bool, n: int, reps: int = 4096, blocks: int = 148):
+    """(cycles per tcgen05.mma instruction on one SM, TFLOP/s of the whole launch) for M = 128, N = n;
+    kind 0 = tf32, 1 = bf16."""
+    cycles, tflops = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    st = load_library().vgc_probe_mma_rate(int(kind), int(bool(a_tmem)), int(n), int(reps), int(blocks),
+                                           ctypes.byref(cycles), ctypes.byref(tflops))
+    _check(st, "vgc_probe_mma_rate")
+    return cycles.value, tflops.value
 
 
 def vgc_sqgrad_conv_batch_workspace_bytes(n_layers, B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, exact: bool = False) -> int:

@@ -77,7 +77,7 @@ constexpr int kSplitA = 4, kSplitB = 7, kSplitLo = 3;              // 16-KB unit
 static_assert((kSplitA + kSplitB + kSplitLo) * kRawBytesA <= (kRawSlots + kLoSlots) * kRawStageBytes, "smem budget");
 // Pair form (two CTAs of a cluster share one 256 x 128 tile, tcgen05 cta_group::2): each CTA holds its own 128 A rows
 // and half of the B rows, so a B slot is 8 KB and the rings get deeper: A raw, B raw/hi, B bf16 (+ A in TMEM)
-constexpr int kPairA = 5, kPairB = 10, kPairLo = 4;
+constexpr int kPairA = 8, kPairB = 8, kPairLo = 4;
 constexpr uint32_t kPairBBytes = kRawBytesB / 2;
 static_assert(kPairA * kRawBytesA + (kPairB + kPairLo) * kPairBBytes <= (kRawSlots + kLoSlots) * kRawStageBytes, "smem budget");
 constexpr uint32_t kTmemColsA = 64;                                 // per slot: 32 columns hi + 32 columns lo
@@ -1521,12 +1521,6 @@ static vgc_status tc_launch(KernelFn kernel, const Batch &bt, int n_layers, Para
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr; cfg.numAttrs = 1;
-        if (getenv("VGC_DEBUG")) {
-            int n_clusters = -1;
-            const cudaError_t oe = cudaOccupancyMaxActiveClusters(&n_clusters, kernel, &cfg);
-            fprintf(stderr, "vgc: pair launch grid (%u, %u, %u), smem %u: max active clusters %d (%s)\n", grid.x, grid.y,
-                    grid.z, (unsigned)kSmemBytes, n_clusters, cudaGetErrorString(oe));
-        }
         VGC_CUDA_OK(cudaLaunchKernelEx(&cfg, kernel, bt, prm));
     } else {
         kernel<<<grid, kThreadsTc, kSmemBytes, st>>>(bt, prm);

@@ -243,3 +243,18 @@ def test_plan_hint_changes_the_split_not_the_result():
             _check(run_conv(x, d, 1, 1, 0, 1.0), want)
     finally:
         vgc.vgc_sqgrad_plan_hint(1)
+
+
+def test_mma_rate_probe_reports_the_instruction_floor():
+    """The diagnostic behind the kernel's tensor-pipe ceiling: with M = 128 an instruction takes as long for N = 64 as
+    for N = 128 (so half-width tiles run at half the rate) and less than twice as long for N = 256."""
+    c64, _ = vgc.vgc_probe_mma_rate(0, True, 64, reps=2048, blocks=8)
+    c128, tf128 = vgc.vgc_probe_mma_rate(0, True, 128, reps=2048, blocks=8)
+    c256, tf256 = vgc.vgc_probe_mma_rate(0, True, 256, reps=2048, blocks=8)
+    assert 20 < c128 < 1000 and tf128 > 0
+    assert c64 > 0.9 * c128
+    assert c128 < c256 < 1.9 * c128 and tf256 > tf128
+    with pytest.raises(vgc.VgcError):
+        vgc.vgc_probe_mma_rate(0, True, 100)
+    with pytest.raises(vgc.VgcError):
+        vgc.vgc_probe_mma_rate(2, True, 128)
