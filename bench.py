@@ -694,6 +694,9 @@ def main():
                     "traffic": NCU_SQGRAD_PASS_BYTES_RESNET50 if args.workload == "resnet50" else None,
                     "issued_tflops": issue_factor * ach, "issue_factor": issue_factor, "tf32_peak": tf32_peak,
                     "frac_of_3xtf32_ceiling": ach / (tf32_peak / 3.0),
+                    # measured with `bench.py --mma-rates` (profiles/tcgen05_mma_rates.md): the rate of back-to-back
+                    # tf32 MMAs of the 128 x 128 shape this kernel issues, all SMs, 1965 MHz
+                    "shape_ceiling_tflops": 620.8, "issued_frac_of_shape_ceiling": issue_factor * ach / 620.8,
                     "algorithmic_frac_of_tf32_peak": ach / tf32_peak,
                     "peak_source": f"{pk['source']} bf16 sustained x 1/2 (tf32 nominal ratio) / issue_factor, of measured",
                     "note": "achieved = algorithmic flops 2*M*N*K per layer / sqgrad time; frac = tensor-pipe load: "
