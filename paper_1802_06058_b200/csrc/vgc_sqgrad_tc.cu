@@ -103,6 +103,7 @@ struct Params {
     uint32_t tx_bytes_a;     // of which the A tile's
     float scale;
     int accumulate;
+    int tiles_x;             // 128-column tiles of the output (wide form: the scratch is indexed in these)
     int splits;              // blocks along the reduction per layer (blockIdx.z = layer * splits + split)
     int C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, Wo, P;     // conv geometry (gathered tiles)
     int chw;                 // C*H*W
@@ -718,7 +719,15 @@ struct Gatherer<kMode, kHalf, true> {
 // the B rows, which halves the B share of the shared-memory traffic.  The even CTA issues the MMAs; the transform and
 // epilogue warps of the odd one signal its barriers through the cluster's shared-memory window, and a commit
 // arrives on the barriers of both.
-template <int kMajor, int kModeA, int kModeB, bool kATmem, bool kExact = false, bool kBf = false, bool kPair = false>
+// kWide (a pair form): the pair's tile is 256 x 256 and its instructions have N = 256, the shape at which the tensor
+// pipe delivers its full rate (an instruction takes 138 cycles there against 96 - 110 for any N up to 128).  Each CTA
+// holds 128 of the 256 B rows, i.e. the tiles, rings and transform load of the single-CTA kernel.  Tensor memory has room
+// for one accumulator of 256 columns next to the A ring, so chunks are not double-buffered: the MMAs pause while a chunk
+// is drained.  The epilogue keeps no running sums (256 per lane do not fit in registers): it stores the first chunk to
+// the split-K scratch and adds the later ones there with red.global.add (one thread per address, in program order), and
+// the combine kernel, which always runs in this form, writes the result.
+template <int kMajor, int kModeA, int kModeB, bool kATmem, bool kExact = false, bool kBf = false, bool kPair = false,
+          bool kWide = false>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
 {
@@ -730,12 +739,15 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
     constexpr bool kSplit = kATmem && !kAnyGather;                         // A raw tiles in a ring of their own
     static_assert(!kBf || (kSplit && !kExact), "bf16 cross terms: the TMA-fed form with A in tensor memory");
     static_assert(!kPair || kBf, "the pair form exists for the TMA-fed form with bf16 cross terms");
-    constexpr int kNA = kPair ? kPairA : kSplitA;                          // slots of the raw A ring (split form)
+    static_assert(!kWide || kPair, "N = 256 instructions are issued by CTA pairs");
+    constexpr bool kHalfB = kPair && !kWide;                               // this CTA's B tile has 64 rows (else 128)
+    constexpr int kTileN = kWide ? 2 * kBN : kBN;                          // columns of the block's (pair's) output tile
+    constexpr int kNA = kHalfB ? kPairA : kSplitA;                         // slots of the raw A ring (split form)
     // the transform warps work as two groups of four on alternate slices (else all eight on every slice)
     constexpr bool kTwoGroups = !kAnyGather || (IsTaps<kModeB>::value && kModeA == kTma);
-    constexpr int kNB = kPair ? kPairB : kSplit ? kSplitB : kRawSlots;     // slots of the raw / hi ring
+    constexpr int kNB = kHalfB ? kPairB : kSplit ? kSplitB : kRawSlots;    // slots of the raw / hi ring
     // lo slots (and A slots in TMEM); the per-example form needs 128 TMEM columns for its sum of squares
-    constexpr int kLoN = kPair ? kPairLo : (kExact && kATmem) ? 2 : kSplit ? kSplitLo : (kATmem ? kLoSlotsAT : kLoSlots);
+    constexpr int kLoN = kHalfB ? kPairLo : (kExact && kATmem) ? 2 : kSplit ? kSplitLo : (kATmem ? kLoSlotsAT : kLoSlots);
     constexpr uint32_t kSqCol = 2 * kBN + (kATmem ? 2 * kTmemColsA : 0);         // where that sum lives
     constexpr uint32_t kLoBytes = kATmem ? kRawBytesB : kRawStageBytes;  // bytes of one lo slot
     // byte offsets of slot s: the [A][B] pair of the raw / hi ring (split form: only its B half exists, the
@@ -748,12 +760,12 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
 
     // bf16-cross form: where the B tile of raw slot s and the [hi bf16][lo bf16] tiles of lo slot s live
     auto b_tile = [&](int s) -> uint32_t {
-        return kPair ? (uint32_t)kPairA * kRawBytesA + (uint32_t)s * kPairBBytes : pair_off(s) + kRawBytesA;
+        return kHalfB ? (uint32_t)kPairA * kRawBytesA + (uint32_t)s * kPairBBytes : pair_off(s) + kRawBytesA;
     };
     auto bf_tile = [&](int s) -> uint32_t {
-        return kPair ? (uint32_t)kPairA * kRawBytesA + (uint32_t)(kPairB + s) * kPairBBytes : lo_off(s) + kRawBytesA;
+        return kHalfB ? (uint32_t)kPairA * kRawBytesA + (uint32_t)(kPairB + s) * kPairBBytes : lo_off(s) + kRawBytesA;
     };
-    constexpr uint32_t kBTile = kPair ? kPairBBytes : kRawBytesB;          // bytes of this CTA's B tile
+    constexpr uint32_t kBTile = kHalfB ? kPairBBytes : kRawBytesB;         // bytes of this CTA's B tile
 
     extern __shared__ uint8_t smem_raw_[];
     __shared__ __align__(8) uint64_t bars[3 * kPairB + kLoSlotsAT + 5 + 2 * kPairA];
@@ -778,8 +790,8 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
     // the two CTAs of a pair, neighbours in rows, must be neighbours along x
     const int tile_n = kPair ? (int)blockIdx.y : (int)blockIdx.x, tile_m = kPair ? (int)blockIdx.x : (int)blockIdx.y;
     const int tiles_n = kPair ? (int)gridDim.y : (int)gridDim.x;
-    const int m0 = tile_m * kBM, n0 = tile_n * kBN;
-    const int n_valid = min(kBN, prm.N - n0);                              // columns of this tile that exist
+    const int m0 = tile_m * kBM, n0 = tile_n * kTileN;
+    const int n_valid = min(kTileN, prm.N - n0);                           // columns of this tile that exist
     const int n_act = kPair ? (n_valid + 31) & ~31 : (n_valid + 15) & ~15; // UMMA N (multiple of 16; of 32 for a pair)
     const int layer = (int)blockIdx.z / prm.splits, split = (int)blockIdx.z - layer * prm.splits;
     const CUtensorMap *map_a = &bt.a[layer], *map_b = &bt.b[layer];
@@ -911,8 +923,8 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
             uint32_t st_phase = 0;
             bool ok = true;
             for (int c = 0; c < n_chunks && ok; ++c) {
-                const int b = c & 1;
-                ok = mbar_wait(smem_u32(&acc_empty[b]), ((uint32_t)(c >> 1) & 1u) ^ 1u, &abort_flag, 0);
+                const int b = kWide ? 0 : c & 1;                             // the wide form has one accumulator
+                ok = mbar_wait(smem_u32(&acc_empty[b]), ((uint32_t)(kWide ? c : c >> 1) & 1u) ^ 1u, &abort_flag, 0);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)b * kBN;
@@ -1170,6 +1182,71 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
             }
         }
         }
+    } else if (kWide) {
+        // ================= epilogue warps, wide form =================
+        // Columns 0..127 of the pair's tile keep their running sums in registers as in the other forms; 256 per lane
+        // do not fit, so columns 128..255 go to the split-K scratch chunk by chunk (first chunk stored, later ones
+        // added with red.global.add -- one thread per address, in program order).  The accumulator is handed back as
+        // soon as its last columns are in registers, before their reds are issued.
+        const uint32_t q = warp & 3;
+        const int r_local = (int)(q * 32u + lane);
+        // this CTA's two 128 x 128 scratch tiles (column halves of its 128 x 256 part), column-major inside a tile
+        const size_t tiles_layer = (size_t)prm.tiles_x * gridDim.x;
+        const size_t tile0 = (size_t)blockIdx.z * tiles_layer + (size_t)tile_m * prm.tiles_x + (size_t)tile_n * 2;
+        float *const dst0 = prm.partial + tile0 * (kBM * kBN) + r_local;
+        float acc[kBN];
+#pragma unroll
+        for (int j = 0; j < kBN; ++j) acc[j] = 0.f;
+        bool ok = true;
+        for (int c = 0; c < n_chunks && ok; ++c) {
+            ok = mbar_wait(smem_u32(&acc_full[0]), (uint32_t)c & 1u, &abort_flag, 32);     // the MMAs wait for this drain
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((q * 32u) << 16);
+#pragma unroll
+            for (int j0 = 0; j0 < kBN; j0 += 32) {
+                if (j0 < n_act) {
+                    uint32_t r[32];
+                    tc_ld_32x32(taddr + j0, r);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) acc[j0 + j] = __fadd_rn(acc[j0 + j], __uint_as_float(r[j]));
+                }
+            }
+            bool released = false;
+            auto release = [&]() {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cta(smem_u32(&acc_empty[0]), 0);
+                released = true;
+            };
+#pragma unroll
+            for (int j0 = kBN; j0 < kTileN; j0 += 32) {
+                if (j0 < n_act) {
+                    uint32_t r[32];
+                    tc_ld_32x32(taddr + j0, r);
+                    tc_wait_ld();
+                    if (j0 + 32 >= n_act) release();              // the last columns are out of tensor memory
+                    float *dst = dst0 + (size_t)j0 * kBM;         // tile 1 follows tile 0 in the scratch
+                    if (c == 0) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j0 + j < n_valid) dst[j * kBM] = __uint_as_float(r[j]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j0 + j < n_valid)
+                                asm volatile("red.global.add.f32 [%0], %1;" ::"l"(dst + j * kBM), "f"(__uint_as_float(r[j])) : "memory");
+                    }
+                }
+            }
+            if (!released) release();
+        }
+        if (ok) {
+#pragma unroll
+            for (int j = 0; j < kBN; ++j)
+                if (j < n_valid) dst0[(size_t)j * kBM] = acc[j];
+        }
     } else {
         // ================= epilogue warps: drain chunks, accumulate in fp32 registers =================
         const uint32_t q = warp & 3;                                      // TMEM lane quarter of this warp
@@ -1426,13 +1503,15 @@ struct Plan {
 static int g_concurrent_launches = 1;
 
 // `unit`: slices that must stay in one block (the per-example form splits the reduction between examples only)
-static Plan make_plan(int M, int N, int k_slices_total, int n_layers = 1, int unit = 1)
+// `wide`: the blocks are CTA pairs' halves of 256 x 256 tiles, i.e. each block covers two 128-column tiles
+static Plan make_plan(int M, int N, int k_slices_total, int n_layers = 1, int unit = 1, bool wide = false)
 {
     Plan p;
     const int k_slices = k_slices_total / unit;                          // planned in units
     p.tiles_x = (N + kBN - 1) / kBN;
     p.tiles_y = (M + kBM - 1) / kBM;
-    const long tiles = (long)p.tiles_x * p.tiles_y * n_layers;          // output tiles of the whole launch
+    // blocks of one split of the whole launch
+    const long tiles = (long)(wide ? (p.tiles_x + 1) / 2 : p.tiles_x) * p.tiles_y * n_layers;
     // Blocks run one per SM, wave after wave.  A caller that runs several launches side by side (separate
     // streams and workspaces, vgc_sqgrad_plan_hint) may also plan for fewer SMs per launch through VGC_TC_BLOCKS.
     const char *env = getenv("VGC_TC_BLOCKS");
@@ -1485,18 +1564,35 @@ bool tc_conv_supported(int B, int C, int H, int W, int Cout, int Kh, int Kw, int
            (long)B * ((P + kBK - 1) / kBK) < (1L << 30);
 }
 
+// the wide pair form (256 x 256 tiles, N = 256 instructions) where the pair form applies: VGC_TC_WIDE=1
+static bool wide_form()
+{
+    const char *e = getenv("VGC_TC_WIDE");
+    return e && atoi(e) != 0;
+}
+
 static size_t tc_workspace_bytes(int M, int N, int k_slices, int n_layers = 1, int unit = 1)
 {
     const Plan p = make_plan(M, N, k_slices, n_layers, unit);
-    return 256 + (p.splits > 1 ? (size_t)n_layers * p.splits * p.tiles_x * p.tiles_y * kBM * kBN * sizeof(float) : 0);
+    size_t need = 256 + (p.splits > 1 ? (size_t)n_layers * p.splits * p.tiles_x * p.tiles_y * kBM * kBN * sizeof(float) : 0);
+    if (wide_form()) {
+        // the wide form always goes through the scratch and splits further (half as many blocks per split); which
+        // operand becomes the row side is decided at launch, so both orientations are covered
+        const Plan a = make_plan(M, N, k_slices, n_layers, unit, true), b = make_plan(N, M, k_slices, n_layers, unit, true);
+        const size_t splits = a.splits > b.splits ? a.splits : b.splits;
+        const size_t w = 256 + (size_t)n_layers * splits * p.tiles_x * p.tiles_y * kBM * kBN * sizeof(float);
+        if (w > need) need = w;
+    }
+    return need;
 }
 
 typedef void (*KernelFn)(const Batch, const Params);
 
 static vgc_status tc_launch(KernelFn kernel, const Batch &bt, int n_layers, Params prm, int M, int N,
-                            int k_slices, void *ws, size_t ws_bytes, cudaStream_t st, int unit = 1, bool pair = false)
+                            int k_slices, void *ws, size_t ws_bytes, cudaStream_t st, int unit = 1, bool pair = false,
+                            bool wide = false)
 {
-    const Plan plan = make_plan(M, N, k_slices, n_layers, unit);
+    const Plan plan = make_plan(M, N, k_slices, n_layers, unit, wide);
     if (ws_bytes < tc_workspace_bytes(M, N, k_slices, n_layers, unit)) return VGC_ERR_WORKSPACE;
     static KernelFn configured[32];
     static int n_configured = 0;
@@ -1508,6 +1604,7 @@ static vgc_status tc_launch(KernelFn kernel, const Batch &bt, int n_layers, Para
     }
     prm.M = M; prm.N = N; prm.k_slices = k_slices; prm.slices_per_split = plan.slices_per_split;
     prm.splits = plan.splits;
+    prm.tiles_x = plan.tiles_x;
     prm.chunk = default_chunk();
     prm.status = static_cast<uint32_t *>(ws);
     prm.partial = reinterpret_cast<float *>(static_cast<char *>(ws) + 256);
@@ -1516,7 +1613,7 @@ static vgc_status tc_launch(KernelFn kernel, const Batch &bt, int n_layers, Para
         // clusters of two CTAs, neighbours along x, which holds the row tiles in this form (the caller made sure
         // their number is even)
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(grid.y, grid.x, grid.z); cfg.blockDim = dim3(kThreadsTc); cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st;
+        cfg.gridDim = dim3(grid.y, wide ? (grid.x + 1) / 2 : grid.x, grid.z); cfg.blockDim = dim3(kThreadsTc); cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
@@ -1526,7 +1623,7 @@ static vgc_status tc_launch(KernelFn kernel, const Batch &bt, int n_layers, Para
         kernel<<<grid, kThreadsTc, kSmemBytes, st>>>(bt, prm);
     }
     count_launch();
-    if (plan.splits > 1) {
+    if (plan.splits > 1 || wide) {
         ResultPtrs results = {};
         for (int l = 0; l < n_layers; ++l) results.S[l] = bt.S[l];
         sqgrad_tc_combine<<<dim3((unsigned)(plan.tiles_x * plan.tiles_y * 64), (unsigned)n_layers), 256, 0, st>>>(
@@ -1818,13 +1915,23 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
     // both tiles by TMA, A in tensor memory, cross terms in bf16; on pairs of CTAs when the number of row tiles is
     // even in one of the two orientations (both operands come the same way, so either can be the A side)
     const bool tma_bf = err_tma && in_tma && a_tmem && bf_cross() && !t_exact;
-    bool pair = false;
-    if (tma_bf && pair_form()) {
-        if (even_row_tiles(swapped ? n_im2col : Cout)) pair = true;
-        else if (even_row_tiles(swapped ? Cout : n_im2col)) { pair = true; swapped = !swapped; }
+    bool pair = false, wide = false;
+    if (tma_bf && (pair_form() || wide_form())) {
+        // the orientation whose number of row tiles is even (the given one first)
+        const bool as_is = even_row_tiles(swapped ? n_im2col : Cout);
+        const bool flipped = !as_is && even_row_tiles(swapped ? Cout : n_im2col);
+        if (as_is || flipped) {
+            const bool sw = flipped ? !swapped : swapped;
+            // 256 x 256 tiles (each CTA of a pair has 128 B rows again) pay where the tile is at least 256 columns
+            // wide and the reduction long enough to cover the unbuffered accumulator's drains and the extra combine pass
+            wide = wide_form() && (sw ? Cout : n_im2col) >= 2 * kBN && k_slices >= 128;
+            pair = wide || pair_form();
+            if (pair) swapped = sw;
+        }
     }
-    // tile heights: 128 rows, or 64 for the B side of a pair (each CTA loads half of the tile's B rows)
-    const int rows_err = swapped ? (pair ? kBN / 2 : kBN) : kBM, rows_in = swapped ? kBM : (pair ? kBN / 2 : kBN);
+    // tile heights: 128 rows, or 64 for the B side of a plain pair (each CTA loads half of the tile's B rows)
+    const int rows_b = pair && !wide ? kBN / 2 : kBN;
+    const int rows_err = swapped ? rows_b : kBM, rows_in = swapped ? kBM : rows_b;
     Batch bt = {};
     uint32_t tx_err = 0, tx_in = 0;
     for (int l = 0; l < n_layers; ++l) {
@@ -1862,21 +1969,25 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
         if (taps) fn = taps == 4 ? VGC_TC_FN(kTma, kGatherTaps4, true) : VGC_TC_FN(kTma, kGatherTaps2, true);
         else if (taps_s2) fn = taps_s2 == 4 ? VGC_TC_FN(kTma, kGatherTaps4S2, true) : VGC_TC_FN(kTma, kGatherTaps2S2, true);
         else if (taps7) fn = VGC_TC_FN(kTma, kGatherTaps7S2, true);
-        else if (tma_bf) fn = pair ? sqgrad_tc<kMajorK, kTma, kTma, true, false, true, true> : sqgrad_tc<kMajorK, kTma, kTma, true, false, true>;
+        else if (tma_bf) fn = wide   ? sqgrad_tc<kMajorK, kTma, kTma, true, false, true, true, true>
+                              : pair ? sqgrad_tc<kMajorK, kTma, kTma, true, false, true, true>
+                                     : sqgrad_tc<kMajorK, kTma, kTma, true, false, true>;
         else if (e == kTma && i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kTma, true) : sqgrad_tc<kMajorK, kTma, kTma, false>;
         else if (e == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kGatherIm2col, true) : sqgrad_tc<kMajorK, kTma, kGatherIm2col, false>;
         else if (i == kTma) fn = VGC_TC_FN(kGatherErr, kTma, false);
         else fn = VGC_TC_FN(kGatherErr, kGatherIm2col, false);
-        return tc_launch(fn, bt, n_layers, prm, Cout, n_im2col, k_slices, ws, ws_bytes, st, unit, pair);
+        return tc_launch(fn, bt, n_layers, prm, Cout, n_im2col, k_slices, ws, ws_bytes, st, unit, pair, wide);
     }
     prm.ld_m = 1; prm.ld_n = n_im2col;   // m = idx, n = o
-    if (tma_bf) fn = pair ? sqgrad_tc<kMajorK, kTma, kTma, true, false, true, true> : sqgrad_tc<kMajorK, kTma, kTma, true, false, true>;
+    if (tma_bf) fn = wide   ? sqgrad_tc<kMajorK, kTma, kTma, true, false, true, true, true>
+                     : pair ? sqgrad_tc<kMajorK, kTma, kTma, true, false, true, true>
+                            : sqgrad_tc<kMajorK, kTma, kTma, true, false, true>;
     else if (e == kTma && i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kTma, true) : sqgrad_tc<kMajorK, kTma, kTma, false>;
     else if (i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kGatherErr, true) : sqgrad_tc<kMajorK, kTma, kGatherErr, false>;
     else if (e == kTma) fn = VGC_TC_FN(kGatherIm2col, kTma, false);
     else fn = VGC_TC_FN(kGatherIm2col, kGatherErr, false);
 #undef VGC_TC_FN
-    return tc_launch(fn, bt, n_layers, prm, n_im2col, Cout, k_slices, ws, ws_bytes, st, unit, pair);
+    return tc_launch(fn, bt, n_layers, prm, n_im2col, Cout, k_slices, ws, ws_bytes, st, unit, pair, wide);
 }
 
 // n_layers layers of one geometry; x, delta, S are host arrays of device pointers

@@ -147,7 +147,7 @@ def test_repacked_and_in_place_forms_agree_with_the_oracle(monkeypatch, B, C, H,
 
 
 @pytest.mark.parametrize("env", [{"VGC_TC_ATMEM": "0"}, {"VGC_TC_GATHER": "1"}, {"VGC_TC_GATHER": "2"},
-                                 {"VGC_TC_GATHER": "3"}, {"VGC_SQGRAD_PATH": "simt"}, {"VGC_TC_TAPS": "0"}, {"VGC_TC_BF16": "0"}, {"VGC_TC_PAIR": "1"}])
+                                 {"VGC_TC_GATHER": "3"}, {"VGC_SQGRAD_PATH": "simt"}, {"VGC_TC_TAPS": "0"}, {"VGC_TC_BF16": "0"}, {"VGC_TC_PAIR": "1"}, {"VGC_TC_WIDE": "1"}])
 @pytest.mark.parametrize("B,C,H,Cout,k,s,p", [(3, 96, 12, 160, 1, 1, 0), (2, 40, 12, 48, 3, 1, 1), (2, 72, 16, 200, 3, 2, 1)])
 def test_every_kernel_variant_gives_the_same_statistic(monkeypatch, env, B, C, H, Cout, k, s, p):
     """The library picks a kernel form per layer (TMA or gathered tiles, A operand in shared or tensor memory,
@@ -178,18 +178,24 @@ def test_constant_inputs_rounding_errors_all_of_one_sign(monkeypatch, bf16_cross
     _check(got, want)
 
 
+@pytest.mark.parametrize("form", ["VGC_TC_PAIR", "VGC_TC_WIDE"])
 @pytest.mark.parametrize("B,C,H,Cout", [(2, 128, 8, 256), (3, 256, 14, 64), (2, 100, 12, 200), (4, 64, 56, 64),
-                                        (8, 256, 14, 1024), (2, 130, 8, 520), (4, 512, 28, 128), (2, 384, 7, 640)])
-def test_pair_form_of_the_1x1_kernel(monkeypatch, B, C, H, Cout):
-    """VGC_TC_PAIR=1: two CTAs of a cluster share a 256 x 128 tile (cta_group::2).  The shapes cover an even number of row
-    tiles as given, one that is even only with the operands' roles exchanged, one with no even side (falls back to
-    single CTAs), ragged last tiles, the repacked 7x7 form and split reductions; one call and a batch of three layers."""
-    monkeypatch.setenv("VGC_TC_PAIR", "1")
+                                        (8, 256, 14, 1024), (2, 130, 8, 520), (4, 512, 28, 128), (2, 384, 7, 640),
+                                        (20, 256, 14, 512), (6, 256, 28, 384)])
+def test_pair_forms_of_the_1x1_kernel(monkeypatch, form, B, C, H, Cout):
+    """VGC_TC_PAIR=1: two CTAs of a cluster share a 256 x 128 tile (cta_group::2); VGC_TC_WIDE=1: a 256 x 256 tile with
+    N = 256 instructions where the layer is wide and deep enough (the last two shapes; the last one only with the
+    operands' roles exchanged and with a half-empty second tile), pairs or single CTAs elsewhere.  The shapes cover an
+    even number of row tiles as given, one that is even only with the roles exchanged, one with no even side (falls back
+    to single CTAs), ragged last tiles, the repacked 7x7 form and split reductions; one call and a batch of three layers."""
+    monkeypatch.setenv(form, "1")
     gen = torch.Generator(device="cuda"); gen.manual_seed(B + C + Cout)
     xs = [torch.randn(B, C, H, H, device="cuda", generator=gen).clamp_(min=0) for _ in range(3)]
     ds = [torch.randn(B, Cout, H, H, device="cuda", generator=gen) * 1e-2 for _ in range(3)]
     wants = [oracle.sqgrad_conv(x.cpu().numpy(), d.cpu().numpy(), (1, 1), (1, 1), (0, 0), scale=0.25) for x, d in zip(xs, ds)]
     _check(run_conv(xs[0], ds[0], 1, 1, 0, 0.25), wants[0])
+    S0 = torch.rand(Cout, C, 1, 1, device="cuda", generator=gen) * float(wants[0].mean())
+    _check(run_conv(xs[0], ds[0], 1, 1, 0, 0.25, S0=S0), S0.cpu().numpy().astype(np.float64) + wants[0])
     Ss = [torch.empty(Cout * C, device="cuda") for _ in range(3)]
     ws = _ws(vgc.vgc_sqgrad_conv_batch_workspace_bytes(3, B, C, H, H, Cout, 1, 1, 1, 1, 0, 0))
     vgc.vgc_sqgrad_conv_batch(xs, ds, (1, 1), (1, 1), (0, 0), 0.25, Ss, ws=ws)
