@@ -46,6 +46,23 @@ def test_workspace_queries_are_pure_host_functions(lib):
     assert lib.vgc_sqgrad_conv_workspace_bytes(32, 64, 2, 2, 64, 3, 3, 1, 1, 0, 0) == 0   # kernel > image
 
 
+def test_workspace_for_the_pair_forms(lib, monkeypatch):
+    """The tile forms are chosen per call from the environment; the workspace query follows the same switches: the wide
+    pair form always goes through the split-K scratch and may split further, so it never needs less; plain pairs use the
+    single-CTA plan."""
+    shapes = [(32, 256, 14, 14, 1024, 1, 1, 1, 1, 0, 0), (32, 1024, 14, 14, 256, 1, 1, 1, 1, 0, 0),
+              (32, 64, 56, 56, 256, 1, 1, 1, 1, 0, 0), (32, 512, 28, 28, 1024, 1, 1, 2, 2, 0, 0),
+              (32, 64, 56, 56, 64, 3, 3, 1, 1, 1, 1)]
+    plain = [lib.vgc_sqgrad_conv_workspace_bytes(*g) for g in shapes]
+    monkeypatch.setenv("VGC_TC_PAIR", "1")
+    assert [lib.vgc_sqgrad_conv_workspace_bytes(*g) for g in shapes] == plain
+    monkeypatch.setenv("VGC_TC_WIDE", "1")
+    wide = [lib.vgc_sqgrad_conv_workspace_bytes(*g) for g in shapes]
+    assert all(w >= p for w, p in zip(wide, plain))
+    assert wide[0] > 256 + 1024 * 256 * 4 - 1                  # at least one scratch copy of the result
+    assert [lib.vgc_sqgrad_conv_batch_workspace_bytes(3, *g) >= w for g, w in zip(shapes, wide)] == [True] * len(shapes)
+
+
 def test_compress_rejects_bad_arguments_on_the_host(lib):
     fake = ctypes.c_void_p(0x1000)          # never dereferenced: every call below fails validation first
     msg = vgc._MessageStruct(0x1000, 16, 0x1000, 0x1000, 0x1000, 0x1000, None, 0x1000)
