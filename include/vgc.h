@@ -79,7 +79,8 @@ uint64_t vgc_kernel_launch_count(void);
  *                  (e.g. when allocating ws): kernels only ever OR bits into it -- VGC_DEV_TIMEOUT
  *                  if a bounded wait inside a kernel gave up, in which case S is invalid.
  *
- * Result within 1e-5 relative of the exact sum.  B, in, out >= 1 (any of them 0: no-op, OK).
+ * Result within 1e-5 relative of the exact sum.  in == 0 or out == 0: no-op, OK.  B == 0: the sum is empty --
+ * S is cleared when accumulate == 0 and left alone otherwise; the workspace is not used.
  * ------------------------------------------------------------------------------------------- */
 size_t vgc_sqgrad_linear_workspace_bytes(int B, int in, int out);
 vgc_status vgc_sqgrad_linear(const float *x, const float *delta, int B, int in, int out,
@@ -94,7 +95,7 @@ vgc_status vgc_sqgrad_linear(const float *x, const float *delta, int B, int in, 
  *
  *   x      [B][C][H][W]        fp32 NCHW        delta  [B][Cout][Ho][Wo]  fp32
  *   S      [Cout][C][Kh][Kw]   fp32 (OIHW, the layer's slice of the flat buffer)
- *   Ho = (H + 2*pad_h - Kh)/stride_h + 1, Wo likewise; both must be >= 1.
+ *   Ho = (H + 2*pad_h - Kh)/stride_h + 1, Wo likewise; both must be >= 1.  B == 0 as for the dense layer.
  * ------------------------------------------------------------------------------------------- */
 size_t vgc_sqgrad_conv_workspace_bytes(int B, int C, int H, int W, int Cout, int Kh, int Kw,
                                        int stride_h, int stride_w, int pad_h, int pad_w);
@@ -128,27 +129,11 @@ vgc_status vgc_sqgrad_conv_exact_batch(int n_layers, const float *const *x, cons
                                        int pad_h, int pad_w, float scale, int accumulate, void *ws, size_t ws_bytes,
                                        vgc_stream_t stream);
 
-/* Planning hint (no counterpart in the paper): how many sqgrad calls the caller keeps in flight side by side
- * on different streams, each with its own workspace (default 1).  Alone, a launch is planned so that its
- * blocks fill whole waves over the SMs; next to other launches a partly filled last wave costs nothing, and
- * the reduction is split less.  Process-wide; set it BEFORE asking for workspace sizes, which depend on it. */
-void vgc_sqgrad_plan_hint(int concurrent_launches);
-
-/* Diagnostic (no counterpart in the paper): how long one tcgen05.mma instruction with M = 128 occupies the tensor
- * pipe of an SM -- the figure that bounds the squared-gradient contraction, whose ceiling depends on the instruction
- * shape it can use and not only on the nominal flop rate.  kind 0: tf32 operands (8 k per instruction), 1: bf16 (16 k);
- * a_tmem != 0: the A operand comes from tensor memory; n: the instruction's N (multiple of 16, <= 256).  `blocks`
- * thread blocks (one per SM when blocks <= the SM count) each issue `reps` back-to-back MMAs on zero operands.
- * Host pointers out: cycles per MMA seen by block 0, and the flop rate of the whole launch from its event time.
- * Synchronises the device; uses the default stream.  VGC_ERR_INVALID_ARG for shapes outside the above,
- * VGC_ERR_CUDA if a launch failed or the bounded wait for the MMAs gave up. */
-vgc_status vgc_probe_mma_rate(int kind, int a_tmem, int n, int reps, int blocks, double *cycles_per_mma, double *tflops);
-
 /* Several conv layers of ONE geometry in one call (the residual stages of a deep network repeat the same
  * layer shapes): layer l computes what vgc_sqgrad_conv computes from x[l], delta[l] into S[l].  The tensor-
- * core path runs up to 8 layers per kernel launch, which shortens the split of the reduction, the scratch
- * traffic and the per-launch fixed cost; results are identical to n_layers single calls only up to the
- * order of the fp32 partial sums (same 1e-5 bound).
+ * core path runs up to 8 layers per kernel launch and cuts their combined work evenly over the SMs, which a
+ * single small layer cannot fill; results are identical to n_layers single calls only up to the order of the
+ * fp32 partial sums (same 1e-5 bound).
  *   x, delta, S   HOST arrays of n_layers DEVICE pointers (read during the call only)
  *   ws            at least vgc_sqgrad_conv_batch_workspace_bytes(n_layers, ...) bytes; status word as above
  * The layers' S ranges must not overlap.  n_layers == 0: no-op, OK. */
@@ -237,18 +222,27 @@ vgc_status vgc_compress_static(const float *g, const float *s, float *r, float *
  *
  * For every word of every message w:  u[idx] += scale * (-1)^sign * 2^(group_exp_w[k] - d), k the
  * tensor that holds idx.  The W messages are summed ("allreduce" semantics of Sec. 4.3 realised
- * after an allgatherv); scale = 1/W gives the mean.  Additions into one element may happen in any
- * order (fp32 atomics), so results match a sequential sum to rounding only.
+ * after an allgatherv); scale = 1/W gives the mean.
  *
  *   msgs   HOST array of W views; each view holds DEVICE pointers; the word count is read on the device.
  *          Words must be in ascending index order, as vgc_compress emits them.
  *   u      [n] fp32, accumulated in place (the caller zeroes it when a fresh sum is wanted)
- * Words whose index is >= n are skipped and VGC_DEV_RANGE is set.  W == 0 or n == 0: no-op, OK.
+ *
+ * Order of the additions.  When the messages together hold at least one word per eight elements, u is moved
+ * through shared memory and every element receives its additions in message order (w = 0, 1, ...): the result
+ * is the fp32 sequence of a sequential sum and does not depend on scheduling, so every worker that decodes the
+ * same messages gets the same bits.  Sparser calls add with fp32 atomics, in any order: an element hit by
+ * three or more messages may then differ from the sequential sum in the last bit.
+ *
+ * Words whose index is >= n are skipped and VGC_DEV_RANGE is set; a word that breaks the ascending order may
+ * be skipped as well (never applied to a wrong element), again with VGC_DEV_RANGE.  A view's word count above
+ * its max_words is clamped (VGC_DEV_CAPACITY).  W == 0 or n == 0: no-op, OK.
  * ------------------------------------------------------------------------------------------- */
 typedef struct {
-    const uint32_t *words;    /* [*nnz] packed words                           */
-    const uint32_t *nnz;      /* [1] number of words                           */
-    const int32_t *group_exp; /* [K]                                           */
+    const uint32_t *words;    /* [max_words] packed words, of which the first min(*nnz, max_words) are read  */
+    const uint32_t *nnz;      /* [1] number of words (a truncated message carries the count that was needed) */
+    const int32_t *group_exp; /* [K]                                                                          */
+    uint32_t max_words;       /* words the buffer holds: the decoder never reads past it                      */
 } vgc_message_view;
 
 vgc_status vgc_decode_accumulate(const vgc_message_view *msgs, int W,

@@ -67,6 +67,11 @@ def _load():
         lib.oracle_decode_hybrid.argtypes = [ctypes.POINTER(u32p), u32p, i, ctypes.c_float, ctypes.c_float, f32p,
                                              ctypes.c_uint64]
         lib.oracle_decode_hybrid.restype = ctypes.c_uint64
+        u8p = ctypes.POINTER(ctypes.c_uint8)
+        lib.oracle_pack_indices.argtypes = [u32p, ctypes.c_uint32, u8p, ctypes.c_uint64]
+        lib.oracle_pack_indices.restype = ctypes.c_uint64
+        lib.oracle_unpack_indices.argtypes = [u8p, ctypes.c_uint32, u32p]
+        lib.oracle_unpack_indices.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -242,3 +247,29 @@ def decode_hybrid(word_arrays, tau, scale, u):
         nnz[k] = w.size
     return int(_load().oracle_decode_hybrid(ptrs, _ptr(nnz, ctypes.c_uint32), W, float(tau), float(scale),
                                             _ptr(u, ctypes.c_float), u.size))
+
+
+PACK_RUN = 256
+
+
+def pack_indices(words) -> np.ndarray:
+    """The message's words (uint32, ascending index) with the index field stored as differences in the base-128
+    variable-length code: uint8 array [run table][payload] (Sec. 4.2, last paragraph; format in vgc_oracle.c)."""
+    words = np.ascontiguousarray(words, dtype=np.uint32)
+    lib = _load()
+    u32p, u8p = ctypes.POINTER(ctypes.c_uint32), ctypes.POINTER(ctypes.c_uint8)
+    runs = (words.size + PACK_RUN - 1) // PACK_RUN
+    out = np.zeros(4 * (runs + 1) + 5 * words.size, np.uint8)
+    size = lib.oracle_pack_indices(words.ctypes.data_as(u32p), words.size, out.ctypes.data_as(u8p), out.size)
+    assert size <= out.size
+    return out[:size].copy()
+
+
+def unpack_indices(packed, nnz: int) -> np.ndarray:
+    """Inverse of pack_indices: the nnz 32-bit words.  Raises ValueError on a malformed stream."""
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    words = np.zeros(nnz, np.uint32)
+    u32p, u8p = ctypes.POINTER(ctypes.c_uint32), ctypes.POINTER(ctypes.c_uint8)
+    if _load().oracle_unpack_indices(packed.ctypes.data_as(u8p), nnz, words.ctypes.data_as(u32p)) != 0:
+        raise ValueError("malformed index stream")
+    return words

@@ -24,14 +24,20 @@
  *   oracle_decode_accumulate    decode half of CommunicateAndUpdate (Sec. 4.3, Fig. 1 caption).
  *   oracle_compress_hybrid      Algorithm 2 (Hybrid) loop body with the variance correction of Sec. 4.5.
  *   oracle_decode_hybrid        its receiver side: every word adds +-tau.
+ *   oracle_pack_indices /       Sec. 4.2, last paragraph ("compressing parameter indexes"): the sorted 28-bit
+ *   oracle_unpack_indices       index field stored as differences in a variable-length code.  The paper names
+ *                               the idea without a format; the format is this build's (see the functions).
  *
  * Parity pins (tests/, run without a GPU): the Appendix B worked example; closed forms
  * of the Algorithm 1 state machine; equivalence of Eq. 2 with Eq. 1 via the last line of
  * Appendix A; residual accounting; brute-force per-example gradients for the squared sums;
  * for the hybrid: its reduction to the plain threshold method (alpha = 0), the "(a-b)^2" identity
  * of Sec. 4.5 on single samples, the never-send limits, agreement with Algorithm 1's test at tau = 0.
+ * For the index code: byte strings written out by hand from the rule, the exact size in closed form, round trips, and
+ * a second writing of the standard base-128 code in the tests.
  * Conventions the paper leaves open (scope of M_k, bit positions in the word, width of
- * the per-group exponent) are choices of this build: "parity unpinned" for those three.
+ * the per-group exponent, the layout of the compressed index stream) are choices of this build:
+ * "parity unpinned" for those.
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -333,4 +339,86 @@ uint64_t oracle_decode_hybrid(const uint32_t *const *words, const uint32_t *nnz,
             u[idx] = u[idx] + term;
         }
     return bad;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Index compression of a packed message (Sec. 4.2, last paragraph)           */
+/* ------------------------------------------------------------------------- */
+
+/* The words of a message are in ascending index order, so an index is the previous one plus a
+ * positive difference, and at send densities of 1e-2 .. 1e-3 the differences need 7 to 10 bits
+ * instead of 28.  Format (a choice of this build):
+ *   - the words are taken in runs of ORACLE_PACK_RUN = 256; a run starts afresh (its first
+ *     "previous index" is 0), so runs can be decoded independently of one another;
+ *   - word i of a run becomes the number  v = (idx_i - prev) << 4 | (word_i & 15)  -- the
+ *     difference above the unchanged 4-bit value field (sign, d) -- written in the standard
+ *     base-128 code: seven bits per byte, least significant group first, the top bit of a byte
+ *     set when another byte follows (1 to 5 bytes, since v < 2^32);
+ *   - the stream is  [table: (runs + 1) x uint32, little endian][payload], table[j] = offset of
+ *     run j's first byte inside the payload, table[runs] = payload length; runs = ceil(nnz/256).
+ * Returns the total size in bytes (table + payload); writes at most `capacity` bytes (a too
+ * small buffer is detected by the caller comparing the two). */
+#define ORACLE_PACK_RUN 256
+
+uint64_t oracle_pack_indices(const uint32_t *words, uint32_t nnz, uint8_t *out, uint64_t capacity)
+{
+    const uint32_t runs = (nnz + ORACLE_PACK_RUN - 1) / ORACLE_PACK_RUN;
+    const uint64_t table_bytes = 4ull * (runs + 1);
+    uint64_t at = table_bytes;                       /* next payload byte, from the start of `out` */
+    for (uint32_t j = 0; j <= runs; ++j) {
+        const uint32_t first = j * ORACLE_PACK_RUN;
+        const uint32_t offset = (uint32_t)(at - table_bytes);
+        for (int b = 0; b < 4; ++b)                  /* table entry j, little endian */
+            if (4ull * j + b < capacity) out[4ull * j + b] = (uint8_t)(offset >> (8 * b));
+        if (j == runs) break;
+        uint32_t prev = 0;
+        for (uint32_t i = first; i < nnz && i < first + ORACLE_PACK_RUN; ++i) {
+            const uint32_t idx = words[i] >> 4;
+            uint32_t v = ((idx - prev) << 4) | (words[i] & 15u);
+            prev = idx;
+            for (;;) {
+                const uint8_t low = (uint8_t)(v & 0x7Fu);
+                v >>= 7;
+                if (at < capacity) out[at] = (uint8_t)(low | (v ? 0x80u : 0u));
+                ++at;
+                if (!v) break;
+            }
+        }
+    }
+    return at;
+}
+
+/* The inverse: rebuilds the `nnz` 32-bit words from a stream written by the rule above.
+ * Returns 0, or -1 when the stream is malformed (a number longer than five bytes, or a run
+ * that does not end where the table says). */
+int oracle_unpack_indices(const uint8_t *in, uint32_t nnz, uint32_t *words)
+{
+    const uint32_t runs = (nnz + ORACLE_PACK_RUN - 1) / ORACLE_PACK_RUN;
+    const uint64_t table_bytes = 4ull * (runs + 1);
+    for (uint32_t j = 0; j < runs; ++j) {
+        uint32_t begin = 0, end = 0;
+        for (int b = 0; b < 4; ++b) {
+            begin |= (uint32_t)in[4ull * j + b] << (8 * b);
+            end |= (uint32_t)in[4ull * (j + 1) + b] << (8 * b);
+        }
+        uint64_t at = table_bytes + begin;
+        uint32_t prev = 0;
+        const uint32_t first = j * ORACLE_PACK_RUN;
+        for (uint32_t i = first; i < nnz && i < first + ORACLE_PACK_RUN; ++i) {
+            uint32_t v = 0;
+            int shift = 0;
+            for (;;) {
+                const uint8_t byte = in[at++];
+                if (shift > 28) return -1;
+                v |= (uint32_t)(byte & 0x7Fu) << shift;
+                shift += 7;
+                if (!(byte & 0x80u)) break;
+            }
+            const uint32_t idx = prev + (v >> 4);
+            words[i] = (idx << 4) | (v & 15u);
+            prev = idx;
+        }
+        if (at != table_bytes + end) return -1;
+    }
+    return 0;
 }

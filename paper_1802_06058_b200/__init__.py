@@ -27,13 +27,13 @@ EXPORTS = [
     "vgc_status_string", "vgc_version", "vgc_kernel_launch_count",
     "vgc_sqgrad_linear_workspace_bytes", "vgc_sqgrad_linear",
     "vgc_sqgrad_conv_workspace_bytes", "vgc_sqgrad_conv",
-    "vgc_sqgrad_conv_batch_workspace_bytes", "vgc_sqgrad_conv_batch", "vgc_sqgrad_plan_hint",
+    "vgc_sqgrad_conv_batch_workspace_bytes", "vgc_sqgrad_conv_batch",
     "vgc_sqgrad_conv_exact_workspace_bytes", "vgc_sqgrad_conv_exact",
     "vgc_sqgrad_conv_exact_batch_workspace_bytes", "vgc_sqgrad_conv_exact_batch",
     "vgc_compress_workspace_bytes", "vgc_compress", "vgc_compress_static",
     "vgc_decode_accumulate", "vgc_step_host",
     "vgc_compress_hybrid_workspace_bytes", "vgc_compress_hybrid", "vgc_decode_accumulate_hybrid",
-    "vgc_decode_sum", "vgc_decode_sum_hybrid", "vgc_probe_mma_rate",
+    "vgc_decode_sum", "vgc_decode_sum_hybrid",
 ]
 
 
@@ -62,7 +62,8 @@ class _HybridMessageStruct(ctypes.Structure):    # mirrors vgc_hybrid_message
 
 
 class _ViewStruct(ctypes.Structure):         # mirrors vgc_message_view
-    _fields_ = [("words", ctypes.c_void_p), ("nnz", ctypes.c_void_p), ("group_exp", ctypes.c_void_p)]
+    _fields_ = [("words", ctypes.c_void_p), ("nnz", ctypes.c_void_p), ("group_exp", ctypes.c_void_p),
+                ("max_words", ctypes.c_uint32)]
 
 
 _lib = None
@@ -93,9 +94,6 @@ def load_library():
     lib.vgc_sqgrad_conv_batch_workspace_bytes.restype = sz
     lib.vgc_sqgrad_conv_batch.argtypes = [i, vp, vp, vp] + [i] * 11 + [f, i, vp, sz, vp]
     lib.vgc_sqgrad_conv_batch.restype = i
-    lib.vgc_sqgrad_plan_hint.argtypes = [i]; lib.vgc_sqgrad_plan_hint.restype = None
-    lib.vgc_probe_mma_rate.argtypes = [i, i, i, i, i, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
-    lib.vgc_probe_mma_rate.restype = i
     lib.vgc_sqgrad_conv_exact_workspace_bytes.argtypes = [i] * 11
     lib.vgc_sqgrad_conv_exact_workspace_bytes.restype = sz
     lib.vgc_sqgrad_conv_exact.argtypes = lib.vgc_sqgrad_conv.argtypes
@@ -242,21 +240,6 @@ def vgc_sqgrad_conv_exact(x, delta, kernel, stride, padding, scale: float, S, ac
     return S
 
 
-def vgc_sqgrad_plan_hint(concurrent_launches: int) -> None:
-    """Tell the planner how many sqgrad calls run side by side (streams with separate workspaces)."""
-    load_library().vgc_sqgrad_plan_hint(int(concurrent_launches))
-
-
-def vgc_probe_mma_rate(kind: int, a_tmem: bool, n: int, reps: int = 4096, blocks: int = 148):
-    """(cycles per tcgen05.mma instruction on one SM, TFLOP/s of the whole launch) for M = 128, N = n;
-    kind 0 = tf32, 1 = bf16."""
-    cycles, tflops = ctypes.c_double(0.0), ctypes.c_double(0.0)
-    st = load_library().vgc_probe_mma_rate(int(kind), int(bool(a_tmem)), int(n), int(reps), int(blocks),
-                                           ctypes.byref(cycles), ctypes.byref(tflops))
-    _check(st, "vgc_probe_mma_rate")
-    return cycles.value, tflops.value
-
-
 def vgc_sqgrad_conv_batch_workspace_bytes(n_layers, B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, exact: bool = False) -> int:
     lib = load_library()
     fn = lib.vgc_sqgrad_conv_exact_batch_workspace_bytes if exact else lib.vgc_sqgrad_conv_batch_workspace_bytes
@@ -321,7 +304,8 @@ class MessageBuffers:
                               self.mask.data_ptr() if self.mask is not None else None, c + 12)
 
     def view(self) -> _ViewStruct:
-        return _ViewStruct(self.words.data_ptr(), self.counters.data_ptr(), self.group_exp.data_ptr())
+        return _ViewStruct(self.words.data_ptr(), self.counters.data_ptr(), self.group_exp.data_ptr(),
+                           min(self.capacity, self.words.numel()))
 
     def read(self):
         """Device -> host copy (synchronises): dict with words (numpy uint32), group_exp, counters."""
@@ -388,7 +372,8 @@ def vgc_decode_accumulate(messages: Sequence, group_offsets, scale: float, u, de
                           overwrite: bool = False):
     """u[idx] += scale * decoded value over all words of all messages.
 
-    ``messages``: MessageBuffers objects, or (words int32, nnz int32[1], group_exp int32) tensor triples.
+    ``messages``: MessageBuffers objects, or (words int32, nnz int32[1], group_exp int32) tensor triples; the
+    decoder reads at most as many words as the words tensor holds.
     ``dev_status``: int32[1] device tensor (zeroed by the caller) receiving VGC_DEV_* bits.
     ``overwrite``: write u = scale * sum instead (vgc_decode_sum): u is neither read nor needs clearing."""
     W = len(messages)
@@ -399,7 +384,7 @@ def vgc_decode_accumulate(messages: Sequence, group_offsets, scale: float, u, de
         else:
             words, nnz, gexp = m
             views[w] = _ViewStruct(_dev(words, torch.int32, "words"), _dev(nnz, torch.int32, "nnz"),
-                                   _dev(gexp, torch.int32, "group_exp"))
+                                   _dev(gexp, torch.int32, "group_exp"), words.numel())
     K = group_offsets.numel() - 1
     lib = load_library()
     fn = lib.vgc_decode_sum if overwrite else lib.vgc_decode_accumulate
@@ -430,7 +415,7 @@ class HybridMessageBuffers:
                                     self.mask.data_ptr() if self.mask is not None else None, c + 4)
 
     def view(self) -> _ViewStruct:
-        return _ViewStruct(self.words.data_ptr(), self.counters.data_ptr(), None)
+        return _ViewStruct(self.words.data_ptr(), self.counters.data_ptr(), None, min(self.capacity, self.words.numel()))
 
     def read(self):
         nnz, dev_status = (int(c) & 0xFFFFFFFF for c in self.counters.tolist())
@@ -475,7 +460,7 @@ def vgc_decode_accumulate_hybrid(messages: Sequence, tau: float, scale: float, u
             views[w] = m.view()
         else:
             words, nnz = m
-            views[w] = _ViewStruct(_dev(words, torch.int32, "words"), _dev(nnz, torch.int32, "nnz"), None)
+            views[w] = _ViewStruct(_dev(words, torch.int32, "words"), _dev(nnz, torch.int32, "nnz"), None, words.numel())
     lib = load_library()
     fn = lib.vgc_decode_sum_hybrid if overwrite else lib.vgc_decode_accumulate_hybrid
     st = fn(views, W, float(tau), float(scale), _dev(u, torch.float32, "u"), u.numel(),

@@ -2,6 +2,8 @@
 // shape occupies the tensor pipe of an SM.  The squared-gradient contraction is bounded by this figure, not by the
 // nominal flop rate: an instruction with M = 128 takes the same time for N = 64 and N = 128, so the ceiling of a
 // kernel depends on the instruction shape it can use.  `bench.py --mma-rates` prints the table.
+// Not part of libvgc.so: built on request into libvgc_probe.so (paper_1802_06058_b200._build.build_probe) and loaded by
+// the benchmark only.
 //
 // One CTA per block issues `reps` back-to-back MMAs (operands: zeros in shared / tensor memory, one accumulator),
 // then commits and waits -- bounded -- for them to retire; the cycle count of block 0 and the event time of the
@@ -102,7 +104,7 @@ __global__ void __launch_bounds__(128, 1) mma_rate(int kind, int a_tmem, int n, 
 
 }  // namespace vgc
 
-extern "C" vgc_status vgc_probe_mma_rate(int kind, int a_tmem, int n, int reps, int blocks, double *cycles_per_mma,
+extern "C" int vgc_probe_mma_rate(int kind, int a_tmem, int n, int reps, int blocks, double *cycles_per_mma,
                                          double *tflops)
 {
     using namespace vgc;
@@ -118,7 +120,7 @@ extern "C" vgc_status vgc_probe_mma_rate(int kind, int a_tmem, int n, int reps, 
     VGC_CUDA_OK(cudaMalloc(&d_cycles, 16));
     uint32_t *d_status = reinterpret_cast<uint32_t *>(d_cycles + 1);
     cudaEvent_t e0 = nullptr, e1 = nullptr;
-    vgc_status rc = VGC_ERR_CUDA;
+    int rc = VGC_ERR_CUDA;
     float ms = 0.f;
     long long h[2] = {0, 0};
     if (cudaMemset(d_cycles, 0, 16) == cudaSuccess && cudaEventCreate(&e0) == cudaSuccess && cudaEventCreate(&e1) == cudaSuccess) {
@@ -126,7 +128,6 @@ extern "C" vgc_status vgc_probe_mma_rate(int kind, int a_tmem, int n, int reps, 
         cudaEventRecord(e0);
         probe::mma_rate<<<blocks, 128, probe::kSmem>>>(kind, a_tmem, n, reps, d_cycles, d_status);
         cudaEventRecord(e1);
-        count_launch(2);
         if (cudaDeviceSynchronize() == cudaSuccess && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess &&
             cudaMemcpy(h, d_cycles, 16, cudaMemcpyDeviceToHost) == cudaSuccess)
             rc = (uint32_t)h[1] ? VGC_ERR_CUDA : VGC_OK;

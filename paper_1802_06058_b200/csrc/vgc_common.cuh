@@ -21,10 +21,15 @@ inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// VGC_DEBUG=1 in the environment: a failing CUDA call is named on stderr before the status is returned
+// VGC_DEBUG=1 in the environment (read once): a failing CUDA call is named on stderr before the status is returned
+inline bool debug_enabled()
+{
+    static const bool on = getenv("VGC_DEBUG") != nullptr;
+    return on;
+}
 inline void report_cuda_error(cudaError_t e, const char *what, const char *file, int line)
 {
-    if (getenv("VGC_DEBUG")) fprintf(stderr, "vgc: %s:%d: %s -> %s\n", file, line, what, cudaGetErrorString(e));
+    if (debug_enabled()) fprintf(stderr, "vgc: %s:%d: %s -> %s\n", file, line, what, cudaGetErrorString(e));
 }
 #define VGC_CUDA_OK(expr)                                                  \
     do {                                                                   \

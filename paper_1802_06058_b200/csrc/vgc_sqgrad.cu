@@ -10,7 +10,6 @@ vgc_status simt_sqgrad_linear(const float *x, const float *delta, int B, int in,
 vgc_status simt_sqgrad_conv(const float *x, const float *delta, int B, int C, int H, int W, int Cout,
                             int Kh, int Kw, int sh, int sw, int ph, int pw, int Ho, int Wo, float scale,
                             int accumulate, float *S, void *ws, size_t ws_bytes, cudaStream_t st);
-void tc_plan_hint(int concurrent_launches);
 bool tc_linear_supported(int B, int in, int out);
 bool tc_conv_supported(int B, int C, int H, int W, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw);
 size_t tc_linear_workspace_bytes(int B, int in, int out);
@@ -26,11 +25,12 @@ vgc_status tc_sqgrad_conv(int n_layers, const float *const *x, const float *cons
 using namespace vgc;
 
 namespace {
-// VGC_SQGRAD_PATH=simt forces the CUDA-core kernel (cross-checks, shapes under suspicion)
-bool use_tensor_cores()
+// B == 0: the sum over the mini-batch is empty -- S is cleared (accumulate == 0) or left alone
+vgc_status empty_batch(float *const *S, int n_layers, size_t n_weights, int accumulate, cudaStream_t st)
 {
-    const char *e = getenv("VGC_SQGRAD_PATH");
-    return !(e && e[0] == 's');
+    if (!accumulate)
+        for (int l = 0; l < n_layers; ++l) VGC_CUDA_OK(cudaMemsetAsync(S[l], 0, n_weights * sizeof(float), st));
+    return VGC_OK;
 }
 
 bool conv_shape_ok(int B, int C, int H, int W, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw,
@@ -63,9 +63,10 @@ extern "C" vgc_status vgc_sqgrad_linear(const float *x, const float *delta, int 
     if (!S || !aligned16(S)) return VGC_ERR_INVALID_ARG;
     if (B > 0 && (!x || !delta || !aligned16(x) || !aligned16(delta))) return VGC_ERR_INVALID_ARG;
     if (!(scale == scale)) return VGC_ERR_INVALID_ARG;
-    if (ws_bytes < vgc_sqgrad_linear_workspace_bytes(B, in, out) || (ws_bytes && !ws)) return VGC_ERR_WORKSPACE;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    if (use_tensor_cores() && tc_linear_supported(B, in, out))
+    if (B == 0) return empty_batch(&S, 1, (size_t)in * out, accumulate, st);
+    if (ws_bytes < vgc_sqgrad_linear_workspace_bytes(B, in, out) || !ws) return VGC_ERR_WORKSPACE;
+    if (tc_linear_supported(B, in, out))
         return tc_sqgrad_linear(x, delta, B, in, out, scale, accumulate, S, ws, ws_bytes, st);
     return simt_sqgrad_linear(x, delta, B, in, out, scale, accumulate, S, static_cast<char *>(ws) + 256,
                               ws_bytes - 256, st);
@@ -105,12 +106,13 @@ extern "C" vgc_status vgc_sqgrad_conv_batch(int n_layers, const float *const *x,
         if (!S[l] || !aligned16(S[l])) return VGC_ERR_INVALID_ARG;
         if (B > 0 && (!x[l] || !delta[l] || !aligned16(x[l]) || !aligned16(delta[l]))) return VGC_ERR_INVALID_ARG;
     }
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (B == 0) return empty_batch(S, n_layers, (size_t)Cout * C * Kh * Kw, accumulate, st);
     if (ws_bytes < vgc_sqgrad_conv_batch_workspace_bytes(n_layers, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h,
                                                          pad_w) ||
-        (ws_bytes && !ws))
+        !ws)
         return VGC_ERR_WORKSPACE;
-    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    if (B > 0 && use_tensor_cores() && tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w))
+    if (tc_conv_supported(B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w))
         return tc_sqgrad_conv(n_layers, x, delta, S, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, Ho, Wo,
                               scale, accumulate, ws, ws_bytes, st);
     for (int l = 0; l < n_layers; ++l) {        // CUDA-core kernel: layer after layer
@@ -180,8 +182,6 @@ extern "C" vgc_status vgc_sqgrad_conv_exact(const float *x, const float *delta, 
                                        accumulate, ws, ws_bytes, stream);
 }
 
-extern "C" void vgc_sqgrad_plan_hint(int concurrent_launches) { tc_plan_hint(concurrent_launches); }
-
 extern "C" const char *vgc_status_string(int status)
 {
     switch (status) {
@@ -194,7 +194,7 @@ extern "C" const char *vgc_status_string(int status)
     }
 }
 
-extern "C" int vgc_version(void) { return 1000; }
+extern "C" int vgc_version(void) { return 2000; }
 
 namespace vgc { unsigned long long g_launches = 0; }
 extern "C" uint64_t vgc_kernel_launch_count(void) { return vgc::g_launches; }

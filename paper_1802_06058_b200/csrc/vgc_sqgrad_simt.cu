@@ -174,6 +174,7 @@ template <class Ops>
 vgc_status simt_launch(const Ops &ops, int M, int N, int K, float scale, int accumulate, float *S,
                        void *ws, size_t ws_bytes, cudaStream_t st)
 {
+    if (M <= 0 || N <= 0 || K <= 0) return VGC_ERR_INVALID_ARG;     // empty sums are the caller's business
     int splits = simt_splits(M, N, K);
     if (splits > 1 && ws_bytes < (size_t)splits * M * N * sizeof(float)) return VGC_ERR_WORKSPACE;
     int k_per_split = (K + splits - 1) / splits;

@@ -17,7 +17,11 @@
 // The tensor core's fp32 accumulation is not trusted over long reductions: every kChunk k slices
 // the accumulator is drained by four epilogue warps (tcgen05.ld) and added, round-to-nearest, to
 // fp32 registers while the next chunk accumulates into the second TMEM buffer.
-// Long reductions are split across blockIdx.z; partial tiles are combined in a fixed order.
+// Work distribution: the (layer, tile, k slice) space of a launch is laid out linearly and cut into one
+// contiguous range per thread block, with at most one block per SM; a block walks its range segment by
+// segment (a segment = consecutive slices of one output tile) with the pipeline running across segment
+// borders.  A segment that covers a tile's whole reduction writes the result; otherwise it writes a partial
+// tile to scratch and a second kernel adds the partial tiles of a tile in a fixed order.
 //
 // Operand layouts:
 //   dense layer: A = delta[z][out], B = x[z][in]  (m / n innermost: MN-major tiles, both by TMA)
@@ -31,6 +35,7 @@
 //                im2col rows become the 128-row A tile and the errors the narrow B tile.
 //
 // Warp roles (448 threads): 0 TMA producer, 1 MMA issuer + TMEM owner, 2-9 transform, 10-13 epilogue.
+// While the epilogue warps write a segment's tile out, the other roles are already working on the next one.
 // Every wait on an mbarrier is bounded; on expiry the block raises an abort flag, all roles fall
 // through to the common exit, outstanding TMA loads are waited for (bounded) and TMEM is freed.
 #include <cuda.h>
@@ -75,11 +80,6 @@ constexpr int kLoSlotsAT = 2 * kLoSlots;
 // early, and the 16-KB units this saves hold more B tiles: more slices in flight from the same shared memory.
 constexpr int kSplitA = 4, kSplitB = 7, kSplitLo = 3;              // 16-KB units: A raw, B raw/hi, B lo (+ A in TMEM)
 static_assert((kSplitA + kSplitB + kSplitLo) * kRawBytesA <= (kRawSlots + kLoSlots) * kRawStageBytes, "smem budget");
-// Pair form (two CTAs of a cluster share one 256 x 128 tile, tcgen05 cta_group::2): each CTA holds its own 128 A rows
-// and half of the B rows, so a B slot is 8 KB and the rings get deeper: A raw, B raw/hi, B bf16 (+ A in TMEM)
-constexpr int kPairA = 8, kPairB = 8, kPairLo = 4;
-constexpr uint32_t kPairBBytes = kRawBytesB / 2;
-static_assert(kPairA * kRawBytesA + (kPairB + kPairLo) * kPairBBytes <= (kRawSlots + kLoSlots) * kRawStageBytes, "smem budget");
 constexpr uint32_t kTmemColsA = 64;                                 // per slot: 32 columns hi + 32 columns lo
 constexpr uint32_t kTmemCols = 512;                                 // two accumulator buffers + the A operand ring
 constexpr uint32_t kWaitLimit = 1u << 22;                           // polls before a wait gives up
@@ -95,21 +95,22 @@ enum { kTma = 0, kGatherErr = 1, kGatherIm2col = 2, kGatherTaps4 = 3, kGatherTap
 
 struct Params {
     int M, N;                // rows of the A tile space / of the B tile space
-    int k_slices;            // total 32-deep slices of the reduction
-    int slices_per_split;
+    int k_slices;            // 32-deep slices of one tile's reduction
     int p_slices;            // conv: slices per example (ceil(P/32)); dense: 1
     int chunk;               // slices per accumulator drain
+    int unit;                // slices that stay in one block: the reduction is cut between units only
+    int units_per_tile;      // k_slices / unit
+    long long units_total;   // layers * tiles * units_per_tile: the launch's work, cut evenly over the blocks
+    int tiles_x, tiles_y;    // 128-column / 128-row tiles of one layer's result
     uint32_t tx_bytes;       // bytes the TMA loads of one slice deliver
     uint32_t tx_bytes_a;     // of which the A tile's
     float scale;
     int accumulate;
-    int tiles_x;             // 128-column tiles of the output (wide form: the scratch is indexed in these)
-    int splits;              // blocks along the reduction per layer (blockIdx.z = layer * splits + split)
     int C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, Wo, P;     // conv geometry (gathered tiles)
     int chw;                 // C*H*W
     unsigned wo_magic;       // floor(2^32 / Wo) + 1: p / Wo == umulhi(p, wo_magic) for p * Wo < 2^32
     long long ld_m, ld_n;    // result: element (m, n) lives at S[m*ld_m + n*ld_n]; one of the two is 1
-    float *partial;          // split-K scratch [layer][split][tile][column][row], used when splits > 1
+    float *partial;          // scratch for partial tiles [2 * block + (0: a block's first segment, 1: its last)][column][row]
     uint32_t *status;        // device word; VGC_DEV_TIMEOUT is OR-ed in if a wait expired
 };
 
@@ -188,63 +189,6 @@ __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// ---- cluster of two CTAs (pair form) ----
-__device__ __forceinline__ uint32_t cluster_ctarank()
-{
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// arrive on the barrier at the same shared-memory offset in CTA `rank` of the cluster.  No cluster-scope release: what
-// the arrival publishes is read by the tensor core of the writing CTA (its shared memory after fence.proxy.async, its
-// tensor memory after tcgen05.wait::st), not by the other CTA's threads, and a cluster-wide release costs a full
-// memory barrier per arrival (measured: the pair form then runs 1.4x slower than single CTAs).
-__device__ __forceinline__ void mbar_arrive_cta(uint32_t bar, uint32_t rank)
-{
-    asm volatile(
-        "{\n\t.reg .b32 rem;\n\t"
-        "mapa.shared::cluster.u32 rem, %0, %1;\n\t"
-        "mbarrier.arrive.shared::cluster.b64 _, [rem];\n\t}"
-        ::"r"(bar), "r"(rank)
-        : "memory");
-}
-// commit of cta_group::2 MMAs: arrives on the barrier at this offset in both CTAs of the pair
-__device__ __forceinline__ void tc_commit_pair(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"((uint16_t)3)
-                 : "memory");
-}
-__device__ __forceinline__ void tc_commit_pair_local(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// cta_group::2, A from tensor memory: D (256 rows over the two CTAs) (+)= A * B, B rows split between the CTAs
-__device__ __forceinline__ void tc_mma_pair_tf32_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                                    uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void tc_mma_pair_bf16_ts_acc(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.eq.u32 p, 1, 1;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc)
-        : "memory");
-}
-
 __device__ __forceinline__ void tc_mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                             uint32_t accumulate)
 {
@@ -706,6 +650,52 @@ struct Gatherer<kMode, kHalf, true> {
     }
 };
 
+// ---- work distribution -----------------------------------------------------------------------
+// One segment of a block's range: slices [s_begin, s_end) of the reduction of one output tile.
+struct Seg {
+    int layer, m0, n0;       // layer of the batch, first row / column of the tile
+    int n_valid, n_act;      // columns of the tile that exist; the MMAs' N (rounded up to a multiple of 16)
+    int s_begin, s_end;
+    bool whole;              // the segment is the tile's whole reduction: its block writes the result itself
+    int slot;                // otherwise: which partial tile of the scratch it writes
+};
+
+// The launch's work is the sequence (layer, tile, unit of the tile's reduction), units_total long; block b owns
+// units [b U / G, (b + 1) U / G).  Every role of a block walks the same segments with an iterator of its own.
+struct SegIter {
+    long long pos, end;
+    int index;
+    __device__ __forceinline__ SegIter(const Params &prm)
+    {
+        pos = (long long)blockIdx.x * prm.units_total / gridDim.x;
+        end = (long long)(blockIdx.x + 1) * prm.units_total / gridDim.x;
+        index = 0;
+    }
+    __device__ __forceinline__ bool next(const Params &prm, Seg &sg)
+    {
+        if (pos >= end) return false;
+        const int upt = prm.units_per_tile;
+        const long long tile = pos / upt;
+        const int u0 = (int)(pos - tile * upt);
+        const int u1 = end - tile * upt < upt ? (int)(end - tile * upt) : upt;
+        const int tiles_layer = prm.tiles_x * prm.tiles_y;
+        sg.layer = (int)(tile / tiles_layer);
+        const int rem = (int)(tile - (long long)sg.layer * tiles_layer);
+        const int tile_m = rem / prm.tiles_x, tile_n = rem - tile_m * prm.tiles_x;
+        sg.m0 = tile_m * kBM;
+        sg.n0 = tile_n * kBN;
+        sg.n_valid = min(kBN, prm.N - sg.n0);
+        sg.n_act = (sg.n_valid + 15) & ~15;
+        sg.s_begin = u0 * prm.unit;
+        sg.s_end = u1 * prm.unit;
+        sg.whole = u0 == 0 && u1 == upt;
+        sg.slot = 2 * (int)blockIdx.x + (index > 0 ? 1 : 0);     // a block's partial segments: its first and / or its last
+        pos += u1 - u0;
+        ++index;
+        return true;
+    }
+};
+
 // ---- the kernel ------------------------------------------------------------------------------
 // kExact: the per-example statistic of a conv layer, S = scale * sum_z (sum_p delta x)^2 -- operands are split without
 // squaring, an accumulator is drained at least at every example's end, the epilogue sums the drains of one example
@@ -714,20 +704,7 @@ struct Gatherer<kMode, kHalf, true> {
 // tensor-pipe time of a tf32 product each; their rounding, 2^-9 relative on a term that is itself 2^-11 of the
 // product, stays below 2^-18 of the result).  A lo slot then holds [B hi as bf16][B lo as bf16], 8 KB each with
 // 64-byte rows, and an A slot in tensor memory [hi tf32: 32 columns][hi bf16: 16][lo bf16: 16].
-// kPair: two CTAs of a cluster (neighbours along the grid's x, which holds the row tiles in this form) work on one 256 x 128 tile with cta_group::2 MMAs.
-// Each keeps its own 128 rows of A (tensor memory) and of the accumulators and loads / transforms only half of
-// the B rows, which halves the B share of the shared-memory traffic.  The even CTA issues the MMAs; the transform and
-// epilogue warps of the odd one signal its barriers through the cluster's shared-memory window, and a commit
-// arrives on the barriers of both.
-// kWide (a pair form): the pair's tile is 256 x 256 and its instructions have N = 256, the shape at which the tensor
-// pipe delivers its full rate (an instruction takes 138 cycles there against 96 - 110 for any N up to 128).  Each CTA
-// holds 128 of the 256 B rows, i.e. the tiles, rings and transform load of the single-CTA kernel.  Tensor memory has room
-// for one accumulator of 256 columns next to the A ring, so chunks are not double-buffered: the MMAs pause while a chunk
-// is drained.  The epilogue keeps no running sums (256 per lane do not fit in registers): it stores the first chunk to
-// the split-K scratch and adds the later ones there with red.global.add (one thread per address, in program order), and
-// the combine kernel, which always runs in this form, writes the result.
-template <int kMajor, int kModeA, int kModeB, bool kATmem, bool kExact = false, bool kBf = false, bool kPair = false,
-          bool kWide = false>
+template <int kMajor, int kModeA, int kModeB, bool kATmem, bool kExact = false, bool kBf = false>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
 {
@@ -738,16 +715,12 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
     constexpr bool kAnyGather = kGatherA || kGatherB;
     constexpr bool kSplit = kATmem && !kAnyGather;                         // A raw tiles in a ring of their own
     static_assert(!kBf || (kSplit && !kExact), "bf16 cross terms: the TMA-fed form with A in tensor memory");
-    static_assert(!kPair || kBf, "the pair form exists for the TMA-fed form with bf16 cross terms");
-    static_assert(!kWide || kPair, "N = 256 instructions are issued by CTA pairs");
-    constexpr bool kHalfB = kPair && !kWide;                               // this CTA's B tile has 64 rows (else 128)
-    constexpr int kTileN = kWide ? 2 * kBN : kBN;                          // columns of the block's (pair's) output tile
-    constexpr int kNA = kHalfB ? kPairA : kSplitA;                         // slots of the raw A ring (split form)
+    constexpr int kNA = kSplitA;                                           // slots of the raw A ring (split form)
     // the transform warps work as two groups of four on alternate slices (else all eight on every slice)
     constexpr bool kTwoGroups = !kAnyGather || (IsTaps<kModeB>::value && kModeA == kTma);
-    constexpr int kNB = kHalfB ? kPairB : kSplit ? kSplitB : kRawSlots;    // slots of the raw / hi ring
+    constexpr int kNB = kSplit ? kSplitB : kRawSlots;                      // slots of the raw / hi ring
     // lo slots (and A slots in TMEM); the per-example form needs 128 TMEM columns for its sum of squares
-    constexpr int kLoN = kHalfB ? kPairLo : (kExact && kATmem) ? 2 : kSplit ? kSplitLo : (kATmem ? kLoSlotsAT : kLoSlots);
+    constexpr int kLoN = (kExact && kATmem) ? 2 : kSplit ? kSplitLo : (kATmem ? kLoSlotsAT : kLoSlots);
     constexpr uint32_t kSqCol = 2 * kBN + (kATmem ? 2 * kTmemColsA : 0);         // where that sum lives
     constexpr uint32_t kLoBytes = kATmem ? kRawBytesB : kRawStageBytes;  // bytes of one lo slot
     // byte offsets of slot s: the [A][B] pair of the raw / hi ring (split form: only its B half exists, the
@@ -757,18 +730,13 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         return kSplit ? (uint32_t)(kSplitA + kSplitB + s - 1) * kRawBytesA
                       : kLoBase + (uint32_t)s * kLoBytes - (kATmem ? kRawBytesA : 0u);
     };
-
     // bf16-cross form: where the B tile of raw slot s and the [hi bf16][lo bf16] tiles of lo slot s live
-    auto b_tile = [&](int s) -> uint32_t {
-        return kHalfB ? (uint32_t)kPairA * kRawBytesA + (uint32_t)s * kPairBBytes : pair_off(s) + kRawBytesA;
-    };
-    auto bf_tile = [&](int s) -> uint32_t {
-        return kHalfB ? (uint32_t)kPairA * kRawBytesA + (uint32_t)(kPairB + s) * kPairBBytes : lo_off(s) + kRawBytesA;
-    };
-    constexpr uint32_t kBTile = kHalfB ? kPairBBytes : kRawBytesB;         // bytes of this CTA's B tile
+    auto b_tile = [&](int s) -> uint32_t { return pair_off(s) + kRawBytesA; };
+    auto bf_tile = [&](int s) -> uint32_t { return lo_off(s) + kRawBytesA; };
+    constexpr uint32_t kBTile = kRawBytesB;
 
     extern __shared__ uint8_t smem_raw_[];
-    __shared__ __align__(8) uint64_t bars[3 * kPairB + kLoSlotsAT + 5 + 2 * kPairA];
+    __shared__ __align__(8) uint64_t bars[3 * kSplitB + kLoSlotsAT + 5 + 2 * kSplitA];
     __shared__ uint32_t tmem_base_slot;
     __shared__ volatile uint32_t abort_flag;
 
@@ -783,33 +751,12 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
     uint64_t *lo_empty = bars + 3 * kNB;
     uint64_t *acc_full = lo_empty + kLoSlotsAT, *acc_empty = acc_full + 2, *drain = acc_empty + 2;
     uint64_t *a_full = drain + 1, *a_empty = a_full + kNA;                 // split form: the A ring
-    // pair form: rank of this CTA in its cluster; rank 0 issues the MMAs and owns the barriers that both CTAs signal
-    const uint32_t cta_rank = kPair ? cluster_ctarank() : 0u;
-
-    // tile coordinates: columns along the grid's x, rows along y; the pair form has them the other way round because
-    // the two CTAs of a pair, neighbours in rows, must be neighbours along x
-    const int tile_n = kPair ? (int)blockIdx.y : (int)blockIdx.x, tile_m = kPair ? (int)blockIdx.x : (int)blockIdx.y;
-    const int tiles_n = kPair ? (int)gridDim.y : (int)gridDim.x;
-    const int m0 = tile_m * kBM, n0 = tile_n * kTileN;
-    const int n_valid = min(kTileN, prm.N - n0);                           // columns of this tile that exist
-    const int n_act = kPair ? (n_valid + 31) & ~31 : (n_valid + 15) & ~15; // UMMA N (multiple of 16; of 32 for a pair)
-    const int layer = (int)blockIdx.z / prm.splits, split = (int)blockIdx.z - layer * prm.splits;
-    const CUtensorMap *map_a = &bt.a[layer], *map_b = &bt.b[layer];
-    float *const S = bt.S[layer];
-    const int slice_begin = split * prm.slices_per_split;
-    const int slice_end = min(prm.k_slices, slice_begin + prm.slices_per_split);
-    const int n_slices = slice_end - slice_begin;                           // >= 1 by construction
-    // an accumulator is drained every prm.chunk slices, and (kExact) at the end of every example: the block's
-    // slices are segments of seg_len slices (whole examples -- the split is planned that way), each cut into cps chunks
-    const int seg_len = kExact ? prm.p_slices : n_slices;
-    const int cps = (seg_len + prm.chunk - 1) / prm.chunk;
-    const int n_chunks = (n_slices / seg_len) * cps;
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int i = 0; i < kNB; ++i) {
             mbar_init(smem_u32(&raw_full[i]), 1);
-            mbar_init(smem_u32(&op_full[i]), (kPair ? 2 : 1) * (kTwoGroups ? kTransformWarps / 2 : kTransformWarps));
+            mbar_init(smem_u32(&op_full[i]), kTwoGroups ? kTransformWarps / 2 : kTransformWarps);
             mbar_init(smem_u32(&empty[i]), 1);
         }
         if (kSplit)
@@ -818,70 +765,68 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                 mbar_init(smem_u32(&a_empty[i]), kTransformWarps / 2);
             }
         for (int i = 0; i < kLoSlotsAT; ++i) mbar_init(smem_u32(&lo_empty[i]), 1);      // unused, kept initialised
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&acc_full[i]), 1); mbar_init(smem_u32(&acc_empty[i]), (kPair ? 2 : 1) * kEpilogueWarps); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&acc_full[i]), 1); mbar_init(smem_u32(&acc_empty[i]), kEpilogueWarps); }
         mbar_init(smem_u32(drain), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {      // TMEM: this warp allocates and, at the end, frees
-        if (kPair) {       // the same warp of both CTAs allocates for the pair
-            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
-                         "r"(kTmemCols)
-                         : "memory");
-            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-        } else {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
                      "r"(kTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-        }
     }
     tc_fence_before();
     __syncthreads();
-    if (kPair) cluster_sync_all();      // the other CTA's barriers are initialised before anything arrives on them
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
 
+    // `it` below is the running number of a slice within this block (over all of its segments): ring slots and
+    // barrier phases follow it, so the pipeline does not drain between segments.
     if (warp == 0) {
         // ================= TMA producer (one thread) =================
         if (lane == 0 && kAnyTma) {
-            int issued = 0;
-            for (int i = 0; i < n_slices; ++i) {
-                const int st = i % kNB;
-                const uint32_t ph = (uint32_t)(i / kNB) & 1u;
-                if (!mbar_wait(smem_u32(&empty[st]), ph ^ 1u, &abort_flag, 64)) break;
-                const uint32_t full = smem_u32(&raw_full[st]);
-                const uint32_t dst_a = smem_base + pair_off(st), dst_b = dst_a + kRawBytesA;
-                const int slice = slice_begin + i;
-                if (kSplit) {
-                    const int sa = i % kNA;
-                    if (!mbar_wait(smem_u32(&a_empty[sa]), ((uint32_t)(i / kNA) & 1u) ^ 1u, &abort_flag, 64)) break;
-                    const uint32_t full_a = smem_u32(&a_full[sa]);
-                    const int z = slice / prm.p_slices, p0 = (slice - z * prm.p_slices) * kBK;
-                    mbar_expect_tx(full_a, prm.tx_bytes_a);
-                    tma_load_3d(smem_base + (uint32_t)sa * kRawBytesA, map_a, full_a, p0, m0, z);
-                    mbar_expect_tx(full, prm.tx_bytes - prm.tx_bytes_a);
-                    // pair form: this CTA's half of the tile's B rows
-                    if (kBf) tma_load_3d(smem_base + b_tile(st), map_b, full, p0, n0 + (kPair ? (int)cta_rank * (n_act >> 1) : 0), z);
-                    else tma_load_3d(dst_b, map_b, full, p0, n0, z);
-                    issued = i + 1;
-                    continue;
-                }
-                mbar_expect_tx(full, prm.tx_bytes);
-                if (kMajor == kMajorK) {
-                    const int z = slice / prm.p_slices, p0 = (slice - z * prm.p_slices) * kBK;
-                    if (!kGatherA) tma_load_3d(dst_a, map_a, full, p0, m0, z);
-                    if (!kGatherB) tma_load_3d(dst_b, map_b, full, p0, n0, z);
-                } else {
-                    const int k0 = slice * kBK;
+            int it = 0;
+            bool ok = true;
+            SegIter iter(prm);
+            Seg sg;
+            while (ok && iter.next(prm, sg)) {
+                const CUtensorMap *map_a = &bt.a[sg.layer], *map_b = &bt.b[sg.layer];
+                const int m0 = sg.m0, n0 = sg.n0;
+                for (int slice = sg.s_begin; slice < sg.s_end; ++slice, ++it) {
+                    const int st = it % kNB;
+                    const uint32_t ph = (uint32_t)(it / kNB) & 1u;
+                    if (!mbar_wait(smem_u32(&empty[st]), ph ^ 1u, &abort_flag, 64)) { ok = false; break; }
+                    const uint32_t full = smem_u32(&raw_full[st]);
+                    const uint32_t dst_a = smem_base + pair_off(st), dst_b = dst_a + kRawBytesA;
+                    if (kSplit) {
+                        const int sa = it % kNA;
+                        if (!mbar_wait(smem_u32(&a_empty[sa]), ((uint32_t)(it / kNA) & 1u) ^ 1u, &abort_flag, 64)) { ok = false; break; }
+                        const uint32_t full_a = smem_u32(&a_full[sa]);
+                        const int z = slice / prm.p_slices, p0 = (slice - z * prm.p_slices) * kBK;
+                        mbar_expect_tx(full_a, prm.tx_bytes_a);
+                        tma_load_3d(smem_base + (uint32_t)sa * kRawBytesA, map_a, full_a, p0, m0, z);
+                        mbar_expect_tx(full, prm.tx_bytes - prm.tx_bytes_a);
+                        if (kBf) tma_load_3d(smem_base + b_tile(st), map_b, full, p0, n0, z);
+                        else tma_load_3d(dst_b, map_b, full, p0, n0, z);
+                        continue;
+                    }
+                    mbar_expect_tx(full, prm.tx_bytes);
+                    if (kMajor == kMajorK) {
+                        const int z = slice / prm.p_slices, p0 = (slice - z * prm.p_slices) * kBK;
+                        if (!kGatherA) tma_load_3d(dst_a, map_a, full, p0, m0, z);
+                        if (!kGatherB) tma_load_3d(dst_b, map_b, full, p0, n0, z);
+                    } else {
+                        const int k0 = slice * kBK;
 #pragma unroll
-                    for (int j = 0; j < kBM / 32; ++j) tma_load_2d(dst_a + j * 4096, map_a, full, m0 + 32 * j, k0);
+                        for (int j = 0; j < kBM / 32; ++j) tma_load_2d(dst_a + j * 4096, map_a, full, m0 + 32 * j, k0);
 #pragma unroll
-                    for (int j = 0; j < kBN / 32; ++j) tma_load_2d(dst_b + j * 4096, map_b, full, n0 + 32 * j, k0);
+                        for (int j = 0; j < kBN / 32; ++j) tma_load_2d(dst_b + j * 4096, map_b, full, n0 + 32 * j, k0);
+                    }
                 }
-                issued = i + 1;
             }
-            // on an abort: loads already issued must land before the block may exit
+            // on an abort: loads already issued (slices 0 .. it-1) must land before the block may exit
             if (abort_flag) {
+                const int issued = it;
                 const int first = issued > kNB ? issued - kNB : 0;
                 for (int i = first; i < issued; ++i) {
                     const uint32_t bar = smem_u32(&raw_full[i % kNB]);
@@ -900,8 +845,7 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         }
     } else if (warp == 1) {
         // ================= MMA issuer (one thread) =================
-        if (lane == 0 && cta_rank == 0) {
-            const uint32_t idesc = instr_desc(kMajor, n_act, kPair ? 2 * kBM : kBM);
+        if (lane == 0) {
             // K-major: rows of 128 B, 8-row groups 1024 B apart (SBO); LBO unused.
             // MN-major: 32-wide column blocks 4096 B apart (LBO); 4-deep k groups 512 B apart (SBO).
             const uint32_t lbo = kMajor == kMajorK ? 16u : 4096u;
@@ -915,79 +859,84 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
             const uint32_t desc_lo0 = (uint32_t)smem_desc(0, lbo, sbo, layout);
             auto desc_at = [&](uint32_t lo16) -> uint64_t { return ((uint64_t)desc_hi << 32) | (desc_lo0 + lo16); };
             // bf16 tiles: K-major rows of 64 B with the 64-byte swizzle (mode 4), 8-row groups 512 B apart
-            const uint32_t idesc_bf = instr_desc_bf16(n_act, kPair ? 2 * kBM : kBM);
             const uint32_t desc_bf_hi = (uint32_t)(smem_desc(0, 16u, 512u, 4u) >> 32);
             const uint32_t desc_bf_lo0 = (uint32_t)smem_desc(0, 16u, 512u, 4u);
             auto desc_bf = [&](uint32_t lo16) -> uint64_t { return ((uint64_t)desc_bf_hi << 32) | (desc_bf_lo0 + lo16); };
-            int i = 0, st = 0, ls = 0;                   // slice, its raw / hi slot, its lo slot
+            int st = 0, ls = 0;                          // the current slice's raw / hi slot and lo slot
             uint32_t st_phase = 0;
+            int c = 0;                                   // running number of the chunk (accumulator buffer c & 1)
             bool ok = true;
-            for (int c = 0; c < n_chunks && ok; ++c) {
-                const int b = kWide ? 0 : c & 1;                             // the wide form has one accumulator
-                ok = mbar_wait(smem_u32(&acc_empty[b]), ((uint32_t)(kWide ? c : c >> 1) & 1u) ^ 1u, &abort_flag, 0);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)b * kBN;
-                const int seg = c / cps, cq = c - seg * cps;                // segment (example) and chunk inside it
-                const int chunk_end = seg * seg_len + min(seg_len, (cq + 1) * prm.chunk);
-                for (bool first = true; i < chunk_end; ++i) {
-                    ok = mbar_wait(smem_u32(&op_full[st]), st_phase, &abort_flag, 0);
+            SegIter iter(prm);
+            Seg sg;
+            while (ok && iter.next(prm, sg)) {
+                const uint32_t idesc = instr_desc(kMajor, sg.n_act, kBM);
+                const uint32_t idesc_bf = instr_desc_bf16(sg.n_act, kBM);
+                // an accumulator is drained every prm.chunk slices, and (kExact) at the end of every example: the
+                // segment's slices are runs of seg_len slices (whole examples -- the work is cut that way), each cut
+                // into cps chunks
+                const int n_slices = sg.s_end - sg.s_begin;
+                const int seg_len = kExact ? prm.p_slices : n_slices;
+                const int cps = (seg_len + prm.chunk - 1) / prm.chunk;
+                const int n_chunks = (n_slices / seg_len) * cps;
+                int i = 0;                               // slice within the segment
+                for (int cc = 0; cc < n_chunks && ok; ++cc, ++c) {
+                    const int b = c & 1;
+                    ok = mbar_wait(smem_u32(&acc_empty[b]), ((uint32_t)(c >> 1) & 1u) ^ 1u, &abort_flag, 0);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t hi_a16 = (smem_base + pair_off(st)) >> 4, hi_b16 = hi_a16 + (kRawBytesA >> 4);
-                    const uint32_t lo_a16 = (smem_base + lo_off(ls)) >> 4, lo_b16 = lo_a16 + (kRawBytesA >> 4);   // lo_a unused with A in TMEM
-                    const uint32_t ta_hi = tmem_base + 2 * kBN + ls * kTmemColsA, ta_lo = ta_hi + 32;
-                    if (kBf) {
-                        const uint32_t b16 = (smem_base + b_tile(st)) >> 4;
+                    const uint32_t d_tmem = tmem_base + (uint32_t)b * kBN;
+                    const int run = cc / cps, cq = cc - run * cps;              // run (example) and chunk inside it
+                    const int chunk_end = run * seg_len + min(seg_len, (cq + 1) * prm.chunk);
+                    for (bool first = true; i < chunk_end; ++i) {
+                        ok = mbar_wait(smem_u32(&op_full[st]), st_phase, &abort_flag, 0);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t hi_a16 = (smem_base + pair_off(st)) >> 4, hi_b16 = hi_a16 + (kRawBytesA >> 4);
+                        const uint32_t lo_a16 = (smem_base + lo_off(ls)) >> 4, lo_b16 = lo_a16 + (kRawBytesA >> 4);   // lo_a unused with A in TMEM
+                        const uint32_t ta_hi = tmem_base + 2 * kBN + ls * kTmemColsA, ta_lo = ta_hi + 32;
+                        if (kBf) {
+                            const uint32_t b16 = (smem_base + b_tile(st)) >> 4;
 #pragma unroll
-                        for (int kk = 0; kk < kBK / 8; ++kk) {
-                            const uint64_t db_hi = desc_at(b16 + kk * k_step16);
-                            if (kPair) tc_mma_pair_tf32_ts(d_tmem, ta_hi + kk * 8, db_hi, idesc, (kk == 0 && first) ? 0u : 1u);
-                            else if (kk == 0) tc_mma_tf32_ts(d_tmem, ta_hi, db_hi, idesc, first ? 0u : 1u);
-                            else tc_mma_tf32_ts_acc(d_tmem, ta_hi + kk * 8, db_hi, idesc);
-                        }
-                        // cross terms, 16 k (32 bytes of a 64-byte row, 8 columns of tensor memory) per instruction
-                        const uint32_t bf_hi16 = (smem_base + bf_tile(ls)) >> 4, bf_lo16 = bf_hi16 + (kBTile >> 5);
+                            for (int kk = 0; kk < kBK / 8; ++kk) {
+                                const uint64_t db_hi = desc_at(b16 + kk * k_step16);
+                                if (kk == 0) tc_mma_tf32_ts(d_tmem, ta_hi, db_hi, idesc, first ? 0u : 1u);
+                                else tc_mma_tf32_ts_acc(d_tmem, ta_hi + kk * 8, db_hi, idesc);
+                            }
+                            // cross terms, 16 k (32 bytes of a 64-byte row, 8 columns of tensor memory) per instruction
+                            const uint32_t bf_hi16 = (smem_base + bf_tile(ls)) >> 4, bf_lo16 = bf_hi16 + (kBTile >> 5);
 #pragma unroll
-                        for (int kk = 0; kk < kBK / 16; ++kk) {
-                            if (kPair) {
-                                tc_mma_pair_bf16_ts_acc(d_tmem, ta_hi + 32 + kk * 8, desc_bf(bf_lo16 + kk * 2), idesc_bf);
-                                tc_mma_pair_bf16_ts_acc(d_tmem, ta_hi + 48 + kk * 8, desc_bf(bf_hi16 + kk * 2), idesc_bf);
-                            } else {
+                            for (int kk = 0; kk < kBK / 16; ++kk) {
                                 tc_mma_bf16_ts_acc(d_tmem, ta_hi + 32 + kk * 8, desc_bf(bf_lo16 + kk * 2), idesc_bf);
                                 tc_mma_bf16_ts_acc(d_tmem, ta_hi + 48 + kk * 8, desc_bf(bf_hi16 + kk * 2), idesc_bf);
                             }
-                        }
-                    } else
+                        } else
 #pragma unroll
-                    for (int kk = 0; kk < kBK / 8; ++kk) {
-                        const uint64_t db_hi = desc_at(hi_b16 + kk * k_step16);
-                        const uint64_t db_lo = desc_at(lo_b16 + kk * k_step16);
-                        if (kATmem) {
-                            if (kk == 0) tc_mma_tf32_ts(d_tmem, ta_hi, db_hi, idesc, first ? 0u : 1u);
-                            else tc_mma_tf32_ts_acc(d_tmem, ta_hi + kk * 8, db_hi, idesc);
-                            tc_mma_tf32_ts_acc(d_tmem, ta_hi + kk * 8, db_lo, idesc);
-                            tc_mma_tf32_ts_acc(d_tmem, ta_lo + kk * 8, db_hi, idesc);
-                        } else {
-                            const uint64_t da_hi = desc_at(hi_a16 + kk * k_step16);
-                            const uint64_t da_lo = desc_at(lo_a16 + kk * k_step16);
-                            if (kk == 0) tc_mma_tf32(d_tmem, da_hi, db_hi, idesc, first ? 0u : 1u);
-                            else tc_mma_tf32_acc(d_tmem, da_hi, db_hi, idesc);
-                            tc_mma_tf32_acc(d_tmem, da_hi, db_lo, idesc);
-                            tc_mma_tf32_acc(d_tmem, da_lo, db_hi, idesc);
+                        for (int kk = 0; kk < kBK / 8; ++kk) {
+                            const uint64_t db_hi = desc_at(hi_b16 + kk * k_step16);
+                            const uint64_t db_lo = desc_at(lo_b16 + kk * k_step16);
+                            if (kATmem) {
+                                if (kk == 0) tc_mma_tf32_ts(d_tmem, ta_hi, db_hi, idesc, first ? 0u : 1u);
+                                else tc_mma_tf32_ts_acc(d_tmem, ta_hi + kk * 8, db_hi, idesc);
+                                tc_mma_tf32_ts_acc(d_tmem, ta_hi + kk * 8, db_lo, idesc);
+                                tc_mma_tf32_ts_acc(d_tmem, ta_lo + kk * 8, db_hi, idesc);
+                            } else {
+                                const uint64_t da_hi = desc_at(hi_a16 + kk * k_step16);
+                                const uint64_t da_lo = desc_at(lo_a16 + kk * k_step16);
+                                if (kk == 0) tc_mma_tf32(d_tmem, da_hi, db_hi, idesc, first ? 0u : 1u);
+                                else tc_mma_tf32_acc(d_tmem, da_hi, db_hi, idesc);
+                                tc_mma_tf32_acc(d_tmem, da_hi, db_lo, idesc);
+                                tc_mma_tf32_acc(d_tmem, da_lo, db_hi, idesc);
+                            }
                         }
+                        first = false;
+                        tc_commit(smem_u32(&empty[st]));              // raw, lo and TMEM-A slots are free once these MMAs retire
+                        if (++st == kNB) { st = 0; st_phase ^= 1u; }
+                        if (++ls == kLoN) ls = 0;
                     }
-                    first = false;
-                    if (kPair) tc_commit_pair(smem_u32(&empty[st]));      // in both CTAs
-                    else
-                    tc_commit(smem_u32(&empty[st]));              // raw, lo and TMEM-A slots are free once these MMAs retire
-                    if (++st == kNB) { st = 0; st_phase ^= 1u; }
-                    if (++ls == kLoN) ls = 0;
+                    if (ok) tc_commit(smem_u32(&acc_full[b]));
                 }
-                if (ok) { if (kPair) tc_commit_pair(smem_u32(&acc_full[b])); else tc_commit(smem_u32(&acc_full[b])); }
             }
             if (!ok) {      // abort: MMAs already issued must retire before TMEM is freed
-                if (kPair) tc_commit_pair_local(smem_u32(drain)); else
                 tc_commit(smem_u32(drain));
                 for (uint32_t t = 0; t < kWaitLimit && !mbar_try(smem_u32(drain), 0); ++t) {}
             }
@@ -1006,14 +955,8 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         Gatherer<kModeB, kTwoGroups> rows_b;
         typedef typename Gatherer<kModeA, kTwoGroups>::Regs RegsA;
         typedef typename Gatherer<kModeB, kTwoGroups>::Regs RegsB;
-        rows_a.init(prm, bt.x[layer], bt.delta[layer], m0, row0, prm.M);
-        rows_b.init(prm, bt.x[layer], bt.delta[layer], n0, row0, prm.N);
         // where the current slice sits: example z, 32-wide block pblk of that example's output positions
         int z = 0, pblk = 0;
-        if (kAnyGather) {
-            z = slice_begin / prm.p_slices;
-            pblk = slice_begin - z * prm.p_slices;
-        }
         auto advance = [&]() {
             if (++pblk == prm.p_slices) { pblk = 0; ++z; }
         };
@@ -1022,7 +965,7 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
             rows_a.load(prm, z, pbase, ga);
             rows_b.load(prm, z, pbase, gb);
         };
-        // transform of slice i; gathered elements come in registers, TMA tiles from the raw stage
+        // transform of the block's slice number i; gathered elements come in registers, TMA tiles from the raw stage
         auto process = [&](int i, const RegsA &ga, const RegsB &gb) -> bool {
             const int st = i % kNB, ls = i % kLoN;
             const uint32_t ph = (uint32_t)(i / kNB) & 1u;
@@ -1148,190 +1091,141 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
             if (kATmem) { tc_wait_st(); tc_fence_before(); }      // TMEM stores complete and ordered before the signal
             fence_async_smem();                                   // generic-proxy writes -> tensor core reads
             __syncwarp();
-            if (lane == 0) {
-                if (kPair) mbar_arrive_cta(smem_u32(&op_full[st]), 0);     // the issuing CTA's barrier
-                else mbar_arrive(smem_u32(&op_full[st]));
-            }
+            if (lane == 0) mbar_arrive(smem_u32(&op_full[st]));
             return true;
         };
 
-        // two register sets in turn: the loads of slice i+1 are in flight while slice i is transformed
         RegsA a0, a1;
         RegsB b0, b1;
-        if (kTwoGroups && kAnyGather) {
-            // this group's slices: group, group + 2, ...
-            // one register set per thread: the other group's work covers this group's load latency (measured
-            // faster than two sets in turn)
-            for (int sk = 0; sk < group; ++sk) advance();
-            for (int i = group; i < n_slices; i += 2) {
-                gather(a0, b0);
-                if (!process(i, a0, b0)) break;
-                advance(); advance();
-            }
-        } else if (kTwoGroups) {
-            for (int i = group; i < n_slices; i += 2)
-                if (!process(i, a0, b0)) break;
-        } else {
-        if (kAnyGather) gather(a0, b0);
-        for (int i = 0; i < n_slices; i += 2) {
-            if (kAnyGather && i + 1 < n_slices) { advance(); gather(a1, b1); }
-            if (!process(i, a0, b0)) break;
-            if (i + 1 < n_slices) {
-                if (kAnyGather && i + 2 < n_slices) { advance(); gather(a0, b0); }
-                if (!process(i + 1, a1, b1)) break;
-            }
-        }
-        }
-    } else if (kWide) {
-        // ================= epilogue warps, wide form =================
-        // Columns 0..127 of the pair's tile keep their running sums in registers as in the other forms; 256 per lane
-        // do not fit, so columns 128..255 go to the split-K scratch chunk by chunk (first chunk stored, later ones
-        // added with red.global.add -- one thread per address, in program order).  The accumulator is handed back as
-        // soon as its last columns are in registers, before their reds are issued.
-        const uint32_t q = warp & 3;
-        const int r_local = (int)(q * 32u + lane);
-        // this CTA's two 128 x 128 scratch tiles (column halves of its 128 x 256 part), column-major inside a tile
-        const size_t tiles_layer = (size_t)prm.tiles_x * gridDim.x;
-        const size_t tile0 = (size_t)blockIdx.z * tiles_layer + (size_t)tile_m * prm.tiles_x + (size_t)tile_n * 2;
-        float *const dst0 = prm.partial + tile0 * (kBM * kBN) + r_local;
-        float acc[kBN];
-#pragma unroll
-        for (int j = 0; j < kBN; ++j) acc[j] = 0.f;
+        int it0 = 0;                                 // block-wide number of the segment's first slice
         bool ok = true;
-        for (int c = 0; c < n_chunks && ok; ++c) {
-            ok = mbar_wait(smem_u32(&acc_full[0]), (uint32_t)c & 1u, &abort_flag, 32);     // the MMAs wait for this drain
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t taddr = tmem_base + ((q * 32u) << 16);
-#pragma unroll
-            for (int j0 = 0; j0 < kBN; j0 += 32) {
-                if (j0 < n_act) {
-                    uint32_t r[32];
-                    tc_ld_32x32(taddr + j0, r);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) acc[j0 + j] = __fadd_rn(acc[j0 + j], __uint_as_float(r[j]));
-                }
+        SegIter iter(prm);
+        Seg sg;
+        while (ok && iter.next(prm, sg)) {
+            const int n_slices = sg.s_end - sg.s_begin;
+            if (kAnyGather) {
+                rows_a.init(prm, bt.x[sg.layer], bt.delta[sg.layer], sg.m0, row0, prm.M);
+                rows_b.init(prm, bt.x[sg.layer], bt.delta[sg.layer], sg.n0, row0, prm.N);
+                z = sg.s_begin / prm.p_slices;
+                pblk = sg.s_begin - z * prm.p_slices;
             }
-            bool released = false;
-            auto release = [&]() {
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cta(smem_u32(&acc_empty[0]), 0);
-                released = true;
-            };
-#pragma unroll
-            for (int j0 = kBN; j0 < kTileN; j0 += 32) {
-                if (j0 < n_act) {
-                    uint32_t r[32];
-                    tc_ld_32x32(taddr + j0, r);
-                    tc_wait_ld();
-                    if (j0 + 32 >= n_act) release();              // the last columns are out of tensor memory
-                    float *dst = dst0 + (size_t)j0 * kBM;         // tile 1 follows tile 0 in the scratch
-                    if (c == 0) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (j0 + j < n_valid) dst[j * kBM] = __uint_as_float(r[j]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (j0 + j < n_valid)
-                                asm volatile("red.global.add.f32 [%0], %1;" ::"l"(dst + j * kBM), "f"(__uint_as_float(r[j])) : "memory");
+            if (kTwoGroups) {
+                // this group's slices: those whose block-wide number has the group's parity.  With a gathered tile:
+                // one register set per thread -- the other group's work covers this group's load latency
+                // (measured faster than two sets in turn)
+                const int i_first = ((it0 & 1) == group) ? 0 : 1;
+                if (kAnyGather && i_first) advance();
+                for (int i = i_first; i < n_slices; i += 2) {
+                    if (kAnyGather) gather(a0, b0);
+                    if (!process(it0 + i, a0, b0)) { ok = false; break; }
+                    if (kAnyGather) { advance(); advance(); }
+                }
+            } else {
+                // two register sets in turn: the loads of slice i+1 are in flight while slice i is transformed
+                if (kAnyGather) gather(a0, b0);
+                for (int i = 0; i < n_slices; i += 2) {
+                    if (kAnyGather && i + 1 < n_slices) { advance(); gather(a1, b1); }
+                    if (!process(it0 + i, a0, b0)) { ok = false; break; }
+                    if (i + 1 < n_slices) {
+                        if (kAnyGather && i + 2 < n_slices) { advance(); gather(a0, b0); }
+                        if (!process(it0 + i + 1, a1, b1)) { ok = false; break; }
                     }
                 }
             }
-            if (!released) release();
-        }
-        if (ok) {
-#pragma unroll
-            for (int j = 0; j < kBN; ++j)
-                if (j < n_valid) dst0[(size_t)j * kBM] = acc[j];
+            it0 += n_slices;
         }
     } else {
         // ================= epilogue warps: drain chunks, accumulate in fp32 registers =================
         const uint32_t q = warp & 3;                                      // TMEM lane quarter of this warp
+        const int r_local = (int)(q * 32u + lane);
         float acc[kBN];
-#pragma unroll
-        for (int j = 0; j < kBN; ++j) acc[j] = 0.f;
         const uint32_t sq_addr = tmem_base + ((q * 32u) << 16) + kSqCol;  // kExact: this warp's rows of the sum of squares
-        if (kExact) {
-            uint32_t zero[16];
-#pragma unroll
-            for (int j = 0; j < 16; ++j) zero[j] = 0u;
-#pragma unroll
-            for (int j0 = 0; j0 < kBN; j0 += 16) tc_st_32x16(sq_addr + j0, zero);
-            tc_wait_st();
-        }
+        int c = 0;                                                        // running number of the chunk
         bool ok = true;
-        for (int c = 0; c < n_chunks && ok; ++c) {
-            const int b = c & 1;
-            ok = mbar_wait(smem_u32(&acc_full[b]), (uint32_t)(c >> 1) & 1u, &abort_flag, 256);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t taddr = tmem_base + ((q * 32u) << 16) + (uint32_t)b * kBN;
+        SegIter iter(prm);
+        Seg sg;
+        while (ok && iter.next(prm, sg)) {
 #pragma unroll
-            for (int j0 = 0; j0 < kBN; j0 += 32) {
-                if (j0 < n_act) {
-                    uint32_t r[32];
-                    tc_ld_32x32(taddr + j0, r);
-                    tc_wait_ld();
+            for (int j = 0; j < kBN; ++j) acc[j] = 0.f;
+            if (kExact) {
+                uint32_t zero[16];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) acc[j0 + j] = __fadd_rn(acc[j0 + j], __uint_as_float(r[j]));
-                }
+                for (int j = 0; j < 16; ++j) zero[j] = 0u;
+#pragma unroll
+                for (int j0 = 0; j0 < kBN; j0 += 16) tc_st_32x16(sq_addr + j0, zero);
+                tc_wait_st();
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                if (kPair) mbar_arrive_cta(smem_u32(&acc_empty[b]), 0);
-                else mbar_arrive(smem_u32(&acc_empty[b]));
-            }
-            if (kExact && (c + 1) % cps == 0) {
-                // end of an example: acc holds its sum over positions; add the squares to the running sum in TMEM
+            const int n_act = sg.n_act, n_valid = sg.n_valid;
+            const int n_slices = sg.s_end - sg.s_begin;
+            const int seg_len = kExact ? prm.p_slices : n_slices;
+            const int cps = (seg_len + prm.chunk - 1) / prm.chunk;
+            const int n_chunks = (n_slices / seg_len) * cps;
+            for (int cc = 0; cc < n_chunks && ok; ++cc, ++c) {
+                const int b = c & 1;
+                ok = mbar_wait(smem_u32(&acc_full[b]), (uint32_t)(c >> 1) & 1u, &abort_flag, 256);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + ((q * 32u) << 16) + (uint32_t)b * kBN;
 #pragma unroll
                 for (int j0 = 0; j0 < kBN; j0 += 32) {
                     if (j0 < n_act) {
                         uint32_t r[32];
-                        tc_ld_32x32(sq_addr + j0, r);
+                        tc_ld_32x32(taddr + j0, r);
                         tc_wait_ld();
-                        uint32_t w0[16], w1[16];
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            w0[j] = __float_as_uint(__fadd_rn(__uint_as_float(r[j]), __fmul_rn(acc[j0 + j], acc[j0 + j])));
-                            w1[j] = __float_as_uint(__fadd_rn(__uint_as_float(r[16 + j]), __fmul_rn(acc[j0 + 16 + j], acc[j0 + 16 + j])));
-                        }
-                        tc_st_32x16(sq_addr + j0, w0);
-                        tc_st_32x16(sq_addr + j0 + 16, w1);
+                        for (int j = 0; j < 32; ++j) acc[j0 + j] = __fadd_rn(acc[j0 + j], __uint_as_float(r[j]));
                     }
                 }
-                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&acc_empty[b]));
+                if (kExact && (cc + 1) % cps == 0) {
+                    // end of an example: acc holds its sum over positions; add the squares to the running sum in TMEM
 #pragma unroll
-                for (int j = 0; j < kBN; ++j) acc[j] = 0.f;
+                    for (int j0 = 0; j0 < kBN; j0 += 32) {
+                        if (j0 < n_act) {
+                            uint32_t r[32];
+                            tc_ld_32x32(sq_addr + j0, r);
+                            tc_wait_ld();
+                            uint32_t w0[16], w1[16];
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                w0[j] = __float_as_uint(__fadd_rn(__uint_as_float(r[j]), __fmul_rn(acc[j0 + j], acc[j0 + j])));
+                                w1[j] = __float_as_uint(__fadd_rn(__uint_as_float(r[16 + j]), __fmul_rn(acc[j0 + 16 + j], acc[j0 + 16 + j])));
+                            }
+                            tc_st_32x16(sq_addr + j0, w0);
+                            tc_st_32x16(sq_addr + j0 + 16, w1);
+                        }
+                    }
+                    tc_wait_st();
+#pragma unroll
+                    for (int j = 0; j < kBN; ++j) acc[j] = 0.f;
+                }
             }
-        }
-        if (kExact && ok) {        // the result is the sum of squares
+            if (!ok) break;
+            if (kExact) {        // the result is the sum of squares
 #pragma unroll
-            for (int j0 = 0; j0 < kBN; j0 += 32) {
-                uint32_t r[32];
-                tc_ld_32x32(sq_addr + j0, r);
-                tc_wait_ld();
+                for (int j0 = 0; j0 < kBN; j0 += 32) {
+                    uint32_t r[32];
+                    tc_ld_32x32(sq_addr + j0, r);
+                    tc_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) acc[j0 + j] = __uint_as_float(r[j]);
+                    for (int j = 0; j < 32; ++j) acc[j0 + j] = __uint_as_float(r[j]);
+                }
             }
-        }
-        if (ok) {
-            const int r_local = (int)(q * 32u + lane);
-            const int m = m0 + r_local;
-            if (prm.splits > 1) {
-                // split-K scratch, column-major inside the tile: consecutive lanes -> consecutive addresses
-                const size_t tile = (size_t)blockIdx.z * (gridDim.x * gridDim.y) + (size_t)tile_m * tiles_n + tile_n;
-                float *dst = prm.partial + tile * (kBM * kBN) + r_local;
+            // ---- the segment's 128 x 128 sums leave the registers (the other roles are already on the next segment)
+            const int m = sg.m0 + r_local;
+            float *const S = bt.S[sg.layer];
+            if (!sg.whole) {
+                // partial tile, column-major inside the tile: consecutive lanes -> consecutive addresses
+                float *dst = prm.partial + (size_t)sg.slot * (kBM * kBN) + r_local;
 #pragma unroll
                 for (int j = 0; j < kBN; ++j)
                     if (j < n_valid) dst[j * kBM] = acc[j];
             } else if (prm.ld_m == 1) {
                 // result is contiguous along m: lanes write neighbouring addresses directly
                 if (m < prm.M) {
-                    float *col = S + (size_t)m + (size_t)n0 * prm.ld_n;
+                    float *col = S + (size_t)m + (size_t)sg.n0 * prm.ld_n;
 #pragma unroll
                     for (int j0 = 0; j0 < kBN; j0 += 16) {        // old values sixteen at a time, all loads in flight
                         float old[16];
@@ -1346,38 +1240,47 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                             }
                     }
                 }
-            } else {
-                // result is contiguous along n: transpose this warp's 32 x 128 block through shared memory
-                // (the pipeline stages are idle: the last accumulator was complete before we got here)
-                float *tile = reinterpret_cast<float *>(smem_gen) + q * (32 * (kBN + 1));
+            } else if (m < prm.M) {
+                // result is contiguous along n: every lane owns a row and writes it 16 bytes at a time (the halves of a
+                // 32-byte sector arrive in consecutive instructions and are merged in L2); rows whose pitch is not a
+                // multiple of 16 bytes go element by element
+                float *row = S + (size_t)m * prm.ld_m + sg.n0;
+                if ((prm.ld_m & 3) == 0) {
 #pragma unroll
-                for (int j = 0; j < kBN; ++j) tile[lane * (kBN + 1) + j] = __fmul_rn(prm.scale, acc[j]);
-                __syncwarp();
-                for (int r0 = 0; r0 < 32; r0 += 8) {              // eight rows at a time, all loads in flight
-                    float old[8][kBN / 32];
+                    for (int j0 = 0; j0 < kBN; j0 += 16) {
+                        float4 old[4];
 #pragma unroll
-                    for (int rr = 0; rr < 8; ++rr) {
-                        const int mr = m0 + (int)(q * 32u) + r0 + rr;
-                        const float *src = S + (size_t)mr * prm.ld_m + n0;
+                        for (int u = 0; u < 4; ++u)
+                            old[u] = (prm.accumulate && j0 + 4 * u + 3 < n_valid) ? *reinterpret_cast<const float4 *>(row + j0 + 4 * u)
+                                                                                  : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                        for (int cblk = 0; cblk < kBN / 32; ++cblk) {
-                            const int j = cblk * 32 + (int)lane;
-                            old[rr][cblk] = (prm.accumulate && mr < prm.M && j < n_valid) ? src[j] : 0.f;
-                        }
-                    }
+                        for (int u = 0; u < 4; ++u) {
+                            const int j = j0 + 4 * u;
+                            if (j + 3 < n_valid) {
+                                float4 res = make_float4(__fmul_rn(prm.scale, acc[j]), __fmul_rn(prm.scale, acc[j + 1]),
+                                                         __fmul_rn(prm.scale, acc[j + 2]), __fmul_rn(prm.scale, acc[j + 3]));
+                                if (prm.accumulate) {
+                                    res.x = __fadd_rn(old[u].x, res.x); res.y = __fadd_rn(old[u].y, res.y);
+                                    res.z = __fadd_rn(old[u].z, res.z); res.w = __fadd_rn(old[u].w, res.w);
+                                }
+                                *reinterpret_cast<float4 *>(row + j) = res;
+                            } else {
 #pragma unroll
-                    for (int rr = 0; rr < 8; ++rr) {
-                        const int mr = m0 + (int)(q * 32u) + r0 + rr;
-                        float *dst = S + (size_t)mr * prm.ld_m + n0;
-#pragma unroll
-                        for (int cblk = 0; cblk < kBN / 32; ++cblk) {
-                            const int j = cblk * 32 + (int)lane;
-                            if (mr < prm.M && j < n_valid) {
-                                const float res = tile[(r0 + rr) * (kBN + 1) + j];
-                                dst[j] = prm.accumulate ? __fadd_rn(old[rr][cblk], res) : res;
+                                for (int e = 0; e < 4; ++e)
+                                    if (j + e < n_valid) {
+                                        const float res = __fmul_rn(prm.scale, acc[j + e]);
+                                        row[j + e] = prm.accumulate ? __fadd_rn(row[j + e], res) : res;
+                                    }
                             }
                         }
                     }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < kBN; ++j)
+                        if (j < n_valid) {
+                            const float res = __fmul_rn(prm.scale, acc[j]);
+                            row[j] = prm.accumulate ? __fadd_rn(row[j], res) : res;
+                        }
                 }
             }
         }
@@ -1386,50 +1289,55 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
     // ---- common exit ----
     tc_fence_before();
     __syncthreads();
-    // pair form: the other CTA's tensor memory and shared memory are operands of this pair's MMAs and its barriers
-    // receive this CTA's arrivals, so neither CTA frees anything or leaves before both are done
-    if (kPair) cluster_sync_all();
     if (warp == 1) {
         tc_fence_after();
-        if (kPair) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
-        else
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
     if (threadIdx.x == 0 && abort_flag) atomicOr(prm.status, VGC_DEV_TIMEOUT);
 }
 
-// Combine split-K partial tiles in a fixed order.  One block per 32 x 8 patch of a tile, one output per
-// thread: partials are read along rows (their unit stride), the result is written along whichever of
-// m / n has unit stride.
+// Adds the partial tiles of every tile that more than one block worked on, in the order of the blocks (a fixed
+// order: the result does not depend on scheduling).  One block per 32 x 8 patch of a tile, one output per thread:
+// partials are read along rows (their unit stride), the result is written along whichever of m / n has unit
+// stride.  Tiles that one block covered alone were written by that block; their patches return at once.
 struct ResultPtrs { float *S[kMaxBatch]; };
 
 __global__ void __launch_bounds__(256)
-sqgrad_tc_combine(const float *__restrict__ partial, int splits, int tiles_x, int tiles_y, int M, int N, float scale,
-                  int accumulate, const ResultPtrs results, long long ld_m, long long ld_n)
+sqgrad_tc_combine(const float *__restrict__ partial, int n_blocks, long long units_total, int units_per_tile,
+                  int tiles_x, int tiles_y, int M, int N, float scale, int accumulate, const ResultPtrs results,
+                  long long ld_m, long long ld_n)
 {
     __shared__ float patch[8][33];
-    float *__restrict__ S = results.S[blockIdx.y];                         // blockIdx.y: layer of the batch
-    partial += (size_t)blockIdx.y * splits * ((size_t)tiles_x * tiles_y) * (kBM * kBN);
     const int tile = blockIdx.x >> 6, sub = blockIdx.x & 63;
+    // the blocks that hold the tile's first and last unit (block b owns units [b U / G, (b + 1) U / G))
+    const long long t_lo = ((long long)blockIdx.y * (tiles_x * tiles_y) + tile) * units_per_tile;
+    const int b_first = (int)(((t_lo + 1) * n_blocks - 1) / units_total);
+    const int b_last = (int)(((t_lo + units_per_tile) * n_blocks - 1) / units_total);
+    if (b_first == b_last) return;
+    float *__restrict__ S = results.S[blockIdx.y];                         // blockIdx.y: layer of the batch
     const int tx = tile % tiles_x, ty = tile / tiles_x;
     const int r0 = (sub & 3) * 32, j0 = (sub >> 2) * 8;                   // patch origin inside the tile
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;              // lane -> row, warp -> column
-    const size_t tiles = (size_t)tiles_x * tiles_y;
     if (ty * kBM + r0 >= M || tx * kBN + j0 >= N) return;
     const int j = j0 + w;
     float sum = 0.f;
     if (tx * kBN + j < N) {
-        const float *src = partial + ((size_t)tile * kBN + j) * kBM + r0 + lane;
-        const size_t stride = tiles * (size_t)(kBM * kBN);
-        int z = 0;
-        for (; z + 8 <= splits; z += 8) {                   // eight loads in flight, summed in split order
+        // the first block's part of this tile is that block's last segment unless its range starts with the tile;
+        // every later block's part is its first segment
+        const long long lo_first = (long long)b_first * units_total / n_blocks;
+        const size_t within = (size_t)j * kBM + r0 + lane;
+        const float *src0 = partial + (size_t)(2 * b_first + (lo_first < t_lo ? 1 : 0)) * (kBM * kBN) + within;
+        sum = __ldcs(src0);
+        const float *src = partial + within;
+        int b = b_first + 1;
+        for (; b + 8 <= b_last + 1; b += 8) {                // eight loads in flight, summed in block order
             float v[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) v[u] = __ldcs(src + (size_t)(z + u) * stride);
+            for (int u = 0; u < 8; ++u) v[u] = __ldcs(src + (size_t)(2 * (b + u)) * (kBM * kBN));
 #pragma unroll
             for (int u = 0; u < 8; ++u) sum = __fadd_rn(sum, v[u]);
         }
-        for (; z < splits; ++z) sum = __fadd_rn(sum, __ldcs(src + (size_t)z * stride));
+        for (; b <= b_last; ++b) sum = __fadd_rn(sum, __ldcs(src + (size_t)(2 * b) * (kBM * kBN)));
     }
     const float res = __fmul_rn(scale, sum);
     if (ld_m == 1) {
@@ -1480,76 +1388,55 @@ static bool make_map(CUtensorMap *map, const float *base, int rank, const cuuint
     const CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<float *>(base), dims,
                            strides_bytes, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (rc != CUDA_SUCCESS && getenv("VGC_DEBUG")) fprintf(stderr, "vgc: tensor map encode failed with CUresult %d\n", (int)rc);
+    if (rc != CUDA_SUCCESS && debug_enabled()) fprintf(stderr, "vgc: tensor map encode failed with CUresult %d\n", (int)rc);
     return rc == CUDA_SUCCESS;
 }
 
-static int default_chunk()
-{
-    static int chunk = 0;
-    if (!chunk) {
-        const char *e = getenv("VGC_TC_CHUNK");
-        chunk = e ? atoi(e) : 8;
-        if (chunk < 1) chunk = 1;
-    }
-    return chunk;
-}
+// Slices per accumulator drain.  The tensor core's fp32 accumulation truncates (a one-sided bias of about 1.3e-8 of the
+// sum per instruction), so an accumulator is handed to the round-to-nearest register sums after at most 8 slices
+// (96 instructions): results then sit 1 - 3e-6 below the exact sum, against the 1e-5 bound.
+constexpr int kChunk = 8;
+constexpr int kBlocksMax = 148;          // thread blocks of a launch: one per SM of a B200
 
 struct Plan {
-    int splits, slices_per_split, k_slices, tiles_x, tiles_y;
+    int unit, units_per_tile, blocks, tiles_x, tiles_y;
+    long long units_total;
+    bool partials;           // some tile is shared by several blocks: partial tiles go through the scratch
 };
 
-// how many sqgrad launches the caller keeps in flight side by side (vgc_sqgrad_plan_hint)
-static int g_concurrent_launches = 1;
-
-// `unit`: slices that must stay in one block (the per-example form splits the reduction between examples only)
-// `wide`: the blocks are CTA pairs' halves of 256 x 256 tiles, i.e. each block covers two 128-column tiles
-static Plan make_plan(int M, int N, int k_slices_total, int n_layers = 1, int unit = 1, bool wide = false)
+// How a launch's work -- n_layers x tiles x k_slices slices -- is cut into one contiguous range per block.
+// `unit_min`: slices that must stay in one block (the per-example form cuts the reduction between examples only).
+// Two candidates: whole tiles per block (no scratch, no second kernel, but the blocks' loads are as even as the
+// tile count allows), or an even cut of the slices over all SMs (tiles at the cuts are shared, their partial
+// sums combined by a second kernel).  Costs in slice times: a block's longest range, plus what the combine pass
+// adds to the call (its launch and the partial tiles' round trip, about 14 slices' worth).
+static Plan make_plan(int M, int N, int k_slices, int n_layers, int unit_min)
 {
     Plan p;
-    const int k_slices = k_slices_total / unit;                          // planned in units
     p.tiles_x = (N + kBN - 1) / kBN;
     p.tiles_y = (M + kBM - 1) / kBM;
-    // blocks of one split of the whole launch
-    const long tiles = (long)(wide ? (p.tiles_x + 1) / 2 : p.tiles_x) * p.tiles_y * n_layers;
-    // Blocks run one per SM, wave after wave.  A caller that runs several launches side by side (separate
-    // streams and workspaces, vgc_sqgrad_plan_hint) may also plan for fewer SMs per launch through VGC_TC_BLOCKS.
-    const char *env = getenv("VGC_TC_BLOCKS");
-    const long target = env && atoi(env) > 0 ? atoi(env) : 148;
-    long want = 1;
-    if (g_concurrent_launches > 1) {
-        // next to other launches a partly filled wave costs nothing (their blocks take the idle SMs): split the
-        // reduction as far as one wave allows and no further -- every extra block pays its fixed cost again
-        want = target / tiles;
-        if (want > k_slices) want = k_slices;
-        if (want < 1) want = 1;
-    } else {
-        // alone, the launch pays for whole waves: take the split with the shortest estimated makespan,
-        // waves x (slices per block + a block's fixed cost, about 8 slices' worth, + about 5 more for writing
-        // and re-reading a partial tile) + the combine pass
-        long best = -1;
-        const long max_split = k_slices < 256 ? k_slices : 256;
-        for (long sp = 1; sp <= max_split; ++sp) {
-            const long per = (k_slices + sp - 1) / sp;
-            if ((k_slices + per - 1) / per != sp) continue;              // splits that would get no slices
-            if (sp > 1 && tiles * sp > 6 * target) break;                 // keeps the split-K scratch L2-sized
-            const long waves = (tiles * sp + target - 1) / target;
-            const long cost = waves * (per * unit + 8 + (sp > 1 ? 5 : 0)) + (sp > 1 ? 6 : 0);
-            if (best < 0 || cost < best) { best = cost; want = sp; }
-        }
-    }
-    p.k_slices = k_slices_total;
-    const int per = (int)((k_slices + want - 1) / want);
-    p.slices_per_split = per * unit;
-    p.splits = (k_slices + per - 1) / per;
+    const long long tiles = (long long)p.tiles_x * p.tiles_y * n_layers;
+    // (a) whole tiles
+    const long long waves = (tiles + kBlocksMax - 1) / kBlocksMax;
+    const long long blocks_a = (tiles + waves - 1) / waves;
+    const long long cost_a = ((tiles + blocks_a - 1) / blocks_a) * k_slices;
+    // (b) even cut
+    const long long upt = k_slices / unit_min, units = tiles * upt;
+    const long long blocks_b = units < kBlocksMax ? units : kBlocksMax;
+    const long long cost_b = ((units + blocks_b - 1) / blocks_b) * unit_min + 14;
+    bool even = cost_b < cost_a;
+    p.unit = even ? unit_min : k_slices;
+    p.units_per_tile = even ? (int)upt : 1;
+    p.units_total = even ? units : tiles;
+    p.blocks = (int)(even ? blocks_b : blocks_a);
+    p.partials = false;
+    for (long long b = 1; b < p.blocks && !p.partials; ++b) p.partials = (b * p.units_total / p.blocks) % p.units_per_tile != 0;
     return p;
 }
 
 }  // namespace tc
 
 using namespace tc;
-
-void tc_plan_hint(int concurrent_launches) { g_concurrent_launches = concurrent_launches > 1 ? concurrent_launches : 1; }
 
 bool tc_linear_supported(int B, int in, int out)
 {
@@ -1564,35 +1451,19 @@ bool tc_conv_supported(int B, int C, int H, int W, int Cout, int Kh, int Kw, int
            (long)B * ((P + kBK - 1) / kBK) < (1L << 30);
 }
 
-// the wide pair form (256 x 256 tiles, N = 256 instructions) where the pair form applies: VGC_TC_WIDE=1
-static bool wide_form()
-{
-    const char *e = getenv("VGC_TC_WIDE");
-    return e && atoi(e) != 0;
-}
-
 static size_t tc_workspace_bytes(int M, int N, int k_slices, int n_layers = 1, int unit = 1)
 {
     const Plan p = make_plan(M, N, k_slices, n_layers, unit);
-    size_t need = 256 + (p.splits > 1 ? (size_t)n_layers * p.splits * p.tiles_x * p.tiles_y * kBM * kBN * sizeof(float) : 0);
-    if (wide_form()) {
-        // the wide form always goes through the scratch and splits further (half as many blocks per split); which
-        // operand becomes the row side is decided at launch, so both orientations are covered
-        const Plan a = make_plan(M, N, k_slices, n_layers, unit, true), b = make_plan(N, M, k_slices, n_layers, unit, true);
-        const size_t splits = a.splits > b.splits ? a.splits : b.splits;
-        const size_t w = 256 + (size_t)n_layers * splits * p.tiles_x * p.tiles_y * kBM * kBN * sizeof(float);
-        if (w > need) need = w;
-    }
-    return need;
+    // status word (256 bytes) + two partial tiles per block (the first and the last segment of its range)
+    return 256 + (p.partials ? (size_t)2 * p.blocks * kBM * kBN * sizeof(float) : 0);
 }
 
 typedef void (*KernelFn)(const Batch, const Params);
 
 static vgc_status tc_launch(KernelFn kernel, const Batch &bt, int n_layers, Params prm, int M, int N,
-                            int k_slices, void *ws, size_t ws_bytes, cudaStream_t st, int unit = 1, bool pair = false,
-                            bool wide = false)
+                            int k_slices, void *ws, size_t ws_bytes, cudaStream_t st, int unit = 1)
 {
-    const Plan plan = make_plan(M, N, k_slices, n_layers, unit, wide);
+    const Plan plan = make_plan(M, N, k_slices, n_layers, unit);
     if (ws_bytes < tc_workspace_bytes(M, N, k_slices, n_layers, unit)) return VGC_ERR_WORKSPACE;
     static KernelFn configured[32];
     static int n_configured = 0;
@@ -1602,33 +1473,20 @@ static vgc_status tc_launch(KernelFn kernel, const Batch &bt, int n_layers, Para
         VGC_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
         if (n_configured < 32) configured[n_configured++] = kernel;
     }
-    prm.M = M; prm.N = N; prm.k_slices = k_slices; prm.slices_per_split = plan.slices_per_split;
-    prm.splits = plan.splits;
-    prm.tiles_x = plan.tiles_x;
-    prm.chunk = default_chunk();
+    prm.M = M; prm.N = N; prm.k_slices = k_slices;
+    prm.unit = plan.unit; prm.units_per_tile = plan.units_per_tile; prm.units_total = plan.units_total;
+    prm.tiles_x = plan.tiles_x; prm.tiles_y = plan.tiles_y;
+    prm.chunk = kChunk;
     prm.status = static_cast<uint32_t *>(ws);
     prm.partial = reinterpret_cast<float *>(static_cast<char *>(ws) + 256);
-    dim3 grid(plan.tiles_x, plan.tiles_y, plan.splits * n_layers);
-    if (pair) {
-        // clusters of two CTAs, neighbours along x, which holds the row tiles in this form (the caller made sure
-        // their number is even)
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(grid.y, wide ? (grid.x + 1) / 2 : grid.x, grid.z); cfg.blockDim = dim3(kThreadsTc); cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        VGC_CUDA_OK(cudaLaunchKernelEx(&cfg, kernel, bt, prm));
-    } else {
-        kernel<<<grid, kThreadsTc, kSmemBytes, st>>>(bt, prm);
-    }
+    kernel<<<plan.blocks, kThreadsTc, kSmemBytes, st>>>(bt, prm);
     count_launch();
-    if (plan.splits > 1 || wide) {
+    if (plan.partials) {
         ResultPtrs results = {};
         for (int l = 0; l < n_layers; ++l) results.S[l] = bt.S[l];
         sqgrad_tc_combine<<<dim3((unsigned)(plan.tiles_x * plan.tiles_y * 64), (unsigned)n_layers), 256, 0, st>>>(
-            prm.partial, plan.splits, plan.tiles_x, plan.tiles_y, M, N, prm.scale, prm.accumulate, results, prm.ld_m,
-            prm.ld_n);
+            prm.partial, plan.blocks, plan.units_total, plan.units_per_tile, plan.tiles_x, plan.tiles_y, M, N, prm.scale,
+            prm.accumulate, results, prm.ld_m, prm.ld_n);
         count_launch();
     }
     VGC_CUDA_OK(cudaGetLastError());
@@ -1664,20 +1522,6 @@ struct ExactScope {
 };
 
 // Cout <= 64: the im2col rows take the 128-row A tile and the errors the narrow B tile
-// cross terms of the TMA-fed form with bf16 operands unless VGC_TC_BF16=0
-static bool bf_cross()
-{
-    const char *e = getenv("VGC_TC_BF16");
-    return !(e && atoi(e) == 0);
-}
-// the TMA-fed form on pairs of CTAs (256 x 128 tiles) where the number of row tiles allows: VGC_TC_PAIR=1
-static bool pair_form()
-{
-    const char *e = getenv("VGC_TC_PAIR");
-    return e && atoi(e) != 0;
-}
-static bool even_row_tiles(int M) { return ((M + kBM - 1) / kBM) % 2 == 0; }
-
 static bool conv_swapped(int Cout, int n_im2col) { return Cout <= 64 && n_im2col > Cout; }
 
 // ---- repacking pre-pass for 1x1 convolutions whose tiles TMA cannot address in place ----------
@@ -1699,8 +1543,6 @@ enum { kRepackNone = 0, kRepackPlanes = 1, kRepackFlat = 2, kRepackPadW = 3 };
 static int repack_mode(int B, int C, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw, int P, int W = 0, int Ho = 0,
                        int Wo = 0)
 {
-    const char *e = getenv("VGC_TC_REPACK");
-    if (e && atoi(e) == 0) return kRepackNone;
     if ((long)B * C >= (1L << 31) || (long)B * Cout >= (1L << 31)) return kRepackNone;      // 32-bit row index
     if (Kw == 3 && pw == 1 && Wo % 2 == 1 && Wo >= 3 && (long)Ho * ((Wo + 3) / 4 * 4) >= kBK &&
         ((sw == 1 && sh == 1 && W == Wo) || (sw == 2 && W == 2 * Wo)))
@@ -1887,51 +1729,26 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
                               inner, st);
         return conv_group(n_layers, xr, dr, S, B, C, Ho, Wo, Cout, 1, 1, 1, 1, 0, 0, Ho, Wo, scale, accumulate, ws, inner, st);
     }
-    // VGC_TC_GATHER (bit 0: error tile, bit 1: input tile) forces the gathered form of a tile and
-    // VGC_TC_ATMEM=0 keeps the A operand in shared memory: every variant computes the same thing, the
-    // switches exist so that tests can reach each of them on any shape.
-    const int force_gather = getenv("VGC_TC_GATHER") ? atoi(getenv("VGC_TC_GATHER")) : 0;
-    const bool err_tma = P >= kBK && P % 4 == 0 && !(force_gather & 1);
-    const bool in_tma = P >= kBK && P % 4 == 0 && !(force_gather & 2) && Kh == 1 && Kw == 1 && sh == 1 && sw == 1 &&
-                        ph == 0 && pw == 0;
-    const bool a_tmem = !(getenv("VGC_TC_ATMEM") && atoi(getenv("VGC_TC_ATMEM")) == 0);
+    // which tiles TMA can deliver: rows of P positions with a 16-byte pitch, at least one slice long; the input
+    // tile only when the im2col view is the tensor itself (1x1 kernel, stride 1, no padding)
+    const bool err_tma = P >= kBK && P % 4 == 0;
+    const bool in_tma = err_tma && Kh == 1 && Kw == 1 && sh == 1 && sw == 1 && ph == 0 && pw == 0;
     const int p_slices = (P + kBK - 1) / kBK;
     const int k_slices = B * p_slices;
     // three taps at a time: Kw = 3, stride 1 along w with pad 1 (then Wo == W), output width even, errors by TMA
-    const char *taps_env = getenv("VGC_TC_TAPS");
-    const int taps = (!(taps_env && atoi(taps_env) == 0) && !in_tma && err_tma && Kw == 3 && sw == 1 && sh == 1 &&
-                      pw == 1 && Wo == W && W % 2 == 0 && a_tmem)
+    const int taps = (!in_tma && err_tma && Kw == 3 && sw == 1 && sh == 1 && pw == 1 && Wo == W && W % 2 == 0)
                          ? (W % 4 == 0 ? 4 : 2) : 0;
     // the same with stride 2 along w: W == 2 Wo, output width even
-    const int taps_s2 = (!(taps_env && atoi(taps_env) == 0) && !in_tma && err_tma && Kw == 3 && sw == 2 && pw == 1 &&
-                         W == 2 * Wo && Wo % 2 == 0 && a_tmem)
+    const int taps_s2 = (!in_tma && err_tma && Kw == 3 && sw == 2 && pw == 1 && W == 2 * Wo && Wo % 2 == 0)
                             ? (Wo % 4 == 0 ? 4 : 2) : 0;
     // seven taps at a time: Kw = 7, stride 2, pad 3
-    const bool taps7 = !(taps_env && atoi(taps_env) == 0) && !in_tma && err_tma && Kw == 7 && sw == 2 && pw == 3 &&
-                       W == 2 * Wo && Wo % 4 == 0 && a_tmem;
+    const bool taps7 = !in_tma && err_tma && Kw == 7 && sw == 2 && pw == 3 && W == 2 * Wo && Wo % 4 == 0;
     // with few output channels the roles are swapped -- except in the three-tap form, where keeping the errors as
     // the A operand (in tensor memory, half of its rows unused) measures faster than both operands in shared memory
-    bool swapped = conv_swapped(Cout, n_im2col) && !taps && !taps_s2 && !taps7;
-    // both tiles by TMA, A in tensor memory, cross terms in bf16; on pairs of CTAs when the number of row tiles is
-    // even in one of the two orientations (both operands come the same way, so either can be the A side)
-    const bool tma_bf = err_tma && in_tma && a_tmem && bf_cross() && !t_exact;
-    bool pair = false, wide = false;
-    if (tma_bf && (pair_form() || wide_form())) {
-        // the orientation whose number of row tiles is even (the given one first)
-        const bool as_is = even_row_tiles(swapped ? n_im2col : Cout);
-        const bool flipped = !as_is && even_row_tiles(swapped ? Cout : n_im2col);
-        if (as_is || flipped) {
-            const bool sw = flipped ? !swapped : swapped;
-            // 256 x 256 tiles (each CTA of a pair has 128 B rows again) pay where the tile is at least 256 columns
-            // wide and the reduction long enough to cover the unbuffered accumulator's drains and the extra combine pass
-            wide = wide_form() && (sw ? Cout : n_im2col) >= 2 * kBN && k_slices >= 128;
-            pair = wide || pair_form();
-            if (pair) swapped = sw;
-        }
-    }
-    // tile heights: 128 rows, or 64 for the B side of a plain pair (each CTA loads half of the tile's B rows)
-    const int rows_b = pair && !wide ? kBN / 2 : kBN;
-    const int rows_err = swapped ? rows_b : kBM, rows_in = swapped ? kBM : rows_b;
+    const bool swapped = conv_swapped(Cout, n_im2col) && !taps && !taps_s2 && !taps7;
+    // both tiles by TMA: A in tensor memory, cross terms in bf16 (the per-example form keeps tf32 cross terms)
+    const bool tma_bf = err_tma && in_tma && !t_exact;
+    const int rows_err = swapped ? kBN : kBM, rows_in = swapped ? kBM : kBN;
     Batch bt = {};
     uint32_t tx_err = 0, tx_in = 0;
     for (int l = 0; l < n_layers; ++l) {
@@ -1959,7 +1776,6 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
     prm.ph = ph; prm.pw = pw; prm.Wo = Wo; prm.P = P;
     prm.chw = C * H * W;
     prm.wo_magic = (unsigned)(0x100000000ull / (unsigned)Wo) + 1u;
-    const int e = err_tma ? kTma : kGatherErr, i = in_tma ? kTma : kGatherIm2col;
     const bool ex = t_exact;
     const int unit = ex ? p_slices : 1;
     KernelFn fn = nullptr;
@@ -1969,25 +1785,19 @@ static vgc_status conv_group(int n_layers, const float *const *x, const float *c
         if (taps) fn = taps == 4 ? VGC_TC_FN(kTma, kGatherTaps4, true) : VGC_TC_FN(kTma, kGatherTaps2, true);
         else if (taps_s2) fn = taps_s2 == 4 ? VGC_TC_FN(kTma, kGatherTaps4S2, true) : VGC_TC_FN(kTma, kGatherTaps2S2, true);
         else if (taps7) fn = VGC_TC_FN(kTma, kGatherTaps7S2, true);
-        else if (tma_bf) fn = wide   ? sqgrad_tc<kMajorK, kTma, kTma, true, false, true, true, true>
-                              : pair ? sqgrad_tc<kMajorK, kTma, kTma, true, false, true, true>
-                                     : sqgrad_tc<kMajorK, kTma, kTma, true, false, true>;
-        else if (e == kTma && i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kTma, true) : sqgrad_tc<kMajorK, kTma, kTma, false>;
-        else if (e == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kGatherIm2col, true) : sqgrad_tc<kMajorK, kTma, kGatherIm2col, false>;
-        else if (i == kTma) fn = VGC_TC_FN(kGatherErr, kTma, false);
+        else if (tma_bf) fn = sqgrad_tc<kMajorK, kTma, kTma, true, false, true>;
+        else if (err_tma && in_tma) fn = sqgrad_tc<kMajorK, kTma, kTma, true, true>;
+        else if (err_tma) fn = VGC_TC_FN(kTma, kGatherIm2col, true);
         else fn = VGC_TC_FN(kGatherErr, kGatherIm2col, false);
-        return tc_launch(fn, bt, n_layers, prm, Cout, n_im2col, k_slices, ws, ws_bytes, st, unit, pair, wide);
+        return tc_launch(fn, bt, n_layers, prm, Cout, n_im2col, k_slices, ws, ws_bytes, st, unit);
     }
     prm.ld_m = 1; prm.ld_n = n_im2col;   // m = idx, n = o
-    if (tma_bf) fn = wide   ? sqgrad_tc<kMajorK, kTma, kTma, true, false, true, true, true>
-                     : pair ? sqgrad_tc<kMajorK, kTma, kTma, true, false, true, true>
-                            : sqgrad_tc<kMajorK, kTma, kTma, true, false, true>;
-    else if (e == kTma && i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kTma, true) : sqgrad_tc<kMajorK, kTma, kTma, false>;
-    else if (i == kTma) fn = (a_tmem || ex) ? VGC_TC_FN(kTma, kGatherErr, true) : sqgrad_tc<kMajorK, kTma, kGatherErr, false>;
-    else if (e == kTma) fn = VGC_TC_FN(kGatherIm2col, kTma, false);
+    if (tma_bf) fn = sqgrad_tc<kMajorK, kTma, kTma, true, false, true>;
+    else if (err_tma && in_tma) fn = sqgrad_tc<kMajorK, kTma, kTma, true, true>;
+    else if (err_tma) fn = VGC_TC_FN(kGatherIm2col, kTma, false);
     else fn = VGC_TC_FN(kGatherIm2col, kGatherErr, false);
 #undef VGC_TC_FN
-    return tc_launch(fn, bt, n_layers, prm, n_im2col, Cout, k_slices, ws, ws_bytes, st, unit, pair, wide);
+    return tc_launch(fn, bt, n_layers, prm, n_im2col, Cout, k_slices, ws, ws_bytes, st, unit);
 }
 
 // n_layers layers of one geometry; x, delta, S are host arrays of device pointers

@@ -9,6 +9,32 @@ import paper_1802_06058_b200 as vgc
 F32 = np.float32
 
 
+class Guarded:
+    """A device buffer with a 4-KB band of 0xA5 bytes on either side (the stand-in for a memory checker: a kernel
+    that writes one element before or after a buffer it was given changes a band, and ``check`` sees it).
+    ``t`` is the buffer itself, 256-byte aligned, its last byte directly followed by the upper band."""
+    BAND = 4096
+
+    def __init__(self, numel, dtype=torch.float32, fill=None, device="cuda"):
+        item = torch.empty(0, dtype=dtype).element_size()
+        self.nbytes = int(numel) * item
+        self.raw = torch.full((2 * self.BAND + self.nbytes,), 0xA5, dtype=torch.uint8, device=device)
+        self.t = self.raw[self.BAND:self.BAND + self.nbytes].view(dtype)
+        if fill is not None:
+            self.t.fill_(fill)
+
+    def check(self, what="buffer"):
+        lower, upper = self.raw[:self.BAND], self.raw[self.BAND + self.nbytes:]
+        assert bool((lower == 0xA5).all()), f"{what}: bytes below the buffer were overwritten"
+        assert bool((upper == 0xA5).all()), f"{what}: bytes above the buffer were overwritten"
+
+
+def guarded_like(t):
+    g = Guarded(t.numel(), t.dtype, device=t.device)
+    g.t.copy_(t.reshape(-1))
+    return g
+
+
 class GpuCompressor:
     """State + buffers for repeated vgc_compress calls on one flat buffer."""
 
@@ -17,16 +43,34 @@ class GpuCompressor:
         self.offsets = np.asarray(offsets, np.uint32)
         self.K = len(self.offsets) - 1
         self.offs_dev = vgc.offsets_tensor(self.offsets)
-        self.r = torch.zeros(n, dtype=torch.float32, device="cuda")
-        self.v = torch.zeros(n, dtype=torch.float32, device="cuda")
-        self.out = vgc.MessageBuffers(n if capacity is None else capacity, self.K, n, with_mask=with_mask)
+        # every buffer the kernels write sits between guard bands
+        self._r, self._v = Guarded(n, fill=0.0), Guarded(n, fill=0.0)
+        self.r, self.v = self._r.t, self._v.t
+        cap = n if capacity is None else capacity
+        self.out = vgc.MessageBuffers(cap, self.K, n, with_mask=with_mask)
+        self._words = Guarded(max(cap, 1), torch.int32)
+        self._gexp = Guarded(max(self.K, 1), torch.int32)
+        self.out.words, self.out.group_exp = self._words.t, self._gexp.t
+        self._mask = None
+        if with_mask:
+            self._mask = Guarded(n, torch.uint8, fill=0)
+            self.out.mask = self._mask.t
         ws_bytes = vgc.vgc_compress_workspace_bytes(n, self.K)
-        self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+        self._ws = Guarded(ws_bytes, torch.uint8)
+        self.ws = self._ws.t
+
+    def check_guards(self):
+        for name, gd in (("r", self._r), ("v", self._v), ("words", self._words), ("group_exp", self._gexp),
+                         ("mask", self._mask), ("workspace", self._ws)):
+            if gd is not None:
+                gd.check(name)
 
     def step(self, g, s, alpha, zeta):
         self.out.counters.zero_()
         vgc.vgc_compress(g, s, self.r, self.v, self.offs_dev, alpha, zeta, self.out, self.ws)
-        return self.out.read()
+        res = self.out.read()
+        self.check_guards()
+        return res
 
 
 class OracleCompressor:

@@ -46,21 +46,15 @@ def test_workspace_queries_are_pure_host_functions(lib):
     assert lib.vgc_sqgrad_conv_workspace_bytes(32, 64, 2, 2, 64, 3, 3, 1, 1, 0, 0) == 0   # kernel > image
 
 
-def test_workspace_for_the_pair_forms(lib, monkeypatch):
-    """The tile forms are chosen per call from the environment; the workspace query follows the same switches: the wide
-    pair form always goes through the split-K scratch and may split further, so it never needs less; plain pairs use the
-    single-CTA plan."""
-    shapes = [(32, 256, 14, 14, 1024, 1, 1, 1, 1, 0, 0), (32, 1024, 14, 14, 256, 1, 1, 1, 1, 0, 0),
-              (32, 64, 56, 56, 256, 1, 1, 1, 1, 0, 0), (32, 512, 28, 28, 1024, 1, 1, 2, 2, 0, 0),
-              (32, 64, 56, 56, 64, 3, 3, 1, 1, 1, 1)]
-    plain = [lib.vgc_sqgrad_conv_workspace_bytes(*g) for g in shapes]
-    monkeypatch.setenv("VGC_TC_PAIR", "1")
-    assert [lib.vgc_sqgrad_conv_workspace_bytes(*g) for g in shapes] == plain
-    monkeypatch.setenv("VGC_TC_WIDE", "1")
-    wide = [lib.vgc_sqgrad_conv_workspace_bytes(*g) for g in shapes]
-    assert all(w >= p for w, p in zip(wide, plain))
-    assert wide[0] > 256 + 1024 * 256 * 4 - 1                  # at least one scratch copy of the result
-    assert [lib.vgc_sqgrad_conv_batch_workspace_bytes(3, *g) >= w for g, w in zip(shapes, wide)] == [True] * len(shapes)
+def test_sqgrad_workspace_follows_the_work_plan(lib):
+    """A launch whose tiles are shared between thread blocks needs two partial tiles (64 KB each) per block beside the
+    status word; one whose blocks take whole tiles needs the status word only."""
+    shared = lib.vgc_sqgrad_conv_workspace_bytes(32, 64, 56, 56, 64, 1, 1, 1, 1, 0, 0)        # one tile, 3136 slices
+    assert shared >= 256 + 2 * 148 * 65536
+    whole = lib.vgc_sqgrad_conv_workspace_bytes(2, 640, 8, 8, 1280, 1, 1, 1, 1, 0, 0)         # 50 tiles, 4 slices
+    assert 256 <= whole < 65536
+    assert lib.vgc_sqgrad_conv_batch_workspace_bytes(8, 32, 256, 14, 14, 1024, 1, 1, 1, 1, 0, 0) >= 256
+    assert lib.vgc_sqgrad_conv_batch_workspace_bytes(0, 32, 256, 14, 14, 1024, 1, 1, 1, 1, 0, 0) == 0
 
 
 def test_compress_rejects_bad_arguments_on_the_host(lib):
@@ -82,11 +76,16 @@ def test_compress_rejects_bad_arguments_on_the_host(lib):
 
 def test_decode_and_sqgrad_reject_bad_arguments_on_the_host(lib):
     fake = ctypes.c_void_p(0x1000)
-    views = (vgc._ViewStruct * 1)(vgc._ViewStruct(0x1000, 0x1000, None))
+    views = (vgc._ViewStruct * 1)(vgc._ViewStruct(0x1000, 0x1000, None, 16))
     assert lib.vgc_decode_accumulate(views, 0, fake, 1, 1.0, fake, 10, fake, None) == 0
     assert lib.vgc_decode_accumulate(views, 1, fake, 1, 1.0, fake, 10, fake, None) == 1   # null group_exp
     assert lib.vgc_decode_accumulate(views, 1, fake, 1, 1.0, None, 10, fake, None) == 1
     assert lib.vgc_sqgrad_linear(fake, fake, 4, 0, 8, 1.0, 0, fake, None, 0, None) == 0   # empty layer
+    # empty mini-batch, accumulate: nothing to add, no workspace needed, nothing enqueued
+    assert lib.vgc_sqgrad_linear(None, None, 0, 8, 8, 1.0, 1, fake, None, 0, None) == 0
+    assert lib.vgc_sqgrad_conv(None, None, 0, 3, 8, 8, 5, 3, 3, 1, 1, 1, 1, 1.0, 1, fake, None, 0, None) == 0
+    assert lib.vgc_sqgrad_linear_workspace_bytes(0, 8, 8) == 0
+    assert lib.vgc_sqgrad_linear(fake, fake, 4, 8, 8, 1.0, 0, fake, None, 0, None) == 3   # B > 0 needs its workspace
     assert lib.vgc_sqgrad_linear(fake, fake, -1, 8, 8, 1.0, 0, fake, None, 0, None) == 1
     assert lib.vgc_sqgrad_linear(None, fake, 4, 8, 8, 1.0, 0, fake, None, 0, None) == 1
     assert lib.vgc_sqgrad_conv(fake, fake, 2, 3, 4, 4, 5, 7, 7, 1, 1, 0, 0, 1.0, 0, fake, None, 0, None) == 1

@@ -107,7 +107,59 @@ def test_config2_mlp_100_steps_then_decode_8_messages():
     decode_and_check(comps, msgs, offs, 1861632, 1.0 / W)
 
 
-def test_config3_resnet50_sampled_sqgrad_and_alpha_sweep():
+def sample_entries(spec, rng, at_least=4096):
+    """Flat weight indices to compare: one in every 128 x 128 tile of the layer's [Cout] x [C*k*k] result (the kernels'
+    tile grid, so that every tile, every shared tile's partial sums and every ragged edge is looked at), the four
+    corners, and random ones up to `at_least` (all entries of a layer that has fewer)."""
+    M, N = spec.cout, spec.cin * spec.k * spec.k
+    if M * N <= at_least:
+        return np.arange(M * N)
+    rows0, cols0 = np.arange(0, M, 128), np.arange(0, N, 128)
+    rr = np.minimum(rows0[:, None] + rng.integers(0, 128, (rows0.size, cols0.size)), M - 1)
+    cc = np.minimum(cols0[None, :] + rng.integers(0, 128, (rows0.size, cols0.size)), N - 1)
+    per_tile = (rr * N + cc).reshape(-1)
+    corners = np.array([0, N - 1, (M - 1) * N, M * N - 1])
+    extra = rng.integers(0, M * N, max(at_least - per_tile.size, 0))
+    return np.unique(np.concatenate([per_tile, corners, extra]))
+
+
+def check_sampled_sqgrad(layers, inputs, s, offs, scale, rng):
+    """s (flat, device) against the oracle on sampled entries of every layer; returns the largest relative error."""
+    worst = 0.0
+    for li, spec in enumerate(layers):
+        x, d = inputs[li]
+        idx = sample_entries(spec, rng)
+        got = s[int(offs[li]):int(offs[li + 1])].cpu().numpy()[idx]
+        if spec.kind == "conv":
+            ref = oracle.sqgrad_conv_entries(x.cpu().numpy(), d.cpu().numpy(), (spec.k, spec.k), (spec.stride, spec.stride),
+                                             (spec.pad, spec.pad), scale, idx)
+        else:
+            ref = oracle.sqgrad_linear(x.cpu().numpy(), d.cpu().numpy(), scale=scale).reshape(-1)[idx]
+        assert_close_rel(got, ref)
+        worst = max(worst, float((np.abs(got.astype(np.float64) - ref) / np.maximum(np.abs(ref), 1e-300)).max()))
+    return worst
+
+
+def lockstep_alpha_sweep(s, offs, n):
+    """Three compressor steps per alpha over the whole flat buffer, bit-exact against the oracle fed the same bytes;
+    g is a noise draw with variance s."""
+    root_s = s.sqrt()
+    s_host = s.cpu().numpy()
+    for alpha in (1.0, 2.0, 4.0):
+        gpu, cpu = GpuCompressor(n, offs, with_mask=False), OracleCompressor(n, offs)
+        for t in range(3):
+            gen = torch.Generator(device="cuda"); gen.manual_seed(workloads.seed_for(2, 0, t, 0, 3))
+            g = torch.empty(n, device="cuda").normal_(generator=gen).mul_(root_s)
+            got = gpu.step(g, s, alpha, ZETA)
+            want = cpu.step(g.cpu().numpy(), s_host, alpha, ZETA, want_mask=False)
+            assert_same_message(got, want, check_mask=False)
+        assert_same_state(gpu, cpu)
+        density = want.n_criterion / n
+        assert 0.005 < density < 0.5
+        del gpu
+
+
+def test_config3_resnet50_layer_by_layer_and_alpha_sweep():
     layers, B = workloads.resnet50_layers(), 32
     offs = workloads.group_offsets(layers)
     n = int(offs[-1])
@@ -120,31 +172,41 @@ def test_config3_resnet50_sampled_sqgrad_and_alpha_sweep():
         x, d = workloads.layer_inputs(spec, B, 2, 0, 0, li, "half_normal", 1e-4, "cuda")
         S = s[int(offs[li]):int(offs[li + 1])]
         sqgrad_layer(spec, x, d, scale, S, ws)
-        idx = np.unique(np.concatenate([rng.integers(0, spec.n_params, 24), [0, spec.n_params - 1]]))
-        got = S.cpu().numpy()[idx]
-        if spec.kind == "conv":
-            ref = oracle.sqgrad_conv_entries(x.cpu().numpy(), d.cpu().numpy(), (spec.k, spec.k), (spec.stride, spec.stride),
-                                             (spec.pad, spec.pad), scale, idx)
-        else:
-            ref = oracle.sqgrad_linear(x.cpu().numpy(), d.cpu().numpy(), scale=scale).reshape(-1)[idx]
-        assert_close_rel(got, ref)
+        check_sampled_sqgrad([spec], [(x, d)], S, np.array([0, spec.n_params]), scale, rng)
         del x, d
     assert int(ws[:4].view(torch.int32).item()) == 0
     assert bool((s >= 0).all())
-    # compress over the whole flat buffer for three steps, alpha sweep; g is a noise draw with variance s
-    root_s = s.sqrt()
-    for alpha in (1.0, 2.0, 4.0):
-        gpu, cpu = GpuCompressor(n, offs, with_mask=False), OracleCompressor(n, offs)
-        s_host = s.cpu().numpy()
-        for t in range(3):
-            gen = torch.Generator(device="cuda"); gen.manual_seed(workloads.seed_for(2, 0, t, 0, 3))
-            g = torch.empty(n, device="cuda").normal_(generator=gen).mul_(root_s)
-            got = gpu.step(g, s, alpha, ZETA)
-            want = cpu.step(g.cpu().numpy(), s_host, alpha, ZETA, want_mask=False)
-            assert_same_message(got, want, check_mask=False)
-        assert_same_state(gpu, cpu)
-        density = want.n_criterion / n
-        assert 0.005 < density < 0.5
+    lockstep_alpha_sweep(s, offs, n)
+
+
+def test_config3_as_the_benchmark_runs_it():
+    """The configuration bench.py times, driven through bench.py's own HotPath: full ResNet-50 sizes at batch 32, layers
+    of one geometry grouped into vgc_sqgrad_conv_batch calls of up to 8, the calls spread over 4 streams with a
+    workspace each, replayed as a CUDA graph.  Every layer is compared on at least one entry per 128 x 128 output tile
+    and at least 4096 entries in all; then the compressor runs in lock-step on the resulting sums, and the decoded mean
+    of the benchmark's 8 messages is compared."""
+    import bench
+    hp = bench.HotPath("resnet50", worker=0, n_input_sets=1, n_g_sets=2, n_streams=4)
+    assert hp.n == 25502912 and len(hp.groups) < len(hp.layers)
+    hp.s.fill_(float("nan"))
+    hp.sqgrad(0)                                    # eager once (first-call set-up), then as a graph replay
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        hp.sqgrad(0)
+    hp.s.fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    for ws in [hp.ws_s] + hp.ws_side:
+        assert int(ws[:4].view(torch.int32).item()) == 0
+    assert bool((hp.s >= 0).all())
+    worst = check_sampled_sqgrad(hp.layers, hp.inputs[0], hp.s, hp.offsets, hp.scale, np.random.default_rng(33))
+    assert worst <= 1e-5
+    # compressor + decoder exactly as a step runs them, against the oracle on the same bytes
+    parity = bench.parity_check(hp)
+    assert parity["message_bit_exact"] and parity["state_bit_exact"]
+    assert parity["decode_max_abs"] <= 1e-6 and parity["decode_bit_exact"]
+    lockstep_alpha_sweep(hp.s, hp.offsets, hp.n)
 
 
 def test_config4_vgg16_flat_buffer_compress_only():

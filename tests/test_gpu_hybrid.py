@@ -110,12 +110,9 @@ def hybrid_message(rng, n, density):
     return (idx << 4) | (sign << 3)
 
 
-@pytest.mark.parametrize("path", [None, "merge", "scatter"])
 @pytest.mark.parametrize("n,W,density", [(1, 1, 1.0), (4097, 3, 0.3), (300007, 8, 0.05), (300007, 2, 0.0005),
                                          ((1 << 21) + 3, 16, 0.02), (70000, 70, 0.2)])
-def test_decode(n, W, density, path, monkeypatch):
-    if path:
-        monkeypatch.setenv("VGC_DECODE_PATH", path)
+def test_decode(n, W, density):
     rng = np.random.default_rng(n + W)
     msgs = [hybrid_message(rng, n, density) for _ in range(W)]
     tau, scale = 0.0123, 1.0 / W

@@ -5,6 +5,7 @@ import torch
 
 import oracle
 import paper_1802_06058_b200 as vgc
+from gpu_harness import Guarded, guarded_like
 
 pytestmark = pytest.mark.gpu
 RTOL = 1e-5
@@ -25,24 +26,33 @@ def _check(got, want):
     assert np.all(got[want == 0] == 0)
 
 
+def _guarded_ws(nbytes):
+    g = Guarded(max(nbytes, 256), torch.uint8)
+    g.t.zero_()                                                               # status word starts at 0
+    return g
+
+
 def run_linear(x, d, scale, S0=None):
+    """Result and workspace sit between guard bands: a store past either end of S or of the scratch fails the run."""
     B, n_in = x.shape
     n_out = d.shape[1]
-    S = torch.empty(n_out, n_in, device="cuda") if S0 is None else S0.clone()
-    ws = _ws(vgc.vgc_sqgrad_linear_workspace_bytes(B, n_in, n_out))
-    vgc.vgc_sqgrad_linear(x, d, scale, S, accumulate=S0 is not None, ws=ws)
-    assert _status(ws) == 0
-    return S.cpu().numpy()
+    S = Guarded(n_out * n_in, fill=float("nan")) if S0 is None else guarded_like(S0)
+    ws = _guarded_ws(vgc.vgc_sqgrad_linear_workspace_bytes(B, n_in, n_out))
+    vgc.vgc_sqgrad_linear(x, d, scale, S.t, accumulate=S0 is not None, ws=ws.t)
+    assert _status(ws.t) == 0
+    S.check("S"); ws.check("sqgrad workspace")
+    return S.t.cpu().numpy().reshape(n_out, n_in)
 
 
 def run_conv(x, d, k, s, p, scale, S0=None):
     B, C, H, W = x.shape
     Cout = d.shape[1]
-    S = torch.empty(Cout, C, k, k, device="cuda") if S0 is None else S0.clone()
-    ws = _ws(vgc.vgc_sqgrad_conv_workspace_bytes(B, C, H, W, Cout, k, k, s, s, p, p))
-    vgc.vgc_sqgrad_conv(x, d, (k, k), (s, s), (p, p), scale, S, accumulate=S0 is not None, ws=ws)
-    assert _status(ws) == 0
-    return S.cpu().numpy()
+    S = Guarded(Cout * C * k * k, fill=float("nan")) if S0 is None else guarded_like(S0)
+    ws = _guarded_ws(vgc.vgc_sqgrad_conv_workspace_bytes(B, C, H, W, Cout, k, k, s, s, p, p))
+    vgc.vgc_sqgrad_conv(x, d, (k, k), (s, s), (p, p), scale, S.t, accumulate=S0 is not None, ws=ws.t)
+    assert _status(ws.t) == 0
+    S.check("S"); ws.check("sqgrad workspace")
+    return S.t.cpu().numpy().reshape(Cout, C, k, k)
 
 
 @pytest.mark.parametrize("B,n_in,n_out", [(32, 256, 128), (128, 784, 1024), (128, 1024, 10), (1, 5, 3),
@@ -131,7 +141,7 @@ def test_long_reduction_all_ones_is_exact():
 
 
 @pytest.mark.parametrize("B,C,H,Cout,k,s,p", REPACKED)
-def test_repacked_and_in_place_forms_agree_with_the_oracle(monkeypatch, B, C, H, Cout, k, s, p):
+def test_repacked_forms_agree_with_the_oracle(B, C, H, Cout, k, s, p):
     gen = torch.Generator(device="cuda"); gen.manual_seed(C + H)
     Ho = (H + 2 * p - k) // s + 1
     x = torch.randn(B, C, H, H, device="cuda", generator=gen)
@@ -140,36 +150,41 @@ def test_repacked_and_in_place_forms_agree_with_the_oracle(monkeypatch, B, C, H,
     S0 = torch.rand(Cout, C, k, k, device="cuda")
     want_acc = S0.cpu().numpy().copy()
     oracle.sqgrad_conv(x.cpu().numpy(), d.cpu().numpy(), (k, k), (s, s), (p, p), scale=0.5, out=want_acc)
-    for repack in ("1", "0"):
-        monkeypatch.setenv("VGC_TC_REPACK", repack)
-        _check(run_conv(x, d, k, s, p, 0.5), want)
-        _check(run_conv(x, d, k, s, p, 0.5, S0=S0), want_acc)
+    _check(run_conv(x, d, k, s, p, 0.5), want)
+    _check(run_conv(x, d, k, s, p, 0.5, S0=S0), want_acc)
 
 
-@pytest.mark.parametrize("env", [{"VGC_TC_ATMEM": "0"}, {"VGC_TC_GATHER": "1"}, {"VGC_TC_GATHER": "2"},
-                                 {"VGC_TC_GATHER": "3"}, {"VGC_SQGRAD_PATH": "simt"}, {"VGC_TC_TAPS": "0"}, {"VGC_TC_BF16": "0"}, {"VGC_TC_PAIR": "1"}, {"VGC_TC_WIDE": "1"}])
-@pytest.mark.parametrize("B,C,H,Cout,k,s,p", [(3, 96, 12, 160, 1, 1, 0), (2, 40, 12, 48, 3, 1, 1), (2, 72, 16, 200, 3, 2, 1)])
-def test_every_kernel_variant_gives_the_same_statistic(monkeypatch, env, B, C, H, Cout, k, s, p):
-    """The library picks a kernel form per layer (TMA or gathered tiles, A operand in shared or tensor memory,
-    roles swapped for few output channels, CUDA-core kernel); the switches force each form on shapes that would
-    otherwise take another one."""
-    for key, val in env.items():
-        monkeypatch.setenv(key, val)
+# The library picks a kernel form from the layer's geometry.  One shape (at least) per form that is left:
+KERNEL_FORMS = [  # B, C, H, Cout, k, stride, pad
+    (3, 96, 12, 160, 1, 1, 0),      # both tiles by TMA, errors as the tensor-memory operand, bf16 cross terms
+    (3, 256, 14, 64, 1, 1, 0),      # ... few output channels: the input takes the 128-row side, result written transposed
+    (2, 40, 12, 80, 5, 1, 2),       # errors by TMA, im2col rows gathered element-wise (5x5 kernel)
+    (2, 40, 12, 48, 5, 1, 2),       # ... roles swapped: gathered im2col rows on the 128-row side
+    (2, 40, 9, 80, 5, 1, 2),        # 9x9 planes: neither tile TMA-addressable, both gathered
+    (2, 40, 9, 48, 5, 1, 2),        # ... roles swapped
+    (2, 24, 16, 130, 3, 1, 1),      # three taps at a time
+    (2, 24, 12, 130, 3, 2, 1),      # three taps, stride 2
+    (2, 3, 32, 16, 7, 2, 3),        # seven taps, stride 2
+    (2, 8, 10, 24, 3, 3, 0),        # stride 3, no padding, 3x3 output: gathered, one slice per example
+]
+
+
+@pytest.mark.parametrize("B,C,H,Cout,k,s,p", KERNEL_FORMS)
+def test_every_kernel_form_gives_the_statistic(B, C, H, Cout, k, s, p):
     gen = torch.Generator(device="cuda"); gen.manual_seed(C + H)
     Ho = (H + 2 * p - k) // s + 1
     x = torch.randn(B, C, H, H, device="cuda", generator=gen).abs_()
     d = torch.randn(B, Cout, Ho, Ho, device="cuda", generator=gen) * 1e-4
-    got = run_conv(x, d, k, s, p, 0.5)
     want = oracle.sqgrad_conv(x.cpu().numpy(), d.cpu().numpy(), (k, k), (s, s), (p, p), scale=0.5)
-    _check(got, want)
+    _check(run_conv(x, d, k, s, p, 0.5), want)
+    S0 = torch.rand(Cout, C, k, k, device="cuda", generator=gen) * float(want.mean())
+    _check(run_conv(x, d, k, s, p, 0.5, S0=S0), S0.cpu().numpy().astype(np.float64) + want)
 
 
-@pytest.mark.parametrize("bf16_cross", ["1", "0"])
 @pytest.mark.parametrize("xv,dv", [(1.2345678, 0.0031415926), (1.7320508, 0.0027182818), (0.99999994, 1.0000001)])
-def test_constant_inputs_rounding_errors_all_of_one_sign(monkeypatch, bf16_cross, xv, dv):
+def test_constant_inputs_rounding_errors_all_of_one_sign(xv, dv):
     """Every product has the same rounding error when all inputs are equal, so nothing averages out: the error of
     the split operands (and of the bf16 cross terms) shows at its full size and must still be inside the tolerance."""
-    monkeypatch.setenv("VGC_TC_BF16", bf16_cross)
     B, C, H, Cout = 8, 128, 28, 256
     x = torch.full((B, C, H, H), xv, device="cuda"); d = torch.full((B, Cout, H, H), dv, device="cuda")
     got = run_conv(x, d, 1, 1, 0, 1.0 / B)
@@ -178,30 +193,50 @@ def test_constant_inputs_rounding_errors_all_of_one_sign(monkeypatch, bf16_cross
     _check(got, want)
 
 
-@pytest.mark.parametrize("form", ["VGC_TC_PAIR", "VGC_TC_WIDE"])
-@pytest.mark.parametrize("B,C,H,Cout", [(2, 128, 8, 256), (3, 256, 14, 64), (2, 100, 12, 200), (4, 64, 56, 64),
-                                        (8, 256, 14, 1024), (2, 130, 8, 520), (4, 512, 28, 128), (2, 384, 7, 640),
-                                        (20, 256, 14, 512), (6, 256, 28, 384)])
-def test_pair_forms_of_the_1x1_kernel(monkeypatch, form, B, C, H, Cout):
-    """VGC_TC_PAIR=1: two CTAs of a cluster share a 256 x 128 tile (cta_group::2); VGC_TC_WIDE=1: a 256 x 256 tile with
-    N = 256 instructions where the layer is wide and deep enough (the last two shapes; the last one only with the
-    operands' roles exchanged and with a half-empty second tile), pairs or single CTAs elsewhere.  The shapes cover an
-    even number of row tiles as given, one that is even only with the roles exchanged, one with no even side (falls back
-    to single CTAs), ragged last tiles, the repacked 7x7 form and split reductions; one call and a batch of three layers."""
-    monkeypatch.setenv(form, "1")
+# How a launch's work is cut over the thread blocks depends on the number of tiles and the length of the reduction:
+# whole tiles per block, or an even cut of all slices with tiles shared between blocks (partial tiles through the
+# scratch, a block finishing one tile and starting the next).  Shapes on either side, results written in both layouts.
+@pytest.mark.parametrize("B,C,H,Cout,n_layers", [(8, 256, 14, 1024, 3),      # 48 tiles, 49 slices each: even cut
+                                                  (2, 640, 8, 1280, 1),       # 50 tiles, 4 slices: whole tiles
+                                                  (16, 64, 28, 64, 2),        # 2 tiles, 400 slices: every block inside one tile
+                                                  (4, 192, 16, 40, 5),        # swapped roles, ragged tiles, 10 tiles
+                                                  (3, 1152, 8, 1408, 2)])     # 198 tiles of 6 slices: more tiles than blocks
+def test_work_is_cut_evenly_over_the_blocks(B, C, H, Cout, n_layers):
     gen = torch.Generator(device="cuda"); gen.manual_seed(B + C + Cout)
-    xs = [torch.randn(B, C, H, H, device="cuda", generator=gen).clamp_(min=0) for _ in range(3)]
-    ds = [torch.randn(B, Cout, H, H, device="cuda", generator=gen) * 1e-2 for _ in range(3)]
+    xs = [torch.randn(B, C, H, H, device="cuda", generator=gen).clamp_(min=0) for _ in range(n_layers)]
+    ds = [torch.randn(B, Cout, H, H, device="cuda", generator=gen) * 1e-2 for _ in range(n_layers)]
     wants = [oracle.sqgrad_conv(x.cpu().numpy(), d.cpu().numpy(), (1, 1), (1, 1), (0, 0), scale=0.25) for x, d in zip(xs, ds)]
-    _check(run_conv(xs[0], ds[0], 1, 1, 0, 0.25), wants[0])
-    S0 = torch.rand(Cout, C, 1, 1, device="cuda", generator=gen) * float(wants[0].mean())
-    _check(run_conv(xs[0], ds[0], 1, 1, 0, 0.25, S0=S0), S0.cpu().numpy().astype(np.float64) + wants[0])
-    Ss = [torch.empty(Cout * C, device="cuda") for _ in range(3)]
-    ws = _ws(vgc.vgc_sqgrad_conv_batch_workspace_bytes(3, B, C, H, H, Cout, 1, 1, 1, 1, 0, 0))
-    vgc.vgc_sqgrad_conv_batch(xs, ds, (1, 1), (1, 1), (0, 0), 0.25, Ss, ws=ws)
-    assert _status(ws) == 0
+    flat = Guarded(n_layers * Cout * C, fill=float("nan"))
+    Ss = [flat.t[l * Cout * C:(l + 1) * Cout * C] for l in range(n_layers)]
+    ws = _guarded_ws(vgc.vgc_sqgrad_conv_batch_workspace_bytes(n_layers, B, C, H, H, Cout, 1, 1, 1, 1, 0, 0))
+    vgc.vgc_sqgrad_conv_batch(xs, ds, (1, 1), (1, 1), (0, 0), 0.25, Ss, ws=ws.t)
+    assert _status(ws.t) == 0
+    flat.check("S"); ws.check("sqgrad workspace")
     for S, want in zip(Ss, wants):
         _check(S.cpu().numpy().reshape(Cout, C, 1, 1), want)
+    # accumulate on top of what is there
+    before = flat.t.clone()
+    vgc.vgc_sqgrad_conv_batch(xs, ds, (1, 1), (1, 1), (0, 0), 0.25, Ss, accumulate=True, ws=ws.t)
+    flat.check("S"); ws.check("sqgrad workspace")
+    for l, want in enumerate(wants):
+        base = before[l * Cout * C:(l + 1) * Cout * C].cpu().numpy().astype(np.float64).reshape(Cout, C, 1, 1)
+        _check(Ss[l].cpu().numpy().reshape(Cout, C, 1, 1), base + want)
+
+
+def test_empty_batch_clears_or_keeps_the_result():
+    """B = 0: the sum over the mini-batch is empty."""
+    x = torch.empty(0, 72, device="cuda"); d = torch.empty(0, 40, device="cuda")
+    S = torch.full((40, 72), 3.0, device="cuda")
+    vgc.vgc_sqgrad_linear(x, d, 1.0, S, accumulate=True)
+    assert float(S.min().item()) == 3.0
+    vgc.vgc_sqgrad_linear(x, d, 1.0, S)
+    assert float(S.abs().max().item()) == 0.0
+    xc = torch.empty(0, 8, 6, 6, device="cuda"); dc = torch.empty(0, 16, 6, 6, device="cuda")
+    Sc = torch.full((16 * 8 * 9,), 2.0, device="cuda")
+    vgc.vgc_sqgrad_conv(xc, dc, (3, 3), (1, 1), (1, 1), 1.0, Sc, accumulate=True)
+    assert float(Sc.min().item()) == 2.0
+    vgc.vgc_sqgrad_conv(xc, dc, (3, 3), (1, 1), (1, 1), 1.0, Sc)
+    assert float(Sc.abs().max().item()) == 0.0
 
 
 @pytest.mark.parametrize("n_layers", [1, 3, 9])
@@ -235,32 +270,3 @@ def test_batch_argument_checks():
     with pytest.raises(vgc.VgcError):                         # workspace too small for two layers
         vgc.vgc_sqgrad_conv_batch([x, x], [d, d], (1, 1), (1, 1), (0, 0), 1.0, [S, S.clone()], ws=_ws(256)[:16])
     assert vgc.vgc_sqgrad_conv_batch([], [], (1, 1), (1, 1), (0, 0), 1.0, []) == []
-
-
-def test_plan_hint_changes_the_split_not_the_result():
-    B, C, H, Cout = 4, 256, 14, 512
-    gen = torch.Generator(device="cuda"); gen.manual_seed(5)
-    x = torch.randn(B, C, H, H, device="cuda", generator=gen)
-    d = torch.randn(B, Cout, H, H, device="cuda", generator=gen) * 1e-2
-    want = oracle.sqgrad_conv(x.cpu().numpy(), d.cpu().numpy(), (1, 1), (1, 1), (0, 0), scale=1.0)
-    try:
-        for hint in (4, 1):
-            vgc.vgc_sqgrad_plan_hint(hint)
-            _check(run_conv(x, d, 1, 1, 0, 1.0), want)
-    finally:
-        vgc.vgc_sqgrad_plan_hint(1)
-
-
-def test_mma_rate_probe_reports_the_instruction_floor():
-    """The diagnostic behind the kernel's tensor-pipe ceiling: with M = 128 an instruction takes as long for N = 64 as
-    for N = 128 (so half-width tiles run at half the rate) and less than twice as long for N = 256."""
-    c64, _ = vgc.vgc_probe_mma_rate(0, True, 64, reps=2048, blocks=8)
-    c128, tf128 = vgc.vgc_probe_mma_rate(0, True, 128, reps=2048, blocks=8)
-    c256, tf256 = vgc.vgc_probe_mma_rate(0, True, 256, reps=2048, blocks=8)
-    assert 20 < c128 < 1000 and tf128 > 0
-    assert c64 > 0.9 * c128
-    assert c128 < c256 < 1.9 * c128 and tf256 > tf128
-    with pytest.raises(vgc.VgcError):
-        vgc.vgc_probe_mma_rate(0, True, 100)
-    with pytest.raises(vgc.VgcError):
-        vgc.vgc_probe_mma_rate(2, True, 128)
