@@ -210,6 +210,7 @@ class HotPath:
             self.s_sets = [s for _, s in gs]
             self.ws_s = None
         else:
+            vgc.vgc_sqgrad_plan_hint(n_streams)
             ws_bytes = 16
             # conv layers of one geometry go to the library together (one launch per group of up to 8)
             groups = {}

@@ -129,6 +129,13 @@ vgc_status vgc_sqgrad_conv_exact_batch(int n_layers, const float *const *x, cons
                                        int pad_h, int pad_w, float scale, int accumulate, void *ws, size_t ws_bytes,
                                        vgc_stream_t stream);
 
+/* Planning hint (no counterpart in the paper): how many sqgrad calls the caller keeps in flight side by side on
+ * different streams, each with its own workspace (default 1).  A call's kernel runs one thread block per SM it may
+ * use; alone it takes every SM, with c calls in flight each takes 1/c of them, so that the calls run next to one
+ * another and the start and tail of one is covered by the others.  Process-wide; set it BEFORE asking for workspace
+ * sizes, which depend on it. */
+void vgc_sqgrad_plan_hint(int concurrent_launches);
+
 /* Several conv layers of ONE geometry in one call (the residual stages of a deep network repeat the same
  * layer shapes): layer l computes what vgc_sqgrad_conv computes from x[l], delta[l] into S[l].  The tensor-
  * core path runs up to 8 layers per kernel launch and cuts their combined work evenly over the SMs, which a

@@ -27,7 +27,7 @@ EXPORTS = [
     "vgc_status_string", "vgc_version", "vgc_kernel_launch_count",
     "vgc_sqgrad_linear_workspace_bytes", "vgc_sqgrad_linear",
     "vgc_sqgrad_conv_workspace_bytes", "vgc_sqgrad_conv",
-    "vgc_sqgrad_conv_batch_workspace_bytes", "vgc_sqgrad_conv_batch",
+    "vgc_sqgrad_conv_batch_workspace_bytes", "vgc_sqgrad_conv_batch", "vgc_sqgrad_plan_hint",
     "vgc_sqgrad_conv_exact_workspace_bytes", "vgc_sqgrad_conv_exact",
     "vgc_sqgrad_conv_exact_batch_workspace_bytes", "vgc_sqgrad_conv_exact_batch",
     "vgc_compress_workspace_bytes", "vgc_compress", "vgc_compress_static",
@@ -94,6 +94,7 @@ def load_library():
     lib.vgc_sqgrad_conv_batch_workspace_bytes.restype = sz
     lib.vgc_sqgrad_conv_batch.argtypes = [i, vp, vp, vp] + [i] * 11 + [f, i, vp, sz, vp]
     lib.vgc_sqgrad_conv_batch.restype = i
+    lib.vgc_sqgrad_plan_hint.argtypes = [i]; lib.vgc_sqgrad_plan_hint.restype = None
     lib.vgc_sqgrad_conv_exact_workspace_bytes.argtypes = [i] * 11
     lib.vgc_sqgrad_conv_exact_workspace_bytes.restype = sz
     lib.vgc_sqgrad_conv_exact.argtypes = lib.vgc_sqgrad_conv.argtypes
@@ -238,6 +239,12 @@ def vgc_sqgrad_conv_exact(x, delta, kernel, stride, padding, scale: float, S, ac
                                               _stream(stream))
     _check(st, "vgc_sqgrad_conv_exact")
     return S
+
+
+def vgc_sqgrad_plan_hint(concurrent_launches: int) -> None:
+    """Tell the planner how many sqgrad calls run side by side (streams with separate workspaces): each then
+    takes that share of the SMs.  Set it before asking for workspace sizes."""
+    load_library().vgc_sqgrad_plan_hint(int(concurrent_launches))
 
 
 def vgc_sqgrad_conv_batch_workspace_bytes(n_layers, B, C, H, W, Cout, Kh, Kw, sh, sw, ph, pw, exact: bool = False) -> int:

@@ -10,13 +10,14 @@
 // search).  Then, per call:
 //   sparse (fewer than one word per eight elements): the block's words are added straight into global memory
 //     with fp32 atomics -- u is touched only where a word points;
-//   dense: every WARP owns a contiguous part of the block's range and walks it in sub-tiles of a few hundred
-//     elements held in shared memory.  For a sub-tile it looks at the next words of every message (a window of
-//     32 - 128 words per message, all windows of eight messages in flight together), adds those that fall into the
-//     sub-tile -- message after message, so an element receives its additions in the order w = 0, 1, ..., the
-//     fp32 sequence of a sequential sum, whatever the scheduling -- advances the message cursors past them and
-//     writes the sub-tile out.  u is read and written once, coalesced; there is no block-wide barrier and no
-//     search inside the loop: a warp's cursors simply move forward with its range.
+//   dense: the block walks its range in tiles of up to 24576 elements (96 KB of shared memory, two blocks of 512
+//     threads per SM).  The tile comes in by cp.async while one warp per message finds where the message's run
+//     leaves the tile (a search confined to the at most tile-length words that can lie in it); the messages are
+//     then applied one after the other by the whole block, 8 x 512 words at a time with the next batch's loads in
+//     flight (indices inside a message are distinct, so plain read-modify-writes, a block barrier between
+//     messages): an element receives its additions in the order w = 0, 1, ..., the fp32 sequence of a sequential
+//     sum, whatever the scheduling.  A word's value is one look-up in a 16-entry table per message (its low four
+//     bits are sign and d) when the tile lies inside one weight tensor.  u is read and written once, coalesced.
 // kOverwrite: the range starts from zero instead of the old contents of u (u = scale * sum of the messages).
 // kHybrid: messages of the hybrid algorithm (Algorithm 2) -- every word stands for +-tau, no exponents.
 #include "vgc_common.cuh"
@@ -25,12 +26,6 @@ namespace vgc {
 
 constexpr int kMaxViews = 64;
 constexpr int kDecOffsSmem = 1024;
-constexpr int kTileThreads = 512;
-constexpr int kTileWarps = kTileThreads / 32;
-constexpr int kSubMax = 1280;                    // largest sub-tile of a warp (elements; 5 KB -- two blocks per SM fit)
-constexpr int kSubMin = 256;
-constexpr int kGroup = 8;                        // messages whose windows are in flight together
-constexpr int kWinMax = 4;                       // 32-word loads per lane and window
 
 struct DecodeViews {
     const uint32_t *words[kMaxViews];
@@ -57,16 +52,31 @@ __device__ __forceinline__ uint32_t warp_lower_bound(const uint32_t *__restrict_
     return lo;
 }
 
+constexpr int kTileThreads = 512;
+constexpr int kTileWarps = kTileThreads / 32;
+constexpr int kTileMax = 24576;                  // elements per tile
+constexpr int kTilePre = 8;                      // words per thread in one batch
+
+__device__ __forceinline__ void cp_async_16(void *smem, const void *gmem)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all()
+{
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+
 template <bool kHybrid, bool kOverwrite>
 __global__ void __launch_bounds__(kTileThreads, 2)
 decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *__restrict__ group_offsets, int K,
-             float scale, float tau, float *__restrict__ u, size_t n, uint32_t chunk_elems, uint32_t *dev_status)
+             float scale, float tau, float *__restrict__ u, size_t n, uint32_t chunk_elems, uint32_t tile_elems,
+             uint32_t *dev_status)
 {
-    extern __shared__ __align__(16) float tiles[];               // kTileWarps sub-tiles of kSubMax floats
+    extern __shared__ __align__(16) float tile[];                // tile_elems floats
     __shared__ uint32_t sm_offs[kDecOffsSmem];
-    __shared__ uint32_t cur[kMaxViews];                          // where each message's run enters the block's range
-    __shared__ uint32_t wcur[kTileWarps][kMaxViews];             // per warp: its cursor into each message
-    __shared__ float lut[kTileWarps][kGroup * 16];
+    __shared__ uint32_t cur[kMaxViews], end[kMaxViews];
+    __shared__ float lut[kMaxViews * 16];
     __shared__ uint32_t total_words;
     // the messages' pointers, copied out of the kernel parameters once: parameters cannot be indexed with a
     // run-time value (the compiler turns such an access into a chain of selects over all kMaxViews entries)
@@ -101,6 +111,7 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
         const uint32_t b = warp_lower_bound(words, count, (uint32_t)lo);
         if (lane == 0) {
             cur[w] = b;
+            end[w] = count;
             atomicAdd(&total_words, count);
             if (last_chunk && count && (words[count - 1] >> 4) >= n) atomicOr(dev_status, VGC_DEV_RANGE);   // skipped
         }
@@ -108,8 +119,8 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
     __syncthreads();
     const uint32_t total = total_words;
     if (total == 0 && !kOverwrite) return;
-
     bool bad = false;                                           // a word out of place: skipped, reported
+
     auto value_of = [&](uint32_t word, const int32_t *gexp, int &k) -> float {
         if (kHybrid) return __fmul_rn(scale, (word & 8u) ? -tau : tau);
         const uint32_t idx = word >> 4;
@@ -130,12 +141,11 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
         for (int w = warp; w < W; w += kTileWarps) {
             const uint32_t *words = sm_words[w];
             const int32_t *gexp = sm_gexp[w];
-            const uint32_t end = sm_count[w];
             int k = 0;
-            for (uint32_t i0 = cur[w]; i0 < end; i0 += 32) {           // warp-uniform trip count
+            for (uint32_t i0 = cur[w]; i0 < end[w]; i0 += 32) {       // warp-uniform trip count
                 const uint32_t i = i0 + lane;
-                const uint32_t word = i < end ? words[i] : 0xFFFFFFFFu;
-                const bool in = i < end && (word >> 4) < hi;
+                const uint32_t word = i < end[w] ? words[i] : 0xFFFFFFFFu;
+                const bool in = i < end[w] && (word >> 4) < hi;
                 if (in) {
                     if ((word >> 4) >= lo) atomicAdd(u + (word >> 4), value_of(word, gexp, k));
                     else bad = true;                                 // behind the run's start: the message is not sorted
@@ -147,169 +157,128 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
         return;
     }
 
-    // ---- dense: every warp walks its own part of the block's range
-    // sub-tile length: about 100 words of an average message per sub-tile, so that one window (at most 128 words)
-    // usually holds all of a message's words for it
-    const uint32_t per_msg = total / (uint32_t)W + 1;
-    const uint64_t sub_want = ((uint64_t)n * 100u) / per_msg;
-    uint32_t sub = sub_want > kSubMax ? kSubMax : (sub_want < kSubMin ? kSubMin : (uint32_t)sub_want);
-    sub &= ~127u;
-    // 32-word loads per window: the expected words per message and sub-tile plus a quarter
-    const uint32_t expect = (uint32_t)(((uint64_t)sub * per_msg) / n) + 1;
-    const uint32_t nl = expect > 76 ? 4u : expect > 51 ? 3u : expect > 25 ? 2u : 1u;
-
-    uint32_t wchunk = (uint32_t)((hi - lo + kTileWarps - 1) / kTileWarps);
-    wchunk = (wchunk + 3u) & ~3u;                                // sub-tiles start on 16-byte boundaries of u
-    const size_t wlo = lo + (size_t)warp * wchunk < hi ? lo + (size_t)warp * wchunk : hi;
-    const size_t whi = wlo + wchunk < hi ? wlo + wchunk : hi;
-    if (wlo >= whi) return;
-
-    // where every message's run enters this warp's part: searched inside the block's run, whose words in this
-    // chunk cannot be more than the chunk has elements; eight messages' probes in flight together
-    for (int m0 = 0; m0 < W; m0 += kGroup) {
-        uint32_t s_lo[kGroup], s_hi[kGroup];
-#pragma unroll
-        for (int g = 0; g < kGroup; ++g) {
-            const int m = m0 + g < W ? m0 + g : W - 1;
-            const uint32_t c = cur[m], left = sm_count[m] - c;
-            s_lo[g] = c;
-            s_hi[g] = c + (left < chunk_elems ? left : chunk_elems);
-            if (m0 + g >= W || warp == 0) s_hi[g] = s_lo[g];       // warp 0 starts where the block's run starts
-        }
-        bool busy = true;
-        while (busy) {
-            uint32_t probe[kGroup], step[kGroup];
-#pragma unroll
-            for (int g = 0; g < kGroup; ++g) {
-                step[g] = (s_hi[g] - s_lo[g]) / 32 + 1;
-                const uint32_t pos = s_lo[g] + step[g] * lane;
-                probe[g] = pos < s_hi[g] ? sm_words[m0 + g < W ? m0 + g : W - 1][pos] >> 4 : 0xFFFFFFFFu;
-            }
-            busy = false;
-#pragma unroll
-            for (int g = 0; g < kGroup; ++g) {
-                if (s_hi[g] > s_lo[g]) {                             // warp-uniform
-                    const uint32_t nb = __popc(__ballot_sync(0xffffffffu, probe[g] < (uint32_t)wlo));
-                    if (nb == 0) s_hi[g] = s_lo[g];
-                    else {
-                        const uint32_t new_hi = s_lo[g] + step[g] * nb;
-                        s_lo[g] = s_lo[g] + step[g] * (nb - 1) + 1;
-                        s_hi[g] = new_hi < s_hi[g] ? new_hi : s_hi[g];
-                    }
-                    busy = busy || s_hi[g] > s_lo[g];
-                }
-            }
-        }
-        if (lane < kGroup && m0 + (int)lane < W) {
-            uint32_t mine = 0;
-#pragma unroll
-            for (int g = 0; g < kGroup; ++g) mine = lane == (uint32_t)g ? s_lo[g] : mine;
-            wcur[warp][m0 + lane] = mine;
-        }
-    }
-    __syncwarp();
-
-    float *const tile = tiles + (size_t)warp * kSubMax;
-    const uint32_t tile_addr0 = (uint32_t)__cvta_generic_to_shared(tile);
-    const uint32_t lut_addr = (uint32_t)__cvta_generic_to_shared(&lut[warp][0]);
-    for (size_t t0 = wlo; t0 < whi; t0 += sub) {
-        const uint32_t t_lo = (uint32_t)t0;
-        const uint32_t t_len = (uint32_t)(whi - t0 < sub ? whi - t0 : sub);
-        const uint32_t t_hi = t_lo + t_len;
-        const uint32_t n_vec = t_len / 4;
+    // ---- dense: tile by tile
+    for (size_t t0 = lo; t0 < hi; t0 += tile_elems) {
+        const uint32_t t_len = (uint32_t)(hi - t0 < tile_elems ? hi - t0 : tile_elems);
+        const uint32_t t_hi = (uint32_t)(t0 + t_len);
+        const uint32_t n_vec = t_len / 4;                           // t0 is a multiple of 4 elements
         if (kOverwrite) {
-            for (uint32_t q = lane; q < (t_len + 3) / 4; q += 32) reinterpret_cast<float4 *>(tile)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (uint32_t q = tid; q < (t_len + 3) / 4; q += kTileThreads)
+                reinterpret_cast<float4 *>(tile)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
         } else {
-            for (uint32_t q = lane; q < n_vec; q += 32)
-                reinterpret_cast<float4 *>(tile)[q] = *reinterpret_cast<const float4 *>(u + t0 + 4 * (size_t)q);
-            if (lane < t_len - 4 * n_vec) tile[4 * n_vec + lane] = u[t0 + 4 * n_vec + lane];
+            for (uint32_t q = tid; q < n_vec; q += kTileThreads) cp_async_16(tile + 4 * q, u + t0 + 4 * (size_t)q);
+            if (tid < t_len - 4 * n_vec) tile[4 * n_vec + tid] = u[t0 + 4 * n_vec + tid];
         }
-        int tile_group = -1;                                        // weight tensor of the sub-tile, -1 if it spans several
+        // where every message's run leaves the tile: at most t_len of its words can lie inside
+        for (int w = warp; w < W; w += kTileWarps) {
+            const uint32_t *words = sm_words[w];
+            const uint32_t count = sm_count[w];
+            const uint32_t c = cur[w];
+            const uint32_t span = count - c < t_len ? count - c : t_len;
+            const uint32_t e = c + warp_lower_bound(words + c, span, t_hi);
+            if (lane == 0) end[w] = e;
+        }
+        int tile_group = -1;                                        // weight tensor of the tile, -1 if it spans several
         if (!kHybrid) {
-            tile_group = group_of(offs, K, t_lo);
+            tile_group = group_of(offs, K, (uint32_t)t0);
             if (t_hi - 1 >= offs[tile_group + 1]) tile_group = -1;
         }
+        // the 16 values a word's low four bits (sign, d) can stand for, per message, when the tile lies in one tensor
         const bool use_lut = kHybrid || tile_group >= 0;
-        // element idx lives at tile_addr + 4 * idx (shared-memory byte address)
-        const uint32_t tile_addr = tile_addr0 - 4u * t_lo;
+        if (use_lut)
+            for (int i = tid; i < W * 16; i += kTileThreads) {
+                const int w = i >> 4;
+                const uint32_t code = (uint32_t)i & 15u;
+                float val;
+                if (kHybrid) val = (code & 8u) ? -tau : tau;
+                else {
+                    const uint32_t ebits = (uint32_t)(sm_gexp[w][tile_group] + 127) << 23;
+                    val = __uint_as_float((ebits - ((code & 7u) << 23)) | ((code & 8u) << 28));
+                }
+                lut[i] = __fmul_rn(scale, val);
+            }
+        if (!kOverwrite) cp_async_wait_all();
+        __syncthreads();
 
-        for (int m0 = 0; m0 < W; m0 += kGroup) {
-            // the next words of eight messages: loads of all windows in flight before the first is looked at
-            uint32_t win[kGroup][kWinMax];
+        // messages one after the other, each in batches of kTileBatch words per thread; the loads of the next batch
+        // (of this message or of the next one) are in flight while a batch is applied
+        constexpr uint32_t kBatchWords = kTilePre * kTileThreads;
+        auto batches_of = [&](int w) -> uint32_t { return (end[w] - cur[w] + kBatchWords - 1) / kBatchWords; };
+        auto load_batch = [&](int w, uint32_t b, uint32_t (&dst)[kTilePre]) {
+            const uint32_t first = cur[w] + b * kBatchWords + tid, e = end[w];
+            const uint32_t *p = sm_words[w] + first;
+            if (first + (kTilePre - 1) * kTileThreads < e) {         // whole column of this thread inside the run
 #pragma unroll
-            for (int g = 0; g < kGroup; ++g) {
-                const int m = m0 + g < W ? m0 + g : W - 1;
-                const uint32_t c = wcur[warp][m], cnt = m0 + g < W ? sm_count[m] : 0u;
-                const uint32_t *p = sm_words[m] + c + lane;
+                for (int j = 0; j < kTilePre; ++j) dst[j] = p[j * kTileThreads];
+            } else {
 #pragma unroll
-                for (int j = 0; j < kWinMax; ++j)
-                    win[g][j] = ((uint32_t)j < nl && c + lane + 32u * j < cnt) ? p[32 * j] : 0xFFFFFFFFu;
+                for (int j = 0; j < kTilePre; ++j) dst[j] = first + j * kTileThreads < e ? p[j * kTileThreads] : 0u;
             }
-            __syncwarp();                                           // the previous group's look-ups are done with the table
-            // the 16 values a word's low four bits (sign, d) can stand for, per message of the group
-            if (use_lut)
-                for (uint32_t i = lane; i < kGroup * 16; i += 32) {
-                    const int m = m0 + (int)(i >> 4) < W ? m0 + (int)(i >> 4) : W - 1;
-                    const uint32_t code = i & 15u;
-                    float val;
-                    if (kHybrid) val = (code & 8u) ? -tau : tau;
-                    else {
-                        const uint32_t ebits = (uint32_t)(sm_gexp[m][tile_group] + 127) << 23;
-                        val = __uint_as_float((ebits - ((code & 7u) << 23)) | ((code & 8u) << 28));
-                    }
-                    lut[warp][i] = __fmul_rn(scale, val);
+        };
+        // shared-memory byte addresses: element idx of u lives at tile_addr + 4 * (idx - t0); a word carries
+        // idx << 4, so 4 * idx = (word >> 2) & ~3
+        const uint32_t tile_addr = (uint32_t)__cvta_generic_to_shared(tile) - 4u * (uint32_t)t0;
+        const uint32_t lut_addr = (uint32_t)__cvta_generic_to_shared(lut);
+        auto add_at = [&](uint32_t word, uint32_t lut_w) {
+            // a word of a sorted message lies inside the tile; one that does not (the message is not sorted) is skipped
+            if ((word >> 4) - (uint32_t)t0 >= t_len) { bad = true; return; }
+            const uint32_t at = tile_addr + ((word >> 2) & 0xFFFFFFFCu);
+            float x, v;
+            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(lut_w + ((word & 15u) << 2)));
+            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(x) : "r"(at) : "memory");
+            x = __fadd_rn(x, v);
+            asm volatile("st.shared.f32 [%0], %1;" ::"r"(at), "f"(x) : "memory");
+        };
+        int w = 0;
+        uint32_t b = 0;
+        while (w < W && batches_of(w) == 0) ++w;
+        uint32_t held[kTilePre], next[kTilePre];
+        uint32_t nb = w < W ? batches_of(w) : 0;                     // batches of the current message
+        if (w < W) load_batch(w, 0, held);
+        int k = 0;
+        while (w < W) {
+            int w2 = w;
+            uint32_t b2 = b + 1, nb2 = nb;
+            if (b2 >= nb) {
+                w2 = w + 1; b2 = 0;
+                while (w2 < W && (nb2 = batches_of(w2)) == 0) ++w2;
+            }
+            if (w2 < W) load_batch(w2, b2, next);
+            const uint32_t first = cur[w] + b * kBatchWords + tid, e = end[w];
+            const bool whole = first + (kTilePre - 1) * kTileThreads < e;
+            if (use_lut) {
+                const uint32_t lut_w = lut_addr + 64u * (uint32_t)w;
+                if (whole) {
+#pragma unroll
+                    for (int j = 0; j < kTilePre; ++j) add_at(held[j], lut_w);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < kTilePre; ++j)
+                        if (first + j * kTileThreads < e) add_at(held[j], lut_w);
                 }
-            __syncwarp();
+            } else {
+                const int32_t *gexp = sm_gexp[w];
 #pragma unroll
-            for (int g = 0; g < kGroup; ++g) {
-                const int m = m0 + g;
-                if (m < W) {                                         // warp-uniform
-                    const uint32_t c = wcur[warp][m], cnt = sm_count[m];
-                    const uint32_t lut_m = lut_addr + 64u * (uint32_t)g;
-                    const int32_t *gexp = sm_gexp[m];
-                    int k = 0;
-                    uint32_t adv = 0;
-                    // one batch of 32 words starting at cursor + adv: adds the leading words that fall below the
-                    // sub-tile's end; returns whether all 32 did (then the run may continue in the next batch)
-                    auto batch = [&](uint32_t word) -> bool {
-                        const uint32_t idx = word >> 4;
-                        const bool in = c + adv + lane < cnt && idx < t_hi;
-                        const uint32_t ballot = __ballot_sync(0xffffffffu, in);
-                        const uint32_t lead = ballot == 0xFFFFFFFFu ? 32u : (uint32_t)__ffs(~ballot) - 1u;   // leading words that are in
-                        if (lane < lead) {
-                            if (idx - t_lo < t_len) {               // also false for an index behind the sub-tile
-                                if (use_lut) {
-                                    float x, v;
-                                    const uint32_t at = tile_addr + 4u * idx;
-                                    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(lut_m + ((word & 15u) << 2)));
-                                    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(x) : "r"(at) : "memory");
-                                    x = __fadd_rn(x, v);
-                                    asm volatile("st.shared.f32 [%0], %1;" ::"r"(at), "f"(x) : "memory");
-                                } else {
-                                    tile[idx - t_lo] = __fadd_rn(tile[idx - t_lo], value_of(word, gexp, k));
-                                }
-                            } else bad = true;
-                        }
-                        adv += lead;
-                        return lead == 32u;
-                    };
-                    bool more = true;
-#pragma unroll
-                    for (int j = 0; j < kWinMax; ++j)
-                        if (more && (uint32_t)j < nl) more = batch(win[g][j]);
-                    while (more) {                                   // more words than the window held
-                        const uint32_t pos = c + adv + lane;
-                        more = batch(pos < cnt ? sm_words[m][pos] : 0xFFFFFFFFu);
+                for (int j = 0; j < kTilePre; ++j) {
+                    const uint32_t word = held[j];
+                    if (first + j * kTileThreads < e) {
+                        if ((word >> 4) - (uint32_t)t0 < t_len) tile[(word >> 4) - (uint32_t)t0] += value_of(word, gexp, k);
+                        else bad = true;
                     }
-                    if (lane == 0) wcur[warp][m] = c + adv;
-                    __syncwarp();                                    // the next message may hit the same elements
                 }
             }
+            if (w2 != w) __syncthreads();                            // the next message may hit the same elements
+#pragma unroll
+            for (int j = 0; j < kTilePre; ++j) held[j] = next[j];
+            w = w2; b = b2; nb = nb2;
         }
-        for (uint32_t q = lane; q < n_vec; q += 32)
+        __syncthreads();
+        for (uint32_t q = tid; q < n_vec; q += kTileThreads)
             *reinterpret_cast<float4 *>(u + t0 + 4 * (size_t)q) = reinterpret_cast<const float4 *>(tile)[q];
-        if (lane < t_len - 4 * n_vec) u[t0 + 4 * n_vec + lane] = tile[4 * n_vec + lane];
-        __syncwarp();
+        if (tid < t_len - 4 * n_vec) u[t0 + 4 * n_vec + tid] = tile[4 * n_vec + tid];
+        __syncthreads();
+        for (int w = tid; w < W; w += kTileThreads) cur[w] = end[w];
+        __syncthreads();
     }
     if (bad) atomicOr(dev_status, VGC_DEV_RANGE);
 }
@@ -319,7 +288,8 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
 using namespace vgc;
 
 namespace {
-typedef void (*TilesFn)(const DecodeViews, int, const uint32_t *, int, float, float, float *, size_t, uint32_t, uint32_t *);
+typedef void (*TilesFn)(const DecodeViews, int, const uint32_t *, int, float, float, float *, size_t, uint32_t, uint32_t,
+                        uint32_t *);
 
 vgc_status decode_launch(bool hybrid, bool overwrite, const vgc_message_view *msgs, int W, const uint32_t *group_offsets,
                          int K, float scale, float tau, float *u, size_t n, uint32_t *dev_status, cudaStream_t st)
@@ -345,23 +315,25 @@ vgc_status decode_launch(bool hybrid, bool overwrite, const vgc_message_view *ms
             views.group_exp[w] = m.group_exp;
             views.max_words[w] = m.max_words;
         }
-        // one contiguous range per block, two blocks per SM
+        // one contiguous range per block, two blocks per SM, three or four tiles per range
         size_t chunk = (n + (size_t)sm_count * 2 - 1) / ((size_t)sm_count * 2);
         chunk = (chunk + 3) / 4 * 4;
+        const size_t tiles = (chunk + kTileMax - 1) / kTileMax;
+        const uint32_t tile_elems = (uint32_t)(((chunk + tiles - 1) / tiles + 3) / 4 * 4);
         const unsigned blocks = (unsigned)((n + chunk - 1) / chunk);
         const bool ow = overwrite && w0 == 0;                    // later groups of messages add to the first
         TilesFn fn = hybrid ? (ow ? decode_tiles<true, true> : decode_tiles<true, false>)
                             : (ow ? decode_tiles<false, true> : decode_tiles<false, false>);
-        constexpr size_t kDynSmem = (size_t)kTileWarps * kSubMax * sizeof(float);
         static TilesFn configured[4];
         static int n_configured = 0;
         bool seen = false;
         for (int i = 0; i < n_configured; ++i) seen = seen || configured[i] == fn;
         if (!seen) {
-            VGC_CUDA_OK(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem));
+            VGC_CUDA_OK(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileMax * 4));
             if (n_configured < 4) configured[n_configured++] = fn;
         }
-        fn<<<blocks, kTileThreads, kDynSmem, st>>>(views, wb, group_offsets, K, scale, tau, u, n, (uint32_t)chunk, dev_status);
+        fn<<<blocks, kTileThreads, (size_t)tile_elems * 4, st>>>(views, wb, group_offsets, K, scale, tau, u, n, (uint32_t)chunk,
+                                                                 tile_elems, dev_status);
         count_launch();
     }
     VGC_CUDA_OK(cudaGetLastError());

@@ -10,6 +10,7 @@ vgc_status simt_sqgrad_linear(const float *x, const float *delta, int B, int in,
 vgc_status simt_sqgrad_conv(const float *x, const float *delta, int B, int C, int H, int W, int Cout,
                             int Kh, int Kw, int sh, int sw, int ph, int pw, int Ho, int Wo, float scale,
                             int accumulate, float *S, void *ws, size_t ws_bytes, cudaStream_t st);
+void tc_plan_hint(int concurrent_launches);
 bool tc_linear_supported(int B, int in, int out);
 bool tc_conv_supported(int B, int C, int H, int W, int Cout, int Kh, int Kw, int sh, int sw, int ph, int pw);
 size_t tc_linear_workspace_bytes(int B, int in, int out);
@@ -181,6 +182,8 @@ extern "C" vgc_status vgc_sqgrad_conv_exact(const float *x, const float *delta, 
     return vgc_sqgrad_conv_exact_batch(1, &x, &delta, &S, B, C, H, W, Cout, Kh, Kw, stride_h, stride_w, pad_h, pad_w, scale,
                                        accumulate, ws, ws_bytes, stream);
 }
+
+extern "C" void vgc_sqgrad_plan_hint(int concurrent_launches) { tc_plan_hint(concurrent_launches); }
 
 extern "C" const char *vgc_status_string(int status)
 {

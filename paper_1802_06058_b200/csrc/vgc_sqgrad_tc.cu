@@ -100,7 +100,8 @@ struct Params {
     int chunk;               // slices per accumulator drain
     int unit;                // slices that stay in one block: the reduction is cut between units only
     int units_per_tile;      // k_slices / unit
-    long long units_total;   // layers * tiles * units_per_tile: the launch's work, cut evenly over the blocks
+    int units_total;         // layers * tiles * units_per_tile: the launch's work, cut evenly over the blocks:
+    int units_q, units_r;    // block b owns units [b q + min(b, r), ...) with q = total / blocks, r = total % blocks
     int tiles_x, tiles_y;    // 128-column / 128-row tiles of one layer's result
     uint32_t tx_bytes;       // bytes the TMA loads of one slice deliver
     uint32_t tx_bytes_a;     // of which the A tile's
@@ -663,24 +664,25 @@ struct Seg {
 // The launch's work is the sequence (layer, tile, unit of the tile's reduction), units_total long; block b owns
 // units [b U / G, (b + 1) U / G).  Every role of a block walks the same segments with an iterator of its own.
 struct SegIter {
-    long long pos, end;
+    int pos, end;
     int index;
     __device__ __forceinline__ SegIter(const Params &prm)
     {
-        pos = (long long)blockIdx.x * prm.units_total / gridDim.x;
-        end = (long long)(blockIdx.x + 1) * prm.units_total / gridDim.x;
+        const int b = (int)blockIdx.x;
+        pos = b * prm.units_q + min(b, prm.units_r);
+        end = pos + prm.units_q + (b < prm.units_r ? 1 : 0);
         index = 0;
     }
     __device__ __forceinline__ bool next(const Params &prm, Seg &sg)
     {
         if (pos >= end) return false;
         const int upt = prm.units_per_tile;
-        const long long tile = pos / upt;
-        const int u0 = (int)(pos - tile * upt);
-        const int u1 = end - tile * upt < upt ? (int)(end - tile * upt) : upt;
+        const int tile = pos / upt;
+        const int u0 = pos - tile * upt;
+        const int u1 = min(end - tile * upt, upt);
         const int tiles_layer = prm.tiles_x * prm.tiles_y;
-        sg.layer = (int)(tile / tiles_layer);
-        const int rem = (int)(tile - (long long)sg.layer * tiles_layer);
+        sg.layer = tile / tiles_layer;
+        const int rem = tile - sg.layer * tiles_layer;
         const int tile_m = rem / prm.tiles_x, tile_n = rem - tile_m * prm.tiles_x;
         sg.m0 = tile_m * kBM;
         sg.n0 = tile_n * kBN;
@@ -1240,8 +1242,43 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                             }
                     }
                 }
+            } else if (iter.pos >= iter.end) {
+                // result is contiguous along n, and this is the block's last segment: the pipeline stages are idle
+                // (the last accumulator was complete before we got here), so this warp's 32 x 128 block is transposed
+                // through shared memory and written row by row with consecutive lanes on consecutive addresses
+                float *tile = reinterpret_cast<float *>(smem_gen) + q * (32 * (kBN + 1));
+#pragma unroll
+                for (int j = 0; j < kBN; ++j) tile[lane * (kBN + 1) + j] = __fmul_rn(prm.scale, acc[j]);
+                __syncwarp();
+                for (int r0 = 0; r0 < 32; r0 += 8) {              // eight rows at a time, all loads in flight
+                    float old[8][kBN / 32];
+#pragma unroll
+                    for (int rr = 0; rr < 8; ++rr) {
+                        const int mr = sg.m0 + (int)(q * 32u) + r0 + rr;
+                        const float *src = S + (size_t)mr * prm.ld_m + sg.n0;
+#pragma unroll
+                        for (int cblk = 0; cblk < kBN / 32; ++cblk) {
+                            const int j = cblk * 32 + (int)lane;
+                            old[rr][cblk] = (prm.accumulate && mr < prm.M && j < n_valid) ? src[j] : 0.f;
+                        }
+                    }
+#pragma unroll
+                    for (int rr = 0; rr < 8; ++rr) {
+                        const int mr = sg.m0 + (int)(q * 32u) + r0 + rr;
+                        float *dst = S + (size_t)mr * prm.ld_m + sg.n0;
+#pragma unroll
+                        for (int cblk = 0; cblk < kBN / 32; ++cblk) {
+                            const int j = cblk * 32 + (int)lane;
+                            if (mr < prm.M && j < n_valid) {
+                                const float res = tile[(r0 + rr) * (kBN + 1) + j];
+                                dst[j] = prm.accumulate ? __fadd_rn(old[rr][cblk], res) : res;
+                            }
+                        }
+                    }
+                }
             } else if (m < prm.M) {
-                // result is contiguous along n: every lane owns a row and writes it 16 bytes at a time (the halves of a
+                // result is contiguous along n, more segments follow (the pipeline is busy with the next one): every
+                // lane owns a row and writes it 16 bytes at a time (the halves of a
                 // 32-byte sector arrive in consecutive instructions and are merged in L2); rows whose pitch is not a
                 // multiple of 16 bytes go element by element
                 float *row = S + (size_t)m * prm.ld_m + sg.n0;
@@ -1303,16 +1340,18 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
 struct ResultPtrs { float *S[kMaxBatch]; };
 
 __global__ void __launch_bounds__(256)
-sqgrad_tc_combine(const float *__restrict__ partial, int n_blocks, long long units_total, int units_per_tile,
+sqgrad_tc_combine(const float *__restrict__ partial, int units_q, int units_r, int units_per_tile,
                   int tiles_x, int tiles_y, int M, int N, float scale, int accumulate, const ResultPtrs results,
                   long long ld_m, long long ld_n)
 {
     __shared__ float patch[8][33];
     const int tile = blockIdx.x >> 6, sub = blockIdx.x & 63;
-    // the blocks that hold the tile's first and last unit (block b owns units [b U / G, (b + 1) U / G))
-    const long long t_lo = ((long long)blockIdx.y * (tiles_x * tiles_y) + tile) * units_per_tile;
-    const int b_first = (int)(((t_lo + 1) * n_blocks - 1) / units_total);
-    const int b_last = (int)(((t_lo + units_per_tile) * n_blocks - 1) / units_total);
+    // the blocks that hold the tile's first and last unit: the first units_r blocks own units_q + 1 units each, the
+    // others units_q
+    const int t_lo = ((int)blockIdx.y * (tiles_x * tiles_y) + tile) * units_per_tile;
+    const int big = units_r * (units_q + 1);
+    auto block_of = [&](int u) -> int { return u < big ? u / (units_q + 1) : units_r + (u - big) / units_q; };
+    const int b_first = block_of(t_lo), b_last = block_of(t_lo + units_per_tile - 1);
     if (b_first == b_last) return;
     float *__restrict__ S = results.S[blockIdx.y];                         // blockIdx.y: layer of the batch
     const int tx = tile % tiles_x, ty = tile / tiles_x;
@@ -1324,7 +1363,7 @@ sqgrad_tc_combine(const float *__restrict__ partial, int n_blocks, long long uni
     if (tx * kBN + j < N) {
         // the first block's part of this tile is that block's last segment unless its range starts with the tile;
         // every later block's part is its first segment
-        const long long lo_first = (long long)b_first * units_total / n_blocks;
+        const int lo_first = b_first * units_q + min(b_first, units_r);
         const size_t within = (size_t)j * kBM + r0 + lane;
         const float *src0 = partial + (size_t)(2 * b_first + (lo_first < t_lo ? 1 : 0)) * (kBM * kBN) + within;
         sum = __ldcs(src0);
@@ -1396,11 +1435,13 @@ static bool make_map(CUtensorMap *map, const float *base, int rank, const cuuint
 // sum per instruction), so an accumulator is handed to the round-to-nearest register sums after at most 8 slices
 // (96 instructions): results then sit 1 - 3e-6 below the exact sum, against the 1e-5 bound.
 constexpr int kChunk = 8;
-constexpr int kBlocksMax = 148;          // thread blocks of a launch: one per SM of a B200
+constexpr int kSmCount = 148;            // SMs of a B200
+// how many sqgrad launches the caller keeps in flight side by side (vgc_sqgrad_plan_hint)
+static int g_concurrent = 1;
 
 struct Plan {
     int unit, units_per_tile, blocks, tiles_x, tiles_y;
-    long long units_total;
+    int units_total;
     bool partials;           // some tile is shared by several blocks: partial tiles go through the scratch
 };
 
@@ -1416,27 +1457,51 @@ static Plan make_plan(int M, int N, int k_slices, int n_layers, int unit_min)
     p.tiles_x = (N + kBN - 1) / kBN;
     p.tiles_y = (M + kBM - 1) / kBM;
     const long long tiles = (long long)p.tiles_x * p.tiles_y * n_layers;
-    // (a) whole tiles
-    const long long waves = (tiles + kBlocksMax - 1) / kBlocksMax;
-    const long long blocks_a = (tiles + waves - 1) / waves;
-    const long long cost_a = ((tiles + blocks_a - 1) / blocks_a) * k_slices;
-    // (b) even cut
     const long long upt = k_slices / unit_min, units = tiles * upt;
-    const long long blocks_b = units < kBlocksMax ? units : kBlocksMax;
-    const long long cost_b = ((units + blocks_b - 1) / blocks_b) * unit_min + 14;
-    bool even = cost_b < cost_a;
+    bool even;
+    long long blocks;
+    if (g_concurrent > 1) {
+        // Next to other launches the hardware's block scheduler does the balancing: blocks of all launches in flight
+        // queue for the SMs, so a launch is cut into many short blocks -- each tile's reduction into as many parts as
+        // fit one wave of SMs -- and a partly filled wave costs nothing (the neighbours' blocks take the idle SMs).
+        long long parts = kSmCount / tiles;
+        parts = parts > upt ? upt : (parts < 1 ? 1 : parts);
+        even = parts > 1;
+        blocks = tiles * parts;
+    } else {
+        // Alone, the launch is one block per SM at most.  Two candidates, costs in slice times: whole tiles per block
+        // (a block's longest range), or an even cut of all slices (plus what the combine pass adds to the call: its
+        // launch and the partial tiles' round trip, about 14 slices' worth).
+        const long long waves = (tiles + kSmCount - 1) / kSmCount;
+        const long long blocks_a = (tiles + waves - 1) / waves;
+        const long long cost_a = ((tiles + blocks_a - 1) / blocks_a) * k_slices;
+        const long long blocks_b = units < kSmCount ? units : kSmCount;
+        const long long cost_b = ((units + blocks_b - 1) / blocks_b) * unit_min + 14;
+        even = cost_b < cost_a;
+        blocks = even ? blocks_b : blocks_a;
+    }
+    if (even && units >= (1LL << 31)) {          // unit positions are 32-bit in the kernel: whole tiles then
+        even = false;
+        blocks = tiles < kSmCount ? tiles : kSmCount;
+    }
     p.unit = even ? unit_min : k_slices;
     p.units_per_tile = even ? (int)upt : 1;
-    p.units_total = even ? units : tiles;
-    p.blocks = (int)(even ? blocks_b : blocks_a);
+    p.units_total = (int)(even ? units : tiles);
+    p.blocks = (int)blocks;
     p.partials = false;
-    for (long long b = 1; b < p.blocks && !p.partials; ++b) p.partials = (b * p.units_total / p.blocks) % p.units_per_tile != 0;
+    const int q = p.units_total / p.blocks, r = p.units_total % p.blocks;
+    for (int b = 1; b < p.blocks && !p.partials; ++b) p.partials = (b * q + (b < r ? b : r)) % p.units_per_tile != 0;
     return p;
 }
 
 }  // namespace tc
 
 using namespace tc;
+
+void tc_plan_hint(int concurrent_launches)
+{
+    g_concurrent = concurrent_launches > 1 ? concurrent_launches : 1;
+}
 
 bool tc_linear_supported(int B, int in, int out)
 {
@@ -1475,6 +1540,7 @@ static vgc_status tc_launch(KernelFn kernel, const Batch &bt, int n_layers, Para
     }
     prm.M = M; prm.N = N; prm.k_slices = k_slices;
     prm.unit = plan.unit; prm.units_per_tile = plan.units_per_tile; prm.units_total = plan.units_total;
+    prm.units_q = plan.units_total / plan.blocks; prm.units_r = plan.units_total % plan.blocks;
     prm.tiles_x = plan.tiles_x; prm.tiles_y = plan.tiles_y;
     prm.chunk = kChunk;
     prm.status = static_cast<uint32_t *>(ws);
@@ -1485,7 +1551,7 @@ static vgc_status tc_launch(KernelFn kernel, const Batch &bt, int n_layers, Para
         ResultPtrs results = {};
         for (int l = 0; l < n_layers; ++l) results.S[l] = bt.S[l];
         sqgrad_tc_combine<<<dim3((unsigned)(plan.tiles_x * plan.tiles_y * 64), (unsigned)n_layers), 256, 0, st>>>(
-            prm.partial, plan.blocks, plan.units_total, plan.units_per_tile, plan.tiles_x, plan.tiles_y, M, N, prm.scale,
+            prm.partial, prm.units_q, prm.units_r, plan.units_per_tile, plan.tiles_x, plan.tiles_y, M, N, prm.scale,
             prm.accumulate, results, prm.ld_m, prm.ld_n);
         count_launch();
     }

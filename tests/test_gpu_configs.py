@@ -186,6 +186,13 @@ def test_config3_as_the_benchmark_runs_it():
     and at least 4096 entries in all; then the compressor runs in lock-step on the resulting sums, and the decoded mean
     of the benchmark's 8 messages is compared."""
     import bench
+    try:
+        _benchmark_configuration(bench)
+    finally:
+        vgc.vgc_sqgrad_plan_hint(1)               # HotPath asked for a quarter of the SMs per call; process-wide
+
+
+def _benchmark_configuration(bench):
     hp = bench.HotPath("resnet50", worker=0, n_input_sets=1, n_g_sets=2, n_streams=4)
     assert hp.n == 25502912 and len(hp.groups) < len(hp.layers)
     hp.s.fill_(float("nan"))

@@ -270,3 +270,17 @@ def test_batch_argument_checks():
     with pytest.raises(vgc.VgcError):                         # workspace too small for two layers
         vgc.vgc_sqgrad_conv_batch([x, x], [d, d], (1, 1), (1, 1), (0, 0), 1.0, [S, S.clone()], ws=_ws(256)[:16])
     assert vgc.vgc_sqgrad_conv_batch([], [], (1, 1), (1, 1), (0, 0), 1.0, []) == []
+
+
+def test_plan_hint_changes_the_share_of_the_sms_not_the_result():
+    B, C, H, Cout = 4, 256, 14, 512
+    gen = torch.Generator(device="cuda"); gen.manual_seed(5)
+    x = torch.randn(B, C, H, H, device="cuda", generator=gen)
+    d = torch.randn(B, Cout, H, H, device="cuda", generator=gen) * 1e-2
+    want = oracle.sqgrad_conv(x.cpu().numpy(), d.cpu().numpy(), (1, 1), (1, 1), (0, 0), scale=1.0)
+    try:
+        for hint in (4, 148, 1000, 1):
+            vgc.vgc_sqgrad_plan_hint(hint)
+            _check(run_conv(x, d, 1, 1, 0, 1.0), want)
+    finally:
+        vgc.vgc_sqgrad_plan_hint(1)
