@@ -331,6 +331,39 @@ vgc_status vgc_decode_accumulate_hybrid(const vgc_message_view *msgs, int W, flo
 vgc_status vgc_decode_sum_hybrid(const vgc_message_view *msgs, int W, float tau, float scale, float *u, size_t n,
                                  uint32_t *dev_status, vgc_stream_t stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * (5) Index compression of a packed message (Sec. 4.2, last paragraph: the index field can be stored in
+ * fewer bits).  The paper names the idea without a format; this one is the library's.  The words of a
+ * message are in ascending index order, so the 28-bit index field is replaced by the difference to the
+ * previous index:  v = (idx_i - idx_{i-1}) << 4 | (word_i & 15), written in the base-128 variable-length
+ * code (seven bits per byte, least significant first, top bit = "another byte follows": 1 to 5 bytes).
+ * Words are taken in runs of VGC_PACK_RUN; every run starts from idx_{-1} = 0, so runs are independent.
+ *
+ *   stream = [table: (runs + 1) x uint32 little endian][payload]     runs = ceil(nnz / VGC_PACK_RUN)
+ *            table[j] = offset of run j's first byte inside the payload, table[runs] = payload length
+ *
+ * At send densities of 1e-2 .. 1e-3 a word takes 2 bytes instead of 4.  The 4-bit value field, the
+ * per-tensor exponents and the word count travel unchanged.
+ *
+ * vgc_pack_indices     words [min(*nnz, max_words)] (device, as vgc_compress wrote them) -> packed (device,
+ *                      at least vgc_pack_bound_bytes(max_words) bytes for a guaranteed fit); *packed_bytes
+ *                      (device) receives the stream's length.  A too small buffer: the stream is cut,
+ *                      VGC_DEV_CAPACITY is set and *packed_bytes still holds the length that was needed.
+ *                      ws: vgc_pack_workspace_bytes(max_words) bytes of device scratch.
+ * vgc_unpack_indices   the inverse: rebuilds min(*nnz, max_words) words from a stream.  A run whose bytes do not
+ *                      parse (wrong length, a number longer than five bytes) sets VGC_DEV_RANGE and its words are
+ *                      written as 0xFFFFFFFF, an index no buffer has, so that a decoder skips them.
+ * Both only enqueue work on `stream`; nnz is read on the device.
+ * ------------------------------------------------------------------------------------------- */
+#define VGC_PACK_RUN 256
+size_t vgc_pack_bound_bytes(uint32_t max_words);
+size_t vgc_pack_workspace_bytes(uint32_t max_words);
+vgc_status vgc_pack_indices(const uint32_t *words, const uint32_t *nnz, uint32_t max_words, uint8_t *packed,
+                            size_t packed_capacity, uint32_t *packed_bytes, uint32_t *dev_status, void *ws,
+                            size_t ws_bytes, vgc_stream_t stream);
+vgc_status vgc_unpack_indices(const uint8_t *packed, const uint32_t *nnz, uint32_t max_words, uint32_t *words,
+                              uint32_t *dev_status, vgc_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

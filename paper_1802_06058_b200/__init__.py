@@ -34,6 +34,7 @@ EXPORTS = [
     "vgc_decode_accumulate", "vgc_step_host",
     "vgc_compress_hybrid_workspace_bytes", "vgc_compress_hybrid", "vgc_decode_accumulate_hybrid",
     "vgc_decode_sum", "vgc_decode_sum_hybrid",
+    "vgc_pack_bound_bytes", "vgc_pack_workspace_bytes", "vgc_pack_indices", "vgc_unpack_indices",
 ]
 
 
@@ -124,6 +125,12 @@ def load_library():
     lib.vgc_decode_accumulate_hybrid.restype = i
     lib.vgc_decode_sum_hybrid.argtypes = lib.vgc_decode_accumulate_hybrid.argtypes
     lib.vgc_decode_sum_hybrid.restype = i
+    lib.vgc_pack_bound_bytes.argtypes = [ctypes.c_uint32]; lib.vgc_pack_bound_bytes.restype = sz
+    lib.vgc_pack_workspace_bytes.argtypes = [ctypes.c_uint32]; lib.vgc_pack_workspace_bytes.restype = sz
+    lib.vgc_pack_indices.argtypes = [vp, vp, ctypes.c_uint32, vp, sz, vp, vp, vp, sz, vp]
+    lib.vgc_pack_indices.restype = i
+    lib.vgc_unpack_indices.argtypes = [vp, vp, ctypes.c_uint32, vp, vp, vp]
+    lib.vgc_unpack_indices.restype = i
     _lib = lib
     return lib
 
@@ -474,6 +481,36 @@ def vgc_decode_accumulate_hybrid(messages: Sequence, tau: float, scale: float, u
             _dev(dev_status, torch.int32, "dev_status"), _stream(stream))
     _check(st, "vgc_decode_accumulate_hybrid")
     return u
+
+
+# ------------------------------------------------------------------------------------------ (5)
+def vgc_pack_bound_bytes(max_words: int) -> int:
+    return load_library().vgc_pack_bound_bytes(int(max_words))
+
+
+def vgc_pack_workspace_bytes(max_words: int) -> int:
+    return load_library().vgc_pack_workspace_bytes(int(max_words))
+
+
+def vgc_pack_indices(words, nnz, packed, packed_bytes, dev_status, ws, stream=None):
+    """words int32 [max_words] + nnz int32 [1] (device) -> packed uint8 (device): the index field as differences in
+    the base-128 code; packed_bytes int32 [1] (device) receives the stream's length."""
+    wp, wb = _ws(ws)
+    st = load_library().vgc_pack_indices(_dev(words, torch.int32, "words"), _dev(nnz, torch.int32, "nnz"), words.numel(),
+                                         _dev(packed, torch.uint8, "packed"), packed.numel(),
+                                         _dev(packed_bytes, torch.int32, "packed_bytes"),
+                                         _dev(dev_status, torch.int32, "dev_status"), wp, wb, _stream(stream))
+    _check(st, "vgc_pack_indices")
+    return packed
+
+
+def vgc_unpack_indices(packed, nnz, words, dev_status, stream=None):
+    """The inverse of vgc_pack_indices: rebuilds min(nnz, words.numel()) words (device int32)."""
+    st = load_library().vgc_unpack_indices(_dev(packed, torch.uint8, "packed"), _dev(nnz, torch.int32, "nnz"), words.numel(),
+                                           _dev(words, torch.int32, "words"), _dev(dev_status, torch.int32, "dev_status"),
+                                           _stream(stream))
+    _check(st, "vgc_unpack_indices")
+    return words
 
 
 def _host(t: torch.Tensor, dtype, name: str) -> int:

@@ -63,10 +63,18 @@ constexpr int kBK = 32;             // k per pipeline slice (= 128 bytes of fp32
 // lo parts, which only exist between the transform and the MMAs that consume them.
 constexpr int kRawSlots = VGC_TC_RAW_SLOTS;
 constexpr int kLoSlots = VGC_TC_LO_SLOTS;
-constexpr int kThreadsTc = 448;
-constexpr int kTransformWarps = 8;
-constexpr int kTransformThreads = 32 * kTransformWarps;
+#ifndef VGC_TC_GROUPS
+#define VGC_TC_GROUPS 2
+#endif
+// Transform warps: groups of four warps; in the forms whose slices are taken by one group each, the groups work on
+// consecutive slices side by side (a slice's transform is a chain of shared-memory round trips, waits and fences: its
+// latency, not the arithmetic, sets the pace, so slices in flight are what counts).  The element-wise gathers share a
+// slice among eight warps (the first two groups).
+constexpr int kGroups = VGC_TC_GROUPS;
+constexpr int kTransformWarps = 4 * kGroups;
+constexpr int kGatherThreads = 256;                                 // threads sharing a slice in the one-group forms
 constexpr int kEpilogueWarps = 4;
+constexpr int kThreadsTc = 32 * (2 + kTransformWarps + kEpilogueWarps);
 constexpr uint32_t kRawBytesA = kBM * kBK * 4;                      // 16 KB
 constexpr uint32_t kRawBytesB = kBN * kBK * 4;                      // 16 KB
 constexpr uint32_t kRawStageBytes = kRawBytesA + kRawBytesB;        // 32 KB: [A raw/hi][B raw/hi], same for lo
@@ -78,7 +86,7 @@ constexpr int kLoSlotsAT = 2 * kLoSlots;
 // Pure TMA form with A in tensor memory ("split rings"): the raw A tile is dead as soon as the transform has
 // read it, long before the MMAs of its slice retire.  It therefore gets a ring of its own that is freed
 // early, and the 16-KB units this saves hold more B tiles: more slices in flight from the same shared memory.
-constexpr int kSplitA = 4, kSplitB = 7, kSplitLo = 3;              // 16-KB units: A raw, B raw/hi, B lo (+ A in TMEM)
+constexpr int kSplitA = 4, kSplitB = kGroups > 2 ? 6 : 7, kSplitLo = kGroups > 2 ? 4 : 3;   // 16-KB units: A raw, B raw/hi, B lo (+ A in TMEM)
 static_assert((kSplitA + kSplitB + kSplitLo) * kRawBytesA <= (kRawSlots + kLoSlots) * kRawStageBytes, "smem budget");
 constexpr uint32_t kTmemColsA = 64;                                 // per slot: 32 columns hi + 32 columns lo
 constexpr uint32_t kTmemCols = 512;                                 // two accumulator buffers + the A operand ring
@@ -335,7 +343,7 @@ __device__ __forceinline__ void split_store(uint8_t *hi_tile, uint8_t *lo_tile, 
     *reinterpret_cast<uint4 *>(lo_tile + off) = l;
 }
 
-constexpr int kRowsPerThread = kBM * 8 / kTransformThreads;        // 4 gathered chunks per thread per tile
+constexpr int kRowsPerThread = kBM * 8 / kGatherThreads;        // 4 gathered chunks per thread per tile
 
 // The four rows (row0 + 32*i) of a gathered tile that one transform thread owns.
 template <int kMode>
@@ -758,13 +766,13 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         abort_flag = 0;
         for (int i = 0; i < kNB; ++i) {
             mbar_init(smem_u32(&raw_full[i]), 1);
-            mbar_init(smem_u32(&op_full[i]), kTwoGroups ? kTransformWarps / 2 : kTransformWarps);
+            mbar_init(smem_u32(&op_full[i]), kTwoGroups ? 4 : kGatherThreads / 32);
             mbar_init(smem_u32(&empty[i]), 1);
         }
         if (kSplit)
             for (int i = 0; i < kNA; ++i) {
                 mbar_init(smem_u32(&a_full[i]), 1);
-                mbar_init(smem_u32(&a_empty[i]), kTransformWarps / 2);
+                mbar_init(smem_u32(&a_empty[i]), 4);
             }
         for (int i = 0; i < kLoSlotsAT; ++i) mbar_init(smem_u32(&lo_empty[i]), 1);      // unused, kept initialised
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&acc_full[i]), 1); mbar_init(smem_u32(&acc_empty[i]), kEpilogueWarps); }
@@ -945,11 +953,12 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         }
     } else if (warp < 2 + kTransformWarps) {
         // ================= transform warps: square and split into TF32 hi / lo =================
-        const int t = (int)threadIdx.x - 64;                               // 0..255
-        // With nothing to gather the eight warps work as two groups of four that take alternate slices: the
-        // waits, fences and tensor-memory stores of one slice then overlap the arithmetic of the next one.
-        // The same split is used when the B tile is gathered three taps at a time next to a TMA-fed A tile.
-        constexpr int kTT = kTwoGroups ? kTransformThreads / 2 : kTransformThreads;   // threads sharing a slice
+        const int t = (int)threadIdx.x - 64;                               // 0 .. 128 * kGroups - 1
+        // With nothing to gather the warps work as groups of four that take consecutive slices in turn: the waits,
+        // fences and tensor-memory stores of one slice then overlap the arithmetic of the others.  The same split
+        // is used when the B tile is gathered several taps at a time next to a TMA-fed A tile.  The element-wise
+        // gathers share every slice among the first eight warps; further warps have nothing to do there.
+        constexpr int kTT = kTwoGroups ? 128 : kGatherThreads;             // threads sharing a slice
         const int group = kTwoGroups ? (t >> 7) : 0;
         const int tt = kTwoGroups ? (t & 127) : t;
         const int kq = tt & 7, row0 = tt >> 3;                             // gathered chunks: rows row0 + 32*i, k = 4*kq..4*kq+3
@@ -1103,6 +1112,7 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
         bool ok = true;
         SegIter iter(prm);
         Seg sg;
+        if (!kTwoGroups && t >= kGatherThreads) ok = false;
         while (ok && iter.next(prm, sg)) {
             const int n_slices = sg.s_end - sg.s_begin;
             if (kAnyGather) {
@@ -1112,15 +1122,17 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
                 pblk = sg.s_begin - z * prm.p_slices;
             }
             if (kTwoGroups) {
-                // this group's slices: those whose block-wide number has the group's parity.  With a gathered tile:
-                // one register set per thread -- the other group's work covers this group's load latency
+                // this group's slices: those whose block-wide number is the group's modulo kGroups.  With a gathered
+                // tile: one register set per thread -- the other groups' work covers this group's load latency
                 // (measured faster than two sets in turn)
-                const int i_first = ((it0 & 1) == group) ? 0 : 1;
-                if (kAnyGather && i_first) advance();
-                for (int i = i_first; i < n_slices; i += 2) {
+                const int i_first = (group - it0 % kGroups + kGroups) % kGroups;
+                if (kAnyGather)
+                    for (int sk = 0; sk < i_first; ++sk) advance();
+                for (int i = i_first; i < n_slices; i += kGroups) {
                     if (kAnyGather) gather(a0, b0);
                     if (!process(it0 + i, a0, b0)) { ok = false; break; }
-                    if (kAnyGather) { advance(); advance(); }
+                    if (kAnyGather)
+                        for (int sk = 0; sk < kGroups; ++sk) advance();
                 }
             } else {
                 // two register sets in turn: the loads of slice i+1 are in flight while slice i is transformed

@@ -85,7 +85,7 @@ def test_size_in_closed_form_round_trip_and_second_writing(n, density, seed):
     assert packed[4 * (runs + 1):4 * (runs + 1) + len(want)].tobytes() == want
     # round trip
     assert np.array_equal(oracle.unpack_indices(packed, m), words)
-    if density <= 1e-2 and m > 1000:
+    if 1e-3 <= density <= 1e-2 and m > 1000:
         assert packed.size < 0.7 * 4 * m            # the point of it: well under four bytes a word
 
 
