@@ -120,6 +120,25 @@ def test_dense_calls_add_in_message_order_bit_for_bit(n, K, W, density):
     assert int(st.item()) == 0 and np.array_equal(gu.t.cpu().numpy().view(np.uint32), ref.view(np.uint32))
 
 
+@pytest.mark.parametrize("n,K,W,density,exps,scale", [(1 << 20, 54, 8, 0.14, (-10, -8), 0.125), (2500000, 40, 17, 0.05, (-14, -9), 1.0),
+                                                      (700001, 5, 64, 0.05, (-3, 0), 2.0 ** -6), (400003, 9, 5, 0.3, (-20, -6), 0.5),
+                                                      (300000, 3, 4, 0.5, (-125, -120), 1.0), (300000, 3, 4, 0.5, (100, 110), 0.25)])
+def test_decode_sum_over_the_exponent_range_bit_for_bit(n, K, W, density, exps, scale):
+    """vgc_decode_sum against the oracle's sequential sum, bit for bit, with power-of-two scales, many messages per
+    element, exponents close together and far apart, values next to the smallest normal number and large ones."""
+    offs = random_offsets(np.random.default_rng(31), n, K)
+    msgs = [workloads.random_message(n, offs, density, seed=700 + w, device="cuda", exp_lo=exps[0], exp_hi=exps[1])
+            for w in range(W)]
+    gu = Guarded(n, fill=float("nan"))
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    triples = [(w, torch.tensor([w.numel()], dtype=torch.int32, device="cuda"), e) for w, e in msgs]
+    vgc.vgc_decode_sum(triples, vgc.offsets_tensor(offs), scale, gu.t, st)
+    gu.check("u")
+    ref = np.zeros(n, F32)
+    oracle.decode_accumulate([(w.cpu().numpy().view(np.uint32), e.cpu().numpy()) for w, e in msgs], offs, scale, ref)
+    assert int(st.item()) == 0 and np.array_equal(gu.t.cpu().numpy().view(np.uint32), ref.view(np.uint32))
+
+
 @pytest.mark.parametrize("n,K,W,density", [(400003, 9, 5, 0.002), (2500000, 40, 17, 0.0005)])
 def test_sparse_calls_are_relative_to_the_sum(n, K, W, density):
     """Sparse calls add with atomics in any order: an element hit by three or more messages may differ from the
