@@ -734,6 +734,95 @@ def config5_decode_sweep(pk):
 
 
 # ----------------------------------------------------------------------------------------------
+# one small launch of every kernel of the library (for ncu captures; see profiles/)
+# ----------------------------------------------------------------------------------------------
+def profile_kernels():
+    """Runs every kernel form once on a small case (after one warm-up call each): ResNet-50 layer shapes at batch 4-8
+    for the squared-gradient kernels, a flat buffer of 2^24 parameters (state larger than L2) for the compressor, the
+    hybrid compressor, the decoder and the index coder.  Prints one line per case; meant to run under ncu."""
+    import paper_1802_06058_b200 as vgc
+    from paper_1802_06058_b200 import workloads
+    dev = "cuda"
+    conv_cases = [  # name, layers, B, C, H, Cout, k, stride, pad
+        ("1x1 both tiles by TMA, bf16 cross terms (layer-3 expansion)", 2, 8, 256, 14, 1024, 1, 1, 0),
+        ("1x1 roles swapped (layer-1 reduction, Cout 64)", 2, 4, 256, 56, 64, 1, 1, 0),
+        ("3x3 three taps, width % 4 == 0 (layer-1)", 1, 4, 64, 56, 64, 3, 1, 1),
+        ("3x3 three taps, width % 4 == 2 (layer-3)", 2, 8, 256, 14, 256, 3, 1, 1),
+        ("3x3 stride 2 three taps (layer-2 first block)", 1, 4, 128, 56, 128, 3, 2, 1),
+        ("7x7 stride 2 seven taps (first layer)", 1, 4, 3, 224, 64, 7, 2, 3),
+        ("1x1 on 7x7 planes: repacked channel-major (layer-4 expansion)", 2, 8, 512, 7, 2048, 1, 1, 0),
+        ("1x1 stride 2: subsampled planes (layer-3 downsample)", 1, 8, 512, 28, 1024, 1, 2, 0),
+        ("3x3 on 7x7 planes: padded planes + three taps (layer-4)", 1, 8, 512, 7, 512, 3, 1, 1),
+        ("5x5: element-wise gather (not a ResNet shape)", 1, 4, 64, 28, 128, 5, 1, 2),
+    ]
+    for name, nl, B, C, H, Cout, k, st, pd in conv_cases:
+        Ho = (H + 2 * pd - k) // st + 1
+        xs = [torch.randn(B, C, H, H, device=dev).abs_() for _ in range(nl)]
+        ds = [torch.randn(B, Cout, Ho, Ho, device=dev) * 1e-4 for _ in range(nl)]
+        Ss = [torch.empty(Cout * C * k * k, device=dev) for _ in range(nl)]
+        ws = torch.zeros(vgc.vgc_sqgrad_conv_batch_workspace_bytes(nl, B, C, H, H, Cout, k, k, st, st, pd, pd), dtype=torch.uint8, device=dev)
+        for _ in range(2):
+            vgc.vgc_sqgrad_conv_batch(xs, ds, (k, k), (st, st), (pd, pd), 1.0 / (B * B), Ss, ws=ws)
+        torch.cuda.synchronize()
+        print(json.dumps({"case": "sqgrad_conv: " + name, "layers": nl, "B": B, "M": Cout, "N": C * k * k, "K": B * Ho * Ho,
+                          "gflop": nl * 2 * Cout * C * k * k * B * Ho * Ho / 1e9}))
+    # per-example statistic (kExact), dense layers (tensor cores and CUDA cores)
+    B, C, H, Cout = 8, 256, 14, 256
+    x = torch.randn(B, C, H, H, device=dev); d = torch.randn(B, Cout, H, H, device=dev) * 1e-4
+    S = torch.empty(Cout * C * 9, device=dev)
+    ws = torch.zeros(vgc.vgc_sqgrad_conv_exact_workspace_bytes(B, C, H, H, Cout, 3, 3, 1, 1, 1, 1), dtype=torch.uint8, device=dev)
+    for _ in range(2):
+        vgc.vgc_sqgrad_conv_exact(x, d, (3, 3), (1, 1), (1, 1), 1.0, S, ws=ws)
+    print(json.dumps({"case": "sqgrad_conv_exact: 3x3 layer-3 shape, per-example statistic", "B": B}))
+    for B, n_in, n_out, what in ((32, 2048, 1000, "tensor cores (fc of ResNet-50)"), (8, 1000, 333, "CUDA cores (batch < 32)")):
+        x = torch.randn(B, n_in, device=dev); d = torch.randn(B, n_out, device=dev)
+        S = torch.empty(n_out * n_in, device=dev)
+        ws = torch.zeros(vgc.vgc_sqgrad_linear_workspace_bytes(B, n_in, n_out), dtype=torch.uint8, device=dev)
+        for _ in range(2):
+            vgc.vgc_sqgrad_linear(x, d, 1.0, S, ws=ws)
+        print(json.dumps({"case": "sqgrad_linear: " + what, "B": B, "in": n_in, "out": n_out}))
+    # flat buffer: compress, hybrid compress, decode (dense and sparse), index coder
+    n, K = 1 << 24, 16
+    offs = np.linspace(0, n, K + 1).astype(np.uint32)
+    offs_dev = vgc.offsets_tensor(offs)
+    g, s = workloads.per_parameter_gs(n, 64, 1e-4, 11, dev)
+    r = torch.zeros(n, device=dev); v = torch.zeros(n, device=dev)
+    out = vgc.MessageBuffers(n, K, n)
+    ws = torch.empty(max(vgc.vgc_compress_workspace_bytes(n, K), vgc.vgc_compress_hybrid_workspace_bytes(n)), dtype=torch.uint8, device=dev)
+    for _ in range(2):
+        vgc.vgc_compress(g, s, r, v, offs_dev, 2.0, ZETA, out, ws)
+    torch.cuda.synchronize()
+    c = out.read()
+    print(json.dumps({"case": "compress", "n": n, "n_criterion": c["n_criterion"], "nnz": c["nnz"]}))
+    hout = vgc.HybridMessageBuffers(n, n)
+    r.zero_(); v.zero_()
+    tau = float(s.sqrt().median().item())
+    for _ in range(2):
+        vgc.vgc_compress_hybrid(g, s, r, v, 2.0, ZETA, tau, hout, ws)
+    torch.cuda.synchronize()
+    print(json.dumps({"case": "compress_hybrid", "n": n, "nnz": hout.read()["nnz"]}))
+    u = torch.zeros(n, device=dev); status = torch.zeros(1, dtype=torch.int32, device=dev)
+    for density, W in ((0.1, 4), (1e-3, 4)):
+        msgs = [workloads.random_message(n, offs, density, 50 + w, dev) for w in range(W)]
+        triples = [(m[0], torch.tensor([m[0].numel()], dtype=torch.int32, device=dev), m[1]) for m in msgs]
+        for _ in range(2):
+            vgc.vgc_decode_accumulate(triples, offs_dev, 1.0 / W, u, status)
+            vgc.vgc_decode_sum(triples, offs_dev, 1.0 / W, u, status)
+        torch.cuda.synchronize()
+        print(json.dumps({"case": "decode_accumulate + decode_sum", "n": n, "W": W, "density": density,
+                          "sum_nnz": sum(m[0].numel() for m in msgs)}))
+    packed = torch.empty(vgc.vgc_pack_bound_bytes(out.words.numel()), dtype=torch.uint8, device=dev)
+    pws = torch.empty(vgc.vgc_pack_workspace_bytes(out.words.numel()), dtype=torch.uint8, device=dev)
+    nbytes = torch.zeros(1, dtype=torch.int32, device=dev)
+    back = torch.empty_like(out.words)
+    for _ in range(2):
+        vgc.vgc_pack_indices(out.words, out.counters[0:1], packed, nbytes, status, pws)
+        vgc.vgc_unpack_indices(packed, out.counters[0:1], back, status)
+    torch.cuda.synchronize()
+    print(json.dumps({"case": "pack_indices + unpack_indices", "words": c["nnz"], "packed_bytes": int(nbytes.item())}))
+
+
+# ----------------------------------------------------------------------------------------------
 # CPU oracle timing (cpu_baseline and --impl reference)
 # ----------------------------------------------------------------------------------------------
 def oracle_sample_time(name: str, n_params: int = 1 << 25):
@@ -830,6 +919,8 @@ def main():
     ap.add_argument("--mma-rates", action="store_true",
                     help="print the measured time of one tcgen05.mma instruction per shape (the tensor-pipe ceiling "
                          "the sqgrad kernel is bounded by) instead of the bench line")
+    ap.add_argument("--profile-kernels", action="store_true",
+                    help="run every kernel form once on a small case and exit (what the ncu captures of profiles/ run)")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--streams", type=int, default=4, help="streams the independent sqgrad layers are spread over")
     ap.add_argument("--fused", action="store_true",
@@ -883,6 +974,10 @@ def main():
                                           "tflops_all_sms": round(tf.value, 1)}))
         return
     vgc.load_library()
+    if args.profile_kernels:
+        if rank == 0:
+            profile_kernels()
+        return
     pk = peaks()
     hp = HotPath(args.workload, worker=rank * 16, n_input_sets=2, n_g_sets=max(4, min(args.steps + args.warmup, 16)),
                  n_params=args.n_params, n_streams=1 if args.per_layer else max(args.streams, 1), algorithm=args.algorithm,

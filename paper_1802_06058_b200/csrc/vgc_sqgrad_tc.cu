@@ -1346,9 +1346,10 @@ sqgrad_tc(const __grid_constant__ Batch bt, const Params prm)
 }
 
 // Adds the partial tiles of every tile that more than one block worked on, in the order of the blocks (a fixed
-// order: the result does not depend on scheduling).  One block per 32 x 8 patch of a tile, one output per thread:
-// partials are read along rows (their unit stride), the result is written along whichever of m / n has unit
-// stride.  Tiles that one block covered alone were written by that block; their patches return at once.
+// order: the result does not depend on scheduling).  One thread block per 32 x 32 patch of a tile: a warp takes
+// four columns, a lane one row -- partials are read along rows (their unit stride), four independent sums per
+// thread -- and the result is written along whichever of m / n has unit stride.  Tiles that one block covered
+// alone were written by that block; their patches return at once.
 struct ResultPtrs { float *S[kMaxBatch]; };
 
 __global__ void __launch_bounds__(256)
@@ -1356,8 +1357,8 @@ sqgrad_tc_combine(const float *__restrict__ partial, int units_q, int units_r, i
                   int tiles_x, int tiles_y, int M, int N, float scale, int accumulate, const ResultPtrs results,
                   long long ld_m, long long ld_n)
 {
-    __shared__ float patch[8][33];
-    const int tile = blockIdx.x >> 6, sub = blockIdx.x & 63;
+    __shared__ float patch[32][33];
+    const int tile = blockIdx.x >> 4, sub = blockIdx.x & 15;
     // the blocks that hold the tile's first and last unit: the first units_r blocks own units_q + 1 units each, the
     // others units_q
     const int t_lo = ((int)blockIdx.y * (tiles_x * tiles_y) + tile) * units_per_tile;
@@ -1367,47 +1368,67 @@ sqgrad_tc_combine(const float *__restrict__ partial, int units_q, int units_r, i
     if (b_first == b_last) return;
     float *__restrict__ S = results.S[blockIdx.y];                         // blockIdx.y: layer of the batch
     const int tx = tile % tiles_x, ty = tile / tiles_x;
-    const int r0 = (sub & 3) * 32, j0 = (sub >> 2) * 8;                   // patch origin inside the tile
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;              // lane -> row, warp -> column
+    const int r0 = (sub & 3) * 32, j0 = (sub >> 2) * 32;                  // patch origin inside the tile
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;              // lane -> row, warp -> four columns
     if (ty * kBM + r0 >= M || tx * kBN + j0 >= N) return;
-    const int j = j0 + w;
-    float sum = 0.f;
-    if (tx * kBN + j < N) {
-        // the first block's part of this tile is that block's last segment unless its range starts with the tile;
-        // every later block's part is its first segment
-        const int lo_first = b_first * units_q + min(b_first, units_r);
-        const size_t within = (size_t)j * kBM + r0 + lane;
-        const float *src0 = partial + (size_t)(2 * b_first + (lo_first < t_lo ? 1 : 0)) * (kBM * kBN) + within;
-        sum = __ldcs(src0);
-        const float *src = partial + within;
-        int b = b_first + 1;
-        for (; b + 8 <= b_last + 1; b += 8) {                // eight loads in flight, summed in block order
-            float v[8];
+    // the first block's part of this tile is that block's last segment unless its range starts with the tile;
+    // every later block's part is its first segment
+    const int lo_first = b_first * units_q + min(b_first, units_r);
+    const size_t within = (size_t)(j0 + 4 * w) * kBM + r0 + lane;
+    const float *src0 = partial + (size_t)(2 * b_first + (lo_first < t_lo ? 1 : 0)) * (kBM * kBN) + within;
+    const float *src = partial + within;
+    float sum[4];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) v[u] = __ldcs(src + (size_t)(2 * (b + u)) * (kBM * kBN));
+    for (int c = 0; c < 4; ++c) sum[c] = __ldcs(src0 + c * kBM);
+    int b = b_first + 1;
+    for (; b + 2 <= b_last + 1; b += 2) {                // eight loads in flight, summed in block order
+        float v[2][4];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) sum = __fadd_rn(sum, v[u]);
-        }
-        for (; b <= b_last; ++b) sum = __fadd_rn(sum, __ldcs(src + (size_t)(2 * b) * (kBM * kBN)));
+        for (int u = 0; u < 2; ++u)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) v[u][c] = __ldcs(src + (size_t)(2 * (b + u)) * (kBM * kBN) + c * kBM);
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) sum[c] = __fadd_rn(sum[c], v[u][c]);
     }
-    const float res = __fmul_rn(scale, sum);
+    for (; b <= b_last; ++b)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) sum[c] = __fadd_rn(sum[c], __ldcs(src + (size_t)(2 * b) * (kBM * kBN) + c * kBM));
     if (ld_m == 1) {
-        const int m = ty * kBM + r0 + lane, n = tx * kBN + j;
-        if (m < M && n < N) {
-            float *dst = S + (size_t)m + (size_t)n * ld_n;
-            *dst = accumulate ? __fadd_rn(*dst, res) : res;
+        const int m = ty * kBM + r0 + lane;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int n = tx * kBN + j0 + 4 * w + c;
+            if (m < M && n < N) {
+                float *dst = S + (size_t)m + (size_t)n * ld_n;
+                const float res = __fmul_rn(scale, sum[c]);
+                *dst = accumulate ? __fadd_rn(*dst, res) : res;
+            }
         }
         return;
     }
-    patch[w][lane] = res;                                                  // patch[column][row]
+#pragma unroll
+    for (int c = 0; c < 4; ++c) patch[4 * w + c][lane] = __fmul_rn(scale, sum[c]);      // patch[column][row]
     __syncthreads();
     {
-        const int c = threadIdx.x & 7, r = threadIdx.x >> 3;              // 8 consecutive columns per row
-        const int m = ty * kBM + r0 + r, n = tx * kBN + j0 + c;
-        if (m < M && n < N) {
+        const int c0 = (threadIdx.x & 7) * 4, r = threadIdx.x >> 3;       // four consecutive columns of one row
+        const int m = ty * kBM + r0 + r, n = tx * kBN + j0 + c0;
+        if (m < M) {
             float *dst = S + (size_t)m * ld_m + n;
-            const float out = patch[c][r];
-            *dst = accumulate ? __fadd_rn(*dst, out) : out;
+            if ((ld_m & 3) == 0 && n + 3 < N) {
+                float4 out = make_float4(patch[c0][r], patch[c0 + 1][r], patch[c0 + 2][r], patch[c0 + 3][r]);
+                if (accumulate) {
+                    const float4 old = *reinterpret_cast<const float4 *>(dst);
+                    out.x = __fadd_rn(old.x, out.x); out.y = __fadd_rn(old.y, out.y);
+                    out.z = __fadd_rn(old.z, out.z); out.w = __fadd_rn(old.w, out.w);
+                }
+                *reinterpret_cast<float4 *>(dst) = out;
+            } else {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    if (n + c < N) dst[c] = accumulate ? __fadd_rn(dst[c], patch[c0 + c][r]) : patch[c0 + c][r];
+            }
         }
     }
 }
@@ -1562,7 +1583,7 @@ static vgc_status tc_launch(KernelFn kernel, const Batch &bt, int n_layers, Para
     if (plan.partials) {
         ResultPtrs results = {};
         for (int l = 0; l < n_layers; ++l) results.S[l] = bt.S[l];
-        sqgrad_tc_combine<<<dim3((unsigned)(plan.tiles_x * plan.tiles_y * 64), (unsigned)n_layers), 256, 0, st>>>(
+        sqgrad_tc_combine<<<dim3((unsigned)(plan.tiles_x * plan.tiles_y * 16), (unsigned)n_layers), 256, 0, st>>>(
             prm.partial, prm.units_q, prm.units_r, plan.units_per_tile, plan.tiles_x, plan.tiles_y, M, N, prm.scale,
             prm.accumulate, results, prm.ld_m, prm.ld_n);
         count_launch();
