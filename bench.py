@@ -164,7 +164,7 @@ class HotPath:
     """All device buffers of one worker and the launches of one step."""
 
     def __init__(self, name: str, worker: int, n_input_sets: int, n_g_sets: int, device="cuda",
-                 n_params: int = 1 << 25, n_streams: int = 4, algorithm: str = "basic", batch_layers: bool = True,
+                 n_params: int = 1 << 25, n_streams: int = 5, algorithm: str = "basic", batch_layers: bool = True,
                  exact_conv: bool = False):
         import paper_1802_06058_b200 as vgc
         from paper_1802_06058_b200 import workloads
@@ -922,7 +922,7 @@ def main():
     ap.add_argument("--profile-kernels", action="store_true",
                     help="run every kernel form once on a small case and exit (what the ncu captures of profiles/ run)")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
-    ap.add_argument("--streams", type=int, default=4, help="streams the independent sqgrad layers are spread over")
+    ap.add_argument("--streams", type=int, default=5, help="streams the independent sqgrad layers are spread over")
     ap.add_argument("--fused", action="store_true",
                     help="sqgrad adds its sums straight into v and vgc_compress runs without s (12 B read per parameter)")
     ap.add_argument("--algorithm", default="basic", choices=["basic", "hybrid"],

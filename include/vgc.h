@@ -130,10 +130,10 @@ vgc_status vgc_sqgrad_conv_exact_batch(int n_layers, const float *const *x, cons
                                        vgc_stream_t stream);
 
 /* Planning hint (no counterpart in the paper): how many sqgrad calls the caller keeps in flight side by side on
- * different streams, each with its own workspace (default 1).  A call's kernel runs one thread block per SM it may
- * use; alone it takes every SM, with c calls in flight each takes 1/c of them, so that the calls run next to one
- * another and the start and tail of one is covered by the others.  Process-wide; set it BEFORE asking for workspace
- * sizes, which depend on it. */
+ * different streams, each with its own workspace (default 1).  A call's kernel runs one thread block per SM at a
+ * time.  Alone (1), a call's work is cut evenly over all SMs, one long block each.  With several calls in flight
+ * (> 1), each call is cut into about half a wave of shorter blocks, and the hardware's block scheduler balances the
+ * SMs across the calls.  Process-wide; set it BEFORE asking for workspace sizes, which depend on it. */
 void vgc_sqgrad_plan_hint(int concurrent_launches);
 
 /* Several conv layers of ONE geometry in one call (the residual stages of a deep network repeat the same
