@@ -238,8 +238,11 @@ vgc_status vgc_compress_static(const float *g, const float *s, float *r, float *
  * Order of the additions.  When the messages together hold at least one word per eight elements, u is moved
  * through shared memory and every element receives its additions in message order (w = 0, 1, ...): the result
  * is the fp32 sequence of a sequential sum and does not depend on scheduling, so every worker that decodes the
- * same messages gets the same bits.  Sparser calls add with fp32 atomics, in any order: an element hit by
- * three or more messages may then differ from the sequential sum in the last bit.
+ * same messages gets the same bits.  (vgc_decode_sum with a power-of-two scale and per-tensor exponents close
+ * enough together adds exact integer multiples of one power of two in any order instead: then every partial sum is
+ * an exact fp32 number and the result is the sequential sum's, bit for bit, all the same.)  Sparser calls add with
+ * fp32 atomics, in any order: an element hit by three or more messages may then differ from the sequential sum in
+ * the last bit.
  *
  * Words whose index is >= n are skipped and VGC_DEV_RANGE is set; a word that breaks the ascending order may
  * be skipped as well (never applied to a wrong element), again with VGC_DEV_RANGE.  A view's word count above

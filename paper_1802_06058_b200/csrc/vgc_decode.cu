@@ -75,7 +75,7 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
 {
     extern __shared__ __align__(16) float tile[];                // tile_elems floats
     __shared__ uint32_t sm_offs[kDecOffsSmem];
-    __shared__ uint32_t cur[kMaxViews], end[kMaxViews];
+    __shared__ uint32_t cur[kMaxViews], end[kMaxViews], taken[kMaxViews];
     __shared__ float lut[kMaxViews * 16];
     __shared__ uint32_t total_words;
     // the messages' pointers, copied out of the kernel parameters once: parameters cannot be indexed with a
@@ -169,19 +169,45 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
             for (uint32_t q = tid; q < n_vec; q += kTileThreads) cp_async_16(tile + 4 * q, u + t0 + 4 * (size_t)q);
             if (tid < t_len - 4 * n_vec) tile[4 * n_vec + tid] = u[t0 + 4 * n_vec + tid];
         }
-        // where every message's run leaves the tile: at most t_len of its words can lie inside
-        for (int w = warp; w < W; w += kTileWarps) {
-            const uint32_t *words = sm_words[w];
-            const uint32_t count = sm_count[w];
-            const uint32_t c = cur[w];
-            const uint32_t span = count - c < t_len ? count - c : t_len;
-            const uint32_t e = c + warp_lower_bound(words + c, span, t_hi);
-            if (lane == 0) end[w] = e;
-        }
         int tile_group = -1;                                        // weight tensor of the tile, -1 if it spans several
         if (!kHybrid) {
             tile_group = group_of(offs, K, (uint32_t)t0);
             if (t_hi - 1 >= offs[tile_group + 1]) tile_group = -1;
+        }
+        // Exact form (vgc_decode_sum only).  When the scale is a power of two and the exponents of all messages for the
+        // tile's tensor lie close enough together, every word is an integer multiple of one power of two, 2^base, and
+        // every partial sum of up to W of them stays below 2^24 multiples: all of them are exact fp32 numbers, fp32
+        // addition of them is associative, and the sequential sum the decoder stands for equals the exact sum.  The
+        // tile is then accumulated as int32 multiples of 2^base with shared-memory integer atomics, in any order:
+        // no barrier between messages, no search for the runs' ends -- the warps stream every message's words from
+        // its cursor until the indices leave the tile -- and one conversion at the end.  Same bits, much less waiting.
+        int fast_base = INT32_MIN;                                  // INT32_MIN: not applicable
+        if (kOverwrite && !kHybrid && tile_group >= 0) {
+            const uint32_t sbits = __float_as_uint(scale);
+            const int s_exp = (int)((sbits >> 23) & 0xFFu) - 127;
+            if ((sbits & 0x807FFFFFu) == 0u && s_exp > -127 && s_exp < 128) {      // positive, a power of two, normal
+                int e_max = INT32_MIN, e_min = INT32_MAX;
+                for (int w = 0; w < W; ++w) {
+                    const int e = sm_gexp[w][tile_group];
+                    if (e != VGC_EXP_NONE) { e_max = max(e_max, e); e_min = min(e_min, e); }
+                }
+                const int base = e_min - 7;                         // the smallest value a word can stand for
+                if (e_max >= e_min && e_max - base + (32 - __clz((W - 1) | 1)) <= 23 && base + s_exp >= -126 && e_max + s_exp <= 127)
+                    fast_base = base;
+            }
+        }
+        const bool fast = fast_base != INT32_MIN;
+        if (tid < (uint32_t)W) taken[tid] = 0;
+        if (!fast) {
+        // where every message's run leaves the tile: at most t_len of its words can lie inside
+            for (int w = warp; w < W; w += kTileWarps) {
+                const uint32_t *words = sm_words[w];
+                const uint32_t count = sm_count[w];
+                const uint32_t c = cur[w];
+                const uint32_t span = count - c < t_len ? count - c : t_len;
+                const uint32_t e = c + warp_lower_bound(words + c, span, t_hi);
+                if (lane == 0) end[w] = e;
+            }
         }
         // the 16 values a word's low four bits (sign, d) can stand for, per message, when the tile lies in one tensor
         const bool use_lut = kHybrid || tile_group >= 0;
@@ -191,7 +217,12 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
                 const uint32_t code = (uint32_t)i & 15u;
                 float val;
                 if (kHybrid) val = (code & 8u) ? -tau : tau;
-                else {
+                else if (fast) {
+                    const int e = sm_gexp[w][tile_group];
+                    const int mult = e == VGC_EXP_NONE ? 0 : 1 << (e - (int)(code & 7u) - fast_base);
+                    reinterpret_cast<int *>(lut)[i] = (code & 8u) ? -mult : mult;
+                    continue;
+                } else {
                     const uint32_t ebits = (uint32_t)(sm_gexp[w][tile_group] + 127) << 23;
                     val = __uint_as_float((ebits - ((code & 7u) << 23)) | ((code & 8u) << 28));
                 }
@@ -200,6 +231,60 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
         if (!kOverwrite) cp_async_wait_all();
         __syncthreads();
 
+        if (fast) {
+            // ---- exact form: warps stream the messages' words from their cursors.  Message m is shared by the warps
+            // m, m + W, ... (W <= 16) in turns of 256 words -- or a warp takes the messages warp, warp + 16, ... -- and a
+            // warp stops at its first turn that reaches past the tile (or the message's end); the words it found inside
+            // are added to the message's count, which moves the cursor once all warps are done.
+            const uint32_t tile_addr = (uint32_t)__cvta_generic_to_shared(tile) - 4u * (uint32_t)t0;
+            const uint32_t lut_addr = (uint32_t)__cvta_generic_to_shared(lut);
+            const int sharers = W < kTileWarps ? kTileWarps / W : 1;   // warps per message
+            for (int m = (int)warp % W + (W < kTileWarps ? 0 : 0); m < W; m += kTileWarps) {
+                if (W < kTileWarps && (int)warp >= sharers * W) break;   // warps left over when W does not divide 16
+                const int turn0 = W < kTileWarps ? (int)warp / W : 0;
+                const uint32_t *words = sm_words[m];
+                const uint32_t c = cur[m], cnt = sm_count[m];
+                const uint32_t lut_m = lut_addr + 64u * (uint32_t)m;
+                uint32_t inside = 0;
+                // a turn is kTurn x 32 consecutive words; the next turn's loads are issued before this turn's words are
+                // looked at (they stay inside the message's buffer), so the DRAM latency of one turn hides under the other
+                constexpr int kTurn = 8;
+                uint32_t nxt[kTurn];
+                auto fetch = [&](uint32_t turn, uint32_t (&dst)[kTurn]) {
+                    const uint32_t first = c + turn * (32u * kTurn) + lane;
+#pragma unroll
+                    for (int j = 0; j < kTurn; ++j) dst[j] = first + 32u * j < cnt ? words[first + 32u * j] : 0xFFFFFFFFu;
+                };
+                fetch((uint32_t)turn0, nxt);
+                for (uint32_t turn = (uint32_t)turn0;; turn += (uint32_t)sharers) {
+                    const uint32_t first = c + turn * (32u * kTurn) + lane;
+                    uint32_t wd[kTurn];
+#pragma unroll
+                    for (int j = 0; j < kTurn; ++j) wd[j] = nxt[j];
+                    fetch(turn + (uint32_t)sharers, nxt);
+                    bool past = false;
+#pragma unroll
+                    for (int j = 0; j < kTurn; ++j) {
+                        const uint32_t idx = wd[j] >> 4;
+                        const bool in = first + 32u * j < cnt && idx < t_hi;
+                        if (in) {
+                            if (idx - (uint32_t)t0 < t_len) {          // false only for an index behind the tile (unsorted)
+                                int iv;
+                                asm volatile("ld.shared.s32 %0, [%1];" : "=r"(iv) : "r"(lut_m + ((wd[j] & 15u) << 2)));
+                                asm volatile("red.shared.add.s32 [%0], %1;" ::"r"(tile_addr + 4u * idx), "r"(iv) : "memory");
+                            } else bad = true;
+                        }
+                        const uint32_t ballot = __ballot_sync(0xffffffffu, in);
+                        inside += __popc(ballot);
+                        past = past || ballot != 0xFFFFFFFFu;
+                    }
+                    if (past) break;
+                }
+                if (lane == 0 && inside) atomicAdd(&taken[m], inside);
+            }
+            __syncthreads();
+            if (tid < (uint32_t)W) end[tid] = cur[tid] + taken[tid];
+        } else {
         // messages one after the other, each in batches of kTileBatch words per thread; the loads of the next batch
         // (of this message or of the next one) are in flight while a batch is applied
         constexpr uint32_t kBatchWords = kTilePre * kTileThreads;
@@ -272,10 +357,24 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
             for (int j = 0; j < kTilePre; ++j) held[j] = next[j];
             w = w2; b = b2; nb = nb2;
         }
+        }
         __syncthreads();
+        if (fast) {
+            // multiples of 2^base -> fp32, times the scale: both factors powers of two, every product exact
+            const float unit = __uint_as_float((uint32_t)(fast_base + ((int)((__float_as_uint(scale) >> 23) & 0xFFu) - 127) + 127) << 23);
+            for (uint32_t q = tid; q < n_vec; q += kTileThreads) {
+                const int4 mlt = reinterpret_cast<const int4 *>(tile)[q];
+                *reinterpret_cast<float4 *>(u + t0 + 4 * (size_t)q) =
+                    make_float4(__fmul_rn((float)mlt.x, unit), __fmul_rn((float)mlt.y, unit), __fmul_rn((float)mlt.z, unit),
+                                __fmul_rn((float)mlt.w, unit));
+            }
+            if (tid < t_len - 4 * n_vec)
+                u[t0 + 4 * n_vec + tid] = __fmul_rn((float)reinterpret_cast<const int *>(tile)[4 * n_vec + tid], unit);
+        } else {
         for (uint32_t q = tid; q < n_vec; q += kTileThreads)
             *reinterpret_cast<float4 *>(u + t0 + 4 * (size_t)q) = reinterpret_cast<const float4 *>(tile)[q];
         if (tid < t_len - 4 * n_vec) u[t0 + 4 * n_vec + tid] = tile[4 * n_vec + tid];
+        }
         __syncthreads();
         for (int w = tid; w < W; w += kTileThreads) cur[w] = end[w];
         __syncthreads();

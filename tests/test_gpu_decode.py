@@ -124,8 +124,10 @@ def test_dense_calls_add_in_message_order_bit_for_bit(n, K, W, density):
                                                       (700001, 5, 64, 0.05, (-3, 0), 2.0 ** -6), (400003, 9, 5, 0.3, (-20, -6), 0.5),
                                                       (300000, 3, 4, 0.5, (-125, -120), 1.0), (300000, 3, 4, 0.5, (100, 110), 0.25)])
 def test_decode_sum_over_the_exponent_range_bit_for_bit(n, K, W, density, exps, scale):
-    """vgc_decode_sum against the oracle's sequential sum, bit for bit, with power-of-two scales, many messages per
-    element, exponents close together and far apart, values next to the smallest normal number and large ones."""
+    """vgc_decode_sum with a power-of-two scale and per-tensor exponents that lie close together accumulates integer
+    multiples of one power of two in any order (no barrier between messages, no search for the runs' ends); the sums
+    are exact, so the result is still the oracle's sequential sum, bit for bit.  Wider exponent ranges (fourth case),
+    values next to the smallest normal number and large ones take whichever form applies tile by tile."""
     offs = random_offsets(np.random.default_rng(31), n, K)
     msgs = [workloads.random_message(n, offs, density, seed=700 + w, device="cuda", exp_lo=exps[0], exp_hi=exps[1])
             for w in range(W)]
