@@ -76,6 +76,7 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
     extern __shared__ __align__(16) float tile[];                // tile_elems floats
     __shared__ uint32_t sm_offs[kDecOffsSmem];
     __shared__ uint32_t cur[kMaxViews], end[kMaxViews], taken[kMaxViews];
+    __shared__ int32_t sm_ex[kMaxViews];                         // the messages' exponents for the current tile's tensor
     __shared__ float lut[kMaxViews * 16];
     __shared__ uint32_t total_words;
     // the messages' pointers, copied out of the kernel parameters once: parameters cannot be indexed with a
@@ -158,8 +159,17 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
     }
 
     // ---- dense: tile by tile
-    for (size_t t0 = lo; t0 < hi; t0 += tile_elems) {
-        const uint32_t t_len = (uint32_t)(hi - t0 < tile_elems ? hi - t0 : tile_elems);
+    int cached_group = -1;
+    uint32_t t_len = 0;
+    for (size_t t0 = lo; t0 < hi; t0 += t_len) {
+        t_len = (uint32_t)(hi - t0 < tile_elems ? hi - t0 : tile_elems);
+        if (!kHybrid) {
+            // a tile ends where its weight tensor ends (when that keeps the next tile on a 16-byte boundary): a tile
+            // inside one tensor has one exponent per message -- the table look-up and the exact form below apply
+            const uint32_t next = offs[group_of(offs, K, (uint32_t)t0) + 1];
+            // (not for a run of tiny tensors: a tile has a fixed cost of a few microseconds)
+            if (next >= (uint32_t)t0 + 2048u && next - (uint32_t)t0 < t_len && (next & 3u) == 0u) t_len = next - (uint32_t)t0;
+        }
         const uint32_t t_hi = (uint32_t)(t0 + t_len);
         const uint32_t n_vec = t_len / 4;                           // t0 is a multiple of 4 elements
         if (kOverwrite) {
@@ -173,6 +183,11 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
         if (!kHybrid) {
             tile_group = group_of(offs, K, (uint32_t)t0);
             if (t_hi - 1 >= offs[tile_group + 1]) tile_group = -1;
+        }
+        if (tile_group >= 0 && tile_group != cached_group) {       // block-uniform; the previous tile ended with a barrier
+            if (tid < (uint32_t)W) sm_ex[tid] = sm_gexp[tid][tile_group];
+            __syncthreads();
+            cached_group = tile_group;
         }
         // Exact form (vgc_decode_sum only).  When the scale is a power of two and the exponents of all messages for the
         // tile's tensor lie close enough together, every word is an integer multiple of one power of two, 2^base, and
@@ -188,7 +203,7 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
             if ((sbits & 0x807FFFFFu) == 0u && s_exp > -127 && s_exp < 128) {      // positive, a power of two, normal
                 int e_max = INT32_MIN, e_min = INT32_MAX;
                 for (int w = 0; w < W; ++w) {
-                    const int e = sm_gexp[w][tile_group];
+                    const int e = sm_ex[w];
                     if (e != VGC_EXP_NONE) { e_max = max(e_max, e); e_min = min(e_min, e); }
                 }
                 const int base = e_min - 7;                         // the smallest value a word can stand for
@@ -218,12 +233,12 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
                 float val;
                 if (kHybrid) val = (code & 8u) ? -tau : tau;
                 else if (fast) {
-                    const int e = sm_gexp[w][tile_group];
+                    const int e = sm_ex[w];
                     const int mult = e == VGC_EXP_NONE ? 0 : 1 << (e - (int)(code & 7u) - fast_base);
                     reinterpret_cast<int *>(lut)[i] = (code & 8u) ? -mult : mult;
                     continue;
                 } else {
-                    const uint32_t ebits = (uint32_t)(sm_gexp[w][tile_group] + 127) << 23;
+                    const uint32_t ebits = (uint32_t)(sm_ex[w] + 127) << 23;
                     val = __uint_as_float((ebits - ((code & 7u) << 23)) | ((code & 8u) << 28));
                 }
                 lut[i] = __fmul_rn(scale, val);
@@ -248,12 +263,16 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
                 uint32_t inside = 0;
                 // a turn is kTurn x 32 consecutive words; the next turn's loads are issued before this turn's words are
                 // looked at (they stay inside the message's buffer), so the DRAM latency of one turn hides under the other
-                constexpr int kTurn = 8;
+                constexpr int kTurn = 8, kAhead = 4;
                 uint32_t nxt[kTurn];
                 auto fetch = [&](uint32_t turn, uint32_t (&dst)[kTurn]) {
                     const uint32_t first = c + turn * (32u * kTurn) + lane;
 #pragma unroll
                     for (int j = 0; j < kTurn; ++j) dst[j] = first + 32u * j < cnt ? words[first + 32u * j] : 0xFFFFFFFFu;
+                    // ... and the turns after it are asked into L2 (no registers held): a turn's loads then find their lines there
+                    const uint32_t ahead = first + (uint32_t)(kAhead * sharers) * (32u * kTurn);
+                    if (lane < kTurn && ahead - lane + 32u * lane < cnt)
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(words + (ahead - lane + 32u * lane)));
                 };
                 fetch((uint32_t)turn0, nxt);
                 for (uint32_t turn = (uint32_t)turn0;; turn += (uint32_t)sharers) {
