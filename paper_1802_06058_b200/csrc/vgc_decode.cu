@@ -161,59 +161,72 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
     // ---- dense: tile by tile
     int cached_group = -1;
     uint32_t t_len = 0;
+    // the exact form (below) needs a scale that is a positive, normal power of two, and reads the messages 16 bytes at a time
+    const int s_exp = (int)((__float_as_uint(scale) >> 23) & 0xFFu) - 127;
+    bool exact_possible = kOverwrite && !kHybrid && (__float_as_uint(scale) & 0x807FFFFFu) == 0u && s_exp > -127 && s_exp < 128;
+    if (exact_possible)
+        for (int w = 0; w < W; ++w) exact_possible = exact_possible && (reinterpret_cast<uintptr_t>(sm_words[w]) & 15u) == 0u;
+    if (kOverwrite) {
+        // the whole tile buffer starts as zeros; from then on whoever writes a tile out leaves zeros behind
+        for (uint32_t q = tid; q < kTileMax / 4; q += kTileThreads)
+            reinterpret_cast<float4 *>(tile)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     for (size_t t0 = lo; t0 < hi; t0 += t_len) {
-        t_len = (uint32_t)(hi - t0 < tile_elems ? hi - t0 : tile_elems);
+        const uint32_t left = (uint32_t)(hi - t0);
+        t_len = left < tile_elems ? left : tile_elems;
+        int tile_group = -1;                                        // weight tensor of the tile, -1 if it spans several
         if (!kHybrid) {
-            // a tile ends where its weight tensor ends (when that keeps the next tile on a 16-byte boundary): a tile
-            // inside one tensor has one exponent per message -- the table look-up and the exact form below apply
-            const uint32_t next = offs[group_of(offs, K, (uint32_t)t0) + 1];
-            // (not for a run of tiny tensors: a tile has a fixed cost of a few microseconds)
-            if (next >= (uint32_t)t0 + 2048u && next - (uint32_t)t0 < t_len && (next & 3u) == 0u) t_len = next - (uint32_t)t0;
+            // A tile ends where its weight tensor ends (when that keeps the next tile on a 16-byte boundary): a tile
+            // inside one tensor has one exponent per message -- the table look-up and the exact form below apply.
+            // The buffer holds kTileMax elements, so a tile may grow a little to reach that end; a tensor that needs
+            // two more tiles gets two of the same size rather than a sliver at its end.
+            const int g = group_of(offs, K, (uint32_t)t0);
+            const uint32_t next = offs[g + 1], rem = next - (uint32_t)t0;
+            if ((next & 3u) == 0u && rem <= left) {
+                // (not for a run of tiny tensors: a tile has a fixed cost of a few microseconds)
+                // (a sliver is cut off only where the exact form can make it cheap)
+                const bool worth = rem >= 2048u || (exact_possible && g + 2 <= K && offs[g + 2] - next >= 8192u);
+                if (rem <= (uint32_t)kTileMax) { if (worth) t_len = rem; }
+                else if (rem < t_len + 2048u || rem <= 2u * (uint32_t)kTileMax) {
+                    const uint32_t half = (rem / 2u + 3u) & ~3u;
+                    if (half <= (uint32_t)kTileMax) t_len = half;
+                }
+            }
+            if ((uint32_t)t0 + t_len - 1u < next) tile_group = g;
         }
         const uint32_t t_hi = (uint32_t)(t0 + t_len);
         const uint32_t n_vec = t_len / 4;                           // t0 is a multiple of 4 elements
-        if (kOverwrite) {
-            for (uint32_t q = tid; q < (t_len + 3) / 4; q += kTileThreads)
-                reinterpret_cast<float4 *>(tile)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-        } else {
+        if (!kOverwrite) {
             for (uint32_t q = tid; q < n_vec; q += kTileThreads) cp_async_16(tile + 4 * q, u + t0 + 4 * (size_t)q);
             if (tid < t_len - 4 * n_vec) tile[4 * n_vec + tid] = u[t0 + 4 * n_vec + tid];
         }
-        int tile_group = -1;                                        // weight tensor of the tile, -1 if it spans several
-        if (!kHybrid) {
-            tile_group = group_of(offs, K, (uint32_t)t0);
-            if (t_hi - 1 >= offs[tile_group + 1]) tile_group = -1;
-        }
-        if (tile_group >= 0 && tile_group != cached_group) {       // block-uniform; the previous tile ended with a barrier
+        if (tile_group >= 0 && tile_group != cached_group) {       // block-uniform; nobody reads sm_ex between the tiles
             if (tid < (uint32_t)W) sm_ex[tid] = sm_gexp[tid][tile_group];
             __syncthreads();
             cached_group = tile_group;
         }
         // Exact form (vgc_decode_sum only).  When the scale is a power of two and the exponents of all messages for the
         // tile's tensor lie close enough together, every word is an integer multiple of one power of two, 2^base, and
-        // every partial sum of up to W of them stays below 2^24 multiples: all of them are exact fp32 numbers, fp32
+        // every partial sum of up to W of them stays within 2^22 multiples: all of them are exact fp32 numbers, fp32
         // addition of them is associative, and the sequential sum the decoder stands for equals the exact sum.  The
         // tile is then accumulated as int32 multiples of 2^base with shared-memory integer atomics, in any order:
         // no barrier between messages, no search for the runs' ends -- the warps stream every message's words from
         // its cursor until the indices leave the tile -- and one conversion at the end.  Same bits, much less waiting.
         int fast_base = INT32_MIN;                                  // INT32_MIN: not applicable
-        if (kOverwrite && !kHybrid && tile_group >= 0) {
-            const uint32_t sbits = __float_as_uint(scale);
-            const int s_exp = (int)((sbits >> 23) & 0xFFu) - 127;
-            if ((sbits & 0x807FFFFFu) == 0u && s_exp > -127 && s_exp < 128) {      // positive, a power of two, normal
-                int e_max = INT32_MIN, e_min = INT32_MAX;
-                for (int w = 0; w < W; ++w) {
-                    const int e = sm_ex[w];
-                    if (e != VGC_EXP_NONE) { e_max = max(e_max, e); e_min = min(e_min, e); }
-                }
-                const int base = e_min - 7;                         // the smallest value a word can stand for
-                if (e_max >= e_min && e_max - base + (32 - __clz((W - 1) | 1)) <= 23 && base + s_exp >= -126 && e_max + s_exp <= 127)
-                    fast_base = base;
+        if (exact_possible && tile_group >= 0 && t_hi < (1u << 28)) {
+            int e_max = INT32_MIN, e_min = INT32_MAX;
+            for (int w = 0; w < W; ++w) {
+                const int e = sm_ex[w];
+                if (e != VGC_EXP_NONE) { e_max = max(e_max, e); e_min = min(e_min, e); }
             }
+            const int base = e_min - 7;                             // the smallest value a word can stand for
+            if (e_max >= e_min && e_max - base + (32 - __clz((W - 1) | 1)) <= 22 && base + s_exp >= -126 && e_max + s_exp <= 127)
+                fast_base = base;
         }
         const bool fast = fast_base != INT32_MIN;
         if (tid < (uint32_t)W) taken[tid] = 0;
         if (!fast) {
+            if (kOverwrite) __syncthreads();                        // the cursors of the tile before
         // where every message's run leaves the tile: at most t_len of its words can lie inside
             for (int w = warp; w < W; w += kTileWarps) {
                 const uint32_t *words = sm_words[w];
@@ -251,58 +264,84 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
             // m, m + W, ... (W <= 16) in turns of 256 words -- or a warp takes the messages warp, warp + 16, ... -- and a
             // warp stops at its first turn that reaches past the tile (or the message's end); the words it found inside
             // are added to the message's count, which moves the cursor once all warps are done.
-            const uint32_t tile_addr = (uint32_t)__cvta_generic_to_shared(tile) - 4u * (uint32_t)t0;
+            const uint32_t tile_addr = (uint32_t)__cvta_generic_to_shared(tile);
             const uint32_t lut_addr = (uint32_t)__cvta_generic_to_shared(lut);
+            // a word minus t0 << 4 keeps its low four bits and turns its index into the offset inside the tile; one
+            // unsigned comparison then says "inside the tile" (a word behind the tile wraps around to a huge number,
+            // and so does the filler 0xFFFFFFFF, because t_hi < 2^28)
+            const uint32_t t0s = (uint32_t)t0 << 4, t_len16 = t_len << 4;
             const int sharers = W < kTileWarps ? kTileWarps / W : 1;   // warps per message
-            for (int m = (int)warp % W + (W < kTileWarps ? 0 : 0); m < W; m += kTileWarps) {
+            for (int m = (int)warp % W; m < W; m += kTileWarps) {
                 if (W < kTileWarps && (int)warp >= sharers * W) break;   // warps left over when W does not divide 16
-                const int turn0 = W < kTileWarps ? (int)warp / W : 0;
+                const uint32_t turn0 = W < kTileWarps ? warp / (uint32_t)W : 0u;
                 const uint32_t *words = sm_words[m];
                 const uint32_t c = cur[m], cnt = sm_count[m];
+                const uint32_t a = c & ~3u;                          // 16-byte loads: start at the boundary before the cursor
                 const uint32_t lut_m = lut_addr + 64u * (uint32_t)m;
-                uint32_t inside = 0;
-                // a turn is kTurn x 32 consecutive words; the next turn's loads are issued before this turn's words are
-                // looked at (they stay inside the message's buffer), so the DRAM latency of one turn hides under the other
-                constexpr int kTurn = 8, kAhead = 4;
-                uint32_t nxt[kTurn];
-                auto fetch = [&](uint32_t turn, uint32_t (&dst)[kTurn]) {
-                    const uint32_t first = c + turn * (32u * kTurn) + lane;
+                uint32_t inside = 0, n_in = 0;                       // words up to the tile's end; words added
+                // a turn is 256 consecutive words, two 16-byte loads per lane; the next turn's loads are issued before
+                // this turn's words are looked at, so the latency of one turn hides under the work of the other
+                constexpr int kVecs = 2, kAhead = 4;
+                constexpr uint32_t kTurnWords = 128u * kVecs;
+                uint4 nxt[kVecs];
+                auto fetch = [&](uint32_t turn, uint4 (&dst)[kVecs]) {
+                    const uint32_t p0 = a + turn * kTurnWords + 4u * lane;
 #pragma unroll
-                    for (int j = 0; j < kTurn; ++j) dst[j] = first + 32u * j < cnt ? words[first + 32u * j] : 0xFFFFFFFFu;
-                    // ... and the turns after it are asked into L2 (no registers held): a turn's loads then find their lines there
-                    const uint32_t ahead = first + (uint32_t)(kAhead * sharers) * (32u * kTurn);
-                    if (lane < kTurn && ahead - lane + 32u * lane < cnt)
-                        asm volatile("prefetch.global.L2 [%0];" ::"l"(words + (ahead - lane + 32u * lane)));
-                };
-                fetch((uint32_t)turn0, nxt);
-                for (uint32_t turn = (uint32_t)turn0;; turn += (uint32_t)sharers) {
-                    const uint32_t first = c + turn * (32u * kTurn) + lane;
-                    uint32_t wd[kTurn];
-#pragma unroll
-                    for (int j = 0; j < kTurn; ++j) wd[j] = nxt[j];
-                    fetch(turn + (uint32_t)sharers, nxt);
-                    bool past = false;
-#pragma unroll
-                    for (int j = 0; j < kTurn; ++j) {
-                        const uint32_t idx = wd[j] >> 4;
-                        const bool in = first + 32u * j < cnt && idx < t_hi;
-                        if (in) {
-                            if (idx - (uint32_t)t0 < t_len) {          // false only for an index behind the tile (unsorted)
-                                int iv;
-                                asm volatile("ld.shared.s32 %0, [%1];" : "=r"(iv) : "r"(lut_m + ((wd[j] & 15u) << 2)));
-                                asm volatile("red.shared.add.s32 [%0], %1;" ::"r"(tile_addr + 4u * idx), "r"(iv) : "memory");
-                            } else bad = true;
+                    for (int v = 0; v < kVecs; ++v) {
+                        const uint32_t p = p0 + 128u * v;
+                        if (p + 4u <= cnt) dst[v] = *reinterpret_cast<const uint4 *>(words + p);
+                        else {
+                            dst[v].x = p < cnt ? words[p] : 0xFFFFFFFFu;
+                            dst[v].y = p + 1u < cnt ? words[p + 1] : 0xFFFFFFFFu;
+                            dst[v].z = p + 2u < cnt ? words[p + 2] : 0xFFFFFFFFu;
+                            dst[v].w = 0xFFFFFFFFu;
                         }
-                        const uint32_t ballot = __ballot_sync(0xffffffffu, in);
-                        inside += __popc(ballot);
-                        past = past || ballot != 0xFFFFFFFFu;
                     }
-                    if (past) break;
+                    // ... and the turns after it are asked into L2 (no registers held): a turn's loads then find their lines there
+                    const uint32_t ahead = a + (turn + (uint32_t)(kAhead * sharers)) * kTurnWords + 32u * lane;
+                    if (lane < kTurnWords / 32u && ahead < cnt) asm volatile("prefetch.global.L2 [%0];" ::"l"(words + ahead));
+                };
+                auto add = [&](uint32_t word) {
+                    const uint32_t off16 = word - t0s;
+                    if (off16 < t_len16) {
+                        int iv;
+                        asm volatile("ld.shared.s32 %0, [%1];" : "=r"(iv) : "r"(lut_m + ((word & 15u) << 2)));
+                        asm volatile("red.shared.add.s32 [%0], %1;" ::"r"(tile_addr + ((off16 >> 2) & 0xFFFFFFFCu)), "r"(iv) : "memory");
+                        ++n_in;
+                    }
+                };
+                fetch(turn0, nxt);
+                for (uint32_t turn = turn0;; turn += (uint32_t)sharers) {
+                    uint4 wd[kVecs];
+#pragma unroll
+                    for (int v = 0; v < kVecs; ++v) wd[v] = nxt[v];
+                    fetch(turn + (uint32_t)sharers, nxt);
+#pragma unroll
+                    for (int v = 0; v < kVecs; ++v) { add(wd[v].x); add(wd[v].y); add(wd[v].z); add(wd[v].w); }
+                    // sorted words: the turn lies inside the tile when its last word does (and the message goes on)
+                    const uint32_t turn_end = a + (turn + 1u) * kTurnWords;
+                    const bool last_in = wd[kVecs - 1].w - t0s < t_len16;
+                    if (turn_end <= cnt && (__ballot_sync(0xffffffffu, last_in) >> 31)) {
+                        inside += kTurnWords - (turn == 0u ? c - a : 0u);
+                        continue;
+                    }
+                    // the last turn of this warp: count the words from the cursor on that lie before the tile's end
+                    uint32_t mine = 0;
+                    const uint32_t p0 = a + turn * kTurnWords + 4u * lane;
+#pragma unroll
+                    for (int v = 0; v < kVecs; ++v) {
+                        const uint32_t p = p0 + 128u * v;
+                        const uint32_t x[4] = {wd[v].x, wd[v].y, wd[v].z, wd[v].w};
+#pragma unroll
+                        for (uint32_t i = 0; i < 4; ++i) mine += (p + i >= c && p + i < cnt && (x[i] >> 4) < t_hi) ? 1u : 0u;
+                    }
+                    inside += __reduce_add_sync(0xffffffffu, mine);
+                    break;
                 }
+                // a word before the tile's end that was not added lies behind the tile: the message is not sorted
+                if (__reduce_add_sync(0xffffffffu, n_in) != inside) bad = true;
                 if (lane == 0 && inside) atomicAdd(&taken[m], inside);
             }
-            __syncthreads();
-            if (tid < (uint32_t)W) end[tid] = cur[tid] + taken[tid];
         } else {
         // messages one after the other, each in batches of kTileBatch words per thread; the loads of the next batch
         // (of this message or of the next one) are in flight while a batch is applied
@@ -378,25 +417,34 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
         }
         }
         __syncthreads();
+        if (tid < (uint32_t)W) cur[tid] = fast ? cur[tid] + taken[tid] : end[tid];
         if (fast) {
-            // multiples of 2^base -> fp32, times the scale: both factors powers of two, every product exact
-            const float unit = __uint_as_float((uint32_t)(fast_base + ((int)((__float_as_uint(scale) >> 23) & 0xFFu) - 127) + 127) << 23);
+            // multiples of 2^base -> fp32, times the scale: both factors powers of two, every product exact.  A sum is
+            // at most 2^22 multiples either way, so 1.5 * 2^23 plus it is a float whose bits are 0x4B400000 plus it.
+            const float unit = __uint_as_float((uint32_t)(fast_base + s_exp + 127) << 23);
+            auto value = [&](int mult) { return __fmul_rn(__fsub_rn(__int_as_float(0x4B400000 + mult), 12582912.f), unit); };
             for (uint32_t q = tid; q < n_vec; q += kTileThreads) {
                 const int4 mlt = reinterpret_cast<const int4 *>(tile)[q];
-                *reinterpret_cast<float4 *>(u + t0 + 4 * (size_t)q) =
-                    make_float4(__fmul_rn((float)mlt.x, unit), __fmul_rn((float)mlt.y, unit), __fmul_rn((float)mlt.z, unit),
-                                __fmul_rn((float)mlt.w, unit));
+                reinterpret_cast<int4 *>(tile)[q] = make_int4(0, 0, 0, 0);
+                *reinterpret_cast<float4 *>(u + t0 + 4 * (size_t)q) = make_float4(value(mlt.x), value(mlt.y), value(mlt.z), value(mlt.w));
             }
-            if (tid < t_len - 4 * n_vec)
-                u[t0 + 4 * n_vec + tid] = __fmul_rn((float)reinterpret_cast<const int *>(tile)[4 * n_vec + tid], unit);
+            if (tid < t_len - 4 * n_vec) {
+                u[t0 + 4 * n_vec + tid] = value(reinterpret_cast<const int *>(tile)[4 * n_vec + tid]);
+                tile[4 * n_vec + tid] = 0.f;
+            }
         } else {
-        for (uint32_t q = tid; q < n_vec; q += kTileThreads)
-            *reinterpret_cast<float4 *>(u + t0 + 4 * (size_t)q) = reinterpret_cast<const float4 *>(tile)[q];
-        if (tid < t_len - 4 * n_vec) u[t0 + 4 * n_vec + tid] = tile[4 * n_vec + tid];
+            for (uint32_t q = tid; q < n_vec; q += kTileThreads) {
+                *reinterpret_cast<float4 *>(u + t0 + 4 * (size_t)q) = reinterpret_cast<const float4 *>(tile)[q];
+                if (kOverwrite) reinterpret_cast<float4 *>(tile)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            if (tid < t_len - 4 * n_vec) {
+                u[t0 + 4 * n_vec + tid] = tile[4 * n_vec + tid];
+                if (kOverwrite) tile[4 * n_vec + tid] = 0.f;
+            }
         }
-        __syncthreads();
-        for (int w = tid; w < W; w += kTileThreads) cur[w] = end[w];
-        __syncthreads();
+        // vgc_decode_sum: every thread put zeros back where it read, and the next tile's barrier orders them before
+        // the next additions.  vgc_decode_accumulate loads the next tile over this one: wait for the readers.
+        if (!kOverwrite) __syncthreads();
     }
     if (bad) atomicOr(dev_status, VGC_DEV_RANGE);
 }
@@ -450,7 +498,7 @@ vgc_status decode_launch(bool hybrid, bool overwrite, const vgc_message_view *ms
             VGC_CUDA_OK(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileMax * 4));
             if (n_configured < 4) configured[n_configured++] = fn;
         }
-        fn<<<blocks, kTileThreads, (size_t)tile_elems * 4, st>>>(views, wb, group_offsets, K, scale, tau, u, n, (uint32_t)chunk,
+        fn<<<blocks, kTileThreads, (size_t)kTileMax * 4, st>>>(views, wb, group_offsets, K, scale, tau, u, n, (uint32_t)chunk,
                                                                  tile_elems, dev_status);
         count_launch();
     }

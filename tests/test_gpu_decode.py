@@ -141,6 +141,30 @@ def test_decode_sum_over_the_exponent_range_bit_for_bit(n, K, W, density, exps, 
     assert int(st.item()) == 0 and np.array_equal(gu.t.cpu().numpy().view(np.uint32), ref.view(np.uint32))
 
 
+@pytest.mark.parametrize("shift", [0, 1, 2, 3])
+def test_decode_sum_reads_messages_at_any_word_alignment(shift):
+    """The exact form reads the messages 16 bytes at a time from the boundary before each cursor; a message that does
+    not start on a 16-byte boundary takes the ordered form.  Same bits either way, and nothing before a message's
+    first word or after its last one changes the result: each message sits between two words that point at element 0."""
+    n, K, W = 600001, 7, 6
+    offs = random_offsets(np.random.default_rng(77), n, K)
+    msgs = [workloads.random_message(n, offs, 0.2, seed=1200 + w, device="cuda", exp_lo=-9, exp_hi=-7) for w in range(W)]
+    triples = []
+    for w, (words, exps) in enumerate(msgs):
+        m = words.numel() - (w % 4)                                 # counts that are not multiples of four
+        buf = torch.full((m + shift + 8,), 0x0000000F, dtype=words.dtype, device="cuda")      # element 0, largest code
+        buf[shift:shift + m] = words[:m]
+        msgs[w] = (words[:m], exps)
+        triples.append((buf[shift:shift + m], torch.tensor([m], dtype=torch.int32, device="cuda"), exps))
+    gu = Guarded(n, fill=float("nan"))
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    vgc.vgc_decode_sum(triples, vgc.offsets_tensor(offs), 0.25, gu.t, st)
+    gu.check("u")
+    ref = np.zeros(n, F32)
+    oracle.decode_accumulate([(w.cpu().numpy().view(np.uint32), e.cpu().numpy()) for w, e in msgs], offs, 0.25, ref)
+    assert int(st.item()) == 0 and np.array_equal(gu.t.cpu().numpy().view(np.uint32), ref.view(np.uint32))
+
+
 @pytest.mark.parametrize("n,K,W,density", [(400003, 9, 5, 0.002), (2500000, 40, 17, 0.0005)])
 def test_sparse_calls_are_relative_to_the_sum(n, K, W, density):
     """Sparse calls add with atomics in any order: an element hit by three or more messages may differ from the
@@ -191,7 +215,8 @@ def test_truncated_message_is_decoded_up_to_its_buffer():
 
 
 @pytest.mark.parametrize("density", [0.3, 0.001])
-def test_unsorted_words_never_touch_a_wrong_element(density):
+@pytest.mark.parametrize("entry", ["vgc_decode_accumulate", "vgc_decode_sum"])
+def test_unsorted_words_never_touch_a_wrong_element(density, entry):
     """Messages must be sorted; one that is not may lose words (VGC_DEV_RANGE says so), but no word is ever added to
     an element other than its own and nothing outside u is written."""
     n, W = 200003, 3
@@ -204,7 +229,7 @@ def test_unsorted_words_never_touch_a_wrong_element(density):
     gu = Guarded(n, fill=0.0)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     triples = [(w, torch.tensor([w.numel()], dtype=torch.int32, device="cuda"), e) for w, e in msgs]
-    vgc.vgc_decode_accumulate(triples, vgc.offsets_tensor(offs), 1.0, gu.t, status)
+    getattr(vgc, entry)(triples, vgc.offsets_tensor(offs), 1.0, gu.t, status)        # u starts as zeros: same result
     gu.check("u")
     ref = np.zeros(n, F32)
     oracle.decode_accumulate([(w.cpu().numpy().view(np.uint32), e.cpu().numpy()) for w, e in msgs], offs, 1.0, ref)
