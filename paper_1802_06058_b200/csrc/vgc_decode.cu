@@ -52,9 +52,11 @@ __device__ __forceinline__ uint32_t warp_lower_bound(const uint32_t *__restrict_
     return lo;
 }
 
-constexpr int kTileThreads = 512;
+// three blocks of eight warps per SM: while one block waits at a barrier or for its first words, the others add
+constexpr int kTileThreads = 256;
+constexpr int kBlocksPerSm = 3;
 constexpr int kTileWarps = kTileThreads / 32;
-constexpr int kTileMax = 24576;                  // elements per tile
+constexpr int kTileMax = 16384;                  // elements per tile
 constexpr int kTilePre = 8;                      // words per thread in one batch
 
 __device__ __forceinline__ void cp_async_16(void *smem, const void *gmem)
@@ -68,7 +70,7 @@ __device__ __forceinline__ void cp_async_wait_all()
 }
 
 template <bool kHybrid, bool kOverwrite>
-__global__ void __launch_bounds__(kTileThreads, 2)
+__global__ void __launch_bounds__(kTileThreads, kBlocksPerSm)
 decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *__restrict__ group_offsets, int K,
              float scale, float tau, float *__restrict__ u, size_t n, uint32_t chunk_elems, uint32_t tile_elems,
              uint32_t *dev_status)
@@ -261,7 +263,7 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
 
         if (fast) {
             // ---- exact form: warps stream the messages' words from their cursors.  Message m is shared by the warps
-            // m, m + W, ... (W <= 16) in turns of 256 words -- or a warp takes the messages warp, warp + 16, ... -- and a
+            // m, m + W, ... (W < 8) in turns of 256 words -- or a warp takes the messages warp, warp + 8, ... -- and a
             // warp stops at its first turn that reaches past the tile (or the message's end); the words it found inside
             // are added to the message's count, which moves the cursor once all warps are done.
             const uint32_t tile_addr = (uint32_t)__cvta_generic_to_shared(tile);
@@ -272,7 +274,7 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
             const uint32_t t0s = (uint32_t)t0 << 4, t_len16 = t_len << 4;
             const int sharers = W < kTileWarps ? kTileWarps / W : 1;   // warps per message
             for (int m = (int)warp % W; m < W; m += kTileWarps) {
-                if (W < kTileWarps && (int)warp >= sharers * W) break;   // warps left over when W does not divide 16
+                if (W < kTileWarps && (int)warp >= sharers * W) break;   // warps left over when W does not divide the warps
                 const uint32_t turn0 = W < kTileWarps ? warp / (uint32_t)W : 0u;
                 const uint32_t *words = sm_words[m];
                 const uint32_t c = cur[m], cnt = sm_count[m];
@@ -286,29 +288,44 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
                 uint4 nxt[kVecs];
                 auto fetch = [&](uint32_t turn, uint4 (&dst)[kVecs]) {
                     const uint32_t p0 = a + turn * kTurnWords + 4u * lane;
+                    if (a + (turn + 1u) * kTurnWords <= cnt) {          // warp-uniform: the whole turn lies inside the message
 #pragma unroll
-                    for (int v = 0; v < kVecs; ++v) {
-                        const uint32_t p = p0 + 128u * v;
-                        if (p + 4u <= cnt) dst[v] = *reinterpret_cast<const uint4 *>(words + p);
-                        else {
+                        for (int v = 0; v < kVecs; ++v) dst[v] = *reinterpret_cast<const uint4 *>(words + p0 + 128u * v);
+                    } else {
+#pragma unroll
+                        for (int v = 0; v < kVecs; ++v) {
+                            const uint32_t p = p0 + 128u * v;
                             dst[v].x = p < cnt ? words[p] : 0xFFFFFFFFu;
                             dst[v].y = p + 1u < cnt ? words[p + 1] : 0xFFFFFFFFu;
                             dst[v].z = p + 2u < cnt ? words[p + 2] : 0xFFFFFFFFu;
-                            dst[v].w = 0xFFFFFFFFu;
+                            dst[v].w = p + 3u < cnt ? words[p + 3] : 0xFFFFFFFFu;
                         }
                     }
                     // ... and the turns after it are asked into L2 (no registers held): a turn's loads then find their lines there
                     const uint32_t ahead = a + (turn + (uint32_t)(kAhead * sharers)) * kTurnWords + 32u * lane;
                     if (lane < kTurnWords / 32u && ahead < cnt) asm volatile("prefetch.global.L2 [%0];" ::"l"(words + ahead));
                 };
+                // one word: inside the tile -> look its multiple up and add it; all of it predicated, no branch
                 auto add = [&](uint32_t word) {
-                    const uint32_t off16 = word - t0s;
-                    if (off16 < t_len16) {
-                        int iv;
-                        asm volatile("ld.shared.s32 %0, [%1];" : "=r"(iv) : "r"(lut_m + ((word & 15u) << 2)));
-                        asm volatile("red.shared.add.s32 [%0], %1;" ::"r"(tile_addr + ((off16 >> 2) & 0xFFFFFFFCu)), "r"(iv) : "memory");
-                        ++n_in;
-                    }
+                    asm volatile("{\n\t"
+                                 ".reg .pred p;\n\t"
+                                 ".reg .s32 iv;\n\t"
+                                 ".reg .u32 o, at, l;\n\t"
+                                 "sub.u32 o, %1, %2;\n\t"
+                                 "setp.lt.u32 p, o, %3;\n\t"
+                                 "and.b32 l, %1, 15;\n\t"
+                                 "shl.b32 l, l, 2;\n\t"
+                                 "add.u32 l, l, %4;\n\t"
+                                 "shr.u32 at, o, 2;\n\t"
+                                 "and.b32 at, at, 0xFFFFFFFC;\n\t"
+                                 "add.u32 at, at, %5;\n\t"
+                                 "@p ld.shared.s32 iv, [l];\n\t"
+                                 "@p red.shared.add.s32 [at], iv;\n\t"
+                                 "@p add.u32 %0, %0, 1;\n\t"
+                                 "}"
+                                 : "+r"(n_in)
+                                 : "r"(word), "r"(t0s), "r"(t_len16), "r"(lut_m), "r"(tile_addr)
+                                 : "memory");
                 };
                 fetch(turn0, nxt);
                 for (uint32_t turn = turn0;; turn += (uint32_t)sharers) {
@@ -481,8 +498,8 @@ vgc_status decode_launch(bool hybrid, bool overwrite, const vgc_message_view *ms
             views.group_exp[w] = m.group_exp;
             views.max_words[w] = m.max_words;
         }
-        // one contiguous range per block, two blocks per SM, three or four tiles per range
-        size_t chunk = (n + (size_t)sm_count * 2 - 1) / ((size_t)sm_count * 2);
+        // one contiguous range per block, kBlocksPerSm blocks per SM, three or four tiles per range
+        size_t chunk = (n + (size_t)sm_count * kBlocksPerSm - 1) / ((size_t)sm_count * kBlocksPerSm);
         chunk = (chunk + 3) / 4 * 4;
         const size_t tiles = (chunk + kTileMax - 1) / kTileMax;
         const uint32_t tile_elems = (uint32_t)(((chunk + tiles - 1) / tiles + 3) / 4 * 4);
