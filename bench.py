@@ -1047,6 +1047,14 @@ def main():
                          "traffic": compress_traffic * n if compress_traffic else None,
                          "traffic_source": traffic.get("source"),
                          "algorithmic_bytes": compress_bytes, "peak_source": f"{pk['source']} copy bandwidth, of measured"}
+    decode_roofline = None
+    if hp.W:
+        decode_roofline = {"kernel": "decode_tiles (vgc_decode_sum)", "bound": "hbm", "achieved": gbs(decode_bytes, de_ms),
+                           "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": gbs(decode_bytes, de_ms) / pk["hbm_gbs"],
+                           "frac_of_8tbs": gbs(decode_bytes, de_ms) / HBM_NOMINAL_GBS,
+                           "traffic": traffic.get("decode_bytes_resnet50_w8") if args.workload == "resnet50" and hp.W == 8 else None,
+                           "traffic_source": traffic.get("source"), "algorithmic_bytes": decode_bytes,
+                           "peak_source": f"{pk['source']} copy bandwidth, of measured"}
     extras = rank == 0 and world == 1 and not args.no_extra
     # dominant kernel of the step
     if sq_ms >= co_ms + de_ms and hp.flops_useful:
@@ -1101,7 +1109,7 @@ def main():
                        "fused_sqgrad_into_v": bool(args.fused),
                        "l2": "inputs larger than L2 (no flush)" if n * 16 > 126e6 else "state fits in L2 (no flush): cache-resident numbers"},
             "gpu_launches": int(launches), "clocks": clocks, "sections": sections, "roofline": roofline,
-            "roofline_compress": compress_roofline}
+            "roofline_compress": compress_roofline, "roofline_decode": decode_roofline}
 
     if not args.no_e2e:
         e2e_ms, h2d, d2h = run_e2e(hp, min(args.steps, 5), 1)

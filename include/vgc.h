@@ -235,14 +235,20 @@ vgc_status vgc_compress_static(const float *g, const float *s, float *r, float *
  *          Words must be in ascending index order, as vgc_compress emits them.
  *   u      [n] fp32, accumulated in place (the caller zeroes it when a fresh sum is wanted)
  *
- * Order of the additions.  When the messages together hold at least one word per eight elements, u is moved
- * through shared memory and every element receives its additions in message order (w = 0, 1, ...): the result
- * is the fp32 sequence of a sequential sum and does not depend on scheduling, so every worker that decodes the
- * same messages gets the same bits.  (vgc_decode_sum with a power-of-two scale and per-tensor exponents close
- * enough together adds exact integer multiples of one power of two in any order instead: then every partial sum is
- * an exact fp32 number and the result is the sequential sum's, bit for bit, all the same.)  Sparser calls add with
- * fp32 atomics, in any order: an element hit by three or more messages may then differ from the sequential sum in
- * the last bit.
+ * Arithmetic.  Every result is a deterministic function of the inputs' bits when the messages together hold at
+ * least one word per eight elements (u then moves through shared memory, tensor by tensor), so every worker that
+ * decodes the same messages gets the same bits.  Two forms, chosen per weight tensor:
+ *   exact    taken when all messages start on 16-byte boundaries and, for the tensor, the messages' exponents lie
+ *            close together (E_max - E_min + 7 + ceil(log2 W) <= 22).  The words of an element are then integer
+ *            multiples of one power of two and are summed exactly; the element becomes scale * sum (vgc_decode_sum)
+ *            or u + scale * sum (vgc_decode_accumulate), each operation rounded once.  With a scale that is a
+ *            power of two nothing is rounded before the final addition, and vgc_decode_sum returns the bits of the
+ *            sum taken message by message in fp32.  Elements no word points at keep their bits (accumulate).
+ *   ordered  otherwise: u[idx] += scale * value, rounded per word, in message order (w = 0, 1, ...) -- the fp32
+ *            sequence of a sequential loop.
+ *   The two differ by at most the roundings of the sequential loop: (W + 2) half-ulps of |u| + sum |scale * value|.
+ * Sparser calls add scale * value with fp32 atomics, in any order: an element hit by three or more messages may
+ * then differ from the sequential sum in the last bit.
  *
  * Words whose index is >= n are skipped and VGC_DEV_RANGE is set; a word that breaks the ascending order may
  * be skipped as well (never applied to a wrong element), again with VGC_DEV_RANGE.  A view's word count above

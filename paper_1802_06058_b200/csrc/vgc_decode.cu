@@ -163,12 +163,14 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
     // ---- dense: tile by tile
     int cached_group = -1;
     uint32_t t_len = 0;
-    // the exact form (below) needs a scale that is a positive, normal power of two, and reads the messages 16 bytes at a time
+    // the exact form (below) reads the messages 16 bytes at a time; with a scale that is a positive, normal power of two
+    // its result is the sequential sum's, bit for bit
     const int s_exp = (int)((__float_as_uint(scale) >> 23) & 0xFFu) - 127;
-    bool exact_possible = kOverwrite && !kHybrid && (__float_as_uint(scale) & 0x807FFFFFu) == 0u && s_exp > -127 && s_exp < 128;
+    const bool pow2 = (__float_as_uint(scale) & 0x807FFFFFu) == 0u && s_exp > -127 && s_exp < 128;
+    bool exact_possible = !kHybrid && s_exp < 128;              // a finite scale
     if (exact_possible)
         for (int w = 0; w < W; ++w) exact_possible = exact_possible && (reinterpret_cast<uintptr_t>(sm_words[w]) & 15u) == 0u;
-    if (kOverwrite) {
+    if (kOverwrite || exact_possible) {
         // the whole tile buffer starts as zeros; from then on whoever writes a tile out leaves zeros behind
         for (uint32_t q = tid; q < kTileMax / 4; q += kTileThreads)
             reinterpret_cast<float4 *>(tile)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -198,19 +200,17 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
         }
         const uint32_t t_hi = (uint32_t)(t0 + t_len);
         const uint32_t n_vec = t_len / 4;                           // t0 is a multiple of 4 elements
-        if (!kOverwrite) {
-            for (uint32_t q = tid; q < n_vec; q += kTileThreads) cp_async_16(tile + 4 * q, u + t0 + 4 * (size_t)q);
-            if (tid < t_len - 4 * n_vec) tile[4 * n_vec + tid] = u[t0 + 4 * n_vec + tid];
-        }
         if (tile_group >= 0 && tile_group != cached_group) {       // block-uniform; nobody reads sm_ex between the tiles
             if (tid < (uint32_t)W) sm_ex[tid] = sm_gexp[tid][tile_group];
             __syncthreads();
             cached_group = tile_group;
         }
-        // Exact form (vgc_decode_sum only).  When the scale is a power of two and the exponents of all messages for the
-        // tile's tensor lie close enough together, every word is an integer multiple of one power of two, 2^base, and
+        // Exact form.  When the exponents of all messages for the tile's tensor lie close enough together, every word
+        // is an integer multiple of one power of two, 2^base, and
         // every partial sum of up to W of them stays within 2^22 multiples: all of them are exact fp32 numbers, fp32
-        // addition of them is associative, and the sequential sum the decoder stands for equals the exact sum.  The
+        // addition of them is associative, and the sequential sum of the words equals the exact sum (with a power-of-two
+        // scale that is the decoder's result bit for bit; otherwise the scale is applied to the exact sum, one rounding
+        // instead of one per message, and vgc_decode_accumulate adds the scaled sum to u in one addition).  The
         // tile is then accumulated as int32 multiples of 2^base with shared-memory integer atomics, in any order:
         // no barrier between messages, no search for the runs' ends -- the warps stream every message's words from
         // its cursor until the indices leave the tile -- and one conversion at the end.  Same bits, much less waiting.
@@ -222,10 +222,19 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
                 if (e != VGC_EXP_NONE) { e_max = max(e_max, e); e_min = min(e_min, e); }
             }
             const int base = e_min - 7;                             // the smallest value a word can stand for
-            if (e_max >= e_min && e_max - base + (32 - __clz((W - 1) | 1)) <= 22 && base + s_exp >= -126 && e_max + s_exp <= 127)
+            // 2^base and every sum of multiples are normal numbers; with a power-of-two scale so are their products
+            if (e_max >= e_min && e_max - base + (32 - __clz((W - 1) | 1)) <= 22 && base >= -126 && base + 22 <= 127 &&
+                (!pow2 || (base + s_exp >= -126 && base + 22 + s_exp <= 127)))
                 fast_base = base;
         }
         const bool fast = fast_base != INT32_MIN;
+        if (!kOverwrite && fast)                                    // the exact form reads u at the tile's end: ask it into L2 now
+            for (uint32_t line = tid; line < (t_len + 31u) / 32u; line += kTileThreads)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(u + t0 + 32u * (size_t)line));
+        if (!kOverwrite && !fast) {                                 // the ordered form adds to the tile's old content
+            for (uint32_t q = tid; q < n_vec; q += kTileThreads) cp_async_16(tile + 4 * q, u + t0 + 4 * (size_t)q);
+            if (tid < t_len - 4 * n_vec) tile[4 * n_vec + tid] = u[t0 + 4 * n_vec + tid];
+        }
         if (tid < (uint32_t)W) taken[tid] = 0;
         if (!fast) {
             if (kOverwrite) __syncthreads();                        // the cursors of the tile before
@@ -258,7 +267,7 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
                 }
                 lut[i] = __fmul_rn(scale, val);
             }
-        if (!kOverwrite) cp_async_wait_all();
+        if (!kOverwrite && !fast) cp_async_wait_all();
         __syncthreads();
 
         if (fast) {
@@ -436,27 +445,61 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
         __syncthreads();
         if (tid < (uint32_t)W) cur[tid] = fast ? cur[tid] + taken[tid] : end[tid];
         if (fast) {
-            // multiples of 2^base -> fp32, times the scale: both factors powers of two, every product exact.  A sum is
-            // at most 2^22 multiples either way, so 1.5 * 2^23 plus it is a float whose bits are 0x4B400000 plus it.
-            const float unit = __uint_as_float((uint32_t)(fast_base + s_exp + 127) << 23);
-            auto value = [&](int mult) { return __fmul_rn(__fsub_rn(__int_as_float(0x4B400000 + mult), 12582912.f), unit); };
-            for (uint32_t q = tid; q < n_vec; q += kTileThreads) {
-                const int4 mlt = reinterpret_cast<const int4 *>(tile)[q];
-                reinterpret_cast<int4 *>(tile)[q] = make_int4(0, 0, 0, 0);
-                *reinterpret_cast<float4 *>(u + t0 + 4 * (size_t)q) = make_float4(value(mlt.x), value(mlt.y), value(mlt.z), value(mlt.w));
+            // multiples of 2^base -> fp32 (a sum is at most 2^22 multiples either way, so 1.5 * 2^23 plus it is a float
+            // whose bits are 0x4B400000 plus it), times 2^base (exact), times the scale: one rounding, none when the
+            // scale is a power of two.  vgc_decode_accumulate adds the result to u; an element no word points at keeps
+            // its bits.
+            const float unit = __uint_as_float((uint32_t)(fast_base + 127) << 23);
+            auto value = [&](int mult) {
+                return __fmul_rn(__fmul_rn(__fsub_rn(__int_as_float(0x4B400000 + mult), 12582912.f), unit), scale);
+            };
+            if (kOverwrite) {
+                for (uint32_t q = tid; q < n_vec; q += kTileThreads) {
+                    const int4 mlt = reinterpret_cast<const int4 *>(tile)[q];
+                    reinterpret_cast<int4 *>(tile)[q] = make_int4(0, 0, 0, 0);
+                    *reinterpret_cast<float4 *>(u + t0 + 4 * (size_t)q) =
+                        make_float4(value(mlt.x), value(mlt.y), value(mlt.z), value(mlt.w));
+                }
+            } else {
+                // four vectors of u per thread in flight (asked into L2 when the tile began)
+                for (uint32_t q0 = tid; q0 < n_vec; q0 += 4 * kTileThreads) {
+                    float4 o[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t q = q0 + j * kTileThreads;
+                        if (q < n_vec) o[j] = *reinterpret_cast<const float4 *>(u + t0 + 4 * (size_t)q);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t q = q0 + j * kTileThreads;
+                        if (q >= n_vec) break;
+                        const int4 mlt = reinterpret_cast<const int4 *>(tile)[q];
+                        if ((mlt.x | mlt.y | mlt.z | mlt.w) == 0) continue;
+                        reinterpret_cast<int4 *>(tile)[q] = make_int4(0, 0, 0, 0);
+                        if (mlt.x) o[j].x = __fadd_rn(o[j].x, value(mlt.x));
+                        if (mlt.y) o[j].y = __fadd_rn(o[j].y, value(mlt.y));
+                        if (mlt.z) o[j].z = __fadd_rn(o[j].z, value(mlt.z));
+                        if (mlt.w) o[j].w = __fadd_rn(o[j].w, value(mlt.w));
+                        *reinterpret_cast<float4 *>(u + t0 + 4 * (size_t)q) = o[j];
+                    }
+                }
             }
             if (tid < t_len - 4 * n_vec) {
-                u[t0 + 4 * n_vec + tid] = value(reinterpret_cast<const int *>(tile)[4 * n_vec + tid]);
+                const int mult = reinterpret_cast<const int *>(tile)[4 * n_vec + tid];
+                float *dst = u + t0 + 4 * n_vec + tid;
+                if (kOverwrite) *dst = value(mult);
+                else if (mult) *dst = __fadd_rn(*dst, value(mult));
                 tile[4 * n_vec + tid] = 0.f;
             }
         } else {
+            const bool zero_after = kOverwrite || exact_possible;
             for (uint32_t q = tid; q < n_vec; q += kTileThreads) {
                 *reinterpret_cast<float4 *>(u + t0 + 4 * (size_t)q) = reinterpret_cast<const float4 *>(tile)[q];
-                if (kOverwrite) reinterpret_cast<float4 *>(tile)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (zero_after) reinterpret_cast<float4 *>(tile)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
             }
             if (tid < t_len - 4 * n_vec) {
                 u[t0 + 4 * n_vec + tid] = tile[4 * n_vec + tid];
-                if (kOverwrite) tile[4 * n_vec + tid] = 0.f;
+                if (zero_after) tile[4 * n_vec + tid] = 0.f;
             }
         }
         // vgc_decode_sum: every thread put zeros back where it read, and the next tile's barrier orders them before

@@ -1,6 +1,7 @@
-"""GPU parity: vgc_decode_accumulate / vgc_decode_sum against the CPU oracle.  The bound is 1e-6 absolute; where the
-decoder adds in message order (dense calls, and any element hit by at most two messages) the result must be the
-oracle's bit for bit."""
+"""GPU parity: vgc_decode_accumulate / vgc_decode_sum against the CPU oracle.  The bound is 1e-6 absolute.  Where the
+decoder adds in message order (the ordered form of dense calls, and any element hit by at most two messages) and where
+it sums exactly under a power-of-two scale (vgc_decode_sum's exact form) the result must be the oracle's bit for bit;
+where it applies the scale to the exact sum, the difference is bounded by the roundings of the sequential sum."""
 import numpy as np
 import pytest
 import torch
@@ -94,16 +95,26 @@ def test_round_trip_of_compressed_messages():
     assert np.abs(u.cpu().numpy().astype(np.float64) - want).max() <= ATOL
 
 
-@pytest.mark.parametrize("n,K,W,density", [(400003, 9, 5, 0.1), (3 * 24576 * 2 + 5, 3, 9, 0.15), (2500000, 40, 17, 0.05),
-                                           (1 << 20, 54, 8, 0.14), (700001, 5, 3, 0.9), (300000, 2, 64, 0.004),
-                                           (33, 1, 2, 1.0), (5000, 1, 1, 0.5)])
-def test_dense_calls_add_in_message_order_bit_for_bit(n, K, W, density):
-    """At one word per eight elements or more the decoder moves u through shared memory and adds message after
-    message -- the oracle's own sequence of fp32 additions -- so the result is the oracle's, bit for bit, with several
-    messages hitting most elements and a scale that is not a power of two."""
+DENSE_CASES = [(400003, 9, 5, 0.1), (3 * 24576 * 2 + 5, 3, 9, 0.15), (2500000, 40, 17, 0.05), (1 << 20, 54, 8, 0.14),
+               (700001, 5, 3, 0.9), (300000, 2, 64, 0.004), (33, 1, 2, 1.0), (5000, 1, 1, 0.5)]
+
+
+def _off_boundary(words):
+    """The same words at an address that is 4 bytes past a 16-byte boundary: such a message takes the ordered form."""
+    buf = torch.empty(words.numel() + 1, dtype=words.dtype, device=words.device)
+    buf[1:] = words
+    return buf[1:]
+
+
+@pytest.mark.parametrize("n,K,W,density", DENSE_CASES)
+def test_ordered_form_adds_in_message_order_bit_for_bit(n, K, W, density):
+    """At one word per eight elements or more the decoder moves u through shared memory; messages that do not start on
+    16-byte boundaries are added message after message -- the oracle's own sequence of fp32 additions -- so the result
+    is the oracle's, bit for bit, with several messages hitting most elements and a scale that is not a power of two."""
     offs = random_offsets(np.random.default_rng(21), n, K)
     msgs = [workloads.random_message(n, offs, density * (1.5 if w % 2 else 0.5), seed=900 + w, device="cuda",
                                      exp_lo=-12, exp_hi=3) for w in range(W)]
+    msgs = [(_off_boundary(w), e) for w, e in msgs]
     assert sum(m[0].numel() for m in msgs) * 8 >= n
     u0 = torch.randn(n, device="cuda") * 1e-2
     got, want, status, _ = _decode_both(n, offs, msgs, 1.0 / 3, u0=u0)
@@ -118,6 +129,45 @@ def test_dense_calls_add_in_message_order_bit_for_bit(n, K, W, density):
     ref = np.zeros(n, F32)
     oracle.decode_accumulate([(w.cpu().numpy().view(np.uint32), e.cpu().numpy()) for w, e in msgs], offs, 1.0 / 3, ref)
     assert int(st.item()) == 0 and np.array_equal(gu.t.cpu().numpy().view(np.uint32), ref.view(np.uint32))
+
+
+@pytest.mark.parametrize("scale", [1.0 / 3, 0.25, -1.0 / 7])
+@pytest.mark.parametrize("n,K,W,density", DENSE_CASES)
+def test_exact_form_differs_from_the_sequential_sum_by_its_roundings_only(n, K, W, density, scale):
+    """Messages on 16-byte boundaries whose exponents lie close together are summed exactly and scaled once; the
+    sequential sum rounds after every message.  Per element the two differ by at most the sequential sum's W roundings
+    plus the exact form's two, each half an ulp of a number no larger than |u0| + sum |scale * value|.  Elements no
+    word points at keep their bits.  (Tensors whose exponents lie too far apart take the ordered form: no difference.)"""
+    offs = random_offsets(np.random.default_rng(21), n, K)
+    msgs = [workloads.random_message(n, offs, density * (1.5 if w % 2 else 0.5), seed=900 + w, device="cuda",
+                                     exp_lo=-9, exp_hi=-4) for w in range(W)]
+    assert sum(m[0].numel() for m in msgs) * 8 >= n
+    u0 = torch.randn(n, device="cuda") * 1e-2
+    u0[::7] = -0.0
+    got, want, status, _ = _decode_both(n, offs, msgs, scale, u0=u0)
+    assert status == 0
+    mag = np.abs(u0.cpu().numpy()).astype(np.float64)
+    touched = np.zeros(n, bool)
+    for w, e in msgs:
+        one = np.zeros(n, F32)
+        oracle.decode_accumulate([(w.cpu().numpy().view(np.uint32), e.cpu().numpy())], offs, scale, one)
+        mag += np.abs(one)
+        touched[w.cpu().numpy().view(np.uint32) >> 4] = True
+    err = np.abs(got.astype(np.float64) - want.astype(np.float64))
+    assert np.all(err <= (W + 2) * 2.0 ** -24 * mag) and err.max() <= ATOL
+    assert np.array_equal(got.view(np.uint32)[~touched], u0.cpu().numpy().view(np.uint32)[~touched])
+    # the same messages written instead of added: scale times the exact sum, one rounding
+    gu = Guarded(n, fill=float("nan"))
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    triples = [(w, torch.tensor([w.numel()], dtype=torch.int32, device="cuda"), e) for w, e in msgs]
+    vgc.vgc_decode_sum(triples, vgc.offsets_tensor(offs), scale, gu.t, st)
+    gu.check("u")
+    ref = np.zeros(n, F32)
+    oracle.decode_accumulate([(w.cpu().numpy().view(np.uint32), e.cpu().numpy()) for w, e in msgs], offs, scale, ref)
+    err = np.abs(gu.t.cpu().numpy().astype(np.float64) - ref.astype(np.float64))
+    assert int(st.item()) == 0 and np.all(err <= (W + 2) * 2.0 ** -24 * (mag - np.abs(u0.cpu().numpy())))
+    if scale == 0.25:                                         # a power of two: every product exact, the same bits
+        assert np.array_equal(gu.t.cpu().numpy().view(np.uint32), ref.view(np.uint32))
 
 
 @pytest.mark.parametrize("n,K,W,density,exps,scale", [(1 << 20, 54, 8, 0.14, (-10, -8), 0.125), (2500000, 40, 17, 0.05, (-14, -9), 1.0),
