@@ -693,8 +693,10 @@ def config4_compress(pk, steps: int = 8):
 
 def config5_decode_sweep(pk):
     """vgc_decode_accumulate over N in {ResNet-50, VGG-16 buffer} x W in {4, 16, 64} x density in {1e-4, 1e-3, 1e-2}
-    generated messages (sorted distinct uniform indices, codes from the quantiser's grid), plus one point per N where
-    all W = 16 messages share one index set.  Bytes: 'strict' counts 4 B per word and 8 B (read + write) per element
+    generated messages (sorted distinct uniform indices, codes from the quantiser's grid; per-tensor exponents shared by
+    the workers up to +-1, as workers of one job have them), plus per N one point where all W = 16 messages share one
+    index set and one where every message draws its exponents independently over 13 binades (workers with nothing in
+    common: the decoder's ordered form).  Bytes: 'strict' counts 4 B per word and 8 B (read + write) per element
     touched; 'moved' is what the form that ran has to move -- sparse calls (atomics) one 32-byte sector read and written
     per word plus the word, dense calls the whole of u once in and out plus the words."""
     import paper_1802_06058_b200 as vgc
@@ -707,20 +709,23 @@ def config5_decode_sweep(pk):
         offs_dev = vgc.offsets_tensor(offs)
         u = torch.zeros(n, dtype=torch.float32, device="cuda")
         status = torch.zeros(1, dtype=torch.int32, device="cuda")
-        points = [(W, rho, False) for W in (4, 16, 64) for rho in (1e-4, 1e-3, 1e-2)] + [(16, 1e-3, True)]
-        for W, rho, shared in points:
+        points = ([(W, rho, False, True) for W in (4, 16, 64) for rho in (1e-4, 1e-3, 1e-2)] + [(16, 1e-3, True, True)] +
+                  [(16, 1e-2, False, False)])
+        for W, rho, shared, common_exps in points:
             mask = None
             if shared:
                 gen = torch.Generator(device="cuda"); gen.manual_seed(5)
                 mask = torch.empty(n, device="cuda").uniform_(generator=gen) < rho
             msgs = [workloads.random_message(n, offs, rho, workloads.seed_for(4, w, 1 if shared else 0, 0, 2), "cuda",
-                                             index_mask=mask) for w in range(W)]
+                                             index_mask=mask, exp_seed=workloads.seed_for(4, 0, 0, 0, 3) if common_exps else None)
+                    for w in range(W)]
             triples = [(m[0], torch.tensor([m[0].numel()], dtype=torch.int32, device="cuda"), m[1]) for m in msgs]
             sum_nnz = sum(m[0].numel() for m in msgs)
             ms = time_graph(lambda: vgc.vgc_decode_accumulate(triples, offs_dev, 1.0 / W, u, status))
             dense = sum_nnz * 8 >= n
             moved = (4 * sum_nnz + 8 * n) if dense else (4 + 64) * sum_nnz
-            rows.append({"net": net, "n": n, "W": W, "density": rho, "shared_index_set": shared, "sum_nnz": sum_nnz,
+            rows.append({"net": net, "n": n, "W": W, "density": rho, "shared_index_set": shared,
+                         "exponents": "shared per tensor +-1" if common_exps else "independent per message", "sum_nnz": sum_nnz,
                          "form": "tiles in shared memory" if dense else "atomics", "ms": ms,
                          "gelem_s": sum_nnz / (ms * 1e-3) / 1e9, "gbs_strict": 12 * sum_nnz / (ms * 1e-3) / 1e9,
                          "gbs_moved": moved / (ms * 1e-3) / 1e9,

@@ -203,9 +203,16 @@ def planted_density_gs(n: int, alpha: float, q: float, seed: int, device="cpu"):
 # generated messages for the decoder sweep
 # ----------------------------------------------------------------------------------------
 def random_message(n: int, offsets: np.ndarray, density: float, seed: int, device="cpu",
-                   exp_lo: int = -20, exp_hi: int = -8, index_mask: torch.Tensor = None):
+                   exp_lo: int = -20, exp_hi: int = -8, index_mask: torch.Tensor = None,
+                   exp_seed: int = None, exp_jitter: int = 1):
     """A packed message with ~density*n sorted distinct uniform indices, uniform sign, uniform
     3-bit code, and per-group exponents uniform on [exp_lo, exp_hi].
+
+    exp_seed: the workers of one job see the same parameters and mini-batches of the same distribution, so the
+    largest residual of a weight tensor (whose exponent is the group exponent, Sec. 4.2) is of the same magnitude
+    on every worker.  With exp_seed the per-group exponents are drawn once from that seed (shared by all messages
+    built with it) and each message moves every group by a draw from [-exp_jitter, exp_jitter]; without it every
+    message draws its own exponents over the whole range (workers that have nothing in common).
 
     Word layout: index << 4 | sign << 3 | code.  Returns (words, group_exp): words is an int32
     tensor holding the 32-bit patterns (view it as uint32), group_exp an int32 tensor."""
@@ -217,5 +224,9 @@ def random_message(n: int, offsets: np.ndarray, density: float, seed: int, devic
     w64 = (idx << 4) | low
     words = torch.where(w64 >= 2 ** 31, w64 - 2 ** 32, w64).to(torch.int32)   # same 32 bits
     k = len(offsets) - 1
-    gexp = torch.randint(exp_lo, exp_hi + 1, (k,), generator=gen, device=device, dtype=torch.int32)
+    if exp_seed is None:
+        gexp = torch.randint(exp_lo, exp_hi + 1, (k,), generator=gen, device=device, dtype=torch.int32)
+    else:
+        base = torch.randint(exp_lo, exp_hi + 1, (k,), generator=_gen(exp_seed, device), device=device, dtype=torch.int32)
+        gexp = base + torch.randint(-exp_jitter, exp_jitter + 1, (k,), generator=gen, device=device, dtype=torch.int32)
     return words, gexp

@@ -231,14 +231,19 @@ def test_config4_vgg16_flat_buffer_compress_only():
     assert_same_state(gpu, cpu)
 
 
-@pytest.mark.parametrize("net,W,density", [("resnet50", 4, 1e-4), ("resnet50", 16, 1e-3), ("resnet50", 64, 1e-2),
-                                           ("vgg16", 4, 1e-2), ("vgg16", 64, 1e-3)])
-def test_config5_decode_sweep(net, W, density):
+@pytest.mark.parametrize("net,W,density,common_exps", [("resnet50", 4, 1e-4, True), ("resnet50", 16, 1e-3, True),
+                                                       ("resnet50", 64, 1e-2, True), ("resnet50", 16, 1e-2, False),
+                                                       ("vgg16", 4, 1e-2, True), ("vgg16", 64, 1e-3, True),
+                                                       ("vgg16", 16, 1e-2, True)])
+def test_config5_decode_sweep(net, W, density, common_exps):
+    """The points of the benchmark's decode sweep, with the messages the benchmark generates (per-tensor exponents
+    shared by the workers up to +-1, or drawn independently per message)."""
     layers = workloads.resnet50_layers() if net == "resnet50" else workloads.vgg16_layers()
     offs = workloads.group_offsets(layers)
     n = int(offs[-1])
     offs_dev = vgc.offsets_tensor(offs)
-    msgs = [workloads.random_message(n, offs, density, workloads.seed_for(4, w, 0, 0, 2), "cuda") for w in range(W)]
+    msgs = [workloads.random_message(n, offs, density, workloads.seed_for(4, w, 0, 0, 2), "cuda",
+                                     exp_seed=workloads.seed_for(4, 0, 0, 0, 3) if common_exps else None) for w in range(W)]
     counts = [torch.tensor([m[0].numel()], dtype=torch.int32, device="cuda") for m in msgs]
     u = torch.zeros(n, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
