@@ -167,7 +167,7 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
     // its result is the sequential sum's, bit for bit
     const int s_exp = (int)((__float_as_uint(scale) >> 23) & 0xFFu) - 127;
     const bool pow2 = (__float_as_uint(scale) & 0x807FFFFFu) == 0u && s_exp > -127 && s_exp < 128;
-    bool exact_possible = !kHybrid && s_exp < 128;              // a finite scale
+    bool exact_possible = s_exp < 128;                          // a finite scale
     if (exact_possible)
         for (int w = 0; w < W; ++w) exact_possible = exact_possible && (reinterpret_cast<uintptr_t>(sm_words[w]) & 15u) == 0u;
     if (kOverwrite || exact_possible) {
@@ -215,7 +215,10 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
         // no barrier between messages, no search for the runs' ends -- the warps stream every message's words from
         // its cursor until the indices leave the tile -- and one conversion at the end.  Same bits, much less waiting.
         int fast_base = INT32_MIN;                                  // INT32_MIN: not applicable
-        if (exact_possible && tile_group >= 0 && t_hi < (1u << 28)) {
+        if (kHybrid) {
+            // every word stands for +tau or -tau: the multiples are +-1 and a sum is at most W of them
+            if (exact_possible && t_hi < (1u << 28)) fast_base = 0;
+        } else if (exact_possible && tile_group >= 0 && t_hi < (1u << 28)) {
             int e_max = INT32_MIN, e_min = INT32_MAX;
             for (int w = 0; w < W; ++w) {
                 const int e = sm_ex[w];
@@ -255,7 +258,10 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
                 const int w = i >> 4;
                 const uint32_t code = (uint32_t)i & 15u;
                 float val;
-                if (kHybrid) val = (code & 8u) ? -tau : tau;
+                if (kHybrid && fast) {
+                    reinterpret_cast<int *>(lut)[i] = (code & 8u) ? -1 : 1;
+                    continue;
+                } else if (kHybrid) val = (code & 8u) ? -tau : tau;
                 else if (fast) {
                     const int e = sm_ex[w];
                     const int mult = e == VGC_EXP_NONE ? 0 : 1 << (e - (int)(code & 7u) - fast_base);
@@ -449,9 +455,10 @@ decode_tiles(const __grid_constant__ DecodeViews views, int W, const uint32_t *_
             // whose bits are 0x4B400000 plus it), times 2^base (exact), times the scale: one rounding, none when the
             // scale is a power of two.  vgc_decode_accumulate adds the result to u; an element no word points at keeps
             // its bits.
-            const float unit = __uint_as_float((uint32_t)(fast_base + 127) << 23);
+            const float unit = kHybrid ? __fmul_rn(scale, tau) : __uint_as_float((uint32_t)(fast_base + 127) << 23);
             auto value = [&](int mult) {
-                return __fmul_rn(__fmul_rn(__fsub_rn(__int_as_float(0x4B400000 + mult), 12582912.f), unit), scale);
+                const float m = __fmul_rn(__fsub_rn(__int_as_float(0x4B400000 + mult), 12582912.f), unit);
+                return kHybrid ? m : __fmul_rn(m, scale);       // hybrid: a word is worth scale * tau, rounded once
             };
             if (kOverwrite) {
                 for (uint32_t q = tid; q < n_vec; q += kTileThreads) {

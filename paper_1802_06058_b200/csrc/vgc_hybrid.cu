@@ -186,24 +186,26 @@ hybrid_totals(const uint32_t *__restrict__ tile_count, uint32_t n_tiles, uint32_
     if (lane == 0) chunk_total[chunk] = c;
 }
 
-__global__ void __launch_bounds__(kThreads)
+constexpr int kThreadsPack = kSegPerChunk * kWarp;   // 1024: one warp per segment of the chunk
+
+__global__ void __launch_bounds__(kThreadsPack)
 hybrid_pack(const uint32_t *__restrict__ tile_count, uint32_t n_tiles, const uint32_t *__restrict__ chunk_total,
             const uint32_t *__restrict__ stage, uint32_t *__restrict__ words, uint32_t capacity,
             uint32_t *nnz_out, uint32_t *dev_status)
 {
-    __shared__ uint32_t sm_tot[kWarps];
+    __shared__ uint32_t sm_tot[kSegPerChunk];
     __shared__ uint32_t sm_pos[kSegPerChunk];
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     uint32_t before = 0;                               // words of all chunks before this one
-    for (uint32_t c = tid; c < blockIdx.x; c += kThreads) before += chunk_total[c];
+    for (uint32_t c = tid; c < blockIdx.x; c += kThreadsPack) before += chunk_total[c];
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) before += __shfl_xor_sync(0xffffffffu, before, d);
     if (lane == 0) sm_tot[warp] = before;
     __syncthreads();
     before = 0;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) before += sm_tot[w];
+    for (int w = 0; w < kSegPerChunk; ++w) before += sm_tot[w];
 
     if (warp == 0) {
         const uint32_t seg = blockIdx.x * kSegPerChunk + lane;
@@ -222,15 +224,23 @@ hybrid_pack(const uint32_t *__restrict__ tile_count, uint32_t n_tiles, const uin
         }
     }
     __syncthreads();
-#pragma unroll 1
-    for (int i = 0; i < kSegPerChunk / kWarps; ++i) {
-        const uint32_t local = i * kWarps + warp;
-        const uint32_t seg = blockIdx.x * kSegPerChunk + local;
-        if (seg >= n_tiles) break;
-        const uint32_t count = tile_count[seg], pos = sm_pos[local];
-        const uint32_t *src = stage + (size_t)seg * kTile;
-        for (uint32_t q = lane; q < count; q += 32)
-            if (pos + q < capacity) words[pos + q] = src[q];
+    // one warp per segment, four 32-wide slices per round so that the loads of a round are in flight together
+    const uint32_t seg = blockIdx.x * kSegPerChunk + warp;
+    if (seg >= n_tiles) return;
+    const uint32_t count = tile_count[seg], pos = sm_pos[warp];
+    const uint32_t *src = stage + (size_t)seg * kTile;
+    for (uint32_t q0 = 0; q0 < count; q0 += 128) {
+        uint32_t held[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t q = q0 + 32 * j + lane;
+            held[j] = q < count ? src[q] : 0u;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t q = q0 + 32 * j + lane;
+            if (q < count && pos + q < capacity) words[pos + q] = held[j];
+        }
     }
 }
 
@@ -282,7 +292,7 @@ extern "C" vgc_status vgc_compress_hybrid(const float *g, const float *s, float 
 #undef VGC_HYBRID_LAUNCH
     hybrid::hybrid_totals<<<(L.chunks + hybrid::kWarps - 1) / hybrid::kWarps, hybrid::kThreads, 0, st>>>(
         tile_count, L.tiles, chunk_total, L.chunks);
-    hybrid::hybrid_pack<<<L.chunks, hybrid::kThreads, 0, st>>>(tile_count, L.tiles, chunk_total, stage, out->words,
+    hybrid::hybrid_pack<<<L.chunks, hybrid::kThreadsPack, 0, st>>>(tile_count, L.tiles, chunk_total, stage, out->words,
                                                                out->capacity, out->nnz, out->dev_status);
     count_launch(3);
     VGC_CUDA_OK(cudaGetLastError());
