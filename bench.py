@@ -1043,6 +1043,10 @@ def main():
         "send_density": nnz_a / n, "nnz": nnz, "n_dropped": counters["n_dropped"], "sum_nnz_decoded": sum_nnz,
         "dev_status": counters["dev_status"],
     }
+    if args.fused:
+        # replayed on their own the sections cannot share v the way the fused step does (the sums would be added
+        # without the compressor's reset in between), so the split is taken in the unfused form; the step is fused
+        sections["note"] = "section split measured in the unfused form (s written, then read by compress); ms_per_step is the fused step"
     traffic = ncu_traffic()
     compress_traffic = traffic.get("compress_bytes_per_param")
     compress_roofline = {"kernel": "compress_phase_a + compress_count + compress_emit", "bound": "hbm",
