@@ -14,7 +14,7 @@
 //           pack_emit    a block adds up the totals of the blocks before it (no waiting on other blocks), a warp scans
 //                        its lanes' sizes and every lane writes the bytes of its 8 words
 //   unpack: one kernel   a warp copies its run's bytes to shared memory, every lane finds the numbers that END in its
-//                        40-byte part (a byte with a clear top bit ends one), a warp scan of their counts gives each
+//                        32nd of them (a byte with a clear top bit ends one), a warp scan of their counts gives each
 //                        its place in the run, and a second scan over the differences gives the indices
 #include "vgc_common.cuh"
 
@@ -145,7 +145,7 @@ __global__ void __launch_bounds__(kPackThreads)
 unpack_runs(const uint8_t *__restrict__ packed, const uint32_t *__restrict__ nnz, uint32_t max_words,
             uint32_t *__restrict__ words, uint32_t *dev_status)
 {
-    __shared__ uint8_t sm_bytes[kPackWarps][kRunBytesMax];
+    __shared__ __align__(4) uint8_t sm_bytes[kPackWarps][kRunBytesMax + 8];
     __shared__ uint32_t sm_vals[kPackWarps][kPackRun];
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t n = min(*nnz, max_words);
@@ -168,12 +168,22 @@ unpack_runs(const uint8_t *__restrict__ packed, const uint32_t *__restrict__ nnz
         return;
     }
     const uint8_t *src = packed + table_bytes + begin;
-    for (uint32_t i = lane; i < nb; i += 32) sm_bytes[warp][i] = src[i];
+    // the bytes keep their alignment in shared memory (byte i sits at off + i), so whole 4-byte words can be copied;
+    // the word that holds the first byte starts up to 3 bytes earlier (inside the stream: the table is before it), the
+    // bytes after the last whole word are copied one by one
+    const uint32_t off = (uint32_t)(reinterpret_cast<uintptr_t>(src) & 3u);
+    const uint32_t whole = (off + nb) / 4u;
+    const uint32_t *src_w = reinterpret_cast<const uint32_t *>(src - off);
+    uint32_t *dst_w = reinterpret_cast<uint32_t *>(&sm_bytes[warp][0]);
+    for (uint32_t i = lane; i < whole; i += 32) dst_w[i] = src_w[i];
+    for (uint32_t i = 4u * whole + lane; i < off + nb; i += 32) sm_bytes[warp][i] = src[i - off];
     __syncwarp();
+    const uint8_t *bytes = &sm_bytes[warp][off];
     // numbers that end in this lane's part of the bytes
-    const uint32_t p0 = lane * kBytesPerLane, p1 = min(p0 + kBytesPerLane, nb);
+    const uint32_t span = (nb + 31u) / 32u;                               // at most kBytesPerLane: every lane has a part
+    const uint32_t p0 = min(lane * span, nb), p1 = min(p0 + span, nb);
     uint32_t ends = 0;
-    for (uint32_t p = p0; p < p1; ++p) ends += (sm_bytes[warp][p] & 0x80u) ? 0u : 1u;
+    for (uint32_t p = p0; p < p1; ++p) ends += (bytes[p] & 0x80u) ? 0u : 1u;
     uint32_t incl = ends;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
@@ -182,17 +192,17 @@ unpack_runs(const uint8_t *__restrict__ packed, const uint32_t *__restrict__ nnz
     }
     const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
     // as many numbers as the run has words, the last byte ending one
-    bool bad = total != in_run || (sm_bytes[warp][nb - 1] & 0x80u);
+    bool bad = total != in_run || (bytes[nb - 1] & 0x80u);
     uint32_t k = incl - ends;                                             // place in the run of the first number ending here
     if (!bad) {
         for (uint32_t p = p0; p < p1; ++p) {
-            if (sm_bytes[warp][p] & 0x80u) continue;
+            if (bytes[p] & 0x80u) continue;
             // the number's bytes: this one and the bytes before it whose top bit is set (at most four)
             uint32_t first = p;
-            while (first > 0 && p - first < 5 && (sm_bytes[warp][first - 1] & 0x80u)) --first;
+            while (first > 0 && p - first < 5 && (bytes[first - 1] & 0x80u)) --first;
             if (p - first > 4) { bad = true; break; }
             uint32_t v = 0;
-            for (uint32_t q = first; q <= p; ++q) v |= (uint32_t)(sm_bytes[warp][q] & 0x7Fu) << (7 * (q - first));
+            for (uint32_t q = first; q <= p; ++q) v |= (uint32_t)(bytes[q] & 0x7Fu) << (7 * (q - first));
             sm_vals[warp][k++] = v;
         }
     }
