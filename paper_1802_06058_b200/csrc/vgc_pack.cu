@@ -60,6 +60,8 @@ pack_count(const uint32_t *__restrict__ words, const uint32_t *__restrict__ nnz,
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t n = min(*nnz, max_words);
     const uint32_t run = blockIdx.x * kPackWarps + warp;
+    // the grid covers the buffer's capacity; blocks past the message's last run have nothing anyone reads
+    if ((size_t)blockIdx.x * kPackWarps * kPackRun >= n) return;
     uint32_t v[kPerLane];
     const uint32_t have = lane_numbers(words, n, run, lane, v);
     uint32_t bytes = 0;
