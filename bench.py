@@ -967,15 +967,15 @@ def main():
             import ctypes
             from paper_1802_06058_b200 import _build
             probe = ctypes.CDLL(_build.build_probe())
-            probe.vgc_probe_mma_rate.argtypes = [ctypes.c_int] * 5 + [ctypes.POINTER(ctypes.c_double)] * 2
+            probe.vgc_probe_mma_rate.argtypes = [ctypes.c_int] * 6 + [ctypes.POINTER(ctypes.c_double)] * 2
             sms = torch.cuda.get_device_properties(local_rank).multi_processor_count
             for kind, name in ((0, "tf32 (8 k)"), (1, "bf16 (16 k)")):
-                for a_tmem in (False, True):
+                for m_rows, a_tmem in ((128, False), (128, True), (64, False)):
                     for n_cols in (64, 128, 256):
                         cyc, tf = ctypes.c_double(0.0), ctypes.c_double(0.0)
-                        rc = probe.vgc_probe_mma_rate(kind, int(a_tmem), n_cols, 4096, sms, ctypes.byref(cyc), ctypes.byref(tf))
+                        rc = probe.vgc_probe_mma_rate(kind, int(a_tmem), m_rows, n_cols, 4096, sms, ctypes.byref(cyc), ctypes.byref(tf))
                         print(json.dumps({"operands": name, "A_from": "tensor memory" if a_tmem else "shared memory",
-                                          "M": 128, "N": n_cols, "status": rc, "cycles_per_mma": round(cyc.value, 1),
+                                          "M": m_rows, "N": n_cols, "status": rc, "cycles_per_mma": round(cyc.value, 1),
                                           "tflops_all_sms": round(tf.value, 1)}))
         return
     vgc.load_library()

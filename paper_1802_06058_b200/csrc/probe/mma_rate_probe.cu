@@ -34,7 +34,7 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr)
 }
 
 // kind: 0 = tf32 (8 k per instruction), 1 = bf16 (16 k); a_tmem: A operand from tensor memory instead of shared memory
-__global__ void __launch_bounds__(128, 1) mma_rate(int kind, int a_tmem, int n, int reps, long long *cycles, uint32_t *status)
+__global__ void __launch_bounds__(128, 1) mma_rate(int kind, int a_tmem, int m, int n, int reps, long long *cycles, uint32_t *status)
 {
     extern __shared__ uint8_t raw[];
     __shared__ __align__(8) uint64_t bar;
@@ -58,7 +58,7 @@ __global__ void __launch_bounds__(128, 1) mma_rate(int kind, int a_tmem, int n, 
     const uint32_t tmem = tmem_slot;
     if (threadIdx.x == 0) {
         const uint32_t fmt = kind ? 1u : 2u;
-        const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+        const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
         const uint64_t da = smem_desc(base), db = smem_desc(base + 16384);
         const long long t0 = clock64();
         for (int r = 0; r < reps; ++r) {
@@ -104,12 +104,13 @@ __global__ void __launch_bounds__(128, 1) mma_rate(int kind, int a_tmem, int n, 
 
 }  // namespace vgc
 
-extern "C" int vgc_probe_mma_rate(int kind, int a_tmem, int n, int reps, int blocks, double *cycles_per_mma,
+// m: rows of the instruction, 128 (n a multiple of 16) or 64 (n a multiple of 8, A operand from shared memory)
+extern "C" int vgc_probe_mma_rate(int kind, int a_tmem, int m, int n, int reps, int blocks, double *cycles_per_mma,
                                          double *tflops)
 {
     using namespace vgc;
-    if ((kind != 0 && kind != 1) || n < 16 || n > 256 || n % 16 != 0 || reps < 1 || reps > (1 << 20) || blocks < 1 ||
-        blocks > 4096 || !cycles_per_mma || !tflops)
+    if ((kind != 0 && kind != 1) || (m != 64 && m != 128) || (m == 64 && a_tmem) || n < 16 || n > 256 || n % 16 != 0 ||
+        reps < 1 || reps > (1 << 20) || blocks < 1 || blocks > 4096 || !cycles_per_mma || !tflops)
         return VGC_ERR_INVALID_ARG;
     static bool configured = false;
     if (!configured) {
@@ -124,9 +125,9 @@ extern "C" int vgc_probe_mma_rate(int kind, int a_tmem, int n, int reps, int blo
     float ms = 0.f;
     long long h[2] = {0, 0};
     if (cudaMemset(d_cycles, 0, 16) == cudaSuccess && cudaEventCreate(&e0) == cudaSuccess && cudaEventCreate(&e1) == cudaSuccess) {
-        probe::mma_rate<<<blocks, 128, probe::kSmem>>>(kind, a_tmem, n, reps, d_cycles, d_status);      // warm-up
+        probe::mma_rate<<<blocks, 128, probe::kSmem>>>(kind, a_tmem, m, n, reps, d_cycles, d_status);   // warm-up
         cudaEventRecord(e0);
-        probe::mma_rate<<<blocks, 128, probe::kSmem>>>(kind, a_tmem, n, reps, d_cycles, d_status);
+        probe::mma_rate<<<blocks, 128, probe::kSmem>>>(kind, a_tmem, m, n, reps, d_cycles, d_status);
         cudaEventRecord(e1);
         if (cudaDeviceSynchronize() == cudaSuccess && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess &&
             cudaMemcpy(h, d_cycles, 16, cudaMemcpyDeviceToHost) == cudaSuccess)
@@ -137,6 +138,6 @@ extern "C" int vgc_probe_mma_rate(int kind, int a_tmem, int n, int reps, int blo
     cudaFree(d_cycles);
     if (rc != VGC_OK) return rc;
     *cycles_per_mma = (double)h[0] / reps;
-    *tflops = 2.0 * 128.0 * n * (kind ? 16.0 : 8.0) * reps * blocks / (ms * 1e-3) / 1e12;
+    *tflops = 2.0 * m * n * (kind ? 16.0 : 8.0) * reps * blocks / (ms * 1e-3) / 1e12;
     return VGC_OK;
 }
