@@ -19,7 +19,7 @@ def allgather_messages(words: torch.Tensor, nnz: torch.Tensor, group_exp: torch.
     (all_words int32 [W, L], all_nnz int32 [W], all_exp int32 [W, K]); row w is rank w's message."""
     if not dist.is_available() or not dist.is_initialized():
         L = int(nnz.item()) if pad_to is None else int(pad_to)
-        L = max(L, 4)
+        L = max((L + 3) // 4 * 4, 4)
         buf = torch.zeros(L, dtype=torch.int32, device=words.device)
         take = min(L, words.numel())
         buf[:take] = words[:take]
@@ -28,7 +28,7 @@ def allgather_messages(words: torch.Tensor, nnz: torch.Tensor, group_exp: torch.
     all_nnz = torch.empty(W, dtype=torch.int32, device=nnz.device)
     dist.all_gather_into_tensor(all_nnz, nnz.reshape(1).contiguous(), group=group)
     L = int(all_nnz.max().item()) if pad_to is None else int(pad_to)       # host read only when no length is agreed
-    L = max(L, 4)
+    L = max((L + 3) // 4 * 4, 4)        # rows on 16-byte boundaries: the decoder then reads them 16 bytes at a time
     mine = torch.zeros(L, dtype=torch.int32, device=words.device)
     take = min(L, words.numel())
     mine[:take] = words[:take]

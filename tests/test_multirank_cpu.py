@@ -85,7 +85,7 @@ words, nnz, gexp = message(rank)
 padded = torch.cat([words, torch.full((9,), -1, dtype=torch.int32)])        # capacity larger than the message
 for pad_to in (None, 16):
     all_words, all_nnz, all_exp = exchange.allgather_messages(padded, nnz, gexp, pad_to=pad_to)
-    assert all_words.shape == (W, 11 if pad_to is None else 16), all_words.shape
+    assert all_words.shape == (W, 12 if pad_to is None else 16), all_words.shape   # the longest message (11), rounded up to 16-byte rows
     for r in range(W):
         w, c, e = message(r)
         assert int(all_nnz[r]) == int(c[0])
