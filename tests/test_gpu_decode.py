@@ -191,6 +191,30 @@ def test_decode_sum_over_the_exponent_range_bit_for_bit(n, K, W, density, exps, 
     assert int(st.item()) == 0 and np.array_equal(gu.t.cpu().numpy().view(np.uint32), ref.view(np.uint32))
 
 
+def test_more_messages_than_one_launch_takes():
+    """70 messages are decoded by two launches (64 + 6); the second adds to what the first wrote.  With the workers'
+    exponents close together both take the exact form: the result is within the roundings of the sequential sum."""
+    n, K, W, scale = 500003, 6, 70, 1.0 / 70
+    offs = random_offsets(np.random.default_rng(3), n, K)
+    msgs = [workloads.random_message(n, offs, 0.01, seed=1500 + w, device="cuda", exp_seed=77) for w in range(W)]
+    assert sum(m[0].numel() for m in msgs) * 8 >= n
+    for entry in ("vgc_decode_sum", "vgc_decode_accumulate"):
+        gu = Guarded(n, fill=0.0)
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        triples = [(w, torch.tensor([w.numel()], dtype=torch.int32, device="cuda"), e) for w, e in msgs]
+        getattr(vgc, entry)(triples, vgc.offsets_tensor(offs), scale, gu.t, st)
+        gu.check("u")
+        ref = np.zeros(n, F32)
+        mag = np.zeros(n, np.float64)
+        for w, e in msgs:
+            one = np.zeros(n, F32)
+            oracle.decode_accumulate([(w.cpu().numpy().view(np.uint32), e.cpu().numpy())], offs, scale, one)
+            mag += np.abs(one)
+        oracle.decode_accumulate([(w.cpu().numpy().view(np.uint32), e.cpu().numpy()) for w, e in msgs], offs, scale, ref)
+        err = np.abs(gu.t.cpu().numpy().astype(np.float64) - ref.astype(np.float64))
+        assert int(st.item()) == 0 and np.all(err <= (W + 4) * 2.0 ** -24 * mag) and err.max() <= ATOL
+
+
 @pytest.mark.parametrize("shift", [0, 1, 2, 3])
 def test_decode_sum_reads_messages_at_any_word_alignment(shift):
     """The exact form reads the messages 16 bytes at a time from the boundary before each cursor; a message that does
